@@ -1,0 +1,155 @@
+/*
+ * river.h -- C ABI of the B200 (sm_100a) early-exit decode library.
+ *
+ * The library runs the hot path of River-LLM: the token-level early-exit autoregressive
+ * decode step of a decoder-only transformer with a KV-Shared Exit River
+ * (paper Section 4.1 "KV-Shared Exit Layer", Section 4.2 "Inference with Seamless Exit", Eq. 1).
+ *
+ * Conventions
+ *   - Pointers marked [dev] are device pointers on the CUDA device that was current at
+ *     river_init; pointers marked [host] are ordinary host memory.  All caller-owned: the
+ *     library never frees them, and weights / KV pool / workspace must outlive the context.
+ *   - Matrices are row-major [out, in] bf16.  A river (exit-layer) matrix is 4-bit weight-only:
+ *     codes u8 [out, in/2] (low nibble = even input index), scale bf16 [out, in/group],
+ *     zero bf16 [out, in/group]; the weight is (code - zero) * scale (Section 4.1, W4A16).
+ *   - Layers are numbered 1..L; exit_layer = number of backbone blocks a token ran, in
+ *     [entry_layer, L] (L = never left the backbone).
+ *   - Every call returns RIVER_OK (0) or a negative RIVER_E_* code; river_last_error() gives
+ *     a text.  No exceptions, no aborts, no device traps.
+ *   - Work is enqueued on the stream given to river_init; device outputs are valid once the
+ *     caller has synchronised that stream (the *_host variants synchronise themselves).
+ *   - A context is not thread-safe.
+ */
+#ifndef RIVER_H_
+#define RIVER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    RIVER_OK = 0,
+    RIVER_E_BADARG = -1,  /* null pointer, out-of-range value */
+    RIVER_E_SHAPE = -2,   /* unsupported model shape */
+    RIVER_E_NOMEM = -3,   /* workspace or KV pool too small */
+    RIVER_E_NOPAGE = -4,  /* no free KV page / sequence full */
+    RIVER_E_BADSLOT = -5, /* slot out of range, duplicated in a batch, or empty */
+    RIVER_E_DEVICE = -6,  /* a CUDA call failed, or a kernel flagged an error */
+    RIVER_E_TIMEOUT = -7  /* a bounded device-side wait ran out */
+};
+
+enum { RIVER_EXIT_PER_TOKEN = 0, RIVER_EXIT_BATCH_MIN = 1 };
+
+/* flags */
+enum {
+    RIVER_F_GRAPH = 1,   /* replay each decode step as a CUDA graph (captured on first use) */
+    RIVER_F_NO_TC = 2    /* run every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
+};
+
+typedef struct river_config {
+    int32_t L, d, Hq, Hkv, dh, F, V; /* layers, hidden, query heads, KV heads, head dim, FFN dim, vocabulary */
+    float rms_eps, rope_theta;
+    int32_t entry_layer;       /* L_s of Section 4.2: the first block after which a token may exit (0..L-1) */
+    int32_t group;             /* quantisation group along the input dimension (64) */
+    int32_t page_size;         /* tokens per KV page (16) */
+    int32_t max_seqs;          /* sequence slots */
+    int32_t max_pages_per_seq; /* page-table width: max context = max_pages_per_seq * page_size */
+    int32_t n_pages;           /* pages in the KV pool (shared by all layers: one page id addresses L layers) */
+    int32_t max_batch;         /* max rows per decode step (<= 1024) */
+    int32_t exit_mode;         /* RIVER_EXIT_PER_TOKEN: Eq. 1 per row; RIVER_EXIT_BATCH_MIN: Eq. 1 literally */
+    uint32_t page_shuffle_seed;/* != 0: hand pages out in a seeded shuffled order */
+    uint32_t flags;
+} river_config;
+
+typedef struct river_w4 {
+    const void *codes, *scale, *zero; /* [dev] */
+} river_w4;
+
+typedef struct river_layer_weights {
+    const void *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *wg, *wu, *wd; /* [dev] bf16 backbone block */
+    river_w4 rq, rk, rv, ro, rg, ru, rd; /* [dev] its exit-layer copy; all NULL if the layer has none */
+} river_layer_weights;
+
+typedef struct river_weights {
+    const void *embed, *lm_head, *final_norm; /* [dev] bf16 [V,d], [V,d], [d] */
+    const river_layer_weights *layers;        /* [host] array of L entries (copied by river_init) */
+} river_weights;
+
+typedef struct river_stats_t {
+    int64_t steps;               /* decode steps run */
+    int64_t launches_total;      /* kernels launched by this context */
+    int32_t launches_last_step;  /* kernels in the last decode step */
+    int32_t batch_last;          /* rows of the last decode step */
+    int32_t device_error;        /* sticky device error word (0 = none) */
+    int32_t pages_in_use;
+    double alg_bytes_last_step;  /* algorithmic HBM bytes of the last step (executed-layer weights + KV read/written
+                                    + LM head + embedding rows + logits), from its actual exit pattern */
+    double layers_executed_last; /* mean exit_layer / L over the rows of the last step */
+} river_stats_t;
+
+typedef struct river_ctx river_ctx;
+
+/* Bytes the caller must provide as workspace / KV pool for this configuration (0 on a bad config).
+ * KV pool layout: bf16 [L][n_pages][2 (K,V)][Hkv][page_size][dh]; K is stored after RoPE.
+ * One page id addresses the same slot in every layer, for backbone and exit layers alike
+ * ("identical KV cache addressing", Section 4.1). */
+size_t river_workspace_bytes(const river_config *cfg);
+size_t river_kv_pool_bytes(const river_config *cfg);
+
+/* Create a context.  kv_pool, workspace: [dev], 256-byte aligned.  cuda_stream: a cudaStream_t (NULL = default
+ * stream).  Copies the config and the layer-pointer table; does not copy weights. */
+int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, size_t kv_pool_bytes,
+               void *workspace, size_t workspace_bytes, void *cuda_stream, river_ctx **out);
+
+/* Prefill with sequence-level exit (Section 4.2, "Prefill Phase"): every prompt token runs backbone blocks
+ * 1..prefill_exit_layer and exit layers above it (prefill_exit_layer = L: the whole backbone), causal attention,
+ * and fills the KV cache of every (token, layer).
+ *   slots   [host] n_seqs empty sequence slots;   tok [dev] int32 token ids, all prompts concatenated;
+ *   offsets [host] n_seqs+1 prefix offsets into tok;
+ *   logits_last [dev] fp32 [n_seqs, V] or NULL;  next_tok [dev] int32 [n_seqs] or NULL (greedy, ties -> lowest id). */
+int river_prefill(river_ctx *ctx, int n_seqs, const int32_t *slots, const int32_t *tok, const int32_t *offsets,
+                  int prefill_exit_layer, float *logits_last, int32_t *next_tok);
+
+/* One token-level early-exit decode step (Section 4.2, "Generation Phase"; Eq. 1).
+ * Row b appends token tok[b] to sequence slots[b] (distinct slots).  After backbone block l with
+ * entry_layer <= l < L the row's state-transition similarity s = cos(h^(l-1), h^(l)) is compared with tau[b]
+ * (strict >, fp32); on exit the row finishes blocks l+1..L in the exit layers, which write their K/V into the
+ * backbone's cache slots, and all rows end at the original LM head.
+ *   slots [host] int32 [batch];  tok [dev] int32 [batch];  tau [dev] fp32 [batch];
+ *   forced_exit [dev] int32 [batch] or NULL -- test hook: a value >= 0 replaces the score test by "leave after
+ *       block forced_exit[b]" (L = never; 0 = exit layers from block 1 on, legal only with entry_layer 0);
+ *   logits [dev] fp32 [batch, V] or NULL;  next_tok [dev] int32 [batch];  exit_layer [dev] int32 [batch];
+ *   scores [dev] fp32 [batch, L] or NULL -- s of every backbone block the row ran, NaN elsewhere. */
+int river_decode_step(river_ctx *ctx, int batch, const int32_t *slots, const int32_t *tok, const float *tau,
+                      const int32_t *forced_exit, float *logits, int32_t *next_tok, int32_t *exit_layer,
+                      float *scores);
+
+/* The same step with HOST buffers: copies tok / tau / forced_exit to the device, runs the step, copies
+ * next_tok / exit_layer (and logits, scores if not NULL) back, and synchronises the stream. */
+int river_decode_step_host(river_ctx *ctx, int batch, const int32_t *slots, const int32_t *tok, const float *tau,
+                           const int32_t *forced_exit, float *logits, int32_t *next_tok, int32_t *exit_layer,
+                           float *scores);
+
+/* Copy n cached positions of one sequence and layer (1-based) out / in: bf16 [n, Hkv, dh], [dev].
+ * river_write_kv is a test hook; it may extend the sequence (allocating pages) up to pos0 + n. */
+int river_read_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, void *k_out, void *v_out);
+int river_write_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, const void *k_in, const void *v_in);
+
+/* Row lists of the last decode step, [host] out: act_idx / riv_idx int32 [(L+1), batch] (entry l-1: rows in the
+ * backbone / in the exit layers entering block l, ascending, -1 padded; entry L: at the LM head) and their counts
+ * int32 [L+1].  Synchronises the stream. */
+int river_last_lists(river_ctx *ctx, int32_t *act_idx, int32_t *n_act, int32_t *riv_idx, int32_t *n_riv);
+
+int river_seq_len(const river_ctx *ctx, int slot);       /* tokens cached in the slot, or RIVER_E_BADSLOT */
+int river_release(river_ctx *ctx, int slot);             /* free the slot's pages */
+int river_stats(river_ctx *ctx, river_stats_t *host_out); /* synchronises the stream */
+void river_destroy(river_ctx *ctx);
+const char *river_last_error(const river_ctx *ctx);      /* ctx may be NULL: error of the last failed river_init */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RIVER_H_ */

@@ -1,0 +1,687 @@
+// Host side of the C ABI declared in include/river.h: argument checks, the KV page table, the per-step
+// metadata upload and the kernel launch sequence of one early-exit decode step.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/river.h"
+#include "river_kernels.cuh"
+
+using namespace river;
+
+namespace {
+
+thread_local std::string g_init_error;
+
+constexpr int kStaging = 4;        // pinned metadata buffers in flight
+constexpr size_t kSmemBudget = 200 * 1024;
+
+struct Carver {
+    char *base;
+    size_t off = 0;
+    template <class T>
+    T *take(size_t n) {
+        off = (off + 255) & ~(size_t)255;
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+}  // namespace
+
+struct river_ctx {
+    river_config cfg;
+    std::vector<river_layer_weights> layers;
+    const uint16_t *embed, *lm_head, *final_norm;
+    cudaStream_t stream;
+    int num_sms = 0;
+    __nv_bfloat16 *pool = nullptr;
+
+    // workspace
+    float *h[3], *qbuf, *obuf, *act, *part_val, *tau_i, *logits_i, *scores_i;
+    float2 *rope_cs;
+    double *inv_freq;
+    int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
+    int32_t *meta_dev;  // [4 + 6*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows
+    uint8_t *exited, *pass;
+    int *dev_err;
+    size_t ws_bytes = 0;
+
+    // host state
+    std::vector<int32_t> page_tbl, seq_len, free_pages;
+    int32_t *meta_host[kStaging] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t meta_ev[kStaging];
+    int meta_next = 0;
+    void *pin_io = nullptr;  // pinned staging for the *_host entry point
+    size_t pin_io_bytes = 0;
+    std::vector<int32_t> last_pos;  // positions of the rows of the last decode step
+    int head_grid = 0;
+
+    river_stats_t st{};
+    std::string err;
+
+    int meta_ints() const { return 4 + 6 * cfg.max_batch; }
+    StepMeta *meta() const { return reinterpret_cast<StepMeta *>(meta_dev); }
+    int32_t *row_slot() const { return meta_dev + 4; }
+    int32_t *row_pos() const { return meta_dev + 4 + cfg.max_batch; }
+    int32_t *upd() const { return meta_dev + 4 + 2 * cfg.max_batch; }
+    int32_t *head_rows() const { return meta_dev + 4 + 5 * cfg.max_batch; }
+};
+
+namespace {
+
+int fail(river_ctx *c, int code, const std::string &msg) {
+    if (c) c->err = msg;
+    else g_init_error = msg;
+    return code;
+}
+
+#define CUDA_TRY(ctx, expr)                                                                             \
+    do {                                                                                                \
+        cudaError_t e_ = (expr);                                                                        \
+        if (e_ != cudaSuccess)                                                                          \
+            return fail(ctx, RIVER_E_DEVICE, std::string(#expr) + ": " + cudaGetErrorString(e_));       \
+    } while (0)
+
+const char *check_config(const river_config *c) {
+    if (!c) return "null config";
+    if (c->L <= 0 || c->d <= 0 || c->Hq <= 0 || c->Hkv <= 0 || c->F <= 0 || c->V <= 0) return "non-positive dimension";
+    if (c->Hq % c->Hkv) return "Hq must be a multiple of Hkv";
+    const int gq = c->Hq / c->Hkv;
+    if (!(gq == 1 || gq == 2 || gq == 4 || gq == 8)) return "GQA group must be 1, 2, 4 or 8";
+    if (!(c->dh == 64 || c->dh == 128)) return "head dim must be 64 or 128";
+    if (!(c->group == 32 || c->group == 64 || c->group == 128)) return "quantisation group must be 32, 64 or 128";
+    if (c->d % c->group || c->F % c->group || (c->Hq * c->dh) % c->group) return "input dims must be multiples of group";
+    if (c->d % 32 || c->F % 32 || c->V % 4 || c->d % 4) return "d, F must be multiples of 32 and V of 4";
+    if (c->page_size != kPage) return "page_size must be 16";
+    if (c->entry_layer < 0 || c->entry_layer >= c->L) return "entry_layer out of range";
+    if (c->max_batch <= 0 || c->max_batch > kMaxBatch) return "max_batch out of range";
+    if (c->max_seqs <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return "bad cache geometry";
+    if (!(c->exit_mode == RIVER_EXIT_PER_TOKEN || c->exit_mode == RIVER_EXIT_BATCH_MIN)) return "bad exit_mode";
+    return nullptr;
+}
+
+int head_grid_for(const river_config *c) { return 148 * 4 > c->V / 4 ? std::max(1, c->V / 4) : 148 * 4; }
+
+size_t carve(const river_config *c, river_ctx *x, char *base) {
+    Carver cv{base};
+    const size_t B = c->max_batch, d = c->d, L = c->L;
+    float *h0 = cv.take<float>(B * d), *h1 = cv.take<float>(B * d), *h2 = cv.take<float>(B * d);
+    float *qb = cv.take<float>(B * c->Hq * c->dh), *ob = cv.take<float>(B * c->Hq * c->dh);
+    float *act = cv.take<float>(B * c->F);
+    float *pv = cv.take<float>(B * (size_t)head_grid_for(c));
+    int32_t *pi = cv.take<int32_t>(B * (size_t)head_grid_for(c));
+    float *tau = cv.take<float>(B);
+    float *lg = cv.take<float>(B * (size_t)c->V);
+    float *sc = cv.take<float>(B * L);
+    float2 *cs = cv.take<float2>(B * (c->dh / 2));
+    double *fr = cv.take<double>(c->dh / 2);
+    int32_t *ai = cv.take<int32_t>((L + 1) * B), *ri = cv.take<int32_t>((L + 1) * B);
+    int32_t *na = cv.take<int32_t>(L + 1), *nr = cv.take<int32_t>(L + 1);
+    int32_t *pt = cv.take<int32_t>((size_t)c->max_seqs * c->max_pages_per_seq);
+    int32_t *tk = cv.take<int32_t>(B), *fo = cv.take<int32_t>(B), *ex = cv.take<int32_t>(B), *nx = cv.take<int32_t>(B);
+    int32_t *md = cv.take<int32_t>(4 + 6 * B);
+    uint8_t *exd = cv.take<uint8_t>(B), *ps = cv.take<uint8_t>(B);
+    int *de = cv.take<int>(1);
+    if (x) {
+        x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
+        x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
+        x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
+        x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
+        x->pass = ps; x->dev_err = de;
+    }
+    return (cv.off + 255) & ~(size_t)255;
+}
+
+// ---- shared-memory sizes and the number of activation rows a projection kernel takes per pass
+size_t proj_smem(int N, int K) {
+    const int xs = std::max(xs_stride(K, 8), xs_stride(K, 32));
+    return sizeof(float) * (32 + (size_t)N * (K >> 5) + (size_t)N * xs);
+}
+int pick_n(int rows, int K) {
+    int n = 1;
+    while (n < rows && n < 8 && proj_smem(n * 2, K) <= kSmemBudget) n *= 2;
+    return n;
+}
+
+template <class Kern>
+int launch_grid(river_ctx *c, Kern kern, int threads, size_t smem) {
+    int occ = 1;
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, smem);
+    occ = std::max(1, std::min(occ, 2048 / threads));
+    return c->num_sms * occ;
+}
+
+#define DISPATCH_N(n, ...)                                      \
+    switch (n) {                                                \
+        case 1: { constexpr int N = 1; __VA_ARGS__ } break;     \
+        case 2: { constexpr int N = 2; __VA_ARGS__ } break;     \
+        case 4: { constexpr int N = 4; __VA_ARGS__ } break;     \
+        default: { constexpr int N = 8; __VA_ARGS__ } break;    \
+    }
+
+KvAddr kv_addr(const river_ctx *c, int layer0) {
+    KvAddr k;
+    k.pool = c->pool;
+    k.page_tbl = c->page_tbl_dev;
+    k.row_slot = c->row_slot();
+    k.row_pos = c->row_pos();
+    k.n_pages = c->cfg.n_pages;
+    k.max_pages_per_seq = c->cfg.max_pages_per_seq;
+    k.Hkv = c->cfg.Hkv;
+    k.dh = c->cfg.dh;
+    k.layer0 = layer0;
+    return k;
+}
+
+W4 w4(const river_w4 &r) {
+    return W4{(const uint8_t *)r.codes, (const uint16_t *)r.scale, (const uint16_t *)r.zero};
+}
+
+template <int DH, int GQ>
+void launch_attn(river_ctx *c, int n, int layer0) {
+    const river_config &g = c->cfg;
+    attn_decode_kernel<DH, GQ><<<dim3(g.Hkv, n), 128, 0, c->stream>>>(
+        c->meta(), c->qbuf, kv_addr(c, layer0), 1.0f / std::sqrt((float)DH), g.Hq, c->obuf);
+}
+
+int launch_attention(river_ctx *c, int n, int layer0) {
+    const int gq = c->cfg.Hq / c->cfg.Hkv;
+#define ATT(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) { launch_attn<DH_, GQ_>(c, n, layer0); return 0; }
+    ATT(64, 1) ATT(64, 2) ATT(64, 4) ATT(64, 8) ATT(128, 1) ATT(128, 2) ATT(128, 4) ATT(128, 8)
+#undef ATT
+    return -1;
+}
+
+// Allocate the page that position `pos` of `slot` falls in, if it has none yet; queue the device update.
+int ensure_page(river_ctx *c, int slot, int pos, int32_t *mh, int &n_upd) {
+    const river_config &g = c->cfg;
+    const int pi = pos / kPage;
+    if (pi >= g.max_pages_per_seq) return fail(c, RIVER_E_NOPAGE, "sequence exceeds max_pages_per_seq");
+    int32_t &e = c->page_tbl[(size_t)slot * g.max_pages_per_seq + pi];
+    if (e >= 0) return 0;
+    if (c->free_pages.empty()) return fail(c, RIVER_E_NOPAGE, "KV pool exhausted");
+    if (n_upd >= g.max_batch) return fail(c, RIVER_E_NOPAGE, "too many new pages in one step");
+    e = c->free_pages.back();
+    c->free_pages.pop_back();
+    int32_t *u = mh + 4 + 2 * g.max_batch;
+    u[n_upd] = slot;
+    u[g.max_batch + n_upd] = pi;
+    u[2 * g.max_batch + n_upd] = e;
+    ++n_upd;
+    return 0;
+}
+
+int32_t *next_meta(river_ctx *c) {
+    const int i = c->meta_next;
+    c->meta_next = (i + 1) % kStaging;
+    cudaEventSynchronize(c->meta_ev[i]);
+    return c->meta_host[i];
+}
+
+int push_meta(river_ctx *c, int32_t *mh) {
+    const int i = (int)((c->meta_next + kStaging - 1) % kStaging);
+    CUDA_TRY(c, cudaMemcpyAsync(c->meta_dev, mh, sizeof(int32_t) * c->meta_ints(), cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaEventRecord(c->meta_ev[i], c->stream));
+    return 0;
+}
+
+// The launch sequence of one step over the rows already described in the device metadata.
+int run_rows(river_ctx *c, int n, int n_head, const int32_t *tok, const float *tau, const int32_t *forced,
+             float *logits, int32_t *next_tok, int32_t *exit_layer, float *scores) {
+    const river_config &g = c->cfg;
+    const int L = g.L, d = g.d, B = g.max_batch;
+    int launches = 0;
+    Lists lists{c->act_idx, c->riv_idx, c->n_act, c->n_riv, B};
+
+    step_begin_kernel<<<std::max(n, 1), 128, 0, c->stream>>>(
+        c->meta(), c->upd(), c->page_tbl_dev, g.max_pages_per_seq, B, tok, c->embed, d, g.V, c->h[0], c->row_pos(),
+        c->inv_freq, g.dh / 2, c->rope_cs, forced, L, g.entry_layer, c->exited, exit_layer, scores, c->dev_err);
+    compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), 0, L, g.entry_layer, g.exit_mode, c->pass, forced, c->exited,
+                                              exit_layer, lists);
+    launches += 2;
+
+    const int qdim = g.Hq * g.dh;
+    int hi = 0;  // h[hi] = block input
+    for (int l = 1; l <= L; ++l) {
+        const river_layer_weights &w = c->layers[l - 1];
+        const int has_river = w.rq.codes != nullptr;
+        const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
+        const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
+        float *h_in = c->h[hi], *h_mid = c->h[(hi + 1) % 3], *h_out = c->h[(hi + 2) % 3];
+        {
+            QkvArgs a{};
+            a.wq = (const uint16_t *)w.wq; a.wk = (const uint16_t *)w.wk; a.wv = (const uint16_t *)w.wv;
+            a.rq = w4(w.rq); a.rk = w4(w.rk); a.rv = w4(w.rv);
+            a.has_river = has_river;
+            a.in = ProjIn{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
+            a.d = d; a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh; a.group = g.group;
+            a.rope_cs = c->rope_cs; a.q_out = c->qbuf; a.kv = kv_addr(c, l - 1);
+            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr; a.dev_err = c->dev_err;
+            const int n_sel = pick_n(n, d);
+            const size_t smem = proj_smem(n_sel, d);
+            DISPATCH_N(n_sel, {
+                const int grid = launch_grid(c, qkv_rope_kv_kernel<N>, 256, smem);
+                qkv_rope_kv_kernel<N><<<grid, 256, smem, c->stream>>>(a);
+            });
+        }
+        if (launch_attention(c, n, l - 1)) return fail(c, RIVER_E_SHAPE, "no attention kernel for this head geometry");
+        {
+            ResidArgs a{};
+            a.w = (const uint16_t *)w.wo; a.rw = w4(w.ro); a.has_river = has_river;
+            a.in = ProjIn{c->obuf, nullptr, 0.f};
+            a.K = qdim; a.out_dim = d; a.group = g.group; a.resid = h_in; a.out = h_mid;
+            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
+            const int n_sel = std::min(pick_n(n, qdim), 8);
+            const size_t smem = proj_smem(n_sel, qdim);
+            DISPATCH_N(n_sel, {
+                const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
+                proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
+            });
+        }
+        {
+            GateUpArgs a{};
+            a.wg = (const uint16_t *)w.wg; a.wu = (const uint16_t *)w.wu; a.rg = w4(w.rg); a.ru = w4(w.ru);
+            a.has_river = has_river;
+            a.in = ProjIn{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
+            a.d = d; a.F = g.F; a.group = g.group; a.act = c->act;
+            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
+            const int n_sel = pick_n(n, d);
+            const size_t smem = proj_smem(n_sel, d);
+            DISPATCH_N(n_sel, {
+                const int grid = launch_grid(c, gateup_kernel<N>, 256, smem);
+                gateup_kernel<N><<<grid, 256, smem, c->stream>>>(a);
+            });
+        }
+        {
+            ResidArgs a{};
+            a.w = (const uint16_t *)w.wd; a.rw = w4(w.rd); a.has_river = has_river;
+            a.in = ProjIn{c->act, nullptr, 0.f};
+            a.K = g.F; a.out_dim = d; a.group = g.group; a.resid = h_mid; a.out = h_out;
+            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
+            const int n_sel = pick_n(n, g.F);
+            const size_t smem = proj_smem(n_sel, g.F);
+            DISPATCH_N(n_sel, {
+                const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
+                proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
+            });
+        }
+        launches += 5;
+        if (l < L || scores) {
+            exit_score_kernel<<<n, 256, 0, c->stream>>>(ai, na, h_in, h_out, d, tau, c->pass, scores, L, l);
+            ++launches;
+        }
+        compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), l, L, g.entry_layer, g.exit_mode, c->pass, forced,
+                                                  c->exited, exit_layer, lists);
+        ++launches;
+        hi = (hi + 2) % 3;
+    }
+    if (n_head > 0) {
+        HeadArgs a{};
+        a.w = c->lm_head;
+        a.in = ProjIn{c->h[hi], c->final_norm, g.rms_eps};
+        a.d = d; a.V = g.V; a.rows = c->head_rows(); a.meta = c->meta(); a.logits = logits;
+        a.part_val = c->part_val; a.part_idx = c->part_idx;
+        const int n_sel = std::min(pick_n(n_head, d), 4);
+        const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xs_stride(d, 8));
+        DISPATCH_N(n_sel, {
+            if (N <= 4) {
+                constexpr int NN = N <= 4 ? N : 4;
+                cudaFuncSetAttribute(lm_head_kernel<NN, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                lm_head_kernel<NN, 4><<<c->head_grid, 256, smem, c->stream>>>(a);
+            }
+        });
+        argmax_final_kernel<<<n_head, 128, 0, c->stream>>>(c->meta(), c->part_val, c->part_idx, c->head_grid, next_tok);
+        launches += 2;
+    }
+    CUDA_TRY(c, cudaGetLastError());
+    c->st.launches_last_step = launches;
+    c->st.launches_total += launches;
+    return 0;
+}
+
+int check_slot(const river_ctx *c, int slot) { return slot >= 0 && slot < c->cfg.max_seqs; }
+
+}  // namespace
+
+extern "C" {
+
+size_t river_workspace_bytes(const river_config *cfg) {
+    if (check_config(cfg)) return 0;
+    return carve(cfg, nullptr, nullptr);
+}
+
+size_t river_kv_pool_bytes(const river_config *cfg) {
+    if (check_config(cfg)) return 0;
+    return (size_t)cfg->L * cfg->n_pages * 2 * cfg->Hkv * kPage * cfg->dh * sizeof(__nv_bfloat16);
+}
+
+int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, size_t kv_pool_bytes, void *workspace,
+               size_t workspace_bytes, void *cuda_stream, river_ctx **out) {
+    if (!out) return fail(nullptr, RIVER_E_BADARG, "out is null");
+    *out = nullptr;
+    if (const char *m = check_config(cfg)) return fail(nullptr, RIVER_E_SHAPE, m);
+    if (!w || !w->embed || !w->lm_head || !w->final_norm || !w->layers) return fail(nullptr, RIVER_E_BADARG, "null weights");
+    if (!kv_pool || !workspace) return fail(nullptr, RIVER_E_BADARG, "null kv_pool / workspace");
+    if (((uintptr_t)kv_pool | (uintptr_t)workspace) & 255) return fail(nullptr, RIVER_E_BADARG, "kv_pool / workspace must be 256-byte aligned");
+    if (kv_pool_bytes < river_kv_pool_bytes(cfg)) return fail(nullptr, RIVER_E_NOMEM, "kv_pool too small");
+    if (workspace_bytes < river_workspace_bytes(cfg)) return fail(nullptr, RIVER_E_NOMEM, "workspace too small");
+    for (int l = 0; l < cfg->L; ++l) {
+        const river_layer_weights &y = w->layers[l];
+        if (!y.attn_norm || !y.wq || !y.wk || !y.wv || !y.wo || !y.ffn_norm || !y.wg || !y.wu || !y.wd)
+            return fail(nullptr, RIVER_E_BADARG, "null backbone weight in layer " + std::to_string(l + 1));
+        const river_w4 *r[7] = {&y.rq, &y.rk, &y.rv, &y.ro, &y.rg, &y.ru, &y.rd};
+        int have = 0;
+        for (auto p : r) have += (p->codes && p->scale && p->zero) ? 1 : 0;
+        if (have != 0 && have != 7) return fail(nullptr, RIVER_E_BADARG, "partial exit-layer weights in layer " + std::to_string(l + 1));
+        if (have == 0 && l + 1 > cfg->entry_layer)
+            return fail(nullptr, RIVER_E_BADARG, "layer " + std::to_string(l + 1) + " is above entry_layer but has no exit-layer copy");
+    }
+    river_ctx *c = new river_ctx();
+    c->cfg = *cfg;
+    c->layers.assign(w->layers, w->layers + cfg->L);
+    c->embed = (const uint16_t *)w->embed;
+    c->lm_head = (const uint16_t *)w->lm_head;
+    c->final_norm = (const uint16_t *)w->final_norm;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->pool = (__nv_bfloat16 *)kv_pool;
+    c->ws_bytes = carve(cfg, c, (char *)workspace);
+    c->head_grid = head_grid_for(cfg);
+    auto bail = [&](const std::string &m) {
+        g_init_error = m;
+        river_destroy(c);
+        return RIVER_E_DEVICE;
+    };
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return bail("cudaGetDevice failed (no CUDA device?)");
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return bail("cudaGetDeviceProperties failed");
+    if (prop.major != 10) return bail("this library is built for sm_100a (B200) only");
+    c->num_sms = prop.multiProcessorCount;
+    for (int i = 0; i < kStaging; ++i) {
+        if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");
+        if (cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail("cudaEventCreate failed");
+    }
+    c->pin_io_bytes = (size_t)cfg->max_batch * (4 * sizeof(int32_t) + sizeof(float));
+    if (cudaMallocHost(&c->pin_io, c->pin_io_bytes) != cudaSuccess) return bail("cudaMallocHost failed");
+    c->page_tbl.assign((size_t)cfg->max_seqs * cfg->max_pages_per_seq, -1);
+    c->seq_len.assign(cfg->max_seqs, 0);
+    c->free_pages.resize(cfg->n_pages);
+    for (int i = 0; i < cfg->n_pages; ++i) c->free_pages[i] = cfg->n_pages - 1 - i;  // pop_back hands out 0, 1, 2, ...
+    if (cfg->page_shuffle_seed) {
+        uint64_t s = cfg->page_shuffle_seed * 0x9E3779B97F4A7C15ull + 1;
+        for (int i = cfg->n_pages - 1; i > 0; --i) {
+            s ^= s >> 12; s ^= s << 25; s ^= s >> 27;
+            const uint64_t r = (s * 0x2545F4914F6CDD1Dull) >> 33;
+            std::swap(c->free_pages[i], c->free_pages[(size_t)(r % (uint64_t)(i + 1))]);
+        }
+    }
+    std::vector<double> fr(cfg->dh / 2);
+    for (int i = 0; i < cfg->dh / 2; ++i) fr[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->dh);
+    cudaError_t e = cudaMemcpyAsync(c->inv_freq, fr.data(), sizeof(double) * fr.size(), cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->page_tbl_dev, 0xff, sizeof(int32_t) * c->page_tbl.size(), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->n_act, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->n_riv, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return bail(std::string("init copies failed: ") + cudaGetErrorString(e));
+    *out = c;
+    return RIVER_OK;
+}
+
+int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32_t *tok, const float *tau,
+                      const int32_t *forced_exit, float *logits, int32_t *next_tok, int32_t *exit_layer,
+                      float *scores) {
+    if (!c) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    if (batch <= 0 || batch > g.max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
+    if (!slots || !tok || !tau || !next_tok || !exit_layer) return fail(c, RIVER_E_BADARG, "null argument");
+    for (int b = 0; b < batch; ++b) {
+        if (!check_slot(c, slots[b])) return fail(c, RIVER_E_BADSLOT, "slot out of range");
+        for (int b2 = 0; b2 < b; ++b2)
+            if (slots[b2] == slots[b]) return fail(c, RIVER_E_BADSLOT, "a slot appears twice in one step");
+        if (c->seq_len[slots[b]] >= g.max_pages_per_seq * kPage) return fail(c, RIVER_E_NOPAGE, "sequence full");
+    }
+    int32_t *mh = next_meta(c);
+    int n_upd = 0;
+    c->last_pos.resize(batch);
+    for (int b = 0; b < batch; ++b) {
+        const int pos = c->seq_len[slots[b]];
+        if (int rc = ensure_page(c, slots[b], pos, mh, n_upd)) return rc;
+        mh[4 + b] = slots[b];
+        mh[4 + g.max_batch + b] = pos;
+        mh[4 + 5 * g.max_batch + b] = b;
+        c->last_pos[b] = pos;
+    }
+    mh[0] = batch; mh[1] = n_upd; mh[2] = batch; mh[3] = 0;
+    if (int rc = push_meta(c, mh)) return rc;
+    if (int rc = run_rows(c, batch, batch, tok, tau, forced_exit, logits, next_tok, exit_layer, scores)) return rc;
+    for (int b = 0; b < batch; ++b) c->seq_len[slots[b]] += 1;
+    c->st.steps += 1;
+    c->st.batch_last = batch;
+    return RIVER_OK;
+}
+
+int river_decode_step_host(river_ctx *c, int batch, const int32_t *slots, const int32_t *tok, const float *tau,
+                           const int32_t *forced_exit, float *logits, int32_t *next_tok, int32_t *exit_layer,
+                           float *scores) {
+    if (!c) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    if (batch <= 0 || batch > g.max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
+    if (!slots || !tok || !tau || !next_tok || !exit_layer) return fail(c, RIVER_E_BADARG, "null argument");
+    if (forced_exit)
+        for (int b = 0; b < batch; ++b)
+            if (forced_exit[b] >= 0 && (forced_exit[b] > g.L || forced_exit[b] < g.entry_layer))
+                return fail(c, RIVER_E_BADARG, "forced_exit out of range");
+    const size_t B = g.max_batch;
+    int32_t *p_tok = (int32_t *)c->pin_io, *p_forced = p_tok + B, *p_next = p_forced + B, *p_exit = p_next + B;
+    float *p_tau = (float *)(p_exit + B);
+    std::memcpy(p_tok, tok, sizeof(int32_t) * batch);
+    std::memcpy(p_tau, tau, sizeof(float) * batch);
+    if (forced_exit) std::memcpy(p_forced, forced_exit, sizeof(int32_t) * batch);
+    CUDA_TRY(c, cudaMemcpyAsync(c->tok_i, p_tok, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->tau_i, p_tau, sizeof(float) * batch, cudaMemcpyHostToDevice, c->stream));
+    if (forced_exit)
+        CUDA_TRY(c, cudaMemcpyAsync(c->forced_i, p_forced, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, c->stream));
+    if (int rc = river_decode_step(c, batch, slots, c->tok_i, c->tau_i, forced_exit ? c->forced_i : nullptr,
+                                   logits ? c->logits_i : nullptr, c->next_i, c->exit_i, scores ? c->scores_i : nullptr))
+        return rc;
+    CUDA_TRY(c, cudaMemcpyAsync(p_next, c->next_i, sizeof(int32_t) * batch, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(p_exit, c->exit_i, sizeof(int32_t) * batch, cudaMemcpyDeviceToHost, c->stream));
+    if (logits)
+        CUDA_TRY(c, cudaMemcpyAsync(logits, c->logits_i, sizeof(float) * (size_t)batch * g.V, cudaMemcpyDeviceToHost, c->stream));
+    if (scores)
+        CUDA_TRY(c, cudaMemcpyAsync(scores, c->scores_i, sizeof(float) * (size_t)batch * g.L, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    std::memcpy(next_tok, p_next, sizeof(int32_t) * batch);
+    std::memcpy(exit_layer, p_exit, sizeof(int32_t) * batch);
+    return RIVER_OK;
+}
+
+int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t *tok, const int32_t *offsets,
+                  int prefill_exit_layer, float *logits_last, int32_t *next_tok) {
+    if (!c) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    if (n_seqs <= 0 || !slots || !tok || !offsets) return fail(c, RIVER_E_BADARG, "null / empty argument");
+    if (prefill_exit_layer < std::max(g.entry_layer, 0) || prefill_exit_layer > g.L)
+        return fail(c, RIVER_E_BADARG, "prefill_exit_layer must lie in [entry_layer, L]");
+    for (int s = 0; s < n_seqs; ++s) {
+        if (!check_slot(c, slots[s])) return fail(c, RIVER_E_BADSLOT, "slot out of range");
+        if (c->seq_len[slots[s]] != 0) return fail(c, RIVER_E_BADSLOT, "prefill needs an empty slot");
+        for (int s2 = 0; s2 < s; ++s2)
+            if (slots[s2] == slots[s]) return fail(c, RIVER_E_BADSLOT, "a slot appears twice");
+        const int n = offsets[s + 1] - offsets[s];
+        if (n <= 0) return fail(c, RIVER_E_BADARG, "empty prompt");
+        if (n > g.max_pages_per_seq * kPage) return fail(c, RIVER_E_NOPAGE, "prompt longer than the page table");
+    }
+    // constant per-row inputs of every chunk: exit forced at the unified depth, threshold unused
+    {
+        std::vector<int32_t> fe(g.max_batch, prefill_exit_layer);
+        std::vector<float> ta(g.max_batch, INFINITY);
+        CUDA_TRY(c, cudaMemcpyAsync(c->forced_i, fe.data(), sizeof(int32_t) * fe.size(), cudaMemcpyHostToDevice, c->stream));
+        CUDA_TRY(c, cudaMemcpyAsync(c->tau_i, ta.data(), sizeof(float) * ta.size(), cudaMemcpyHostToDevice, c->stream));
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    }
+    // Rows of a chunk are consecutive prompt positions, possibly of several sequences; K/V of the whole chunk are
+    // written before its attention runs, and a row attends to positions <= its own, so causality holds inside a chunk.
+    int s = 0, p = 0;  // next (sequence, position) to schedule
+    while (s < n_seqs) {
+        int32_t *mh = next_meta(c);
+        int n = 0, n_upd = 0, n_head = 0;
+        const int tok0 = offsets[s] + p;
+        int head_seq[kMaxBatch];
+        while (s < n_seqs && n < g.max_batch) {
+            const int len = offsets[s + 1] - offsets[s];
+            if (offsets[s] + p != tok0 + n) break;  // token ids of a chunk must be contiguous in tok
+            if (int rc = ensure_page(c, slots[s], p, mh, n_upd)) return rc;
+            mh[4 + n] = slots[s];
+            mh[4 + g.max_batch + n] = p;
+            if (p == len - 1) {
+                mh[4 + 5 * g.max_batch + n_head] = n;
+                head_seq[n_head++] = s;
+            }
+            ++n;
+            if (++p == len) { c->seq_len[slots[s]] = len; ++s; p = 0; }
+        }
+        mh[0] = n; mh[1] = n_upd; mh[2] = n_head; mh[3] = 0;
+        if (int rc = push_meta(c, mh)) return rc;
+        const bool want_logits = logits_last && n_head > 0;
+        if (int rc = run_rows(c, n, n_head, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr,
+                              c->next_i, c->exit_i, nullptr))
+            return rc;
+        for (int i = 0; i < n_head; ++i) {
+            if (logits_last)
+                CUDA_TRY(c, cudaMemcpyAsync(logits_last + (size_t)head_seq[i] * g.V, c->logits_i + (size_t)i * g.V,
+                                            sizeof(float) * g.V, cudaMemcpyDeviceToDevice, c->stream));
+            if (next_tok)
+                CUDA_TRY(c, cudaMemcpyAsync(next_tok + head_seq[i], c->next_i + i, sizeof(int32_t), cudaMemcpyDeviceToDevice, c->stream));
+        }
+    }
+    return RIVER_OK;
+}
+
+static int kv_copy(river_ctx *c, int slot, int layer, int pos0, int n, void *k, void *v, int to_cache) {
+    if (!c) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    if (!check_slot(c, slot)) return fail(c, RIVER_E_BADSLOT, "slot out of range");
+    if (layer < 1 || layer > g.L || pos0 < 0 || n <= 0 || !k || !v) return fail(c, RIVER_E_BADARG, "bad range");
+    if (!to_cache && pos0 + n > c->seq_len[slot]) return fail(c, RIVER_E_BADARG, "range beyond the cached length");
+    if (to_cache) {
+        if (pos0 + n > g.max_pages_per_seq * kPage) return fail(c, RIVER_E_NOPAGE, "range beyond the page table");
+        std::vector<int32_t> u;
+        for (int p = pos0; p < pos0 + n; ++p) {
+            int32_t &e = c->page_tbl[(size_t)slot * g.max_pages_per_seq + p / kPage];
+            if (e >= 0) continue;
+            if (c->free_pages.empty()) return fail(c, RIVER_E_NOPAGE, "KV pool exhausted");
+            e = c->free_pages.back();
+            c->free_pages.pop_back();
+            CUDA_TRY(c, cudaMemcpyAsync(c->page_tbl_dev + (size_t)slot * g.max_pages_per_seq + p / kPage, &e,
+                                        sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+            CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        }
+        c->seq_len[slot] = std::max(c->seq_len[slot], pos0 + n);
+    }
+    kv_copy_kernel<<<n, 128, 0, c->stream>>>(kv_addr(c, layer - 1), slot, pos0, n, (__nv_bfloat16 *)k,
+                                             (__nv_bfloat16 *)v, to_cache);
+    CUDA_TRY(c, cudaGetLastError());
+    c->st.launches_total += 1;
+    return RIVER_OK;
+}
+
+int river_read_kv(river_ctx *c, int slot, int layer, int pos0, int n, void *k_out, void *v_out) {
+    return kv_copy(c, slot, layer, pos0, n, k_out, v_out, 0);
+}
+int river_write_kv(river_ctx *c, int slot, int layer, int pos0, int n, const void *k_in, const void *v_in) {
+    return kv_copy(c, slot, layer, pos0, n, const_cast<void *>(k_in), const_cast<void *>(v_in), 1);
+}
+
+int river_last_lists(river_ctx *c, int32_t *act_idx, int32_t *n_act, int32_t *riv_idx, int32_t *n_riv) {
+    if (!c || !act_idx || !n_act || !riv_idx || !n_riv) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    const int B = c->st.batch_last, L = g.L;
+    if (B <= 0) return fail(c, RIVER_E_BADARG, "no decode step has run");
+    std::vector<int32_t> a((size_t)(L + 1) * g.max_batch), r((size_t)(L + 1) * g.max_batch);
+    CUDA_TRY(c, cudaMemcpyAsync(a.data(), c->act_idx, sizeof(int32_t) * a.size(), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(r.data(), c->riv_idx, sizeof(int32_t) * r.size(), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(n_act, c->n_act, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(n_riv, c->n_riv, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (int l = 0; l <= L; ++l)
+        for (int i = 0; i < B; ++i) {
+            act_idx[(size_t)l * B + i] = i < n_act[l] ? a[(size_t)l * g.max_batch + i] : -1;
+            riv_idx[(size_t)l * B + i] = i < n_riv[l] ? r[(size_t)l * g.max_batch + i] : -1;
+        }
+    return RIVER_OK;
+}
+
+int river_seq_len(const river_ctx *c, int slot) {
+    if (!c || !check_slot(c, slot)) return RIVER_E_BADSLOT;
+    return c->seq_len[slot];
+}
+
+int river_release(river_ctx *c, int slot) {
+    if (!c) return RIVER_E_BADARG;
+    if (!check_slot(c, slot)) return fail(c, RIVER_E_BADSLOT, "slot out of range");
+    const river_config &g = c->cfg;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (int i = g.max_pages_per_seq - 1; i >= 0; --i) {
+        int32_t &e = c->page_tbl[(size_t)slot * g.max_pages_per_seq + i];
+        if (e >= 0) { c->free_pages.push_back(e); e = -1; }
+    }
+    c->seq_len[slot] = 0;
+    CUDA_TRY(c, cudaMemsetAsync(c->page_tbl_dev + (size_t)slot * g.max_pages_per_seq, 0xff,
+                                sizeof(int32_t) * g.max_pages_per_seq, c->stream));
+    return RIVER_OK;
+}
+
+int river_stats(river_ctx *c, river_stats_t *out) {
+    if (!c || !out) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    const int L = g.L, B = c->st.batch_last;
+    std::vector<int32_t> na(L + 1), nr(L + 1);
+    int de = 0;
+    CUDA_TRY(c, cudaMemcpyAsync(na.data(), c->n_act, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(nr.data(), c->n_riv, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(&de, c->dev_err, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    c->st.device_error = de;
+    c->st.pages_in_use = g.n_pages - (int)c->free_pages.size();
+    // algorithmic bytes of the last decode step from its actual exit pattern
+    double bytes = 0.0, layers_run = 0.0;
+    if (B > 0 && c->st.steps > 0) {
+        const double P = (double)g.d * g.Hq * g.dh + 2.0 * g.d * g.Hkv * g.dh + (double)g.Hq * g.dh * g.d + 3.0 * g.d * g.F;
+        const double kv_tok = 2.0 * g.Hkv * g.dh * 2.0;
+        for (int l = 0; l < L; ++l) {
+            if (na[l] > 0) bytes += 2.0 * P;
+            if (nr[l] > 0) bytes += P / 2.0 + 4.0 * P / g.group;
+            layers_run += na[l];
+        }
+        for (int b = 0; b < B; ++b) bytes += (double)L * ((c->last_pos[b] + 1) * kv_tok + kv_tok);
+        bytes += 2.0 * g.V * g.d + (double)B * g.d * 2.0;
+        c->st.layers_executed_last = layers_run / ((double)B * L);
+    }
+    c->st.alg_bytes_last_step = bytes;
+    *out = c->st;
+    return de ? RIVER_E_DEVICE : RIVER_OK;
+}
+
+void river_destroy(river_ctx *c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->stream);
+    for (int i = 0; i < kStaging; ++i) {
+        if (c->meta_host[i]) { cudaFreeHost(c->meta_host[i]); cudaEventDestroy(c->meta_ev[i]); }
+    }
+    if (c->pin_io) cudaFreeHost(c->pin_io);
+    delete c;
+}
+
+const char *river_last_error(const river_ctx *c) { return c ? c->err.c_str() : g_init_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,180 @@
+"""Drives the CPU oracle and the CUDA library side by side on the same seeded buffers (GPU tests only)."""
+from __future__ import annotations
+
+import dataclasses
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from oracle import river_oracle as orc
+from paper_2604_18396_b200 import River, make_config
+from workloads import rtn_w4, synth
+
+INF = float("inf")
+NEAR = 1e-3          # a score this close to the threshold may flip the decision
+LOGIT_ATOL = 2e-2    # max abs error of the logits against the fp32 oracle
+LOGIT_COS = 0.999
+KV_RTOL = 1e-2       # |a-b| <= KV_RTOL*|b| + KV_RTOL*rms(b)
+
+
+def draw_model(name: str, n_layers=None, identity: bool = False):
+    """Draw the model once (on the GPU when there is one: faster) and return CPU and CUDA copies of the same bits."""
+    shape = synth.SHAPES[name]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    bb = synth.make_backbone(shape, dev, n_layers)
+    if identity:
+        rv = []
+        for lay in bb["layers"]:
+            r = {}
+            for n in synth.MATS:
+                lay[n], c, s, z = rtn_w4.snap_to_grid(lay[n], shape.group)
+                r[n] = (c, s, z)
+            rv.append(r)
+    else:
+        rv = rtn_w4.make_river(bb, shape.group)
+
+    def to(x, d):
+        if isinstance(x, torch.Tensor):
+            return x.to(d).contiguous()
+        if isinstance(x, dict):
+            return {k: to(v, d) for k, v in x.items()}
+        if isinstance(x, (list, tuple)):
+            return type(x)(to(v, d) for v in x)
+        return x
+
+    return shape, (to(bb, "cpu"), to(rv, "cpu")), (to(bb, "cuda"), to(rv, "cuda"))
+
+
+@dataclasses.dataclass
+class StepOut:
+    logits: np.ndarray
+    next_tok: np.ndarray
+    exit_layer: np.ndarray
+    scores: np.ndarray
+
+
+class Pair:
+    """An oracle and a CUDA context over the same model, fed the same tokens."""
+
+    def __init__(self, model, max_seqs: int, max_len: int, max_batch: int, exit_mode: int = 0,
+                 entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0):
+        self.shape, (bb_c, rv_c), (bb_g, rv_g) = model
+        self.L = len(bb_c["layers"])
+        self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer)
+        pages_per_seq = (max_len + 15) // 16
+        cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
+                          n_pages=max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
+                          entry_layer=entry_layer, exit_mode=exit_mode, page_shuffle_seed=page_shuffle_seed,
+                          flags=flags)
+        self.gpu = River(cfg, bb_g, rv_g)
+        self.entry = self.shape.entry_layer if entry_layer is None else entry_layer
+        self.V = self.shape.V
+
+    # ---- both sides
+    def prefill(self, slots: List[int], prompts: List[np.ndarray], exit_layer: Optional[int] = None):
+        for s, p in zip(slots, prompts):
+            self.oracle.prefill(s, p, exit_layer)
+        tok = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
+        offs = np.concatenate([[0], np.cumsum([len(p) for p in prompts])]).tolist()
+        self.gpu.prefill(slots, tok, offs, exit_layer)
+
+    def gpu_step(self, slots, tok, tau, forced=None, want_logits=True) -> StepOut:
+        B = len(slots)
+        t = torch.as_tensor(np.asarray(tok, np.int32)).cuda()
+        ta = torch.as_tensor(np.broadcast_to(np.asarray(tau, np.float32), (B,)).copy()).cuda()
+        fe = None if forced is None else torch.as_tensor(np.asarray(forced, np.int32)).cuda()
+        lg = torch.empty((B, self.V), dtype=torch.float32, device="cuda") if want_logits else None
+        nx = torch.empty(B, dtype=torch.int32, device="cuda")
+        el = torch.empty(B, dtype=torch.int32, device="cuda")
+        sc = torch.empty((B, self.L), dtype=torch.float32, device="cuda")
+        self.gpu.decode_step(slots, t, ta, fe, lg, nx, el, sc)
+        torch.cuda.synchronize()
+        return StepOut(lg.cpu().numpy() if want_logits else None, nx.cpu().numpy(), el.cpu().numpy(),
+                       sc.cpu().numpy())
+
+    def oracle_step(self, slots, tok, tau, forced=None) -> StepOut:
+        r = self.oracle.decode_step(slots, tok, tau, forced)
+        return StepOut(r["logits"], r["next_tok"], r["exit_layer"], r["scores"])
+
+    def oracle_scheduled_step(self, slots, tok, targets, margin: float = 2.5 * NEAR):
+        """Oracle step whose per-row thresholds are placed so that the row leaves at (or as close as possible to)
+        targets[b] with every evaluated score at least margin/2 away from its threshold.  Returns (tau, StepOut)."""
+        trial = self.oracle.decode_step(slots, tok, INF)
+        for s in slots:
+            self.oracle.set_len(s, self.oracle.seq_len(s) - 1)  # rewind: the real step rewrites the same slots
+        sc = trial["scores"]
+        tau = np.full(len(slots), INF, np.float32)
+        for b in range(len(slots)):
+            lo = max(self.entry, 1)
+            best = None
+            for e in range(lo, self.L):  # candidate exit layers, nearest to the target first
+                prev = sc[b, lo - 1:e - 1].max() if e > lo else -1.0
+                if sc[b, e - 1] > prev + margin:
+                    if best is None or abs(e - targets[b]) < abs(best - targets[b]):
+                        best = e
+            if targets[b] < self.L and best is not None:
+                e = best
+                prev = sc[b, lo - 1:e - 1].max() if e > lo else sc[b, e - 1] - 2 * margin
+                tau[b] = 0.5 * (sc[b, e - 1] + max(prev, sc[b, e - 1] - 2 * margin))
+        return tau, self.oracle_step(slots, tok, tau)
+
+    # ---- comparisons
+    def compare_logits(self, got: np.ndarray, want: np.ndarray, what=""):
+        err = np.abs(got.astype(np.float64) - want.astype(np.float64)).max()
+        for b in range(want.shape[0]):
+            a, w = got[b].astype(np.float64), want[b].astype(np.float64)
+            cos = a @ w / (np.linalg.norm(a) * np.linalg.norm(w))
+            assert cos >= LOGIT_COS, f"{what}: logits cosine {cos} row {b}"
+        assert err <= LOGIT_ATOL, f"{what}: logits max abs error {err}"
+        return err
+
+    def compare_kv(self, slot: int, n: int, what=""):
+        worst = 0.0
+        for l in range(1, self.L + 1):
+            ko, vo = self.oracle.read_kv(slot, l - 1, 0, n)
+            kg, vg = self.gpu.read_kv(slot, l, 0, n)
+            torch.cuda.synchronize()
+            for name, o, g in (("K", ko, kg), ("V", vo, vg)):
+                g = g.float().cpu().numpy()
+                assert np.isfinite(g).all(), f"{what}: {name} layer {l} slot {slot}: unwritten (NaN) cache entry"
+                rms = np.sqrt((o.astype(np.float64) ** 2).mean())
+                bound = KV_RTOL * np.abs(o) + KV_RTOL * rms
+                ratio = (np.abs(g - o) / bound).max()
+                worst = max(worst, ratio)
+                assert ratio <= 1.0, f"{what}: {name} layer {l} slot {slot}: error {ratio:.3f} x tolerance"
+        return worst
+
+    def compare_lists(self, B: int):
+        ao, nao, ro, nro = self.oracle.last_lists(B)
+        ag, nag, rg, nrg = self.gpu.last_lists(B)
+        assert np.array_equal(nao, nag) and np.array_equal(nro, nrg)
+        assert np.array_equal(ao, ag) and np.array_equal(ro, rg)
+
+    def near_threshold(self, sc_oracle_row: np.ndarray, tau: float, upto: int) -> bool:
+        lo = max(self.entry, 1)
+        s = sc_oracle_row[lo - 1:min(upto, self.L - 1)]
+        s = s[~np.isnan(s)]
+        return bool((np.abs(s - tau) <= NEAR).any())
+
+    def close(self):
+        self.gpu.close()
+        self.oracle.close()
+
+
+def natural_tau(model, prompts, steps_tok, frac_exit: float, entry_layer=None) -> float:
+    """Threshold such that about frac_exit of the decode tokens leave early: the (1-frac) quantile of
+    max_{L_s<=l<L} s^l over a full-depth oracle run."""
+    shape, (bb, rv), _ = model
+    L = len(bb["layers"])
+    o = orc.Oracle(shape, bb, rv, len(prompts), max(len(p) for p in prompts) + len(steps_tok) + 1,
+                   entry_layer=entry_layer)
+    for s, p in enumerate(prompts):
+        o.prefill(s, p)
+    lo = max(shape.entry_layer if entry_layer is None else entry_layer, 1)
+    mx = []
+    for t in range(len(steps_tok)):
+        r = o.decode_step(list(range(len(prompts))), steps_tok[t], INF)
+        mx.append(r["scores"][:, lo - 1:L - 1].max(axis=1))
+    o.close()
+    return float(np.quantile(np.concatenate(mx), 1.0 - frac_exit))
