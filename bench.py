@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the early-exit decode step (one JSON line on stdout).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8b_b1|1b_b8|8b_b64|tiny] [--impl reference]
+
+A step is one decode step of the whole hot path (embed, every block on the backbone or exit-layer weights with
+paged GQA attention, exit score, compaction, LM head) over one batch of synthetic, seeded input.  The default
+workload is the 8B-class decoder at batch 1 with a 1024-token prompt and thresholds scheduled so that about half
+of the tokens leave the backbone early.  value = tokens/s with inputs resident in HBM (CUDA events); e2e = the
+same through the host-buffer entry point, host<->device copies inside the timed region.  With --gpus N (under
+torchrun) every rank runs an independent replica: the path has no exchange step, so no collective is on it.
+--impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import rtn_w4, synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (shape, batch, prompt (lo, hi), seed)
+    "tiny": ("tiny", 1, (32, 32), 0),
+    "1b_b8": ("1b", 8, (512, 512), 1),
+    "8b_b1": ("8b", 1, (1024, 1024), 2),
+    "8b_b64": ("8b", 64, (256, 4096), 3),
+}
+EARLY_FRACTION = 0.5   # share of decode tokens that leave the backbone early
+EARLY_MEAN_LAYER = 3.0  # their mean exit layer (the paper's benchmark table reports about 3 of 16 / 32 at tau = 0.5)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.rows.append([c.strip() for c in ln.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.t.join(timeout=2)
+
+    def summary(self):
+        mhz, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                mhz.append(float(r[0])); mx = max(mx, float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(mhz)}
+
+
+def alg_bytes_step(shape, L, exit_layers, positions, want_logits=True):
+    """Algorithmic HBM bytes of one decode step from its exit pattern: weights of every (layer, weight set) that
+    ran, KV read by every row in every layer (exit-layer rows attend too), KV written, LM head, embedding rows."""
+    P = shape.layer_params()
+    B = len(exit_layers)
+    total = 0.0
+    for l in range(1, L + 1):
+        n_act = sum(1 for e in exit_layers if e >= l)
+        if n_act > 0:
+            total += 2.0 * P
+        if n_act < B:
+            total += P / 2.0 + 4.0 * P / shape.group
+    kv_tok = 2.0 * shape.Hkv * shape.dh * 2.0
+    total += L * sum((p + 1) * kv_tok + kv_tok for p in positions)
+    total += 2.0 * shape.V * shape.d + B * shape.d * 2.0 + (4.0 * B * shape.V if want_logits else 0.0)
+    return total
+
+
+def exit_targets(seed, n, L, entry):
+    """Seeded target exit layers: EARLY_FRACTION of the tokens leave early (geometric, mean EARLY_MEAN_LAYER)."""
+    early = synth.uniform_int(seed, 5000, n, 0, 1000).numpy() < int(1000 * EARLY_FRACTION)
+    geo = synth.forced_exit_schedule(seed, 77, n, L - 1, entry, "geometric", EARLY_MEAN_LAYER).numpy()
+    return np.where(early, np.minimum(geo, L - 1), L).astype(np.int32)
+
+
+def draw_model(shape, device):
+    bb = synth.make_backbone(shape, device)
+    rv = rtn_w4.make_river(bb, shape.group)
+    return bb, rv
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle timing
+def time_oracle(shape, bb_cpu, rv_cpu, B, ctx_len, n_steps, n_warm, seed):
+    """Oracle decode steps at context ctx_len on the host cores.  The KV history is synthetic N(0,1) (an oracle
+    prefill of the whole prompt would take minutes); exits are forced at the scheduled layers."""
+    from oracle import river_oracle as orc
+    L = len(bb_cpu["layers"])
+    o = orc.Oracle(shape, bb_cpu, rv_cpu, B, ctx_len + n_steps + n_warm + 1)
+    w = shape.Hkv * shape.dh
+    for b in range(B):
+        k = synth.normal(seed, 9000 + b, (ctx_len, w), 1.0, "cpu", torch.float32).numpy()
+        for l in range(L):
+            o.write_kv(b, l, 0, k, k)
+        o.set_len(b, ctx_len)
+    targets = exit_targets(seed, (n_steps + n_warm) * B, L, shape.entry_layer).reshape(-1, B)
+    toks = synth.tokens(seed, 50, (n_steps + n_warm) * B, shape.V).numpy().reshape(-1, B)
+    slots = list(range(B))
+    times = []
+    for t in range(n_warm + n_steps):
+        t0 = time.perf_counter()
+        o.decode_step(slots, toks[t], float("inf"), targets[t], want_logits=True, want_scores=False)
+        times.append(time.perf_counter() - t0)
+    o.close()
+    dt = float(np.sum(times[n_warm:]))
+    return {"tokens_per_s": B * n_steps / dt, "seconds": dt, "threads": orc.threads(),
+            "layers_executed": float(targets[n_warm:].mean() / L)}
+
+
+def reference_arm(args, wl):
+    shape_name, B, (plo, phi), seed = WORKLOADS[wl]
+    shape = synth.SHAPES[shape_name]
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    bb, rv = draw_model(shape, dev)
+    to_cpu = lambda x: x.cpu() if isinstance(x, torch.Tensor) else (
+        {k: to_cpu(v) for k, v in x.items()} if isinstance(x, dict) else type(x)(to_cpu(v) for v in x))
+    bb, rv = to_cpu(bb), to_cpu(rv)
+    ctx = (plo + phi) // 2
+    # bound the run to a few minutes: time one step, then fit the row count of the sample
+    Bs = min(B, 4)
+    r = time_oracle(shape, bb, rv, Bs, ctx, args.steps, args.warmup, seed)
+    from oracle import river_oracle as orc
+    cores = orc.threads()
+    sample = (f"{args.steps} oracle decode steps, {Bs} of {B} rows, {shape_name} shape, context {ctx} "
+              f"(synthetic N(0,1) KV history instead of an oracle prefill), exits forced at the scheduled layers")
+    line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": r["tokens_per_s"], "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * r["seconds"] / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl, "shape": shape_name, "batch": Bs, "context": ctx},
+            "cpu_baseline": {"value": r["tokens_per_s"], "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": r["tokens_per_s"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "layers_executed_fraction": r["layers_executed"]}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------- distributed glue
+def dist_setup(n_gpus):
+    """Replicas only: torch.distributed serves the barrier and the max over ranks of the timed region."""
+    import torch.distributed as dist
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if torch.cuda.is_available():
+            torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        dist.init_process_group(backend)
+        return dist.get_rank(), dist.get_world_size()
+    return 0, 1
+
+
+def dist_barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def dist_max(x: float) -> float:
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        t = torch.tensor([x], dtype=torch.float64, device="cuda" if dist.get_backend() == "nccl" else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return x
+
+
+def dist_sum(x: float) -> float:
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        t = torch.tensor([x], dtype=torch.float64, device="cuda" if dist.get_backend() == "nccl" else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+    return x
+
+
+# ---------------------------------------------------------------------------------------------- our arm
+def timed_steps(rv, slots_c, slots, toks, taus, logits, nxt, exits, t0, n):
+    """n decode steps with device-resident inputs, timed with CUDA events on the launching stream."""
+    torch.cuda.synchronize()
+    dist_barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(t0, t0 + n):
+        rv.decode_step(slots, toks[t], taus[t], None, logits, nxt, exits[t], None, slots_c=slots_c)
+    e1.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    return e0.elapsed_time(e1)
+
+
+def ours(args, wl):
+    import ctypes
+    from paper_2604_18396_b200 import River, buildlib, make_config
+    rank, world = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    buildlib.build()
+    dev = torch.device("cuda", torch.cuda.current_device())
+    shape_name, B, (plo, phi), seed = WORKLOADS[wl]
+    seed = seed + 1000 * rank  # replicas draw their own prompts; the model is the same
+    shape = synth.SHAPES[shape_name]
+    L = shape.L
+    K, W = args.steps, args.warmup
+    n_cal, n_prof, n_e2e = 8, 4, min(K, 64)
+    total_steps = n_cal + 2 * (W + K) + n_prof + (W + n_e2e) + 4
+    bb, rvw = draw_model(shape, dev)
+    lens = synth.prompt_lengths(WORKLOADS[wl][3] + 1000 * rank, B, plo, phi) if plo != phi else [plo] * B
+    max_len = max(lens) + total_steps
+    pages_per_seq = (max_len + 15) // 16
+    n_pages = sum((l + total_steps + 15) // 16 for l in lens)
+    flags = args.flags
+    cfg = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=n_pages, max_batch=max(B, 8),
+                      page_shuffle_seed=seed + 1, flags=flags)
+    rv = River(cfg, bb, rvw)
+    slots = list(range(B))
+    slots_c = (ctypes.c_int32 * B)(*slots)
+
+    # ---- prefill (untimed; whole backbone)
+    prompt = torch.cat([synth.tokens(seed, 100 + b, n, shape.V) for b, n in enumerate(lens)]).to(dev)
+    offs = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    t_pf = time.perf_counter()
+    rv.prefill(slots, prompt, offs)
+    torch.cuda.synchronize()
+    t_pf = time.perf_counter() - t_pf
+
+    toks = synth.tokens(seed, 50, total_steps * B, shape.V).view(total_steps, B).to(dev)
+    logits = torch.empty((B, shape.V), dtype=torch.float32, device=dev)
+    nxt = torch.empty(B, dtype=torch.int32, device=dev)
+    exits = torch.full((total_steps, B), -1, dtype=torch.int32, device=dev)
+    inf = torch.full((total_steps, B), float("inf"), dtype=torch.float32, device=dev)
+
+    # ---- calibration: full-depth steps with score read-out give the mean score per layer
+    sc = torch.empty((B, L), dtype=torch.float32, device=dev)
+    acc = []
+    step = 0
+    for _ in range(n_cal):
+        rv.decode_step(slots, toks[step], inf[step], None, logits, nxt, exits[step], sc, slots_c=slots_c)
+        acc.append(sc.clone())
+        step += 1
+    torch.cuda.synchronize()
+    s_mean = torch.stack(acc).float().mean(dim=(0, 1)).cpu().numpy()  # [L]
+    lo = max(shape.entry_layer, 1)
+    targets = exit_targets(seed, total_steps * B, L, shape.entry_layer).reshape(total_steps, B)
+    run_max = np.maximum.accumulate(np.concatenate([[-1.0], s_mean[lo - 1:L - 1]]))  # max score below layer e
+    tau_np = np.full((total_steps, B), np.inf, np.float32)
+    for e in range(lo, L):
+        prev = run_max[e - lo]
+        tau_e = 0.5 * (s_mean[e - 1] + prev) if prev > -1.0 else s_mean[e - 1] - 0.05
+        tau_np[targets == e] = tau_e
+    taus = torch.from_numpy(tau_np).to(dev)
+
+    # ---- timed: early-exit run, then the same kernels at full depth
+    timed_steps(rv, slots_c, slots, toks, taus, logits, nxt, exits, step, W)
+    step += W
+    pos0 = [rv.seq_len(s) for s in slots]
+    launches0 = rv.stats().launches_total
+    with ClockSampler(torch.cuda.current_device()) as clk:
+        ms = timed_steps(rv, slots_c, slots, toks, taus, logits, nxt, exits, step, K)
+    launches = rv.stats().launches_total - launches0
+    ex = exits[step:step + K].cpu().numpy()
+    step += K
+    ms = dist_max(ms)
+    bytes_exit = sum(alg_bytes_step(shape, L, ex[t], [p + t for p in pos0]) for t in range(K)) / K
+
+    timed_steps(rv, slots_c, slots, toks, inf, logits, nxt, exits, step, W)
+    step += W
+    pos1 = [rv.seq_len(s) for s in slots]
+    ms_full = timed_steps(rv, slots_c, slots, toks, inf, logits, nxt, exits, step, K)
+    step += K
+    ms_full = dist_max(ms_full)
+    bytes_full = sum(alg_bytes_step(shape, L, [L] * B, [p + t for p in pos1]) for t in range(K)) / K
+
+    # ---- end to end: host buffers in, results out, every step
+    tok_h = toks.cpu().pin_memory()
+    tau_h = taus.cpu().pin_memory()
+    lg_h = torch.empty((B, shape.V), dtype=torch.float32).pin_memory()
+    nx_h = torch.empty(B, dtype=torch.int32).pin_memory()
+    el_h = torch.empty(B, dtype=torch.int32).pin_memory()
+    for t in range(step, step + W):
+        rv.decode_step_host(slots, tok_h[t], tau_h[t], None, lg_h, nx_h, el_h, None, slots_c=slots_c)
+    step += W
+    torch.cuda.synchronize()
+    dist_barrier()
+    t0 = time.perf_counter()
+    for t in range(step, step + n_e2e):
+        rv.decode_step_host(slots, tok_h[t], tau_h[t], None, lg_h, nx_h, el_h, None, slots_c=slots_c)
+    torch.cuda.synchronize()
+    dist_barrier()
+    ms_e2e = dist_max((time.perf_counter() - t0) * 1e3)
+    step += n_e2e
+
+    # ---- per-kernel timing pass (events around every launch; outside every timed region), full depth
+    rv.profile(True)
+    for t in range(step, step + n_prof):
+        rv.decode_step(slots, toks[t], inf[t], None, logits, nxt, exits[t], None, slots_c=slots_c)
+    step += n_prof
+    prof = rv.profile_read()
+    rv.profile(False)
+    st = rv.stats()
+
+    peak, peak_kind = peaks()
+    tok_s = world * B * K / (ms / 1e3)
+    line = None
+    if rank == 0:
+        dom = max(prof, key=lambda r: r["ms_total"])
+        per_launch_ms = dom["ms_total"] / dom["launches"]
+        ach = dom["alg_bytes_total"] / dom["launches"] / (per_launch_ms * 1e-3) / 1e9
+        tot_ms = sum(r["ms_total"] for r in prof)
+        kernels = {r["name"]: {"launches_per_step": r["launches"] // n_prof,
+                               "ms_per_step": round(r["ms_total"] / n_prof, 4),
+                               "share": round(r["ms_total"] / tot_ms, 4),
+                               "GBps": round(r["alg_bytes_total"] / max(r["ms_total"], 1e-9) / 1e6, 1)} for r in prof}
+        step_gbs = bytes_exit / (ms / K * 1e-3) / 1e9
+        full_gbs = bytes_full / (ms_full / K * 1e-3) / 1e9
+        line = {
+            "metric": "decode_tokens_per_s", "value": tok_s, "unit": "tokens/s", "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl, "shape": shape_name, "batch": B, "prompt": [plo, phi], "context_at_start": pos0[:4],
+                       "early_exit_target_fraction": EARLY_FRACTION, "thresholds": "per-step, from calibrated mean scores",
+                       "l2": "inputs (weights + KV) larger than L2, no flush", "flags": flags,
+                       "parallelism": "replicas only" if world > 1 else "1 GPU", "prefill_s": round(t_pf, 3)},
+            "layers_executed_fraction": float(ex.mean() / L), "early_exit_fraction": float((ex < L).mean()),
+            "mean_exit_layer": float(ex.mean()),
+            "alg_bytes_per_step": bytes_exit,
+            "hbm_roofline_step": {"achieved_GBps": step_gbs, "frac_of_measured_peak": step_gbs / peak,
+                                  "frac_of_8TBps": step_gbs / 8000.0, "peak_GBps": peak, "peak_kind": peak_kind},
+            "full_depth": {"tokens_per_s": world * B * K / (ms_full / 1e3), "ms_per_step": ms_full / K,
+                           "alg_bytes_per_step": bytes_full, "achieved_GBps": full_gbs,
+                           "frac_of_measured_peak": full_gbs / peak, "frac_of_8TBps": full_gbs / 8000.0},
+            "early_exit_speedup_vs_full_depth": ms_full / ms,
+            "roofline": {"bound": "hbm", "kernel": dom["name"], "achieved": ach, "peak": peak, "unit": "GB/s",
+                         "frac": ach / peak, "traffic": None, "peak_kind": peak_kind,
+                         "launch_ms": per_launch_ms, "alg_bytes_per_launch": dom["alg_bytes_total"] / dom["launches"],
+                         "pass": "full depth, events around every launch"},
+            "kernels": kernels,
+            "e2e": {"value": world * B * n_e2e / (ms_e2e / 1e3), "unit": "tokens/s", "steps": n_e2e,
+                    "h2d_bytes_per_step": B * 8, "d2h_bytes_per_step": B * (4 * shape.V + 8)},
+            "gpu_launches": int(launches),
+            "clocks": clk.summary(),
+            "device_error": st.device_error,
+        }
+    # ---- the oracle on the host cores, rank 0 at N = 1 only
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        to_cpu = lambda x: x.cpu() if isinstance(x, torch.Tensor) else (
+            {k: to_cpu(v) for k, v in x.items()} if isinstance(x, dict) else type(x)(to_cpu(v) for v in x))
+        Bs = min(B, 2)
+        n_or = 12 if shape_name == "8b" else 24
+        r = time_oracle(shape, to_cpu(bb), to_cpu(rvw), Bs, int(np.mean(pos0)), n_or, 1, WORKLOADS[wl][3])
+        line["cpu_baseline"] = {
+            "value": r["tokens_per_s"], "unit": "tokens/s", "cores": r["threads"], "kind": "oracle",
+            "sample": f"{n_or} oracle decode steps after 1 warm-up, {Bs} of {B} rows, {shape_name} shape, context "
+                      f"{int(np.mean(pos0))} (synthetic N(0,1) KV history), exits forced at the scheduled layers"}
+    if rank == 0:
+        if "cpu_baseline" not in line:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    rv.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b_b1", choices=sorted(WORKLOADS))
+    ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        reference_arm(args, args.workload)
+    else:
+        ours(args, args.workload)
+
+
+if __name__ == "__main__":
+    main()

@@ -143,6 +143,21 @@ int river_write_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, const v
  * int32 [L+1].  Synchronises the stream. */
 int river_last_lists(river_ctx *ctx, int32_t *act_idx, int32_t *n_act, int32_t *riv_idx, int32_t *n_riv);
 
+/* Per-kernel timing.  river_profile(ctx, 1) zeroes the counters and makes every later step record a CUDA event
+ * before and after each kernel launch on the context's stream and synchronise at the end of the step (the step gets
+ * slower: use it for a separate measuring pass, never inside a timed region); river_profile(ctx, 0) turns it off.
+ * river_profile_read fills out[0..*n_out) ([host], cap entries) with one record per kernel of the step sequence:
+ * its launches, summed device time, and summed algorithmic HBM bytes (weights of the weight sets that actually ran,
+ * KV bytes read / written, LM head, logits). */
+typedef struct river_kernel_time {
+    char name[24];
+    int64_t launches;
+    double ms_total;
+    double alg_bytes_total;
+} river_kernel_time;
+int river_profile(river_ctx *ctx, int enable);
+int river_profile_read(river_ctx *ctx, river_kernel_time *out, int cap, int *n_out);
+
 int river_seq_len(const river_ctx *ctx, int slot);       /* tokens cached in the slot, or RIVER_E_BADSLOT */
 int river_release(river_ctx *ctx, int slot);             /* free the slot's pages */
 int river_stats(river_ctx *ctx, river_stats_t *host_out); /* synchronises the stream */

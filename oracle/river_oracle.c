@@ -45,6 +45,8 @@ typedef struct {
     int32_t group;       /* quantisation group along the input dimension */
     int32_t max_seqs, max_len;
     int32_t exit_mode;   /* 0 = per token, 1 = whole batch switches together (Eq. 1 literal) */
+    int32_t kv_store;    /* 0 = cache holds fp32 values; 1 = cache entries are rounded to bf16 when stored: the
+                            method keeps the KV cache in a 16-bit format (Section 4.1) */
 } orc_config;
 
 /* backbone pointers per layer: attn_norm, wq, wk, wv, wo, ffn_norm, wg, wu, wd (all bf16) */
@@ -64,6 +66,17 @@ typedef struct {
     int32_t *act_idx, *riv_idx, *n_act, *n_riv; /* [(L+1)][maxB], [(L+1)] */
     int32_t lists_cap;
 } orc_ctx;
+
+/* round an fp32 value to the nearest bf16 (ties to even) and return it as fp32 */
+static inline float round_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return f; /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&f, &u, 4);
+    return f;
+}
 
 static inline float bf16_to_f32(uint16_t v) {
     uint32_t u = ((uint32_t)v) << 16;
@@ -213,6 +226,8 @@ static void block(orc_ctx *o, int l0, int river, int slot, int pos, const float 
     matvec(&m[2], Hkv * dh, d, x, vdst);
     for (int i = 0; i < Hq; ++i) rope(q + (size_t)i * dh, dh, pos, c->rope_theta);
     for (int j = 0; j < Hkv; ++j) rope(kdst + (size_t)j * dh, dh, pos, c->rope_theta);
+    if (c->kv_store == 1)
+        for (int i = 0; i < Hkv * dh; ++i) { kdst[i] = round_to_bf16(kdst[i]); vdst[i] = round_to_bf16(vdst[i]); }
     {
         uint8_t *w = &o->written[((size_t)l0 * c->max_seqs + slot) * c->max_len + pos];
         if (*w < 255) ++*w;

@@ -49,7 +49,12 @@ class river_stats_t(C.Structure):
                 ("alg_bytes_last_step", C.c_double), ("layers_executed_last", C.c_double)]
 
 
-EXPORTS = ("river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
+class river_kernel_time(C.Structure):
+    _fields_ = [("name", C.c_char * 24), ("launches", C.c_int64), ("ms_total", C.c_double),
+                ("alg_bytes_total", C.c_double)]
+
+
+EXPORTS = ("river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error")
 
@@ -84,6 +89,8 @@ def load():
     L.river_seq_len.argtypes = [vp, C.c_int]
     L.river_release.argtypes = [vp, C.c_int]
     L.river_stats.argtypes = [vp, C.POINTER(river_stats_t)]
+    L.river_profile.argtypes = [vp, C.c_int]
+    L.river_profile_read.argtypes = [vp, C.POINTER(river_kernel_time), C.c_int, C.POINTER(C.c_int)]
     L.river_destroy.argtypes = [vp]
     L.river_destroy.restype = None
     L.river_last_error.argtypes = [vp]
@@ -233,6 +240,17 @@ class River:
 
     def release(self, slot: int):
         self._check(load().river_release(self.h, slot))
+
+    def profile(self, enable: bool):
+        self._check(load().river_profile(self.h, int(enable)))
+
+    def profile_read(self):
+        """-> [{name, launches, ms_total, alg_bytes_total}] for the kernels timed since profile(True)."""
+        buf = (river_kernel_time * 16)()
+        n = C.c_int(0)
+        self._check(load().river_profile_read(self.h, buf, 16, C.byref(n)))
+        return [dict(name=buf[i].name.decode(), launches=buf[i].launches, ms_total=buf[i].ms_total,
+                     alg_bytes_total=buf[i].alg_bytes_total) for i in range(n.value)]
 
     def stats(self) -> river_stats_t:
         st = river_stats_t()

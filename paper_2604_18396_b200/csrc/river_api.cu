@@ -19,6 +19,9 @@ namespace {
 thread_local std::string g_init_error;
 
 constexpr int kStaging = 4;        // pinned metadata buffers in flight
+enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, kNumClasses };
+const char *const kClassNames[kNumClasses] = {"step_begin", "compact", "qkv_rope_kv", "attn_decode", "o_proj_resid",
+                                              "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final"};
 constexpr size_t kSmemBudget = 200 * 1024;
 
 struct Carver {
@@ -65,6 +68,14 @@ struct river_ctx {
 
     river_stats_t st{};
     std::string err;
+
+    // optional per-kernel timing (river_profile): events around every launch of a step
+    bool profiling = false;
+    std::vector<cudaEvent_t> prof_ev;
+    struct ProfRec { int cls; double bytes_act, bytes_riv; int list_idx; };
+    std::vector<ProfRec> prof_rec;
+    double prof_ms[kNumClasses] = {0}, prof_bytes[kNumClasses] = {0};
+    int64_t prof_launches[kNumClasses] = {0};
 
     int meta_ints() const { return 4 + 6 * cfg.max_batch; }
     StepMeta *meta() const { return reinterpret_cast<StepMeta *>(meta_dev); }
@@ -233,22 +244,69 @@ int push_meta(river_ctx *c, int32_t *mh) {
     return 0;
 }
 
+// Per-kernel timing support: an event before and after every launch while profiling is on.
+struct LaunchScope {
+    river_ctx *c;
+    int idx = -1;
+    LaunchScope(river_ctx *c_, int cls, double bytes_act, double bytes_riv, int list_idx) : c(c_) {
+        ++c->st.launches_last_step;
+        if (!c->profiling) return;
+        idx = (int)c->prof_rec.size();
+        if ((size_t)(2 * idx + 1) >= c->prof_ev.size()) { idx = -1; return; }
+        c->prof_rec.push_back({cls, bytes_act, bytes_riv, list_idx});
+        cudaEventRecord(c->prof_ev[2 * idx], c->stream);
+    }
+    ~LaunchScope() {
+        if (idx >= 0) cudaEventRecord(c->prof_ev[2 * idx + 1], c->stream);
+    }
+};
+
+int profile_collect(river_ctx *c) {
+    const int L = c->cfg.L;
+    std::vector<int32_t> na(L + 1), nr(L + 1);
+    CUDA_TRY(c, cudaMemcpyAsync(na.data(), c->n_act, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(nr.data(), c->n_riv, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (size_t i = 0; i < c->prof_rec.size(); ++i) {
+        const auto &r = c->prof_rec[i];
+        float ms = 0.f;
+        CUDA_TRY(c, cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]));
+        c->prof_ms[r.cls] += ms;
+        c->prof_launches[r.cls] += 1;
+        double bytes = 0.0;
+        if (r.list_idx < 0) bytes = r.bytes_act;
+        else bytes = (na[r.list_idx] > 0 ? r.bytes_act : 0.0) + (nr[r.list_idx] > 0 ? r.bytes_riv : 0.0);
+        c->prof_bytes[r.cls] += bytes;
+    }
+    c->prof_rec.clear();
+    return 0;
+}
+
 // The launch sequence of one step over the rows already described in the device metadata.
-int run_rows(river_ctx *c, int n, int n_head, const int32_t *tok, const float *tau, const int32_t *forced,
-             float *logits, int32_t *next_tok, int32_t *exit_layer, float *scores) {
+int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, const int32_t *tok, const float *tau,
+             const int32_t *forced, float *logits, int32_t *next_tok, int32_t *exit_layer, float *scores) {
     const river_config &g = c->cfg;
     const int L = g.L, d = g.d, B = g.max_batch;
-    int launches = 0;
+    c->st.launches_last_step = 0;
     Lists lists{c->act_idx, c->riv_idx, c->n_act, c->n_riv, B};
+    const int qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
+    const double w4f = 0.25 + 2.0 / g.group;  // bytes of a 4-bit copy relative to bf16: (1/2 + 4/G) / 2
+    double kv_read = 0.0;
+    for (int i = 0; i < n; ++i) kv_read += (double)(row_pos_host[i] + 1) * 2.0 * kvdim * 2.0;
+    const double kv_write = (double)n * 2.0 * kvdim * 2.0;
 
-    step_begin_kernel<<<std::max(n, 1), 128, 0, c->stream>>>(
-        c->meta(), c->upd(), c->page_tbl_dev, g.max_pages_per_seq, B, tok, c->embed, d, g.V, c->h[0], c->row_pos(),
-        c->inv_freq, g.dh / 2, c->rope_cs, forced, L, g.entry_layer, c->exited, exit_layer, scores, c->dev_err);
-    compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), 0, L, g.entry_layer, g.exit_mode, c->pass, forced, c->exited,
-                                              exit_layer, lists);
-    launches += 2;
+    {
+        LaunchScope ls(c, K_BEGIN, (double)n * d * 2.0, 0, -1);
+        step_begin_kernel<<<std::max(n, 1), 128, 0, c->stream>>>(
+            c->meta(), c->upd(), c->page_tbl_dev, g.max_pages_per_seq, B, tok, c->embed, d, g.V, c->h[0], c->row_pos(),
+            c->inv_freq, g.dh / 2, c->rope_cs, forced, L, g.entry_layer, c->exited, exit_layer, scores, c->dev_err);
+    }
+    {
+        LaunchScope ls(c, K_COMPACT, 0, 0, -1);
+        compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), 0, L, g.entry_layer, g.exit_mode, c->pass, forced,
+                                                  c->exited, exit_layer, lists);
+    }
 
-    const int qdim = g.Hq * g.dh;
     int hi = 0;  // h[hi] = block input
     for (int l = 1; l <= L; ++l) {
         const river_layer_weights &w = c->layers[l - 1];
@@ -267,20 +325,27 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *tok, const float *t
             a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr; a.dev_err = c->dev_err;
             const int n_sel = pick_n(n, d);
             const size_t smem = proj_smem(n_sel, d);
+            const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
+            LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
             DISPATCH_N(n_sel, {
                 const int grid = launch_grid(c, qkv_rope_kv_kernel<N>, 256, smem);
                 qkv_rope_kv_kernel<N><<<grid, 256, smem, c->stream>>>(a);
             });
         }
-        if (launch_attention(c, n, l - 1)) return fail(c, RIVER_E_SHAPE, "no attention kernel for this head geometry");
+        {
+            LaunchScope ls(c, K_ATTN, kv_read, 0, -1);
+            if (launch_attention(c, n, l - 1)) return fail(c, RIVER_E_SHAPE, "no attention kernel for this head geometry");
+        }
         {
             ResidArgs a{};
             a.w = (const uint16_t *)w.wo; a.rw = w4(w.ro); a.has_river = has_river;
             a.in = ProjIn{c->obuf, nullptr, 0.f};
             a.K = qdim; a.out_dim = d; a.group = g.group; a.resid = h_in; a.out = h_mid;
             a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-            const int n_sel = std::min(pick_n(n, qdim), 8);
+            const int n_sel = pick_n(n, qdim);
             const size_t smem = proj_smem(n_sel, qdim);
+            const double wb = 2.0 * qdim * d;
+            LaunchScope ls(c, K_OPROJ, wb, wb * w4f, l - 1);
             DISPATCH_N(n_sel, {
                 const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
                 proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
@@ -295,6 +360,8 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *tok, const float *t
             a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
             const int n_sel = pick_n(n, d);
             const size_t smem = proj_smem(n_sel, d);
+            const double wb = 2.0 * 2.0 * g.F * d;
+            LaunchScope ls(c, K_GATEUP, wb, wb * w4f, l - 1);
             DISPATCH_N(n_sel, {
                 const int grid = launch_grid(c, gateup_kernel<N>, 256, smem);
                 gateup_kernel<N><<<grid, 256, smem, c->stream>>>(a);
@@ -308,19 +375,22 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *tok, const float *t
             a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
             const int n_sel = pick_n(n, g.F);
             const size_t smem = proj_smem(n_sel, g.F);
+            const double wb = 2.0 * g.F * d;
+            LaunchScope ls(c, K_DOWN, wb, wb * w4f, l - 1);
             DISPATCH_N(n_sel, {
                 const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
                 proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
             });
         }
-        launches += 5;
         if (l < L || scores) {
+            LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
             exit_score_kernel<<<n, 256, 0, c->stream>>>(ai, na, h_in, h_out, d, tau, c->pass, scores, L, l);
-            ++launches;
         }
-        compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), l, L, g.entry_layer, g.exit_mode, c->pass, forced,
-                                                  c->exited, exit_layer, lists);
-        ++launches;
+        {
+            LaunchScope ls(c, K_COMPACT, 0, 0, -1);
+            compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), l, L, g.entry_layer, g.exit_mode, c->pass, forced,
+                                                      c->exited, exit_layer, lists);
+        }
         hi = (hi + 2) % 3;
     }
     if (n_head > 0) {
@@ -331,19 +401,25 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *tok, const float *t
         a.part_val = c->part_val; a.part_idx = c->part_idx;
         const int n_sel = std::min(pick_n(n_head, d), 4);
         const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xs_stride(d, 8));
-        DISPATCH_N(n_sel, {
-            if (N <= 4) {
-                constexpr int NN = N <= 4 ? N : 4;
-                cudaFuncSetAttribute(lm_head_kernel<NN, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                lm_head_kernel<NN, 4><<<c->head_grid, 256, smem, c->stream>>>(a);
+        {
+            LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + (logits ? 4.0 * n_head * g.V : 0.0), 0, -1);
+            switch (n_sel) {
+                case 1: cudaFuncSetAttribute(lm_head_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                        lm_head_kernel<1, 4><<<c->head_grid, 256, smem, c->stream>>>(a); break;
+                case 2: cudaFuncSetAttribute(lm_head_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                        lm_head_kernel<2, 4><<<c->head_grid, 256, smem, c->stream>>>(a); break;
+                default: cudaFuncSetAttribute(lm_head_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                        lm_head_kernel<4, 4><<<c->head_grid, 256, smem, c->stream>>>(a); break;
             }
-        });
-        argmax_final_kernel<<<n_head, 128, 0, c->stream>>>(c->meta(), c->part_val, c->part_idx, c->head_grid, next_tok);
-        launches += 2;
+        }
+        {
+            LaunchScope ls(c, K_ARGMAX, 0, 0, -1);
+            argmax_final_kernel<<<n_head, 128, 0, c->stream>>>(c->meta(), c->part_val, c->part_idx, c->head_grid, next_tok);
+        }
     }
     CUDA_TRY(c, cudaGetLastError());
-    c->st.launches_last_step = launches;
-    c->st.launches_total += launches;
+    c->st.launches_total += c->st.launches_last_step;
+    if (c->profiling) return profile_collect(c);
     return 0;
 }
 
@@ -462,7 +538,7 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
     }
     mh[0] = batch; mh[1] = n_upd; mh[2] = batch; mh[3] = 0;
     if (int rc = push_meta(c, mh)) return rc;
-    if (int rc = run_rows(c, batch, batch, tok, tau, forced_exit, logits, next_tok, exit_layer, scores)) return rc;
+    if (int rc = run_rows(c, batch, batch, c->last_pos.data(), tok, tau, forced_exit, logits, next_tok, exit_layer, scores)) return rc;
     for (int b = 0; b < batch; ++b) c->seq_len[slots[b]] += 1;
     c->st.steps += 1;
     c->st.batch_last = batch;
@@ -553,7 +629,7 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
         mh[0] = n; mh[1] = n_upd; mh[2] = n_head; mh[3] = 0;
         if (int rc = push_meta(c, mh)) return rc;
         const bool want_logits = logits_last && n_head > 0;
-        if (int rc = run_rows(c, n, n_head, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr,
+        if (int rc = run_rows(c, n, n_head, mh + 4 + g.max_batch, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr,
                               c->next_i, c->exit_i, nullptr))
             return rc;
         for (int i = 0; i < n_head; ++i) {
@@ -672,9 +748,41 @@ int river_stats(river_ctx *c, river_stats_t *out) {
     return de ? RIVER_E_DEVICE : RIVER_OK;
 }
 
+int river_profile(river_ctx *c, int enable) {
+    if (!c) return RIVER_E_BADARG;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (enable && c->prof_ev.empty()) {
+        c->prof_ev.resize(2 * (size_t)(8 * c->cfg.L + 8));
+        for (auto &e : c->prof_ev) CUDA_TRY(c, cudaEventCreate(&e));
+    }
+    if (enable) {
+        for (int i = 0; i < kNumClasses; ++i) { c->prof_ms[i] = 0; c->prof_bytes[i] = 0; c->prof_launches[i] = 0; }
+        c->prof_rec.clear();
+    }
+    c->profiling = enable != 0;
+    return RIVER_OK;
+}
+
+int river_profile_read(river_ctx *c, river_kernel_time *out, int cap, int *n_out) {
+    if (!c || !out || !n_out) return RIVER_E_BADARG;
+    int n = 0;
+    for (int i = 0; i < kNumClasses && n < cap; ++i) {
+        if (!c->prof_launches[i]) continue;
+        std::memset(&out[n], 0, sizeof(out[n]));
+        std::strncpy(out[n].name, kClassNames[i], sizeof(out[n].name) - 1);
+        out[n].launches = c->prof_launches[i];
+        out[n].ms_total = c->prof_ms[i];
+        out[n].alg_bytes_total = c->prof_bytes[i];
+        ++n;
+    }
+    *n_out = n;
+    return RIVER_OK;
+}
+
 void river_destroy(river_ctx *c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
+    for (auto &e : c->prof_ev) cudaEventDestroy(e);
     for (int i = 0; i < kStaging; ++i) {
         if (c->meta_host[i]) { cudaFreeHost(c->meta_host[i]); cudaEventDestroy(c->meta_ev[i]); }
     }

@@ -58,10 +58,10 @@ class Pair:
     """An oracle and a CUDA context over the same model, fed the same tokens."""
 
     def __init__(self, model, max_seqs: int, max_len: int, max_batch: int, exit_mode: int = 0,
-                 entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0):
+                 entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0, kv_store: int = 0):
         self.shape, (bb_c, rv_c), (bb_g, rv_g) = model
         self.L = len(bb_c["layers"])
-        self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer)
+        self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, kv_store)
         pages_per_seq = (max_len + 15) // 16
         cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
                           n_pages=max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
