@@ -1,0 +1,297 @@
+// a3: ragged GQA decode attention over the paged bf16 KV cache (sm_100a).
+//
+// Work item = (row, kv head, KV split).  A producer warp stages K/V pages of the split in shared memory with TMA
+// (2-D tiled copies, 128-byte swizzle, one mbarrier pair per pipeline stage); four consumer warps each own one page
+// (16 positions) of every 64-position tile and run an independent online softmax over their share: a lane owns one
+// position and half of the head dim for q.K (the GQ query heads of the group share every K/V read), the tile maximum
+// and the probabilities move with warp shuffles, and for P.V a lane owns DH/32 head dims.  The four warp states
+// merge through shared memory into one partial (max, sum, unnormalised output) per (row, head, split); a second
+// small kernel merges the splits.  All arithmetic is fp32, exponentials are base 2 (q is pre-scaled by log2 e).
+#pragma once
+#include <cuda.h>
+
+#include "river_kernels.cuh"
+
+namespace river {
+
+constexpr int kAttnTile = 64;      // positions per pipeline stage (4 pages)
+constexpr int kAttnStages = 3;
+constexpr int kAttnConsumers = 4;  // consumer warps = pages per tile
+constexpr int kAttnThreads = 32 * (kAttnConsumers + 1);
+constexpr uint32_t kWaitLimit = 1u << 20;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kWaitLimit polls (or when another thread of the CTA already gave up), records the
+// timeout in the device error word and raises the CTA's abort flag.  Returns false on give-up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *dev_err) {
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(dev_err, DEV_WAIT_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+struct AttnArgs {
+    const StepMeta *meta;
+    const float *q;        // [rows][Hq*DH]
+    const int32_t *page_tbl, *row_slot, *row_pos;
+    int n_pages, max_pages_per_seq, Hkv, Hq, layer0;
+    float qscale;          // log2(e) / sqrt(DH)
+    float *part_o;         // [(row*Hq + head)*splits + split][DH]  unnormalised
+    float2 *part_ml;       // same index: (max, sum) in the base-2 domain
+    int *dev_err;
+};
+
+template <int DH, int GQ>
+__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                  const AttnArgs a) {
+    constexpr int NB = DH / 64;                  // 128-byte boxes per cache row
+    constexpr int PAGE_BYTES = kPage * DH * 2;   // one page of K (or V) of one kv head
+    constexpr int STAGE_BYTES = 2 * kAttnConsumers * PAGE_BYTES;
+    constexpr int NCH = DH / 16;                 // 16-byte chunks per lane half in q.K
+    constexpr int VE = DH / 32;                  // head dims per lane in P.V
+
+    const int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
+    if (row >= a.meta->n_rows) return;
+    const int chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
+    const int pos = a.row_pos[row], slot = a.row_slot[row];
+    const int p0 = split * chunk;
+    if (p0 > pos) return;
+    const int p1 = min(p0 + chunk, pos + 1);     // positions [p0, p1)
+    const int n_tiles = (p1 - p0 + kAttnTile - 1) / kAttnTile;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *stages = smem;                                            // kAttnStages * STAGE_BYTES, 1024-aligned
+    float *sq = reinterpret_cast<float *>(stages + kAttnStages * STAGE_BYTES);  // [GQ][DH]
+    float *sp = sq + GQ * DH;                                          // [4 warps][16][GQ]
+    float *sm = sp + kAttnConsumers * kPage * GQ;                      // merge: [4][GQ][DH + 2]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sm + kAttnConsumers * GQ * (DH + 2));  // full[S], empty[S]
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < kAttnStages; ++s) {
+            mbar_init(smem_u32(&bars[s]), 1);
+            mbar_init(smem_u32(&bars[kAttnStages + s]), kAttnConsumers);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    for (int i = tid; i < GQ * DH; i += kAttnThreads)
+        sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
+    __syncthreads();
+    volatile int *abortp = &s_abort;
+
+    if (warp == kAttnConsumers) {
+        // ---------------- producer: one lane issues the TMA copies, at most kAttnStages tiles ahead
+        if (lane == 0) {
+            const int32_t *pt = a.page_tbl + (size_t)slot * a.max_pages_per_seq;
+            for (int t = 0; t < n_tiles; ++t) {
+                const int s = t % kAttnStages;
+                if (t >= kAttnStages &&
+                    !mbar_wait(smem_u32(&bars[kAttnStages + s]), ((t / kAttnStages) - 1) & 1, abortp, a.dev_err))
+                    break;
+                const int first_page = (p0 + t * kAttnTile) / kPage;
+                const int n_valid = min(kAttnConsumers, (p1 - 1) / kPage - first_page + 1);
+                const uint32_t full = smem_u32(&bars[s]);
+                mbar_expect_tx(full, (uint32_t)(n_valid * 2 * PAGE_BYTES));
+                for (int j = 0; j < n_valid; ++j) {
+                    int page = pt[first_page + j];
+                    if (page < 0 || page >= a.n_pages) { atomicExch(a.dev_err, DEV_BAD_PAGE); page = 0; }
+                    // cache rows of (layer, page, K|V, kv head): 16 consecutive rows of the [rows][DH] view
+                    const int yk = ((((a.layer0 * a.n_pages + page) * 2 + 0) * a.Hkv) + kvh) * kPage;
+                    const int yv = ((((a.layer0 * a.n_pages + page) * 2 + 1) * a.Hkv) + kvh) * kPage;
+                    const uint32_t dk = smem_u32(stages + s * STAGE_BYTES + j * PAGE_BYTES);
+                    const uint32_t dv = dk + kAttnConsumers * PAGE_BYTES;
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        tma_load_2d(dk + b * (kPage * 128), &tmap, b * 64, yk, full);
+                        tma_load_2d(dv + b * (kPage * 128), &tmap, b * 64, yv, full);
+                    }
+                }
+            }
+        }
+    } else {
+        // ---------------- consumers: warp w owns page w of every tile
+        const int r = lane & 15, hsel = lane >> 4;
+        float m[GQ], l[GQ], acc[GQ][VE];
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            m[g] = -CUDART_INF_F;
+            l[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
+        }
+        float *my_sp = sp + warp * kPage * GQ;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int s = t % kAttnStages;
+            if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
+            const int page_pos0 = p0 + t * kAttnTile + warp * kPage;  // first position of this warp's page
+            if (page_pos0 < p1) {
+                const uint8_t *kpg = stages + s * STAGE_BYTES + warp * PAGE_BYTES;
+                const uint8_t *vpg = kpg + kAttnConsumers * PAGE_BYTES;
+                // q.K for position r, dims [hsel*DH/2, (hsel+1)*DH/2)
+                float sc[GQ];
+#pragma unroll
+                for (int g = 0; g < GQ; ++g) sc[g] = 0.f;
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) {
+                    const int cg = hsel * NCH + i, box = cg >> 3, c = cg & 7;
+                    const uint4 kw = *reinterpret_cast<const uint4 *>(kpg + box * (kPage * 128) + r * 128 +
+                                                                     ((c ^ (r & 7)) << 4));
+                    const float k0 = bf16lo(kw.x), k1 = bf16hi(kw.x), k2 = bf16lo(kw.y), k3 = bf16hi(kw.y);
+                    const float k4 = bf16lo(kw.z), k5 = bf16hi(kw.z), k6 = bf16lo(kw.w), k7 = bf16hi(kw.w);
+#pragma unroll
+                    for (int g = 0; g < GQ; ++g) {
+                        const float4 qa = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8);
+                        const float4 qb = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8 + 4);
+                        float v = sc[g];
+                        v = fmaf(qa.x, k0, v); v = fmaf(qa.y, k1, v); v = fmaf(qa.z, k2, v); v = fmaf(qa.w, k3, v);
+                        v = fmaf(qb.x, k4, v); v = fmaf(qb.y, k5, v); v = fmaf(qb.z, k6, v); v = fmaf(qb.w, k7, v);
+                        sc[g] = v;
+                    }
+                }
+                const bool live = page_pos0 + r < p1;
+                float corr[GQ];
+#pragma unroll
+                for (int g = 0; g < GQ; ++g) {
+                    float v = sc[g] + __shfl_xor_sync(0xffffffffu, sc[g], 16);
+                    v = live ? v : -CUDART_INF_F;  // select, never arithmetic: stale cache rows may hold anything
+                    float mx = v;
+#pragma unroll
+                    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    const float mn = fmaxf(m[g], mx);  // finite: position page_pos0 is live
+                    corr[g] = ex2(m[g] - mn);
+                    m[g] = mn;
+                    const float p = live ? ex2(v - mn) : 0.f;
+                    if (hsel == 0) my_sp[r * GQ + g] = p;
+                    l[g] *= corr[g];
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) acc[g][e] *= corr[g];
+                }
+                __syncwarp();
+                // P.V: lane owns dims [lane*VE, lane*VE + VE)
+                const int n_live = min(kPage, p1 - page_pos0);
+                const int vbyte = lane * VE * 2, vbox = vbyte >> 7, vc = (vbyte & 127) >> 4, vo = vbyte & 15;
+                for (int j = 0; j < n_live; ++j) {
+                    const uint8_t *vp = vpg + vbox * (kPage * 128) + j * 128 + ((vc ^ (j & 7)) << 4) + vo;
+                    float vf[VE];
+                    if (VE == 4) {
+                        const uint2 w = *reinterpret_cast<const uint2 *>(vp);
+                        vf[0] = bf16lo(w.x); vf[1] = bf16hi(w.x); vf[2 % VE] = bf16lo(w.y); vf[3 % VE] = bf16hi(w.y);
+                    } else {
+                        const uint32_t w = *reinterpret_cast<const uint32_t *>(vp);
+                        vf[0] = bf16lo(w); vf[1] = bf16hi(w);
+                    }
+#pragma unroll
+                    for (int g = 0; g < GQ; ++g) {
+                        const float p = my_sp[j * GQ + g];
+                        l[g] += p;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) acc[g][e] = fmaf(p, vf[e], acc[g][e]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars[kAttnStages + s]));
+        }
+        // publish this warp's state
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            float *dst = sm + (warp * GQ + g) * (DH + 2);
+#pragma unroll
+            for (int e = 0; e < VE; ++e) dst[lane * VE + e] = acc[g][e];
+            if (lane == 0) { dst[DH] = m[g]; dst[DH + 1] = l[g]; }
+        }
+    }
+    __syncthreads();
+    if (s_abort) {
+        // give copies that are still in flight time to land before the CTA's shared memory is handed on
+        for (int i = 0; i < 2000; ++i) __nanosleep(100);
+        return;
+    }
+    // merge the four warp states -> one partial per head
+    for (int t = tid; t < GQ * DH; t += kAttnThreads) {
+        const int g = t / DH, e = t % DH;
+        float M = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < kAttnConsumers; ++w) M = fmaxf(M, sm[(w * GQ + g) * (DH + 2) + DH]);
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int w = 0; w < kAttnConsumers; ++w) {
+            const float *src = sm + (w * GQ + g) * (DH + 2);
+            const float c = (src[DH] == -CUDART_INF_F) ? 0.f : ex2(src[DH] - M);
+            num = fmaf(c, src[e], num);
+            den = fmaf(c, src[DH + 1], den);
+        }
+        const size_t idx = ((size_t)row * a.Hq + kvh * GQ + g) * n_splits + split;
+        a.part_o[idx * DH + e] = num;
+        if (e == 0) a.part_ml[idx] = make_float2(M, den);
+    }
+}
+
+// Merge the KV splits of every (row, head): out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s.
+template <int DH>
+__global__ void __launch_bounds__(DH) attn_combine_kernel(const StepMeta *meta, const int32_t *row_pos, int Hq,
+                                                          const float *part_o, const float2 *part_ml, float *out) {
+    const int head = blockIdx.x, row = blockIdx.y;
+    if (row >= meta->n_rows) return;
+    const int chunk = meta->attn_chunk, n_splits = meta->attn_splits;
+    const int ns = row_pos[row] / chunk + 1;
+    const size_t base = ((size_t)row * Hq + head) * n_splits;
+    float M = -CUDART_INF_F;
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, part_ml[base + s].x);
+    float num = 0.f, den = 0.f;
+    for (int s = 0; s < ns; ++s) {
+        const float2 ml = part_ml[base + s];
+        const float c = ex2(ml.x - M);
+        num = fmaf(c, part_o[(base + s) * DH + threadIdx.x], num);
+        den = fmaf(c, ml.y, den);
+    }
+    out[((size_t)row * Hq + head) * DH + threadIdx.x] = num / den;
+}
+
+inline size_t attn_smem_bytes(int DH, int GQ) {
+    const size_t stage = 2 * kAttnConsumers * (size_t)(kPage * DH * 2);
+    return 1024 + kAttnStages * stage + sizeof(float) * ((size_t)GQ * DH + kAttnConsumers * kPage * GQ +
+                                                         (size_t)kAttnConsumers * GQ * (DH + 2)) +
+           2 * kAttnStages * sizeof(uint64_t) + 64;
+}
+
+}  // namespace river

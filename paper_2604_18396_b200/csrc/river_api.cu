@@ -11,6 +11,7 @@
 
 #include "../../include/river.h"
 #include "river_kernels.cuh"
+#include "attn_decode.cuh"
 
 using namespace river;
 
@@ -48,10 +49,13 @@ struct river_ctx {
 
     // workspace
     float *h[3], *qbuf, *obuf, *act, *part_val, *tau_i, *logits_i, *scores_i;
-    float2 *rope_cs;
+    float2 *rope_cs, *part_ml;
+    float *part_o;
+    CUtensorMap kv_tmap;
+    int attn_splits_now = 1;
     double *inv_freq;
     int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
-    int32_t *meta_dev;  // [4 + 6*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows
+    int32_t *meta_dev;  // [kMetaHdr + 6*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows
     uint8_t *exited, *pass;
     int *dev_err;
     size_t ws_bytes = 0;
@@ -77,12 +81,12 @@ struct river_ctx {
     double prof_ms[kNumClasses] = {0}, prof_bytes[kNumClasses] = {0};
     int64_t prof_launches[kNumClasses] = {0};
 
-    int meta_ints() const { return 4 + 6 * cfg.max_batch; }
+    int meta_ints() const { return kMetaHdr + 6 * cfg.max_batch; }
     StepMeta *meta() const { return reinterpret_cast<StepMeta *>(meta_dev); }
-    int32_t *row_slot() const { return meta_dev + 4; }
-    int32_t *row_pos() const { return meta_dev + 4 + cfg.max_batch; }
-    int32_t *upd() const { return meta_dev + 4 + 2 * cfg.max_batch; }
-    int32_t *head_rows() const { return meta_dev + 4 + 5 * cfg.max_batch; }
+    int32_t *row_slot() const { return meta_dev + kMetaHdr; }
+    int32_t *row_pos() const { return meta_dev + kMetaHdr + cfg.max_batch; }
+    int32_t *upd() const { return meta_dev + kMetaHdr + 2 * cfg.max_batch; }
+    int32_t *head_rows() const { return meta_dev + kMetaHdr + 5 * cfg.max_batch; }
 };
 
 namespace {
@@ -137,7 +141,9 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     int32_t *na = cv.take<int32_t>(L + 1), *nr = cv.take<int32_t>(L + 1);
     int32_t *pt = cv.take<int32_t>((size_t)c->max_seqs * c->max_pages_per_seq);
     int32_t *tk = cv.take<int32_t>(B), *fo = cv.take<int32_t>(B), *ex = cv.take<int32_t>(B), *nx = cv.take<int32_t>(B);
-    int32_t *md = cv.take<int32_t>(4 + 6 * B);
+    int32_t *md = cv.take<int32_t>(kMetaHdr + 6 * B);
+    float *po = cv.take<float>((B + 600) * (size_t)c->Hq * c->dh);
+    float2 *pml = cv.take<float2>((B + 600) * (size_t)c->Hq);
     uint8_t *exd = cv.take<uint8_t>(B), *ps = cv.take<uint8_t>(B);
     int *de = cv.take<int>(1);
     if (x) {
@@ -145,7 +151,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
         x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
-        x->pass = ps; x->dev_err = de;
+        x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml;
     }
     return (cv.off + 255) & ~(size_t)255;
 }
@@ -196,11 +202,45 @@ W4 w4(const river_w4 &r) {
     return W4{(const uint8_t *)r.codes, (const uint16_t *)r.scale, (const uint16_t *)r.zero};
 }
 
+// KV split geometry of this step: enough (row, kv head, split) work items to fill the GPU about four times over,
+// splits of at least one 64-position tile.  The split count depends only on the row count, so a captured launch
+// stays valid while the chunk length grows with the context.
+void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
+    const river_config &g = c->cfg;
+    int max_pos = 0;
+    for (int i = 0; i < n; ++i) max_pos = std::max(max_pos, mh[kMetaHdr + g.max_batch + i]);
+    int S = (4 * c->num_sms + n * g.Hkv - 1) / (n * g.Hkv);
+    S = std::max(1, std::min(S, 64));
+    int chunk = (max_pos + 1 + S - 1) / S;
+    chunk = std::max(kAttnTile, (chunk + kAttnTile - 1) / kAttnTile * kAttnTile);
+    mh[3] = chunk;
+    mh[4] = S;
+    mh[5] = mh[6] = mh[7] = 0;
+    c->attn_splits_now = S;
+}
+
 template <int DH, int GQ>
 void launch_attn(river_ctx *c, int n, int layer0) {
     const river_config &g = c->cfg;
-    attn_decode_kernel<DH, GQ><<<dim3(g.Hkv, n), 128, 0, c->stream>>>(
-        c->meta(), c->qbuf, kv_addr(c, layer0), 1.0f / std::sqrt((float)DH), g.Hq, c->obuf);
+    if (g.flags & RIVER_F_SIMPLE_ATTN) {
+        attn_decode_kernel<DH, GQ><<<dim3(g.Hkv, n), 128, 0, c->stream>>>(
+            c->meta(), c->qbuf, kv_addr(c, layer0), 1.0f / std::sqrt((float)DH), g.Hq, c->obuf);
+        return;
+    }
+    AttnArgs a{};
+    a.meta = c->meta(); a.q = c->qbuf; a.page_tbl = c->page_tbl_dev; a.row_slot = c->row_slot(); a.row_pos = c->row_pos();
+    a.n_pages = g.n_pages; a.max_pages_per_seq = g.max_pages_per_seq; a.Hkv = g.Hkv; a.Hq = g.Hq; a.layer0 = layer0;
+    a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.dev_err = c->dev_err;
+    const size_t smem = attn_smem_bytes(DH, GQ);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(attn_split_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_set = true;
+    }
+    attn_split_kernel<DH, GQ><<<dim3(c->attn_splits_now, g.Hkv, n), kAttnThreads, smem, c->stream>>>(c->kv_tmap, a);
+    attn_combine_kernel<DH><<<dim3(g.Hq, n), DH, 0, c->stream>>>(c->meta(), c->row_pos(), g.Hq, c->part_o, c->part_ml,
+                                                               c->obuf);
 }
 
 int launch_attention(river_ctx *c, int n, int layer0) {
@@ -209,6 +249,30 @@ int launch_attention(river_ctx *c, int n, int layer0) {
     ATT(64, 1) ATT(64, 2) ATT(64, 4) ATT(64, 8) ATT(128, 1) ATT(128, 2) ATT(128, 4) ATT(128, 8)
 #undef ATT
     return -1;
+}
+
+// 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
+// 128-byte swizzle: one box is the K (or V) of one page, one kv head, one half of the head dim.
+int make_kv_tensor_map(river_ctx *c) {
+    const river_config &g = c->cfg;
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+        return fail(nullptr, RIVER_E_DEVICE, "cuTensorMapEncodeTiled is not available");
+    const cuuint64_t rows = (cuuint64_t)g.L * g.n_pages * 2 * g.Hkv * kPage;
+    if (rows >= (1ull << 31)) return fail(nullptr, RIVER_E_SHAPE, "KV pool has too many cache rows for one tensor map");
+    const cuuint64_t gdim[2] = {(cuuint64_t)g.dh, rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)g.dh * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = ((EncodeFn)fn)(&c->kv_tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->pool, gdim, gstride, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(nullptr, RIVER_E_DEVICE, "cuTensorMapEncodeTiled failed: " + std::to_string((int)r));
+    return 0;
 }
 
 // Allocate the page that position `pos` of `slot` falls in, if it has none yet; queue the device update.
@@ -222,7 +286,7 @@ int ensure_page(river_ctx *c, int slot, int pos, int32_t *mh, int &n_upd) {
     if (n_upd >= g.max_batch) return fail(c, RIVER_E_NOPAGE, "too many new pages in one step");
     e = c->free_pages.back();
     c->free_pages.pop_back();
-    int32_t *u = mh + 4 + 2 * g.max_batch;
+    int32_t *u = mh + kMetaHdr + 2 * g.max_batch;
     u[n_upd] = slot;
     u[g.max_batch + n_upd] = pi;
     u[2 * g.max_batch + n_upd] = e;
@@ -334,6 +398,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, const
         }
         {
             LaunchScope ls(c, K_ATTN, kv_read, 0, -1);
+            if (!(g.flags & RIVER_F_SIMPLE_ATTN)) ++c->st.launches_last_step;  // split kernel + combine kernel
             if (launch_attention(c, n, l - 1)) return fail(c, RIVER_E_SHAPE, "no attention kernel for this head geometry");
         }
         {
@@ -481,6 +546,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return bail("cudaGetDeviceProperties failed");
     if (prop.major != 10) return bail("this library is built for sm_100a (B200) only");
     c->num_sms = prop.multiProcessorCount;
+    if (make_kv_tensor_map(c)) { river_destroy(c); return RIVER_E_DEVICE; }
     for (int i = 0; i < kStaging; ++i) {
         if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");
         if (cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail("cudaEventCreate failed");
@@ -531,12 +597,13 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
     for (int b = 0; b < batch; ++b) {
         const int pos = c->seq_len[slots[b]];
         if (int rc = ensure_page(c, slots[b], pos, mh, n_upd)) return rc;
-        mh[4 + b] = slots[b];
-        mh[4 + g.max_batch + b] = pos;
-        mh[4 + 5 * g.max_batch + b] = b;
+        mh[kMetaHdr + b] = slots[b];
+        mh[kMetaHdr + g.max_batch + b] = pos;
+        mh[kMetaHdr + 5 * g.max_batch + b] = b;
         c->last_pos[b] = pos;
     }
-    mh[0] = batch; mh[1] = n_upd; mh[2] = batch; mh[3] = 0;
+    mh[0] = batch; mh[1] = n_upd; mh[2] = batch;
+    set_attn_meta(c, mh, batch);
     if (int rc = push_meta(c, mh)) return rc;
     if (int rc = run_rows(c, batch, batch, c->last_pos.data(), tok, tau, forced_exit, logits, next_tok, exit_layer, scores)) return rc;
     for (int b = 0; b < batch; ++b) c->seq_len[slots[b]] += 1;
@@ -617,19 +684,20 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
             const int len = offsets[s + 1] - offsets[s];
             if (offsets[s] + p != tok0 + n) break;  // token ids of a chunk must be contiguous in tok
             if (int rc = ensure_page(c, slots[s], p, mh, n_upd)) return rc;
-            mh[4 + n] = slots[s];
-            mh[4 + g.max_batch + n] = p;
+            mh[kMetaHdr + n] = slots[s];
+            mh[kMetaHdr + g.max_batch + n] = p;
             if (p == len - 1) {
-                mh[4 + 5 * g.max_batch + n_head] = n;
+                mh[kMetaHdr + 5 * g.max_batch + n_head] = n;
                 head_seq[n_head++] = s;
             }
             ++n;
             if (++p == len) { c->seq_len[slots[s]] = len; ++s; p = 0; }
         }
-        mh[0] = n; mh[1] = n_upd; mh[2] = n_head; mh[3] = 0;
+        mh[0] = n; mh[1] = n_upd; mh[2] = n_head;
+        set_attn_meta(c, mh, n);
         if (int rc = push_meta(c, mh)) return rc;
         const bool want_logits = logits_last && n_head > 0;
-        if (int rc = run_rows(c, n, n_head, mh + 4 + g.max_batch, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr,
+        if (int rc = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr,
                               c->next_i, c->exit_i, nullptr))
             return rc;
         for (int i = 0; i < n_head; ++i) {

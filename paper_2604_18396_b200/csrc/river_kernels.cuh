@@ -60,8 +60,11 @@ struct StepMeta {  // device-resident, rewritten by the host before every step
     int32_t n_rows;
     int32_t n_updates;
     int32_t n_head_rows;
-    int32_t pad;
+    int32_t attn_chunk;   // positions per KV split of the attention kernel (multiple of 64)
+    int32_t attn_splits;  // split slots per (row, head) in the partial buffers
+    int32_t pad[3];
 };
+constexpr int kMetaHdr = sizeof(StepMeta) / sizeof(int32_t);
 
 struct Lists {  // rows entering each block, per layer index 0..L
     int32_t *act_idx;  // [(L+1)][max_batch]

@@ -31,8 +31,14 @@ def _rope(X, n_heads, dh, theta):
     return X.reshape(T, n_heads * dh)
 
 
-def recompute(shape, bb, rv, tokens, exit_layers):
-    """-> logits [T,V], K [L,T,Hkv*dh] (after RoPE), V [L,T,Hkv*dh], scores [T,L]."""
+def _bf16(x):
+    import torch
+    return torch.from_numpy(x).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False):
+    """-> logits [T,V], K [L,T,Hkv*dh] (after RoPE), V [L,T,Hkv*dh], scores [T,L].
+    kv_bf16: keys and values are rounded to bf16 (through torch's cast) before they are used or returned."""
     tokens = np.asarray(tokens)
     e = np.asarray(exit_layers)
     T = len(tokens)
@@ -57,6 +63,8 @@ def recompute(shape, bb, rv, tokens, exit_layers):
         q = _rope(proj("wq", x), Hq, dh, shape.rope_theta).reshape(T, Hq, dh)
         k = _rope(proj("wk", x), Hkv, dh, shape.rope_theta)
         v = proj("wv", x)
+        if kv_bf16:
+            k, v = _bf16(k), _bf16(v)
         Ks.append(k)
         Vs.append(v)
         k3, v3 = k.reshape(T, Hkv, dh), v.reshape(T, Hkv, dh)

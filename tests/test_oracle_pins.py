@@ -97,6 +97,31 @@ def test_matches_bruteforce_recompute(tiny, mode):
         np.testing.assert_allclose(v, V[l], rtol=0, atol=1e-6)
 
 
+def test_bf16_cache_storage_matches_bruteforce(tiny):
+    # the optional 16-bit cache storage: every key / value is rounded to bf16 (ties to even) before any use
+    shape, bb, rv = tiny
+    prompt, steps = _tokens(shape, 9), _tokens(shape, 7, 1)
+    forced = synth.forced_exit_schedule(5, 0, len(steps), shape.L, shape.entry_layer).numpy()
+    o = orc.Oracle(shape, bb, rv, 1, 32, kv_store=1)
+    outs = _run(o, 0, prompt, steps, INF, forced, prefill_exit=3)
+    e = np.array([3] * len(prompt) + [int(r["exit_layer"][0]) for r in outs])
+    toks = np.concatenate([prompt, steps])
+    logits, K, V, _ = bruteforce.recompute(shape, bb, rv, toks, e, kv_bf16=True)
+    for t, r in enumerate(outs):
+        np.testing.assert_allclose(r["logits"][0], logits[len(prompt) + t], rtol=0, atol=1e-4)
+    mism = 0
+    for l in range(shape.L):
+        k, v = o.read_kv(0, l, 0, len(toks))
+        for got, want in ((k, K[l]), (v, V[l])):
+            assert np.array_equal(got, torch.from_numpy(got).to(torch.bfloat16).float().numpy())  # bf16 values
+            mism += int((got != want).sum())
+            assert np.abs(got - want).max() <= 2.0 ** -7 * np.abs(want).max()  # at most one bf16 step apart
+    assert mism <= 0.001 * 2 * shape.L * K[0].size  # rounding ties may fall either way, rarely
+    plain = orc.Oracle(shape, bb, rv, 1, 32)
+    ref = _run(plain, 0, prompt, steps, INF, forced, prefill_exit=3)
+    assert not np.array_equal(ref[-1]["logits"], outs[-1]["logits"])
+
+
 # ------------------------------------------------------------------ P3: identity river
 def test_identity_river_makes_exits_invisible():
     shape = synth.SHAPES["tiny"]
