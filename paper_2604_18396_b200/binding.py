@@ -169,7 +169,10 @@ class River:
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
         # NaN-filled pool: a cache position that is read before it was written shows up at once
         self.kv_pool = torch.full((kb // 2,), float("nan"), dtype=torch.bfloat16, device=dev)
-        self.stream = stream if stream is not None else torch.cuda.current_stream(dev)
+        if stream is None:
+            # graph replay cannot be captured on the legacy default stream: give the context a stream of its own
+            stream = torch.cuda.Stream(dev) if (cfg.flags & RIVER_F_GRAPH) else torch.cuda.current_stream(dev)
+        self.stream = stream
         h = C.c_void_p()
         rc = L.river_init(C.byref(cfg), C.byref(self._w), self.kv_pool.data_ptr(), kb, self.workspace.data_ptr(), ws,
                           C.c_void_p(self.stream.cuda_stream), C.byref(h))
@@ -179,6 +182,12 @@ class River:
         self.device = dev
 
     # -- helpers
+    def _order_after_current(self):
+        """Work queued on torch's current stream (input tensors) must precede the step on the context's stream."""
+        cur = torch.cuda.current_stream(self.device)
+        if cur != self.stream:
+            self.stream.wait_stream(cur)
+
     def _check(self, rc: int):
         if rc:
             raise RiverError(rc, load().river_last_error(self.h).decode())
@@ -198,6 +207,7 @@ class River:
     def prefill(self, slots: Sequence[int], tok: torch.Tensor, offsets: Sequence[int], prefill_exit_layer=None,
                 logits_last: Optional[torch.Tensor] = None, next_tok: Optional[torch.Tensor] = None):
         e = self.cfg.L if prefill_exit_layer is None else prefill_exit_layer
+        self._order_after_current()
         self._check(load().river_prefill(self.h, len(slots), _i32_host(slots), _dp(tok), _i32_host(offsets), e,
                                          _dp(logits_last), _dp(next_tok)))
 
@@ -205,6 +215,7 @@ class River:
                     forced_exit: Optional[torch.Tensor], logits: Optional[torch.Tensor], next_tok: torch.Tensor,
                     exit_layer: torch.Tensor, scores: Optional[torch.Tensor] = None, slots_c=None):
         sc = slots_c if slots_c is not None else _i32_host(slots)
+        self._order_after_current()
         self._check(load().river_decode_step(self.h, len(slots), sc, _dp(tok), _dp(tau), _dp(forced_exit),
                                              _dp(logits), _dp(next_tok), _dp(exit_layer), _dp(scores)))
 
@@ -219,10 +230,12 @@ class River:
         w = self.cfg.Hkv * self.cfg.dh
         k = torch.empty((n, w), dtype=torch.bfloat16, device=self.device)
         v = torch.empty((n, w), dtype=torch.bfloat16, device=self.device)
+        self._order_after_current()
         self._check(load().river_read_kv(self.h, slot, layer, pos0, n, k.data_ptr(), v.data_ptr()))
         return k, v
 
     def write_kv(self, slot: int, layer: int, pos0: int, k: torch.Tensor, v: torch.Tensor):
+        self._order_after_current()
         self._check(load().river_write_kv(self.h, slot, layer, pos0, k.shape[0], _dp(k), _dp(v)))
 
     def last_lists(self, batch: int):

@@ -73,6 +73,8 @@ struct AttnArgs {
     float qscale;          // log2(e) / sqrt(DH)
     float *part_o;         // [(row*Hq + head)*splits + split][DH]  unnormalised
     float2 *part_ml;       // same index: (max, sum) in the base-2 domain
+    unsigned *tickets;     // [rows][Hkv], zero between launches: the last split of a (row, kv head) merges them all
+    float *out;            // [rows][Hq*DH]
     int *dev_err;
 };
 
@@ -86,6 +88,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     constexpr int VE = DH / 32;                  // head dims per lane in P.V
 
     const int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
+    pdl_launch();
+    pdl_wait();
     if (row >= a.meta->n_rows) return;
     const int chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
     const int pos = a.row_pos[row], slot = a.row_slot[row];
@@ -102,6 +106,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     float *sm = sp + kAttnConsumers * kPage * GQ;                      // merge: [4][GQ][DH + 2]
     uint64_t *bars = reinterpret_cast<uint64_t *>(sm + kAttnConsumers * GQ * (DH + 2));  // full[S], empty[S]
     __shared__ int s_abort;
+    __shared__ bool s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -264,27 +269,30 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
         a.part_o[idx * DH + e] = num;
         if (e == 0) a.part_ml[idx] = make_float2(M, den);
     }
-}
-
-// Merge the KV splits of every (row, head): out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s.
-template <int DH>
-__global__ void __launch_bounds__(DH) attn_combine_kernel(const StepMeta *meta, const int32_t *row_pos, int Hq,
-                                                          const float *part_o, const float2 *part_ml, float *out) {
-    const int head = blockIdx.x, row = blockIdx.y;
-    if (row >= meta->n_rows) return;
-    const int chunk = meta->attn_chunk, n_splits = meta->attn_splits;
-    const int ns = row_pos[row] / chunk + 1;
-    const size_t base = ((size_t)row * Hq + head) * n_splits;
-    float M = -CUDART_INF_F;
-    for (int s = 0; s < ns; ++s) M = fmaxf(M, part_ml[base + s].x);
-    float num = 0.f, den = 0.f;
-    for (int s = 0; s < ns; ++s) {
-        const float2 ml = part_ml[base + s];
-        const float c = ex2(ml.x - M);
-        num = fmaf(c, part_o[(base + s) * DH + threadIdx.x], num);
-        den = fmaf(c, ml.y, den);
+    // the last split of this (row, kv head) to finish merges all of them:
+    // out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s  (atomic ticket, no spinning)
+    const int ns = pos / chunk + 1;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(&a.tickets[row * a.Hkv + kvh], 1u) == (unsigned)(ns - 1));
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int t = tid; t < GQ * DH; t += kAttnThreads) {
+        const int g = t / DH, e = t % DH;
+        const size_t base = ((size_t)row * a.Hq + kvh * GQ + g) * n_splits;
+        float M = -CUDART_INF_F;
+        for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&a.part_ml[base + s]).x);
+        float num = 0.f, den = 0.f;
+        for (int s = 0; s < ns; ++s) {
+            const float2 ml = __ldcg(&a.part_ml[base + s]);
+            const float c = ex2(ml.x - M);
+            num = fmaf(c, __ldcg(&a.part_o[(base + s) * DH + e]), num);
+            den = fmaf(c, ml.y, den);
+        }
+        a.out[((size_t)row * a.Hq + kvh * GQ + g) * DH + e] = num / den;
     }
-    out[((size_t)row * Hq + head) * DH + threadIdx.x] = num / den;
+    if (tid == 0) a.tickets[row * a.Hkv + kvh] = 0;
 }
 
 inline size_t attn_smem_bytes(int DH, int GQ) {

@@ -12,6 +12,7 @@
 #include "../../include/river.h"
 #include "river_kernels.cuh"
 #include "attn_decode.cuh"
+#include "gemv_ring.cuh"
 
 using namespace river;
 
@@ -53,6 +54,10 @@ struct river_ctx {
     float *part_o;
     CUtensorMap kv_tmap;
     int attn_splits_now = 1;
+    unsigned *attn_tickets, *tickets;  // [max_batch*Hkv], [4]
+    int32_t *hint_act;
+    struct GraphEntry { int n; bool scores; cudaGraphExec_t exec; int launches; };
+    std::vector<GraphEntry> graphs;
     double *inv_freq;
     int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
     int32_t *meta_dev;  // [kMetaHdr + 6*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows
@@ -146,12 +151,14 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     float2 *pml = cv.take<float2>((B + 600) * (size_t)c->Hq);
     uint8_t *exd = cv.take<uint8_t>(B), *ps = cv.take<uint8_t>(B);
     int *de = cv.take<int>(1);
+    unsigned *atk = cv.take<unsigned>(B * (size_t)c->Hkv), *tk4 = cv.take<unsigned>(4);
+    int32_t *hint = cv.take<int32_t>(1);
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
         x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
-        x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml;
+        x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
     }
     return (cv.off + 255) & ~(size_t)255;
 }
@@ -183,6 +190,25 @@ int launch_grid(river_ctx *c, Kern kern, int threads, size_t smem) {
         case 4: { constexpr int N = 4; __VA_ARGS__ } break;     \
         default: { constexpr int N = 8; __VA_ARGS__ } break;    \
     }
+
+// Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the
+// stream is still running and orders itself with griddepcontrol.wait.  Every kernel launched this way calls
+// griddepcontrol.wait before it touches anything a predecessor writes.
+template <class... KArgs, class... Args>
+cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                     Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
+}
 
 KvAddr kv_addr(const river_ctx *c, int layer0) {
     KvAddr k;
@@ -219,36 +245,97 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     c->attn_splits_now = S;
 }
 
+void set_io_meta(int32_t *mh, const int32_t *tok, const float *tau, const int32_t *forced, float *logits,
+                 int32_t *next_tok, int32_t *exit_layer, float *scores) {
+    StepMeta *m = reinterpret_cast<StepMeta *>(mh);
+    m->tok = tok; m->tau = tau; m->forced = forced; m->logits = logits; m->next_tok = next_tok;
+    m->exit_layer = exit_layer; m->scores = scores;
+}
+
 template <int DH, int GQ>
-void launch_attn(river_ctx *c, int n, int layer0) {
+cudaError_t launch_attn(river_ctx *c, int n, int layer0, bool pdl) {
     const river_config &g = c->cfg;
     if (g.flags & RIVER_F_SIMPLE_ATTN) {
         attn_decode_kernel<DH, GQ><<<dim3(g.Hkv, n), 128, 0, c->stream>>>(
             c->meta(), c->qbuf, kv_addr(c, layer0), 1.0f / std::sqrt((float)DH), g.Hq, c->obuf);
-        return;
+        return cudaGetLastError();
     }
     AttnArgs a{};
     a.meta = c->meta(); a.q = c->qbuf; a.page_tbl = c->page_tbl_dev; a.row_slot = c->row_slot(); a.row_pos = c->row_pos();
     a.n_pages = g.n_pages; a.max_pages_per_seq = g.max_pages_per_seq; a.Hkv = g.Hkv; a.Hq = g.Hq; a.layer0 = layer0;
     a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.dev_err = c->dev_err;
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.tickets = c->attn_tickets; a.out = c->obuf; a.dev_err = c->dev_err;
     const size_t smem = attn_smem_bytes(DH, GQ);
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(attn_split_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_set = true;
     }
-    attn_split_kernel<DH, GQ><<<dim3(c->attn_splits_now, g.Hkv, n), kAttnThreads, smem, c->stream>>>(c->kv_tmap, a);
-    attn_combine_kernel<DH><<<dim3(g.Hq, n), DH, 0, c->stream>>>(c->meta(), c->row_pos(), g.Hq, c->part_o, c->part_ml,
-                                                               c->obuf);
+    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(kAttnThreads), smem, c->stream,
+                    pdl, c->kv_tmap, a);
 }
 
-int launch_attention(river_ctx *c, int n, int layer0) {
+cudaError_t launch_attention(river_ctx *c, int n, int layer0, bool pdl) {
     const int gq = c->cfg.Hq / c->cfg.Hkv;
-#define ATT(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) { launch_attn<DH_, GQ_>(c, n, layer0); return 0; }
+#define ATT(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn<DH_, GQ_>(c, n, layer0, pdl);
     ATT(64, 1) ATT(64, 2) ATT(64, 4) ATT(64, 8) ATT(128, 1) ATT(128, 2) ATT(128, 4) ATT(128, 8)
 #undef ATT
-    return -1;
+    return cudaErrorInvalidValue;
+}
+
+// ---- ring projection launch: rows per stage for the two weight formats, ring depth, shared memory
+int ring_rb(int K) { return K > 2048 ? 2 : (K > 1024 ? 4 : 8); }  // rows x min(K, 4096) x 2 B <= 16 KB
+int ring_rw(int K, int group, int nrun) {
+    for (int r = 8; r >= 2; r >>= 1) {
+        const size_t bytes = (size_t)r * ((K >> 1) + 4 * (K / group));
+        const int rr = r / nrun;
+        if (rr < 1) continue;
+        if (bytes <= (size_t)kRingStageBytes && (size_t)r * (K >> 1) <= 16384 && (rr * (K / group) * 2) % 16 == 0)
+            return r;
+    }
+    return 0;  // this shape cannot use the ring kernel for 4-bit weights
+}
+
+template <class P, int N, int RB, int RW>
+cudaError_t launch_ring_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int has_river,
+                          bool pdl) {
+    RingGeom geom;
+    geom.xstride = xs_stride(K, 32);
+    int S = 6;
+    while (S > 4 && ring_smem_bytes(S, N, K) > 110 * 1024) --S;  // two kernels of the chain fit one SM together
+    geom.n_stages = S;
+    const size_t smem = ring_smem_bytes(S, N, K);
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaFuncSetAttribute(ring_proj_kernel<P, N, RB, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_smem = smem;
+    }
+    return launch_k(ring_proj_kernel<P, N, RB, RW>, dim3(c->num_sms), dim3(kRingThreads), smem, c->stream, pdl, p, in, rl,
+                    geom, has_river, c->dev_err);
+}
+
+template <class P>
+cudaError_t launch_ring(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int n, int has_river,
+                        bool pdl) {
+    const int rb = ring_rb(K), rw = ring_rw(K, c->cfg.group, P::NRUN);
+    int n_sel = 1;
+    while (n_sel < n && n_sel < 4 && ring_smem_bytes(4, n_sel * 2, K) <= 210 * 1024) n_sel *= 2;
+#define RING_CASE(N_, RB_, RW_) \
+    if (n_sel == N_ && rb == RB_ && rw == RW_) return launch_ring_t<P, N_, RB_, RW_>(c, p, in, rl, K, has_river, pdl);
+#define RING_N(RB_, RW_) RING_CASE(1, RB_, RW_) RING_CASE(2, RB_, RW_) RING_CASE(4, RB_, RW_)
+    RING_N(2, 8) RING_N(2, 4) RING_N(2, 2) RING_N(4, 8) RING_N(4, 4) RING_N(8, 8)
+#undef RING_N
+#undef RING_CASE
+    return cudaErrorInvalidValue;
+}
+
+bool ring_ok(const river_ctx *c, int K, int nrun) {
+    if (c->cfg.flags & RIVER_F_NO_RING) return false;
+    const int rb = ring_rb(K), rw = ring_rw(K, c->cfg.group, nrun);
+    if (rw == 0) return false;
+    const bool combo = (rb == 2 && (rw == 8 || rw == 4 || rw == 2)) || (rb == 4 && (rw == 8 || rw == 4)) ||
+                       (rb == 8 && rw == 8);
+    return combo;
 }
 
 // 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
@@ -346,9 +433,8 @@ int profile_collect(river_ctx *c) {
     return 0;
 }
 
-// The launch sequence of one step over the rows already described in the device metadata.
-int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, const int32_t *tok, const float *tau,
-             const int32_t *forced, float *logits, int32_t *next_tok, int32_t *exit_layer, float *scores) {
+// The launch sequence of one step over the rows described in the device metadata (rows, positions, caller buffers).
+int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
     const river_config &g = c->cfg;
     const int L = g.L, d = g.d, B = g.max_batch;
     c->st.launches_last_step = 0;
@@ -358,103 +444,133 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, const
     double kv_read = 0.0;
     for (int i = 0; i < n; ++i) kv_read += (double)(row_pos_host[i] + 1) * 2.0 * kvdim * 2.0;
     const double kv_write = (double)n * 2.0 * kvdim * 2.0;
+    cudaError_t err = cudaSuccess;
+    auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
 
     {
         LaunchScope ls(c, K_BEGIN, (double)n * d * 2.0, 0, -1);
-        step_begin_kernel<<<std::max(n, 1), 128, 0, c->stream>>>(
-            c->meta(), c->upd(), c->page_tbl_dev, g.max_pages_per_seq, B, tok, c->embed, d, g.V, c->h[0], c->row_pos(),
-            c->inv_freq, g.dh / 2, c->rope_cs, forced, L, g.entry_layer, c->exited, exit_layer, scores, c->dev_err);
+        note(launch_k(step_begin_kernel, dim3(std::max(n, 1)), dim3(128), 0, c->stream, false, c->meta(), c->upd(),
+                      c->page_tbl_dev, g.max_pages_per_seq, B, c->embed, d, g.V, c->h[0], c->row_pos(), c->inv_freq,
+                      g.dh / 2, c->rope_cs, L, g.entry_layer, c->exited, c->dev_err, lists, c->hint_act, c->tickets));
     }
-    {
-        LaunchScope ls(c, K_COMPACT, 0, 0, -1);
-        compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), 0, L, g.entry_layer, g.exit_mode, c->pass, forced,
-                                                  c->exited, exit_layer, lists);
-    }
-
-    int hi = 0;  // h[hi] = block input
+    int hi = 0;                  // h[hi] = block input
     for (int l = 1; l <= L; ++l) {
         const river_layer_weights &w = c->layers[l - 1];
         const int has_river = w.rq.codes != nullptr;
         const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
         const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
+        const RowLists rl{ai, na, ri, nr, c->hint_act};
         float *h_in = c->h[hi], *h_mid = c->h[(hi + 1) % 3], *h_out = c->h[(hi + 2) % 3];
+        // ---- a2: attention norm + QKV + RoPE + KV write
         {
-            QkvArgs a{};
-            a.wq = (const uint16_t *)w.wq; a.wk = (const uint16_t *)w.wk; a.wv = (const uint16_t *)w.wv;
-            a.rq = w4(w.rq); a.rk = w4(w.rk); a.rv = w4(w.rv);
-            a.has_river = has_river;
-            a.in = ProjIn{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
-            a.d = d; a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh; a.group = g.group;
-            a.rope_cs = c->rope_cs; a.q_out = c->qbuf; a.kv = kv_addr(c, l - 1);
-            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr; a.dev_err = c->dev_err;
-            const int n_sel = pick_n(n, d);
-            const size_t smem = proj_smem(n_sel, d);
             const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
             LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
-            DISPATCH_N(n_sel, {
-                const int grid = launch_grid(c, qkv_rope_kv_kernel<N>, 256, smem);
-                qkv_rope_kv_kernel<N><<<grid, 256, smem, c->stream>>>(a);
-            });
+            const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
+            if (ring_ok(c, d, 2)) {
+                QkvProblem p{};
+                p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
+                p.rq = w4(w.rq); p.rk = w4(w.rk); p.rv = w4(w.rv);
+                p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
+                p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
+                note(launch_ring(c, p, in, rl, d, n, has_river, true));
+            } else {
+                QkvArgs a{};
+                a.wq = (const uint16_t *)w.wq; a.wk = (const uint16_t *)w.wk; a.wv = (const uint16_t *)w.wv;
+                a.rq = w4(w.rq); a.rk = w4(w.rk); a.rv = w4(w.rv);
+                a.has_river = has_river; a.in = in;
+                a.d = d; a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh; a.group = g.group;
+                a.rope_cs = c->rope_cs; a.q_out = c->qbuf; a.kv = kv_addr(c, l - 1);
+                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr; a.dev_err = c->dev_err;
+                const int n_sel = pick_n(n, d);
+                const size_t smem = proj_smem(n_sel, d);
+                DISPATCH_N(n_sel, {
+                    const int grid = launch_grid(c, qkv_rope_kv_kernel<N>, 256, smem);
+                    qkv_rope_kv_kernel<N><<<grid, 256, smem, c->stream>>>(a);
+                });
+            }
         }
+        // ---- a3: paged GQA decode attention
         {
             LaunchScope ls(c, K_ATTN, kv_read, 0, -1);
-            if (!(g.flags & RIVER_F_SIMPLE_ATTN)) ++c->st.launches_last_step;  // split kernel + combine kernel
-            if (launch_attention(c, n, l - 1)) return fail(c, RIVER_E_SHAPE, "no attention kernel for this head geometry");
+            note(launch_attention(c, n, l - 1, !(g.flags & RIVER_F_SIMPLE_ATTN)));
         }
+        // ---- a4: O projection + residual
         {
-            ResidArgs a{};
-            a.w = (const uint16_t *)w.wo; a.rw = w4(w.ro); a.has_river = has_river;
-            a.in = ProjIn{c->obuf, nullptr, 0.f};
-            a.K = qdim; a.out_dim = d; a.group = g.group; a.resid = h_in; a.out = h_mid;
-            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-            const int n_sel = pick_n(n, qdim);
-            const size_t smem = proj_smem(n_sel, qdim);
             const double wb = 2.0 * qdim * d;
             LaunchScope ls(c, K_OPROJ, wb, wb * w4f, l - 1);
-            DISPATCH_N(n_sel, {
-                const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
-                proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
-            });
+            const ProjIn in{c->obuf, nullptr, 0.f};
+            if (ring_ok(c, qdim, 1)) {
+                ResidProblem p{};
+                p.w = (const uint16_t *)w.wo; p.rw = w4(w.ro); p.K = qdim; p.out_dim = d; p.group = g.group;
+                p.resid = h_in; p.out = h_mid;
+                note(launch_ring(c, p, in, rl, qdim, n, has_river, !(g.flags & RIVER_F_SIMPLE_ATTN)));
+            } else {
+                ResidArgs a{};
+                a.w = (const uint16_t *)w.wo; a.rw = w4(w.ro); a.has_river = has_river; a.in = in;
+                a.K = qdim; a.out_dim = d; a.group = g.group; a.resid = h_in; a.out = h_mid;
+                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
+                const int n_sel = pick_n(n, qdim);
+                const size_t smem = proj_smem(n_sel, qdim);
+                DISPATCH_N(n_sel, {
+                    const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
+                    proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
+                });
+            }
         }
+        // ---- a5: FFN norm + gate/up + SwiGLU
         {
-            GateUpArgs a{};
-            a.wg = (const uint16_t *)w.wg; a.wu = (const uint16_t *)w.wu; a.rg = w4(w.rg); a.ru = w4(w.ru);
-            a.has_river = has_river;
-            a.in = ProjIn{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
-            a.d = d; a.F = g.F; a.group = g.group; a.act = c->act;
-            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-            const int n_sel = pick_n(n, d);
-            const size_t smem = proj_smem(n_sel, d);
             const double wb = 2.0 * 2.0 * g.F * d;
             LaunchScope ls(c, K_GATEUP, wb, wb * w4f, l - 1);
-            DISPATCH_N(n_sel, {
-                const int grid = launch_grid(c, gateup_kernel<N>, 256, smem);
-                gateup_kernel<N><<<grid, 256, smem, c->stream>>>(a);
-            });
+            const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
+            if (ring_ok(c, d, 2)) {
+                GateUpProblem p{};
+                p.wg = (const uint16_t *)w.wg; p.wu = (const uint16_t *)w.wu; p.rg = w4(w.rg); p.ru = w4(w.ru);
+                p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
+                note(launch_ring(c, p, in, rl, d, n, has_river, ring_ok(c, qdim, 1)));
+            } else {
+                GateUpArgs a{};
+                a.wg = (const uint16_t *)w.wg; a.wu = (const uint16_t *)w.wu; a.rg = w4(w.rg); a.ru = w4(w.ru);
+                a.has_river = has_river; a.in = in;
+                a.d = d; a.F = g.F; a.group = g.group; a.act = c->act;
+                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
+                const int n_sel = pick_n(n, d);
+                const size_t smem = proj_smem(n_sel, d);
+                DISPATCH_N(n_sel, {
+                    const int grid = launch_grid(c, gateup_kernel<N>, 256, smem);
+                    gateup_kernel<N><<<grid, 256, smem, c->stream>>>(a);
+                });
+            }
         }
+        // ---- a5: down projection + residual
+        bool down_ring = ring_ok(c, g.F, 1);
         {
-            ResidArgs a{};
-            a.w = (const uint16_t *)w.wd; a.rw = w4(w.rd); a.has_river = has_river;
-            a.in = ProjIn{c->act, nullptr, 0.f};
-            a.K = g.F; a.out_dim = d; a.group = g.group; a.resid = h_mid; a.out = h_out;
-            a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-            const int n_sel = pick_n(n, g.F);
-            const size_t smem = proj_smem(n_sel, g.F);
             const double wb = 2.0 * g.F * d;
             LaunchScope ls(c, K_DOWN, wb, wb * w4f, l - 1);
-            DISPATCH_N(n_sel, {
-                const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
-                proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
-            });
+            const ProjIn in{c->act, nullptr, 0.f};
+            if (down_ring) {
+                ResidProblem p{};
+                p.w = (const uint16_t *)w.wd; p.rw = w4(w.rd); p.K = g.F; p.out_dim = d; p.group = g.group;
+                p.resid = h_mid; p.out = h_out;
+                note(launch_ring(c, p, in, rl, g.F, n, has_river, ring_ok(c, d, 2)));
+            } else {
+                ResidArgs a{};
+                a.w = (const uint16_t *)w.wd; a.rw = w4(w.rd); a.has_river = has_river; a.in = in;
+                a.K = g.F; a.out_dim = d; a.group = g.group; a.resid = h_mid; a.out = h_out;
+                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
+                const int n_sel = pick_n(n, g.F);
+                const size_t smem = proj_smem(n_sel, g.F);
+                DISPATCH_N(n_sel, {
+                    const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
+                    proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
+                });
+            }
         }
-        if (l < L || scores) {
-            LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
-            exit_score_kernel<<<n, 256, 0, c->stream>>>(ai, na, h_in, h_out, d, tau, c->pass, scores, L, l);
-        }
+        // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
         {
-            LaunchScope ls(c, K_COMPACT, 0, 0, -1);
-            compact_kernel<<<1, 1024, 0, c->stream>>>(c->meta(), l, L, g.entry_layer, g.exit_mode, c->pass, forced,
-                                                      c->exited, exit_layer, lists);
+            LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
+            note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, down_ring, c->meta(), l, L,
+                          g.entry_layer, g.exit_mode, (const float *)h_in, (const float *)h_out, d, c->pass, c->exited,
+                          lists, c->hint_act, c->tickets + 1));
         }
         hi = (hi + 2) % 3;
     }
@@ -462,30 +578,61 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, const
         HeadArgs a{};
         a.w = c->lm_head;
         a.in = ProjIn{c->h[hi], c->final_norm, g.rms_eps};
-        a.d = d; a.V = g.V; a.rows = c->head_rows(); a.meta = c->meta(); a.logits = logits;
+        a.d = d; a.V = g.V; a.rows = c->head_rows(); a.meta = c->meta();
         a.part_val = c->part_val; a.part_idx = c->part_idx;
         const int n_sel = std::min(pick_n(n_head, d), 4);
         const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xs_stride(d, 8));
         {
-            LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + (logits ? 4.0 * n_head * g.V : 0.0), 0, -1);
+            LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + 4.0 * n_head * g.V, 0, -1);
             switch (n_sel) {
                 case 1: cudaFuncSetAttribute(lm_head_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        lm_head_kernel<1, 4><<<c->head_grid, 256, smem, c->stream>>>(a); break;
+                        note(launch_k(lm_head_kernel<1, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a)); break;
                 case 2: cudaFuncSetAttribute(lm_head_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        lm_head_kernel<2, 4><<<c->head_grid, 256, smem, c->stream>>>(a); break;
+                        note(launch_k(lm_head_kernel<2, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a)); break;
                 default: cudaFuncSetAttribute(lm_head_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        lm_head_kernel<4, 4><<<c->head_grid, 256, smem, c->stream>>>(a); break;
+                        note(launch_k(lm_head_kernel<4, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a)); break;
             }
         }
         {
             LaunchScope ls(c, K_ARGMAX, 0, 0, -1);
-            argmax_final_kernel<<<n_head, 128, 0, c->stream>>>(c->meta(), c->part_val, c->part_idx, c->head_grid, next_tok);
+            note(launch_k(argmax_final_kernel, dim3(n_head), dim3(128), 0, c->stream, true, c->meta(),
+                          (const float *)c->part_val, (const int32_t *)c->part_idx, c->head_grid));
         }
     }
-    CUDA_TRY(c, cudaGetLastError());
+    if (err == cudaSuccess) err = cudaGetLastError();
+    if (err != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(err));
     c->st.launches_total += c->st.launches_last_step;
     if (c->profiling) return profile_collect(c);
     return 0;
+}
+
+// One decode step through a CUDA graph of the launch sequence (captured the second time a row count is seen; the
+// per-step inputs live in device memory, so the graph never needs new parameters).
+int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
+    const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
+    if (!use_graph) return run_rows(c, n, n, row_pos_host);
+    for (auto &ge : c->graphs)
+        if (ge.n == n) {
+            if (!ge.exec) {  // second use: capture
+                cudaGraph_t graph = nullptr;
+                CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+                const int rc = run_rows(c, n, n, row_pos_host);
+                const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+                if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
+                if (e != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("graph capture failed: ") + cudaGetErrorString(e));
+                const cudaError_t e2 = cudaGraphInstantiate(&ge.exec, graph, 0);
+                cudaGraphDestroy(graph);
+                if (e2 != cudaSuccess) { ge.exec = nullptr; return fail(c, RIVER_E_DEVICE, std::string("graph instantiate failed: ") + cudaGetErrorString(e2)); }
+                ge.launches = c->st.launches_last_step;
+                c->st.launches_total -= ge.launches;  // capturing launched nothing
+            }
+            CUDA_TRY(c, cudaGraphLaunch(ge.exec, c->stream));
+            c->st.launches_last_step = ge.launches;
+            c->st.launches_total += ge.launches;
+            return 0;
+        }
+    c->graphs.push_back({n, false, nullptr, 0});
+    return run_rows(c, n, n, row_pos_host);  // first use: plain launches (also sets the kernels' attributes)
 }
 
 int check_slot(const river_ctx *c, int slot) { return slot >= 0 && slot < c->cfg.max_seqs; }
@@ -532,6 +679,10 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     c->lm_head = (const uint16_t *)w->lm_head;
     c->final_norm = (const uint16_t *)w->final_norm;
     c->stream = (cudaStream_t)cuda_stream;
+    if ((cfg->flags & RIVER_F_GRAPH) && (c->stream == nullptr || c->stream == cudaStreamLegacy)) {
+        delete c;
+        return fail(nullptr, RIVER_E_BADARG, "RIVER_F_GRAPH needs a stream other than the default stream");
+    }
     c->pool = (__nv_bfloat16 *)kv_pool;
     c->ws_bytes = carve(cfg, c, (char *)workspace);
     c->head_grid = head_grid_for(cfg);
@@ -570,6 +721,9 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     cudaError_t e = cudaMemcpyAsync(c->inv_freq, fr.data(), sizeof(double) * fr.size(), cudaMemcpyHostToDevice, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->page_tbl_dev, 0xff, sizeof(int32_t) * c->page_tbl.size(), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->hint_act, 0, sizeof(int32_t), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_act, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_riv, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
@@ -604,8 +758,9 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
     }
     mh[0] = batch; mh[1] = n_upd; mh[2] = batch;
     set_attn_meta(c, mh, batch);
+    set_io_meta(mh, tok, tau, forced_exit, logits, next_tok, exit_layer, scores);
     if (int rc = push_meta(c, mh)) return rc;
-    if (int rc = run_rows(c, batch, batch, c->last_pos.data(), tok, tau, forced_exit, logits, next_tok, exit_layer, scores)) return rc;
+    if (int rc = run_step(c, batch, c->last_pos.data())) return rc;
     for (int b = 0; b < batch; ++b) c->seq_len[slots[b]] += 1;
     c->st.steps += 1;
     c->st.batch_last = batch;
@@ -695,11 +850,11 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
         }
         mh[0] = n; mh[1] = n_upd; mh[2] = n_head;
         set_attn_meta(c, mh, n);
-        if (int rc = push_meta(c, mh)) return rc;
         const bool want_logits = logits_last && n_head > 0;
-        if (int rc = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr,
-                              c->next_i, c->exit_i, nullptr))
-            return rc;
+        set_io_meta(mh, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr, c->next_i, c->exit_i,
+                    nullptr);
+        if (int rc = push_meta(c, mh)) return rc;
+        if (int rc = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch)) return rc;
         for (int i = 0; i < n_head; ++i) {
             if (logits_last)
                 CUDA_TRY(c, cudaMemcpyAsync(logits_last + (size_t)head_seq[i] * g.V, c->logits_i + (size_t)i * g.V,
@@ -851,6 +1006,7 @@ void river_destroy(river_ctx *c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     for (auto &e : c->prof_ev) cudaEventDestroy(e);
+    for (auto &ge : c->graphs) if (ge.exec) cudaGraphExecDestroy(ge.exec);
     for (int i = 0; i < kStaging; ++i) {
         if (c->meta_host[i]) { cudaFreeHost(c->meta_host[i]); cudaEventDestroy(c->meta_ev[i]); }
     }

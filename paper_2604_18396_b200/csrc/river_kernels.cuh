@@ -63,6 +63,14 @@ struct StepMeta {  // device-resident, rewritten by the host before every step
     int32_t attn_chunk;   // positions per KV split of the attention kernel (multiple of 64)
     int32_t attn_splits;  // split slots per (row, head) in the partial buffers
     int32_t pad[3];
+    // the caller's device buffers of this step (read through here so that a captured launch sequence never changes)
+    const int32_t *tok;
+    const float *tau;
+    const int32_t *forced;  // may be null
+    float *logits;          // may be null
+    int32_t *next_tok;
+    int32_t *exit_layer;
+    float *scores;          // may be null
 };
 constexpr int kMetaHdr = sizeof(StepMeta) / sizeof(int32_t);
 
@@ -80,137 +88,182 @@ struct W4 {
     const uint16_t *zero;
 };
 
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Stable partition of the rows by the sticky exit flag, run by ONE CTA (any number of threads >= 32, multiple of
+// 32): ascending row ids of the rows still in the backbone and of the rows in the exit layers, and their counts.
+__device__ __forceinline__ void build_lists(int n, const uint8_t *exited, int l, const Lists &lists,
+                                            int32_t *hint_act, int *s_cnt /* shared, 2 * 32 + 2 ints */) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    int32_t *A = lists.act_idx + (size_t)l * lists.max_batch;
+    int32_t *R = lists.riv_idx + (size_t)l * lists.max_batch;
+    if (tid == 0) { s_cnt[64] = 0; s_cnt[65] = 0; }
+    __syncthreads();
+    for (int b0 = 0; b0 < n; b0 += blockDim.x) {
+        const int b = b0 + tid;
+        const bool valid = b < n;
+        const bool gone = valid && exited[b] != 0;
+        const unsigned ma = __ballot_sync(0xffffffffu, valid && !gone);
+        const unsigned mr = __ballot_sync(0xffffffffu, valid && gone);
+        if (lane == 0) { s_cnt[warp] = __popc(ma); s_cnt[32 + warp] = __popc(mr); }
+        __syncthreads();
+        int base_a = s_cnt[64], base_r = s_cnt[65], tot_a = 0, tot_r = 0;
+        for (int w = 0; w < nwarps; ++w) {
+            if (w < warp) { base_a += s_cnt[w]; base_r += s_cnt[32 + w]; }
+            tot_a += s_cnt[w];
+            tot_r += s_cnt[32 + w];
+        }
+        const unsigned lt = (1u << lane) - 1u;
+        if (valid) {
+            if (!gone) A[base_a + __popc(ma & lt)] = b;
+            else R[base_r + __popc(mr & lt)] = b;
+        }
+        __syncthreads();
+        if (tid == 0) { s_cnt[64] += tot_a; s_cnt[65] += tot_r; }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        lists.n_act[l] = s_cnt[64];
+        lists.n_riv[l] = s_cnt[65];
+        *hint_act = s_cnt[64];
+    }
+}
+
 // ---------------------------------------------------------------- step prologue
 // Applies the page-table updates of this step, embeds the tokens (a0), resets the per-row exit state and the
 // score diagnostics, and tabulates cos/sin of the rotary angles of every row's position.
 __global__ void step_begin_kernel(const StepMeta *meta, const int32_t *upd, /* [3][max_batch]: slot, idx, page */
-                                  int32_t *page_tbl, int max_pages_per_seq, int max_batch, const int32_t *tok,
+                                  int32_t *page_tbl, int max_pages_per_seq, int max_batch,
                                   const uint16_t *embed, int d, int V, float *h0, const int32_t *row_pos,
-                                  const double *inv_freq, int half_dh, float2 *rope_cs, const int32_t *forced,
-                                  int L, int entry_layer, uint8_t *exited, int32_t *exit_layer, float *scores,
-                                  int *dev_err) {
+                                  const double *inv_freq, int half_dh, float2 *rope_cs,
+                                  int L, int entry_layer, uint8_t *exited,
+                                  int *dev_err, Lists lists, int32_t *hint_act, unsigned *ticket) {
+    __shared__ int s_cnt[66];
+    __shared__ bool s_last;
+    pdl_launch();
+    pdl_wait();
     const int b = blockIdx.x;
     const int n_rows = meta->n_rows;
+    const int32_t *tok = meta->tok, *forced = meta->forced;
+    int32_t *exit_layer = meta->exit_layer;
+    float *scores = meta->scores;
     if (b == 0) {
         for (int i = threadIdx.x; i < meta->n_updates; i += blockDim.x)
             page_tbl[(size_t)upd[i] * max_pages_per_seq + upd[max_batch + i]] = upd[2 * max_batch + i];
     }
-    if (b >= n_rows) return;
-    int t = tok[b];
-    if (t < 0 || t >= V) {
-        if (threadIdx.x == 0) atomicExch(dev_err, DEV_BAD_TOKEN);
-        t = 0;
-    }
-    const uint16_t *e = embed + (size_t)t * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) h0[(size_t)b * d + i] = bf16f(e[i]);
-    const int pos = row_pos[b];
-    for (int i = threadIdx.x; i < half_dh; i += blockDim.x) {
-        double s, c;
-        sincos((double)pos * inv_freq[i], &s, &c);
-        rope_cs[(size_t)b * half_dh + i] = make_float2((float)c, (float)s);
-    }
-    if (scores)
-        for (int i = threadIdx.x; i < L; i += blockDim.x) scores[(size_t)b * L + i] = CUDART_NAN_F;
-    if (threadIdx.x == 0) {
-        int f = forced ? forced[b] : -1;
-        if (f >= 0 && (f > L || f < entry_layer)) {
-            atomicExch(dev_err, DEV_BAD_FORCED);
-            f = L;
+    if (b < n_rows) {
+        int t = tok[b];
+        if (t < 0 || t >= V) {
+            if (threadIdx.x == 0) atomicExch(dev_err, DEV_BAD_TOKEN);
+            t = 0;
         }
-        const bool gone = (f == 0);
-        exited[b] = gone ? 1 : 0;
-        exit_layer[b] = gone ? 0 : L;
+        const uint16_t *e = embed + (size_t)t * d;
+        for (int i = threadIdx.x; i < d; i += blockDim.x) h0[(size_t)b * d + i] = bf16f(e[i]);
+        const int pos = row_pos[b];
+        for (int i = threadIdx.x; i < half_dh; i += blockDim.x) {
+            double s, c;
+            sincos((double)pos * inv_freq[i], &s, &c);
+            rope_cs[(size_t)b * half_dh + i] = make_float2((float)c, (float)s);
+        }
+        if (scores)
+            for (int i = threadIdx.x; i < L; i += blockDim.x) scores[(size_t)b * L + i] = CUDART_NAN_F;
+        if (threadIdx.x == 0) {
+            int f = forced ? forced[b] : -1;
+            if (f >= 0 && (f > L || f < entry_layer)) {
+                atomicExch(dev_err, DEV_BAD_FORCED);
+                f = L;
+            }
+            const bool gone = (f == 0);
+            exited[b] = gone ? 1 : 0;
+            exit_layer[b] = gone ? 0 : L;
+        }
+    }
+    // the last CTA to finish builds the row lists entering block 1 (a7)
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        build_lists(n_rows, exited, 0, lists, hint_act, s_cnt);
+        if (threadIdx.x == 0) *ticket = 0;
     }
 }
 
-// ---------------------------------------------------------------- a7: row compaction (bit-exact, one CTA)
-// Takes the pass flags of Eq. 1 for the rows that just ran backbone block l (l = 0: before block 1), applies the
-// eligibility window entry_layer <= l < L, the forced-exit hook and the batch mode, updates the sticky exit state
-// and emits the two ascending row lists (stable partition) and their counts for block l+1.
-__global__ void __launch_bounds__(1024) compact_kernel(const StepMeta *meta, int l, int L, int entry_layer,
-                                                       int exit_mode, const uint8_t *pass, const int32_t *forced,
-                                                       uint8_t *exited, int32_t *exit_layer, Lists lists) {
-    __shared__ int s_warp_a[32], s_warp_r[32], s_allpass;
+// ---------------------------------------------------------------- a6 + a7: exit score, decision, compaction
+// One CTA per row of the step.  A row still in the backbone gets s = <h_in, h_out> / (|h_in| |h_out|) (Eq. 1) in
+// fp32 with a fixed reduction order and the flag s > tau (strict; NaN fails; a zero norm gives s = 0).  The last
+// CTA to finish (atomic ticket, no spinning) applies the eligibility window entry_layer <= l < L, the forced-exit
+// hook and the batch mode to the flags, updates the sticky exit state and emits the two ascending row lists
+// (a stable partition, bit-exact) and their counts for block l+1.
+__global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta, int l, int L, int entry_layer,
+                                                            int exit_mode, const float *h_in, const float *h_out,
+                                                            int d, uint8_t *pass, uint8_t *exited, Lists lists,
+                                                            int32_t *hint_act, unsigned *ticket) {
+    __shared__ float red[3][8];
+    __shared__ int s_cnt[66];
+    __shared__ bool s_last;
+    __shared__ int s_allpass;
+    pdl_launch();
+    pdl_wait();
     const int n = meta->n_rows;
-    const int b = threadIdx.x, lane = b & 31, warp = b >> 5;
-    if (b == 0) s_allpass = 1;
-    __syncthreads();
-    bool gone = false, valid = b < n;
-    if (valid) gone = exited[b] != 0;
+    const float *tau = meta->tau;
+    const int32_t *forced = meta->forced;
+    int32_t *exit_layer = meta->exit_layer;
+    float *scores = meta->scores;
+    const int row = blockIdx.x;
     const bool eligible = (l >= 1) && (l >= entry_layer) && (l < L);
-    bool p = valid && !gone && eligible && pass[b];
-    if (exit_mode == 1) {
-        if (valid && !gone && !(eligible && pass[b])) atomicAnd(&s_allpass, 0);
+    if (row < n && exited[row] == 0 && (eligible || scores)) {
+        const float4 *a = reinterpret_cast<const float4 *>(h_in + (size_t)row * d);
+        const float4 *b = reinterpret_cast<const float4 *>(h_out + (size_t)row * d);
+        float ab = 0.f, aa = 0.f, bb = 0.f;
+        for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+            const float4 x = a[i], y = b[i];
+            ab += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
+            aa += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+            bb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+        }
+        ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        if (lane == 0) { red[0][warp] = ab; red[1][warp] = aa; red[2][warp] = bb; }
         __syncthreads();
-        p = valid && !gone && eligible && (s_allpass != 0);
+        if (threadIdx.x == 0) {
+            ab = aa = bb = 0.f;
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { ab += red[0][w]; aa += red[1][w]; bb += red[2][w]; }
+            float s = 0.f;
+            if (aa > 0.f && bb > 0.f) s = ab / (sqrtf(aa) * sqrtf(bb));
+            pass[row] = (s > tau[row]) ? 1 : 0;
+            if (scores) scores[(size_t)row * L + (l - 1)] = s;
+        }
     }
-    if (valid && !gone && l >= 1) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // ---- decision for every row still in the backbone
+    if (threadIdx.x == 0) s_allpass = 1;
+    __syncthreads();
+    if (exit_mode == 1) {
+        for (int b = threadIdx.x; b < n; b += blockDim.x)
+            if (exited[b] == 0 && !(eligible && pass[b])) atomicAnd(&s_allpass, 0);
+        __syncthreads();
+    }
+    for (int b = threadIdx.x; b < n; b += blockDim.x) {
+        if (exited[b] != 0) continue;
+        bool leave = eligible && (exit_mode == 1 ? (s_allpass != 0) : (pass[b] != 0));
         const int f = forced ? forced[b] : -1;
-        bool leave = p;
         if (f >= 0) leave = (f == l) && (l < L);
         if (leave) {
-            gone = true;
             exited[b] = 1;
             exit_layer[b] = l;
         }
     }
-    const unsigned ma = __ballot_sync(0xffffffffu, valid && !gone);
-    const unsigned mr = __ballot_sync(0xffffffffu, valid && gone);
-    if (lane == 0) {
-        s_warp_a[warp] = __popc(ma);
-        s_warp_r[warp] = __popc(mr);
-    }
     __syncthreads();
-    int base_a = 0, base_r = 0, tot_a = 0, tot_r = 0;
-    for (int w = 0; w < 32; ++w) {
-        if (w < warp) { base_a += s_warp_a[w]; base_r += s_warp_r[w]; }
-        tot_a += s_warp_a[w];
-        tot_r += s_warp_r[w];
-    }
-    const unsigned lt = (1u << lane) - 1u;
-    int32_t *A = lists.act_idx + (size_t)l * lists.max_batch;
-    int32_t *R = lists.riv_idx + (size_t)l * lists.max_batch;
-    if (valid) {
-        if (!gone) A[base_a + __popc(ma & lt)] = b;
-        else R[base_r + __popc(mr & lt)] = b;
-    }
-    if (b == 0) {
-        lists.n_act[l] = tot_a;
-        lists.n_riv[l] = tot_r;
-    }
-}
-
-// ---------------------------------------------------------------- a6: exit score (Eq. 1)
-// One CTA per row still in the backbone: s = <h_in, h_out> / (|h_in| |h_out|) in fp32 with a fixed reduction
-// order; emits the pass flag s > tau (strict; NaN fails; a zero norm gives s = 0) and the score diagnostic.
-__global__ void __launch_bounds__(256) exit_score_kernel(const int32_t *act_idx, const int32_t *n_act,
-                                                         const float *h_in, const float *h_out, int d,
-                                                         const float *tau, uint8_t *pass, float *scores, int L,
-                                                         int l) {
-    if ((int)blockIdx.x >= *n_act) return;
-    const int row = act_idx[blockIdx.x];
-    const float4 *a = reinterpret_cast<const float4 *>(h_in + (size_t)row * d);
-    const float4 *b = reinterpret_cast<const float4 *>(h_out + (size_t)row * d);
-    float ab = 0.f, aa = 0.f, bb = 0.f;
-    for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
-        const float4 x = a[i], y = b[i];
-        ab += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
-        aa += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-        bb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
-    }
-    __shared__ float red[3][8];
-    ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) { red[0][warp] = ab; red[1][warp] = aa; red[2][warp] = bb; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        ab = aa = bb = 0.f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { ab += red[0][w]; aa += red[1][w]; bb += red[2][w]; }
-        float s = 0.f;
-        if (aa > 0.f && bb > 0.f) s = ab / (sqrtf(aa) * sqrtf(bb));
-        pass[row] = (s > tau[row]) ? 1 : 0;
-        if (scores) scores[(size_t)row * L + (l - 1)] = s;
-    }
+    build_lists(n, exited, l, lists, hint_act, s_cnt);
+    if (threadIdx.x == 0) *ticket = 0;
 }
 
 // ---------------------------------------------------------------- projections on CUDA cores
@@ -619,8 +672,7 @@ struct HeadArgs {
     ProjIn in;
     int d, V;
     const int32_t *rows;  // rows that need logits
-    const StepMeta *meta; // n_head_rows
-    float *logits;        // [n_head_rows][V] or nullptr (indexed by position in `rows`)
+    const StepMeta *meta; // n_head_rows, logits [n_head_rows][V] or nullptr (indexed by position in `rows`)
     float *part_val;      // [max_batch][gridDim.x]
     int32_t *part_idx;
 };
@@ -632,7 +684,10 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a) {
     float *xs = smem + 32;
     __shared__ float s_val[16][N];
     __shared__ int s_idx[16][N];
+    pdl_launch();
+    pdl_wait();
     const int cnt = a.meta->n_head_rows;
+    float *logits = a.meta->logits;
     const int K = a.d, xstride = xs_stride(K, 8);
     int t0, t1;
     cta_range(a.V / R, t0, t1);
@@ -657,7 +712,7 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a) {
                 for (int r = 0; r < R; ++r) {
                     const float v = acc[r][n];
                     if (v > best[n]) { best[n] = v; besti[n] = (int)(o0 + r); }  // ascending ids: first max wins
-                    if (a.logits && lane == n * R + r && i0 + n < cnt) a.logits[(size_t)(i0 + n) * a.V + o0 + r] = v;
+                    if (logits && lane == n * R + r && i0 + n < cnt) logits[(size_t)(i0 + n) * a.V + o0 + r] = v;
                 }
         }
         if (lane == 0)
@@ -679,10 +734,12 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a) {
     }
 }
 
-__global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts,
-                                    int32_t *next_tok /* indexed by position in the head-row list */) {
+__global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts) {
+    pdl_launch();
+    pdl_wait();
     const int i = blockIdx.x;
     if (i >= meta->n_head_rows) return;
+    int32_t *next_tok = meta->next_tok;  // indexed by position in the head-row list
     float bv = -CUDART_INF_F;
     int bi = 0x7fffffff;
     for (int p = threadIdx.x; p < nparts; p += blockDim.x) {
