@@ -247,6 +247,11 @@ def ours(args, wl):
     shape_name, B, (plo, phi), seed = WORKLOADS[wl]
     seed = seed + 1000 * rank  # replicas draw their own prompts; the model is the same
     shape = synth.SHAPES[shape_name]
+    if args.layers:
+        import dataclasses
+        shape = dataclasses.replace(shape, L=args.layers)
+    if args.prompt:
+        plo = phi = args.prompt
     L = shape.L
     K, W = args.steps, args.warmup
     n_cal, n_prof, n_e2e = 8, 4, min(K, 64)
@@ -260,6 +265,10 @@ def ours(args, wl):
     cfg = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=n_pages, max_batch=max(B, 8),
                       page_shuffle_seed=seed + 1, flags=flags)
     rv = River(cfg, bb, rvw)
+    torch.cuda.synchronize()
+    # everything below runs on the context's stream (its own stream when graph replay is on)
+    stream_ctx = torch.cuda.stream(rv.stream)
+    stream_ctx.__enter__()
     slots = list(range(B))
     slots_c = (ctypes.c_int32 * B)(*slots)
 
@@ -366,7 +375,7 @@ def ours(args, wl):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl, "shape": shape_name, "batch": B, "prompt": [plo, phi], "context_at_start": pos0[:4],
                        "early_exit_target_fraction": EARLY_FRACTION, "thresholds": "per-step, from calibrated mean scores",
-                       "l2": "inputs (weights + KV) larger than L2, no flush", "flags": flags,
+                       "l2": "inputs (weights + KV) larger than L2, no flush", "flags": flags, "layers": L,
                        "parallelism": "replicas only" if world > 1 else "1 GPU", "prefill_s": round(t_pf, 3)},
             "layers_executed_fraction": float(ex.mean() / L), "early_exit_fraction": float((ex < L).mean()),
             "mean_exit_layer": float(ex.mean()),
@@ -403,6 +412,7 @@ def ours(args, wl):
         if "cpu_baseline" not in line:
             line["cpu_baseline"] = None
         print(json.dumps(line), flush=True)
+    stream_ctx.__exit__(None, None, None)
     rv.close()
 
 
@@ -415,6 +425,8 @@ def main():
     ap.add_argument("--workload", default="8b_b1", choices=sorted(WORKLOADS))
     ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")
+    ap.add_argument("--prompt", type=int, default=0, help="profiling aid: override the prompt length")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

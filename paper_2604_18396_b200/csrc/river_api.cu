@@ -152,7 +152,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     uint8_t *exd = cv.take<uint8_t>(B), *ps = cv.take<uint8_t>(B);
     int *de = cv.take<int>(1);
     unsigned *atk = cv.take<unsigned>(B * (size_t)c->Hkv), *tk4 = cv.take<unsigned>(4);
-    int32_t *hint = cv.take<int32_t>(1);
+    int32_t *hint = md ? md + 5 : nullptr;  // StepMeta::hint_act
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
         x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
@@ -241,7 +241,8 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     chunk = std::max(kAttnTile, (chunk + kAttnTile - 1) / kAttnTile * kAttnTile);
     mh[3] = chunk;
     mh[4] = S;
-    mh[5] = mh[6] = mh[7] = 0;
+    mh[5] = n;  // hint_act: every row starts in the backbone
+    mh[6] = mh[7] = 0;
     c->attn_splits_now = S;
 }
 
@@ -299,12 +300,16 @@ int ring_rw(int K, int group, int nrun) {
 template <class P, int N, int RB, int RW>
 cudaError_t launch_ring_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int has_river,
                           bool pdl) {
+    constexpr int RMAX = RB > RW ? RB : RW;
     RingGeom geom;
     geom.xstride = xs_stride(K, 32);
+    geom.ks = std::min(K, 8192 / RB);
+    // ring depth: as deep as leaves two kernels of the chain resident on one SM together (so that the next kernel's
+    // weight prefetch overlaps this kernel's tail), but at least four stages
     int S = 6;
-    while (S > 4 && ring_smem_bytes(S, N, K) > 110 * 1024) --S;  // two kernels of the chain fit one SM together
-    geom.n_stages = S;
-    const size_t smem = ring_smem_bytes(S, N, K);
+    while (S > 4 && ring_smem_bytes(S, N, K, RMAX) > 110 * 1024) --S;
+    geom.n_slots = S;
+    const size_t smem = ring_smem_bytes(S, N, K, RMAX);
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
         cudaFuncSetAttribute(ring_proj_kernel<P, N, RB, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -319,7 +324,7 @@ cudaError_t launch_ring(river_ctx *c, const P &p, const ProjIn &in, const RowLis
                         bool pdl) {
     const int rb = ring_rb(K), rw = ring_rw(K, c->cfg.group, P::NRUN);
     int n_sel = 1;
-    while (n_sel < n && n_sel < 4 && ring_smem_bytes(4, n_sel * 2, K) <= 210 * 1024) n_sel *= 2;
+    while (n_sel < n && n_sel < 4 && ring_smem_bytes(4, n_sel * 2, K, 8) <= 220 * 1024) n_sel *= 2;
 #define RING_CASE(N_, RB_, RW_) \
     if (n_sel == N_ && rb == RB_ && rw == RW_) return launch_ring_t<P, N_, RB_, RW_>(c, p, in, rl, K, has_river, pdl);
 #define RING_N(RB_, RW_) RING_CASE(1, RB_, RW_) RING_CASE(2, RB_, RW_) RING_CASE(4, RB_, RW_)
@@ -331,8 +336,9 @@ cudaError_t launch_ring(river_ctx *c, const P &p, const ProjIn &in, const RowLis
 
 bool ring_ok(const river_ctx *c, int K, int nrun) {
     if (c->cfg.flags & RIVER_F_NO_RING) return false;
+    if (K % 1024) return false;  // the 4-bit consumer wants K/32 chunks per row to fill whole warps
     const int rb = ring_rb(K), rw = ring_rw(K, c->cfg.group, nrun);
-    if (rw == 0) return false;
+    if (rw == 0 || rw * (K / 32) > 4 * kRingCThreads) return false;
     const bool combo = (rb == 2 && (rw == 8 || rw == 4 || rw == 2)) || (rb == 4 && (rw == 8 || rw == 4)) ||
                        (rb == 8 && rw == 8);
     return combo;
@@ -723,7 +729,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(c->hint_act, 0, sizeof(int32_t), c->stream);
+
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_act, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_riv, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
