@@ -47,8 +47,7 @@ enum { RIVER_EXIT_PER_TOKEN = 0, RIVER_EXIT_BATCH_MIN = 1 };
 enum {
     RIVER_F_GRAPH = 1,   /* replay each decode step as a CUDA graph (captured on first use) */
     RIVER_F_NO_TC = 2,   /* run every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
-    RIVER_F_SIMPLE_ATTN = 4, /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
-    RIVER_F_NO_RING = 8      /* debugging aid: projections on the plain register-streaming kernels, not the TMA ring */
+    RIVER_F_SIMPLE_ATTN = 4  /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
 };
 
 typedef struct river_config {

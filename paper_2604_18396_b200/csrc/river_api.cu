@@ -12,7 +12,7 @@
 #include "../../include/river.h"
 #include "river_kernels.cuh"
 #include "attn_decode.cuh"
-#include "gemv_ring.cuh"
+#include "gemv_stream.cuh"
 
 using namespace river;
 
@@ -24,7 +24,6 @@ constexpr int kStaging = 4;        // pinned metadata buffers in flight
 enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, kNumClasses };
 const char *const kClassNames[kNumClasses] = {"step_begin", "compact", "qkv_rope_kv", "attn_decode", "o_proj_resid",
                                               "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final"};
-constexpr size_t kSmemBudget = 200 * 1024;
 
 struct Carver {
     char *base;
@@ -163,34 +162,6 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     return (cv.off + 255) & ~(size_t)255;
 }
 
-// ---- shared-memory sizes and the number of activation rows a projection kernel takes per pass
-size_t proj_smem(int N, int K) {
-    const int xs = std::max(xs_stride(K, 8), xs_stride(K, 32));
-    return sizeof(float) * (32 + (size_t)N * (K >> 5) + (size_t)N * xs);
-}
-int pick_n(int rows, int K) {
-    int n = 1;
-    while (n < rows && n < 8 && proj_smem(n * 2, K) <= kSmemBudget) n *= 2;
-    return n;
-}
-
-template <class Kern>
-int launch_grid(river_ctx *c, Kern kern, int threads, size_t smem) {
-    int occ = 1;
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, smem);
-    occ = std::max(1, std::min(occ, 2048 / threads));
-    return c->num_sms * occ;
-}
-
-#define DISPATCH_N(n, ...)                                      \
-    switch (n) {                                                \
-        case 1: { constexpr int N = 1; __VA_ARGS__ } break;     \
-        case 2: { constexpr int N = 2; __VA_ARGS__ } break;     \
-        case 4: { constexpr int N = 4; __VA_ARGS__ } break;     \
-        default: { constexpr int N = 8; __VA_ARGS__ } break;    \
-    }
-
 // Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the
 // stream is still running and orders itself with griddepcontrol.wait.  Every kernel launched this way calls
 // griddepcontrol.wait before it touches anything a predecessor writes.
@@ -284,64 +255,69 @@ cudaError_t launch_attention(river_ctx *c, int n, int layer0, bool pdl) {
     return cudaErrorInvalidValue;
 }
 
-// ---- ring projection launch: rows per stage for the two weight formats, ring depth, shared memory
-int ring_rb(int K) { return K > 2048 ? 2 : (K > 1024 ? 4 : 8); }  // rows x min(K, 4096) x 2 B <= 16 KB
-int ring_rw(int K, int group, int nrun) {
-    for (int r = 8; r >= 2; r >>= 1) {
-        const size_t bytes = (size_t)r * ((K >> 1) + 4 * (K / group));
-        const int rr = r / nrun;
-        if (rr < 1) continue;
-        if (bytes <= (size_t)kRingStageBytes && (size_t)r * (K >> 1) <= 16384 && (rr * (K / group) * 2) % 16 == 0)
-            return r;
+// ---- streaming projection launch
+// Launch geometry: warps per CTA and CTAs per SM such that every warp gets the same number of tasks (a task is R
+// weight rows) and at least 16 warps per SM have loads in flight; searched once per (kernel, task count).
+struct StreamGeom { int threads, grid; };
+
+template <class Kern>
+StreamGeom pick_geometry(river_ctx *c, Kern kern, int tasks, size_t smem) {
+    StreamGeom best{256, c->num_sms};
+    double best_cost = 1e30;
+    int best_w = 0;
+    for (int w = 4; w <= 16; ++w) {
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, w * 32, smem) != cudaSuccess || occ < 1) continue;
+        occ = std::min(occ, 64 / w);
+        for (int o = 1; o <= occ; ++o) {
+            const int ctas = c->num_sms * o;
+            const int per_cta = (tasks + ctas - 1) / ctas;
+            const int rounds = (per_cta + w - 1) / w;
+            const int W = w * o;
+            const double cost = rounds * (W < 16 ? 16.0 / W : 1.0) * (1.0 + 0.002 * o);  // few large CTAs share x loads
+            if (cost < best_cost - 1e-9 || (std::fabs(cost - best_cost) < 1e-9 && W > best_w)) {
+                best_cost = cost; best_w = W; best = StreamGeom{w * 32, ctas};
+            }
+        }
     }
-    return 0;  // this shape cannot use the ring kernel for 4-bit weights
+    return best;
 }
 
-template <class P, int N, int RB, int RW>
-cudaError_t launch_ring_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int has_river,
-                          bool pdl) {
-    constexpr int RMAX = RB > RW ? RB : RW;
-    RingGeom geom;
-    geom.xstride = xs_stride(K, 32);
-    geom.ks = std::min(K, 8192 / RB);
-    // ring depth: as deep as leaves two kernels of the chain resident on one SM together (so that the next kernel's
-    // weight prefetch overlaps this kernel's tail), but at least four stages
-    int S = 6;
-    while (S > 4 && ring_smem_bytes(S, N, K, RMAX) > 110 * 1024) --S;
-    geom.n_slots = S;
-    const size_t smem = ring_smem_bytes(S, N, K, RMAX);
+template <class P, int N, int R>
+cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks,
+                            int has_river, bool pdl) {
+    const size_t smem = stream_smem_bytes(N, K);
+    // one kernel instantiation serves several projections (O and down): cache the geometry per (tasks, K)
+    struct Entry { int tasks, K; StreamGeom g; };
+    static std::vector<Entry> cache;
     static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaFuncSetAttribute(ring_proj_kernel<P, N, RB, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_smem = smem;
+    const StreamGeom *geom = nullptr;
+    for (auto &e : cache)
+        if (e.tasks == tasks && e.K == K) geom = &e.g;
+    if (!geom) {
+        if (smem > attr_smem) attr_smem = smem;
+        cudaFuncSetAttribute(stream_proj_kernel<P, N, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attr_smem);
+        cache.push_back({tasks, K, pick_geometry(c, stream_proj_kernel<P, N, R>, tasks, smem)});
+        geom = &cache.back().g;
     }
-    return launch_k(ring_proj_kernel<P, N, RB, RW>, dim3(c->num_sms), dim3(kRingThreads), smem, c->stream, pdl, p, in, rl,
-                    geom, has_river, c->dev_err);
+    return launch_k(stream_proj_kernel<P, N, R>, dim3(geom->grid), dim3(geom->threads), smem, c->stream, pdl, p, in, rl,
+                    has_river, xs_stride(K, 32));
 }
+
+int stream_rows_per_task(int K) { return K >= 4096 ? 2 : 4; }
 
 template <class P>
-cudaError_t launch_ring(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int n, int has_river,
-                        bool pdl) {
-    const int rb = ring_rb(K), rw = ring_rw(K, c->cfg.group, P::NRUN);
+cudaError_t launch_stream(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks_r2, int n,
+                          int has_river, bool pdl) {
     int n_sel = 1;
-    while (n_sel < n && n_sel < 4 && ring_smem_bytes(4, n_sel * 2, K, 8) <= 220 * 1024) n_sel *= 2;
-#define RING_CASE(N_, RB_, RW_) \
-    if (n_sel == N_ && rb == RB_ && rw == RW_) return launch_ring_t<P, N_, RB_, RW_>(c, p, in, rl, K, has_river, pdl);
-#define RING_N(RB_, RW_) RING_CASE(1, RB_, RW_) RING_CASE(2, RB_, RW_) RING_CASE(4, RB_, RW_)
-    RING_N(2, 8) RING_N(2, 4) RING_N(2, 2) RING_N(4, 8) RING_N(4, 4) RING_N(8, 8)
-#undef RING_N
-#undef RING_CASE
+    while (n_sel < n && n_sel < 4 && stream_smem_bytes(n_sel * 2, K) <= 200 * 1024) n_sel *= 2;
+    const int r = stream_rows_per_task(K);
+    const int tasks = tasks_r2 * 2 / r;
+#define STREAM_CASE(N_, R_) if (n_sel == N_ && r == R_) return launch_stream_t<P, N_, R_>(c, p, in, rl, K, tasks, has_river, pdl);
+    STREAM_CASE(1, 2) STREAM_CASE(2, 2) STREAM_CASE(4, 2)
+    STREAM_CASE(1, 4) STREAM_CASE(2, 4) STREAM_CASE(4, 4)
+#undef STREAM_CASE
     return cudaErrorInvalidValue;
-}
-
-bool ring_ok(const river_ctx *c, int K, int nrun) {
-    if (c->cfg.flags & RIVER_F_NO_RING) return false;
-    if (K % 1024) return false;  // the 4-bit consumer wants K/32 chunks per row to fill whole warps
-    const int rb = ring_rb(K), rw = ring_rw(K, c->cfg.group, nrun);
-    if (rw == 0 || rw * (K / 32) > 4 * kRingCThreads) return false;
-    const bool combo = (rb == 2 && (rw == 8 || rw == 4 || rw == 2)) || (rb == 4 && (rw == 8 || rw == 4)) ||
-                       (rb == 8 && rw == 8);
-    return combo;
 }
 
 // 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
@@ -471,29 +447,13 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         {
             const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
             LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
-            const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
-            if (ring_ok(c, d, 2)) {
-                QkvProblem p{};
-                p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
-                p.rq = w4(w.rq); p.rk = w4(w.rk); p.rv = w4(w.rv);
-                p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
-                p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
-                note(launch_ring(c, p, in, rl, d, n, has_river, true));
-            } else {
-                QkvArgs a{};
-                a.wq = (const uint16_t *)w.wq; a.wk = (const uint16_t *)w.wk; a.wv = (const uint16_t *)w.wv;
-                a.rq = w4(w.rq); a.rk = w4(w.rk); a.rv = w4(w.rv);
-                a.has_river = has_river; a.in = in;
-                a.d = d; a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh; a.group = g.group;
-                a.rope_cs = c->rope_cs; a.q_out = c->qbuf; a.kv = kv_addr(c, l - 1);
-                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr; a.dev_err = c->dev_err;
-                const int n_sel = pick_n(n, d);
-                const size_t smem = proj_smem(n_sel, d);
-                DISPATCH_N(n_sel, {
-                    const int grid = launch_grid(c, qkv_rope_kv_kernel<N>, 256, smem);
-                    qkv_rope_kv_kernel<N><<<grid, 256, smem, c->stream>>>(a);
-                });
-            }
+            QkvProblem p{};
+            p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
+            p.rq = w4(w.rq); p.rk = w4(w.rk); p.rv = w4(w.rv);
+            p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
+            p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
+            note(launch_stream(c, p, ProjIn{h_in, (const uint16_t *)w.attn_norm, g.rms_eps}, rl, d,
+                               (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true));
         }
         // ---- a3: paged GQA decode attention
         {
@@ -504,77 +464,35 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         {
             const double wb = 2.0 * qdim * d;
             LaunchScope ls(c, K_OPROJ, wb, wb * w4f, l - 1);
-            const ProjIn in{c->obuf, nullptr, 0.f};
-            if (ring_ok(c, qdim, 1)) {
-                ResidProblem p{};
-                p.w = (const uint16_t *)w.wo; p.rw = w4(w.ro); p.K = qdim; p.out_dim = d; p.group = g.group;
-                p.resid = h_in; p.out = h_mid;
-                note(launch_ring(c, p, in, rl, qdim, n, has_river, !(g.flags & RIVER_F_SIMPLE_ATTN)));
-            } else {
-                ResidArgs a{};
-                a.w = (const uint16_t *)w.wo; a.rw = w4(w.ro); a.has_river = has_river; a.in = in;
-                a.K = qdim; a.out_dim = d; a.group = g.group; a.resid = h_in; a.out = h_mid;
-                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-                const int n_sel = pick_n(n, qdim);
-                const size_t smem = proj_smem(n_sel, qdim);
-                DISPATCH_N(n_sel, {
-                    const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
-                    proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
-                });
-            }
+            ResidProblem p{};
+            p.w = (const uint16_t *)w.wo; p.rw = w4(w.ro); p.K = qdim; p.out_dim = d; p.group = g.group;
+            p.resid = h_in; p.out = h_mid;
+            note(launch_stream(c, p, ProjIn{c->obuf, nullptr, 0.f}, rl, qdim, d / 2, n, has_river,
+                               !(g.flags & RIVER_F_SIMPLE_ATTN)));
         }
         // ---- a5: FFN norm + gate/up + SwiGLU
         {
             const double wb = 2.0 * 2.0 * g.F * d;
             LaunchScope ls(c, K_GATEUP, wb, wb * w4f, l - 1);
-            const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
-            if (ring_ok(c, d, 2)) {
-                GateUpProblem p{};
-                p.wg = (const uint16_t *)w.wg; p.wu = (const uint16_t *)w.wu; p.rg = w4(w.rg); p.ru = w4(w.ru);
-                p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
-                note(launch_ring(c, p, in, rl, d, n, has_river, ring_ok(c, qdim, 1)));
-            } else {
-                GateUpArgs a{};
-                a.wg = (const uint16_t *)w.wg; a.wu = (const uint16_t *)w.wu; a.rg = w4(w.rg); a.ru = w4(w.ru);
-                a.has_river = has_river; a.in = in;
-                a.d = d; a.F = g.F; a.group = g.group; a.act = c->act;
-                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-                const int n_sel = pick_n(n, d);
-                const size_t smem = proj_smem(n_sel, d);
-                DISPATCH_N(n_sel, {
-                    const int grid = launch_grid(c, gateup_kernel<N>, 256, smem);
-                    gateup_kernel<N><<<grid, 256, smem, c->stream>>>(a);
-                });
-            }
+            GateUpProblem p{};
+            p.wg = (const uint16_t *)w.wg; p.wu = (const uint16_t *)w.wu; p.rg = w4(w.rg); p.ru = w4(w.ru);
+            p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
+            note(launch_stream(c, p, ProjIn{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps}, rl, d, g.F, n, has_river,
+                               true));
         }
         // ---- a5: down projection + residual
-        bool down_ring = ring_ok(c, g.F, 1);
         {
             const double wb = 2.0 * g.F * d;
             LaunchScope ls(c, K_DOWN, wb, wb * w4f, l - 1);
-            const ProjIn in{c->act, nullptr, 0.f};
-            if (down_ring) {
-                ResidProblem p{};
-                p.w = (const uint16_t *)w.wd; p.rw = w4(w.rd); p.K = g.F; p.out_dim = d; p.group = g.group;
-                p.resid = h_mid; p.out = h_out;
-                note(launch_ring(c, p, in, rl, g.F, n, has_river, ring_ok(c, d, 2)));
-            } else {
-                ResidArgs a{};
-                a.w = (const uint16_t *)w.wd; a.rw = w4(w.rd); a.has_river = has_river; a.in = in;
-                a.K = g.F; a.out_dim = d; a.group = g.group; a.resid = h_mid; a.out = h_out;
-                a.act_idx = ai; a.n_act = na; a.riv_idx = ri; a.n_riv = nr;
-                const int n_sel = pick_n(n, g.F);
-                const size_t smem = proj_smem(n_sel, g.F);
-                DISPATCH_N(n_sel, {
-                    const int grid = launch_grid(c, proj_resid_kernel<N, 2>, 256, smem);
-                    proj_resid_kernel<N, 2><<<grid, 256, smem, c->stream>>>(a);
-                });
-            }
+            ResidProblem p{};
+            p.w = (const uint16_t *)w.wd; p.rw = w4(w.rd); p.K = g.F; p.out_dim = d; p.group = g.group;
+            p.resid = h_mid; p.out = h_out;
+            note(launch_stream(c, p, ProjIn{c->act, nullptr, 0.f}, rl, g.F, d / 2, n, has_river, true));
         }
         // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
         {
             LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
-            note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, down_ring, c->meta(), l, L,
+            note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, true, c->meta(), l, L,
                           g.entry_layer, g.exit_mode, (const float *)h_in, (const float *)h_out, d, c->pass, c->exited,
                           lists, c->hint_act, c->tickets + 1));
         }
@@ -586,17 +504,19 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         a.in = ProjIn{c->h[hi], c->final_norm, g.rms_eps};
         a.d = d; a.V = g.V; a.rows = c->head_rows(); a.meta = c->meta();
         a.part_val = c->part_val; a.part_idx = c->part_idx;
-        const int n_sel = std::min(pick_n(n_head, d), 4);
-        const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xs_stride(d, 8));
+        int n_sel = 1;
+        while (n_sel < n_head && n_sel < 4) n_sel *= 2;
+        const int xstride = xs_stride(d, 8);
+        const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xstride);
         {
             LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + 4.0 * n_head * g.V, 0, -1);
             switch (n_sel) {
                 case 1: cudaFuncSetAttribute(lm_head_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        note(launch_k(lm_head_kernel<1, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a)); break;
+                        note(launch_k(lm_head_kernel<1, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride)); break;
                 case 2: cudaFuncSetAttribute(lm_head_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        note(launch_k(lm_head_kernel<2, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a)); break;
+                        note(launch_k(lm_head_kernel<2, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride)); break;
                 default: cudaFuncSetAttribute(lm_head_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        note(launch_k(lm_head_kernel<4, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a)); break;
+                        note(launch_k(lm_head_kernel<4, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride)); break;
             }
         }
         {

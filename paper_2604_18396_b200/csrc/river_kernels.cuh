@@ -267,119 +267,7 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     if (threadIdx.x == 0) *ticket = 0;
 }
 
-// ---------------------------------------------------------------- projections on CUDA cores
-// A warp computes R output features for up to N activation rows at once: the weight rows stream from HBM with
-// 128-bit loads, the N activation rows sit in shared memory (fp32, lane-interleaved).
-
-// bf16 weights: 8 weights per 16-byte chunk.
-template <int N, int R>
-__device__ __forceinline__ void warp_dots_bf16(const uint16_t *const (&wrow)[R], const float *xs, int K, int xstride,
-                                               float (&acc)[R][N]) {
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
-    const int nchunks = K >> 3;
-#pragma unroll 2
-    for (int c0 = 0; c0 < nchunks; c0 += 32) {
-        const int c = c0 + lane;
-        if (c < nchunks) {
-            uint4 w[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) w[r] = ldg_stream16(wrow[r] + (size_t)c * 8);
-            const float *xb = xs + (c0 >> 5) * 256 + lane * 4;
-#pragma unroll
-            for (int n = 0; n < N; ++n) {
-                const float4 x0 = *reinterpret_cast<const float4 *>(xb + n * xstride);
-                const float4 x1 = *reinterpret_cast<const float4 *>(xb + n * xstride + 128);
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float a = acc[r][n];
-                    a = fmaf(bf16lo(w[r].x), x0.x, a);
-                    a = fmaf(bf16hi(w[r].x), x0.y, a);
-                    a = fmaf(bf16lo(w[r].y), x0.z, a);
-                    a = fmaf(bf16hi(w[r].y), x0.w, a);
-                    a = fmaf(bf16lo(w[r].z), x1.x, a);
-                    a = fmaf(bf16hi(w[r].z), x1.y, a);
-                    a = fmaf(bf16lo(w[r].w), x1.z, a);
-                    a = fmaf(bf16hi(w[r].w), x1.w, a);
-                    acc[r][n] = a;
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int n = 0; n < N; ++n) acc[r][n] = warp_sum(acc[r][n]);
-}
-
-// 4-bit weights: 32 weights per 16-byte chunk of codes, one (scale, zero) per `group` inputs.
-// sum_k (q_k - z) s x_k over a chunk = s * ( sum_k (128 + q_k) x_k  -  (z + 128) * sum_k x_k ):
-// 128 + q is what OR-ing a nibble into the bf16 pattern 0x4300 gives, and the chunk sums of x are precomputed.
-template <int N, int R>
-__device__ __forceinline__ void warp_dots_w4(const W4 (&wrow)[R], const float *xs, const float *xsum, int K,
-                                             int xstride, int xsum_stride, int group, float (&acc)[R][N]) {
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
-    const int nchunks = K >> 5;
-    const int gshift = (group == 64) ? 1 : (group == 32 ? 0 : 2);  // chunks per group = group / 32
-    for (int c0 = 0; c0 < nchunks; c0 += 32) {
-        const int c = c0 + lane;
-        if (c < nchunks) {
-            uint4 q[R];
-            float s[R], zz[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                q[r] = ldg_stream16(wrow[r].codes + (size_t)c * 16);
-                s[r] = bf16f(ldg_u16(wrow[r].scale + (c >> gshift)));
-                zz[r] = bf16f(ldg_u16(wrow[r].zero + (c >> gshift))) + 128.f;
-            }
-            const float *xb = xs + (c0 >> 5) * 1024 + lane * 4;
-#pragma unroll
-            for (int n = 0; n < N; ++n) {
-                float part[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) part[r] = 0.f;
-#pragma unroll
-                for (int wd = 0; wd < 4; ++wd) {  // code word wd holds inputs 8*wd .. 8*wd+7 of the chunk
-                    const float4 x0 = *reinterpret_cast<const float4 *>(xb + n * xstride + (2 * wd) * 128);
-                    const float4 x1 = *reinterpret_cast<const float4 *>(xb + n * xstride + (2 * wd + 1) * 128);
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const uint32_t v = wd == 0 ? q[r].x : (wd == 1 ? q[r].y : (wd == 2 ? q[r].z : q[r].w));
-                        const uint32_t p0 = (v & 0x000f000fu) | 0x43004300u;         // inputs 0, 4
-                        const uint32_t p1 = ((v >> 4) & 0x000f000fu) | 0x43004300u;  // inputs 1, 5
-                        const uint32_t p2 = ((v >> 8) & 0x000f000fu) | 0x43004300u;  // inputs 2, 6
-                        const uint32_t p3 = ((v >> 12) & 0x000f000fu) | 0x43004300u; // inputs 3, 7
-                        float a = part[r];
-                        a = fmaf(bf16lo(p0), x0.x, a);
-                        a = fmaf(bf16lo(p1), x0.y, a);
-                        a = fmaf(bf16lo(p2), x0.z, a);
-                        a = fmaf(bf16lo(p3), x0.w, a);
-                        a = fmaf(bf16hi(p0), x1.x, a);
-                        a = fmaf(bf16hi(p1), x1.y, a);
-                        a = fmaf(bf16hi(p2), x1.z, a);
-                        a = fmaf(bf16hi(p3), x1.w, a);
-                        part[r] = a;
-                    }
-                }
-                const float sx = xsum[n * xsum_stride + c];
-#pragma unroll
-                for (int r = 0; r < R; ++r) acc[r][n] = fmaf(s[r], part[r] - zz[r] * sx, acc[r][n]);
-            }
-        }
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int n = 0; n < N; ++n) acc[r][n] = warp_sum(acc[r][n]);
-}
-
+// ---------------------------------------------------------------- shared by the projection kernels
 // What feeds a projection: either rows of an fp32 buffer as they are, or their RMSNorm (x = h * rsqrt(mean h^2 +
 // eps) * gain), computed by every CTA for itself.
 struct ProjIn {
@@ -387,65 +275,6 @@ struct ProjIn {
     const uint16_t *gain;  // bf16 [K] or nullptr = no normalisation
     float eps;
 };
-
-// Fill shared memory with up to N activation rows idx[i0 .. i0+N) (E = inputs per chunk: 8 bf16 / 32 w4) and, for
-// the 4-bit path, the per-chunk sums.  Rows beyond cnt are zero.
-template <int N, int E>
-__device__ __forceinline__ void load_rows(const ProjIn &in, const int32_t *idx, int i0, int cnt, int K, int xstride,
-                                          float *xs, float *xsum, int xsum_stride, float *red /* [32] */) {
-    const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int n = 0; n < N; ++n) {
-        float *dst = xs + n * xstride;
-        if (i0 + n >= cnt) {
-            for (int k = tid; k < xstride; k += nthr) dst[k] = 0.f;
-            continue;
-        }
-        const float *src = in.src + (size_t)idx[i0 + n] * K;
-        float scale = 1.f;
-        if (in.gain) {
-            float ss = 0.f;
-            for (int k = tid; k < K; k += nthr) { const float v = src[k]; ss = fmaf(v, v, ss); }
-            ss = warp_sum(ss);
-            __syncthreads();
-            if ((tid & 31) == 0) red[tid >> 5] = ss;
-            __syncthreads();
-            ss = 0.f;
-            for (int w = 0; w < (nthr >> 5); ++w) ss += red[w];
-            scale = rsqrtf(ss / (float)K + in.eps);
-        }
-        for (int k = tid; k < xstride; k += nthr) {
-            float v = 0.f;
-            if (k < K) {
-                v = src[k] * scale;
-                if (in.gain) v *= bf16f(in.gain[k]);
-            }
-            if (k < K) dst[xs_index<E>(k)] = v;
-        }
-        // padding beyond K inside the last 32-chunk block is never read (lanes with c >= nchunks are idle)
-    }
-    __syncthreads();
-    if (E == 32) {
-        const int nchunks = K >> 5;
-        for (int t = tid; t < N * nchunks; t += nthr) {
-            const int n = t / nchunks, c = t % nchunks;
-            const float *xb = xs + n * xstride + (c >> 5) * 1024 + (c & 31) * 4;
-            float sx = 0.f;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float4 v = *reinterpret_cast<const float4 *>(xb + j * 128);
-                sx += (v.x + v.y) + (v.z + v.w);
-            }
-            xsum[n * xsum_stride + c] = sx;
-        }
-        __syncthreads();
-    }
-}
-
-// Contiguous share of `total` tasks for CTA `cta` of `ncta`.
-__device__ __forceinline__ void cta_range(int total, int &t0, int &t1) {
-    t0 = (int)(((long long)total * blockIdx.x) / gridDim.x);
-    t1 = (int)(((long long)total * (blockIdx.x + 1)) / gridDim.x);
-}
 
 struct KvAddr {
     __nv_bfloat16 *pool;  // [L][n_pages][2][Hkv][16][dh]
@@ -458,314 +287,8 @@ struct KvAddr {
     }
 };
 
-// ---- a2: attention-norm + QKV projection + RoPE + paged KV write (both weight sets in one launch)
-// Task = (head hh of the concatenated [q heads | k heads | v heads], pair i): output features hh*dh + i and
-// hh*dh + i + dh/2, the two halves a rotary pair needs.
-struct QkvArgs {
-    const uint16_t *wq, *wk, *wv, *attn_norm;
-    W4 rq, rk, rv;
-    int has_river;
-    ProjIn in;
-    int d, Hq, Hkv, dh, group;
-    const float2 *rope_cs;  // [rows][dh/2]
-    float *q_out;           // [rows][Hq*dh]
-    KvAddr kv;
-    const int32_t *act_idx, *n_act, *riv_idx, *n_riv;
-    int *dev_err;
-};
-
-template <int N, bool RIVER>
-__device__ __forceinline__ void qkv_pass(const QkvArgs &a, const int32_t *idx, int cnt, float *xs, float *xsum,
-                                         float *red) {
-    constexpr int E = RIVER ? 32 : 8;
-    const int K = a.d, xstride = xs_stride(K, E), xsum_stride = K >> 5;
-    const int half = a.dh >> 1;
-    const int tasks = (a.Hq + 2 * a.Hkv) * half;
-    int t0, t1;
-    cta_range(tasks, t0, t1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int i0 = 0; i0 < cnt; i0 += N) {
-        __syncthreads();
-        load_rows<N, E>(a.in, idx, i0, cnt, K, xstride, xs, xsum, xsum_stride, red);
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            const int hh = t / half, i = t % half;
-            int which, hl;  // 0 q, 1 k, 2 v; head index inside its matrix
-            if (hh < a.Hq) { which = 0; hl = hh; }
-            else if (hh < a.Hq + a.Hkv) { which = 1; hl = hh - a.Hq; }
-            else { which = 2; hl = hh - a.Hq - a.Hkv; }
-            const size_t r0 = (size_t)hl * a.dh + i, r1 = r0 + half;
-            float acc[2][N];
-            if (!RIVER) {
-                const uint16_t *w = which == 0 ? a.wq : (which == 1 ? a.wk : a.wv);
-                const uint16_t *const rows[2] = {w + r0 * K, w + r1 * K};
-                warp_dots_bf16<N, 2>(rows, xs, K, xstride, acc);
-            } else {
-                const W4 &w = which == 0 ? a.rq : (which == 1 ? a.rk : a.rv);
-                const int ng = K / a.group;
-                const W4 rows[2] = {{w.codes + r0 * (K >> 1), w.scale + r0 * ng, w.zero + r0 * ng},
-                                    {w.codes + r1 * (K >> 1), w.scale + r1 * ng, w.zero + r1 * ng}};
-                warp_dots_w4<N, 2>(rows, xs, xsum, K, xstride, xsum_stride, a.group, acc);
-            }
-#pragma unroll
-            for (int n = 0; n < N; ++n) {
-                if (lane == n && i0 + n < cnt) {
-                    const int row = idx[i0 + n];
-                    float lo = acc[0][n], hi = acc[1][n];
-                    if (which != 2) {
-                        const float2 cs = a.rope_cs[(size_t)row * half + i];
-                        const float rl = lo * cs.x - hi * cs.y;
-                        const float rh = hi * cs.x + lo * cs.y;
-                        lo = rl; hi = rh;
-                    }
-                    if (which == 0) {
-                        a.q_out[(size_t)row * (a.Hq * a.dh) + r0] = lo;
-                        a.q_out[(size_t)row * (a.Hq * a.dh) + r1] = hi;
-                    } else {
-                        const int pos = a.kv.row_pos[row], slot = a.kv.row_slot[row];
-                        const int page = a.kv.page_tbl[(size_t)slot * a.kv.max_pages_per_seq + pos / kPage];
-                        if (page < 0 || page >= a.kv.n_pages) {
-                            atomicExch(a.dev_err, DEV_BAD_PAGE);
-                        } else {
-                            const size_t o = a.kv.base(page, which - 1, hl, pos % kPage);
-                            a.kv.pool[o + i] = __float2bfloat16_rn(lo);
-                            a.kv.pool[o + i + half] = __float2bfloat16_rn(hi);
-                        }
-                    }
-                }
-            }
-        }
-    }
-}
-
-template <int N>
-__global__ void __launch_bounds__(256) qkv_rope_kv_kernel(const QkvArgs a) {
-    extern __shared__ __align__(16) float smem[];
-    float *red = smem;             // 32
-    float *xsum = smem + 32;       // N * (K/32)
-    float *xs = xsum + N * (a.d >> 5);
-    const int na = *a.n_act, nr = *a.n_riv;
-    if (na > 0) qkv_pass<N, false>(a, a.act_idx, na, xs, xsum, red);
-    if (nr > 0 && a.has_river) qkv_pass<N, true>(a, a.riv_idx, nr, xs, xsum, red);
-}
-
-// ---- a4 / a5b: plain projection with residual: out[row][o] = resid[row][o] + sum_k W[o][k] x[row][k]
-struct ResidArgs {
-    const uint16_t *w;
-    W4 rw;
-    int has_river;
-    ProjIn in;
-    int K, out_dim, group;
-    const float *resid;  // [rows][out_dim]
-    float *out;          // [rows][out_dim]
-    const int32_t *act_idx, *n_act, *riv_idx, *n_riv;
-};
-
-template <int N, int R, bool RIVER>
-__device__ __forceinline__ void resid_pass(const ResidArgs &a, const int32_t *idx, int cnt, float *xs, float *xsum,
-                                           float *red) {
-    constexpr int E = RIVER ? 32 : 8;
-    const int K = a.K, xstride = xs_stride(K, E), xsum_stride = K >> 5;
-    const int tasks = a.out_dim / R;
-    int t0, t1;
-    cta_range(tasks, t0, t1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int i0 = 0; i0 < cnt; i0 += N) {
-        __syncthreads();
-        load_rows<N, E>(a.in, idx, i0, cnt, K, xstride, xs, xsum, xsum_stride, red);
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            const size_t o0 = (size_t)t * R;
-            float acc[R][N];
-            if (!RIVER) {
-                const uint16_t *rows[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) rows[r] = a.w + (o0 + r) * K;
-                warp_dots_bf16<N, R>(rows, xs, K, xstride, acc);
-            } else {
-                const int ng = K / a.group;
-                W4 rows[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-                    rows[r] = W4{a.rw.codes + (o0 + r) * (K >> 1), a.rw.scale + (o0 + r) * ng,
-                                 a.rw.zero + (o0 + r) * ng};
-                warp_dots_w4<N, R>(rows, xs, xsum, K, xstride, xsum_stride, a.group, acc);
-            }
-#pragma unroll
-            for (int n = 0; n < N; ++n)
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-                    if (lane == n * R + r && i0 + n < cnt) {
-                        const size_t o = (size_t)idx[i0 + n] * a.out_dim + o0 + r;
-                        a.out[o] = a.resid[o] + acc[r][n];
-                    }
-        }
-    }
-}
-
-template <int N, int R>
-__global__ void __launch_bounds__(256) proj_resid_kernel(const ResidArgs a) {
-    extern __shared__ __align__(16) float smem[];
-    float *red = smem;
-    float *xsum = smem + 32;
-    float *xs = xsum + N * (a.K >> 5);
-    const int na = *a.n_act, nr = *a.n_riv;
-    if (na > 0) resid_pass<N, R, false>(a, a.act_idx, na, xs, xsum, red);
-    if (nr > 0 && a.has_river) resid_pass<N, R, true>(a, a.riv_idx, nr, xs, xsum, red);
-}
-
-// ---- a5a: FFN-norm + gate/up projection + SwiGLU: act[row][f] = silu(Wg y) * (Wu y)
-struct GateUpArgs {
-    const uint16_t *wg, *wu;
-    W4 rg, ru;
-    int has_river;
-    ProjIn in;
-    int d, F, group;
-    float *act;  // [rows][F]
-    const int32_t *act_idx, *n_act, *riv_idx, *n_riv;
-};
-
-template <int N, bool RIVER>
-__device__ __forceinline__ void gateup_pass(const GateUpArgs &a, const int32_t *idx, int cnt, float *xs, float *xsum,
-                                            float *red) {
-    constexpr int E = RIVER ? 32 : 8;
-    const int K = a.d, xstride = xs_stride(K, E), xsum_stride = K >> 5;
-    int t0, t1;
-    cta_range(a.F, t0, t1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int i0 = 0; i0 < cnt; i0 += N) {
-        __syncthreads();
-        load_rows<N, E>(a.in, idx, i0, cnt, K, xstride, xs, xsum, xsum_stride, red);
-        for (int f = t0 + warp; f < t1; f += nwarps) {
-            float acc[2][N];
-            if (!RIVER) {
-                const uint16_t *const rows[2] = {a.wg + (size_t)f * K, a.wu + (size_t)f * K};
-                warp_dots_bf16<N, 2>(rows, xs, K, xstride, acc);
-            } else {
-                const int ng = K / a.group;
-                const W4 rows[2] = {
-                    {a.rg.codes + (size_t)f * (K >> 1), a.rg.scale + (size_t)f * ng, a.rg.zero + (size_t)f * ng},
-                    {a.ru.codes + (size_t)f * (K >> 1), a.ru.scale + (size_t)f * ng, a.ru.zero + (size_t)f * ng}};
-                warp_dots_w4<N, 2>(rows, xs, xsum, K, xstride, xsum_stride, a.group, acc);
-            }
-#pragma unroll
-            for (int n = 0; n < N; ++n)
-                if (lane == n && i0 + n < cnt) {
-                    const float g = acc[0][n], u = acc[1][n];
-                    a.act[(size_t)idx[i0 + n] * a.F + f] = g / (1.f + __expf(-g)) * u;
-                }
-        }
-    }
-}
-
-template <int N>
-__global__ void __launch_bounds__(256) gateup_kernel(const GateUpArgs a) {
-    extern __shared__ __align__(16) float smem[];
-    float *red = smem;
-    float *xsum = smem + 32;
-    float *xs = xsum + N * (a.d >> 5);
-    const int na = *a.n_act, nr = *a.n_riv;
-    if (na > 0) gateup_pass<N, false>(a, a.act_idx, na, xs, xsum, red);
-    if (nr > 0 && a.has_river) gateup_pass<N, true>(a, a.riv_idx, nr, xs, xsum, red);
-}
-
-// ---- a8: final norm + LM head (+ per-CTA argmax partials; ties -> lowest id)
-struct HeadArgs {
-    const uint16_t *w;  // [V][d]
-    ProjIn in;
-    int d, V;
-    const int32_t *rows;  // rows that need logits
-    const StepMeta *meta; // n_head_rows, logits [n_head_rows][V] or nullptr (indexed by position in `rows`)
-    float *part_val;      // [max_batch][gridDim.x]
-    int32_t *part_idx;
-};
-
-template <int N, int R>
-__global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a) {
-    extern __shared__ __align__(16) float smem[];
-    float *red = smem;
-    float *xs = smem + 32;
-    __shared__ float s_val[16][N];
-    __shared__ int s_idx[16][N];
-    pdl_launch();
-    pdl_wait();
-    const int cnt = a.meta->n_head_rows;
-    float *logits = a.meta->logits;
-    const int K = a.d, xstride = xs_stride(K, 8);
-    int t0, t1;
-    cta_range(a.V / R, t0, t1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int i0 = 0; i0 < cnt; i0 += N) {
-        __syncthreads();
-        load_rows<N, 8>(a.in, a.rows, i0, cnt, K, xstride, xs, nullptr, 0, red);
-        float best[N];
-        int besti[N];
-#pragma unroll
-        for (int n = 0; n < N; ++n) { best[n] = -CUDART_INF_F; besti[n] = 0x7fffffff; }
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            const size_t o0 = (size_t)t * R;
-            const uint16_t *rows[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) rows[r] = a.w + (o0 + r) * K;
-            float acc[R][N];
-            warp_dots_bf16<N, R>(rows, xs, K, xstride, acc);
-#pragma unroll
-            for (int n = 0; n < N; ++n)
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float v = acc[r][n];
-                    if (v > best[n]) { best[n] = v; besti[n] = (int)(o0 + r); }  // ascending ids: first max wins
-                    if (logits && lane == n * R + r && i0 + n < cnt) logits[(size_t)(i0 + n) * a.V + o0 + r] = v;
-                }
-        }
-        if (lane == 0)
-#pragma unroll
-            for (int n = 0; n < N; ++n) { s_val[warp][n] = best[n]; s_idx[warp][n] = besti[n]; }
-        __syncthreads();
-        if (threadIdx.x < N && i0 + (int)threadIdx.x < cnt) {
-            const int n = threadIdx.x;
-            float bv = -CUDART_INF_F;
-            int bi = 0x7fffffff;
-            for (int w = 0; w < nwarps; ++w) {
-                const float v = s_val[w][n];
-                const int id = s_idx[w][n];
-                if (v > bv || (v == bv && id < bi)) { bv = v; bi = id; }
-            }
-            a.part_val[(size_t)(i0 + n) * gridDim.x + blockIdx.x] = bv;
-            a.part_idx[(size_t)(i0 + n) * gridDim.x + blockIdx.x] = bi;
-        }
-    }
-}
-
-__global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts) {
-    pdl_launch();
-    pdl_wait();
-    const int i = blockIdx.x;
-    if (i >= meta->n_head_rows) return;
-    int32_t *next_tok = meta->next_tok;  // indexed by position in the head-row list
-    float bv = -CUDART_INF_F;
-    int bi = 0x7fffffff;
-    for (int p = threadIdx.x; p < nparts; p += blockDim.x) {
-        const float v = part_val[(size_t)i * nparts + p];
-        const int id = part_idx[(size_t)i * nparts + p];
-        if (v > bv || (v == bv && id < bi)) { bv = v; bi = id; }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-    }
-    __shared__ float sv[32];
-    __shared__ int si[32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) { sv[warp] = bv; si[warp] = bi; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
-            if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
-        next_tok[i] = bi;
-    }
-}
-
-// ---------------------------------------------------------------- a3: paged GQA decode attention (first version)
+// ---------------------------------------------------------------- a3: paged GQA decode attention, plain version
+// (a debugging aid selected by RIVER_F_SIMPLE_ATTN; the production kernel is in attn_decode.cuh)
 // One CTA per (row, kv head): its GQ query heads share every K/V load.  A warp walks positions warp, warp+W, ...;
 // a lane owns DH/32 head dims; softmax is online in fp32; the warps' partial states merge through shared memory.
 template <int DH, int GQ>
@@ -850,12 +373,6 @@ __global__ void kv_copy_kernel(KvAddr kv, int slot, int pos0, int n, __nv_bfloat
             v_io[(size_t)i * w + t] = kv.pool[ov];
         }
     }
-}
-
-__global__ void apply_page_updates_kernel(const int32_t *upd, int n, int max_batch, int32_t *page_tbl,
-                                          int max_pages_per_seq) {
-    for (int i = threadIdx.x + blockIdx.x * blockDim.x; i < n; i += blockDim.x * gridDim.x)
-        page_tbl[(size_t)upd[i] * max_pages_per_seq + upd[max_batch + i]] = upd[2 * max_batch + i];
 }
 
 }  // namespace river
