@@ -159,6 +159,23 @@ typedef struct river_kernel_time {
 int river_profile(river_ctx *ctx, int enable);
 int river_profile_read(river_ctx *ctx, river_kernel_time *out, int cap, int *n_out);
 
+/* Greedy token selection over logits the caller already holds, without allocating anything.
+ * (The paper has no counterpart: this is a utility for callers of the library.)
+ * For callers that cannot allocate at the point of the call and have no context workspace to lend: a sampling hook
+ * inside a serving loop whose device memory was all handed out at start-up, or a latency-critical loop where an
+ * allocation would serialise the device.  The scratch (per-CTA partial maxima, per-row arrival counters, 66 KB)
+ * is a fixed array in the library's device image; every GPU that loads the library holds it until process exit.
+ *   logits [dev] fp32 [n_rows, V];  next_tok [dev] int32 [n_rows]: index of the row maximum, ties -> lowest id
+ *   (the rule river_decode_step uses);  cuda_stream: a cudaStream_t (NULL = default stream); the call is
+ *   asynchronous on it.
+ * n_rows > RIVER_NOALLOC_MAX_ROWS returns RIVER_E_NOMEM (split the batch); bad pointers / sizes RIVER_E_BADARG.
+ * The first call on a device looks up the scratch array's device address (with that device current); make that
+ * first call before any stream capture.  Calls no cudaMalloc / cudaFree or allocating library routine.  All calls
+ * on a device share the one array: two calls that overlap on the GPU (different streams) race; issue them on one
+ * stream or order them yourself. */
+#define RIVER_NOALLOC_MAX_ROWS 64
+int river_argmax_noalloc(const float *logits, int n_rows, int V, int32_t *next_tok, void *cuda_stream);
+
 int river_seq_len(const river_ctx *ctx, int slot);       /* tokens cached in the slot, or RIVER_E_BADSLOT */
 int river_release(river_ctx *ctx, int slot);             /* free the slot's pages */
 int river_stats(river_ctx *ctx, river_stats_t *host_out); /* synchronises the stream */

@@ -54,7 +54,7 @@ class river_kernel_time(C.Structure):
                 ("alg_bytes_total", C.c_double)]
 
 
-EXPORTS = ("river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
+EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error")
 
@@ -91,6 +91,7 @@ def load():
     L.river_stats.argtypes = [vp, C.POINTER(river_stats_t)]
     L.river_profile.argtypes = [vp, C.c_int]
     L.river_profile_read.argtypes = [vp, C.POINTER(river_kernel_time), C.c_int, C.POINTER(C.c_int)]
+    L.river_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, vp]
     L.river_destroy.argtypes = [vp]
     L.river_destroy.restype = None
     L.river_last_error.argtypes = [vp]
@@ -132,6 +133,20 @@ def _hp(t: Optional[torch.Tensor]) -> int:
 
 def _i32_host(xs: Sequence[int]):
     return (C.c_int32 * len(xs))(*[int(v) for v in xs])
+
+
+def argmax_noalloc(logits: torch.Tensor, next_tok: torch.Tensor, stream=None) -> None:
+    """river_argmax_noalloc: next_tok[r] = index of the maximum of logits[r] (ties -> lowest id), no allocation.
+
+    logits: CUDA fp32 [n_rows, V] (n_rows <= 64); next_tok: CUDA int32 [n_rows].  Asynchronous on `stream`
+    (default: torch's current stream).  For callers that cannot allocate device memory at this point."""
+    assert logits.dtype == torch.float32 and next_tok.dtype == torch.int32 and logits.dim() == 2
+    st = stream if stream is not None else torch.cuda.current_stream(logits.device)
+    with torch.cuda.device(logits.device):
+        rc = load().river_argmax_noalloc(_dp(logits), logits.shape[0], logits.shape[1], _dp(next_tok),
+                                         C.c_void_p(st.cuda_stream))
+    if rc:
+        raise RiverError(rc, "river_argmax_noalloc rejected the call")
 
 
 class River:
