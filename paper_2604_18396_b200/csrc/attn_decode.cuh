@@ -88,15 +88,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     constexpr int VE = DH / 32;                  // head dims per lane in P.V
 
     const int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     pdl_launch();
-    pdl_wait();
-    if (row >= a.meta->n_rows) return;
-    const int chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
-    const int pos = a.row_pos[row], slot = a.row_slot[row];
-    const int p0 = split * chunk;
-    if (p0 > pos) return;
-    const int p1 = min(p0 + chunk, pos + 1);     // positions [p0, p1)
-    const int n_tiles = (p1 - p0 + kAttnTile - 1) / kAttnTile;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -107,9 +100,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     uint64_t *bars = reinterpret_cast<uint64_t *>(sm + kAttnConsumers * GQ * (DH + 2));  // full[S], empty[S]
     __shared__ int s_abort;
     __shared__ bool s_last;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) {
+    const bool is_producer = tid == kAttnConsumers * 32;
+    if (is_producer) {  // nothing here depends on the previous kernel
         s_abort = 0;
         for (int s = 0; s < kAttnStages; ++s) {
             mbar_init(smem_u32(&bars[s]), 1);
@@ -118,40 +110,54 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    pdl_wait();
+    // independent loads first, decisions after (every index below is valid for any row of the grid)
+    const int n_rows = a.meta->n_rows, chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
+    const int pos = a.row_pos[row], slot = a.row_slot[row];
+    if (row >= n_rows) return;
+    const int p0 = split * chunk;
+    if (p0 > pos) return;
+    const int p1 = min(p0 + chunk, pos + 1);     // positions [p0, p1)
+    const int n_tiles = (p1 - p0 + kAttnTile - 1) / kAttnTile;
+    volatile int *abortp = &s_abort;
+
+    // one lane issues the TMA copies, at most kAttnStages tiles ahead; the first tiles go out before anything else
+    auto issue_tile = [&](int t) {
+        const int32_t *pt = a.page_tbl + (size_t)slot * a.max_pages_per_seq;
+        const int s = t % kAttnStages;
+        if (t >= kAttnStages &&
+            !mbar_wait(smem_u32(&bars[kAttnStages + s]), ((t / kAttnStages) - 1) & 1, abortp, a.dev_err))
+            return false;
+        const int first_page = (p0 + t * kAttnTile) / kPage;
+        const int n_valid = min(kAttnConsumers, (p1 - 1) / kPage - first_page + 1);
+        const uint32_t full = smem_u32(&bars[s]);
+        mbar_expect_tx(full, (uint32_t)(n_valid * 2 * PAGE_BYTES));
+        for (int j = 0; j < n_valid; ++j) {
+            int page = pt[first_page + j];
+            if (page < 0 || page >= a.n_pages) { atomicExch(a.dev_err, DEV_BAD_PAGE); page = 0; }
+            // cache rows of (layer, page, K|V, kv head): 16 consecutive rows of the [rows][DH] view
+            const int yk = ((((a.layer0 * a.n_pages + page) * 2 + 0) * a.Hkv) + kvh) * kPage;
+            const int yv = ((((a.layer0 * a.n_pages + page) * 2 + 1) * a.Hkv) + kvh) * kPage;
+            const uint32_t dk = smem_u32(stages + s * STAGE_BYTES + j * PAGE_BYTES);
+            const uint32_t dv = dk + kAttnConsumers * PAGE_BYTES;
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                tma_load_2d(dk + b * (kPage * 128), &tmap, b * 64, yk, full);
+                tma_load_2d(dv + b * (kPage * 128), &tmap, b * 64, yv, full);
+            }
+        }
+        return true;
+    };
+    if (is_producer)
+        for (int t = 0; t < min(n_tiles, kAttnStages); ++t) issue_tile(t);
     for (int i = tid; i < GQ * DH; i += kAttnThreads)
         sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
     __syncthreads();
-    volatile int *abortp = &s_abort;
 
     if (warp == kAttnConsumers) {
-        // ---------------- producer: one lane issues the TMA copies, at most kAttnStages tiles ahead
-        if (lane == 0) {
-            const int32_t *pt = a.page_tbl + (size_t)slot * a.max_pages_per_seq;
-            for (int t = 0; t < n_tiles; ++t) {
-                const int s = t % kAttnStages;
-                if (t >= kAttnStages &&
-                    !mbar_wait(smem_u32(&bars[kAttnStages + s]), ((t / kAttnStages) - 1) & 1, abortp, a.dev_err))
-                    break;
-                const int first_page = (p0 + t * kAttnTile) / kPage;
-                const int n_valid = min(kAttnConsumers, (p1 - 1) / kPage - first_page + 1);
-                const uint32_t full = smem_u32(&bars[s]);
-                mbar_expect_tx(full, (uint32_t)(n_valid * 2 * PAGE_BYTES));
-                for (int j = 0; j < n_valid; ++j) {
-                    int page = pt[first_page + j];
-                    if (page < 0 || page >= a.n_pages) { atomicExch(a.dev_err, DEV_BAD_PAGE); page = 0; }
-                    // cache rows of (layer, page, K|V, kv head): 16 consecutive rows of the [rows][DH] view
-                    const int yk = ((((a.layer0 * a.n_pages + page) * 2 + 0) * a.Hkv) + kvh) * kPage;
-                    const int yv = ((((a.layer0 * a.n_pages + page) * 2 + 1) * a.Hkv) + kvh) * kPage;
-                    const uint32_t dk = smem_u32(stages + s * STAGE_BYTES + j * PAGE_BYTES);
-                    const uint32_t dv = dk + kAttnConsumers * PAGE_BYTES;
-#pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        tma_load_2d(dk + b * (kPage * 128), &tmap, b * 64, yk, full);
-                        tma_load_2d(dv + b * (kPage * 128), &tmap, b * 64, yv, full);
-                    }
-                }
-            }
-        }
+        if (lane == 0)
+            for (int t = kAttnStages; t < n_tiles; ++t)
+                if (!issue_tile(t)) break;
     } else {
         // ---------------- consumers: warp w owns page w of every tile
         const int r = lane & 15, hsel = lane >> 4;
@@ -251,7 +257,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
         for (int i = 0; i < 2000; ++i) __nanosleep(100);
         return;
     }
-    // merge the four warp states -> one partial per head
+    // merge the four warp states -> one result per head for this split
+    const int ns = pos / chunk + 1;  // splits of this row
     for (int t = tid; t < GQ * DH; t += kAttnThreads) {
         const int g = t / DH, e = t % DH;
         float M = -CUDART_INF_F;
@@ -265,32 +272,52 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
             num = fmaf(c, src[e], num);
             den = fmaf(c, src[DH + 1], den);
         }
-        const size_t idx = ((size_t)row * a.Hq + kvh * GQ + g) * n_splits + split;
-        a.part_o[idx * DH + e] = num;
-        if (e == 0) a.part_ml[idx] = make_float2(M, den);
+        if (ns == 1) {  // the only split of the row: this is the attention output
+            a.out[((size_t)row * a.Hq + kvh * GQ + g) * DH + e] = num / den;
+        } else {
+            const size_t idx = ((size_t)row * a.Hq + kvh * GQ + g) * n_splits + split;
+            a.part_o[idx * DH + e] = num;
+            if (e == 0) a.part_ml[idx] = make_float2(M, den);
+        }
     }
+    if (ns == 1) return;
     // the last split of this (row, kv head) to finish merges all of them:
     // out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s  (atomic ticket, no spinning)
-    const int ns = pos / chunk + 1;
     __threadfence();
     __syncthreads();
     if (tid == 0) s_last = (atomicAdd(&a.tickets[row * a.Hkv + kvh], 1u) == (unsigned)(ns - 1));
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    float *wgt = sm;  // [GQ][ns] weights 2^(m_s - M) / sum, reusing the merge buffer (ns <= 64)
+    const size_t base0 = ((size_t)row * a.Hq + kvh * GQ) * n_splits;
+    for (int t = tid; t < GQ * ns; t += kAttnThreads) {
+        const int g = t / ns, sidx = t % ns;
+        const float2 ml = __ldcg(&a.part_ml[base0 + (size_t)g * n_splits + sidx]);
+        wgt[g * 64 + sidx] = ml.x;
+        wgt[GQ * 64 + g * 64 + sidx] = ml.y;
+    }
+    __syncthreads();
+    if (tid < GQ) {
+        float M = -CUDART_INF_F;
+        for (int sidx = 0; sidx < ns; ++sidx) M = fmaxf(M, wgt[tid * 64 + sidx]);
+        float den = 0.f;
+        for (int sidx = 0; sidx < ns; ++sidx) {
+            const float c = ex2(wgt[tid * 64 + sidx] - M);
+            den = fmaf(c, wgt[GQ * 64 + tid * 64 + sidx], den);
+            wgt[tid * 64 + sidx] = c;
+        }
+        const float inv = 1.f / den;
+        for (int sidx = 0; sidx < ns; ++sidx) wgt[tid * 64 + sidx] *= inv;
+    }
+    __syncthreads();
     for (int t = tid; t < GQ * DH; t += kAttnThreads) {
         const int g = t / DH, e = t % DH;
-        const size_t base = ((size_t)row * a.Hq + kvh * GQ + g) * n_splits;
-        float M = -CUDART_INF_F;
-        for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&a.part_ml[base + s]).x);
-        float num = 0.f, den = 0.f;
-        for (int s = 0; s < ns; ++s) {
-            const float2 ml = __ldcg(&a.part_ml[base + s]);
-            const float c = ex2(ml.x - M);
-            num = fmaf(c, __ldcg(&a.part_o[(base + s) * DH + e]), num);
-            den = fmaf(c, ml.y, den);
-        }
-        a.out[((size_t)row * a.Hq + kvh * GQ + g) * DH + e] = num / den;
+        const float *po = a.part_o + (base0 + (size_t)g * n_splits) * DH + e;
+        float num = 0.f;
+#pragma unroll 8
+        for (int sidx = 0; sidx < ns; ++sidx) num = fmaf(wgt[g * 64 + sidx], __ldcg(po + (size_t)sidx * DH), num);
+        a.out[((size_t)row * a.Hq + kvh * GQ + g) * DH + e] = num;
     }
     if (tid == 0) a.tickets[row * a.Hkv + kvh] = 0;
 }

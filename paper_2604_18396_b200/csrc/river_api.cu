@@ -199,17 +199,17 @@ W4 w4(const river_w4 &r) {
     return W4{(const uint8_t *)r.codes, (const uint16_t *)r.scale, (const uint16_t *)r.zero};
 }
 
-// KV split geometry of this step: enough (row, kv head, split) work items to fill the GPU about four times over,
-// splits of at least one 64-position tile.  The split count depends only on the row count, so a captured launch
+// KV split geometry of this step: enough (row, kv head, split) work items to fill the GPU about twice over,
+// splits of at least two 64-position tiles.  The split count depends only on the row count, so a captured launch
 // stays valid while the chunk length grows with the context.
 void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     const river_config &g = c->cfg;
     int max_pos = 0;
     for (int i = 0; i < n; ++i) max_pos = std::max(max_pos, mh[kMetaHdr + g.max_batch + i]);
-    int S = (4 * c->num_sms + n * g.Hkv - 1) / (n * g.Hkv);
+    int S = (2 * c->num_sms + n * g.Hkv - 1) / (n * g.Hkv);
     S = std::max(1, std::min(S, 64));
     int chunk = (max_pos + 1 + S - 1) / S;
-    chunk = std::max(kAttnTile, (chunk + kAttnTile - 1) / kAttnTile * kAttnTile);
+    chunk = std::max(2 * kAttnTile, (chunk + kAttnTile - 1) / kAttnTile * kAttnTile);
     mh[3] = chunk;
     mh[4] = S;
     mh[5] = n;  // hint_act: every row starts in the backbone

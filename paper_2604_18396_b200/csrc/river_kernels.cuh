@@ -218,12 +218,23 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     if (row < n && exited[row] == 0 && (eligible || scores)) {
         const float4 *a = reinterpret_cast<const float4 *>(h_in + (size_t)row * d);
         const float4 *b = reinterpret_cast<const float4 *>(h_out + (size_t)row * d);
+        const float tau_row = tau[row];
         float ab = 0.f, aa = 0.f, bb = 0.f;
-        for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
-            const float4 x = a[i], y = b[i];
-            ab += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
-            aa += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-            bb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+        const int nv = d / 4;
+        for (int i0 = 0; i0 < nv; i0 += 4 * 256) {  // four loads of each vector in flight per thread
+            float4 x[4], y[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * 256 + threadIdx.x;
+                x[u] = i < nv ? __ldcg(a + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                y[u] = i < nv ? __ldcg(b + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                ab += x[u].x * y[u].x + x[u].y * y[u].y + x[u].z * y[u].z + x[u].w * y[u].w;
+                aa += x[u].x * x[u].x + x[u].y * x[u].y + x[u].z * x[u].z + x[u].w * x[u].w;
+                bb += y[u].x * y[u].x + y[u].y * y[u].y + y[u].z * y[u].z + y[u].w * y[u].w;
+            }
         }
         ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -234,16 +245,20 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
             for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { ab += red[0][w]; aa += red[1][w]; bb += red[2][w]; }
             float s = 0.f;
             if (aa > 0.f && bb > 0.f) s = ab / (sqrtf(aa) * sqrtf(bb));
-            pass[row] = (s > tau[row]) ? 1 : 0;
+            pass[row] = (s > tau_row) ? 1 : 0;
             if (scores) scores[(size_t)row * L + (l - 1)] = s;
         }
     }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
+    if (gridDim.x > 1) {  // a single CTA is its own last arriver
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+    } else {
+        __syncthreads();
+    }
     // ---- decision for every row still in the backbone
     if (threadIdx.x == 0) s_allpass = 1;
     __syncthreads();
@@ -264,7 +279,7 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     }
     __syncthreads();
     build_lists(n, exited, l, lists, hint_act, s_cnt);
-    if (threadIdx.x == 0) *ticket = 0;
+    if (threadIdx.x == 0 && gridDim.x > 1) *ticket = 0;
 }
 
 // ---------------------------------------------------------------- shared by the projection kernels
