@@ -1,0 +1,367 @@
+// Batched backbone projections on the 5th-generation tensor cores (sm_100a): tcgen05.mma with TMEM accumulators.
+//
+// With more than a handful of activation rows the CUDA-core stream kernel becomes issue-bound, while the projection
+// is still a weight stream: D[128 output features x N rows] = W[128 x K] . X^T[K x N] ("swap-AB": the weights are the
+// M = 128 operand, the rows of the step the N operand, 16 <= N <= 256).  One CTA owns one 128-feature tile and one
+// K-split of it.  A producer lane brings 128 x 64 weight tiles and N x 64 activation tiles into shared memory with
+// 2-D TMA copies (128-byte swizzle, K-major: the canonical UMMA layout); one lane issues tcgen05.mma (kind::f16,
+// bf16 x bf16 -> fp32) against the activations' bf16 high part and again against their low part (x = hi + lo, so the
+// activations keep 16 mantissa bits although the tensor cores take bf16); tcgen05.commit releases the stage.  Four
+// epilogue warps read the accumulator out of TMEM (tcgen05.ld), park it in shared memory and, for split K, in a
+// global partial buffer; the last split of a tile to finish (atomic ticket, no spinning) adds the partials in split
+// order and runs the projection's epilogue (RoPE + KV-cache write, residual add, SwiGLU, logits + argmax partials).
+// Weights do not depend on the previous kernel: their first tiles are requested before the grid dependency resolves.
+#pragma once
+#include "attn_decode.cuh"
+#include "gemv_stream.cuh"
+
+namespace river {
+
+constexpr int kTcBM = 128;      // output features per tile (UMMA M)
+constexpr int kTcBK = 64;       // K per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kTcThreads = 192; // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2..5: epilogue
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major operand tile in shared memory, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t tc_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---------------------------------------------------------------- activation rows -> bf16 hi / lo operand buffers
+// One CTA per operand row i < n_pad: the i-th row of the backbone list (zero beyond the list), optionally
+// RMS-normalised, split as x = hi + lo with hi = bf16(x), lo = bf16(x - hi).
+__global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
+                                                      __nv_bfloat16 *xhi, __nv_bfloat16 *xlo) {
+    __shared__ float red[8];
+    pdl_launch();
+    pdl_wait();
+    const int i = blockIdx.x, n = *cnt;
+    __nv_bfloat16 *hi = xhi + (size_t)i * K, *lo = xlo + (size_t)i * K;
+    if (i >= n) {
+        for (int k = threadIdx.x; k < K; k += blockDim.x) { hi[k] = __float2bfloat16_rn(0.f); lo[k] = hi[k]; }
+        return;
+    }
+    const float *src = in.src + (size_t)idx[i] * K;
+    float scale = 1.f;
+    if (in.gain) {
+        float ss = 0.f;
+        for (int k = threadIdx.x; k < K; k += blockDim.x) { const float v = src[k]; ss = fmaf(v, v, ss); }
+        ss = warp_sum(ss);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        ss = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) ss += red[w];
+        scale = rsqrtf(ss / (float)K + in.eps);
+    }
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float v = src[k] * scale;
+        if (in.gain) v *= bf16f(in.gain[k]);
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[k] = h;
+        lo[k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+// ---------------------------------------------------------------- epilogues on a finished 128 x N tile in smem
+// tile(r, n) = sum over K of W[row0 + r] . x[n]; `rows` maps n to the step's row id; only n < n_live are real.
+struct TcResidEpi {  // out[row][row0 + r] = resid[row][row0 + r] + tile(r, n)
+    const float *resid;
+    float *out;
+    int out_dim;
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr) const {
+        const int row0 = tile_idx * kTcBM;
+        for (int t = tid; t < n_live * kTcBM; t += nthr) {
+            const int n = t / kTcBM, r = t % kTcBM;
+            const size_t o = (size_t)rows[n] * out_dim + row0 + r;
+            out[o] = resid[o] + tile[r * ld + n];
+        }
+    }
+};
+struct TcGateUpEpi {  // tile rows 0..63: gate features f0.., rows 64..127: up features f0..
+    float *act;
+    int F;
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr) const {
+        const int f0 = tile_idx * 64;
+        for (int t = tid; t < n_live * 64; t += nthr) {
+            const int n = t / 64, r = t % 64;
+            const float g = tile[r * ld + n], u = tile[(64 + r) * ld + n];
+            act[(size_t)rows[n] * F + f0 + r] = g / (1.f + __expf(-g)) * u;
+        }
+    }
+};
+struct TcQkvEpi {  // tiles walk the concatenated [q heads | k heads | v heads] features, 128 at a time
+    int Hq, Hkv, dh;
+    const float2 *rope_cs;
+    float *q_out;
+    KvAddr kv;
+    int *dev_err;
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr) const {
+        const int half = dh >> 1, heads_per_tile = kTcBM / dh;
+        const int feat0 = tile_idx * kTcBM;
+        const int qdim = Hq * dh, kvdim = Hkv * dh;
+        const int which = feat0 < qdim ? 0 : (feat0 < qdim + kvdim ? 1 : 2);
+        const int base = which == 0 ? feat0 : (which == 1 ? feat0 - qdim : feat0 - qdim - kvdim);  // inside its matrix
+        for (int t = tid; t < n_live * (kTcBM / 2); t += nthr) {
+            const int n = t / (kTcBM / 2), pr = t % (kTcBM / 2);
+            const int hh = pr / half, i = pr % half;  // head inside the tile, pair index
+            if (hh >= heads_per_tile) continue;
+            const int r_lo = hh * dh + i, r_hi = r_lo + half;
+            const int row = rows[n];
+            float lo = tile[r_lo * ld + n], hi = tile[r_hi * ld + n];
+            if (which != 2) {
+                const float2 cs = rope_cs[(size_t)row * half + i];
+                const float a = lo * cs.x - hi * cs.y, b = hi * cs.x + lo * cs.y;
+                lo = a; hi = b;
+            }
+            const int hl = (base + hh * dh) / dh;
+            if (which == 0) {
+                float *q = q_out + (size_t)row * qdim + (size_t)hl * dh;
+                q[i] = lo;
+                q[i + half] = hi;
+            } else {
+                const int pos = kv.row_pos[row], slot = kv.row_slot[row];
+                const int page = kv.page_tbl[(size_t)slot * kv.max_pages_per_seq + pos / kPage];
+                if (page < 0 || page >= kv.n_pages) { atomicExch(dev_err, DEV_BAD_PAGE); continue; }
+                const size_t o = kv.base(page, which - 1, hl, pos % kPage);
+                kv.pool[o + i] = __float2bfloat16_rn(lo);
+                kv.pool[o + i + half] = __float2bfloat16_rn(hi);
+            }
+        }
+    }
+};
+struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row for the greedy token
+    const StepMeta *meta;
+    int V;
+    float *part_val;
+    int32_t *part_idx;
+    int n_parts;
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *, int tid, int nthr) const {
+        float *logits = meta->logits;
+        const int v0 = tile_idx * kTcBM;
+        if (logits)
+            for (int t = tid; t < n_live * kTcBM; t += nthr) {
+                const int n = t / kTcBM, r = t % kTcBM;
+                logits[(size_t)n * V + v0 + r] = tile[r * ld + n];
+            }
+        for (int n = tid; n < n_live; n += nthr) {
+            float bv = -CUDART_INF_F;
+            int bi = 0x7fffffff;
+            for (int r = 0; r < kTcBM; ++r) {
+                const float v = tile[r * ld + n];
+                if (v > bv) { bv = v; bi = v0 + r; }
+            }
+            part_val[(size_t)n * n_parts + tile_idx] = bv;
+            part_idx[(size_t)n * n_parts + tile_idx] = bi;
+        }
+    }
+};
+
+// ---------------------------------------------------------------- the GEMM kernel
+struct TcArgs {
+    int K;            // inner dimension (multiple of 64)
+    int n_pad;        // N operand rows (multiple of 16, <= 256)
+    int splits;       // K splits per tile
+    int n_stages;     // pipeline depth
+    int a_rows_per_map;  // a tile's 128 rows come from map tile_idx / (rows_per_map / 128) ... see tile_map()
+    int gateup;       // 1: a tile is 64 rows of map 0 + 64 rows of map 1
+    int qkv_q_tiles, qkv_k_tiles;  // QKV: tiles per matrix (0 otherwise)
+    const int32_t *rows;   // step row id of operand row n
+    const int32_t *cnt;    // live operand rows (device)
+    float *partial;        // [tiles][splits][128][n_pad] fp32 (splits > 1)
+    unsigned *tickets;     // [tiles], zero between launches
+    int *dev_err;
+};
+
+template <class Epi>
+__global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0,
+                                                             const __grid_constant__ CUtensorMap map_a1,
+                                                             const __grid_constant__ CUtensorMap map_a2,
+                                                             const __grid_constant__ CUtensorMap map_bhi,
+                                                             const __grid_constant__ CUtensorMap map_blo,
+                                                             const TcArgs a, const Epi epi) {
+    extern __shared__ uint8_t tc_smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int NP = a.n_pad, S = a.n_stages;
+    const uint32_t a_bytes = kTcBM * kTcBK * 2, b_bytes = (uint32_t)NP * kTcBK * 2;
+    const uint32_t stage_bytes = a_bytes + 2 * b_bytes;  // multiples of 1024 (n_pad multiple of 16 -> b_bytes of 2048)
+    uint8_t *stages = smem;
+    float *tile = reinterpret_cast<float *>(stages);     // the finished tile reuses the pipeline memory
+    const int ld = NP + 1;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(stages + (size_t)S * stage_bytes);  // full[S], empty[S], acc
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort;
+    __shared__ bool s_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tile_idx = blockIdx.x / a.splits, split = blockIdx.x % a.splits;
+    const int kb_total = a.K / kTcBK;
+    const int kb0 = (int)(((long long)kb_total * split) / a.splits), kb1 = (int)(((long long)kb_total * (split + 1)) / a.splits);
+    const int nkb = kb1 - kb0;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < NP) tmem_cols <<= 1;
+
+    pdl_launch();
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars[s]), 1); mbar_init(smem_u32(&bars[S + s]), 1); }
+        mbar_init(smem_u32(&bars[2 * S]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {  // TMEM accumulator: 128 lanes x tmem_cols fp32 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(tmem_cols));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+        tc_fence_before();
+    }
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = s_tmem;
+    volatile int *abortp = &s_abort;
+
+    // where this tile's weight rows live
+    const CUtensorMap *ma = &map_a0, *ma2 = nullptr;
+    int ay = tile_idx * kTcBM, ay2 = 0;
+    if (a.gateup) { ma2 = &map_a1; ay = tile_idx * 64; ay2 = tile_idx * 64; }
+    else if (a.qkv_q_tiles) {
+        if (tile_idx >= a.qkv_q_tiles + a.qkv_k_tiles) { ma = &map_a2; ay = (tile_idx - a.qkv_q_tiles - a.qkv_k_tiles) * kTcBM; }
+        else if (tile_idx >= a.qkv_q_tiles) { ma = &map_a1; ay = (tile_idx - a.qkv_q_tiles) * kTcBM; }
+    }
+    auto load_a = [&](int i) {  // weight tile of k-block kb0 + i into stage i % S (expects the stage's whole byte count)
+        const int s = i % S;
+        const uint32_t full = smem_u32(&bars[s]), dst = smem_u32(stages + (size_t)s * stage_bytes);
+        mbar_expect_tx(full, stage_bytes);
+        const int x = (kb0 + i) * kTcBK;
+        if (ma2) {
+            // two 64-row boxes: gate rows then up rows (each box 64 x 64 bf16 = 8 KB, 1024-aligned)
+            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                         ::"r"(dst), "l"(ma), "r"(x), "r"(ay), "r"(full) : "memory");
+            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                         ::"r"(dst + a_bytes / 2), "l"(ma2), "r"(x), "r"(ay2), "r"(full) : "memory");
+        } else {
+            tma_load_2d(dst, ma, x, ay, full);
+        }
+    };
+    auto load_b = [&](int i) {
+        const int s = i % S;
+        const uint32_t full = smem_u32(&bars[s]), dst = smem_u32(stages + (size_t)s * stage_bytes) + a_bytes;
+        const int x = (kb0 + i) * kTcBK;
+        tma_load_2d(dst, &map_bhi, x, 0, full);
+        tma_load_2d(dst + b_bytes, &map_blo, x, 0, full);
+    };
+
+    // weights first: they depend on nothing
+    const int pre = min(S, nkb);
+    if (tid == 0)
+        for (int i = 0; i < pre; ++i) load_a(i);
+    pdl_wait();
+    const int n_live = *a.cnt;  // rows of the backbone list; the stream kernel serves the exit-layer rows
+    // even with no live row the requested weight tiles must land before the CTA may exit: run the pipeline once
+    const int nkb_run = n_live > 0 ? nkb : pre;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < nkb_run; ++i) {
+                if (i >= S) {
+                    if (!mbar_wait(smem_u32(&bars[S + i % S]), ((i / S) - 1) & 1, abortp, a.dev_err)) break;
+                    load_a(i);
+                }
+                load_b(i);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = tc_idesc(NP);
+            for (int i = 0; i < nkb_run; ++i) {
+                const int s = i % S;
+                if (!mbar_wait(smem_u32(&bars[s]), (i / S) & 1, abortp, a.dev_err)) break;
+                tc_fence_after();
+                const uint32_t sa = smem_u32(stages + (size_t)s * stage_bytes);
+                const uint64_t da = tc_smem_desc(sa), dhi = tc_smem_desc(sa + a_bytes), dlo = tc_smem_desc(sa + a_bytes + b_bytes);
+#pragma unroll
+                for (int k = 0; k < kTcBK / 16; ++k) {  // UMMA K = 16 bf16 = 32 bytes: +2 in the 16-byte address field
+                    tc_mma(tmem_d, da + 2 * k, dhi + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    tc_mma(tmem_d, da + 2 * k, dlo + 2 * k, idesc, 1u);
+                }
+                tc_commit(smem_u32(&bars[S + s]));  // frees the stage once these MMAs have read it
+            }
+            tc_commit(smem_u32(&bars[2 * S]));      // accumulator complete
+        }
+    }
+    // everyone: wait for the accumulator (bounded), then move it out of TMEM
+    bool ok = mbar_wait(smem_u32(&bars[2 * S]), 0, abortp, a.dev_err);
+    tc_fence_after();
+    __syncthreads();  // all TMA writes and MMA reads of the pipeline memory are over: it now holds the tile
+    if (warp >= 2 && ok && n_live > 0) {
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const int r = q * 32 + lane;
+        for (int c0 = 0; c0 < NP; c0 += 16) {
+            float v[16];
+            tc_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) tile[r * ld + c0 + j] = v[j];
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols));
+    }
+    if (!ok || s_abort || n_live <= 0) return;
+
+    if (a.splits > 1) {
+        // publish this split's partial; the last split of the tile to arrive adds all of them in split order
+        float *mine = a.partial + ((size_t)tile_idx * a.splits + split) * kTcBM * NP;
+        for (int t = tid; t < kTcBM * NP; t += kTcThreads) mine[t] = tile[(t / NP) * ld + (t % NP)];
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = atomicAdd(&a.tickets[tile_idx], 1u) == (unsigned)(a.splits - 1);
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        const float *all = a.partial + (size_t)tile_idx * a.splits * kTcBM * NP;
+        for (int t = tid; t < kTcBM * NP; t += kTcThreads) {
+            float v = 0.f;
+            for (int sp = 0; sp < a.splits; ++sp) v += __ldcg(all + (size_t)sp * kTcBM * NP + t);
+            tile[(t / NP) * ld + (t % NP)] = v;
+        }
+        if (tid == 0) a.tickets[tile_idx] = 0;
+        __syncthreads();
+    }
+    epi.run(tile, ld, tile_idx, n_live, a.rows, tid, kTcThreads);
+}
+
+inline size_t tc_smem_bytes(int n_pad, int n_stages) {
+    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)n_pad * kTcBK * 2;
+    const size_t pipe = (size_t)n_stages * stage, tile = sizeof(float) * (size_t)kTcBM * (n_pad + 1);
+    return 1024 + (pipe > tile ? pipe : tile) + sizeof(uint64_t) * (2 * n_stages + 1) + 64;
+}
+
+}  // namespace river

@@ -328,7 +328,7 @@ __device__ __forceinline__ void stream_rows_bf16(const P &p, int t, const uint16
 
 template <class P, int N, int R>
 __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjIn in, const RowLists rl, int has_river,
-                                                          int xstride) {
+                                                          int xstride, int skip_backbone) {
     extern __shared__ __align__(16) float stream_smem[];
     const int K = p.K;
     float *red = stream_smem;            // 32
@@ -345,14 +345,15 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     // nothing).  The hint never under-counts the backbone rows, so zero means they are certainly not needed.
     uint4 pre[R][kStreamPF];
     bool have_pre = false;
-    if (t0 + warp < t1 && *reinterpret_cast<const volatile int32_t *>(rl.hint_act) > 0) {
+    if (!skip_backbone && t0 + warp < t1 && *reinterpret_cast<const volatile int32_t *>(rl.hint_act) > 0) {
         const uint16_t *rows[R];
         stream_rows_bf16<P, N, R>(p, t0 + warp, rows);
         stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre);
         have_pre = true;
     }
     pdl_wait();
-    const int na = *rl.n_act, nr = has_river ? *rl.n_riv : 0;
+    // skip_backbone: the backbone rows of this step are served by the tensor-core kernel
+    const int na = skip_backbone ? 0 : *rl.n_act, nr = has_river ? *rl.n_riv : 0;
 
     for (int i0 = 0; i0 < na; i0 += N) {
         __syncthreads();

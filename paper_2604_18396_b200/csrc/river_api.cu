@@ -13,6 +13,7 @@
 #include "river_kernels.cuh"
 #include "attn_decode.cuh"
 #include "gemv_stream.cuh"
+#include "gemm_tc.cuh"
 
 using namespace river;
 
@@ -21,6 +22,7 @@ namespace {
 thread_local std::string g_init_error;
 
 constexpr int kStaging = 4;        // pinned metadata buffers in flight
+constexpr int kTcMaxCtas = 320;    // tiles x K-splits of a split-K projection (bounds the partial buffer)
 enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, kNumClasses };
 const char *const kClassNames[kNumClasses] = {"step_begin", "compact", "qkv_rope_kv", "attn_decode", "o_proj_resid",
                                               "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final"};
@@ -54,6 +56,17 @@ struct river_ctx {
     CUtensorMap kv_tmap;
     int attn_splits_now = 1;
     unsigned *attn_tickets, *tickets;  // [max_batch*Hkv], [4]
+    // tensor-core path: operand buffers, split-K partials, tickets, tensor maps of every weight matrix
+    __nv_bfloat16 *tc_xhi = nullptr, *tc_xlo = nullptr;
+    float *tc_partial = nullptr;
+    unsigned *tc_tickets = nullptr;
+    int tc_max_pad = 0, tc_kmax = 0;
+    bool tc_ok = false;
+    struct LayerMaps { CUtensorMap q, k, v, o, g, u, d; };
+    std::vector<LayerMaps> tc_maps;
+    CUtensorMap tc_map_head;
+    struct BMap { int K, np; CUtensorMap hi, lo; };
+    std::vector<BMap> tc_bmaps;
     int32_t *hint_act;
     struct GraphEntry { int n; bool scores; cudaGraphExec_t exec; int launches; };
     std::vector<GraphEntry> graphs;
@@ -127,6 +140,7 @@ const char *check_config(const river_config *c) {
 }
 
 int head_grid_for(const river_config *c) { return 148 * 4 > c->V / 4 ? std::max(1, c->V / 4) : 148 * 4; }
+int head_parts_for(const river_config *c) { return std::max(head_grid_for(c), c->V / 128 + 1); }  // argmax partials per row
 
 size_t carve(const river_config *c, river_ctx *x, char *base) {
     Carver cv{base};
@@ -134,8 +148,8 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     float *h0 = cv.take<float>(B * d), *h1 = cv.take<float>(B * d), *h2 = cv.take<float>(B * d);
     float *qb = cv.take<float>(B * c->Hq * c->dh), *ob = cv.take<float>(B * c->Hq * c->dh);
     float *act = cv.take<float>(B * c->F);
-    float *pv = cv.take<float>(B * (size_t)head_grid_for(c));
-    int32_t *pi = cv.take<int32_t>(B * (size_t)head_grid_for(c));
+    float *pv = cv.take<float>(B * (size_t)head_parts_for(c));
+    int32_t *pi = cv.take<int32_t>(B * (size_t)head_parts_for(c));
     float *tau = cv.take<float>(B);
     float *lg = cv.take<float>(B * (size_t)c->V);
     float *sc = cv.take<float>(B * L);
@@ -152,12 +166,18 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     int *de = cv.take<int>(1);
     unsigned *atk = cv.take<unsigned>(B * (size_t)c->Hkv), *tk4 = cv.take<unsigned>(4);
     int32_t *hint = md ? md + 5 : nullptr;  // StepMeta::hint_act
+    const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
+    const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
+    __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
+    float *tpart = cv.take<float>((size_t)kTcMaxCtas * kTcBM * tc_pad);
+    unsigned *ttk = cv.take<unsigned>(2048);
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
         x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
+        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_partial = tpart; x->tc_tickets = ttk; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
 }
@@ -285,7 +305,7 @@ StreamGeom pick_geometry(river_ctx *c, Kern kern, int tasks, size_t smem) {
 
 template <class P, int N, int R>
 cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks,
-                            int has_river, bool pdl) {
+                            int has_river, bool pdl, int skip_backbone) {
     const size_t smem = stream_smem_bytes(N, K);
     // one kernel instantiation serves several projections (O and down): cache the geometry per (tasks, K)
     struct Entry { int tasks, K; StreamGeom g; };
@@ -301,23 +321,116 @@ cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const Ro
         geom = &cache.back().g;
     }
     return launch_k(stream_proj_kernel<P, N, R>, dim3(geom->grid), dim3(geom->threads), smem, c->stream, pdl, p, in, rl,
-                    has_river, xs_stride(K, 32));
+                    has_river, xs_stride(K, 32), skip_backbone);
 }
 
 int stream_rows_per_task(int K) { return K >= 4096 ? 2 : 4; }
 
 template <class P>
 cudaError_t launch_stream(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks_r2, int n,
-                          int has_river, bool pdl) {
+                          int has_river, bool pdl, int skip_backbone = 0) {
     int n_sel = 1;
     while (n_sel < n && n_sel < 4 && stream_smem_bytes(n_sel * 2, K) <= 200 * 1024) n_sel *= 2;
     const int r = stream_rows_per_task(K);
     const int tasks = tasks_r2 * 2 / r;
-#define STREAM_CASE(N_, R_) if (n_sel == N_ && r == R_) return launch_stream_t<P, N_, R_>(c, p, in, rl, K, tasks, has_river, pdl);
+#define STREAM_CASE(N_, R_) if (n_sel == N_ && r == R_) return launch_stream_t<P, N_, R_>(c, p, in, rl, K, tasks, has_river, pdl, skip_backbone);
     STREAM_CASE(1, 2) STREAM_CASE(2, 2) STREAM_CASE(4, 2)
     STREAM_CASE(1, 4) STREAM_CASE(2, 4) STREAM_CASE(4, 4)
 #undef STREAM_CASE
     return cudaErrorInvalidValue;
+}
+
+typedef CUresult (*TmapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TmapEncodeFn tmap_encoder() {
+    static TmapEncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess) fn = (TmapEncodeFn)p;
+    }
+    return fn;
+}
+// bf16 row-major matrix [rows][inner] -> tiled map with a (box_rows x 64) box and the 128-byte swizzle
+bool make_map_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+    TmapEncodeFn fn = tmap_encoder();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {inner, rows};
+    const cuuint64_t gstride[1] = {inner * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ---- tensor-core projection launch
+// The shapes the tensor-core path takes: every output dimension in whole 128-feature tiles.
+bool tc_shape_ok(const river_config &g) {
+    return g.d % 128 == 0 && (g.Hq * g.dh) % 128 == 0 && (g.Hkv * g.dh) % 128 == 0 && g.F % 64 == 0 && g.V % 128 == 0 &&
+           g.d % 64 == 0 && g.F % 64 == 0 && (g.Hq * g.dh) % 64 == 0 && g.V / 128 <= 2048;
+}
+bool make_tc_maps(river_ctx *c) {
+    const river_config &g = c->cfg;
+    const int qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
+    c->tc_maps.resize(g.L);
+    for (int l = 0; l < g.L; ++l) {
+        const river_layer_weights &w = c->layers[l];
+        river_ctx::LayerMaps &m = c->tc_maps[l];
+        if (!make_map_bf16(&m.q, w.wq, g.d, qdim, 128) || !make_map_bf16(&m.k, w.wk, g.d, kvdim, 128) ||
+            !make_map_bf16(&m.v, w.wv, g.d, kvdim, 128) || !make_map_bf16(&m.o, w.wo, qdim, g.d, 128) ||
+            !make_map_bf16(&m.g, w.wg, g.d, g.F, 64) || !make_map_bf16(&m.u, w.wu, g.d, g.F, 64) ||
+            !make_map_bf16(&m.d, w.wd, g.F, g.d, 128))
+            return false;
+    }
+    return make_map_bf16(&c->tc_map_head, c->lm_head, g.d, g.V, 128);
+}
+const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
+    for (auto &b : c->tc_bmaps)
+        if (b.K == K && b.np == np) return &b;
+    river_ctx::BMap b{K, np, {}, {}};
+    if (!make_map_bf16(&b.hi, c->tc_xhi, K, np, np) || !make_map_bf16(&b.lo, c->tc_xlo, K, np, np)) return nullptr;
+    c->tc_bmaps.push_back(b);
+    return &c->tc_bmaps.back();
+}
+// K-splits per tile: fill whole waves of SMs, keep at least four 64-wide k-blocks per split
+int tc_pick_splits(const river_ctx *c, int tiles, int kb_total) {
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= 16; ++s) {
+        if (s > 1 && (kb_total / s < 4 || tiles * s > kTcMaxCtas)) break;
+        const int ctas = tiles * s, waves = (ctas + c->num_sms - 1) / c->num_sms;
+        const double eff = (double)ctas / (waves * c->num_sms);
+        if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+    }
+    return best;
+}
+
+template <class Epi>
+cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
+                      int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
+                      const int32_t *cnt, const Epi &epi) {
+    const int np = (n + 15) / 16 * 16;
+    const river_ctx::BMap *bm = tc_bmap(c, K, np);
+    if (!bm) return cudaErrorInvalidValue;
+    cudaError_t e = launch_k(tc_prep_kernel, dim3(np), dim3(256), 0, c->stream, true, in, rows, cnt, K, c->tc_xhi, c->tc_xlo);
+    if (e != cudaSuccess) return e;
+    ++c->st.launches_last_step;
+    TcArgs a{};
+    a.K = K; a.n_pad = np; a.splits = tc_pick_splits(c, tiles, K / kTcBK);
+    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
+    a.n_stages = (int)std::max<size_t>(2, std::min<size_t>(8, (200 * 1024) / stage));
+    a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
+    a.rows = rows; a.cnt = cnt; a.partial = c->tc_partial; a.tickets = c->tc_tickets; a.dev_err = c->dev_err;
+    const size_t smem = tc_smem_bytes(np, a.n_stages);
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaFuncSetAttribute(tc_gemm_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_smem = smem;
+    }
+    return launch_k(tc_gemm_kernel<Epi>, dim3(tiles * a.splits), dim3(kTcThreads), smem, c->stream, true, a0, a1, a2,
+                    bm->hi, bm->lo, a, epi);
 }
 
 // 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
@@ -443,6 +556,11 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
         const RowLists rl{ai, na, ri, nr, c->hint_act};
         float *h_in = c->h[hi], *h_mid = c->h[(hi + 1) % 3], *h_out = c->h[(hi + 2) % 3];
+        // With more rows than one CUDA-core pass takes, the backbone rows go to the tensor-core GEMM and the stream
+        // kernel only serves the exit-layer rows of the same launch slot.
+        const bool tc = c->tc_ok && n >= 5 && n <= c->tc_max_pad;
+        const river_ctx::LayerMaps *tm = tc ? &c->tc_maps[l - 1] : nullptr;
+        const int skip_bb = tc ? 1 : 0;
         // ---- a2: attention norm + QKV + RoPE + KV write
         {
             const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
@@ -452,8 +570,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             p.rq = w4(w.rq); p.rk = w4(w.rk); p.rv = w4(w.rv);
             p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
             p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
-            note(launch_stream(c, p, ProjIn{h_in, (const uint16_t *)w.attn_norm, g.rms_eps}, rl, d,
-                               (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true));
+            const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
+            if (tc) {
+                TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
+                note(launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM,
+                               kvdim / kTcBM, ai, na, e));
+            }
+            if (!tc || has_river)
+                note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, skip_bb));
         }
         // ---- a3: paged GQA decode attention
         {
@@ -467,8 +591,13 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             ResidProblem p{};
             p.w = (const uint16_t *)w.wo; p.rw = w4(w.ro); p.K = qdim; p.out_dim = d; p.group = g.group;
             p.resid = h_in; p.out = h_mid;
-            note(launch_stream(c, p, ProjIn{c->obuf, nullptr, 0.f}, rl, qdim, d / 2, n, has_river,
-                               !(g.flags & RIVER_F_SIMPLE_ATTN)));
+            const ProjIn in{c->obuf, nullptr, 0.f};
+            if (tc) {
+                TcResidEpi e{h_in, h_mid, d};
+                note(launch_tc(c, in, tm->o, tm->o, tm->o, qdim, d / kTcBM, n, 0, 0, 0, ai, na, e));
+            }
+            if (!tc || has_river)
+                note(launch_stream(c, p, in, rl, qdim, d / 2, n, has_river, tc || !(g.flags & RIVER_F_SIMPLE_ATTN), skip_bb));
         }
         // ---- a5: FFN norm + gate/up + SwiGLU
         {
@@ -477,8 +606,12 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             GateUpProblem p{};
             p.wg = (const uint16_t *)w.wg; p.wu = (const uint16_t *)w.wu; p.rg = w4(w.rg); p.ru = w4(w.ru);
             p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
-            note(launch_stream(c, p, ProjIn{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps}, rl, d, g.F, n, has_river,
-                               true));
+            const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
+            if (tc) {
+                TcGateUpEpi e{c->act, g.F};
+                note(launch_tc(c, in, tm->g, tm->u, tm->u, d, g.F / 64, n, 1, 0, 0, ai, na, e));
+            }
+            if (!tc || has_river) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb));
         }
         // ---- a5: down projection + residual
         {
@@ -487,7 +620,12 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             ResidProblem p{};
             p.w = (const uint16_t *)w.wd; p.rw = w4(w.rd); p.K = g.F; p.out_dim = d; p.group = g.group;
             p.resid = h_mid; p.out = h_out;
-            note(launch_stream(c, p, ProjIn{c->act, nullptr, 0.f}, rl, g.F, d / 2, n, has_river, true));
+            const ProjIn in{c->act, nullptr, 0.f};
+            if (tc) {
+                TcResidEpi e{h_mid, h_out, d};
+                note(launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e));
+            }
+            if (!tc || has_river) note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb));
         }
         // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
         {
@@ -504,11 +642,18 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         a.in = ProjIn{c->h[hi], c->final_norm, g.rms_eps};
         a.d = d; a.V = g.V; a.rows = c->head_rows(); a.meta = c->meta();
         a.part_val = c->part_val; a.part_idx = c->part_idx;
-        int n_sel = 1;
-        while (n_sel < n_head && n_sel < 4) n_sel *= 2;
-        const int xstride = xs_stride(d, 8);
-        const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xstride);
-        {
+        int n_parts = c->head_grid;
+        if (c->tc_ok && n_head >= 5 && n_head <= c->tc_max_pad) {
+            LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + 4.0 * n_head * g.V, 0, -1);
+            n_parts = g.V / kTcBM;
+            TcHeadEpi e{c->meta(), g.V, c->part_val, c->part_idx, n_parts};
+            note(launch_tc(c, a.in, c->tc_map_head, c->tc_map_head, c->tc_map_head, d, n_parts, n_head, 0, 0, 0,
+                           c->head_rows(), c->meta_dev + 2 /* StepMeta::n_head_rows */, e));
+        } else {
+            int n_sel = 1;
+            while (n_sel < n_head && n_sel < 4) n_sel *= 2;
+            const int xstride = xs_stride(d, 8);
+            const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xstride);
             LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + 4.0 * n_head * g.V, 0, -1);
             switch (n_sel) {
                 case 1: cudaFuncSetAttribute(lm_head_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -522,7 +667,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         {
             LaunchScope ls(c, K_ARGMAX, 0, 0, -1);
             note(launch_k(argmax_final_kernel, dim3(n_head), dim3(128), 0, c->stream, true, c->meta(),
-                          (const float *)c->part_val, (const int32_t *)c->part_idx, c->head_grid));
+                          (const float *)c->part_val, (const int32_t *)c->part_idx, n_parts));
         }
     }
     if (err == cudaSuccess) err = cudaGetLastError();
@@ -624,6 +769,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (prop.major != 10) return bail("this library is built for sm_100a (B200) only");
     c->num_sms = prop.multiProcessorCount;
     if (make_kv_tensor_map(c)) { river_destroy(c); return RIVER_E_DEVICE; }
+    c->tc_ok = !(cfg->flags & RIVER_F_NO_TC) && tc_shape_ok(*cfg) && make_tc_maps(c);
     for (int i = 0; i < kStaging; ++i) {
         if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");
         if (cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail("cudaEventCreate failed");
@@ -649,6 +795,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->tc_tickets, 0, sizeof(unsigned) * 2048, c->stream);
 
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_act, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_riv, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
