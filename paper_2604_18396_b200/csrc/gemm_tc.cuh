@@ -314,6 +314,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
             tc_commit(smem_u32(&bars[2 * S]));      // accumulator complete
         }
     }
+    // The other lanes of the two single-lane warps park at a warp barrier: a spinning (and possibly suspending)
+    // mbarrier wait in the same warp would steal the issuing lane's cycles.
+    __syncwarp();
     // everyone: wait for the accumulator (bounded), then move it out of TMEM
     bool ok = mbar_wait(smem_u32(&bars[2 * S]), 0, abortp, a.dev_err);
     tc_fence_after();
@@ -339,18 +342,29 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     if (a.splits > 1) {
         // publish this split's partial; the last split of the tile to arrive adds all of them in split order
         float *mine = a.partial + ((size_t)tile_idx * a.splits + split) * kTcBM * NP;
-        for (int t = tid; t < kTcBM * NP; t += kTcThreads) mine[t] = tile[(t / NP) * ld + (t % NP)];
+        for (int t = tid; t < kTcBM * NP / 4; t += kTcThreads) {
+            const float *src = tile + (t / (NP / 4)) * ld + (t % (NP / 4)) * 4;
+            reinterpret_cast<float4 *>(mine)[t] = make_float4(src[0], src[1], src[2], src[3]);
+        }
         __threadfence();
         __syncthreads();
         if (tid == 0) s_last = atomicAdd(&a.tickets[tile_idx], 1u) == (unsigned)(a.splits - 1);
         __syncthreads();
         if (!s_last) return;
         __threadfence();
-        const float *all = a.partial + (size_t)tile_idx * a.splits * kTcBM * NP;
-        for (int t = tid; t < kTcBM * NP; t += kTcThreads) {
-            float v = 0.f;
-            for (int sp = 0; sp < a.splits; ++sp) v += __ldcg(all + (size_t)sp * kTcBM * NP + t);
-            tile[(t / NP) * ld + (t % NP)] = v;
+        // all loads of one output vector are issued together (the splits are independent addresses)
+        const float4 *all4 = reinterpret_cast<const float4 *>(a.partial + (size_t)tile_idx * a.splits * kTcBM * NP);
+        const int vec_per_split = kTcBM * NP / 4, vec_per_row = NP / 4;
+        for (int t = tid; t < vec_per_split; t += kTcThreads) {
+            float4 x[16];
+#pragma unroll
+            for (int sp = 0; sp < 16; ++sp)
+                x[sp] = sp < a.splits ? __ldcg(all4 + (size_t)sp * vec_per_split + t) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 v = x[0];
+#pragma unroll
+            for (int sp = 1; sp < 16; ++sp) { v.x += x[sp].x; v.y += x[sp].y; v.z += x[sp].z; v.w += x[sp].w; }
+            float *dst = tile + (t / vec_per_row) * ld + (t % vec_per_row) * 4;
+            dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
         }
         if (tid == 0) a.tickets[tile_idx] = 0;
         __syncthreads();

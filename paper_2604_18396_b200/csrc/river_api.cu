@@ -394,14 +394,16 @@ const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
     c->tc_bmaps.push_back(b);
     return &c->tc_bmaps.back();
 }
-// K-splits per tile: fill whole waves of SMs, keep at least four 64-wide k-blocks per split
-int tc_pick_splits(const river_ctx *c, int tiles, int kb_total) {
+// K-splits per tile: fill whole waves of the CTA slots (two CTAs per SM when the pipeline fits twice), keep at
+// least four 64-wide k-blocks per split.  The kernel is memory-bound, so what matters is that all CTAs are resident
+// together and every SM slot streams.
+int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots) {
     int best = 1;
     double best_eff = 0.0;
     for (int s = 1; s <= 16; ++s) {
         if (s > 1 && (kb_total / s < 4 || tiles * s > kTcMaxCtas)) break;
-        const int ctas = tiles * s, waves = (ctas + c->num_sms - 1) / c->num_sms;
-        const double eff = (double)ctas / (waves * c->num_sms);
+        const int ctas = tiles * s, waves = (ctas + slots - 1) / slots;
+        const double eff = (double)ctas / ((double)waves * slots);
         if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
     }
     return best;
@@ -418,9 +420,11 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
     if (e != cudaSuccess) return e;
     ++c->st.launches_last_step;
     TcArgs a{};
-    a.K = K; a.n_pad = np; a.splits = tc_pick_splits(c, tiles, K / kTcBK);
+    a.K = K; a.n_pad = np;
     const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
-    a.n_stages = (int)std::max<size_t>(2, std::min<size_t>(8, (200 * 1024) / stage));
+    a.n_stages = (int)std::max<size_t>(2, std::min<size_t>(8, (106 * 1024) / stage));  // two CTAs per SM if possible
+    const int occ = tc_smem_bytes(np, a.n_stages) <= 113 * 1024 ? 2 : 1;
+    a.splits = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * occ);
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     a.rows = rows; a.cnt = cnt; a.partial = c->tc_partial; a.tickets = c->tc_tickets; a.dev_err = c->dev_err;
     const size_t smem = tc_smem_bytes(np, a.n_stages);
