@@ -7,9 +7,11 @@
 // 2-D TMA copies (128-byte swizzle, K-major: the canonical UMMA layout); one lane issues tcgen05.mma (kind::f16,
 // bf16 x bf16 -> fp32) against the activations' bf16 high part and again against their low part (x = hi + lo, so the
 // activations keep 16 mantissa bits although the tensor cores take bf16); tcgen05.commit releases the stage.  Four
-// epilogue warps read the accumulator out of TMEM (tcgen05.ld), park it in shared memory and, for split K, in a
-// global partial buffer; the last split of a tile to finish (atomic ticket, no spinning) adds the partials in split
-// order and runs the projection's epilogue (RoPE + KV-cache write, residual add, SwiGLU, logits + argmax partials).
+// epilogue warps read the accumulator out of TMEM (tcgen05.ld) and park it in shared memory.  The K-splits of one
+// tile form a thread-block cluster: after a cluster barrier every split CTA adds, in split order, its own slice of
+// the tile's rows from all peers' shared memory (distributed shared memory: a reduce-scatter with no trip through
+// HBM, no atomics, a fixed summation order) and runs the projection's epilogue on that slice (RoPE + KV-cache
+// write, residual add, SwiGLU, logits + argmax partials).
 // Weights do not depend on the previous kernel: their first tiles are requested before the grid dependency resolves.
 #pragma once
 #include "attn_decode.cuh"
@@ -64,42 +66,80 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int
     pdl_launch();
     pdl_wait();
     const int i = blockIdx.x, n = *cnt;
-    __nv_bfloat16 *hi = xhi + (size_t)i * K, *lo = xlo + (size_t)i * K;
+    uint2 *hi = reinterpret_cast<uint2 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint2 *>(xlo + (size_t)i * K);
+    const int nv = K >> 2;
     if (i >= n) {
-        for (int k = threadIdx.x; k < K; k += blockDim.x) { hi[k] = __float2bfloat16_rn(0.f); lo[k] = hi[k]; }
+        for (int v = threadIdx.x; v < nv; v += blockDim.x) { hi[v] = make_uint2(0u, 0u); lo[v] = make_uint2(0u, 0u); }
         return;
     }
-    const float *src = in.src + (size_t)idx[i] * K;
+    const float4 *src = reinterpret_cast<const float4 *>(in.src + (size_t)idx[i] * K);
     float scale = 1.f;
     if (in.gain) {
         float ss = 0.f;
-        for (int k = threadIdx.x; k < K; k += blockDim.x) { const float v = src[k]; ss = fmaf(v, v, ss); }
+        for (int v0 = 0; v0 < nv; v0 += 4 * 256) {
+            float4 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int v = v0 + u * 256 + threadIdx.x;
+                x[u] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) ss += x[u].x * x[u].x + x[u].y * x[u].y + x[u].z * x[u].z + x[u].w * x[u].w;
+        }
         ss = warp_sum(ss);
         if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
         __syncthreads();
         ss = 0.f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) ss += red[w];
+        for (int w = 0; w < 8; ++w) ss += red[w];
         scale = rsqrtf(ss / (float)K + in.eps);
     }
-    for (int k = threadIdx.x; k < K; k += blockDim.x) {
-        float v = src[k] * scale;
-        if (in.gain) v *= bf16f(in.gain[k]);
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        hi[k] = h;
-        lo[k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    auto split2 = [](float a, float b, uint32_t &h, uint32_t &l) {
+        const __nv_bfloat16 ha = __float2bfloat16_rn(a), hb = __float2bfloat16_rn(b);
+        const __nv_bfloat16 la = __float2bfloat16_rn(a - __bfloat162float(ha)), lb = __float2bfloat16_rn(b - __bfloat162float(hb));
+        h = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
+        l = (uint32_t)__bfloat16_as_ushort(la) | ((uint32_t)__bfloat16_as_ushort(lb) << 16);
+    };
+    for (int v0 = 0; v0 < nv; v0 += 4 * 256) {
+        float4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = v0 + u * 256 + threadIdx.x;
+            x[u] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = v0 + u * 256 + threadIdx.x;
+            if (v < nv) {
+                float4 y = x[u];
+                y.x *= scale; y.y *= scale; y.z *= scale; y.w *= scale;
+                if (in.gain) {
+                    const uint2 gw = *reinterpret_cast<const uint2 *>(in.gain + 4 * v);
+                    y.x *= bf16lo(gw.x); y.y *= bf16hi(gw.x); y.z *= bf16lo(gw.y); y.w *= bf16hi(gw.y);
+                }
+                uint2 h, l;
+                split2(y.x, y.y, h.x, l.x);
+                split2(y.z, y.w, h.y, l.y);
+                hi[v] = h;
+                lo[v] = l;
+            }
+        }
     }
 }
 
 // ---------------------------------------------------------------- epilogues on a finished 128 x N tile in smem
 // tile(r, n) = sum over K of W[row0 + r] . x[n]; `rows` maps n to the step's row id; only n < n_live are real.
+// The 128 tile rows are handled as 64 pairs; an epilogue call covers the pairs [pr0, pr1) (a K-split CTA finishes
+// its own slice of the tile), and pair_rows() tells which two tile rows pair pr is.
 struct TcResidEpi {  // out[row][row0 + r] = resid[row][row0 + r] + tile(r, n)
     const float *resid;
     float *out;
     int out_dim;
-    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr) const {
-        const int row0 = tile_idx * kTcBM;
-        for (int t = tid; t < n_live * kTcBM; t += nthr) {
-            const int n = t / kTcBM, r = t % kTcBM;
+    __device__ void pair_rows(int pr, int &r0, int &r1) const { r0 = 2 * pr; r1 = 2 * pr + 1; }
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
+                        int pr0, int pr1) const {
+        const int row0 = tile_idx * kTcBM, nr = 2 * (pr1 - pr0);
+        for (int t = tid; t < n_live * nr; t += nthr) {
+            const int n = t / nr, r = 2 * pr0 + t % nr;
             const size_t o = (size_t)rows[n] * out_dim + row0 + r;
             out[o] = resid[o] + tile[r * ld + n];
         }
@@ -108,10 +148,12 @@ struct TcResidEpi {  // out[row][row0 + r] = resid[row][row0 + r] + tile(r, n)
 struct TcGateUpEpi {  // tile rows 0..63: gate features f0.., rows 64..127: up features f0..
     float *act;
     int F;
-    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr) const {
-        const int f0 = tile_idx * 64;
-        for (int t = tid; t < n_live * 64; t += nthr) {
-            const int n = t / 64, r = t % 64;
+    __device__ void pair_rows(int pr, int &r0, int &r1) const { r0 = pr; r1 = 64 + pr; }
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
+                        int pr0, int pr1) const {
+        const int f0 = tile_idx * 64, np = pr1 - pr0;
+        for (int t = tid; t < n_live * np; t += nthr) {
+            const int n = t / np, r = pr0 + t % np;
             const float g = tile[r * ld + n], u = tile[(64 + r) * ld + n];
             act[(size_t)rows[n] * F + f0 + r] = g / (1.f + __expf(-g)) * u;
         }
@@ -123,14 +165,21 @@ struct TcQkvEpi {  // tiles walk the concatenated [q heads | k heads | v heads] 
     float *q_out;
     KvAddr kv;
     int *dev_err;
-    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr) const {
+    __device__ void pair_rows(int pr, int &r0, int &r1) const {
+        const int half = dh >> 1;
+        r0 = (pr / half) * dh + pr % half;
+        r1 = r0 + half;
+    }
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
+                        int pr0, int pr1) const {
         const int half = dh >> 1, heads_per_tile = kTcBM / dh;
         const int feat0 = tile_idx * kTcBM;
         const int qdim = Hq * dh, kvdim = Hkv * dh;
         const int which = feat0 < qdim ? 0 : (feat0 < qdim + kvdim ? 1 : 2);
         const int base = which == 0 ? feat0 : (which == 1 ? feat0 - qdim : feat0 - qdim - kvdim);  // inside its matrix
-        for (int t = tid; t < n_live * (kTcBM / 2); t += nthr) {
-            const int n = t / (kTcBM / 2), pr = t % (kTcBM / 2);
+        const int np = pr1 - pr0;
+        for (int t = tid; t < n_live * np; t += nthr) {
+            const int n = t / np, pr = pr0 + t % np;
             const int hh = pr / half, i = pr % half;  // head inside the tile, pair index
             if (hh >= heads_per_tile) continue;
             const int r_lo = hh * dh + i, r_hi = r_lo + half;
@@ -163,7 +212,10 @@ struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row
     float *part_val;
     int32_t *part_idx;
     int n_parts;
-    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *, int tid, int nthr) const {
+    __device__ void pair_rows(int pr, int &r0, int &r1) const { r0 = 2 * pr; r1 = 2 * pr + 1; }
+    // (the LM head is never K-split: the argmax partial below needs all 128 rows of the tile)
+    __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *, int tid, int nthr, int,
+                        int) const {
         float *logits = meta->logits;
         const int v0 = tile_idx * kTcBM;
         if (logits)
@@ -188,15 +240,13 @@ struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row
 struct TcArgs {
     int K;            // inner dimension (multiple of 64)
     int n_pad;        // N operand rows (multiple of 16, <= 256)
-    int splits;       // K splits per tile
+    int splits;       // K splits per tile = CTAs per cluster (<= 8)
     int n_stages;     // pipeline depth
     int a_rows_per_map;  // a tile's 128 rows come from map tile_idx / (rows_per_map / 128) ... see tile_map()
     int gateup;       // 1: a tile is 64 rows of map 0 + 64 rows of map 1
     int qkv_q_tiles, qkv_k_tiles;  // QKV: tiles per matrix (0 otherwise)
     const int32_t *rows;   // step row id of operand row n
     const int32_t *cnt;    // live operand rows (device)
-    float *partial;        // [tiles][splits][128][n_pad] fp32 (splits > 1)
-    unsigned *tickets;     // [tiles], zero between launches
     int *dev_err;
 };
 
@@ -218,7 +268,6 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     uint64_t *bars = reinterpret_cast<uint64_t *>(stages + (size_t)S * stage_bytes);  // full[S], empty[S], acc
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
-    __shared__ bool s_last;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tile_idx = blockIdx.x / a.splits, split = blockIdx.x % a.splits;
     const int kb_total = a.K / kTcBK;
@@ -337,45 +386,59 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols));
     }
-    if (!ok || s_abort || n_live <= 0) return;
-
+    if (n_live <= 0) return;  // uniform over the cluster: nobody waits for anybody
+    const bool good = ok && !s_abort;
+    int pr0 = 0, pr1 = kTcBM / 2;
     if (a.splits > 1) {
-        // publish this split's partial; the last split of the tile to arrive adds all of them in split order
-        float *mine = a.partial + ((size_t)tile_idx * a.splits + split) * kTcBM * NP;
-        for (int t = tid; t < kTcBM * NP / 4; t += kTcThreads) {
-            const float *src = tile + (t / (NP / 4)) * ld + (t % (NP / 4)) * 4;
-            reinterpret_cast<float4 *>(mine)[t] = make_float4(src[0], src[1], src[2], src[3]);
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) s_last = atomicAdd(&a.tickets[tile_idx], 1u) == (unsigned)(a.splits - 1);
-        __syncthreads();
-        if (!s_last) return;
-        __threadfence();
-        // all loads of one output vector are issued together (the splits are independent addresses)
-        const float4 *all4 = reinterpret_cast<const float4 *>(a.partial + (size_t)tile_idx * a.splits * kTcBM * NP);
-        const int vec_per_split = kTcBM * NP / 4, vec_per_row = NP / 4;
-        for (int t = tid; t < vec_per_split; t += kTcThreads) {
-            float4 x[16];
+        // Reduce-scatter over the cluster: CTA `split` owns the pairs [pr0, pr1) of the tile and adds them up from
+        // every peer's shared memory in split order.  Even a CTA that gave up takes part in both barriers: a
+        // cluster barrier has no time-out.
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        pr0 = (kTcBM / 2) * split / a.splits;
+        pr1 = (kTcBM / 2) * (split + 1) / a.splits;
+        float *fin = tile + kTcBM * ld;  // [2 * (pr1 - pr0)][NP] behind the tile
+        const int nrows = 2 * (pr1 - pr0);
+        if (good) {
+            for (int t = tid; t < nrows * NP; t += kTcThreads) {
+                const int j = t / NP, n = t % NP;
+                int r0, r1;
+                epi.pair_rows(pr0 + (j >> 1), r0, r1);
+                const int r = (j & 1) ? r1 : r0;
+                const uint32_t laddr = smem_u32(tile + r * ld + n);
+                float x[8];
 #pragma unroll
-            for (int sp = 0; sp < 16; ++sp)
-                x[sp] = sp < a.splits ? __ldcg(all4 + (size_t)sp * vec_per_split + t) : make_float4(0.f, 0.f, 0.f, 0.f);
-            float4 v = x[0];
+                for (int sp = 0; sp < 8; ++sp) {  // all peers' loads in flight together
+                    x[sp] = 0.f;
+                    if (sp < a.splits) {
+                        uint32_t raddr;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(sp));
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x[sp]) : "r"(raddr) : "memory");
+                    }
+                }
+                float v = x[0];
 #pragma unroll
-            for (int sp = 1; sp < 16; ++sp) { v.x += x[sp].x; v.y += x[sp].y; v.z += x[sp].z; v.w += x[sp].w; }
-            float *dst = tile + (t / vec_per_row) * ld + (t % vec_per_row) * 4;
-            dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+                for (int sp = 1; sp < 8; ++sp) v += x[sp];
+                fin[j * NP + n] = v;
+            }
         }
-        if (tid == 0) a.tickets[tile_idx] = 0;
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (good) {
+            for (int t = tid; t < nrows * NP; t += kTcThreads) {  // peers are done with my tile: put the sums in place
+                const int j = t / NP, n = t % NP;
+                int r0, r1;
+                epi.pair_rows(pr0 + (j >> 1), r0, r1);
+                tile[((j & 1) ? r1 : r0) * ld + n] = fin[j * NP + n];
+            }
+        }
         __syncthreads();
     }
-    epi.run(tile, ld, tile_idx, n_live, a.rows, tid, kTcThreads);
+    if (good) epi.run(tile, ld, tile_idx, n_live, a.rows, tid, kTcThreads, pr0, pr1);
 }
 
 inline size_t tc_smem_bytes(int n_pad, int n_stages) {
     const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)n_pad * kTcBK * 2;
-    const size_t pipe = (size_t)n_stages * stage, tile = sizeof(float) * (size_t)kTcBM * (n_pad + 1);
-    return 1024 + (pipe > tile ? pipe : tile) + sizeof(uint64_t) * (2 * n_stages + 1) + 64;
+    const size_t pipe = (size_t)n_stages * stage;  // the tile and the reduced slice reuse it (the host checks the fit)
+    return 1024 + pipe + sizeof(uint64_t) * (2 * n_stages + 1) + 64;
 }
 
 }  // namespace river

@@ -22,7 +22,6 @@ namespace {
 thread_local std::string g_init_error;
 
 constexpr int kStaging = 4;        // pinned metadata buffers in flight
-constexpr int kTcMaxCtas = 320;    // tiles x K-splits of a split-K projection (bounds the partial buffer)
 enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, kNumClasses };
 const char *const kClassNames[kNumClasses] = {"step_begin", "compact", "qkv_rope_kv", "attn_decode", "o_proj_resid",
                                               "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final"};
@@ -58,8 +57,6 @@ struct river_ctx {
     unsigned *attn_tickets, *tickets;  // [max_batch*Hkv], [4]
     // tensor-core path: operand buffers, split-K partials, tickets, tensor maps of every weight matrix
     __nv_bfloat16 *tc_xhi = nullptr, *tc_xlo = nullptr;
-    float *tc_partial = nullptr;
-    unsigned *tc_tickets = nullptr;
     int tc_max_pad = 0, tc_kmax = 0;
     bool tc_ok = false;
     struct LayerMaps { CUtensorMap q, k, v, o, g, u, d; };
@@ -169,15 +166,14 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
-    float *tpart = cv.take<float>((size_t)kTcMaxCtas * kTcBM * tc_pad);
-    unsigned *ttk = cv.take<unsigned>(2048);
+
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
         x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
-        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_partial = tpart; x->tc_tickets = ttk; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
+        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
 }
@@ -186,19 +182,35 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
 // stream is still running and orders itself with griddepcontrol.wait.  Every kernel launched this way calls
 // griddepcontrol.wait before it touches anything a predecessor writes.
 template <class... KArgs, class... Args>
-cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
-                     Args &&...args) {
+cudaError_t launch_kc(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                      int cluster_x, Args &&...args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (pdl) {
+        at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    if (cluster_x > 1) {  // consecutive CTAs along x form a thread-block cluster
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = cluster_x;
+        at[na].val.clusterDim.y = 1;
+        at[na].val.clusterDim.z = 1;
+        ++na;
+    }
     cfg.attrs = at;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
+}
+template <class... KArgs, class... Args>
+cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                     Args &&...args) {
+    return launch_kc(kern, grid, block, smem, st, pdl, 1, std::forward<Args>(args)...);
 }
 
 KvAddr kv_addr(const river_ctx *c, int layer0) {
@@ -369,7 +381,7 @@ bool make_map_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t ro
 // The shapes the tensor-core path takes: every output dimension in whole 128-feature tiles.
 bool tc_shape_ok(const river_config &g) {
     return g.d % 128 == 0 && (g.Hq * g.dh) % 128 == 0 && (g.Hkv * g.dh) % 128 == 0 && g.F % 64 == 0 && g.V % 128 == 0 &&
-           g.d % 64 == 0 && g.F % 64 == 0 && (g.Hq * g.dh) % 64 == 0 && g.V / 128 <= 2048;
+           g.d % 64 == 0 && g.F % 64 == 0 && (g.Hq * g.dh) % 64 == 0;
 }
 bool make_tc_maps(river_ctx *c) {
     const river_config &g = c->cfg;
@@ -400,8 +412,8 @@ const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
 int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots) {
     int best = 1;
     double best_eff = 0.0;
-    for (int s = 1; s <= 16; ++s) {
-        if (s > 1 && (kb_total / s < 4 || tiles * s > kTcMaxCtas)) break;
+    for (int s = 1; s <= 8; ++s) {  // a cluster holds at most 8 CTAs
+        if (s > 1 && kb_total / s < 4) break;
         const int ctas = tiles * s, waves = (ctas + slots - 1) / slots;
         const double eff = (double)ctas / ((double)waves * slots);
         if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
@@ -412,7 +424,7 @@ int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots) {
 template <class Epi>
 cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
                       int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                      const int32_t *cnt, const Epi &epi) {
+                      const int32_t *cnt, const Epi &epi, bool allow_split = true) {
     const int np = (n + 15) / 16 * 16;
     const river_ctx::BMap *bm = tc_bmap(c, K, np);
     if (!bm) return cudaErrorInvalidValue;
@@ -425,16 +437,20 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
     a.n_stages = (int)std::max<size_t>(2, std::min<size_t>(8, (106 * 1024) / stage));  // two CTAs per SM if possible
     const int occ = tc_smem_bytes(np, a.n_stages) <= 113 * 1024 ? 2 : 1;
     a.splits = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * occ);
+    // the finished tile plus the reduced slice of a split CTA live in the pipeline memory
+    const size_t tile_b = sizeof(float) * (size_t)kTcBM * (np + 1);
+    while (a.splits > 1 && tile_b + tile_b / a.splits + 4096 > (size_t)a.n_stages * stage) --a.splits;
+    if (!allow_split) a.splits = 1;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
-    a.rows = rows; a.cnt = cnt; a.partial = c->tc_partial; a.tickets = c->tc_tickets; a.dev_err = c->dev_err;
+    a.rows = rows; a.cnt = cnt; a.dev_err = c->dev_err;
     const size_t smem = tc_smem_bytes(np, a.n_stages);
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
         cudaFuncSetAttribute(tc_gemm_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_smem = smem;
     }
-    return launch_k(tc_gemm_kernel<Epi>, dim3(tiles * a.splits), dim3(kTcThreads), smem, c->stream, true, a0, a1, a2,
-                    bm->hi, bm->lo, a, epi);
+    return launch_kc(tc_gemm_kernel<Epi>, dim3(tiles * a.splits), dim3(kTcThreads), smem, c->stream, true, a.splits, a0,
+                     a1, a2, bm->hi, bm->lo, a, epi);
 }
 
 // 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
@@ -652,7 +668,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             n_parts = g.V / kTcBM;
             TcHeadEpi e{c->meta(), g.V, c->part_val, c->part_idx, n_parts};
             note(launch_tc(c, a.in, c->tc_map_head, c->tc_map_head, c->tc_map_head, d, n_parts, n_head, 0, 0, 0,
-                           c->head_rows(), c->meta_dev + 2 /* StepMeta::n_head_rows */, e));
+                           c->head_rows(), c->meta_dev + 2 /* StepMeta::n_head_rows */, e, false));
         } else {
             int n_sel = 1;
             while (n_sel < n_head && n_sel < 4) n_sel *= 2;
@@ -799,7 +815,6 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(c->tc_tickets, 0, sizeof(unsigned) * 2048, c->stream);
 
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_act, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_riv, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
