@@ -126,6 +126,11 @@ def draw_model(shape, device):
     return bb, rv
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (taken on a
+# 4-layer model of the same layer shape: kernel, geometry and operands per launch are those of the full model).
+NCU_TRAFFIC = {("8b", "gateup_swiglu"): 235.0e6}
+
+
 # ---------------------------------------------------------------------------------------------- CPU oracle timing
 def time_oracle(shape, bb_cpu, rv_cpu, B, ctx_len, n_steps, n_warm, seed):
     """Oracle decode steps at context ctx_len on the host cores.  The KV history is synthetic N(0,1) (an oracle
@@ -389,7 +394,8 @@ def ours(args, wl):
                            "frac_of_measured_peak": full_gbs / peak, "frac_of_8TBps": full_gbs / 8000.0},
             "early_exit_speedup_vs_full_depth": ms_full / ms,
             "roofline": {"bound": "hbm", "kernel": dom["name"], "achieved": ach, "peak": peak, "unit": "GB/s",
-                         "frac": ach / peak, "traffic": None, "peak_kind": peak_kind,
+                         "frac": ach / peak, "traffic": NCU_TRAFFIC.get((shape_name, dom["name"])),
+                         "peak_kind": peak_kind,
                          "launch_ms": per_launch_ms, "alg_bytes_per_launch": dom["alg_bytes_total"] / dom["launches"],
                          "pass": "full depth, events around every launch"},
             "kernels": kernels,
