@@ -260,7 +260,7 @@ def ours(args, wl):
     L = shape.L
     K, W = args.steps, args.warmup
     n_cal, n_prof, n_e2e = 8, 4, min(K, 64)
-    total_steps = n_cal + 2 * (W + K) + n_prof + (W + n_e2e) + 4
+    total_steps = n_cal + 2 * (W + K) + 2 * n_prof + (W + n_e2e) + 4
     bb, rvw = draw_model(shape, dev)
     lens = synth.prompt_lengths(WORKLOADS[wl][3] + 1000 * rank, B, plo, phi) if plo != phi else [plo] * B
     max_len = max(lens) + total_steps
@@ -353,27 +353,45 @@ def ours(args, wl):
     ms_e2e = dist_max((time.perf_counter() - t0) * 1e3)
     step += n_e2e
 
-    # ---- per-kernel timing pass (events around every launch; outside every timed region), full depth
-    rv.profile(True)
-    for t in range(step, step + n_prof):
-        rv.decode_step(slots, toks[t], inf[t], None, logits, nxt, exits[t], None, slots_c=slots_c)
-    step += n_prof
-    prof = rv.profile_read()
-    rv.profile(False)
+    # ---- per-kernel timing passes (outside every timed region): events around every launch; for the persistent
+    # chain kernel additionally its phases as CTA 0 saw them on the global timer.  Full depth, then scheduled exits.
+    def profile_pass(thresholds):
+        nonlocal step
+        rv.profile(True)
+        for t in range(step, step + n_prof):
+            rv.decode_step(slots, toks[t], thresholds[t], None, logits, nxt, exits[t], None, slots_c=slots_c)
+        step += n_prof
+        out = rv.profile_read()
+        rv.profile(False)
+        return out
+    prof = profile_pass(inf)
+    prof_exit = profile_pass(taus)
     st = rv.stats()
 
     peak, peak_kind = peaks()
     tok_s = world * B * K / (ms / 1e3)
     line = None
     if rank == 0:
-        dom = max(prof, key=lambda r: r["ms_total"])
+        def table(pr):
+            chain = any(r["name"] == "decode_chain" for r in pr)
+            phase_names = ("qkv_rope_kv", "attn_decode", "o_proj_resid", "gateup_swiglu", "down_resid", "exit_score", "lm_head")
+            launches_k = [r for r in pr if not (chain and r["name"] in phase_names)]
+            tot = sum(r["ms_total"] for r in launches_k)
+            row = lambda r, den: {"launches_per_step": r["launches"] // n_prof, "ms_per_step": round(r["ms_total"] / n_prof, 4),
+                                  "share": round(r["ms_total"] / den, 4),
+                                  "GBps": round(r["alg_bytes_total"] / max(r["ms_total"], 1e-9) / 1e6, 1)}
+            out = {r["name"]: row(r, tot) for r in launches_k}
+            if chain:
+                ph = [r for r in pr if r["name"] in phase_names]
+                tot_ph = sum(r["ms_total"] for r in ph)
+                out["decode_chain"]["phases"] = {r["name"]: row(r, tot_ph) for r in ph}
+            return out
+        names = {r["name"]: r for r in prof}
+        dom = names["decode_chain"] if "decode_chain" in names else max(prof, key=lambda r: r["ms_total"])
         per_launch_ms = dom["ms_total"] / dom["launches"]
         ach = dom["alg_bytes_total"] / dom["launches"] / (per_launch_ms * 1e-3) / 1e9
-        tot_ms = sum(r["ms_total"] for r in prof)
-        kernels = {r["name"]: {"launches_per_step": r["launches"] // n_prof,
-                               "ms_per_step": round(r["ms_total"] / n_prof, 4),
-                               "share": round(r["ms_total"] / tot_ms, 4),
-                               "GBps": round(r["alg_bytes_total"] / max(r["ms_total"], 1e-9) / 1e6, 1)} for r in prof}
+        kernels = table(prof)
+        kernels_exit = table(prof_exit)
         step_gbs = bytes_exit / (ms / K * 1e-3) / 1e9
         full_gbs = bytes_full / (ms_full / K * 1e-3) / 1e9
         line = {
@@ -399,6 +417,7 @@ def ours(args, wl):
                          "launch_ms": per_launch_ms, "alg_bytes_per_launch": dom["alg_bytes_total"] / dom["launches"],
                          "pass": "full depth, events around every launch"},
             "kernels": kernels,
+            "kernels_exit_run": kernels_exit,
             "e2e": {"value": world * B * n_e2e / (ms_e2e / 1e3), "unit": "tokens/s", "steps": n_e2e,
                     "h2d_bytes_per_step": B * 8, "d2h_bytes_per_step": B * (4 * shape.V + 8)},
             "gpu_launches": int(launches),

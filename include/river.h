@@ -47,7 +47,10 @@ enum { RIVER_EXIT_PER_TOKEN = 0, RIVER_EXIT_BATCH_MIN = 1 };
 enum {
     RIVER_F_GRAPH = 1,   /* replay each decode step as a CUDA graph (captured on first use) */
     RIVER_F_NO_TC = 2,   /* run every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
-    RIVER_F_SIMPLE_ATTN = 4  /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
+    RIVER_F_SIMPLE_ATTN = 4, /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
+    RIVER_F_NO_CHAIN = 8     /* steps of 1-4 rows as separate kernels per stage instead of the persistent chain kernel */
+    /* bits 8-15: tuning aid for the chain kernel, KiB of the next phase's weights each warp requests from the L2
+       ahead of time (0 = default 4) */
 };
 
 typedef struct river_config {

@@ -1,0 +1,858 @@
+// One persistent kernel for the layer chain of a small-batch decode step (rows <= 4, sm_100a).
+//
+// At one to four rows every projection is a weight stream and what a step costs beyond the weight bytes is the chain
+// of dependent launches: QKV -> attention -> O -> gate/up -> down -> exit score, 32 times.  This kernel runs the whole
+// chain, and the LM head, as phases of ONE cooperative launch with one CTA per SM:
+//   * phases are separated by a grid barrier (arrive counter in global memory, bounded spin);
+//   * a phase splits its weight rows evenly over the CTAs and, inside a CTA, splits (row pair, K slice) units evenly
+//     over the warps, so every warp streams the same number of bytes whatever the projection's shape; the partial
+//     dot products of a row pair meet in shared memory in a fixed order (deterministic);
+//   * a warp that has finished its share of a phase asks the L2 for the first weights it will need in the NEXT phase
+//     (cp.async.bulk.prefetch.L2), so HBM keeps streaming through phase tails, barriers, the attention phase and the
+//     activation staging of the next phase;
+//   * attention (split over KV positions, merged by the last-arriving CTA of a head), the Eq. 1 score, the exit
+//     decision and the row lists are computed in-kernel; the decision is taken redundantly and identically by every
+//     CTA, so no extra barrier is needed for it.
+// Rows still in the backbone use the bf16 weights, rows that left it the 4-bit exit-layer copy (Section 4.1); both
+// write K/V to the same cache slots.
+#pragma once
+#include "gemv_stream.cuh"
+
+namespace river {
+
+struct LayerDev {  // device-resident copy of one block's weight pointers
+    const uint16_t *attn_norm, *ffn_norm, *wq, *wk, *wv, *wo, *wg, *wu, *wd;
+    W4 rq, rk, rv, ro, rg, ru, rd;
+    int32_t has_river, pad;
+};
+
+struct ChainArgs {
+    const StepMeta *meta;
+    const LayerDev *layers;
+    int L, d, Hq, Hkv, dh, F, V, group, entry_layer, exit_mode;
+    float eps, qscale;  // qscale = log2(e) / sqrt(dh)
+    float *h[3], *qbuf, *obuf, *act;
+    const float2 *rope_cs;
+    KvAddr kv;  // layer0 is set per layer
+    float *part_o;      // [row][Hq][splits][dh]
+    float2 *part_ml;    // [row][Hq][splits]
+    unsigned *attn_tickets;  // [row][Hkv], zero between steps
+    uint8_t *exited;    // [max_batch] in: state after the step prologue; out: final state
+    Lists lists;
+    const uint16_t *lm_head, *final_norm;
+    const int32_t *head_rows;
+    float *part_val;    // [row][gridDim.x]
+    int32_t *part_idx;
+    unsigned *bar;      // arrive counter, zero at launch
+    int *dev_err;
+    unsigned long long *stamps;  // optional [2 + 6 L]: globaltimer at the phase boundaries seen by CTA 0
+    unsigned long long *sub;     // optional [5][8]: time CTA 0 spent staging / streaming / finishing / waiting, per phase kind
+    int part_cap;       // partial slots per warp
+    int pf_bytes;       // bytes of the next phase each warp asks the L2 for
+    int xs_floats;      // capacity of the activation staging area
+};
+
+constexpr int kChainThreads = 512;
+constexpr int kChainWarps = kChainThreads / 32;
+constexpr int kChainR = 2;           // weight rows per task
+constexpr unsigned kChainSpinLimit = 1u << 20;
+
+__device__ __forceinline__ unsigned long long chain_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Ask the L2 to fetch [p, p + bytes) (never a byte outside the range; 16-byte granules).
+__device__ __forceinline__ void l2_prefetch(const void *p, size_t bytes) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p);
+    uintptr_t a0 = (a + 15) & ~(uintptr_t)15;
+    if (a0 - a >= bytes) return;
+    size_t n = (bytes - (a0 - a)) & ~(size_t)15;
+    while (n) {
+        const uint32_t c = n > 32768 ? 32768u : (uint32_t)n;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a0), "r"(c) : "memory");
+        a0 += c;
+        n -= c;
+    }
+}
+
+// Optional timing probe of CTA 0 / thread 0: time since the previous mark is added to acc[k] (profiling runs only).
+struct ChainProbe {
+    unsigned long long *acc;
+    unsigned long long last;
+    __device__ __forceinline__ void mark(int k) {
+        if (acc) {
+            const unsigned long long t = chain_now();
+            acc[k] += t - last;
+            last = t;
+        }
+    }
+};
+
+// ---------------------------------------------------------------- grid barrier
+// Every CTA arrives once per barrier on a counter that only grows during the launch.  The wait is bounded: a CTA
+// that gives up flags DEV_WAIT_TIMEOUT, and every other CTA leaves as soon as it sees the flag.
+__device__ __forceinline__ bool chain_grid_sync(unsigned *bar, unsigned &target, int *dev_err, int *s_dead) {
+    target += gridDim.x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(bar, 1u);
+        unsigned it = 0;
+        for (;;) {
+            unsigned v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
+            if ((int)(v - target) >= 0) break;
+            ++it;
+            if (it > kChainSpinLimit) {
+                atomicExch(dev_err, DEV_WAIT_TIMEOUT);
+                *s_dead = 1;
+                break;
+            }
+            if ((it & 63u) == 0 && *reinterpret_cast<volatile int *>(dev_err) == DEV_WAIT_TIMEOUT) {
+                *s_dead = 1;
+                break;
+            }
+        }
+        __threadfence();
+    }
+    __syncthreads();
+    return *s_dead == 0;
+}
+
+// ---------------------------------------------------------------- the share of a phase a CTA / warp owns
+struct ChainShare {
+    int t0, T;        // first task and task count of this CTA
+    int nsl;          // K slices per task
+    int units;        // T * nsl
+    __device__ __forceinline__ int bound(int w) const { return (int)(((long long)units * w) / kChainWarps); }
+};
+__device__ __forceinline__ ChainShare chain_share(int tasks, int nit, int its_per_slice) {
+    ChainShare s;
+    s.t0 = (int)(((long long)tasks * blockIdx.x) / gridDim.x);
+    s.T = (int)(((long long)tasks * (blockIdx.x + 1)) / gridDim.x) - s.t0;
+    s.nsl = max(1, (nit + its_per_slice - 1) / its_per_slice);
+    s.units = s.T * s.nsl;
+    return s;
+}
+
+// ---------------------------------------------------------------- units: bf16 weights
+constexpr int kBfIts = 4;  // 32-lane x 16-byte iterations per slice (1024 inputs)
+
+template <int N, int R>
+__device__ __forceinline__ void chain_fma_bf16(const uint4 (&w)[R][kBfIts], const float *xs, int xstride, int it0, int nch,
+                                               int lane, float (&acc)[R][N]) {
+#pragma unroll
+    for (int u = 0; u < kBfIts; ++u) {
+        const int c = (it0 + u) * 32 + lane;
+        if (c < nch) {
+            const float *xb = xs + (c >> 5) * 256 + lane * 4;
+#pragma unroll
+            for (int n = 0; n < N; ++n) {
+                const float4 x0 = *reinterpret_cast<const float4 *>(xb + n * xstride);
+                const float4 x1 = *reinterpret_cast<const float4 *>(xb + n * xstride + 128);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const uint4 v = w[r][u];
+                    float a0 = bf16lo(v.x) * x0.x, a1 = bf16hi(v.x) * x0.y;
+                    a0 = fmaf(bf16lo(v.y), x0.z, a0); a1 = fmaf(bf16hi(v.y), x0.w, a1);
+                    a0 = fmaf(bf16lo(v.z), x1.x, a0); a1 = fmaf(bf16hi(v.z), x1.y, a1);
+                    a0 = fmaf(bf16lo(v.w), x1.z, a0); a1 = fmaf(bf16hi(v.w), x1.w, a1);
+                    acc[r][n] += a0 + a1;
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- units: 4-bit weights
+constexpr int kW4Its = 2;  // 32-lane x 16-byte iterations per slice (2048 inputs)
+
+struct W4Regs {
+    uint4 q;
+    float s, zz;
+};
+
+template <int R>
+__device__ __forceinline__ void chain_issue_w4(const W4 (&wrow)[R], int nch, int gshift, int it0, int lane,
+                                               W4Regs (&w)[R][kW4Its]) {
+#pragma unroll
+    for (int u = 0; u < kW4Its; ++u) {
+        const int c = (it0 + u) * 32 + lane;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (c < nch) {
+                w[r][u].q = ldg_stream16(wrow[r].codes + (size_t)c * 16);
+                w[r][u].s = bf16f(ldg_u16(wrow[r].scale + (c >> gshift)));
+                w[r][u].zz = bf16f(ldg_u16(wrow[r].zero + (c >> gshift))) + 128.f;
+            } else {
+                w[r][u].q = make_uint4(0u, 0u, 0u, 0u);
+                w[r][u].s = 0.f;
+                w[r][u].zz = 0.f;
+            }
+        }
+    }
+}
+
+// sum_k (q_k - z) s x_k over a 32-input chunk = s * (sum_k (128 + q_k) x_k - (z + 128) * sum_k x_k); 128 + q is the
+// bf16 bit pattern 0x4300 | q, the chunk sums of x are precomputed while staging.
+template <int N, int R>
+__device__ __forceinline__ void chain_fma_w4(const W4Regs (&w)[R][kW4Its], const float *xs, const float *xsum, int xstride,
+                                             int it0, int nch, int lane, float (&acc)[R][N]) {
+#pragma unroll
+    for (int u = 0; u < kW4Its; ++u) {
+        const int c = (it0 + u) * 32 + lane;
+        if (c < nch) {
+#pragma unroll
+            for (int n = 0; n < N; ++n) {
+                const float *xb = xs + n * xstride + (c >> 5) * 1024 + lane * 4;
+                float p0[R], p1[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) { p0[r] = 0.f; p1[r] = 0.f; }
+#pragma unroll
+                for (int wd = 0; wd < 4; ++wd) {
+                    const float4 x0 = *reinterpret_cast<const float4 *>(xb + (2 * wd) * 128);
+                    const float4 x1 = *reinterpret_cast<const float4 *>(xb + (2 * wd + 1) * 128);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const uint4 q = w[r][u].q;
+                        const uint32_t v = wd == 0 ? q.x : (wd == 1 ? q.y : (wd == 2 ? q.z : q.w));
+                        const uint32_t b0 = (v & 0x000f000fu) | 0x43004300u;
+                        const uint32_t b1 = ((v >> 4) & 0x000f000fu) | 0x43004300u;
+                        const uint32_t b2 = ((v >> 8) & 0x000f000fu) | 0x43004300u;
+                        const uint32_t b3 = ((v >> 12) & 0x000f000fu) | 0x43004300u;
+                        p0[r] = fmaf(bf16lo(b0), x0.x, p0[r]); p1[r] = fmaf(bf16lo(b1), x0.y, p1[r]);
+                        p0[r] = fmaf(bf16lo(b2), x0.z, p0[r]); p1[r] = fmaf(bf16lo(b3), x0.w, p1[r]);
+                        p0[r] = fmaf(bf16hi(b0), x1.x, p0[r]); p1[r] = fmaf(bf16hi(b1), x1.y, p1[r]);
+                        p0[r] = fmaf(bf16hi(b2), x1.z, p0[r]); p1[r] = fmaf(bf16hi(b3), x1.w, p1[r]);
+                    }
+                }
+                const float sx = xsum[n * nch + c];
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r][n] = fmaf(w[r][u].s, (p0[r] + p1[r]) - w[r][u].zz * sx, acc[r][n]);
+            }
+        }
+    }
+}
+
+template <class P, int R>
+__device__ __forceinline__ void chain_rows_w4(const P &p, int t, W4 (&rows)[R]) {
+    const int K = p.K, ng = K / p.group;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int run = r / (R / P::NRUN), j = r % (R / P::NRUN);
+        const W4 b = p.template w4_base<R>(t, run);
+        const size_t row = p.template run_row<R>(t, run) + j;
+        rows[r] = W4{b.codes + row * (size_t)(K >> 1), b.scale + row * (size_t)ng, b.zero + row * (size_t)ng};
+    }
+}
+
+// ---------------------------------------------------------------- L2 prefetch of a warp's first units of a phase
+template <class P, int R>
+__device__ __forceinline__ void chain_prefetch(const P &p, bool want_bf16, bool want_w4, int pf_bytes) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int K = p.K;
+    const int tasks = p.template n_tasks<R>();
+    if (want_bf16) {
+        const int nch = K >> 3;
+        const ChainShare sh = chain_share(tasks, (nch + 31) >> 5, kBfIts);
+        const int u0 = sh.bound(warp), u1 = sh.bound(warp + 1);
+        const int per = kBfIts * 32 * 8;  // inputs per slice
+        const int npu = max(1, min(32 / R, pf_bytes / (R * per * 2)));
+        const int u = u0 + lane / R, r = lane % R;
+        if (lane < npu * R && u < u1) {
+            const int t = sh.t0 + u / sh.nsl, s = u % sh.nsl;
+            const int run = r / (R / P::NRUN), j = r % (R / P::NRUN);
+            const uint16_t *row = p.template bf16_base<R>(t, run) + (p.template run_row<R>(t, run) + j) * (size_t)K;
+            const int k0 = s * per;
+            if (k0 < K) l2_prefetch(row + k0, (size_t)min(per, K - k0) * 2);
+        }
+    }
+    if (want_w4) {
+        const int nch = K >> 5;
+        const ChainShare sh = chain_share(tasks, (nch + 31) >> 5, kW4Its);
+        const int u0 = sh.bound(warp), u1 = sh.bound(warp + 1);
+        const int per = kW4Its * 32 * 32;
+        const int npu = max(1, min(32 / R, pf_bytes / (R * (per / 2 + 4 * per / p.group))));
+        const int u = u0 + lane / R, r = lane % R;
+        if (lane < npu * R && u < u1) {
+            const int t = sh.t0 + u / sh.nsl, s = u % sh.nsl;
+            W4 rows[R];
+            chain_rows_w4<P, R>(p, t, rows);
+            const int k0 = s * per;
+            if (k0 < K) {
+                const int len = min(per, K - k0);
+                l2_prefetch(rows[r].codes + (k0 >> 1), (size_t)len >> 1);
+                l2_prefetch(rows[r].scale + k0 / p.group, (size_t)(len / p.group) * 2);
+                l2_prefetch(rows[r].zero + k0 / p.group, (size_t)(len / p.group) * 2);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- one pass of a phase over staged activation rows
+// Every warp streams its units, partial sums of a task meet in `part`, then the CTA's threads finish the tasks:
+// epi(task, n, res[R]) gets the R dot products of activation row n of the pass.
+template <class P, int N, int R, bool W4M, class PF, class EP>
+__device__ __forceinline__ void chain_stream(const P &p, const float *xs, const float *xsum, int xstride, float *part,
+                                             int part_cap, int *dev_err, bool do_pf, PF &&prefetch_next, EP &&epi,
+                                             ChainProbe &probe, int pk) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int K = p.K;
+    const int nch = W4M ? (K >> 5) : (K >> 3);
+    constexpr int ITS = W4M ? kW4Its : kBfIts;
+    const ChainShare sh = chain_share(p.template n_tasks<R>(), (nch + 31) >> 5, ITS);
+    const int u0 = sh.bound(warp), u1 = sh.bound(warp + 1);
+    const int tf = u0 / sh.nsl;
+    float acc[R][N];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
+
+    auto flush = [&](int t) {
+        const int j = t - tf;
+        float *dst = part + (size_t)(warp * part_cap + j) * (R * N);
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int n = 0; n < N; ++n) {
+                const float v = warp_sum(acc[r][n]);
+                if (lane == 0 && j < part_cap) dst[r * N + n] = v;
+                acc[r][n] = 0.f;
+            }
+        if (lane == 0 && j >= part_cap) atomicExch(dev_err, DEV_INTERNAL);
+    };
+
+    if (u0 < u1) {
+        int t = tf, s = u0 - tf * sh.nsl;
+        if constexpr (!W4M) {
+            uint4 wn[R][kBfIts];
+            {
+                const uint16_t *rows[R];
+                stream_rows_bf16<P, N, R>(p, sh.t0 + t, rows);
+                stream_issue_bf16<R>(rows, nch, s * ITS, lane, wn);
+            }
+            for (int u = u0; u < u1; ++u) {
+                uint4 wc[R][kBfIts];
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int i = 0; i < kBfIts; ++i) wc[r][i] = wn[r][i];
+                int tn = t, sn = s + 1;
+                if (sn == sh.nsl) { sn = 0; ++tn; }
+                if (u + 1 < u1) {
+                    const uint16_t *rows[R];
+                    stream_rows_bf16<P, N, R>(p, sh.t0 + tn, rows);
+                    stream_issue_bf16<R>(rows, nch, sn * ITS, lane, wn);
+                }
+                chain_fma_bf16<N, R>(wc, xs, xstride, s * ITS, nch, lane, acc);
+                if (u + 1 == u1 || tn != t) flush(t);
+                t = tn; s = sn;
+            }
+        } else {
+            const int gshift = (p.group == 64) ? 1 : (p.group == 32 ? 0 : 2);
+            W4Regs wn[R][kW4Its];
+            {
+                W4 rows[R];
+                chain_rows_w4<P, R>(p, sh.t0 + t, rows);
+                chain_issue_w4<R>(rows, nch, gshift, s * ITS, lane, wn);
+            }
+            for (int u = u0; u < u1; ++u) {
+                W4Regs wc[R][kW4Its];
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int i = 0; i < kW4Its; ++i) wc[r][i] = wn[r][i];
+                int tn = t, sn = s + 1;
+                if (sn == sh.nsl) { sn = 0; ++tn; }
+                if (u + 1 < u1) {
+                    W4 rows[R];
+                    chain_rows_w4<P, R>(p, sh.t0 + tn, rows);
+                    chain_issue_w4<R>(rows, nch, gshift, sn * ITS, lane, wn);
+                }
+                chain_fma_w4<N, R>(wc, xs, xsum, xstride, s * ITS, nch, lane, acc);
+                if (u + 1 == u1 || tn != t) flush(t);
+                t = tn; s = sn;
+            }
+        }
+    }
+    probe.mark(pk + 1);
+    if (do_pf) prefetch_next();
+    __syncthreads();
+    for (int e = threadIdx.x; e < sh.T * N; e += blockDim.x) {
+        const int tl = e / N, n = e - tl * N;
+        float res[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) res[r] = 0.f;
+        const int ua = tl * sh.nsl, ub = ua + sh.nsl - 1;
+        for (int w = 0; w < kChainWarps; ++w) {  // fixed order: deterministic sums
+            const int b0 = sh.bound(w), b1 = sh.bound(w + 1);
+            if (b1 > b0 && b0 <= ub && b1 > ua) {
+                const int j = tl - b0 / sh.nsl;
+                if (j < part_cap) {
+                    const float *src = part + (size_t)(w * part_cap + j) * (R * N);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) res[r] += src[r * N + n];
+                }
+            }
+        }
+        epi(sh.t0 + tl, n, res);
+    }
+    __syncthreads();
+    probe.mark(pk + 2);
+}
+
+struct ChainSmem {
+    float *red, *xsum, *part, *xs;
+};
+
+// A projection phase: the rows still in the backbone against the bf16 weights, then the rows in the exit layers
+// against the 4-bit copy, N rows per pass.
+template <class P, int N, class PF>
+__device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, const ProjIn &in, const int *s_act, int na,
+                                              const int *s_riv, int nr, const ChainSmem &sm, PF &&prefetch_next,
+                                              ChainProbe &probe, int pk) {
+    constexpr int R = kChainR;
+    const int K = p.K;
+    const int xstride = xs_stride(K, 32);
+    const int passes_a = (na + N - 1) / N, passes_r = (nr + N - 1) / N;
+    for (int ps = 0; ps < passes_a; ++ps) {
+        const int i0 = ps * N;
+        stream_load_rows<N, 8>(in, s_act, i0, na, K, xstride, sm.xs, sm.xsum, sm.red);
+        probe.mark(pk);
+        chain_stream<P, N, R, false>(p, sm.xs, sm.xsum, xstride, sm.part, a.part_cap, a.dev_err,
+                                     ps + 1 == passes_a && passes_r == 0, prefetch_next,
+                                     [&](int t, int n, const float(&res)[R]) {
+                                         if (i0 + n < na) p.template epilogue<R>(t, s_act[i0 + n], res);
+                                     }, probe, pk);
+    }
+    for (int ps = 0; ps < passes_r; ++ps) {
+        const int i0 = ps * N;
+        stream_load_rows<N, 32>(in, s_riv, i0, nr, K, xstride, sm.xs, sm.xsum, sm.red);
+        probe.mark(pk + 4);
+        chain_stream<P, N, R, true>(p, sm.xs, sm.xsum, xstride, sm.part, a.part_cap, a.dev_err, ps + 1 == passes_r,
+                                    prefetch_next, [&](int t, int n, const float(&res)[R]) {
+                                        if (i0 + n < nr) p.template epilogue<R>(t, s_riv[i0 + n], res);
+                                    }, probe, pk + 4);
+    }
+    if (passes_a + passes_r == 0) prefetch_next();
+}
+
+// ---------------------------------------------------------------- a3 inside the chain: split-KV decode attention
+// Work item = (row, kv head, split of the positions).  A warp takes four consecutive positions of one page at a
+// time (a lane owns DH/32 head dims of K and V), keeps a base-2 online softmax per query head of the group, the
+// warps of the CTA merge through shared memory and the CTA writes one partial per item; the last CTA of a (row, kv
+// head) to arrive merges the splits in split order (deterministic) and writes the attention output.
+struct ChainFlags {
+    int exited[4], act[4], riv[4], pass[4];
+    int na, nr, dead, flag;
+};
+
+__device__ __forceinline__ float chain_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int DH, int GQ>
+__device__ __forceinline__ void chain_attention(const ChainArgs &a, const KvAddr &kv, int n_rows, int S, int chunk,
+                                                float *sm, ChainFlags *fl) {
+    constexpr int VE = DH / 32, U = 4, NW = kChainWarps;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float *s_m = sm, *s_l = sm + NW * GQ, *s_acc = sm + 2 * NW * GQ;  // [NW][GQ], [NW][GQ], [NW][GQ][DH]
+    const int items = n_rows * a.Hkv * S;
+    const int Hq = a.Hq;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int sp = item % S, kvh = (item / S) % a.Hkv, row = item / (S * a.Hkv);
+        const int pos = kv.row_pos[row], slot = kv.row_slot[row];
+        const int p0 = sp * chunk, p1 = min(pos + 1, p0 + chunk);
+        float qr[GQ][VE], acc[GQ][VE], m[GQ], l[GQ];
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            m[g] = -CUDART_INF_F;
+            l[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < VE; ++e) {
+                qr[g][e] = __ldcg(a.qbuf + (size_t)row * Hq * DH + (size_t)(kvh * GQ + g) * DH + lane * VE + e) * a.qscale;
+                acc[g][e] = 0.f;
+            }
+        }
+        const int32_t *pt = kv.page_tbl + (size_t)slot * kv.max_pages_per_seq;
+        for (int pb = p0 + warp * U; pb < p1; pb += NW * U) {  // pb is a multiple of 4: one page per batch
+            int page = pt[pb / kPage];
+            if (page < 0 || page >= kv.n_pages) {
+                if (lane == 0) atomicExch(a.dev_err, DEV_BAD_PAGE);
+                page = 0;
+            }
+            float kf[U][VE], vf[U][VE];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int p = pb + u;
+                if (p < p1) {
+                    const __nv_bfloat16 *kp = kv.pool + kv.base(page, 0, kvh, p % kPage) + lane * VE;
+                    const __nv_bfloat16 *vp = kv.pool + kv.base(page, 1, kvh, p % kPage) + lane * VE;
+                    if constexpr (VE == 4) {
+                        const uint2 kr = __ldcg(reinterpret_cast<const uint2 *>(kp));
+                        const uint2 vr = __ldcg(reinterpret_cast<const uint2 *>(vp));
+                        kf[u][0] = bf16lo(kr.x); kf[u][1] = bf16hi(kr.x); kf[u][2] = bf16lo(kr.y); kf[u][3] = bf16hi(kr.y);
+                        vf[u][0] = bf16lo(vr.x); vf[u][1] = bf16hi(vr.x); vf[u][2] = bf16lo(vr.y); vf[u][3] = bf16hi(vr.y);
+                    } else {
+                        const uint32_t kr = __ldcg(reinterpret_cast<const uint32_t *>(kp));
+                        const uint32_t vr = __ldcg(reinterpret_cast<const uint32_t *>(vp));
+                        kf[u][0] = bf16lo(kr); kf[u][1] = bf16hi(kr);
+                        vf[u][0] = bf16lo(vr); vf[u][1] = bf16hi(vr);
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) { kf[u][e] = 0.f; vf[u][e] = 0.f; }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (pb + u < p1) {  // warp-uniform
+#pragma unroll
+                    for (int g = 0; g < GQ; ++g) {
+                        float s = 0.f;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) s = fmaf(qr[g][e], kf[u][e], s);
+                        s = warp_sum(s);
+                        const float mn = fmaxf(m[g], s);
+                        const float corr = chain_ex2(m[g] - mn), pr = chain_ex2(s - mn);
+                        l[g] = l[g] * corr + pr;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) acc[g][e] = fmaf(pr, vf[u][e], acc[g][e] * corr);
+                        m[g] = mn;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+            if (lane == 0) { s_m[warp * GQ + g] = m[g]; s_l[warp * GQ + g] = l[g]; }
+#pragma unroll
+            for (int e = 0; e < VE; ++e) s_acc[(warp * GQ + g) * DH + lane * VE + e] = acc[g][e];
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < GQ * DH; t += blockDim.x) {
+            const int g = t / DH, e = t % DH;
+            float M = -CUDART_INF_F;
+            for (int w = 0; w < NW; ++w) M = fmaxf(M, s_m[w * GQ + g]);
+            float num = 0.f, den = 0.f;
+            for (int w = 0; w < NW; ++w) {
+                const float mw = s_m[w * GQ + g];
+                const float c = (mw == -CUDART_INF_F) ? 0.f : chain_ex2(mw - M);
+                num = fmaf(c, s_acc[(w * GQ + g) * DH + e], num);
+                den = fmaf(c, s_l[w * GQ + g], den);
+            }
+            const int head = kvh * GQ + g;
+            if (S == 1) {
+                a.obuf[(size_t)row * Hq * DH + (size_t)head * DH + e] = num / den;
+            } else {
+                const size_t pi = ((size_t)row * Hq + head) * S + sp;
+                a.part_o[pi * DH + e] = num;
+                if (e == 0) a.part_ml[pi] = make_float2(M, den);
+            }
+        }
+        if (S > 1) {
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const unsigned tk = atomicAdd(a.attn_tickets + row * a.Hkv + kvh, 1u);
+                fl->flag = (tk == (unsigned)(S - 1));
+            }
+            __syncthreads();
+            if (fl->flag) {
+                __threadfence();
+                // (max, sum) of every (head, split) into shared memory, then every thread owns one (head, dim) and
+                // pulls the splits' partial outputs in batches of independent loads
+                float *s_mx = s_acc, *s_sm = s_acc + GQ * 64;
+                for (int t = threadIdx.x; t < GQ * S; t += blockDim.x) {
+                    const int g = t / S, s2 = t % S;
+                    const float2 ml = __ldcg(&a.part_ml[((size_t)row * Hq + kvh * GQ + g) * S + s2]);
+                    s_mx[g * 64 + s2] = ml.x;
+                    s_sm[g * 64 + s2] = ml.y;
+                }
+                __syncthreads();
+                for (int t = threadIdx.x; t < GQ * DH; t += blockDim.x) {
+                    const int g = t / DH, e = t % DH;
+                    const float *po = a.part_o + ((size_t)row * Hq + kvh * GQ + g) * S * DH + e;
+                    float M = -CUDART_INF_F;
+                    for (int s2 = 0; s2 < S; ++s2) M = fmaxf(M, s_mx[g * 64 + s2]);
+                    float num = 0.f, den = 0.f;
+                    for (int s0 = 0; s0 < S; s0 += 8) {
+                        float v[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) v[k] = (s0 + k < S) ? __ldcg(po + (size_t)(s0 + k) * DH) : 0.f;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            if (s0 + k < S) {
+                                const float mx = s_mx[g * 64 + s0 + k];
+                                const float c = (mx == -CUDART_INF_F) ? 0.f : chain_ex2(mx - M);
+                                num = fmaf(c, v[k], num);
+                                den = fmaf(c, s_sm[g * 64 + s0 + k], den);
+                            }
+                    }
+                    a.obuf[(size_t)row * Hq * DH + (size_t)(kvh * GQ + g) * DH + e] = num / den;
+                }
+                if (threadIdx.x == 0) a.attn_tickets[row * a.Hkv + kvh] = 0u;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------- a6 + a7 inside the chain
+// Eq. 1 for every row still in the backbone, the exit decision and the row lists entering block l + 1.  Every CTA
+// runs this on the same inputs with the same reduction order, so all CTAs hold identical lists; CTA 0 publishes
+// them (and the scores / exit layers) to global memory for the host-side queries.
+__device__ __forceinline__ void chain_decide(const ChainArgs &a, int l, const float *h_in, const float *h_out, int n,
+                                             float *red, ChainFlags *fl) {
+    const int L = a.L, d = a.d;
+    const bool eligible = (l >= 1) && (l >= a.entry_layer) && (l < L);
+    float *scores = a.meta->scores;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int row = 0; row < n; ++row) {
+        if (fl->exited[row] != 0 || !(eligible || scores)) continue;  // uniform across the CTA
+        const float4 *x = reinterpret_cast<const float4 *>(h_in + (size_t)row * d);
+        const float4 *y = reinterpret_cast<const float4 *>(h_out + (size_t)row * d);
+        float ab = 0.f, aa = 0.f, bb = 0.f;
+        for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+            const float4 u = __ldcg(x + i), v = __ldcg(y + i);
+            ab += u.x * v.x + u.y * v.y + u.z * v.z + u.w * v.w;
+            aa += u.x * u.x + u.y * u.y + u.z * u.z + u.w * u.w;
+            bb += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+        ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
+        __syncthreads();
+        if (lane == 0) { red[warp] = ab; red[32 + warp] = aa; red[64 + warp] = bb; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            ab = aa = bb = 0.f;
+            for (int w = 0; w < kChainWarps; ++w) { ab += red[w]; aa += red[32 + w]; bb += red[64 + w]; }
+            float s = 0.f;
+            if (aa > 0.f && bb > 0.f) s = ab / (sqrtf(aa) * sqrtf(bb));
+            fl->pass[row] = (s > a.meta->tau[row]) ? 1 : 0;
+            if (scores && blockIdx.x == 0) scores[(size_t)row * L + (l - 1)] = s;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int32_t *forced = a.meta->forced;
+        int allpass = 1;
+        if (a.exit_mode == 1)
+            for (int b = 0; b < n; ++b)
+                if (fl->exited[b] == 0 && !(eligible && fl->pass[b])) allpass = 0;
+        int na = 0, nr = 0;
+        for (int b = 0; b < n; ++b) {
+            if (fl->exited[b] == 0) {
+                bool leave = eligible && (a.exit_mode == 1 ? (allpass != 0) : (fl->pass[b] != 0));
+                const int f = forced ? forced[b] : -1;
+                if (f >= 0) leave = (f == l) && (l < L);
+                if (leave) {
+                    fl->exited[b] = 1;
+                    if (blockIdx.x == 0) { a.meta->exit_layer[b] = l; a.exited[b] = 1; }
+                }
+            }
+            if (fl->exited[b] == 0) fl->act[na++] = b;
+            else fl->riv[nr++] = b;
+        }
+        fl->na = na;
+        fl->nr = nr;
+        if (blockIdx.x == 0) {
+            int32_t *A = a.lists.act_idx + (size_t)l * a.lists.max_batch, *R = a.lists.riv_idx + (size_t)l * a.lists.max_batch;
+            for (int i = 0; i < na; ++i) A[i] = fl->act[i];
+            for (int i = 0; i < nr; ++i) R[i] = fl->riv[i];
+            a.lists.n_act[l] = na;
+            a.lists.n_riv[l] = nr;
+        }
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------- a8 inside the chain: LM head as a stream problem
+struct HeadProblem {
+    static constexpr int NRUN = 1;
+    const uint16_t *w;
+    int K, V, group;
+    template <int R> __device__ int n_tasks() const { return V / R; }
+    template <int R> __device__ size_t run_row(int t, int) const { return (size_t)t * R; }
+    template <int R> __device__ const uint16_t *bf16_base(int, int) const { return w; }
+    template <int R> __device__ W4 w4_base(int, int) const { return W4{nullptr, nullptr, nullptr}; }
+};
+
+struct NoProblem {  // "nothing follows"
+    static constexpr int NRUN = 1;
+    int K, group;
+    template <int R> __device__ int n_tasks() const { return 0; }
+    template <int R> __device__ size_t run_row(int, int) const { return 0; }
+    template <int R> __device__ const uint16_t *bf16_base(int, int) const { return nullptr; }
+    template <int R> __device__ W4 w4_base(int, int) const { return W4{nullptr, nullptr, nullptr}; }
+};
+
+// ---------------------------------------------------------------- the kernel
+// N = activation rows per pass (1, 2 or 4; the host picks the smallest that holds the step's rows, or fewer if the
+// widest input does not fit in shared memory N times).  Launched cooperatively: gridDim.x CTAs are co-resident.
+template <int N, int DH, int GQ>
+__global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const ChainArgs a) {
+    extern __shared__ __align__(16) float chain_smem[];
+    __shared__ ChainFlags fl;
+    __shared__ float s_best[kChainWarps];
+    __shared__ int s_besti[kChainWarps];
+    constexpr int R = kChainR;
+    const int Kmax = max(max(a.d, a.F), a.Hq * a.dh);
+    ChainSmem sm;
+    sm.red = chain_smem;                                  // 96
+    sm.xsum = chain_smem + 96;                            // N * Kmax / 32
+    sm.part = sm.xsum + ((N * (Kmax >> 5) + 3) & ~3);     // kChainWarps * part_cap * R * N
+    sm.xs = sm.part + ((kChainWarps * a.part_cap * R * N + 3) & ~3);
+    const int n = a.meta->n_rows;
+    const int L = a.L;
+    unsigned target = 0;
+    if (threadIdx.x == 0) {
+        fl.dead = 0;
+        fl.flag = 0;
+        int na = 0, nr = 0;
+        for (int b = 0; b < n && b < 4; ++b) {
+            fl.exited[b] = a.exited[b];
+            fl.pass[b] = 0;
+            if (fl.exited[b] == 0) fl.act[na++] = b;
+            else fl.riv[nr++] = b;
+        }
+        fl.na = na;
+        fl.nr = nr;
+    }
+    __syncthreads();
+    const bool stamp = a.stamps != nullptr && blockIdx.x == 0 && threadIdx.x == 0;
+    int si = 0;
+    if (stamp) a.stamps[si++] = chain_now();
+    ChainProbe probe{stamp ? a.sub : nullptr, chain_now()};
+    const int S = a.meta->pad[1], chunk = a.meta->pad[0];
+    int hi = 0;
+    for (int l = 1; l <= L; ++l) {
+        const LayerDev &w = a.layers[l - 1];
+        float *h_in = a.h[hi], *h_mid = a.h[(hi + 1) % 3], *h_out = a.h[(hi + 2) % 3];
+        const int na = fl.na, nr = w.has_river ? fl.nr : 0;
+        const bool riv = nr > 0, act = na > 0;
+
+        QkvProblem pq{};
+        pq.wq = w.wq; pq.wk = w.wk; pq.wv = w.wv; pq.rq = w.rq; pq.rk = w.rk; pq.rv = w.rv;
+        pq.K = a.d; pq.Hq = a.Hq; pq.Hkv = a.Hkv; pq.dh = a.dh; pq.group = a.group;
+        pq.rope_cs = a.rope_cs; pq.q_out = a.qbuf; pq.kv = a.kv; pq.kv.layer0 = l - 1; pq.dev_err = a.dev_err;
+        ResidProblem po{};
+        po.w = w.wo; po.rw = w.ro; po.K = a.Hq * a.dh; po.out_dim = a.d; po.group = a.group; po.resid = h_in; po.out = h_mid;
+        GateUpProblem pg{};
+        pg.wg = w.wg; pg.wu = w.wu; pg.rg = w.rg; pg.ru = w.ru; pg.K = a.d; pg.F = a.F; pg.group = a.group; pg.act = a.act;
+        ResidProblem pd{};
+        pd.w = w.wd; pd.rw = w.rd; pd.K = a.F; pd.out_dim = a.d; pd.group = a.group; pd.resid = h_mid; pd.out = h_out;
+
+        // ---- a2
+        chain_project<QkvProblem, N>(a, pq, ProjIn{h_in, w.attn_norm, a.eps}, fl.act, na, fl.riv, nr, sm,
+                                     [&]() { chain_prefetch<ResidProblem, R>(po, act, riv, a.pf_bytes); }, probe, 0);
+        if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
+        probe.mark(3);
+        if (stamp) a.stamps[si++] = chain_now();
+        // ---- a3
+        chain_attention<DH, GQ>(a, pq.kv, n, S, chunk, sm.xs, &fl);
+        probe.mark(32);
+        if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
+        probe.mark(35);
+        if (stamp) a.stamps[si++] = chain_now();
+        // ---- a4
+        chain_project<ResidProblem, N>(a, po, ProjIn{a.obuf, nullptr, 0.f}, fl.act, na, fl.riv, nr, sm,
+                                       [&]() { chain_prefetch<GateUpProblem, R>(pg, act, riv, a.pf_bytes); }, probe, 8);
+        if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
+        probe.mark(11);
+        if (stamp) a.stamps[si++] = chain_now();
+        // ---- a5: gate / up + SwiGLU
+        chain_project<GateUpProblem, N>(a, pg, ProjIn{h_mid, w.ffn_norm, a.eps}, fl.act, na, fl.riv, nr, sm,
+                                        [&]() { chain_prefetch<ResidProblem, R>(pd, act, riv, a.pf_bytes); }, probe, 16);
+        if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
+        probe.mark(19);
+        if (stamp) a.stamps[si++] = chain_now();
+        // ---- a5: down + residual; what follows is block l + 1 with the lists as they stand (an exit at this layer
+        // makes the bf16 part of that request useless, once per token), or the LM head
+        chain_project<ResidProblem, N>(a, pd, ProjIn{a.act, nullptr, 0.f}, fl.act, na, fl.riv, nr, sm, [&]() {
+            if (l < L) {
+                const LayerDev &wn = a.layers[l];
+                QkvProblem pn = pq;
+                pn.wq = wn.wq; pn.wk = wn.wk; pn.wv = wn.wv; pn.rq = wn.rq; pn.rk = wn.rk; pn.rv = wn.rv;
+                chain_prefetch<QkvProblem, R>(pn, act, wn.has_river && fl.nr > 0, a.pf_bytes);
+            } else {
+                HeadProblem ph{a.lm_head, a.d, a.V, a.group};
+                chain_prefetch<HeadProblem, R>(ph, true, false, a.pf_bytes);
+            }
+        }, probe, 24);
+        if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
+        probe.mark(27);
+        if (stamp) a.stamps[si++] = chain_now();
+        // ---- a6 + a7
+        chain_decide(a, l, h_in, h_out, n, sm.red, &fl);
+        probe.mark(36);
+        if (stamp) a.stamps[si++] = chain_now();
+        hi = (hi + 2) % 3;
+    }
+
+    // ---- a8: final norm + LM head + per-CTA argmax partials (merged by argmax_final_kernel)
+    const int n_head = a.meta->n_head_rows;
+    if (n_head > 0) {
+        HeadProblem ph{a.lm_head, a.d, a.V, a.group};
+        float *logits = a.meta->logits;
+        const ProjIn in{a.h[hi], a.final_norm, a.eps};
+        const int xstride = xs_stride(a.d, 32);
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int i0 = 0; i0 < n_head; i0 += N) {
+            stream_load_rows<N, 8>(in, a.head_rows, i0, n_head, a.d, xstride, sm.xs, sm.xsum, sm.red);
+            float best[N];
+            int besti[N];
+#pragma unroll
+            for (int k = 0; k < N; ++k) { best[k] = -CUDART_INF_F; besti[k] = 0x7fffffff; }
+            NoProblem none{a.d, a.group};
+            chain_stream<HeadProblem, N, R, false>(ph, sm.xs, sm.xsum, xstride, sm.part, a.part_cap, a.dev_err, false,
+                                                   [&]() { (void)none; }, [&](int t, int k, const float(&res)[R]) {
+                                                       if (i0 + k >= n_head) return;
+#pragma unroll
+                                                       for (int r = 0; r < R; ++r) {
+                                                           const int id = t * R + r;
+                                                           if (logits) logits[(size_t)(i0 + k) * a.V + id] = res[r];
+#pragma unroll
+                                                           for (int kk = 0; kk < N; ++kk)
+                                                               if (kk == k && (res[r] > best[kk] || (res[r] == best[kk] && id < besti[kk]))) {
+                                                                   best[kk] = res[r];
+                                                                   besti[kk] = id;
+                                                               }
+                                                       }
+                                                   }, probe, 40);
+#pragma unroll
+            for (int k = 0; k < N; ++k) {
+                float bv = best[k];
+                int bi = besti[k];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                }
+                if (lane == 0) { s_best[warp] = bv; s_besti[warp] = bi; }
+                __syncthreads();
+                if (threadIdx.x == 0 && i0 + k < n_head) {
+                    for (int w2 = 1; w2 < kChainWarps; ++w2)
+                        if (s_best[w2] > bv || (s_best[w2] == bv && s_besti[w2] < bi)) { bv = s_best[w2]; bi = s_besti[w2]; }
+                    a.part_val[(size_t)(i0 + k) * gridDim.x + blockIdx.x] = bv;
+                    a.part_idx[(size_t)(i0 + k) * gridDim.x + blockIdx.x] = bi;
+                }
+                __syncthreads();
+            }
+        }
+    }
+    if (stamp) a.stamps[si++] = chain_now();
+}
+
+// Shared memory the kernel needs for N rows per pass.
+inline size_t chain_smem_bytes(int N, int Kmax, int part_cap, int dh, int gq) {
+    const size_t xs = std::max<size_t>((size_t)N * xs_stride(Kmax, 32), (size_t)kChainWarps * gq * (dh + 2));
+    return sizeof(float) * (96 + (((size_t)N * (Kmax >> 5) + 3) & ~(size_t)3) + (((size_t)kChainWarps * part_cap * kChainR * N + 3) & ~(size_t)3) + xs);
+}
+
+}  // namespace river

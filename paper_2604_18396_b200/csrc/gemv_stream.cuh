@@ -110,7 +110,7 @@ struct ResidProblem {  // out[row][o] = resid[row][o] + W[o] . x[row]
     __device__ void epilogue(int t, int row, const float (&res)[R]) const {
         const size_t o = (size_t)row * out_dim + (size_t)t * R;
 #pragma unroll
-        for (int r = 0; r < R; ++r) out[o + r] = resid[o + r] + res[r];
+        for (int r = 0; r < R; ++r) out[o + r] = __ldcg(resid + o + r) + res[r];  // L2: written by other SMs
     }
 };
 

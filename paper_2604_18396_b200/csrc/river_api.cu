@@ -13,7 +13,10 @@
 #include "river_kernels.cuh"
 #include "attn_decode.cuh"
 #include "gemv_stream.cuh"
+#include <cstdio>
+#include <cstdlib>
 #include "gemm_tc.cuh"
+#include "decode_chain.cuh"
 
 using namespace river;
 
@@ -22,9 +25,10 @@ namespace {
 thread_local std::string g_init_error;
 
 constexpr int kStaging = 4;        // pinned metadata buffers in flight
-enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, kNumClasses };
+enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, K_CHAIN, kNumClasses };
 const char *const kClassNames[kNumClasses] = {"step_begin", "compact", "qkv_rope_kv", "attn_decode", "o_proj_resid",
-                                              "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final"};
+                                              "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final",
+                                              "decode_chain"};
 
 struct Carver {
     char *base;
@@ -65,6 +69,11 @@ struct river_ctx {
     struct BMap { int K, np; CUtensorMap hi, lo; };
     std::vector<BMap> tc_bmaps;
     int32_t *hint_act;
+    // persistent layer-chain kernel for steps of at most four rows
+    LayerDev *layers_dev = nullptr;
+    unsigned long long *chain_stamps = nullptr;
+    bool chain_ok = false;
+    int chain_grid = 0, chain_pf_bytes = 4 * 1024;
     struct GraphEntry { int n; bool scores; cudaGraphExec_t exec; int launches; };
     std::vector<GraphEntry> graphs;
     double *inv_freq;
@@ -166,6 +175,8 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
+    LayerDev *ld = cv.take<LayerDev>(L);
+    unsigned long long *stp = cv.take<unsigned long long>(2 + 6 * L + 48);
 
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
@@ -173,6 +184,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
+        x->layers_dev = ld; x->chain_stamps = stp;
         x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
@@ -245,7 +257,12 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     mh[3] = chunk;
     mh[4] = S;
     mh[5] = n;  // hint_act: every row starts in the backbone
-    mh[6] = mh[7] = 0;
+    // the persistent chain kernel: one CTA per (row, kv head, split), chunks in whole pages
+    int Sc = std::max(1, std::min(64, (c->chain_grid > 0 ? c->chain_grid : c->num_sms) / (n * g.Hkv)));
+    int cchunk = (max_pos + 1 + Sc - 1) / Sc;
+    cchunk = std::max(kPage, (cchunk + kPage - 1) / kPage * kPage);
+    mh[6] = cchunk;  // StepMeta::pad[0]
+    mh[7] = Sc;      // StepMeta::pad[1]
     c->attn_splits_now = S;
 }
 
@@ -527,12 +544,24 @@ struct LaunchScope {
     }
 };
 
-int profile_collect(river_ctx *c) {
-    const int L = c->cfg.L;
+int profile_collect(river_ctx *c, int n = 0, int n_head = 0, const int32_t *row_pos_host = nullptr) {
+    const river_config &g = c->cfg;
+    const int L = g.L;
     std::vector<int32_t> na(L + 1), nr(L + 1);
+    std::vector<unsigned long long> stamps(2 + 6 * (size_t)L + 48);
     CUDA_TRY(c, cudaMemcpyAsync(na.data(), c->n_act, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(nr.data(), c->n_riv, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(stamps.data(), c->chain_stamps, sizeof(unsigned long long) * stamps.size(),
+                                cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (std::getenv("RIVER_CHAIN_PROBE")) {  // debugging aid: where CTA 0 of the chain kernel spent the last step
+        const unsigned long long *sub = stamps.data() + 2 + 6 * (size_t)L;
+        const char *names[6] = {"qkv", "o", "gateup", "down", "attn/decide", "head"};
+        for (int k = 0; k < 6; ++k)
+            std::fprintf(stderr, "chain probe %-12s bf16: stage %7.1f stream %7.1f finish %7.1f wait %7.1f | w4: stage %7.1f stream %7.1f finish %7.1f (us per step)\n",
+                         names[k], sub[8 * k] * 1e-3, sub[8 * k + 1] * 1e-3, sub[8 * k + 2] * 1e-3, sub[8 * k + 3] * 1e-3,
+                         sub[8 * k + 4] * 1e-3, sub[8 * k + 5] * 1e-3, sub[8 * k + 6] * 1e-3);
+    }
     for (size_t i = 0; i < c->prof_rec.size(); ++i) {
         const auto &r = c->prof_rec[i];
         float ms = 0.f;
@@ -540,7 +569,34 @@ int profile_collect(river_ctx *c) {
         c->prof_ms[r.cls] += ms;
         c->prof_launches[r.cls] += 1;
         double bytes = 0.0;
-        if (r.list_idx < 0) bytes = r.bytes_act;
+        if (r.list_idx == -2) {
+            // the chain kernel: weights of the executed (layer, weight set) pairs, cache traffic, LM head; its phases
+            // as CTA 0 saw them (global timer at the phase boundaries) are booked under the per-phase classes
+            const int qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
+            const double w4f = 0.25 + 2.0 / g.group;
+            const double wb[4] = {2.0 * (qdim + 2.0 * kvdim) * g.d, 2.0 * qdim * g.d, 4.0 * g.F * g.d, 2.0 * g.F * g.d};
+            const int cls[6] = {K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE};
+            double kv_read = 0.0;
+            for (int b = 0; b < n; ++b) kv_read += (double)(row_pos_host[b] + 1) * 2.0 * kvdim * 2.0;
+            const double kv_write = (double)n * 2.0 * kvdim * 2.0;
+            for (int l = 0; l < L; ++l) {
+                const double f = (na[l] > 0 ? 1.0 : 0.0) + (nr[l] > 0 ? w4f : 0.0);
+                const double pb[6] = {wb[0] * f + kv_write, kv_read, wb[1] * f, wb[2] * f, wb[3] * f, (double)n * g.d * 8.0};
+                for (int ph = 0; ph < 6; ++ph) {
+                    c->prof_ms[cls[ph]] += (double)(stamps[1 + 6 * l + ph] - stamps[6 * l + ph]) * 1e-6;
+                    c->prof_launches[cls[ph]] += 1;
+                    c->prof_bytes[cls[ph]] += pb[ph];
+                    if (ph != 5) bytes += pb[ph];
+                }
+            }
+            if (n_head > 0) {
+                const double hb = 2.0 * g.V * g.d + 4.0 * n_head * g.V;
+                c->prof_ms[K_HEAD] += (double)(stamps[1 + 6 * (size_t)L] - stamps[6 * (size_t)L]) * 1e-6;
+                c->prof_launches[K_HEAD] += 1;
+                c->prof_bytes[K_HEAD] += hb;
+                bytes += hb;
+            }
+        } else if (r.list_idx < 0) bytes = r.bytes_act;
         else bytes = (na[r.list_idx] > 0 ? r.bytes_act : 0.0) + (nr[r.list_idx] > 0 ? r.bytes_riv : 0.0);
         c->prof_bytes[r.cls] += bytes;
     }
@@ -697,9 +753,150 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
     return 0;
 }
 
+// ---- persistent layer-chain kernel (steps of at most four rows)
+int chain_part_cap(const river_config &g, int grid) {
+    auto cap_for = [&](int tasks, int K, bool w4) {
+        const int nch = w4 ? K / 32 : K / 8;
+        const int nit = (nch + 31) / 32, its = w4 ? kW4Its : kBfIts;
+        const int nsl = std::max(1, (nit + its - 1) / its);
+        const int T = (tasks + grid - 1) / grid;
+        const int upw = (T * nsl + kChainWarps - 1) / kChainWarps;
+        return (upw + nsl - 1) / nsl + 1;
+    };
+    const int qdim = g.Hq * g.dh;
+    int cap = 2;
+    for (int w4 = 0; w4 < 2; ++w4) {
+        cap = std::max(cap, cap_for((g.Hq + 2 * g.Hkv) * (g.dh / 2), g.d, w4));
+        cap = std::max(cap, cap_for(g.d / 2, qdim, w4));
+        cap = std::max(cap, cap_for(g.F, g.d, w4));
+        cap = std::max(cap, cap_for(g.d / 2, g.F, w4));
+    }
+    return std::max(cap, cap_for(g.V / 2, g.d, false));
+}
+
+typedef void (*ChainKern)(const ChainArgs);
+ChainKern chain_kernel_for(int N, int dh, int gq) {
+#define CHAIN_CASE(N_, DH_, GQ_) if (N == N_ && dh == DH_ && gq == GQ_) return decode_chain_kernel<N_, DH_, GQ_>;
+    CHAIN_CASE(1, 64, 2) CHAIN_CASE(2, 64, 2) CHAIN_CASE(4, 64, 2)
+    CHAIN_CASE(1, 64, 4) CHAIN_CASE(2, 64, 4) CHAIN_CASE(4, 64, 4)
+    CHAIN_CASE(1, 128, 4) CHAIN_CASE(2, 128, 4) CHAIN_CASE(4, 128, 4)
+#undef CHAIN_CASE
+    return nullptr;
+}
+
+// Rows per pass for a step of n rows, or 0 if the chain kernel does not take this step.
+int chain_rows_per_pass(const river_ctx *c, int n) {
+    const river_config &g = c->cfg;
+    if (!c->chain_ok || n < 1 || n > 4) return 0;
+    const int N = n == 1 ? 1 : (n == 2 ? 2 : 4);
+    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
+    if (chain_smem_bytes(N, Kmax, chain_part_cap(g, c->chain_grid), g.dh, g.Hq / g.Hkv) > 200 * 1024) return 0;
+    return N;
+}
+
+bool chain_setup(river_ctx *c) {
+    const river_config &g = c->cfg;
+    if (g.flags & RIVER_F_NO_CHAIN) return false;
+    if (g.V % 2 || g.d % 4 || g.F % 2) return false;
+    if (!chain_kernel_for(1, g.dh, g.Hq / g.Hkv)) return false;
+    int dev = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return false;
+    c->chain_grid = c->num_sms;
+    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
+    const int cap = chain_part_cap(g, c->chain_grid);
+    bool any = false;
+    for (int N = 1; N <= 4; N *= 2) {
+        const size_t smem = chain_smem_bytes(N, Kmax, cap, g.dh, g.Hq / g.Hkv);
+        if (smem > 200 * 1024) continue;
+        ChainKern k = chain_kernel_for(N, g.dh, g.Hq / g.Hkv);
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kChainThreads, smem) != cudaSuccess || occ < 1) return false;
+        any = true;
+    }
+    if (!any) return false;
+    std::vector<LayerDev> ld(g.L);
+    for (int l = 0; l < g.L; ++l) {
+        const river_layer_weights &w = c->layers[l];
+        LayerDev &x = ld[l];
+        x.attn_norm = (const uint16_t *)w.attn_norm; x.ffn_norm = (const uint16_t *)w.ffn_norm;
+        x.wq = (const uint16_t *)w.wq; x.wk = (const uint16_t *)w.wk; x.wv = (const uint16_t *)w.wv;
+        x.wo = (const uint16_t *)w.wo; x.wg = (const uint16_t *)w.wg; x.wu = (const uint16_t *)w.wu;
+        x.wd = (const uint16_t *)w.wd;
+        x.rq = w4(w.rq); x.rk = w4(w.rk); x.rv = w4(w.rv); x.ro = w4(w.ro); x.rg = w4(w.rg); x.ru = w4(w.ru); x.rd = w4(w.rd);
+        x.has_river = w.rq.codes != nullptr;
+        x.pad = 0;
+    }
+    if (cudaMemcpy(c->layers_dev, ld.data(), sizeof(LayerDev) * g.L, cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    const int kb = (g.flags >> 8) & 0xff;  // tuning aid: KiB of the next phase each warp requests from the L2
+    if (kb) c->chain_pf_bytes = kb * 1024;
+    return true;
+}
+
+int run_chain(river_ctx *c, int n, int n_head, int N, const int32_t *row_pos_host) {
+    const river_config &g = c->cfg;
+    const int L = g.L, d = g.d, B = g.max_batch;
+    c->st.launches_last_step = 0;
+    Lists lists{c->act_idx, c->riv_idx, c->n_act, c->n_riv, B};
+    cudaError_t err = cudaSuccess;
+    auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
+    {
+        LaunchScope ls(c, K_BEGIN, (double)n * d * 2.0, 0, -1);
+        note(launch_k(step_begin_kernel, dim3(std::max(n, 1)), dim3(128), 0, c->stream, false, c->meta(), c->upd(),
+                      c->page_tbl_dev, g.max_pages_per_seq, B, c->embed, d, g.V, c->h[0], c->row_pos(), c->inv_freq,
+                      g.dh / 2, c->rope_cs, L, g.entry_layer, c->exited, c->dev_err, lists, c->hint_act, c->tickets));
+    }
+    note(cudaMemsetAsync(c->tickets + 2, 0, sizeof(unsigned), c->stream));
+    if (c->profiling) note(cudaMemsetAsync(c->chain_stamps + 2 + 6 * (size_t)L, 0, sizeof(unsigned long long) * 48, c->stream));
+    ChainArgs a{};
+    a.meta = c->meta(); a.layers = c->layers_dev;
+    a.L = L; a.d = d; a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh; a.F = g.F; a.V = g.V; a.group = g.group;
+    a.entry_layer = g.entry_layer; a.exit_mode = g.exit_mode; a.eps = g.rms_eps;
+    a.qscale = 1.4426950408889634f / std::sqrt((float)g.dh);
+    a.h[0] = c->h[0]; a.h[1] = c->h[1]; a.h[2] = c->h[2]; a.qbuf = c->qbuf; a.obuf = c->obuf; a.act = c->act;
+    a.rope_cs = c->rope_cs; a.kv = kv_addr(c, 0);
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.attn_tickets = c->attn_tickets;
+    a.exited = c->exited; a.lists = lists;
+    a.lm_head = c->lm_head; a.final_norm = c->final_norm; a.head_rows = c->head_rows();
+    a.part_val = c->part_val; a.part_idx = c->part_idx;
+    a.bar = c->tickets + 2; a.dev_err = c->dev_err;
+    a.stamps = c->profiling ? c->chain_stamps : nullptr;
+    a.sub = c->profiling ? c->chain_stamps + 2 + 6 * (size_t)L : nullptr;
+    a.part_cap = chain_part_cap(g, c->chain_grid);
+    a.pf_bytes = c->chain_pf_bytes;
+    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
+    const size_t smem = chain_smem_bytes(N, Kmax, a.part_cap, g.dh, g.Hq / g.Hkv);
+    {
+        LaunchScope ls(c, K_CHAIN, 0, 0, -2);
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(c->chain_grid);
+        cfg.blockDim = dim3(kChainThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = c->stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeCooperative;
+        at[0].val.cooperative = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        note(cudaLaunchKernelEx(&cfg, chain_kernel_for(N, g.dh, g.Hq / g.Hkv), a));
+    }
+    if (n_head > 0) {
+        LaunchScope ls(c, K_ARGMAX, 0, 0, -1);
+        note(launch_k(argmax_final_kernel, dim3(n_head), dim3(128), 0, c->stream, false, c->meta(),
+                      (const float *)c->part_val, (const int32_t *)c->part_idx, c->chain_grid));
+    }
+    if (err == cudaSuccess) err = cudaGetLastError();
+    if (err != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(err));
+    c->st.launches_total += c->st.launches_last_step;
+    if (c->profiling) return profile_collect(c, n, n_head, row_pos_host);
+    return 0;
+}
+
 // One decode step through a CUDA graph of the launch sequence (captured the second time a row count is seen; the
 // per-step inputs live in device memory, so the graph never needs new parameters).
 int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
+    if (const int N = chain_rows_per_pass(c, n)) return run_chain(c, n, n, N, row_pos_host);
     const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
     if (!use_graph) return run_rows(c, n, n, row_pos_host);
     for (auto &ge : c->graphs)
@@ -790,6 +987,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     c->num_sms = prop.multiProcessorCount;
     if (make_kv_tensor_map(c)) { river_destroy(c); return RIVER_E_DEVICE; }
     c->tc_ok = !(cfg->flags & RIVER_F_NO_TC) && tc_shape_ok(*cfg) && make_tc_maps(c);
+    c->chain_ok = chain_setup(c);
     for (int i = 0; i < kStaging; ++i) {
         if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");
         if (cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail("cudaEventCreate failed");

@@ -16,7 +16,7 @@ namespace river {
 constexpr int kPage = 16;         // tokens per KV page
 constexpr int kMaxBatch = 1024;   // rows per step (one CTA scans the exit flags)
 
-enum DevErr : int { DEV_OK = 0, DEV_BAD_FORCED = 1, DEV_BAD_TOKEN = 2, DEV_BAD_PAGE = 3, DEV_WAIT_TIMEOUT = 4 };
+enum DevErr : int { DEV_OK = 0, DEV_BAD_FORCED = 1, DEV_BAD_TOKEN = 2, DEV_BAD_PAGE = 3, DEV_WAIT_TIMEOUT = 4, DEV_INTERNAL = 5 };
 
 // ---------------------------------------------------------------- small helpers
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -123,9 +123,10 @@ def test_tiny_geometric_exits_and_wide_batch():
     assert r["n_early"] > r["total"] // 2
 
 
-@pytest.mark.parametrize("flags", [1, 2, 4, 5])
+@pytest.mark.parametrize("flags", [0, 1, 2, 4, 5, 8, 9, 12])
 def test_launch_modes_agree_with_oracle(flags):
-    # 1: CUDA-graph replay; 2: no tensor-core projections; 4: plain attention kernel
+    # 1: CUDA-graph replay; 2: no tensor-core projections; 4: plain attention kernel; 8: separate kernels per stage
+    # instead of the persistent chain kernel (three rows: the chain kernel takes the step unless 8 is set)
     r = run_scheduled(model("mini8"), [37, 16, 3], 6, "uniform", page_seed=11, flags=flags, max_batch=4)
     assert r["n_early"] > 0
 
