@@ -47,9 +47,10 @@ struct ChainArgs {
     int *dev_err;
     unsigned long long *stamps;  // optional [2 + 6 L]: globaltimer at the phase boundaries seen by CTA 0
     unsigned long long *sub;     // optional [5][8]: time CTA 0 spent staging / streaming / finishing / waiting, per phase kind
-    int part_cap;       // partial slots per warp
+    int part_cap;       // unit slots for partial dot products
     int pf_bytes;       // bytes of the next phase each warp asks the L2 for
     int xs_floats;      // capacity of the activation staging area
+    int part_floats;    // capacity of the partial-sum area
 };
 
 constexpr int kChainThreads = 512;
@@ -126,7 +127,6 @@ struct ChainShare {
     int t0, T;        // first task and task count of this CTA
     int nsl;          // K slices per task
     int units;        // T * nsl
-    __device__ __forceinline__ int bound(int w) const { return (int)(((long long)units * w) / kChainWarps); }
 };
 __device__ __forceinline__ ChainShare chain_share(int tasks, int nit, int its_per_slice) {
     ChainShare s;
@@ -248,39 +248,39 @@ __device__ __forceinline__ void chain_rows_w4(const P &p, int t, W4 (&rows)[R]) 
     }
 }
 
-// ---------------------------------------------------------------- L2 prefetch of a warp's first units of a phase
+// ---------------------------------------------------------------- L2 prefetch of the first units of a phase
+// Units are consumed in index order, so the CTA asks for its first kChainWarps * (pf_bytes / unit bytes) units;
+// thread i of the CTA takes (unit i / R, row i % R).
 template <class P, int R>
 __device__ __forceinline__ void chain_prefetch(const P &p, bool want_bf16, bool want_w4, int pf_bytes) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int K = p.K;
     const int tasks = p.template n_tasks<R>();
+    const int i = threadIdx.x;
     if (want_bf16) {
         const int nch = K >> 3;
         const ChainShare sh = chain_share(tasks, (nch + 31) >> 5, kBfIts);
-        const int u0 = sh.bound(warp), u1 = sh.bound(warp + 1);
         const int per = kBfIts * 32 * 8;  // inputs per slice
-        const int npu = max(1, min(32 / R, pf_bytes / (R * per * 2)));
-        const int u = u0 + lane / R, r = lane % R;
-        if (lane < npu * R && u < u1) {
-            const int t = sh.t0 + u / sh.nsl, s = u % sh.nsl;
+        const int count = min(sh.units, kChainWarps * max(1, pf_bytes / (R * per * 2)));
+        const int u = i / R, r = i % R;
+        if (u < count) {
+            const int t = sh.t0 + u / sh.nsl, sl = u % sh.nsl;
             const int run = r / (R / P::NRUN), j = r % (R / P::NRUN);
             const uint16_t *row = p.template bf16_base<R>(t, run) + (p.template run_row<R>(t, run) + j) * (size_t)K;
-            const int k0 = s * per;
+            const int k0 = sl * per;
             if (k0 < K) l2_prefetch(row + k0, (size_t)min(per, K - k0) * 2);
         }
     }
     if (want_w4) {
         const int nch = K >> 5;
         const ChainShare sh = chain_share(tasks, (nch + 31) >> 5, kW4Its);
-        const int u0 = sh.bound(warp), u1 = sh.bound(warp + 1);
         const int per = kW4Its * 32 * 32;
-        const int npu = max(1, min(32 / R, pf_bytes / (R * (per / 2 + 4 * per / p.group))));
-        const int u = u0 + lane / R, r = lane % R;
-        if (lane < npu * R && u < u1) {
-            const int t = sh.t0 + u / sh.nsl, s = u % sh.nsl;
+        const int count = min(sh.units, kChainWarps * max(1, pf_bytes / (R * (per / 2 + 4 * per / p.group))));
+        const int u = i / R, r = i % R;
+        if (u < count) {
+            const int t = sh.t0 + u / sh.nsl, sl = u % sh.nsl;
             W4 rows[R];
             chain_rows_w4<P, R>(p, t, rows);
-            const int k0 = s * per;
+            const int k0 = sl * per;
             if (k0 < K) {
                 const int len = min(per, K - k0);
                 l2_prefetch(rows[r].codes + (k0 >> 1), (size_t)len >> 1);
@@ -292,114 +292,121 @@ __device__ __forceinline__ void chain_prefetch(const P &p, bool want_bf16, bool 
 }
 
 // ---------------------------------------------------------------- one pass of a phase over staged activation rows
-// Every warp streams its units, partial sums of a task meet in `part`, then the CTA's threads finish the tasks:
+// The CTA's share of the phase is T tasks x nsl K-slices = units of equal size.  Warps take units from a shared
+// counter (a warp that met slow memory simply takes fewer), keep the next unit's loads in flight while they
+// multiply the current one, and leave each unit's R x N partial dot products in its own slot; then the CTA's
+// threads add a task's slices in slice order (deterministic, whoever computed them) and finish the task:
 // epi(task, n, res[R]) gets the R dot products of activation row n of the pass.
 template <class P, int N, int R, bool W4M, class PF, class EP>
 __device__ __forceinline__ void chain_stream(const P &p, const float *xs, const float *xsum, int xstride, float *part,
                                              int part_cap, int *dev_err, bool do_pf, PF &&prefetch_next, EP &&epi,
-                                             ChainProbe &probe, int pk) {
+                                             int *s_next, ChainProbe &probe, int pk) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int K = p.K;
     const int nch = W4M ? (K >> 5) : (K >> 3);
     constexpr int ITS = W4M ? kW4Its : kBfIts;
     const ChainShare sh = chain_share(p.template n_tasks<R>(), (nch + 31) >> 5, ITS);
-    const int u0 = sh.bound(warp), u1 = sh.bound(warp + 1);
-    const int tf = u0 / sh.nsl;
+    const int nsl = sh.nsl;
+    int units = sh.units;
+    if (units > part_cap) {  // cannot happen with the host's sizing; flagged rather than trusted
+        if (threadIdx.x == 0) atomicExch(dev_err, DEV_INTERNAL);
+        units = 0;
+    }
+    if (threadIdx.x == 0) *s_next = kChainWarps;
+    __syncthreads();
     float acc[R][N];
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
-
-    auto flush = [&](int t) {
-        const int j = t - tf;
-        float *dst = part + (size_t)(warp * part_cap + j) * (R * N);
+    auto store_unit = [&](int u) {
+        float *dst = part + (size_t)u * (R * N);
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
             for (int n = 0; n < N; ++n) {
                 const float v = warp_sum(acc[r][n]);
-                if (lane == 0 && j < part_cap) dst[r * N + n] = v;
-                acc[r][n] = 0.f;
+                if (lane == 0) dst[r * N + n] = v;
             }
-        if (lane == 0 && j >= part_cap) atomicExch(dev_err, DEV_INTERNAL);
     };
-
-    if (u0 < u1) {
-        int t = tf, s = u0 - tf * sh.nsl;
-        if constexpr (!W4M) {
-            uint4 wn[R][kBfIts];
-            {
+    auto next_unit = [&]() {
+        int un = 0;
+        if (lane == 0) un = atomicAdd(s_next, 1);
+        return __shfl_sync(0xffffffffu, un, 0);
+    };
+    int u = warp;
+    if constexpr (!W4M) {
+        uint4 wn[R][kBfIts];
+        if (u < units) {
+            const int t = u / nsl;
+            const uint16_t *rows[R];
+            stream_rows_bf16<P, N, R>(p, sh.t0 + t, rows);
+            stream_issue_bf16<R>(rows, nch, (u - t * nsl) * ITS, lane, wn);
+        }
+        while (u < units) {
+            uint4 wc[R][kBfIts];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int i = 0; i < kBfIts; ++i) wc[r][i] = wn[r][i];
+            const int un = next_unit();
+            if (un < units) {
+                const int tn = un / nsl;
                 const uint16_t *rows[R];
-                stream_rows_bf16<P, N, R>(p, sh.t0 + t, rows);
-                stream_issue_bf16<R>(rows, nch, s * ITS, lane, wn);
+                stream_rows_bf16<P, N, R>(p, sh.t0 + tn, rows);
+                stream_issue_bf16<R>(rows, nch, (un - tn * nsl) * ITS, lane, wn);
             }
-            for (int u = u0; u < u1; ++u) {
-                uint4 wc[R][kBfIts];
 #pragma unroll
-                for (int r = 0; r < R; ++r)
+            for (int r = 0; r < R; ++r)
 #pragma unroll
-                    for (int i = 0; i < kBfIts; ++i) wc[r][i] = wn[r][i];
-                int tn = t, sn = s + 1;
-                if (sn == sh.nsl) { sn = 0; ++tn; }
-                if (u + 1 < u1) {
-                    const uint16_t *rows[R];
-                    stream_rows_bf16<P, N, R>(p, sh.t0 + tn, rows);
-                    stream_issue_bf16<R>(rows, nch, sn * ITS, lane, wn);
-                }
-                chain_fma_bf16<N, R>(wc, xs, xstride, s * ITS, nch, lane, acc);
-                if (u + 1 == u1 || tn != t) flush(t);
-                t = tn; s = sn;
-            }
-        } else {
-            const int gshift = (p.group == 64) ? 1 : (p.group == 32 ? 0 : 2);
-            W4Regs wn[R][kW4Its];
-            {
+                for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
+            chain_fma_bf16<N, R>(wc, xs, xstride, (u % nsl) * ITS, nch, lane, acc);
+            store_unit(u);
+            u = un;
+        }
+    } else {
+        const int gshift = (p.group == 64) ? 1 : (p.group == 32 ? 0 : 2);
+        W4Regs wn[R][kW4Its];
+        if (u < units) {
+            const int t = u / nsl;
+            W4 rows[R];
+            chain_rows_w4<P, R>(p, sh.t0 + t, rows);
+            chain_issue_w4<R>(rows, nch, gshift, (u - t * nsl) * ITS, lane, wn);
+        }
+        while (u < units) {
+            W4Regs wc[R][kW4Its];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int i = 0; i < kW4Its; ++i) wc[r][i] = wn[r][i];
+            const int un = next_unit();
+            if (un < units) {
+                const int tn = un / nsl;
                 W4 rows[R];
-                chain_rows_w4<P, R>(p, sh.t0 + t, rows);
-                chain_issue_w4<R>(rows, nch, gshift, s * ITS, lane, wn);
+                chain_rows_w4<P, R>(p, sh.t0 + tn, rows);
+                chain_issue_w4<R>(rows, nch, gshift, (un - tn * nsl) * ITS, lane, wn);
             }
-            for (int u = u0; u < u1; ++u) {
-                W4Regs wc[R][kW4Its];
 #pragma unroll
-                for (int r = 0; r < R; ++r)
+            for (int r = 0; r < R; ++r)
 #pragma unroll
-                    for (int i = 0; i < kW4Its; ++i) wc[r][i] = wn[r][i];
-                int tn = t, sn = s + 1;
-                if (sn == sh.nsl) { sn = 0; ++tn; }
-                if (u + 1 < u1) {
-                    W4 rows[R];
-                    chain_rows_w4<P, R>(p, sh.t0 + tn, rows);
-                    chain_issue_w4<R>(rows, nch, gshift, sn * ITS, lane, wn);
-                }
-                chain_fma_w4<N, R>(wc, xs, xsum, xstride, s * ITS, nch, lane, acc);
-                if (u + 1 == u1 || tn != t) flush(t);
-                t = tn; s = sn;
-            }
+                for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
+            chain_fma_w4<N, R>(wc, xs, xsum, xstride, (u % nsl) * ITS, nch, lane, acc);
+            store_unit(u);
+            u = un;
         }
     }
     probe.mark(pk + 1);
     if (do_pf) prefetch_next();
     __syncthreads();
-    for (int e = threadIdx.x; e < sh.T * N; e += blockDim.x) {
-        const int tl = e / N, n = e - tl * N;
-        float res[R];
+    if (!W4M) probe.mark((pk & ~7) + 7);
+    if (units > 0)
+        for (int e = threadIdx.x; e < sh.T * N; e += blockDim.x) {
+            const int tl = e / N, n = e - tl * N;
+            float res[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) res[r] = 0.f;
-        const int ua = tl * sh.nsl, ub = ua + sh.nsl - 1;
-        for (int w = 0; w < kChainWarps; ++w) {  // fixed order: deterministic sums
-            const int b0 = sh.bound(w), b1 = sh.bound(w + 1);
-            if (b1 > b0 && b0 <= ub && b1 > ua) {
-                const int j = tl - b0 / sh.nsl;
-                if (j < part_cap) {
-                    const float *src = part + (size_t)(w * part_cap + j) * (R * N);
+            for (int r = 0; r < R; ++r) res[r] = 0.f;
+            const float *src = part + (size_t)tl * nsl * (R * N) + n;
+            for (int sl = 0; sl < nsl; ++sl)
 #pragma unroll
-                    for (int r = 0; r < R; ++r) res[r] += src[r * N + n];
-                }
-            }
+                for (int r = 0; r < R; ++r) res[r] += src[(sl * R + r) * N];
+            epi(sh.t0 + tl, n, res);
         }
-        epi(sh.t0 + tl, n, res);
-    }
     __syncthreads();
     probe.mark(pk + 2);
 }
@@ -413,7 +420,7 @@ struct ChainSmem {
 template <class P, int N, class PF>
 __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, const ProjIn &in, const int *s_act, int na,
                                               const int *s_riv, int nr, const ChainSmem &sm, PF &&prefetch_next,
-                                              ChainProbe &probe, int pk) {
+                                              int *s_next, ChainProbe &probe, int pk) {
     constexpr int R = kChainR;
     const int K = p.K;
     const int xstride = xs_stride(K, 32);
@@ -426,7 +433,7 @@ __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, co
                                      ps + 1 == passes_a && passes_r == 0, prefetch_next,
                                      [&](int t, int n, const float(&res)[R]) {
                                          if (i0 + n < na) p.template epilogue<R>(t, s_act[i0 + n], res);
-                                     }, probe, pk);
+                                     }, s_next, probe, pk);
     }
     for (int ps = 0; ps < passes_r; ++ps) {
         const int i0 = ps * N;
@@ -435,7 +442,7 @@ __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, co
         chain_stream<P, N, R, true>(p, sm.xs, sm.xsum, xstride, sm.part, a.part_cap, a.dev_err, ps + 1 == passes_r,
                                     prefetch_next, [&](int t, int n, const float(&res)[R]) {
                                         if (i0 + n < nr) p.template epilogue<R>(t, s_riv[i0 + n], res);
-                                    }, probe, pk + 4);
+                                    }, s_next, probe, pk + 4);
     }
     if (passes_a + passes_r == 0) prefetch_next();
 }
@@ -447,7 +454,7 @@ __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, co
 // head) to arrive merges the splits in split order (deterministic) and writes the attention output.
 struct ChainFlags {
     int exited[4], act[4], riv[4], pass[4];
-    int na, nr, dead, flag;
+    int na, nr, dead, flag, next;
 };
 
 __device__ __forceinline__ float chain_ex2(float x) {
@@ -706,7 +713,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
     sm.red = chain_smem;                                  // 96
     sm.xsum = chain_smem + 96;                            // N * Kmax / 32
     sm.part = sm.xsum + ((N * (Kmax >> 5) + 3) & ~3);     // kChainWarps * part_cap * R * N
-    sm.xs = sm.part + ((kChainWarps * a.part_cap * R * N + 3) & ~3);
+    sm.xs = sm.part + a.part_floats;
     const int n = a.meta->n_rows;
     const int L = a.L;
     unsigned target = 0;
@@ -749,7 +756,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
 
         // ---- a2
         chain_project<QkvProblem, N>(a, pq, ProjIn{h_in, w.attn_norm, a.eps}, fl.act, na, fl.riv, nr, sm,
-                                     [&]() { chain_prefetch<ResidProblem, R>(po, act, riv, a.pf_bytes); }, probe, 0);
+                                     [&]() { chain_prefetch<ResidProblem, R>(po, act, riv, a.pf_bytes); }, &fl.next, probe, 0);
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
         probe.mark(3);
         if (stamp) a.stamps[si++] = chain_now();
@@ -761,13 +768,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         if (stamp) a.stamps[si++] = chain_now();
         // ---- a4
         chain_project<ResidProblem, N>(a, po, ProjIn{a.obuf, nullptr, 0.f}, fl.act, na, fl.riv, nr, sm,
-                                       [&]() { chain_prefetch<GateUpProblem, R>(pg, act, riv, a.pf_bytes); }, probe, 8);
+                                       [&]() { chain_prefetch<GateUpProblem, R>(pg, act, riv, a.pf_bytes); }, &fl.next, probe, 8);
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
         probe.mark(11);
         if (stamp) a.stamps[si++] = chain_now();
         // ---- a5: gate / up + SwiGLU
         chain_project<GateUpProblem, N>(a, pg, ProjIn{h_mid, w.ffn_norm, a.eps}, fl.act, na, fl.riv, nr, sm,
-                                        [&]() { chain_prefetch<ResidProblem, R>(pd, act, riv, a.pf_bytes); }, probe, 16);
+                                        [&]() { chain_prefetch<ResidProblem, R>(pd, act, riv, a.pf_bytes); }, &fl.next, probe, 16);
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
         probe.mark(19);
         if (stamp) a.stamps[si++] = chain_now();
@@ -783,7 +790,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                 HeadProblem ph{a.lm_head, a.d, a.V, a.group};
                 chain_prefetch<HeadProblem, R>(ph, true, false, a.pf_bytes);
             }
-        }, probe, 24);
+        }, &fl.next, probe, 24);
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
         probe.mark(27);
         if (stamp) a.stamps[si++] = chain_now();
@@ -823,7 +830,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                                                                    besti[kk] = id;
                                                                }
                                                        }
-                                                   }, probe, 40);
+                                                   }, &fl.next, probe, 40);
 #pragma unroll
             for (int k = 0; k < N; ++k) {
                 float bv = best[k];
@@ -850,9 +857,19 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
 }
 
 // Shared memory the kernel needs for N rows per pass.
-inline size_t chain_smem_bytes(int N, int Kmax, int part_cap, int dh, int gq) {
+struct ChainLayout {
+    int xs_floats, part_floats;
+    size_t bytes;
+};
+// Shared memory of the kernel for N rows per pass: reduction scratch, chunk sums, unit slots, staging area (fp32
+// rows, or the attention scratch).
+inline ChainLayout chain_layout(int N, int Kmax, int part_cap, int dh, int gq) {
+    ChainLayout l;
     const size_t xs = std::max<size_t>((size_t)N * xs_stride(Kmax, 32), (size_t)kChainWarps * gq * (dh + 2));
-    return sizeof(float) * (96 + (((size_t)N * (Kmax >> 5) + 3) & ~(size_t)3) + (((size_t)kChainWarps * part_cap * kChainR * N + 3) & ~(size_t)3) + xs);
+    l.xs_floats = (int)((xs + 3) & ~(size_t)3);
+    l.part_floats = (int)(((size_t)part_cap * kChainR * N + 3) & ~(size_t)3);
+    l.bytes = sizeof(float) * (96 + (((size_t)N * (Kmax >> 5) + 3) & ~(size_t)3) + l.part_floats + l.xs_floats);
+    return l;
 }
 
 }  // namespace river

@@ -558,8 +558,8 @@ int profile_collect(river_ctx *c, int n = 0, int n_head = 0, const int32_t *row_
         const unsigned long long *sub = stamps.data() + 2 + 6 * (size_t)L;
         const char *names[6] = {"qkv", "o", "gateup", "down", "attn/decide", "head"};
         for (int k = 0; k < 6; ++k)
-            std::fprintf(stderr, "chain probe %-12s bf16: stage %7.1f stream %7.1f finish %7.1f wait %7.1f | w4: stage %7.1f stream %7.1f finish %7.1f (us per step)\n",
-                         names[k], sub[8 * k] * 1e-3, sub[8 * k + 1] * 1e-3, sub[8 * k + 2] * 1e-3, sub[8 * k + 3] * 1e-3,
+            std::fprintf(stderr, "chain probe %-12s bf16: stage %7.1f stream %7.1f join %7.1f finish %7.1f wait %7.1f | w4: stage %7.1f stream %7.1f finish %7.1f (us per step)\n",
+                         names[k], sub[8 * k] * 1e-3, sub[8 * k + 1] * 1e-3, sub[8 * k + 7] * 1e-3, sub[8 * k + 2] * 1e-3, sub[8 * k + 3] * 1e-3,
                          sub[8 * k + 4] * 1e-3, sub[8 * k + 5] * 1e-3, sub[8 * k + 6] * 1e-3);
     }
     for (size_t i = 0; i < c->prof_rec.size(); ++i) {
@@ -754,14 +754,12 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
 }
 
 // ---- persistent layer-chain kernel (steps of at most four rows)
-int chain_part_cap(const river_config &g, int grid) {
+int chain_part_cap(const river_config &g, int grid) {  // most units (task x K-slice) a CTA owns in any pass
     auto cap_for = [&](int tasks, int K, bool w4) {
         const int nch = w4 ? K / 32 : K / 8;
         const int nit = (nch + 31) / 32, its = w4 ? kW4Its : kBfIts;
         const int nsl = std::max(1, (nit + its - 1) / its);
-        const int T = (tasks + grid - 1) / grid;
-        const int upw = (T * nsl + kChainWarps - 1) / kChainWarps;
-        return (upw + nsl - 1) / nsl + 1;
+        return ((tasks + grid - 1) / grid) * nsl;
     };
     const int qdim = g.Hq * g.dh;
     int cap = 2;
@@ -772,6 +770,15 @@ int chain_part_cap(const river_config &g, int grid) {
         cap = std::max(cap, cap_for(g.d / 2, g.F, w4));
     }
     return std::max(cap, cap_for(g.V / 2, g.d, false));
+}
+
+struct ChainPlan { ChainLayout lay; };
+ChainPlan chain_plan(const river_ctx *c, int N) {  // bytes == 0: N rows per pass do not fit in shared memory
+    const river_config &g = c->cfg;
+    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
+    const ChainLayout l = chain_layout(N, Kmax, chain_part_cap(g, c->chain_grid), g.dh, g.Hq / g.Hkv);
+    if (l.bytes <= 200 * 1024) return ChainPlan{l};
+    return ChainPlan{ChainLayout{0, 0, 0}};
 }
 
 typedef void (*ChainKern)(const ChainArgs);
@@ -789,8 +796,7 @@ int chain_rows_per_pass(const river_ctx *c, int n) {
     const river_config &g = c->cfg;
     if (!c->chain_ok || n < 1 || n > 4) return 0;
     const int N = n == 1 ? 1 : (n == 2 ? 2 : 4);
-    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
-    if (chain_smem_bytes(N, Kmax, chain_part_cap(g, c->chain_grid), g.dh, g.Hq / g.Hkv) > 200 * 1024) return 0;
+    if (chain_plan(c, N).lay.bytes == 0) return 0;
     return N;
 }
 
@@ -803,16 +809,14 @@ bool chain_setup(river_ctx *c) {
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return false;
     c->chain_grid = c->num_sms;
-    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
-    const int cap = chain_part_cap(g, c->chain_grid);
     bool any = false;
     for (int N = 1; N <= 4; N *= 2) {
-        const size_t smem = chain_smem_bytes(N, Kmax, cap, g.dh, g.Hq / g.Hkv);
-        if (smem > 200 * 1024) continue;
+        const ChainPlan pl = chain_plan(c, N);
+        if (pl.lay.bytes == 0) continue;
         ChainKern k = chain_kernel_for(N, g.dh, g.Hq / g.Hkv);
-        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.lay.bytes) != cudaSuccess) return false;
         int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kChainThreads, smem) != cudaSuccess || occ < 1) return false;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kChainThreads, pl.lay.bytes) != cudaSuccess || occ < 1) return false;
         any = true;
     }
     if (!any) return false;
@@ -865,8 +869,10 @@ int run_chain(river_ctx *c, int n, int n_head, int N, const int32_t *row_pos_hos
     a.sub = c->profiling ? c->chain_stamps + 2 + 6 * (size_t)L : nullptr;
     a.part_cap = chain_part_cap(g, c->chain_grid);
     a.pf_bytes = c->chain_pf_bytes;
-    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
-    const size_t smem = chain_smem_bytes(N, Kmax, a.part_cap, g.dh, g.Hq / g.Hkv);
+    const ChainPlan pl = chain_plan(c, N);
+    a.xs_floats = pl.lay.xs_floats;
+    a.part_floats = pl.lay.part_floats;
+    const size_t smem = pl.lay.bytes;
     {
         LaunchScope ls(c, K_CHAIN, 0, 0, -2);
         cudaLaunchConfig_t cfg{};
