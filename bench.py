@@ -129,6 +129,9 @@ def draw_model(shape, device):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (taken on a
 # 4-layer model of the same layer shape: kernel, geometry and operands per launch are those of the full model).
 NCU_TRAFFIC = {("8b", "gateup_swiglu"): 235.0e6}
+# decode_chain_kernel: DRAM read + write = 1.0016 x the algorithmic bytes of the captured step; every layer moves the same
+# bytes, so the ratio carries over to the full model.
+NCU_TRAFFIC_RATIO = {("8b", "decode_chain"): 1.0016}
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle timing
@@ -412,7 +415,10 @@ def ours(args, wl):
                            "frac_of_measured_peak": full_gbs / peak, "frac_of_8TBps": full_gbs / 8000.0},
             "early_exit_speedup_vs_full_depth": ms_full / ms,
             "roofline": {"bound": "hbm", "kernel": dom["name"], "achieved": ach, "peak": peak, "unit": "GB/s",
-                         "frac": ach / peak, "traffic": NCU_TRAFFIC.get((shape_name, dom["name"])),
+                         "frac": ach / peak,
+                         "traffic": NCU_TRAFFIC.get((shape_name, dom["name"])) or (
+                             NCU_TRAFFIC_RATIO[(shape_name, dom["name"])] * dom["alg_bytes_total"] / dom["launches"]
+                             if (shape_name, dom["name"]) in NCU_TRAFFIC_RATIO else None),
                          "peak_kind": peak_kind,
                          "launch_ms": per_launch_ms, "alg_bytes_per_launch": dom["alg_bytes_total"] / dom["launches"],
                          "pass": "full depth, events around every launch"},
