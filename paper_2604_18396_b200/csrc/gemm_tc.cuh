@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int
     pdl_launch();
     pdl_wait();
     const int i = blockIdx.x, n = *cnt;
+    if (n <= 0) return;  // no row in the backbone any more: the GEMM returns before it reads an operand
     uint2 *hi = reinterpret_cast<uint2 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint2 *>(xlo + (size_t)i * K);
     const int nv = K >> 2;
     if (i >= n) {
@@ -247,6 +248,7 @@ struct TcArgs {
     int qkv_q_tiles, qkv_k_tiles;  // QKV: tiles per matrix (0 otherwise)
     const int32_t *rows;   // step row id of operand row n
     const int32_t *cnt;    // live operand rows (device)
+    const int32_t *hint;   // a count of those rows that is never too low: 0 means there are certainly none
     int *dev_err;
 };
 
@@ -267,7 +269,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     const int ld = NP + 1;
     uint64_t *bars = reinterpret_cast<uint64_t *>(stages + (size_t)S * stage_bytes);  // full[S], empty[S], acc
     __shared__ uint32_t s_tmem;
-    __shared__ int s_abort;
+    __shared__ int s_abort, s_some;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tile_idx = blockIdx.x / a.splits, split = blockIdx.x % a.splits;
     const int kb_total = a.K / kTcBK;
@@ -277,6 +279,12 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     while ((int)tmem_cols < NP) tmem_cols <<= 1;
 
     pdl_launch();
+    if (tid == 0) s_some = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
+    __syncthreads();
+    if (!s_some) {  // every row has left the backbone: nothing to fetch, nothing to compute (uniform over the cluster:
+        pdl_wait();  // the hint only changes between layers); still order this grid behind its predecessor
+        return;
+    }
     if (tid == 0) {
         s_abort = 0;
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars[s]), 1); mbar_init(smem_u32(&bars[S + s]), 1); }

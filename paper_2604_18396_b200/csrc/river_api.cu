@@ -17,6 +17,7 @@
 #include <cstdlib>
 #include "gemm_tc.cuh"
 #include "decode_chain.cuh"
+#include "gemm_tc_w4.cuh"
 
 using namespace river;
 
@@ -65,6 +66,8 @@ struct river_ctx {
     bool tc_ok = false;
     struct LayerMaps { CUtensorMap q, k, v, o, g, u, d; };
     std::vector<LayerMaps> tc_maps;
+    std::vector<LayerMaps> w4_maps;  // code matrices of the exit layers (u8 [rows][K/2], 128-byte boxes)
+    bool w4tc_ok = false;
     CUtensorMap tc_map_head;
     struct BMap { int K, np; CUtensorMap hi, lo; };
     std::vector<BMap> tc_bmaps;
@@ -394,6 +397,19 @@ bool make_map_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t ro
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// u8 code matrix [rows][inner_bytes] -> tiled map with a (box_rows x 128 byte) box and the 128-byte swizzle
+bool make_map_codes(CUtensorMap *m, const void *base, uint64_t inner_bytes, uint64_t rows, uint32_t box_rows) {
+    TmapEncodeFn fn = tmap_encoder();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {inner_bytes, rows};
+    const cuuint64_t gstride[1] = {inner_bytes};
+    const cuuint32_t box[2] = {128, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ---- tensor-core projection launch
 // The shapes the tensor-core path takes: every output dimension in whole 128-feature tiles.
 bool tc_shape_ok(const river_config &g) {
@@ -414,6 +430,25 @@ bool make_tc_maps(river_ctx *c) {
             return false;
     }
     return make_map_bf16(&c->tc_map_head, c->lm_head, g.d, g.V, 128);
+}
+// The exit layers' code matrices for the dequantising tensor-core kernel: one scale / zero per row and 64-input
+// k-block, raw tiles of 256 inputs.
+bool make_w4_maps(river_ctx *c) {
+    const river_config &g = c->cfg;
+    const int qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
+    if (g.group != 64 || g.d % 256 || g.F % 256 || qdim % 256) return false;
+    c->w4_maps.resize(g.L);
+    for (int l = 0; l < g.L; ++l) {
+        const river_layer_weights &w = c->layers[l];
+        if (!w.rq.codes) continue;
+        river_ctx::LayerMaps &m = c->w4_maps[l];
+        if (!make_map_codes(&m.q, w.rq.codes, g.d / 2, qdim, 128) || !make_map_codes(&m.k, w.rk.codes, g.d / 2, kvdim, 128) ||
+            !make_map_codes(&m.v, w.rv.codes, g.d / 2, kvdim, 128) || !make_map_codes(&m.o, w.ro.codes, qdim / 2, g.d, 128) ||
+            !make_map_codes(&m.g, w.rg.codes, g.d / 2, g.F, 64) || !make_map_codes(&m.u, w.ru.codes, g.d / 2, g.F, 64) ||
+            !make_map_codes(&m.d, w.rd.codes, g.F / 2, g.d, 128))
+            return false;
+    }
+    return true;
 }
 const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
     for (auto &b : c->tc_bmaps)
@@ -441,7 +476,7 @@ int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots) {
 template <class Epi>
 cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
                       int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                      const int32_t *cnt, const Epi &epi, bool allow_split = true) {
+                      const int32_t *cnt, const Epi &epi, bool allow_split = true, const int32_t *hint = nullptr) {
     const int np = (n + 15) / 16 * 16;
     const river_ctx::BMap *bm = tc_bmap(c, K, np);
     if (!bm) return cudaErrorInvalidValue;
@@ -460,6 +495,7 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
     if (!allow_split) a.splits = 1;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     a.rows = rows; a.cnt = cnt; a.dev_err = c->dev_err;
+    a.hint = hint ? hint : cnt;
     const size_t smem = tc_smem_bytes(np, a.n_stages);
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
@@ -468,6 +504,43 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
     }
     return launch_kc(tc_gemm_kernel<Epi>, dim3(tiles * a.splits), dim3(kTcThreads), smem, c->stream, true, a.splits, a0,
                      a1, a2, bm->hi, bm->lo, a, epi);
+}
+
+// Exit-layer rows through the dequantising tensor-core kernel: m[0..2] are the code maps, w[0..2] the matching
+// scale / zero arrays (one matrix, gate + up, or q + k + v).
+template <class Epi>
+cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
+                         int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
+                         const int32_t *cnt, const int32_t *hint, const Epi &epi) {
+    const int np = (n + 15) / 16 * 16;
+    const river_ctx::BMap *bm = tc_bmap(c, K, np);
+    if (!bm) return cudaErrorInvalidValue;
+    cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np), dim3(256), 0, c->stream, true, in, rows, cnt, K,
+                             reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(c->tc_xlo));
+    if (e != cudaSuccess) return e;
+    ++c->st.launches_last_step;
+    TcW4Args a{};
+    a.K = K; a.n_pad = np;
+    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
+    const size_t raw = (size_t)kW4RawBufs * kW4RawBytes;
+    // two CTAs per SM (16 dequantisation warps) when two operand stages fit in half of the shared memory
+    const bool two = 2 * stage + raw + 4096 <= 110 * 1024;
+    a.n_stages = two ? (int)std::min<size_t>(4, (110 * 1024 - raw - 4096) / stage)
+                     : (int)std::max<size_t>(2, std::min<size_t>(6, (214 * 1024 - raw) / stage));
+    a.splits = tc_pick_splits(c, tiles, K / (kTcBK * kW4Super), c->num_sms * (two ? 2 : 1));
+    const size_t tile_b = sizeof(float) * (size_t)kTcBM * (np + 1);
+    while (a.splits > 1 && tile_b + tile_b / a.splits + 4096 > (size_t)a.n_stages * stage + raw) --a.splits;
+    a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
+    for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
+    a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
+    const size_t smem = tc_w4_smem_bytes(np, a.n_stages);
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaFuncSetAttribute(tc_gemm_w4_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_smem = smem;
+    }
+    return launch_kc(tc_gemm_w4_kernel<Epi>, dim3(tiles * a.splits), dim3(kW4Threads), smem, c->stream, true, a.splits,
+                     *m[0], *m[1], *m[2], bm->hi, bm->lo, a, epi);
 }
 
 // 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
@@ -636,6 +709,8 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         // kernel only serves the exit-layer rows of the same launch slot.
         const bool tc = c->tc_ok && n >= 5 && n <= c->tc_max_pad;
         const river_ctx::LayerMaps *tm = tc ? &c->tc_maps[l - 1] : nullptr;
+        const river_ctx::LayerMaps *wm = (tc && c->w4tc_ok && has_river) ? &c->w4_maps[l - 1] : nullptr;
+        const int32_t *nrh = c->n_riv + std::max(0, l - 2);  // never above the count entering this block
         const int skip_bb = tc ? 1 : 0;
         // ---- a2: attention norm + QKV + RoPE + KV write
         {
@@ -650,9 +725,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             if (tc) {
                 TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
                 note(launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM,
-                               kvdim / kTcBM, ai, na, e));
+                               kvdim / kTcBM, ai, na, e, true, c->hint_act));
             }
-            if (!tc || has_river)
+            if (wm) {
+                TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
+                const CUtensorMap *const cm[3] = {&wm->q, &wm->k, &wm->v};
+                const river_w4 *const cw[3] = {&w.rq, &w.rk, &w.rv};
+                note(launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ri, nr, nrh, e));
+            } else if (!tc || has_river)
                 note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, skip_bb));
         }
         // ---- a3: paged GQA decode attention
@@ -670,9 +750,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             const ProjIn in{c->obuf, nullptr, 0.f};
             if (tc) {
                 TcResidEpi e{h_in, h_mid, d};
-                note(launch_tc(c, in, tm->o, tm->o, tm->o, qdim, d / kTcBM, n, 0, 0, 0, ai, na, e));
+                note(launch_tc(c, in, tm->o, tm->o, tm->o, qdim, d / kTcBM, n, 0, 0, 0, ai, na, e, true, c->hint_act));
             }
-            if (!tc || has_river)
+            if (wm) {
+                TcResidEpi e{h_in, h_mid, d};
+                const CUtensorMap *const cm[3] = {&wm->o, &wm->o, &wm->o};
+                const river_w4 *const cw[3] = {&w.ro, &w.ro, &w.ro};
+                note(launch_tc_w4(c, in, cm, cw, qdim, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
+            } else if (!tc || has_river)
                 note(launch_stream(c, p, in, rl, qdim, d / 2, n, has_river, tc || !(g.flags & RIVER_F_SIMPLE_ATTN), skip_bb));
         }
         // ---- a5: FFN norm + gate/up + SwiGLU
@@ -685,9 +770,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
             if (tc) {
                 TcGateUpEpi e{c->act, g.F};
-                note(launch_tc(c, in, tm->g, tm->u, tm->u, d, g.F / 64, n, 1, 0, 0, ai, na, e));
+                note(launch_tc(c, in, tm->g, tm->u, tm->u, d, g.F / 64, n, 1, 0, 0, ai, na, e, true, c->hint_act));
             }
-            if (!tc || has_river) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb));
+            if (wm) {
+                TcGateUpEpi e{c->act, g.F};
+                const CUtensorMap *const cm[3] = {&wm->g, &wm->u, &wm->u};
+                const river_w4 *const cw[3] = {&w.rg, &w.ru, &w.ru};
+                note(launch_tc_w4(c, in, cm, cw, d, g.F / 64, n, 1, 0, 0, ri, nr, nrh, e));
+            } else if (!tc || has_river) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb));
         }
         // ---- a5: down projection + residual
         {
@@ -699,9 +789,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             const ProjIn in{c->act, nullptr, 0.f};
             if (tc) {
                 TcResidEpi e{h_mid, h_out, d};
-                note(launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e));
+                note(launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e, true, c->hint_act));
             }
-            if (!tc || has_river) note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb));
+            if (wm) {
+                TcResidEpi e{h_mid, h_out, d};
+                const CUtensorMap *const cm[3] = {&wm->d, &wm->d, &wm->d};
+                const river_w4 *const cw[3] = {&w.rd, &w.rd, &w.rd};
+                note(launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
+            } else if (!tc || has_river) note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb));
         }
         // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
         {
@@ -993,6 +1088,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     c->num_sms = prop.multiProcessorCount;
     if (make_kv_tensor_map(c)) { river_destroy(c); return RIVER_E_DEVICE; }
     c->tc_ok = !(cfg->flags & RIVER_F_NO_TC) && tc_shape_ok(*cfg) && make_tc_maps(c);
+    c->w4tc_ok = c->tc_ok && !(cfg->flags & RIVER_F_NO_W4TC) && make_w4_maps(c);
     c->chain_ok = chain_setup(c);
     for (int i = 0; i < kStaging; ++i) {
         if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");

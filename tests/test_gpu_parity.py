@@ -131,8 +131,11 @@ def test_launch_modes_agree_with_oracle(flags):
     assert r["n_early"] > 0
 
 
-def test_mini8_head_dim_128_gqa4():
-    r = run_scheduled(model("mini8"), [70, 16, 31, 48, 5], 18, "uniform", prefill_exit=3, page_seed=7)
+@pytest.mark.parametrize("flags", [0, 16, 2])
+def test_mini8_head_dim_128_gqa4(flags):
+    # five rows: backbone rows on the tcgen05 GEMM; exit-layer rows on the dequantising tcgen05 GEMM (0), on the
+    # CUDA-core kernel (16), everything on CUDA cores (2)
+    r = run_scheduled(model("mini8"), [70, 16, 31, 48, 5], 18, "uniform", prefill_exit=3, page_seed=7, flags=flags)
     assert r["n_early"] > 0
     print(r)
 
