@@ -997,7 +997,13 @@ int run_chain(river_ctx *c, int n, int n_head, int N, const int32_t *row_pos_hos
 // One decode step through a CUDA graph of the launch sequence (captured the second time a row count is seen; the
 // per-step inputs live in device memory, so the graph never needs new parameters).
 int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
-    if (const int N = chain_rows_per_pass(c, n)) return run_chain(c, n, n, N, row_pos_host);
+    if (const int N = chain_rows_per_pass(c, n)) {
+        const int rc = run_chain(c, n, n, N, row_pos_host);
+        if (rc != RIVER_E_DEVICE || cudaPeekAtLastError() != cudaSuccess) return rc;
+        // the cooperative launch was refused (co-residency cannot be guaranteed in this context): use the
+        // one-kernel-per-stage plan from now on; its first kernel redoes the step prologue
+        c->chain_ok = false;
+    }
     const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
     if (!use_graph) return run_rows(c, n, n, row_pos_host);
     for (auto &ge : c->graphs)
