@@ -98,8 +98,8 @@ __device__ __forceinline__ bool chain_grid_sync(unsigned *bar, unsigned &target,
     target += gridDim.x;
     __syncthreads();
     if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(bar, 1u);
+        // release: the CTA's writes (ordered before this thread by the barrier above) become visible before the count
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
         unsigned it = 0;
         for (;;) {
             unsigned v;
@@ -116,7 +116,6 @@ __device__ __forceinline__ bool chain_grid_sync(unsigned *bar, unsigned &target,
                 break;
             }
         }
-        __threadfence();
     }
     __syncthreads();
     return *s_dead == 0;
@@ -463,9 +462,54 @@ __device__ __forceinline__ float chain_ex2(float x) {
     return y;
 }
 
+// Raw K and V bits of one cached position for this lane's DH / 32 head dims.
+template <int VE>
+__device__ __forceinline__ void attn_load_raw(const KvAddr &kv, int page, int kvh, int p, int lane, uint2 &k, uint2 &v) {
+    const __nv_bfloat16 *kp = kv.pool + kv.base(page, 0, kvh, p % kPage) + lane * VE;
+    const __nv_bfloat16 *vp = kv.pool + kv.base(page, 1, kvh, p % kPage) + lane * VE;
+    if constexpr (VE == 4) {
+        k = __ldcg(reinterpret_cast<const uint2 *>(kp));
+        v = __ldcg(reinterpret_cast<const uint2 *>(vp));
+    } else {
+        k = make_uint2(__ldcg(reinterpret_cast<const uint32_t *>(kp)), 0u);
+        v = make_uint2(__ldcg(reinterpret_cast<const uint32_t *>(vp)), 0u);
+    }
+}
+
+// The cached positions of this warp's first batch of the CTA's first work item, requested BEFORE the grid barrier
+// that ends the QKV phase: everything but the position written in this very step is already in the cache.
+struct AttnPre {
+    uint2 k[4], v[4];
+    unsigned mask;  // bit u: position u of the batch is in k[u], v[u]
+};
+template <int DH>
+__device__ __forceinline__ void chain_attention_preload(const ChainArgs &a, const KvAddr &kv, int n_rows, int S, int chunk,
+                                                        AttnPre &pre) {
+    constexpr int VE = DH / 32, U = 4;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pre.mask = 0u;
+    const int item = blockIdx.x;
+    if (item >= n_rows * a.Hkv * S) return;
+    const int sp = item % S, kvh = (item / S) % a.Hkv, row = item / (S * a.Hkv);
+    const int pos = kv.row_pos[row], slot = kv.row_slot[row];
+    const int p0 = sp * chunk, p1 = min(pos + 1, p0 + chunk);
+    const int pb = p0 + warp * U;
+    if (pb >= p1) return;
+    const int page = kv.page_tbl[(size_t)slot * kv.max_pages_per_seq + pb / kPage];
+    if (page < 0 || page >= kv.n_pages) return;  // the attention phase itself reports it
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int p = pb + u;
+        if (p < p1 && p != pos) {
+            attn_load_raw<VE>(kv, page, kvh, p, lane, pre.k[u], pre.v[u]);
+            pre.mask |= 1u << u;
+        }
+    }
+}
+
 template <int DH, int GQ>
 __device__ __forceinline__ void chain_attention(const ChainArgs &a, const KvAddr &kv, int n_rows, int S, int chunk,
-                                                float *sm, ChainFlags *fl) {
+                                                float *sm, ChainFlags *fl, const AttnPre &pre) {
     constexpr int VE = DH / 32, U = 4, NW = kChainWarps;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float *s_m = sm, *s_l = sm + NW * GQ, *s_acc = sm + 2 * NW * GQ;  // [NW][GQ], [NW][GQ], [NW][GQ][DH]
@@ -480,11 +524,16 @@ __device__ __forceinline__ void chain_attention(const ChainArgs &a, const KvAddr
         for (int g = 0; g < GQ; ++g) {
             m[g] = -CUDART_INF_F;
             l[g] = 0.f;
-#pragma unroll
-            for (int e = 0; e < VE; ++e) {
-                qr[g][e] = __ldcg(a.qbuf + (size_t)row * Hq * DH + (size_t)(kvh * GQ + g) * DH + lane * VE + e) * a.qscale;
-                acc[g][e] = 0.f;
+            const float *qp = a.qbuf + (size_t)row * Hq * DH + (size_t)(kvh * GQ + g) * DH + lane * VE;
+            if constexpr (VE == 4) {
+                const float4 q4 = __ldcg(reinterpret_cast<const float4 *>(qp));
+                qr[g][0] = q4.x * a.qscale; qr[g][1] = q4.y * a.qscale; qr[g][2] = q4.z * a.qscale; qr[g][3] = q4.w * a.qscale;
+            } else {
+                const float2 q2 = __ldcg(reinterpret_cast<const float2 *>(qp));
+                qr[g][0] = q2.x * a.qscale; qr[g][1] = q2.y * a.qscale;
             }
+#pragma unroll
+            for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
         }
         const int32_t *pt = kv.page_tbl + (size_t)slot * kv.max_pages_per_seq;
         for (int pb = p0 + warp * U; pb < p1; pb += NW * U) {  // pb is a multiple of 4: one page per batch
@@ -494,22 +543,19 @@ __device__ __forceinline__ void chain_attention(const ChainArgs &a, const KvAddr
                 page = 0;
             }
             float kf[U][VE], vf[U][VE];
+            const bool first = item == (int)blockIdx.x && pb == p0 + warp * U;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int p = pb + u;
                 if (p < p1) {
-                    const __nv_bfloat16 *kp = kv.pool + kv.base(page, 0, kvh, p % kPage) + lane * VE;
-                    const __nv_bfloat16 *vp = kv.pool + kv.base(page, 1, kvh, p % kPage) + lane * VE;
+                    uint2 kr, vr;
+                    if (first && ((pre.mask >> u) & 1u)) { kr = pre.k[u]; vr = pre.v[u]; }
+                    else attn_load_raw<VE>(kv, page, kvh, p, lane, kr, vr);
+                    kf[u][0] = bf16lo(kr.x); kf[u][1] = bf16hi(kr.x);
+                    vf[u][0] = bf16lo(vr.x); vf[u][1] = bf16hi(vr.x);
                     if constexpr (VE == 4) {
-                        const uint2 kr = __ldcg(reinterpret_cast<const uint2 *>(kp));
-                        const uint2 vr = __ldcg(reinterpret_cast<const uint2 *>(vp));
-                        kf[u][0] = bf16lo(kr.x); kf[u][1] = bf16hi(kr.x); kf[u][2] = bf16lo(kr.y); kf[u][3] = bf16hi(kr.y);
-                        vf[u][0] = bf16lo(vr.x); vf[u][1] = bf16hi(vr.x); vf[u][2] = bf16lo(vr.y); vf[u][3] = bf16hi(vr.y);
-                    } else {
-                        const uint32_t kr = __ldcg(reinterpret_cast<const uint32_t *>(kp));
-                        const uint32_t vr = __ldcg(reinterpret_cast<const uint32_t *>(vp));
-                        kf[u][0] = bf16lo(kr); kf[u][1] = bf16hi(kr);
-                        vf[u][0] = bf16lo(vr); vf[u][1] = bf16hi(vr);
+                        kf[u][2] = bf16lo(kr.y); kf[u][3] = bf16hi(kr.y);
+                        vf[u][2] = bf16lo(vr.y); vf[u][3] = bf16hi(vr.y);
                     }
                 } else {
 #pragma unroll
@@ -757,11 +803,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         // ---- a2
         chain_project<QkvProblem, N>(a, pq, ProjIn{h_in, w.attn_norm, a.eps}, fl.act, na, fl.riv, nr, sm,
                                      [&]() { chain_prefetch<ResidProblem, R>(po, act, riv, a.pf_bytes); }, &fl.next, probe, 0);
+        AttnPre apre;
+        chain_attention_preload<DH>(a, pq.kv, n, S, chunk, apre);  // cached positions travel across the barrier
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
         probe.mark(3);
         if (stamp) a.stamps[si++] = chain_now();
         // ---- a3
-        chain_attention<DH, GQ>(a, pq.kv, n, S, chunk, sm.xs, &fl);
+        chain_attention<DH, GQ>(a, pq.kv, n, S, chunk, sm.xs, &fl, apre);
         probe.mark(32);
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
         probe.mark(35);
