@@ -419,14 +419,14 @@ struct ChainSmem {
 template <class P, int N, class PF>
 __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, const ProjIn &in, const int *s_act, int na,
                                               const int *s_riv, int nr, const ChainSmem &sm, PF &&prefetch_next,
-                                              int *s_next, ChainProbe &probe, int pk) {
+                                              int *s_next, ChainProbe &probe, int pk, bool prestaged = false) {
     constexpr int R = kChainR;
     const int K = p.K;
     const int xstride = xs_stride(K, 32);
     const int passes_a = (na + N - 1) / N, passes_r = (nr + N - 1) / N;
     for (int ps = 0; ps < passes_a; ++ps) {
         const int i0 = ps * N;
-        stream_load_rows<N, 8>(in, s_act, i0, na, K, xstride, sm.xs, sm.xsum, sm.red);
+        if (!(prestaged && ps == 0)) stream_load_rows<N, 8>(in, s_act, i0, na, K, xstride, sm.xs, sm.xsum, sm.red);
         probe.mark(pk);
         chain_stream<P, N, R, false>(p, sm.xs, sm.xsum, xstride, sm.part, a.part_cap, a.dev_err,
                                      ps + 1 == passes_a && passes_r == 0, prefetch_next,
@@ -436,7 +436,7 @@ __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, co
     }
     for (int ps = 0; ps < passes_r; ++ps) {
         const int i0 = ps * N;
-        stream_load_rows<N, 32>(in, s_riv, i0, nr, K, xstride, sm.xs, sm.xsum, sm.red);
+        if (!(prestaged && ps == 0 && passes_a == 0)) stream_load_rows<N, 32>(in, s_riv, i0, nr, K, xstride, sm.xs, sm.xsum, sm.red);
         probe.mark(pk + 4);
         chain_stream<P, N, R, true>(p, sm.xs, sm.xsum, xstride, sm.part, a.part_cap, a.dev_err, ps + 1 == passes_r,
                                     prefetch_next, [&](int t, int n, const float(&res)[R]) {
@@ -454,6 +454,11 @@ __device__ __forceinline__ void chain_project(const ChainArgs &a, const P &p, co
 struct ChainFlags {
     int exited[4], act[4], riv[4], pass[4];
     int na, nr, dead, flag, next;
+    // per-step constants of the decision, read once (the per-layer decision then touches no global memory to decide)
+    float tau[4];
+    int forced[4];
+    float *scores;
+    int32_t *exit_layer;
 };
 
 __device__ __forceinline__ float chain_ex2(float x) {
@@ -664,7 +669,7 @@ __device__ __forceinline__ void chain_decide(const ChainArgs &a, int l, const fl
                                              float *red, ChainFlags *fl) {
     const int L = a.L, d = a.d;
     const bool eligible = (l >= 1) && (l >= a.entry_layer) && (l < L);
-    float *scores = a.meta->scores;
+    float *scores = fl->scores;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int row = 0; row < n; ++row) {
         if (fl->exited[row] != 0 || !(eligible || scores)) continue;  // uniform across the CTA
@@ -686,13 +691,12 @@ __device__ __forceinline__ void chain_decide(const ChainArgs &a, int l, const fl
             for (int w = 0; w < kChainWarps; ++w) { ab += red[w]; aa += red[32 + w]; bb += red[64 + w]; }
             float s = 0.f;
             if (aa > 0.f && bb > 0.f) s = ab / (sqrtf(aa) * sqrtf(bb));
-            fl->pass[row] = (s > a.meta->tau[row]) ? 1 : 0;
+            fl->pass[row] = (s > fl->tau[row]) ? 1 : 0;
             if (scores && blockIdx.x == 0) scores[(size_t)row * L + (l - 1)] = s;
         }
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        const int32_t *forced = a.meta->forced;
         int allpass = 1;
         if (a.exit_mode == 1)
             for (int b = 0; b < n; ++b)
@@ -701,11 +705,11 @@ __device__ __forceinline__ void chain_decide(const ChainArgs &a, int l, const fl
         for (int b = 0; b < n; ++b) {
             if (fl->exited[b] == 0) {
                 bool leave = eligible && (a.exit_mode == 1 ? (allpass != 0) : (fl->pass[b] != 0));
-                const int f = forced ? forced[b] : -1;
+                const int f = fl->forced[b];
                 if (f >= 0) leave = (f == l) && (l < L);
                 if (leave) {
                     fl->exited[b] = 1;
-                    if (blockIdx.x == 0) { a.meta->exit_layer[b] = l; a.exited[b] = 1; }
+                    if (blockIdx.x == 0) { fl->exit_layer[b] = l; a.exited[b] = 1; }
                 }
             }
             if (fl->exited[b] == 0) fl->act[na++] = b;
@@ -722,6 +726,147 @@ __device__ __forceinline__ void chain_decide(const ChainArgs &a, int l, const fl
         }
     }
     __syncthreads();
+}
+
+// ---------------------------------------------------------------- a6 + a7 fused with the next block's first staging
+// The block output that Eq. 1 scores is also the input of the next block's attention norm: one pass loads it
+// (and the block input of the rows that still need a score), yields dot product, both squared norms (the second
+// is the RMS statistic), takes the decision, and writes the normalised rows of the next QKV phase's first pass
+// straight from registers.  Returns false (and falls back to chain_decide) when a row does not fit in two 128-bit
+// values per thread.
+template <int N>
+__device__ __forceinline__ bool chain_decide_stage(const ChainArgs &a, int l, const float *h_in, const float *h_out, int n,
+                                                   const uint16_t *gain_next, const ChainSmem &sm, ChainFlags *fl) {
+    const int L = a.L, d = a.d, nv = d >> 2;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    if (nv > 2 * nthr) {
+        chain_decide(a, l, h_in, h_out, n, sm.red, fl);
+        return false;
+    }
+    const bool eligible = (l >= 1) && (l >= a.entry_layer) && (l < L);
+    float *scores = fl->scores;
+    float4 v[N][2];  // the step has at most N rows
+    float ab[N], aa[N], bb[N];
+#pragma unroll
+    for (int b = 0; b < N; ++b) {
+        ab[b] = aa[b] = bb[b] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) v[b][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (b < n) {
+            const bool need = fl->exited[b] == 0 && (eligible || scores);  // uniform across the CTA
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int i = tid + k * nthr;
+                if (i < nv) {
+                    const float4 y = __ldcg(reinterpret_cast<const float4 *>(h_out + (size_t)b * d) + i);
+                    v[b][k] = y;
+                    bb[b] += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+                    if (need) {
+                        const float4 x = __ldcg(reinterpret_cast<const float4 *>(h_in + (size_t)b * d) + i);
+                        ab[b] += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
+                        aa[b] += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                    }
+                }
+            }
+        }
+    }
+    float *red = sm.red;  // [3][4][kChainWarps]
+#pragma unroll
+    for (int b = 0; b < N; ++b) {
+        if (b < n) {
+            const float sab = warp_sum(ab[b]), saa = warp_sum(aa[b]), sbb = warp_sum(bb[b]);
+            if (lane == 0) {
+                red[(0 * 4 + b) * kChainWarps + warp] = sab;
+                red[(1 * 4 + b) * kChainWarps + warp] = saa;
+                red[(2 * 4 + b) * kChainWarps + warp] = sbb;
+            }
+        }
+    }
+    __syncthreads();
+    float bbt[N];
+#pragma unroll
+    for (int b = 0; b < N; ++b) {
+        bbt[b] = 0.f;
+        if (b < n)
+            for (int w = 0; w < kChainWarps; ++w) bbt[b] += red[(2 * 4 + b) * kChainWarps + w];
+    }
+    if (tid == 0) {
+        for (int b = 0; b < n; ++b) {
+            fl->pass[b] = 0;
+            if (fl->exited[b] == 0 && (eligible || scores)) {
+                float tab = 0.f, taa = 0.f;
+                for (int w = 0; w < kChainWarps; ++w) { tab += red[(0 * 4 + b) * kChainWarps + w]; taa += red[(1 * 4 + b) * kChainWarps + w]; }
+                float sc = 0.f;
+                if (taa > 0.f && bbt[b] > 0.f) sc = tab / (sqrtf(taa) * sqrtf(bbt[b]));
+                fl->pass[b] = (sc > fl->tau[b]) ? 1 : 0;
+                if (scores && blockIdx.x == 0) scores[(size_t)b * L + (l - 1)] = sc;
+            }
+        }
+        int allpass = 1;
+        if (a.exit_mode == 1)
+            for (int b = 0; b < n; ++b)
+                if (fl->exited[b] == 0 && !(eligible && fl->pass[b])) allpass = 0;
+        int na = 0, nr = 0;
+        for (int b = 0; b < n; ++b) {
+            if (fl->exited[b] == 0) {
+                bool leave = eligible && (a.exit_mode == 1 ? (allpass != 0) : (fl->pass[b] != 0));
+                const int f = fl->forced[b];
+                if (f >= 0) leave = (f == l) && (l < L);
+                if (leave) {
+                    fl->exited[b] = 1;
+                    if (blockIdx.x == 0) { fl->exit_layer[b] = l; a.exited[b] = 1; }
+                }
+            }
+            if (fl->exited[b] == 0) fl->act[na++] = b;
+            else fl->riv[nr++] = b;
+        }
+        fl->na = na;
+        fl->nr = nr;
+        if (blockIdx.x == 0) {
+            int32_t *A = a.lists.act_idx + (size_t)l * a.lists.max_batch, *R = a.lists.riv_idx + (size_t)l * a.lists.max_batch;
+            for (int i = 0; i < na; ++i) A[i] = fl->act[i];
+            for (int i = 0; i < nr; ++i) R[i] = fl->riv[i];
+            a.lists.n_act[l] = na;
+            a.lists.n_riv[l] = nr;
+        }
+    }
+    __syncthreads();
+    if (l >= L) return false;  // the LM head stages its own rows
+    // ---- first pass of the next QKV phase: the backbone rows if any are left, else the exit-layer rows
+    const bool bf = fl->na > 0;
+    const int *list = bf ? fl->act : fl->riv;
+    const int len = bf ? fl->na : fl->nr;
+    const int xstride = xs_stride(d, 32);
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        float *dst = sm.xs + j * xstride;
+        if (j >= len) {
+            for (int k = tid; k < xstride; k += nthr) dst[k] = 0.f;
+            continue;
+        }
+        const int rowid = list[j];
+        float4 x[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+        float ssq = 0.f;
+#pragma unroll
+        for (int b = 0; b < N; ++b)
+            if (b == rowid) { x[0] = v[b][0]; x[1] = v[b][1]; ssq = bbt[b]; }
+        const float scale = rsqrtf(ssq / (float)d + a.eps);
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int i = tid + k * nthr;
+            if (i < nv) {
+                const uint2 gw = *reinterpret_cast<const uint2 *>(gain_next + 4 * i);
+                float4 y = x[k];
+                y.x *= scale * bf16lo(gw.x); y.y *= scale * bf16hi(gw.x);
+                y.z *= scale * bf16lo(gw.y); y.w *= scale * bf16hi(gw.y);
+                if (bf) *reinterpret_cast<float4 *>(dst + xs_index<8>(4 * i)) = y;
+                else *reinterpret_cast<float4 *>(dst + xs_index<32>(4 * i)) = y;
+            }
+        }
+    }
+    __syncthreads();
+    if (!bf) stream_chunk_sums<N>(sm.xs, sm.xsum, d, xstride);
+    return true;
 }
 
 // ---------------------------------------------------------------- a8 inside the chain: LM head as a stream problem
@@ -751,13 +896,14 @@ template <int N, int DH, int GQ>
 __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const ChainArgs a) {
     extern __shared__ __align__(16) float chain_smem[];
     __shared__ ChainFlags fl;
+    __shared__ LayerDev s_layer[2];  // this block's and the next block's weight pointers (fetched one block ahead)
     __shared__ float s_best[kChainWarps];
     __shared__ int s_besti[kChainWarps];
     constexpr int R = kChainR;
     const int Kmax = max(max(a.d, a.F), a.Hq * a.dh);
     ChainSmem sm;
-    sm.red = chain_smem;                                  // 96
-    sm.xsum = chain_smem + 96;                            // N * Kmax / 32
+    sm.red = chain_smem;                                  // 256
+    sm.xsum = chain_smem + 256;                            // N * Kmax / 32
     sm.part = sm.xsum + ((N * (Kmax >> 5) + 3) & ~3);     // kChainWarps * part_cap * R * N
     sm.xs = sm.part + a.part_floats;
     const int n = a.meta->n_rows;
@@ -767,7 +913,11 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         fl.dead = 0;
         fl.flag = 0;
         int na = 0, nr = 0;
+        fl.scores = a.meta->scores;
+        fl.exit_layer = a.meta->exit_layer;
         for (int b = 0; b < n && b < 4; ++b) {
+            fl.tau[b] = a.meta->tau[b];
+            fl.forced[b] = a.meta->forced ? a.meta->forced[b] : -1;
             fl.exited[b] = a.exited[b];
             fl.pass[b] = 0;
             if (fl.exited[b] == 0) fl.act[na++] = b;
@@ -776,6 +926,13 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         fl.na = na;
         fl.nr = nr;
     }
+    {
+        constexpr int kWords = (int)(sizeof(LayerDev) / sizeof(unsigned long long));
+        static_assert(sizeof(LayerDev) % sizeof(unsigned long long) == 0, "LayerDev is copied in 8-byte words");
+        const int t = threadIdx.x - 32;  // warp 1 copies; warp 0's thread 0 is busy above
+        if (t >= 0 && t < kWords) reinterpret_cast<unsigned long long *>(&s_layer[0])[t] = reinterpret_cast<const unsigned long long *>(&a.layers[0])[t];
+        if (t >= 0 && t < kWords && a.L > 1) reinterpret_cast<unsigned long long *>(&s_layer[1])[t] = reinterpret_cast<const unsigned long long *>(&a.layers[1])[t];
+    }
     __syncthreads();
     const bool stamp = a.stamps != nullptr && blockIdx.x == 0 && threadIdx.x == 0;
     int si = 0;
@@ -783,8 +940,9 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
     ChainProbe probe{stamp ? a.sub : nullptr, chain_now()};
     const int S = a.meta->pad[1], chunk = a.meta->pad[0];
     int hi = 0;
+    bool prestaged = false;  // the QKV phase's first rows were staged by the previous block's decision pass
     for (int l = 1; l <= L; ++l) {
-        const LayerDev &w = a.layers[l - 1];
+        const LayerDev &w = s_layer[(l - 1) & 1];
         float *h_in = a.h[hi], *h_mid = a.h[(hi + 1) % 3], *h_out = a.h[(hi + 2) % 3];
         const int na = fl.na, nr = w.has_river ? fl.nr : 0;
         const bool riv = nr > 0, act = na > 0;
@@ -802,7 +960,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
 
         // ---- a2
         chain_project<QkvProblem, N>(a, pq, ProjIn{h_in, w.attn_norm, a.eps}, fl.act, na, fl.riv, nr, sm,
-                                     [&]() { chain_prefetch<ResidProblem, R>(po, act, riv, a.pf_bytes); }, &fl.next, probe, 0);
+                                     [&]() { chain_prefetch<ResidProblem, R>(po, act, riv, a.pf_bytes); }, &fl.next, probe, 0, prestaged);
         AttnPre apre;
         chain_attention_preload<DH>(a, pq.kv, n, S, chunk, apre);  // cached positions travel across the barrier
         if (!chain_grid_sync(a.bar, target, a.dev_err, &fl.dead)) return;
@@ -830,7 +988,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         // makes the bf16 part of that request useless, once per token), or the LM head
         chain_project<ResidProblem, N>(a, pd, ProjIn{a.act, nullptr, 0.f}, fl.act, na, fl.riv, nr, sm, [&]() {
             if (l < L) {
-                const LayerDev &wn = a.layers[l];
+                const LayerDev &wn = s_layer[l & 1];
                 QkvProblem pn = pq;
                 pn.wq = wn.wq; pn.wk = wn.wk; pn.wv = wn.wv; pn.rq = wn.rq; pn.rk = wn.rk; pn.rv = wn.rv;
                 chain_prefetch<QkvProblem, R>(pn, act, wn.has_river && fl.nr > 0, a.pf_bytes);
@@ -843,9 +1001,14 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         probe.mark(27);
         if (stamp) a.stamps[si++] = chain_now();
         // ---- a6 + a7
-        chain_decide(a, l, h_in, h_out, n, sm.red, &fl);
+        prestaged = chain_decide_stage<N>(a, l, h_in, h_out, n, l < L ? s_layer[l & 1].attn_norm : nullptr, sm, &fl);
         probe.mark(36);
         if (stamp) a.stamps[si++] = chain_now();
+        if (l + 1 < L) {  // block l + 2's pointers into the slot block l used (its last reader is behind the barrier above)
+            constexpr int kWords = (int)(sizeof(LayerDev) / sizeof(unsigned long long));
+            const int t = threadIdx.x;
+            if (t < kWords) reinterpret_cast<unsigned long long *>(&s_layer[(l + 1) & 1])[t] = reinterpret_cast<const unsigned long long *>(&a.layers[l + 1])[t];
+        }
         hi = (hi + 2) % 3;
     }
 
@@ -916,7 +1079,7 @@ inline ChainLayout chain_layout(int N, int Kmax, int part_cap, int dh, int gq) {
     const size_t xs = std::max<size_t>((size_t)N * xs_stride(Kmax, 32), (size_t)kChainWarps * gq * (dh + 2));
     l.xs_floats = (int)((xs + 3) & ~(size_t)3);
     l.part_floats = (int)(((size_t)part_cap * kChainR * N + 3) & ~(size_t)3);
-    l.bytes = sizeof(float) * (96 + (((size_t)N * (Kmax >> 5) + 3) & ~(size_t)3) + l.part_floats + l.xs_floats);
+    l.bytes = sizeof(float) * (256 + (((size_t)N * (Kmax >> 5) + 3) & ~(size_t)3) + l.part_floats + l.xs_floats);
     return l;
 }
 

@@ -135,6 +135,25 @@ struct GateUpProblem {  // act[row][f] = silu(Wg[f] . y) * (Wu[f] . y)
 };
 
 
+// Sums of every 32-input chunk of the rows staged in the E = 32 order (all threads of the CTA; ends with a barrier).
+template <int N>
+__device__ __forceinline__ void stream_chunk_sums(const float *xs, float *xsum, int K, int xstride) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int nch = K >> 5;
+    for (int t = tid; t < N * nch; t += nthr) {
+        const int n = t / nch, c = t % nch;
+        const float *xb = xs + n * xstride + (c >> 5) * 1024 + (c & 31) * 4;
+        float sx = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float4 v = *reinterpret_cast<const float4 *>(xb + j * 128);
+            sx += (v.x + v.y) + (v.z + v.w);
+        }
+        xsum[n * nch + c] = sx;
+    }
+    __syncthreads();
+}
+
 // ---------------------------------------------------------------- activation rows -> shared memory
 // All threads of the CTA load up to N rows idx[i0..], optionally RMS-normalise them, and store them fp32 in the
 // lane-interleaved order for E inputs per chunk (8: bf16 weights, 32: 4-bit codes, plus the sums of every chunk).
@@ -186,21 +205,7 @@ __device__ __forceinline__ void stream_load_rows(const ProjIn &in, const int32_t
         }
     }
     __syncthreads();
-    if (E == 32) {
-        const int nch = K >> 5;
-        for (int t = tid; t < N * nch; t += nthr) {
-            const int n = t / nch, c = t % nch;
-            const float *xb = xs + n * xstride + (c >> 5) * 1024 + (c & 31) * 4;
-            float sx = 0.f;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float4 v = *reinterpret_cast<const float4 *>(xb + j * 128);
-                sx += (v.x + v.y) + (v.z + v.w);
-            }
-            xsum[n * nch + c] = sx;
-        }
-        __syncthreads();
-    }
+    if (E == 32) stream_chunk_sums<N>(xs, xsum, K, xstride);
 }
 
 // ---------------------------------------------------------------- one task = R weight rows against N activation rows
