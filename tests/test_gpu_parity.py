@@ -316,6 +316,14 @@ def test_8b_class_batch_rows_on_both_paths():
     print("8b batch:", r)
 
 
+def test_8b_class_six_rows_tensor_core_paths():
+    # from five rows on: backbone rows on the tcgen05 GEMM, exit-layer rows on the dequantising tcgen05 GEMM, at the
+    # full 8B layer shape (cluster K-splits of every projection, 128-head-dim cache writes from the GEMM epilogue)
+    r = run_scheduled(model("8b"), [6, 11, 3, 9, 4, 7], 2, "uniform", max_batch=8, kv_store=1, page_seed=5)
+    assert r["n_early"] > 0
+    print("8b six rows:", r)
+
+
 def test_fp32_cache_oracle_deviation_is_storage_noise():
     # against the oracle with an fp32 cache: direction preserved (cosine bound), max-abs reported
     m = model("8b")
