@@ -441,12 +441,33 @@ def ours(args, wl):
             "value": r["tokens_per_s"], "unit": "tokens/s", "cores": r["threads"], "kind": "oracle",
             "sample": f"{n_or} oracle decode steps after 1 warm-up, {Bs} of {B} rows, {shape_name} shape, context "
                       f"{int(np.mean(pos0))} (synthetic N(0,1) KV history), exits forced at the scheduled layers"}
-    if rank == 0:
-        if "cpu_baseline" not in line:
-            line["cpu_baseline"] = None
-        print(json.dumps(line), flush=True)
+    if rank == 0 and "cpu_baseline" not in line:
+        line["cpu_baseline"] = None
     stream_ctx.__exit__(None, None, None)
     rv.close()
+    # ---- the other launch plan for 1-4 rows (persistent chain kernel), same model, prompt, tokens and thresholds:
+    # printed beside the main numbers, outside every timed region of the main arm
+    if rank == 0 and world == 1 and B <= 4 and not (flags & 8) and not args.no_variant:
+        cfg2 = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=n_pages, max_batch=max(B, 8),
+                           page_shuffle_seed=seed + 1, flags=flags | 8)
+        rv2 = River(cfg2, bb, rvw)
+        with torch.cuda.stream(rv2.stream):
+            rv2.prefill(slots, prompt, offs)
+            K2 = min(K, 64)
+            t0s = n_cal  # same tokens / thresholds as the main arm's timed exit run
+            timed_steps(rv2, slots_c, slots, toks, inf, logits, nxt, exits, 0, n_cal)
+            timed_steps(rv2, slots_c, slots, toks, taus, logits, nxt, exits, t0s, W)
+            ms_x = timed_steps(rv2, slots_c, slots, toks, taus, logits, nxt, exits, t0s + W, K2)
+            timed_steps(rv2, slots_c, slots, toks, inf, logits, nxt, exits, t0s + W + K2, W)
+            ms_f = timed_steps(rv2, slots_c, slots, toks, inf, logits, nxt, exits, t0s + 2 * W + K2, K2)
+        rv2.close()
+        line["chain_kernel_variant"] = {
+            "flags": flags | 8, "steps": K2, "ms_per_step": ms_x / K2, "tokens_per_s": B * K2 / (ms_x / 1e3),
+            "full_depth_ms_per_step": ms_f / K2,
+            "full_depth_frac_of_measured_peak": bytes_full / (ms_f / K2 * 1e-3) / 1e9 / peak,
+            "note": "steps of 1-4 rows as ONE cooperative launch (river_config.flags | 8)"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
 
 
 def main():
@@ -456,8 +477,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b_b1", choices=sorted(WORKLOADS))
-    ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
+    ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay, 8 = persistent chain kernel for 1-4 rows)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variant", action="store_true", help="skip the chain-kernel variant measured beside the main arm")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")
     ap.add_argument("--prompt", type=int, default=0, help="profiling aid: override the prompt length")
     args = ap.parse_args()

@@ -48,7 +48,8 @@ enum {
     RIVER_F_GRAPH = 1,   /* replay each decode step as a CUDA graph (captured on first use) */
     RIVER_F_NO_TC = 2,   /* run every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
     RIVER_F_SIMPLE_ATTN = 4, /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
-    RIVER_F_NO_CHAIN = 8,    /* steps of 1-4 rows as separate kernels per stage instead of the persistent chain kernel */
+    RIVER_F_CHAIN = 8,       /* steps of 1-4 rows through the persistent chain kernel (one cooperative launch for all
+                                layers and the LM head) instead of one kernel per stage */
     RIVER_F_NO_W4TC = 16     /* exit-layer rows of batches on the CUDA-core kernel instead of the dequantising tcgen05 GEMM */
     /* bits 8-15: tuning aid for the chain kernel, KiB of the next phase's weights each warp requests from the L2
        ahead of time (0 = default 4) */

@@ -897,7 +897,7 @@ int chain_rows_per_pass(const river_ctx *c, int n) {
 
 bool chain_setup(river_ctx *c) {
     const river_config &g = c->cfg;
-    if (g.flags & RIVER_F_NO_CHAIN) return false;
+    if (!(g.flags & RIVER_F_CHAIN)) return false;
     if (g.V % 2 || g.d % 4 || g.F % 2) return false;
     if (!chain_kernel_for(1, g.dh, g.Hq / g.Hkv)) return false;
     int dev = 0, coop = 0;

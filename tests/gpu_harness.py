@@ -54,6 +54,9 @@ class StepOut:
     scores: np.ndarray
 
 
+EXTRA_FLAGS = 0  # OR-ed into every context's river_config.flags (the parity tests run under both launch plans)
+
+
 class Pair:
     """An oracle and a CUDA context over the same model, fed the same tokens."""
 
@@ -66,7 +69,7 @@ class Pair:
         cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
                           n_pages=max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
                           entry_layer=entry_layer, exit_mode=exit_mode, page_shuffle_seed=page_shuffle_seed,
-                          flags=flags)
+                          flags=flags | EXTRA_FLAGS)
         self.gpu = River(cfg, bb_g, rv_g)
         self.entry = self.shape.entry_layer if entry_layer is None else entry_layer
         self.V = self.shape.V

@@ -31,6 +31,16 @@ def model(name, n_layers=None, identity=False):
     return _models[key]
 
 
+@pytest.fixture(autouse=True, params=[0, 8], ids=["stage-kernels", "chain-kernel"])
+def launch_plan(request):
+    """Every test runs twice: steps of 1-4 rows as one kernel per stage (default), and through the persistent chain
+    kernel (flag 8).  Steps of five or more rows take the same tensor-core kernels either way."""
+    import tests.gpu_harness as gh
+    gh.EXTRA_FLAGS = request.param
+    yield
+    gh.EXTRA_FLAGS = 0
+
+
 def toks(shape, n, stream):
     return synth.tokens(shape.seed, stream, n, shape.V).numpy()
 
@@ -125,8 +135,8 @@ def test_tiny_geometric_exits_and_wide_batch():
 
 @pytest.mark.parametrize("flags", [0, 1, 2, 4, 5, 8, 9, 12])
 def test_launch_modes_agree_with_oracle(flags):
-    # 1: CUDA-graph replay; 2: no tensor-core projections; 4: plain attention kernel; 8: separate kernels per stage
-    # instead of the persistent chain kernel (three rows: the chain kernel takes the step unless 8 is set)
+    # 1: CUDA-graph replay; 2: no tensor-core projections; 4: plain attention kernel; 8: the persistent chain kernel
+    # (three rows per step: the chain kernel takes them when 8 is set, by the parameter or by the fixture)
     r = run_scheduled(model("mini8"), [37, 16, 3], 6, "uniform", page_seed=11, flags=flags, max_batch=4)
     assert r["n_early"] > 0
 
