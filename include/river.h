@@ -50,7 +50,8 @@ enum {
     RIVER_F_SIMPLE_ATTN = 4, /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
     RIVER_F_CHAIN = 8,       /* steps of 1-4 rows through the persistent chain kernel (one cooperative launch for all
                                 layers and the LM head) instead of one kernel per stage */
-    RIVER_F_NO_W4TC = 16     /* exit-layer rows of batches on the CUDA-core kernel instead of the dequantising tcgen05 GEMM */
+    RIVER_F_NO_W4TC = 16,    /* exit-layer rows of batches on the CUDA-core kernel instead of the dequantising tcgen05 GEMM */
+    RIVER_F_TMA_ATTN = 32    /* steps of 1-4 rows through the TMA-fed attention kernel too (default: the small-step kernel) */
     /* bits 8-15: tuning aid for the chain kernel, KiB of the next phase's weights each warp requests from the L2
        ahead of time (0 = default 4) */
 };

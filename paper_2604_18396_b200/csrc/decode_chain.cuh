@@ -661,6 +661,29 @@ __device__ __forceinline__ void chain_attention(const ChainArgs &a, const KvAddr
     }
 }
 
+// ---------------------------------------------------------------- the same attention as a kernel of its own
+// For steps of 1-4 rows in the one-kernel-per-stage plan: one CTA per (row, KV head, split).  The cached positions do
+// of a decode step do not depend on the preceding QKV kernel (it writes only each row's newest position), so they
+// are requested before griddepcontrol.wait; after it only q and the newest position remain.  (Larger steps use the
+// TMA-fed kernel.)
+template <int DH, int GQ>
+__global__ void __launch_bounds__(kChainThreads) attn_small_kernel(const ChainArgs a, int layer0, int early) {
+    extern __shared__ __align__(16) float attn_small_smem[];
+    __shared__ ChainFlags fl;
+    pdl_launch();
+    KvAddr kv = a.kv;
+    kv.layer0 = layer0;
+    const int n = a.meta->n_rows, S = a.meta->pad[1], chunk = a.meta->pad[0];
+    AttnPre pre;
+    pre.mask = 0u;
+    // early: every row of the step belongs to a different sequence (a decode step), so the QKV kernel in flight
+    // writes nothing but each row's newest position.  Prefill chunks hold consecutive positions of one sequence and
+    // must wait.
+    if (early) chain_attention_preload<DH>(a, kv, n, S, chunk, pre);
+    pdl_wait();
+    chain_attention<DH, GQ>(a, kv, n, S, chunk, attn_small_smem, &fl, pre);
+}
+
 // ---------------------------------------------------------------- a6 + a7 inside the chain
 // Eq. 1 for every row still in the backbone, the exit decision and the row lists entering block l + 1.  Every CTA
 // runs this on the same inputs with the same reduction order, so all CTAs hold identical lists; CTA 0 publishes

@@ -76,6 +76,7 @@ struct river_ctx {
     LayerDev *layers_dev = nullptr;
     unsigned long long *chain_stamps = nullptr;
     bool chain_ok = false;
+    bool rows_distinct = true;  // every row of the current step is a different sequence (decode), not a prefill chunk
     int chain_grid = 0, chain_pf_bytes = 4 * 1024;
     struct GraphEntry { int n; bool scores; cudaGraphExec_t exec; int launches; };
     std::vector<GraphEntry> graphs;
@@ -261,7 +262,7 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     mh[4] = S;
     mh[5] = n;  // hint_act: every row starts in the backbone
     // the persistent chain kernel: one CTA per (row, kv head, split), chunks in whole pages
-    int Sc = std::max(1, std::min(64, (c->chain_grid > 0 ? c->chain_grid : c->num_sms) / (n * g.Hkv)));
+    int Sc = std::max(1, std::min(64, c->num_sms / (n * g.Hkv)));
     int cchunk = (max_pos + 1 + Sc - 1) / Sc;
     cchunk = std::max(kPage, (cchunk + kPage - 1) / kPage * kPage);
     mh[6] = cchunk;  // StepMeta::pad[0]
@@ -299,8 +300,33 @@ cudaError_t launch_attn(river_ctx *c, int n, int layer0, bool pdl) {
                     pdl, c->kv_tmap, a);
 }
 
+// Steps of 1-4 rows: the split-KV kernel that fetches the cached positions before the grid dependency resolves.
+template <int DH, int GQ>
+cudaError_t launch_attn_small(river_ctx *c, int n, int layer0, int early) {
+    const river_config &g = c->cfg;
+    ChainArgs a{};
+    a.meta = c->meta();
+    a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh;
+    a.qscale = 1.4426950408889634f / std::sqrt((float)g.dh);
+    a.qbuf = c->qbuf; a.obuf = c->obuf; a.kv = kv_addr(c, layer0);
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.attn_tickets = c->attn_tickets; a.dev_err = c->dev_err;
+    const int S = std::max(1, std::min(64, c->num_sms / (n * g.Hkv)));  // as set_attn_meta puts into the metadata
+    const size_t smem = sizeof(float) * (size_t)kChainWarps * GQ * (DH + 2);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(attn_small_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_set = true;
+    }
+    return launch_k(attn_small_kernel<DH, GQ>, dim3(n * g.Hkv * S), dim3(kChainThreads), smem, c->stream, true, a, layer0, early);
+}
+
 cudaError_t launch_attention(river_ctx *c, int n, int layer0, bool pdl) {
     const int gq = c->cfg.Hq / c->cfg.Hkv;
+    if (n <= 4 && !(c->cfg.flags & RIVER_F_SIMPLE_ATTN) && !(c->cfg.flags & RIVER_F_TMA_ATTN)) {
+#define ATTS(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn_small<DH_, GQ_>(c, n, layer0, c->rows_distinct ? 1 : 0);
+        ATTS(64, 1) ATTS(64, 2) ATTS(64, 4) ATTS(64, 8) ATTS(128, 1) ATTS(128, 2) ATTS(128, 4) ATTS(128, 8)
+#undef ATTS
+    }
 #define ATT(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn<DH_, GQ_>(c, n, layer0, pdl);
     ATT(64, 1) ATT(64, 2) ATT(64, 4) ATT(64, 8) ATT(128, 1) ATT(128, 2) ATT(128, 4) ATT(128, 8)
 #undef ATT
@@ -1252,7 +1278,10 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
         set_io_meta(mh, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr, c->next_i, c->exit_i,
                     nullptr);
         if (int rc = push_meta(c, mh)) return rc;
-        if (int rc = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch)) return rc;
+        c->rows_distinct = false;  // consecutive positions of one sequence share a chunk
+        const int rc_rows = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch);
+        c->rows_distinct = true;
+        if (rc_rows) return rc_rows;
         for (int i = 0; i < n_head; ++i) {
             if (logits_last)
                 CUDA_TRY(c, cudaMemcpyAsync(logits_last + (size_t)head_seq[i] * g.V, c->logits_i + (size_t)i * g.V,
