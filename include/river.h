@@ -51,7 +51,9 @@ enum {
     RIVER_F_CHAIN = 8,       /* steps of 1-4 rows through the persistent chain kernel (one cooperative launch for all
                                 layers and the LM head) instead of one kernel per stage */
     RIVER_F_NO_W4TC = 16,    /* exit-layer rows of batches on the CUDA-core kernel instead of the dequantising tcgen05 GEMM */
-    RIVER_F_TMA_ATTN = 32    /* steps of 1-4 rows through the TMA-fed attention kernel too (default: the small-step kernel) */
+    RIVER_F_TMA_ATTN = 32,   /* steps of 1-4 rows through the TMA-fed attention kernel too (default: the small-step kernel) */
+    RIVER_F_FUSED_SCORE = 64 /* small steps: exit score / decision / compaction by the last CTA of the down projection
+                                instead of a kernel of its own (measured 1 % slower: the separate kernel overlaps) */
     /* bits 8-15: tuning aid for the chain kernel, KiB of the next phase's weights each warp requests from the L2
        ahead of time (0 = default 4) */
 };

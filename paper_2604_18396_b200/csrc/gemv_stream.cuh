@@ -333,7 +333,7 @@ __device__ __forceinline__ void stream_rows_bf16(const P &p, int t, const uint16
 
 template <class P, int N, int R>
 __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjIn in, const RowLists rl, int has_river,
-                                                          int xstride, int skip_backbone) {
+                                                          int xstride, int skip_backbone, const ScoreTail tail) {
     extern __shared__ __align__(16) float stream_smem[];
     const int K = p.K;
     float *red = stream_smem;            // 32
@@ -401,6 +401,7 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
             }
         }
     }
+    if (tail.meta) score_tail(tail);  // the kernel that ends a block also scores it (small steps)
 }
 
 // ---------------------------------------------------------------- a8: final norm + LM head + argmax partials

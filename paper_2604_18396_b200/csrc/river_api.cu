@@ -363,7 +363,7 @@ StreamGeom pick_geometry(river_ctx *c, Kern kern, int tasks, size_t smem) {
 
 template <class P, int N, int R>
 cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks,
-                            int has_river, bool pdl, int skip_backbone) {
+                            int has_river, bool pdl, int skip_backbone, const ScoreTail &tail) {
     const size_t smem = stream_smem_bytes(N, K);
     // one kernel instantiation serves several projections (O and down): cache the geometry per (tasks, K)
     struct Entry { int tasks, K; StreamGeom g; };
@@ -379,19 +379,19 @@ cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const Ro
         geom = &cache.back().g;
     }
     return launch_k(stream_proj_kernel<P, N, R>, dim3(geom->grid), dim3(geom->threads), smem, c->stream, pdl, p, in, rl,
-                    has_river, xs_stride(K, 32), skip_backbone);
+                    has_river, xs_stride(K, 32), skip_backbone, tail);
 }
 
 int stream_rows_per_task(int K) { return K >= 4096 ? 2 : 4; }
 
 template <class P>
 cudaError_t launch_stream(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks_r2, int n,
-                          int has_river, bool pdl, int skip_backbone = 0) {
+                          int has_river, bool pdl, int skip_backbone = 0, const ScoreTail &tail = ScoreTail{}) {
     int n_sel = 1;
     while (n_sel < n && n_sel < 4 && stream_smem_bytes(n_sel * 2, K) <= 200 * 1024) n_sel *= 2;
     const int r = stream_rows_per_task(K);
     const int tasks = tasks_r2 * 2 / r;
-#define STREAM_CASE(N_, R_) if (n_sel == N_ && r == R_) return launch_stream_t<P, N_, R_>(c, p, in, rl, K, tasks, has_river, pdl, skip_backbone);
+#define STREAM_CASE(N_, R_) if (n_sel == N_ && r == R_) return launch_stream_t<P, N_, R_>(c, p, in, rl, K, tasks, has_river, pdl, skip_backbone, tail);
     STREAM_CASE(1, 2) STREAM_CASE(2, 2) STREAM_CASE(4, 2)
     STREAM_CASE(1, 4) STREAM_CASE(2, 4) STREAM_CASE(4, 4)
 #undef STREAM_CASE
@@ -737,6 +737,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         const river_ctx::LayerMaps *tm = tc ? &c->tc_maps[l - 1] : nullptr;
         const river_ctx::LayerMaps *wm = (tc && c->w4tc_ok && has_river) ? &c->w4_maps[l - 1] : nullptr;
         const int32_t *nrh = c->n_riv + std::max(0, l - 2);  // never above the count entering this block
+        const bool fuse_score = !tc && (g.flags & RIVER_F_FUSED_SCORE);  // opt-in; needs the down projection on the stream kernel
         const int skip_bb = tc ? 1 : 0;
         // ---- a2: attention norm + QKV + RoPE + KV write
         {
@@ -822,10 +823,19 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
                 const CUtensorMap *const cm[3] = {&wm->d, &wm->d, &wm->d};
                 const river_w4 *const cw[3] = {&w.rd, &w.rd, &w.rd};
                 note(launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
-            } else if (!tc || has_river) note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb));
+            } else if (!tc || has_river) {
+                ScoreTail st{};
+                if (fuse_score) {
+                    st.meta = c->meta(); st.l = l; st.L = L; st.entry_layer = g.entry_layer; st.exit_mode = g.exit_mode;
+                    st.d = d; st.h_in = h_in; st.h_out = h_out; st.pass = c->pass; st.exited = c->exited; st.lists = lists;
+                    st.hint_act = c->hint_act; st.ticket = c->tickets + 1;
+                }
+                note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb, st));
+            }
         }
-        // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
-        {
+        // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1 (with RIVER_F_FUSED_SCORE: done
+        // by the last CTA of the down projection above)
+        if (!fuse_score) {
             LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
             note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, true, c->meta(), l, L,
                           g.entry_layer, g.exit_mode, (const float *)h_in, (const float *)h_out, d, c->pass, c->exited,

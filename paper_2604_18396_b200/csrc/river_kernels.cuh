@@ -282,6 +282,85 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     if (threadIdx.x == 0 && gridDim.x > 1) *ticket = 0;
 }
 
+// ---------------------------------------------------------------- a6 + a7 as the tail of the kernel that ends a block
+// An alternative to the score kernel above for small steps (RIVER_F_FUSED_SCORE): the kernel that writes the block
+// output (the down projection) finishes it: the last CTA to arrive (atomic ticket, no spinning)
+// computes Eq. 1 for every row still in the backbone, takes the decisions and emits the row lists, exactly as
+// score_compact_kernel does.
+struct ScoreTail {
+    const StepMeta *meta;   // null: the kernel has no tail
+    int l, L, entry_layer, exit_mode, d;
+    const float *h_in, *h_out;
+    uint8_t *pass, *exited;
+    Lists lists;
+    int32_t *hint_act;
+    unsigned *ticket;
+};
+
+__device__ __forceinline__ void score_tail(const ScoreTail &t) {
+    __shared__ float red[3][32];
+    __shared__ int s_cnt[66];
+    __shared__ bool s_last;
+    __shared__ int s_allpass;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(t.ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const int n = t.meta->n_rows, l = t.l, L = t.L, d = t.d;
+    const float *tau = t.meta->tau;
+    const int32_t *forced = t.meta->forced;
+    int32_t *exit_layer = t.meta->exit_layer;
+    float *scores = t.meta->scores;
+    const bool eligible = (l >= 1) && (l >= t.entry_layer) && (l < L);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int row = 0; row < n; ++row) {
+        if (t.exited[row] != 0 || !(eligible || scores)) continue;  // uniform
+        const float4 *a = reinterpret_cast<const float4 *>(t.h_in + (size_t)row * d);
+        const float4 *b = reinterpret_cast<const float4 *>(t.h_out + (size_t)row * d);
+        float ab = 0.f, aa = 0.f, bb = 0.f;
+        for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+            const float4 x = __ldcg(a + i), y = __ldcg(b + i);
+            ab += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
+            aa += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+            bb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+        }
+        ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
+        __syncthreads();
+        if (lane == 0) { red[0][warp] = ab; red[1][warp] = aa; red[2][warp] = bb; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            ab = aa = bb = 0.f;
+            for (int w = 0; w < nwarps; ++w) { ab += red[0][w]; aa += red[1][w]; bb += red[2][w]; }
+            float s = 0.f;
+            if (aa > 0.f && bb > 0.f) s = ab / (sqrtf(aa) * sqrtf(bb));
+            t.pass[row] = (s > tau[row]) ? 1 : 0;
+            if (scores) scores[(size_t)row * L + (l - 1)] = s;
+        }
+    }
+    if (threadIdx.x == 0) s_allpass = 1;
+    __syncthreads();
+    if (t.exit_mode == 1) {
+        for (int b = threadIdx.x; b < n; b += blockDim.x)
+            if (t.exited[b] == 0 && !(eligible && t.pass[b])) atomicAnd(&s_allpass, 0);
+        __syncthreads();
+    }
+    for (int b = threadIdx.x; b < n; b += blockDim.x) {
+        if (t.exited[b] != 0) continue;
+        bool leave = eligible && (t.exit_mode == 1 ? (s_allpass != 0) : (t.pass[b] != 0));
+        const int f = forced ? forced[b] : -1;
+        if (f >= 0) leave = (f == l) && (l < L);
+        if (leave) {
+            t.exited[b] = 1;
+            exit_layer[b] = l;
+        }
+    }
+    __syncthreads();
+    build_lists(n, t.exited, l, t.lists, t.hint_act, s_cnt);
+    if (threadIdx.x == 0) *t.ticket = 0;
+}
+
 // ---------------------------------------------------------------- shared by the projection kernels
 // What feeds a projection: either rows of an fp32 buffer as they are, or their RMSNorm (x = h * rsqrt(mean h^2 +
 // eps) * gain), computed by every CTA for itself.

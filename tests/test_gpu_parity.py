@@ -133,11 +133,12 @@ def test_tiny_geometric_exits_and_wide_batch():
     assert r["n_early"] > r["total"] // 2
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2, 4, 5, 8, 9, 12, 32, 33])
+@pytest.mark.parametrize("flags", [0, 1, 2, 4, 5, 8, 9, 12, 32, 33, 64, 97])
 def test_launch_modes_agree_with_oracle(flags):
     # 1: CUDA-graph replay; 2: no tensor-core projections; 4: plain attention kernel; 8: the persistent chain kernel
     # (three rows per step: the chain kernel takes them when 8 is set, by the parameter or by the fixture);
-    # 32: the TMA-fed attention kernel for small steps too (default there: the kernel that fetches the cache early)
+    # 32: the TMA-fed attention kernel for small steps too (default there: the kernel that fetches the cache early);
+    # 64: exit score / decision / compaction by the last CTA of the down projection instead of a kernel of its own
     r = run_scheduled(model("mini8"), [37, 16, 3], 6, "uniform", page_seed=11, flags=flags, max_batch=4)
     assert r["n_early"] > 0
 
