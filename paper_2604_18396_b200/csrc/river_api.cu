@@ -59,6 +59,7 @@ struct river_ctx {
     float *part_o;
     CUtensorMap kv_tmap;
     int attn_splits_now = 1;
+    bool attn_small_now = false;  // this step's attention runs on the small-step kernel (short contexts, 1-4 rows)
     unsigned *attn_tickets, *tickets;  // [max_batch*Hkv], [4]
     // tensor-core path: operand buffers, split-K partials, tickets, tensor maps of every weight matrix
     __nv_bfloat16 *tc_xhi = nullptr, *tc_xlo = nullptr;
@@ -78,7 +79,7 @@ struct river_ctx {
     bool chain_ok = false;
     bool rows_distinct = true;  // every row of the current step is a different sequence (decode), not a prefill chunk
     int chain_grid = 0, chain_pf_bytes = 4 * 1024;
-    struct GraphEntry { int n; bool scores; cudaGraphExec_t exec; int launches; };
+    struct GraphEntry { int n; bool small_attn; cudaGraphExec_t exec; int launches; };
     std::vector<GraphEntry> graphs;
     double *inv_freq;
     int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
@@ -267,6 +268,9 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     cchunk = std::max(kPage, (cchunk + kPage - 1) / kPage * kPage);
     mh[6] = cchunk;  // StepMeta::pad[0]
     mh[7] = Sc;      // StepMeta::pad[1]
+    // the small-step kernel walks a split in batches of 4 positions per warp without a load pipeline: worth it up to
+    // two batches per warp, beyond that the TMA-fed kernel's staging pays
+    c->attn_small_now = n <= 4 && cchunk <= 2 * 4 * kChainWarps && !(g.flags & (RIVER_F_SIMPLE_ATTN | RIVER_F_TMA_ATTN));
     c->attn_splits_now = S;
 }
 
@@ -322,7 +326,7 @@ cudaError_t launch_attn_small(river_ctx *c, int n, int layer0, int early) {
 
 cudaError_t launch_attention(river_ctx *c, int n, int layer0, bool pdl) {
     const int gq = c->cfg.Hq / c->cfg.Hkv;
-    if (n <= 4 && !(c->cfg.flags & RIVER_F_SIMPLE_ATTN) && !(c->cfg.flags & RIVER_F_TMA_ATTN)) {
+    if (c->attn_small_now) {
 #define ATTS(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn_small<DH_, GQ_>(c, n, layer0, c->rows_distinct ? 1 : 0);
         ATTS(64, 1) ATTS(64, 2) ATTS(64, 4) ATTS(64, 8) ATTS(128, 1) ATTS(128, 2) ATTS(128, 4) ATTS(128, 8)
 #undef ATTS
@@ -1043,7 +1047,7 @@ int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
     const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
     if (!use_graph) return run_rows(c, n, n, row_pos_host);
     for (auto &ge : c->graphs)
-        if (ge.n == n) {
+        if (ge.n == n && ge.small_attn == c->attn_small_now) {
             if (!ge.exec) {  // second use: capture
                 cudaGraph_t graph = nullptr;
                 CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -1062,7 +1066,7 @@ int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
             c->st.launches_total += ge.launches;
             return 0;
         }
-    c->graphs.push_back({n, false, nullptr, 0});
+    c->graphs.push_back({n, c->attn_small_now, nullptr, 0});
     return run_rows(c, n, n, row_pos_host);  // first use: plain launches (also sets the kernels' attributes)
 }
 
