@@ -207,18 +207,22 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     __shared__ bool s_last;
     __shared__ int s_allpass;
     pdl_launch();
-    pdl_wait();
+    // per-step constants (uploaded before the step's first kernel): fetched while the predecessor still runs, so the
+    // decision below waits for nothing but the scores
     const int n = meta->n_rows;
     const float *tau = meta->tau;
     const int32_t *forced = meta->forced;
     int32_t *exit_layer = meta->exit_layer;
     float *scores = meta->scores;
     const int row = blockIdx.x;
+    const float tau_row = row < n ? tau[row] : 0.f;
+    int forced_mine = -1;  // thread b of the deciding CTA keeps row b's forced exit layer (rows beyond blockDim: read later)
+    if (forced && (int)threadIdx.x < n) forced_mine = forced[threadIdx.x];
+    pdl_wait();
     const bool eligible = (l >= 1) && (l >= entry_layer) && (l < L);
     if (row < n && exited[row] == 0 && (eligible || scores)) {
         const float4 *a = reinterpret_cast<const float4 *>(h_in + (size_t)row * d);
         const float4 *b = reinterpret_cast<const float4 *>(h_out + (size_t)row * d);
-        const float tau_row = tau[row];
         float ab = 0.f, aa = 0.f, bb = 0.f;
         const int nv = d / 4;
         for (int i0 = 0; i0 < nv; i0 += 4 * 256) {  // four loads of each vector in flight per thread
@@ -270,7 +274,7 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     for (int b = threadIdx.x; b < n; b += blockDim.x) {
         if (exited[b] != 0) continue;
         bool leave = eligible && (exit_mode == 1 ? (s_allpass != 0) : (pass[b] != 0));
-        const int f = forced ? forced[b] : -1;
+        const int f = forced ? (b == (int)threadIdx.x ? forced_mine : forced[b]) : -1;
         if (f >= 0) leave = (f == l) && (l < L);
         if (leave) {
             exited[b] = 1;
