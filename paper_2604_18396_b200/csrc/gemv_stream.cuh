@@ -281,7 +281,7 @@ __device__ __forceinline__ void stream_dots_w4(const W4 (&wrow)[R], const float 
     for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
-#pragma unroll 2
+#pragma unroll 4
     for (int c = lane; c < nch; c += 32) {
         uint4 q[R];
         float s[R], zz[R];
