@@ -197,8 +197,8 @@ struct TcQkvEpi {  // tiles walk the concatenated [q heads | k heads | v heads] 
                 q[i] = lo;
                 q[i + half] = hi;
             } else {
-                const int pos = kv.row_pos[row], slot = kv.row_slot[row];
-                const int page = kv.page_tbl[(size_t)slot * kv.max_pages_per_seq + pos / kPage];
+                const int pos = kv.row_pos[row];
+                const int page = kv.row_page[row];
                 if (page < 0 || page >= kv.n_pages) { atomicExch(dev_err, DEV_BAD_PAGE); continue; }
                 const size_t o = kv.base(page, which - 1, hl, pos % kPage);
                 kv.pool[o + i] = __float2bfloat16_rn(lo);

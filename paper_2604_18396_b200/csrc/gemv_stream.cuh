@@ -20,6 +20,8 @@ namespace river {
 struct RowLists {
     const int32_t *act_idx, *n_act, *riv_idx, *n_riv;
     const int32_t *hint_act;  // backbone row count as of the latest compaction; never under-counts (a prefetch hint)
+    const int32_t *n_rows;    // rows of the step (per-step metadata, stable while the step runs)
+    const uint8_t *exited;    // the sticky exit flags the lists were built from
 };
 
 struct QkvProblem {
@@ -67,10 +69,10 @@ struct QkvProblem {
         int which, hl, i0;
         locate<R>(t, which, hl, i0);
         const int half = dh / 2;
-        const int pos = kv.row_pos[row], slot = kv.row_slot[row];
+        const int pos = kv.row_pos[row];
         int page = 0;
         if (which != 0) {
-            page = kv.page_tbl[(size_t)slot * kv.max_pages_per_seq + pos / kPage];
+            page = kv.row_page[row];
             if (page < 0 || page >= kv.n_pages) { atomicExch(dev_err, DEV_BAD_PAGE); return; }
         }
 #pragma unroll
@@ -356,13 +358,81 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
         stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre);
         have_pre = true;
     }
+    // A step of ONE row (the latency-critical case): which weight set the row takes follows from its exit flag, its
+    // index is 0, and its data can be requested at once - one memory round trip after the grid dependency instead of
+    // three (count -> index -> data).  The norm gain, a constant, is fetched before the wait.
+    constexpr int XF = 4;  // 128-bit pieces of the row a thread keeps in registers
+    const int nv = K >> 2, tid = threadIdx.x, nthr = blockDim.x;
+    const bool single = N == 1 && *rl.n_rows == 1;
+    const bool fast = single && nv <= XF * nthr;
+    uint2 gr[XF];
+    if (fast && in.gain) {
+#pragma unroll
+        for (int k = 0; k < XF; ++k) {
+            const int v = tid + k * nthr;
+            gr[k] = v < nv ? *reinterpret_cast<const uint2 *>(in.gain + 4 * v) : make_uint2(0u, 0u);
+        }
+    }
     pdl_wait();
-    // skip_backbone: the backbone rows of this step are served by the tensor-core kernel
-    const int na = skip_backbone ? 0 : *rl.n_act, nr = has_river ? *rl.n_riv : 0;
+    int na, nr;
+    bool prestaged = false;
+    __shared__ int32_t s_row0;
+    const int32_t *act_idx = rl.act_idx, *riv_idx = rl.riv_idx;
+    if (single) {
+        if (tid == 0) s_row0 = 0;
+        const bool riv = rl.exited[0] != 0;
+        na = (riv || skip_backbone) ? 0 : 1;
+        nr = (riv && has_river) ? 1 : 0;
+        act_idx = riv_idx = &s_row0;
+        if (fast && na + nr == 1) {
+            float4 xr[XF];
+            float ss = 0.f;
+            const float4 *src = reinterpret_cast<const float4 *>(in.src);
+#pragma unroll
+            for (int k = 0; k < XF; ++k) {
+                const int v = tid + k * nthr;
+                xr[k] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                ss += xr[k].x * xr[k].x + xr[k].y * xr[k].y + xr[k].z * xr[k].z + xr[k].w * xr[k].w;
+            }
+            float scale = 1.f;
+            if (in.gain) {
+                ss = warp_sum(ss);
+                if (lane == 0) red[warp] = ss;
+                __syncthreads();
+                ss = 0.f;
+                for (int w = 0; w < nwarps; ++w) ss += red[w];
+                scale = rsqrtf(ss / (float)K + in.eps);
+            }
+#pragma unroll
+            for (int k = 0; k < XF; ++k) {
+                const int v = tid + k * nthr;
+                if (v < nv) {
+                    float4 y = xr[k];
+                    if (in.gain) {
+                        y.x *= scale * bf16lo(gr[k].x); y.y *= scale * bf16hi(gr[k].x);
+                        y.z *= scale * bf16lo(gr[k].y); y.w *= scale * bf16hi(gr[k].y);
+                    }
+                    if (riv) *reinterpret_cast<float4 *>(xs + xs_index<32>(4 * v)) = y;
+                    else *reinterpret_cast<float4 *>(xs + xs_index<8>(4 * v)) = y;
+                }
+            }
+            __syncthreads();
+            if (riv) stream_chunk_sums<1>(xs, xsum, K, xstride);
+            prestaged = true;
+        } else {
+            __syncthreads();  // s_row0
+        }
+    } else {
+        // skip_backbone: the backbone rows of this step are served by the tensor-core kernel
+        na = skip_backbone ? 0 : *rl.n_act;
+        nr = has_river ? *rl.n_riv : 0;
+    }
 
     for (int i0 = 0; i0 < na; i0 += N) {
-        __syncthreads();
-        stream_load_rows<N, 8>(in, rl.act_idx, i0, na, K, xstride, xs, xsum, red);
+        if (!prestaged) {
+            __syncthreads();
+            stream_load_rows<N, 8>(in, act_idx, i0, na, K, xstride, xs, xsum, red);
+        }
         for (int t = t0 + warp; t < t1; t += nwarps) {
             const uint16_t *rows[R];
             stream_rows_bf16<P, N, R>(p, t, rows);
@@ -373,13 +443,15 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
                 float res[R];
 #pragma unroll
                 for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n]);
-                if (lane == n && i0 + n < na) p.template epilogue<R>(t, rl.act_idx[i0 + n], res);
+                if (lane == n && i0 + n < na) p.template epilogue<R>(t, single ? 0 : act_idx[i0 + n], res);
             }
         }
     }
     for (int i0 = 0; i0 < nr; i0 += N) {
-        __syncthreads();
-        stream_load_rows<N, 32>(in, rl.riv_idx, i0, nr, K, xstride, xs, xsum, red);
+        if (!prestaged) {
+            __syncthreads();
+            stream_load_rows<N, 32>(in, riv_idx, i0, nr, K, xstride, xs, xsum, red);
+        }
         const int ng = K / p.group;
         for (int t = t0 + warp; t < t1; t += nwarps) {
             W4 rows[R];
@@ -397,7 +469,7 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
                 float res[R];
 #pragma unroll
                 for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n]);
-                if (lane == n && i0 + n < nr) p.template epilogue<R>(t, rl.riv_idx[i0 + n], res);
+                if (lane == n && i0 + n < nr) p.template epilogue<R>(t, single ? 0 : riv_idx[i0 + n], res);
             }
         }
     }

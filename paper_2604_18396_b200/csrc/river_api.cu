@@ -83,7 +83,7 @@ struct river_ctx {
     std::vector<GraphEntry> graphs;
     double *inv_freq;
     int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
-    int32_t *meta_dev;  // [kMetaHdr + 6*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows
+    int32_t *meta_dev;  // [kMetaHdr + 7*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows, row_page
     uint8_t *exited, *pass;
     int *dev_err;
     size_t ws_bytes = 0;
@@ -109,12 +109,13 @@ struct river_ctx {
     double prof_ms[kNumClasses] = {0}, prof_bytes[kNumClasses] = {0};
     int64_t prof_launches[kNumClasses] = {0};
 
-    int meta_ints() const { return kMetaHdr + 6 * cfg.max_batch; }
+    int meta_ints() const { return kMetaHdr + 7 * cfg.max_batch; }
     StepMeta *meta() const { return reinterpret_cast<StepMeta *>(meta_dev); }
     int32_t *row_slot() const { return meta_dev + kMetaHdr; }
     int32_t *row_pos() const { return meta_dev + kMetaHdr + cfg.max_batch; }
     int32_t *upd() const { return meta_dev + kMetaHdr + 2 * cfg.max_batch; }
     int32_t *head_rows() const { return meta_dev + kMetaHdr + 5 * cfg.max_batch; }
+    int32_t *row_page() const { return meta_dev + kMetaHdr + 6 * cfg.max_batch; }  // page of each row's new position
 };
 
 namespace {
@@ -170,7 +171,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     int32_t *na = cv.take<int32_t>(L + 1), *nr = cv.take<int32_t>(L + 1);
     int32_t *pt = cv.take<int32_t>((size_t)c->max_seqs * c->max_pages_per_seq);
     int32_t *tk = cv.take<int32_t>(B), *fo = cv.take<int32_t>(B), *ex = cv.take<int32_t>(B), *nx = cv.take<int32_t>(B);
-    int32_t *md = cv.take<int32_t>(kMetaHdr + 6 * B);
+    int32_t *md = cv.take<int32_t>(kMetaHdr + 7 * B);
     float *po = cv.take<float>((B + 600) * (size_t)c->Hq * c->dh);
     float2 *pml = cv.take<float2>((B + 600) * (size_t)c->Hq);
     uint8_t *exd = cv.take<uint8_t>(B), *ps = cv.take<uint8_t>(B);
@@ -236,6 +237,7 @@ KvAddr kv_addr(const river_ctx *c, int layer0) {
     k.page_tbl = c->page_tbl_dev;
     k.row_slot = c->row_slot();
     k.row_pos = c->row_pos();
+    k.row_page = c->row_page();
     k.n_pages = c->cfg.n_pages;
     k.max_pages_per_seq = c->cfg.max_pages_per_seq;
     k.Hkv = c->cfg.Hkv;
@@ -733,7 +735,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         const int has_river = w.rq.codes != nullptr;
         const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
         const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
-        const RowLists rl{ai, na, ri, nr, c->hint_act};
+        const RowLists rl{ai, na, ri, nr, c->hint_act, c->meta_dev /* StepMeta::n_rows */, c->exited};
         float *h_in = c->h[hi], *h_mid = c->h[(hi + 1) % 3], *h_out = c->h[(hi + 2) % 3];
         // With more rows than one CUDA-core pass takes, the backbone rows go to the tensor-core GEMM and the stream
         // kernel only serves the exit-layer rows of the same launch slot.
@@ -1192,6 +1194,7 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
         mh[kMetaHdr + b] = slots[b];
         mh[kMetaHdr + g.max_batch + b] = pos;
         mh[kMetaHdr + 5 * g.max_batch + b] = b;
+        mh[kMetaHdr + 6 * g.max_batch + b] = c->page_tbl[(size_t)slots[b] * g.max_pages_per_seq + pos / kPage];
         c->last_pos[b] = pos;
     }
     mh[0] = batch; mh[1] = n_upd; mh[2] = batch;
@@ -1279,6 +1282,7 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
             if (int rc = ensure_page(c, slots[s], p, mh, n_upd)) return rc;
             mh[kMetaHdr + n] = slots[s];
             mh[kMetaHdr + g.max_batch + n] = p;
+            mh[kMetaHdr + 6 * g.max_batch + n] = c->page_tbl[(size_t)slots[s] * g.max_pages_per_seq + p / kPage];
             if (p == len - 1) {
                 mh[kMetaHdr + 5 * g.max_batch + n_head] = n;
                 head_seq[n_head++] = s;

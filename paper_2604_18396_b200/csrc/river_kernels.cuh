@@ -378,6 +378,7 @@ struct KvAddr {
     __nv_bfloat16 *pool;  // [L][n_pages][2][Hkv][16][dh]
     const int32_t *page_tbl;
     const int32_t *row_slot, *row_pos;
+    const int32_t *row_page;  // page that holds each row's new position (host-computed: no table walk on the write path)
     int n_pages, max_pages_per_seq, Hkv, dh;
     int layer0;
     __device__ __forceinline__ size_t base(int page, int kv, int kvh, int inpage) const {
