@@ -95,6 +95,42 @@ struct QkvProblem {
             }
         }
     }
+    // What the epilogue of a two-row task reads besides the dot products, requested BEFORE the dot products are
+    // computed so that the loads travel meanwhile: rotary cos / sin, position and write page of the row.
+    __device__ void epi_pre(int t, int row, float (&e)[4]) const {
+        int which, hl, i0;
+        locate<2>(t, which, hl, i0);
+        if (which != 2) {
+            const float2 cs = rope_cs[(size_t)row * (dh / 2) + i0];
+            e[0] = cs.x;
+            e[1] = cs.y;
+        }
+        if (which != 0) {
+            e[2] = __int_as_float(kv.row_pos[row]);
+            e[3] = __int_as_float(kv.row_page[row]);
+        }
+    }
+    __device__ void epilogue_pre(int t, int row, const float (&res)[2], const float (&e)[4]) const {
+        int which, hl, i0;
+        locate<2>(t, which, hl, i0);
+        const int half = dh / 2;
+        float lo = res[0], hi = res[1];
+        if (which != 2) {
+            const float rl = lo * e[0] - hi * e[1], rh = hi * e[0] + lo * e[1];
+            lo = rl; hi = rh;
+        }
+        if (which == 0) {
+            float *q = q_out + (size_t)row * (Hq * dh) + (size_t)hl * dh;
+            q[i0] = lo;
+            q[i0 + half] = hi;
+        } else {
+            const int pos = __float_as_int(e[2]), page = __float_as_int(e[3]);
+            if (page < 0 || page >= kv.n_pages) { atomicExch(dev_err, DEV_BAD_PAGE); return; }
+            const size_t o = kv.base(page, which - 1, hl, pos % kPage);
+            kv.pool[o + i0] = __float2bfloat16_rn(lo);
+            kv.pool[o + i0 + half] = __float2bfloat16_rn(hi);
+        }
+    }
 };
 
 struct ResidProblem {  // out[row][o] = resid[row][o] + W[o] . x[row]
@@ -113,6 +149,14 @@ struct ResidProblem {  // out[row][o] = resid[row][o] + W[o] . x[row]
         const size_t o = (size_t)row * out_dim + (size_t)t * R;
 #pragma unroll
         for (int r = 0; r < R; ++r) out[o + r] = __ldcg(resid + o + r) + res[r];  // L2: written by other SMs
+    }
+    __device__ void epi_pre(int t, int row, float (&e)[4]) const {
+        const float2 v = __ldcg(reinterpret_cast<const float2 *>(resid + (size_t)row * out_dim + (size_t)t * 2));
+        e[0] = v.x;
+        e[1] = v.y;
+    }
+    __device__ void epilogue_pre(int t, int row, const float (&res)[2], const float (&e)[4]) const {
+        *reinterpret_cast<float2 *>(out + (size_t)row * out_dim + (size_t)t * 2) = make_float2(e[0] + res[0], e[1] + res[1]);
     }
 };
 
@@ -134,6 +178,8 @@ struct GateUpProblem {  // act[row][f] = silu(Wg[f] . y) * (Wu[f] . y)
             act[(size_t)row * F + (size_t)t * (R / 2) + j] = g / (1.f + __expf(-g)) * u;
         }
     }
+    __device__ void epi_pre(int, int, float (&)[4]) const {}
+    __device__ void epilogue_pre(int t, int row, const float (&res)[2], const float (&)[4]) const { epilogue<2>(t, row, res); }
 };
 
 
@@ -437,13 +483,24 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
             const uint16_t *rows[R];
             stream_rows_bf16<P, N, R>(p, t, rows);
             float acc[R][N];
+            float ep[4] = {0.f, 0.f, 0.f, 0.f};
+            if constexpr (N == 1 && R == 2) {
+                if (single && lane == 0) p.epi_pre(t, 0, ep);  // travels while the dot products are computed
+            }
             stream_dots_bf16<N, R>(rows, xs, K, xstride, have_pre && i0 == 0 && t == t0 + warp, pre, acc);
 #pragma unroll
             for (int n = 0; n < N; ++n) {
                 float res[R];
 #pragma unroll
                 for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n]);
-                if (lane == n && i0 + n < na) p.template epilogue<R>(t, single ? 0 : act_idx[i0 + n], res);
+                if (lane == n && i0 + n < na) {
+                    if constexpr (N == 1 && R == 2) {
+                        if (single) p.epilogue_pre(t, 0, res, ep);
+                        else p.template epilogue<R>(t, act_idx[i0 + n], res);
+                    } else {
+                        p.template epilogue<R>(t, single ? 0 : act_idx[i0 + n], res);
+                    }
+                }
             }
         }
     }
@@ -463,13 +520,24 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
                 rows[r] = W4{b.codes + row * (K >> 1), b.scale + row * ng, b.zero + row * ng};
             }
             float acc[R][N];
+            float ep[4] = {0.f, 0.f, 0.f, 0.f};
+            if constexpr (N == 1 && R == 2) {
+                if (single && lane == 0) p.epi_pre(t, 0, ep);
+            }
             stream_dots_w4<N, R>(rows, xs, xsum, K, xstride, p.group, acc);
 #pragma unroll
             for (int n = 0; n < N; ++n) {
                 float res[R];
 #pragma unroll
                 for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n]);
-                if (lane == n && i0 + n < nr) p.template epilogue<R>(t, single ? 0 : riv_idx[i0 + n], res);
+                if (lane == n && i0 + n < nr) {
+                    if constexpr (N == 1 && R == 2) {
+                        if (single) p.epilogue_pre(t, 0, res, ep);
+                        else p.template epilogue<R>(t, riv_idx[i0 + n], res);
+                    } else {
+                        p.template epilogue<R>(t, single ? 0 : riv_idx[i0 + n], res);
+                    }
+                }
             }
         }
     }
