@@ -151,7 +151,7 @@ const char *check_config(const river_config *c) {
     return nullptr;
 }
 
-int head_grid_for(const river_config *c) { return 148 * 4 > c->V / 4 ? std::max(1, c->V / 4) : 148 * 4; }
+int head_grid_for(const river_config *c) { return 148 * 2 > c->V / 4 ? std::max(1, c->V / 4) : 148 * 2; }
 int head_parts_for(const river_config *c) { return std::max(head_grid_for(c), c->V / 128 + 1); }  // argmax partials per row
 
 size_t carve(const river_config *c, river_ctx *x, char *base) {
