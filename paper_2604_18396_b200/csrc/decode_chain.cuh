@@ -614,15 +614,15 @@ __device__ __forceinline__ void chain_attention(const ChainArgs &a, const KvAddr
             }
         }
         if (S > 1) {
-            __threadfence();
-            __syncthreads();
+            __syncthreads();  // the CTA's partial is written ...
             if (threadIdx.x == 0) {
+                __threadfence();  // ... and made visible before the ticket (one fence, cumulative over the barrier)
                 const unsigned tk = atomicAdd(a.attn_tickets + row * a.Hkv + kvh, 1u);
                 fl->flag = (tk == (unsigned)(S - 1));
+                __threadfence();
             }
             __syncthreads();
             if (fl->flag) {
-                __threadfence();
                 // (max, sum) of every (head, split) into shared memory, then every thread owns one (head, dim) and
                 // pulls the splits' partial outputs in batches of independent loads
                 float *s_mx = s_acc, *s_sm = s_acc + GQ * 64;
