@@ -220,6 +220,52 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     if (forced && (int)threadIdx.x < n) forced_mine = forced[threadIdx.x];
     pdl_wait();
     const bool eligible = (l >= 1) && (l >= entry_layer) && (l < L);
+    if (n == 1 && gridDim.x == 1) {
+        // A step of one row: its exit flag and both state vectors are requested together (one round trip), and one
+        // thread takes the decision and writes the two one-element lists - no ballots, no second pass over flags.
+        const int gone_before = exited[0];
+        float ab = 0.f, aa = 0.f, bb = 0.f;
+        if (eligible || scores) {
+            const float4 *a = reinterpret_cast<const float4 *>(h_in);
+            const float4 *b = reinterpret_cast<const float4 *>(h_out);
+            for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+                const float4 x = __ldcg(a + i), y = __ldcg(b + i);
+                ab += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
+                aa += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                bb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+            }
+            ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            if (lane == 0) { red[0][warp] = ab; red[1][warp] = aa; red[2][warp] = bb; }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            bool pass1 = false;
+            if (gone_before == 0 && (eligible || scores)) {
+                ab = aa = bb = 0.f;
+                for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { ab += red[0][w]; aa += red[1][w]; bb += red[2][w]; }
+                float sc = 0.f;
+                if (aa > 0.f && bb > 0.f) sc = ab / (sqrtf(aa) * sqrtf(bb));
+                pass1 = sc > tau_row;
+                if (scores) scores[l - 1] = sc;
+            }
+            bool gone = gone_before != 0;
+            if (!gone) {
+                bool leave = eligible && pass1;  // with one row the batch minimum is the row itself
+                if (forced_mine >= 0) leave = (forced_mine == l) && (l < L);
+                if (leave) {
+                    exited[0] = 1;
+                    exit_layer[0] = l;
+                    gone = true;
+                }
+            }
+            (gone ? lists.riv_idx : lists.act_idx)[(size_t)l * lists.max_batch] = 0;
+            lists.n_act[l] = gone ? 0 : 1;
+            lists.n_riv[l] = gone ? 1 : 0;
+            *hint_act = gone ? 0 : 1;
+        }
+        return;
+    }
     if (row < n && exited[row] == 0 && (eligible || scores)) {
         const float4 *a = reinterpret_cast<const float4 *>(h_in + (size_t)row * d);
         const float4 *b = reinterpret_cast<const float4 *>(h_out + (size_t)row * d);
