@@ -58,48 +58,14 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
 }
 
 // ---------------------------------------------------------------- activation rows -> bf16 hi / lo operand buffers
-// One CTA per operand row i < n_pad: the i-th row of the backbone list (zero beyond the list), optionally
-// RMS-normalised, split as x = hi + lo with hi = bf16(x), lo = bf16(x - hi).
-__global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
-                                                      __nv_bfloat16 *xhi, __nv_bfloat16 *xlo) {
-    __shared__ float red[8];
-    pdl_launch();
-    pdl_wait();
-    const int i = blockIdx.x, n = *cnt;
-    if (n <= 0) return;  // no row in the backbone any more: the GEMM returns before it reads an operand
-    uint2 *hi = reinterpret_cast<uint2 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint2 *>(xlo + (size_t)i * K);
+// CTA (i, j) writes inputs [1024 j, 1024 j + 1024) of operand row i < n_pad: the i-th row of the backbone list (zero
+// beyond the list), optionally RMS-normalised (every CTA of a row sums the whole row's squares itself: the row is a
+// few KB in L2), split as x = hi + lo with hi = bf16(x), lo = bf16(x - hi).  One 128-bit load per thread.
+constexpr int kPrepChunk = 1024;
+__device__ __forceinline__ float tc_prep_scale(const ProjIn &in, const float4 *src, int K, float *red) {
+    if (!in.gain) return 1.f;
+    float ss = 0.f;
     const int nv = K >> 2;
-    if (i >= n) {
-        for (int v = threadIdx.x; v < nv; v += blockDim.x) { hi[v] = make_uint2(0u, 0u); lo[v] = make_uint2(0u, 0u); }
-        return;
-    }
-    const float4 *src = reinterpret_cast<const float4 *>(in.src + (size_t)idx[i] * K);
-    float scale = 1.f;
-    if (in.gain) {
-        float ss = 0.f;
-        for (int v0 = 0; v0 < nv; v0 += 4 * 256) {
-            float4 x[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int v = v0 + u * 256 + threadIdx.x;
-                x[u] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) ss += x[u].x * x[u].x + x[u].y * x[u].y + x[u].z * x[u].z + x[u].w * x[u].w;
-        }
-        ss = warp_sum(ss);
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-        __syncthreads();
-        ss = 0.f;
-        for (int w = 0; w < 8; ++w) ss += red[w];
-        scale = rsqrtf(ss / (float)K + in.eps);
-    }
-    auto split2 = [](float a, float b, uint32_t &h, uint32_t &l) {
-        const __nv_bfloat16 ha = __float2bfloat16_rn(a), hb = __float2bfloat16_rn(b);
-        const __nv_bfloat16 la = __float2bfloat16_rn(a - __bfloat162float(ha)), lb = __float2bfloat16_rn(b - __bfloat162float(hb));
-        h = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
-        l = (uint32_t)__bfloat16_as_ushort(la) | ((uint32_t)__bfloat16_as_ushort(lb) << 16);
-    };
     for (int v0 = 0; v0 < nv; v0 += 4 * 256) {
         float4 x[4];
 #pragma unroll
@@ -108,54 +74,84 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int
             x[u] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int v = v0 + u * 256 + threadIdx.x;
-            if (v < nv) {
-                float4 y = x[u];
-                y.x *= scale; y.y *= scale; y.z *= scale; y.w *= scale;
-                if (in.gain) {
-                    const uint2 gw = *reinterpret_cast<const uint2 *>(in.gain + 4 * v);
-                    y.x *= bf16lo(gw.x); y.y *= bf16hi(gw.x); y.z *= bf16lo(gw.y); y.w *= bf16hi(gw.y);
-                }
-                uint2 h, l;
-                split2(y.x, y.y, h.x, l.x);
-                split2(y.z, y.w, h.y, l.y);
-                hi[v] = h;
-                lo[v] = l;
-            }
-        }
+        for (int u = 0; u < 4; ++u) ss += x[u].x * x[u].x + x[u].y * x[u].y + x[u].z * x[u].z + x[u].w * x[u].w;
     }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    ss = 0.f;
+    for (int w = 0; w < 8; ++w) ss += red[w];
+    return rsqrtf(ss / (float)K + in.eps);
+}
+__global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
+                                                      __nv_bfloat16 *xhi, __nv_bfloat16 *xlo) {
+    __shared__ float red[8];
+    pdl_launch();
+    pdl_wait();
+    const int i = blockIdx.x, n = *cnt;
+    if (n <= 0) return;  // no row in the backbone any more: the GEMM returns before it reads an operand
+    const int v = blockIdx.y * (kPrepChunk / 4) + threadIdx.x;  // 4-input group of the row
+    const bool mine = v < (K >> 2);
+    uint2 *hi = reinterpret_cast<uint2 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint2 *>(xlo + (size_t)i * K);
+    if (i >= n) {
+        if (mine) { hi[v] = make_uint2(0u, 0u); lo[v] = make_uint2(0u, 0u); }
+        return;
+    }
+    const float4 *src = reinterpret_cast<const float4 *>(in.src + (size_t)idx[i] * K);
+    float4 y = mine ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+    uint2 gw = make_uint2(0u, 0u);
+    if (in.gain && mine) gw = *reinterpret_cast<const uint2 *>(in.gain + 4 * v);
+    const float scale = tc_prep_scale(in, src, K, red);
+    if (!mine) return;
+    if (in.gain) {
+        y.x = y.x * scale * bf16lo(gw.x); y.y = y.y * scale * bf16hi(gw.x);
+        y.z = y.z * scale * bf16lo(gw.y); y.w = y.w * scale * bf16hi(gw.y);
+    }
+    auto split2 = [](float a, float b, uint32_t &h, uint32_t &l) {
+        const __nv_bfloat16 ha = __float2bfloat16_rn(a), hb = __float2bfloat16_rn(b);
+        const __nv_bfloat16 la = __float2bfloat16_rn(a - __bfloat162float(ha)), lb = __float2bfloat16_rn(b - __bfloat162float(hb));
+        h = (uint32_t)__bfloat16_as_ushort(ha) | ((uint32_t)__bfloat16_as_ushort(hb) << 16);
+        l = (uint32_t)__bfloat16_as_ushort(la) | ((uint32_t)__bfloat16_as_ushort(lb) << 16);
+    };
+    uint2 h, l;
+    split2(y.x, y.y, h.x, l.x);
+    split2(y.z, y.w, h.y, l.y);
+    hi[v] = h;
+    lo[v] = l;
 }
 
 // ---------------------------------------------------------------- epilogues on a finished 128 x N tile in smem
-// tile(r, n) = sum over K of W[row0 + r] . x[n]; `rows` maps n to the step's row id; only n < n_live are real.
-// The 128 tile rows are handled as 64 pairs; an epilogue call covers the pairs [pr0, pr1) (a K-split CTA finishes
-// its own slice of the tile), and pair_rows() tells which two tile rows pair pr is.
+// tile(r, n) = sum over K of W[row0 + r] . x[n], stored column by column: tile[n * ld + r] (consecutive threads take
+// consecutive features r: no bank conflicts, coalesced global writes); `rows` maps n to the step's row id; only
+// n < n_live are real.  The 128 tile rows are handled as 64 pairs in 16 quads of four pairs; an epilogue call covers
+// the pairs [pr0, pr1) (a K-split CTA finishes its own slice of the tile: whole quads), and quad_row(i, q0, nq) names
+// the first of four consecutive tile rows behind item i of the 2 nq four-row runs that make up the quads [q0, q0 + nq).
+constexpr int kTcLd = kTcBM + 4;  // column stride of the tile in floats (16-byte aligned columns)
 struct TcResidEpi {  // out[row][row0 + r] = resid[row][row0 + r] + tile(r, n)
     const float *resid;
     float *out;
     int out_dim;
-    __device__ void pair_rows(int pr, int &r0, int &r1) const { r0 = 2 * pr; r1 = 2 * pr + 1; }
+    __device__ int quad_row(int i, int q0, int) const { return 8 * q0 + 4 * i; }  // pairs (2 pr, 2 pr + 1): one range
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
                         int pr0, int pr1) const {
         const int row0 = tile_idx * kTcBM, nr = 2 * (pr1 - pr0);
         for (int t = tid; t < n_live * nr; t += nthr) {
             const int n = t / nr, r = 2 * pr0 + t % nr;
             const size_t o = (size_t)rows[n] * out_dim + row0 + r;
-            out[o] = resid[o] + tile[r * ld + n];
+            out[o] = resid[o] + tile[n * ld + r];
         }
     }
 };
 struct TcGateUpEpi {  // tile rows 0..63: gate features f0.., rows 64..127: up features f0..
     float *act;
     int F;
-    __device__ void pair_rows(int pr, int &r0, int &r1) const { r0 = pr; r1 = 64 + pr; }
+    __device__ int quad_row(int i, int q0, int nq) const { return i < nq ? 4 * (q0 + i) : 64 + 4 * (q0 + i - nq); }
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
                         int pr0, int pr1) const {
         const int f0 = tile_idx * 64, np = pr1 - pr0;
         for (int t = tid; t < n_live * np; t += nthr) {
             const int n = t / np, r = pr0 + t % np;
-            const float g = tile[r * ld + n], u = tile[(64 + r) * ld + n];
+            const float g = tile[n * ld + r], u = tile[n * ld + 64 + r];
             act[(size_t)rows[n] * F + f0 + r] = g / (1.f + __expf(-g)) * u;
         }
     }
@@ -166,10 +162,9 @@ struct TcQkvEpi {  // tiles walk the concatenated [q heads | k heads | v heads] 
     float *q_out;
     KvAddr kv;
     int *dev_err;
-    __device__ void pair_rows(int pr, int &r0, int &r1) const {
-        const int half = dh >> 1;
-        r0 = (pr / half) * dh + pr % half;
-        r1 = r0 + half;
+    __device__ int quad_row(int i, int q0, int nq) const {  // pair pr = rows (head * dh + j, head * dh + j + dh / 2)
+        const int half = dh >> 1, pr = 4 * (q0 + (i < nq ? i : i - nq));
+        return (pr / half) * dh + pr % half + (i < nq ? 0 : half);
     }
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
                         int pr0, int pr1) const {
@@ -185,7 +180,7 @@ struct TcQkvEpi {  // tiles walk the concatenated [q heads | k heads | v heads] 
             if (hh >= heads_per_tile) continue;
             const int r_lo = hh * dh + i, r_hi = r_lo + half;
             const int row = rows[n];
-            float lo = tile[r_lo * ld + n], hi = tile[r_hi * ld + n];
+            float lo = tile[n * ld + r_lo], hi = tile[n * ld + r_hi];
             if (which != 2) {
                 const float2 cs = rope_cs[(size_t)row * half + i];
                 const float a = lo * cs.x - hi * cs.y, b = hi * cs.x + lo * cs.y;
@@ -213,7 +208,7 @@ struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row
     float *part_val;
     int32_t *part_idx;
     int n_parts;
-    __device__ void pair_rows(int pr, int &r0, int &r1) const { r0 = 2 * pr; r1 = 2 * pr + 1; }
+    __device__ int quad_row(int i, int q0, int) const { return 8 * q0 + 4 * i; }
     // (the LM head is never K-split: the argmax partial below needs all 128 rows of the tile)
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *, int tid, int nthr, int,
                         int) const {
@@ -222,17 +217,28 @@ struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row
         if (logits)
             for (int t = tid; t < n_live * kTcBM; t += nthr) {
                 const int n = t / kTcBM, r = t % kTcBM;
-                logits[(size_t)n * V + v0 + r] = tile[r * ld + n];
+                logits[(size_t)n * V + v0 + r] = tile[n * ld + r];
             }
-        for (int n = tid; n < n_live; n += nthr) {
+        // one warp per column: a lane scans four consecutive features, then (max, lowest id) over the warp
+        const int lane = tid & 31;
+        for (int n = tid >> 5; n < n_live; n += nthr >> 5) {
+            const float4 x = *reinterpret_cast<const float4 *>(tile + n * ld + 4 * lane);
             float bv = -CUDART_INF_F;
             int bi = 0x7fffffff;
-            for (int r = 0; r < kTcBM; ++r) {
-                const float v = tile[r * ld + n];
-                if (v > bv) { bv = v; bi = v0 + r; }
+            if (x.x > bv) { bv = x.x; bi = v0 + 4 * lane; }
+            if (x.y > bv) { bv = x.y; bi = v0 + 4 * lane + 1; }
+            if (x.z > bv) { bv = x.z; bi = v0 + 4 * lane + 2; }
+            if (x.w > bv) { bv = x.w; bi = v0 + 4 * lane + 3; }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
             }
-            part_val[(size_t)n * n_parts + tile_idx] = bv;
-            part_idx[(size_t)n * n_parts + tile_idx] = bi;
+            if (lane == 0) {
+                part_val[(size_t)n * n_parts + tile_idx] = bv;
+                part_idx[(size_t)n * n_parts + tile_idx] = bi;
+            }
         }
     }
 };
@@ -250,7 +256,89 @@ struct TcArgs {
     const int32_t *cnt;    // live operand rows (device)
     const int32_t *hint;   // a count of those rows that is never too low: 0 means there are certainly none
     int *dev_err;
+    unsigned long long *probe;  // optional [8]: global timer at the milestones of CTA 0 (debugging aid)
 };
+
+__device__ __forceinline__ void tc_stamp(unsigned long long *probe, int k) {
+    if (probe && blockIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        probe[k] = t;
+    }
+}
+
+// ---------------------------------------------------------------- the common tail of the tensor-core GEMM kernels
+// Called by every thread once the accumulator is complete and the pipeline memory is free: moves the accumulator
+// from TMEM to shared memory (column by column, see the epilogues), frees TMEM, adds up the K-split partial tiles over
+// the cluster and runs the epilogue.
+//
+// Reduce-scatter over the cluster: CTA `split` owns whole quads of row pairs and adds them up, in split order, from
+// every peer's shared memory with 128-bit distributed-shared-memory loads, all peers' loads in flight together; the
+// sums replace its own partial values in place (peers only ever read the rows of THEIR slices).  A CTA may not
+// exit while a peer still reads its tile: it arrives at the second cluster barrier right after its own reads and waits
+// for it after its epilogue.  Even a CTA that gave up takes part in both barriers: a cluster barrier has no time-out.
+template <class Epi>
+__device__ __forceinline__ void tc_finish(const Epi &epi, float *tile, uint32_t tmem_d, uint32_t tmem_cols, int NP,
+                                          int splits, int split, int tile_idx, int n_live, const int32_t *rows, bool ok,
+                                          const int *s_abort, int nthr, unsigned long long *probe) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (warp >= 2 && warp < 6 && ok && n_live > 0) {
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        float *col = tile + q * 32 + lane;
+        for (int c0 = 0; c0 < NP; c0 += 16) {
+            float v[16];
+            tc_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) col[(c0 + j) * kTcLd] = v[j];
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols));
+    }
+    if (n_live <= 0) return;  // uniform over the cluster: nobody waits for anybody
+    const bool good = ok && !*reinterpret_cast<const volatile int *>(s_abort);
+    int pr0 = 0, pr1 = kTcBM / 2;
+    if (splits > 1) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        const int q0 = 16 * split / splits, nq = 16 * (split + 1) / splits - q0;
+        pr0 = 4 * q0;
+        pr1 = 4 * (q0 + nq);
+        if (good) {
+            const int per_col = 2 * nq;
+            for (int t = tid; t < NP * per_col; t += nthr) {
+                const int n = t / per_col, r = epi.quad_row(t % per_col, q0, nq);
+                float *p = tile + n * kTcLd + r;
+                const uint32_t laddr = smem_u32(p);
+                float4 x[8];
+#pragma unroll
+                for (int sp = 0; sp < 8; ++sp) {
+                    x[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (sp < splits) {
+                        uint32_t raddr;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(sp));
+                        asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(x[sp].x), "=f"(x[sp].y), "=f"(x[sp].z), "=f"(x[sp].w)
+                                     : "r"(raddr)
+                                     : "memory");
+                    }
+                }
+                float4 v = x[0];
+#pragma unroll
+                for (int sp = 1; sp < 8; ++sp) { v.x += x[sp].x; v.y += x[sp].y; v.z += x[sp].z; v.w += x[sp].w; }
+                *reinterpret_cast<float4 *>(p) = v;
+            }
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        __syncthreads();
+    }
+    if (tid == 64) tc_stamp(probe, 6);
+    if (good) epi.run(tile, kTcLd, tile_idx, n_live, rows, tid, nthr, pr0, pr1);
+    if (tid == 64) tc_stamp(probe, 7);
+    if (splits > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 template <class Epi>
 __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0,
@@ -266,7 +354,6 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     const uint32_t stage_bytes = a_bytes + 2 * b_bytes;  // multiples of 1024 (n_pad multiple of 16 -> b_bytes of 2048)
     uint8_t *stages = smem;
     float *tile = reinterpret_cast<float *>(stages);     // the finished tile reuses the pipeline memory
-    const int ld = NP + 1;
     uint64_t *bars = reinterpret_cast<uint64_t *>(stages + (size_t)S * stage_bytes);  // full[S], empty[S], acc
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort, s_some;
@@ -279,6 +366,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     while ((int)tmem_cols < NP) tmem_cols <<= 1;
 
     pdl_launch();
+    if (tid == 0) tc_stamp(a.probe, 0);
     if (tid == 0) s_some = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
     __syncthreads();
     if (!s_some) {  // every row has left the backbone: nothing to fetch, nothing to compute (uniform over the cluster:
@@ -337,7 +425,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     const int pre = min(S, nkb);
     if (tid == 0)
         for (int i = 0; i < pre; ++i) load_a(i);
+    if (tid == 0) tc_stamp(a.probe, 1);
     pdl_wait();
+    if (tid == 0) tc_stamp(a.probe, 2);
     const int n_live = *a.cnt;  // rows of the backbone list; the stream kernel serves the exit-layer rows
     // even with no live row the requested weight tiles must land before the CTA may exit: run the pipeline once
     const int nkb_run = n_live > 0 ? nkb : pre;
@@ -358,6 +448,8 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
             for (int i = 0; i < nkb_run; ++i) {
                 const int s = i % S;
                 if (!mbar_wait(smem_u32(&bars[s]), (i / S) & 1, abortp, a.dev_err)) break;
+                if (i == 0) tc_stamp(a.probe, 3);
+                if (i == nkb_run - 1) tc_stamp(a.probe, 4);
                 tc_fence_after();
                 const uint32_t sa = smem_u32(stages + (size_t)s * stage_bytes);
                 const uint64_t da = tc_smem_desc(sa), dhi = tc_smem_desc(sa + a_bytes), dlo = tc_smem_desc(sa + a_bytes + b_bytes);
@@ -376,76 +468,16 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     __syncwarp();
     // everyone: wait for the accumulator (bounded), then move it out of TMEM
     bool ok = mbar_wait(smem_u32(&bars[2 * S]), 0, abortp, a.dev_err);
+    if (tid == 64) tc_stamp(a.probe, 5);
     tc_fence_after();
     __syncthreads();  // all TMA writes and MMA reads of the pipeline memory are over: it now holds the tile
-    if (warp >= 2 && ok && n_live > 0) {
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
-        const int r = q * 32 + lane;
-        for (int c0 = 0; c0 < NP; c0 += 16) {
-            float v[16];
-            tc_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) tile[r * ld + c0 + j] = v[j];
-        }
-        tc_fence_before();
-    }
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols));
-    }
-    if (n_live <= 0) return;  // uniform over the cluster: nobody waits for anybody
-    const bool good = ok && !s_abort;
-    int pr0 = 0, pr1 = kTcBM / 2;
-    if (a.splits > 1) {
-        // Reduce-scatter over the cluster: CTA `split` owns the pairs [pr0, pr1) of the tile and adds them up from
-        // every peer's shared memory in split order.  Even a CTA that gave up takes part in both barriers: a
-        // cluster barrier has no time-out.
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        pr0 = (kTcBM / 2) * split / a.splits;
-        pr1 = (kTcBM / 2) * (split + 1) / a.splits;
-        float *fin = tile + kTcBM * ld;  // [2 * (pr1 - pr0)][NP] behind the tile
-        const int nrows = 2 * (pr1 - pr0);
-        if (good) {
-            for (int t = tid; t < nrows * NP; t += kTcThreads) {
-                const int j = t / NP, n = t % NP;
-                int r0, r1;
-                epi.pair_rows(pr0 + (j >> 1), r0, r1);
-                const int r = (j & 1) ? r1 : r0;
-                const uint32_t laddr = smem_u32(tile + r * ld + n);
-                float x[8];
-#pragma unroll
-                for (int sp = 0; sp < 8; ++sp) {  // all peers' loads in flight together
-                    x[sp] = 0.f;
-                    if (sp < a.splits) {
-                        uint32_t raddr;
-                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(sp));
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x[sp]) : "r"(raddr) : "memory");
-                    }
-                }
-                float v = x[0];
-#pragma unroll
-                for (int sp = 1; sp < 8; ++sp) v += x[sp];
-                fin[j * NP + n] = v;
-            }
-        }
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        if (good) {
-            for (int t = tid; t < nrows * NP; t += kTcThreads) {  // peers are done with my tile: put the sums in place
-                const int j = t / NP, n = t % NP;
-                int r0, r1;
-                epi.pair_rows(pr0 + (j >> 1), r0, r1);
-                tile[((j & 1) ? r1 : r0) * ld + n] = fin[j * NP + n];
-            }
-        }
-        __syncthreads();
-    }
-    if (good) epi.run(tile, ld, tile_idx, n_live, a.rows, tid, kTcThreads, pr0, pr1);
+    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kTcThreads,
+              a.probe);
 }
 
 inline size_t tc_smem_bytes(int n_pad, int n_stages) {
     const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)n_pad * kTcBK * 2;
-    const size_t pipe = (size_t)n_stages * stage;  // the tile and the reduced slice reuse it (the host checks the fit)
+    const size_t pipe = (size_t)n_stages * stage;  // the finished tile reuses it (the host checks the fit)
     return 1024 + pipe + sizeof(uint64_t) * (2 * n_stages + 1) + 64;
 }
 

@@ -34,7 +34,8 @@ __device__ __forceinline__ uint32_t tc_idesc_f16(int n) {  // D fp32, A and B f1
 }
 
 // ---------------------------------------------------------------- activation rows -> f16 hi / lo operand buffers
-// As tc_prep_kernel, but f16 and with the inputs of every group of eight in the order (0,4,1,5,2,6,3,7).
+// As tc_prep_kernel (CTA (i, j): inputs [2048 j, 2048 j + 2048) of operand row i, eight per thread), but f16 and with
+// the inputs of every group of eight in the order (0,4,1,5,2,6,3,7).
 __global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
                                                          __half *xhi, __half *xlo) {
     __shared__ float red[8];
@@ -42,52 +43,44 @@ __global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in, const 
     pdl_wait();
     const int i = blockIdx.x, n = *cnt;
     if (n <= 0) return;  // no row on the exit layers: the GEMM returns before it reads an operand
+    const int v = blockIdx.y * (2 * kPrepChunk / 8) + threadIdx.x;  // 8-input group of the row
+    const bool mine = v < (K >> 3);
     uint4 *hi = reinterpret_cast<uint4 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint4 *>(xlo + (size_t)i * K);
-    const int n8 = K >> 3;
     if (i >= n) {
-        for (int v = threadIdx.x; v < n8; v += blockDim.x) { hi[v] = make_uint4(0u, 0u, 0u, 0u); lo[v] = make_uint4(0u, 0u, 0u, 0u); }
+        if (mine) { hi[v] = make_uint4(0u, 0u, 0u, 0u); lo[v] = make_uint4(0u, 0u, 0u, 0u); }
         return;
     }
     const float4 *src = reinterpret_cast<const float4 *>(in.src + (size_t)idx[i] * K);
-    float scale = 1.f;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    uint4 gw = make_uint4(0u, 0u, 0u, 0u);
+    if (mine) {
+        a = __ldcg(src + 2 * v);
+        b = __ldcg(src + 2 * v + 1);
+        if (in.gain) gw = *reinterpret_cast<const uint4 *>(in.gain + 8 * v);
+    }
+    const float scale = tc_prep_scale(in, src, K, red);
+    if (!mine) return;
+    float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     if (in.gain) {
-        float ss = 0.f;
-        for (int v = threadIdx.x; v < (K >> 2); v += blockDim.x) {
-            const float4 x = __ldcg(src + v);
-            ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-        }
-        ss = warp_sum(ss);
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-        __syncthreads();
-        ss = 0.f;
-        for (int w = 0; w < 8; ++w) ss += red[w];
-        scale = rsqrtf(ss / (float)K + in.eps);
-    }
-    for (int v = threadIdx.x; v < n8; v += blockDim.x) {
-        const float4 a = __ldcg(src + 2 * v), b = __ldcg(src + 2 * v + 1);
-        float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        if (in.gain) {
-            const uint4 gw = *reinterpret_cast<const uint4 *>(in.gain + 8 * v);
-            const uint32_t g[4] = {gw.x, gw.y, gw.z, gw.w};
+        const uint32_t g[4] = {gw.x, gw.y, gw.z, gw.w};
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                x[2 * q] *= scale * bf16lo(g[q]);
-                x[2 * q + 1] *= scale * bf16hi(g[q]);
-            }
+        for (int q = 0; q < 4; ++q) {
+            x[2 * q] = x[2 * q] * scale * bf16lo(g[q]);
+            x[2 * q + 1] = x[2 * q + 1] * scale * bf16hi(g[q]);
         }
-        unsigned short h[8], l[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const __half hv = __float2half_rn(x[q]);
-            h[q] = __half_as_ushort(hv);
-            l[q] = __half_as_ushort(__float2half_rn(x[q] - __half2float(hv)));
-        }
-        // storage position p holds input perm[p], perm = (0,4,1,5,2,6,3,7)
-        hi[v] = make_uint4((uint32_t)h[0] | ((uint32_t)h[4] << 16), (uint32_t)h[1] | ((uint32_t)h[5] << 16),
-                           (uint32_t)h[2] | ((uint32_t)h[6] << 16), (uint32_t)h[3] | ((uint32_t)h[7] << 16));
-        lo[v] = make_uint4((uint32_t)l[0] | ((uint32_t)l[4] << 16), (uint32_t)l[1] | ((uint32_t)l[5] << 16),
-                           (uint32_t)l[2] | ((uint32_t)l[6] << 16), (uint32_t)l[3] | ((uint32_t)l[7] << 16));
     }
+    unsigned short h[8], l[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const __half hv = __float2half_rn(x[q]);
+        h[q] = __half_as_ushort(hv);
+        l[q] = __half_as_ushort(__float2half_rn(x[q] - __half2float(hv)));
+    }
+    // storage position p holds input perm[p], perm = (0,4,1,5,2,6,3,7)
+    hi[v] = make_uint4((uint32_t)h[0] | ((uint32_t)h[4] << 16), (uint32_t)h[1] | ((uint32_t)h[5] << 16),
+                       (uint32_t)h[2] | ((uint32_t)h[6] << 16), (uint32_t)h[3] | ((uint32_t)h[7] << 16));
+    lo[v] = make_uint4((uint32_t)l[0] | ((uint32_t)l[4] << 16), (uint32_t)l[1] | ((uint32_t)l[5] << 16),
+                       (uint32_t)l[2] | ((uint32_t)l[6] << 16), (uint32_t)l[3] | ((uint32_t)l[7] << 16));
 }
 
 // ---------------------------------------------------------------- the kernel
@@ -141,7 +134,6 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
     uint8_t *stages = smem;
     uint8_t *raw = stages + (size_t)S * stage_bytes;                 // kW4RawBufs raw code tiles, 1024-aligned
     float *tile = reinterpret_cast<float *>(stages);                 // the finished tile reuses stages + raw
-    const int ld = NP + 1;
     // barriers: a_full[S], b_full[S], empty[S], raw_full[R], raw_empty[R], acc
     uint64_t *bars = reinterpret_cast<uint64_t *>(raw + (size_t)kW4RawBufs * kW4RawBytes);
     uint64_t *b_afull = bars, *b_bfull = bars + S, *b_empty = bars + 2 * S, *b_rfull = bars + 3 * S,
@@ -313,66 +305,8 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
     bool ok = n_live > 0 ? mbar_wait(smem_u32(b_acc), 0, abortp, a.dev_err) : true;
     tc_fence_after();
     __syncthreads();  // all copies into and MMA reads of the pipeline memory are over: it now holds the tile
-    if (warp >= 2 && warp < 6 && ok && n_live > 0) {
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
-        const int r = q * 32 + lane;
-        for (int c0 = 0; c0 < NP; c0 += 16) {
-            float v[16];
-            tc_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) tile[r * ld + c0 + j] = v[j];
-        }
-        tc_fence_before();
-    }
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols));
-    }
-    if (n_live <= 0) return;  // uniform over the cluster
-    const bool good = ok && !s_abort;
-    int pr0 = 0, pr1 = kTcBM / 2;
-    if (a.splits > 1) {
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        pr0 = (kTcBM / 2) * split / a.splits;
-        pr1 = (kTcBM / 2) * (split + 1) / a.splits;
-        float *fin = tile + kTcBM * ld;
-        const int nrows = 2 * (pr1 - pr0);
-        if (good) {
-            for (int t = tid; t < nrows * NP; t += kW4Threads) {
-                const int j = t / NP, n = t % NP;
-                int r0, r1;
-                epi.pair_rows(pr0 + (j >> 1), r0, r1);
-                const int r = (j & 1) ? r1 : r0;
-                const uint32_t laddr = smem_u32(tile + r * ld + n);
-                float x[8];
-#pragma unroll
-                for (int sp2 = 0; sp2 < 8; ++sp2) {
-                    x[sp2] = 0.f;
-                    if (sp2 < a.splits) {
-                        uint32_t raddr;
-                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(sp2));
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x[sp2]) : "r"(raddr) : "memory");
-                    }
-                }
-                float v = x[0];
-#pragma unroll
-                for (int sp2 = 1; sp2 < 8; ++sp2) v += x[sp2];
-                fin[j * NP + n] = v;
-            }
-        }
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        if (good) {
-            for (int t = tid; t < nrows * NP; t += kW4Threads) {
-                const int j = t / NP, n = t % NP;
-                int r0, r1;
-                epi.pair_rows(pr0 + (j >> 1), r0, r1);
-                tile[((j & 1) ? r1 : r0) * ld + n] = fin[j * NP + n];
-            }
-        }
-        __syncthreads();
-    }
-    if (good) epi.run(tile, ld, tile_idx, n_live, a.rows, tid, kW4Threads, pr0, pr1);
+    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kW4Threads,
+              nullptr);
 }
 
 inline size_t tc_w4_smem_bytes(int n_pad, int n_stages) {

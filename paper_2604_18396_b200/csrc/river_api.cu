@@ -490,12 +490,13 @@ const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
     c->tc_bmaps.push_back(b);
     return &c->tc_bmaps.back();
 }
-// K-splits per tile: fill whole waves of the CTA slots (two CTAs per SM when the pipeline fits twice), keep at
-// least four 64-wide k-blocks per split.  The kernel is memory-bound, so what matters is that all CTAs are resident
+// K-splits per tile: fill whole waves of the CTA slots, keep at least four 64-wide k-blocks per split; no split at
+// all when there is a tile for every SM.  The kernel is memory-bound, so what matters is that all CTAs are resident
 // together and every SM slot streams.
 int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots) {
     int best = 1;
     double best_eff = 0.0;
+    if (tiles >= c->num_sms) return 1;  // every SM has a tile of its own: splitting only adds reductions
     for (int s = 1; s <= 8; ++s) {  // a cluster holds at most 8 CTAs
         if (s > 1 && kb_total / s < 4) break;
         const int ctas = tiles * s, waves = (ctas + slots - 1) / slots;
@@ -512,22 +513,41 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
     const int np = (n + 15) / 16 * 16;
     const river_ctx::BMap *bm = tc_bmap(c, K, np);
     if (!bm) return cudaErrorInvalidValue;
-    cudaError_t e = launch_k(tc_prep_kernel, dim3(np), dim3(256), 0, c->stream, true, in, rows, cnt, K, c->tc_xhi, c->tc_xlo);
+    cudaError_t e = launch_k(tc_prep_kernel, dim3(np, (K + kPrepChunk - 1) / kPrepChunk), dim3(256), 0, c->stream, true, in, rows, cnt, K,
+                             c->tc_xhi, c->tc_xlo);
     if (e != cudaSuccess) return e;
     ++c->st.launches_last_step;
     TcArgs a{};
     a.K = K; a.n_pad = np;
     const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
-    a.n_stages = (int)std::max<size_t>(2, std::min<size_t>(8, (106 * 1024) / stage));  // two CTAs per SM if possible
-    const int occ = tc_smem_bytes(np, a.n_stages) <= 113 * 1024 ? 2 : 1;
+    // CTAs per SM: two with three stages each, or three with two when that puts more CTAs of one wave to work (while
+    // one CTA drains its accumulator and takes part in the cluster reduction the others keep the weight stream going);
+    // one with deep stages when the operand tiles are too large for that.
+    const size_t sm_smem = 228 * 1024, fixed = 1024 + 1024 + 256;  // per CTA: system reserve, alignment slack, barriers
+    auto stages_at = [&](int occ) {
+        const size_t room = std::min<size_t>(sm_smem / occ, 227 * 1024);
+        return room < fixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : 3, (room - fixed) / stage);
+    };
+    int occ = stages_at(2) ? 2 : 1;
     a.splits = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * occ);
-    // the finished tile plus the reduced slice of a split CTA live in the pipeline memory
-    const size_t tile_b = sizeof(float) * (size_t)kTcBM * (np + 1);
-    while (a.splits > 1 && tile_b + tile_b / a.splits + 4096 > (size_t)a.n_stages * stage) --a.splits;
+    if (occ == 2 && stages_at(3) && allow_split) {
+        const int s3 = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * 3);
+        if (tiles * s3 > tiles * a.splits && tiles * s3 <= c->num_sms * 3) { occ = 3; a.splits = s3; }
+    }
+    a.n_stages = stages_at(occ);
+    // the finished tile lives in the pipeline memory
+    if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage) return cudaErrorInvalidValue;
     if (!allow_split) a.splits = 1;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     a.rows = rows; a.cnt = cnt; a.dev_err = c->dev_err;
     a.hint = hint ? hint : cnt;
+    static const bool probe_on = std::getenv("RIVER_TC_PROBE") != nullptr;
+    if (probe_on && c->profiling) {
+        const int kind = gateup ? 2 : q_tiles ? 0 : K > c->cfg.d ? 3 : 1;
+        a.probe = c->chain_stamps + 2 + 6 * (size_t)c->cfg.L + 8 * kind;
+        static int printed = 0;
+        if (printed++ < 8) std::fprintf(stderr, "tc kind %d: tiles %d splits %d stages %d np %d nkb %d\n", kind, tiles, a.splits, a.n_stages, np, K / kTcBK / a.splits);
+    }
     const size_t smem = tc_smem_bytes(np, a.n_stages);
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
@@ -547,7 +567,8 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
     const int np = (n + 15) / 16 * 16;
     const river_ctx::BMap *bm = tc_bmap(c, K, np);
     if (!bm) return cudaErrorInvalidValue;
-    cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np), dim3(256), 0, c->stream, true, in, rows, cnt, K,
+    cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np, (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk)), dim3(256), 0, c->stream, true, in, rows,
+                             cnt, K,
                              reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(c->tc_xlo));
     if (e != cudaSuccess) return e;
     ++c->st.launches_last_step;
@@ -560,8 +581,7 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
     a.n_stages = two ? (int)std::min<size_t>(4, (110 * 1024 - raw - 4096) / stage)
                      : (int)std::max<size_t>(2, std::min<size_t>(6, (214 * 1024 - raw) / stage));
     a.splits = tc_pick_splits(c, tiles, K / (kTcBK * kW4Super), c->num_sms * (two ? 2 : 1));
-    const size_t tile_b = sizeof(float) * (size_t)kTcBM * (np + 1);
-    while (a.splits > 1 && tile_b + tile_b / a.splits + 4096 > (size_t)a.n_stages * stage + raw) --a.splits;
+    if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage + raw) return cudaErrorInvalidValue;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
     a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
@@ -659,6 +679,16 @@ int profile_collect(river_ctx *c, int n = 0, int n_head = 0, const int32_t *row_
     CUDA_TRY(c, cudaMemcpyAsync(stamps.data(), c->chain_stamps, sizeof(unsigned long long) * stamps.size(),
                                 cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (std::getenv("RIVER_TC_PROBE")) {  // debugging aid: milestones of CTA 0 of the last tensor-core GEMMs
+        const unsigned long long *sub = stamps.data() + 2 + 6 * (size_t)L;
+        const char *names[4] = {"qkv", "o", "gateup", "down"};
+        for (int k = 0; k < 4; ++k) {
+            const unsigned long long *t = sub + 8 * k;
+            std::fprintf(stderr, "tc probe %-7s setup+prefetch %6.2f wait %6.2f first-full %6.2f mainloop %6.2f acc %6.2f drain+reduce %6.2f epilogue %6.2f total %6.2f us\n",
+                         names[k], (t[1] - t[0]) * 1e-3, (t[2] - t[1]) * 1e-3, (t[3] - t[2]) * 1e-3, (t[4] - t[3]) * 1e-3,
+                         (t[5] - t[4]) * 1e-3, (t[6] - t[5]) * 1e-3, (t[7] - t[6]) * 1e-3, (t[7] - t[0]) * 1e-3);
+        }
+    }
     if (std::getenv("RIVER_CHAIN_PROBE")) {  // debugging aid: where CTA 0 of the chain kernel spent the last step
         const unsigned long long *sub = stamps.data() + 2 + 6 * (size_t)L;
         const char *names[6] = {"qkv", "o", "gateup", "down", "attn/decide", "head"};
