@@ -1,12 +1,14 @@
 // a3: ragged GQA decode attention over the paged bf16 KV cache (sm_100a).
 //
 // Work item = (row, kv head, KV split).  A producer warp stages K/V pages of the split in shared memory with TMA
-// (2-D tiled copies, 128-byte swizzle, one mbarrier pair per pipeline stage); four consumer warps each own one page
-// (16 positions) of every 64-position tile and run an independent online softmax over their share: a lane owns one
-// position and half of the head dim for q.K (the GQ query heads of the group share every K/V read), the tile maximum
-// and the probabilities move with warp shuffles, and for P.V a lane owns DH/32 head dims.  The four warp states
-// merge through shared memory into one partial (max, sum, unnormalised output) per (row, head, split); a second
-// small kernel merges the splits.  All arithmetic is fp32, exponentials are base 2 (q is pre-scaled by log2 e).
+// (2-D tiled copies, 128-byte swizzle, one mbarrier pair per pipeline stage); the consumer warps each own one page
+// (16 positions) of every 64-position tile - and, when the group has an even number of query heads, one half of the
+// heads, so that eight warps instead of four hide each other's latencies - and run an independent online softmax over
+// their share: a lane owns one position and half of the head dim for q.K (the query heads of the warp share every
+// K/V read), the tile maximum and the probabilities move with warp shuffles, and for P.V a lane owns DH/32 head dims.
+// The warp states merge through shared memory into one partial (max, sum, unnormalised output) per (row, head,
+// split); the last split of a (row, kv head) to finish merges the splits.  All arithmetic is fp32, exponentials are
+// base 2 (q is pre-scaled by log2 e).
 #pragma once
 #include <cuda.h>
 
@@ -16,8 +18,9 @@ namespace river {
 
 constexpr int kAttnTile = 64;      // positions per pipeline stage (4 pages)
 constexpr int kAttnStages = 3;
-constexpr int kAttnConsumers = 4;  // consumer warps = pages per tile
-constexpr int kAttnThreads = 32 * (kAttnConsumers + 1);
+constexpr int kAttnConsumers = 4;  // pages per tile
+__host__ __device__ constexpr int attn_head_split(int gq) { return gq % 2 == 0 ? 2 : 1; }                          // warps per page
+__host__ __device__ constexpr int attn_threads(int gq) { return 32 * (kAttnConsumers * attn_head_split(gq) + 1); }  // consumers + producer
 constexpr uint32_t kWaitLimit = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -79,8 +82,12 @@ struct AttnArgs {
 };
 
 template <int DH, int GQ>
-__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
-                                                                  const AttnArgs a) {
+__global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                      const AttnArgs a) {
+    constexpr int GS = attn_head_split(GQ);      // warps per page
+    constexpr int GW = GQ / GS;                  // query heads per warp
+    constexpr int NW = kAttnConsumers * GS;      // consumer warps
+    constexpr int kAttnThreads = attn_threads(GQ);
     constexpr int NB = DH / 64;                  // 128-byte boxes per cache row
     constexpr int PAGE_BYTES = kPage * DH * 2;   // one page of K (or V) of one kv head
     constexpr int STAGE_BYTES = 2 * kAttnConsumers * PAGE_BYTES;
@@ -95,17 +102,17 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *stages = smem;                                            // kAttnStages * STAGE_BYTES, 1024-aligned
     float *sq = reinterpret_cast<float *>(stages + kAttnStages * STAGE_BYTES);  // [GQ][DH]
-    float *sp = sq + GQ * DH;                                          // [4 warps][16][GQ]
+    float *sp = sq + GQ * DH;                                          // [NW warps][16][GW]
     float *sm = sp + kAttnConsumers * kPage * GQ;                      // merge: [4][GQ][DH + 2]
     uint64_t *bars = reinterpret_cast<uint64_t *>(sm + kAttnConsumers * GQ * (DH + 2));  // full[S], empty[S]
     __shared__ int s_abort;
     __shared__ bool s_last;
-    const bool is_producer = tid == kAttnConsumers * 32;
+    const bool is_producer = tid == NW * 32;
     if (is_producer) {  // nothing here depends on the previous kernel
         s_abort = 0;
         for (int s = 0; s < kAttnStages; ++s) {
             mbar_init(smem_u32(&bars[s]), 1);
-            mbar_init(smem_u32(&bars[kAttnStages + s]), kAttnConsumers);
+            mbar_init(smem_u32(&bars[kAttnStages + s]), NW);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -154,33 +161,35 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
         sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
     __syncthreads();
 
-    if (warp == kAttnConsumers) {
+    if (warp == NW) {
         if (lane == 0)
             for (int t = kAttnStages; t < n_tiles; ++t)
                 if (!issue_tile(t)) break;
     } else {
-        // ---------------- consumers: warp w owns page w of every tile
+        // ---------------- consumers: warp w owns page w % 4 of every tile and the heads [g0, g0 + GW) of the group
         const int r = lane & 15, hsel = lane >> 4;
-        float m[GQ], l[GQ], acc[GQ][VE];
+        const int pg = warp & (kAttnConsumers - 1), g0 = (warp / kAttnConsumers) * GW;
+        const float *wq = sq + g0 * DH;
+        float m[GW], l[GW], acc[GW][VE];
 #pragma unroll
-        for (int g = 0; g < GQ; ++g) {
+        for (int g = 0; g < GW; ++g) {
             m[g] = -CUDART_INF_F;
             l[g] = 0.f;
 #pragma unroll
             for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
         }
-        float *my_sp = sp + warp * kPage * GQ;
+        float *my_sp = sp + warp * kPage * GW;
         for (int t = 0; t < n_tiles; ++t) {
             const int s = t % kAttnStages;
             if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
-            const int page_pos0 = p0 + t * kAttnTile + warp * kPage;  // first position of this warp's page
+            const int page_pos0 = p0 + t * kAttnTile + pg * kPage;  // first position of this warp's page
             if (page_pos0 < p1) {
-                const uint8_t *kpg = stages + s * STAGE_BYTES + warp * PAGE_BYTES;
+                const uint8_t *kpg = stages + s * STAGE_BYTES + pg * PAGE_BYTES;
                 const uint8_t *vpg = kpg + kAttnConsumers * PAGE_BYTES;
                 // q.K for position r, dims [hsel*DH/2, (hsel+1)*DH/2)
-                float sc[GQ];
+                float sc[GW];
 #pragma unroll
-                for (int g = 0; g < GQ; ++g) sc[g] = 0.f;
+                for (int g = 0; g < GW; ++g) sc[g] = 0.f;
 #pragma unroll
                 for (int i = 0; i < NCH; ++i) {
                     const int cg = hsel * NCH + i, box = cg >> 3, c = cg & 7;
@@ -189,9 +198,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
                     const float k0 = bf16lo(kw.x), k1 = bf16hi(kw.x), k2 = bf16lo(kw.y), k3 = bf16hi(kw.y);
                     const float k4 = bf16lo(kw.z), k5 = bf16hi(kw.z), k6 = bf16lo(kw.w), k7 = bf16hi(kw.w);
 #pragma unroll
-                    for (int g = 0; g < GQ; ++g) {
-                        const float4 qa = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8);
-                        const float4 qb = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8 + 4);
+                    for (int g = 0; g < GW; ++g) {
+                        const float4 qa = *reinterpret_cast<const float4 *>(wq + g * DH + cg * 8);
+                        const float4 qb = *reinterpret_cast<const float4 *>(wq + g * DH + cg * 8 + 4);
                         float v = sc[g];
                         v = fmaf(qa.x, k0, v); v = fmaf(qa.y, k1, v); v = fmaf(qa.z, k2, v); v = fmaf(qa.w, k3, v);
                         v = fmaf(qb.x, k4, v); v = fmaf(qb.y, k5, v); v = fmaf(qb.z, k6, v); v = fmaf(qb.w, k7, v);
@@ -199,9 +208,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
                     }
                 }
                 const bool live = page_pos0 + r < p1;
-                float corr[GQ];
+                float corr[GW];
 #pragma unroll
-                for (int g = 0; g < GQ; ++g) {
+                for (int g = 0; g < GW; ++g) {
                     float v = sc[g] + __shfl_xor_sync(0xffffffffu, sc[g], 16);
                     v = live ? v : -CUDART_INF_F;  // select, never arithmetic: stale cache rows may hold anything
                     float mx = v;
@@ -211,8 +220,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
                     corr[g] = ex2(m[g] - mn);
                     m[g] = mn;
                     const float p = live ? ex2(v - mn) : 0.f;
-                    if (hsel == 0) my_sp[r * GQ + g] = p;
-                    l[g] *= corr[g];
+                    if (hsel == 0) my_sp[r * GW + g] = p;
+                    l[g] = fmaf(l[g], corr[g], hsel == 0 ? p : 0.f);  // this lane's share of the sum; added up at the end
 #pragma unroll
                     for (int e = 0; e < VE; ++e) acc[g][e] *= corr[g];
                 }
@@ -231,9 +240,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
                         vf[0] = bf16lo(w); vf[1] = bf16hi(w);
                     }
 #pragma unroll
-                    for (int g = 0; g < GQ; ++g) {
-                        const float p = my_sp[j * GQ + g];
-                        l[g] += p;
+                    for (int g = 0; g < GW; ++g) {
+                        const float p = my_sp[j * GW + g];
 #pragma unroll
                         for (int e = 0; e < VE; ++e) acc[g][e] = fmaf(p, vf[e], acc[g][e]);
                     }
@@ -244,11 +252,12 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
         }
         // publish this warp's state
 #pragma unroll
-        for (int g = 0; g < GQ; ++g) {
-            float *dst = sm + (warp * GQ + g) * (DH + 2);
+        for (int g = 0; g < GW; ++g) {
+            float *dst = sm + (pg * GQ + g0 + g) * (DH + 2);
 #pragma unroll
             for (int e = 0; e < VE; ++e) dst[lane * VE + e] = acc[g][e];
-            if (lane == 0) { dst[DH] = m[g]; dst[DH + 1] = l[g]; }
+            const float lsum = warp_sum(l[g]);
+            if (lane == 0) { dst[DH] = m[g]; dst[DH + 1] = lsum; }
         }
     }
     __syncthreads();

@@ -79,7 +79,7 @@ struct river_ctx {
     bool chain_ok = false;
     bool rows_distinct = true;  // every row of the current step is a different sequence (decode), not a prefill chunk
     int chain_grid = 0, chain_pf_bytes = 4 * 1024;
-    struct GraphEntry { int n; bool small_attn; cudaGraphExec_t exec; int launches; };
+    struct GraphEntry { int n; bool small_attn; int attn_splits; cudaGraphExec_t exec; int launches; };
     std::vector<GraphEntry> graphs;
     double *inv_freq;
     int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
@@ -250,17 +250,43 @@ W4 w4(const river_w4 &r) {
     return W4{(const uint8_t *)r.codes, (const uint16_t *)r.scale, (const uint16_t *)r.zero};
 }
 
-// KV split geometry of this step: enough (row, kv head, split) work items to fill the GPU about twice over,
-// splits of at least two 64-position tiles.  The split count depends only on the row count, so a captured launch
-// stays valid while the chunk length grows with the context.
+// KV split geometry of this step.  A (row, kv head, split) item costs its positions plus a fixed start-up overhead
+// worth about two 64-position tiles, and splitting at all adds the merge through global memory (about five tiles'
+// time, once); items are handed to the CTA slots in launch order, so a step lasts about (all positions / slots) +
+// half of the longest item + the overheads a slot pays (constants fitted to measurements at 64 rows with equal and
+// with mixed lengths).  The split count that minimises this estimate is taken from a short list: one split when the rows are equally long and outnumber the slots
+// (splitting only adds overhead), several when the lengths are mixed, and at least enough to give every slot an item.  Splits are whole tiles,
+// at least two.  The split count is part of a captured launch's key; the chunk length lives in the step metadata.
 void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     const river_config &g = c->cfg;
     int max_pos = 0;
-    for (int i = 0; i < n; ++i) max_pos = std::max(max_pos, mh[kMetaHdr + g.max_batch + i]);
-    int S = (2 * c->num_sms + n * g.Hkv - 1) / (n * g.Hkv);
-    S = std::max(1, std::min(S, 64));
-    int chunk = (max_pos + 1 + S - 1) / S;
-    chunk = std::max(2 * kAttnTile, (chunk + kAttnTile - 1) / kAttnTile * kAttnTile);
+    double total = 0.0;
+    for (int i = 0; i < n; ++i) {
+        const int pos = mh[kMetaHdr + g.max_batch + i];
+        max_pos = std::max(max_pos, pos);
+        total += pos + 1;
+    }
+    const double slots = 2.0 * c->num_sms, ovh = 120.0 * 128.0 / g.dh, merge = 350.0 * 128.0 / g.dh;
+    const int s_cap = std::max(1, std::min(64, (g.max_batch + 600) / n));  // the partials hold max_batch + 600 (row, split) slots
+    static const int cand[] = {1, 2, 3, 4, 5, 6, 8, 12, 16, 24, 32, 48, 64};
+    int S = 1, chunk = 0;
+    double best = 0.0;
+    // fewer items than slots: at least fill the slots
+    const int s_lo = std::min(s_cap, (int)((slots + n * g.Hkv - 1) / (n * g.Hkv)));
+    for (int k = -1; k < (int)(sizeof(cand) / sizeof(cand[0])); ++k) {
+        const int s = k < 0 ? s_lo : cand[k];
+        if (k >= 0 && (s <= s_lo || s > s_cap)) continue;
+        int ch = (max_pos + 1 + s - 1) / s;
+        ch = std::max(2 * kAttnTile, (ch + kAttnTile - 1) / kAttnTile * kAttnTile);
+        double items = 0.0;
+        for (int i = 0; i < n; ++i) items += (mh[kMetaHdr + g.max_batch + i] + ch) / ch;  // ceil((pos + 1) / ch)
+        items *= g.Hkv;
+        const int longest = std::min(ch, max_pos + 1);
+        const double t = std::max(total * g.Hkv / slots + 0.5 * longest, (double)longest) + ovh * std::max(1.0, items / slots) +
+                         (s > 1 ? merge : 0.0);
+        if (chunk == 0 || t < best * 0.97) { best = t; S = s; chunk = ch; }
+        if (ch == 2 * kAttnTile) break;  // finer splits do not exist
+    }
     mh[3] = chunk;
     mh[4] = S;
     mh[5] = n;  // hint_act: every row starts in the backbone
@@ -302,7 +328,7 @@ cudaError_t launch_attn(river_ctx *c, int n, int layer0, bool pdl) {
         cudaFuncSetAttribute(attn_split_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_set = true;
     }
-    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(kAttnThreads), smem, c->stream,
+    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(attn_threads(GQ)), smem, c->stream,
                     pdl, c->kv_tmap, a);
 }
 
@@ -1078,8 +1104,9 @@ int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
     }
     const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
     if (!use_graph) return run_rows(c, n, n, row_pos_host);
+    const int key_splits = c->attn_small_now ? 0 : c->attn_splits_now;  // the attention grid of the captured launches
     for (auto &ge : c->graphs)
-        if (ge.n == n && ge.small_attn == c->attn_small_now) {
+        if (ge.n == n && ge.small_attn == c->attn_small_now && ge.attn_splits == key_splits) {
             if (!ge.exec) {  // second use: capture
                 cudaGraph_t graph = nullptr;
                 CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -1098,7 +1125,7 @@ int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
             c->st.launches_total += ge.launches;
             return 0;
         }
-    c->graphs.push_back({n, c->attn_small_now, nullptr, 0});
+    c->graphs.push_back({n, c->attn_small_now, key_splits, nullptr, 0});
     return run_rows(c, n, n, row_pos_host);  // first use: plain launches (also sets the kernels' attributes)
 }
 
