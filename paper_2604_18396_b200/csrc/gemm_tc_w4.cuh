@@ -153,13 +153,13 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
         s_abort = 0;
         s_early = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
         for (int s = 0; s < S; ++s) {
-            mbar_init(smem_u32(&b_afull[s]), 32 * kW4DqWarps);
+            mbar_init(smem_u32(&b_afull[s]), kW4DqWarps);  // one arrival per dequantisation warp
             mbar_init(smem_u32(&b_bfull[s]), 1);
             mbar_init(smem_u32(&b_empty[s]), 1);
         }
         for (int r = 0; r < kW4RawBufs; ++r) {
             mbar_init(smem_u32(&b_rfull[r]), 1);
-            mbar_init(smem_u32(&b_rempty[r]), 32 * kW4DqWarps);
+            mbar_init(smem_u32(&b_rempty[r]), kW4DqWarps);
         }
         mbar_init(smem_u32(b_acc), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -273,6 +273,13 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
         uint2 s_next = *reinterpret_cast<const uint2 *>(sp), z_next = *reinterpret_cast<const uint2 *>(zp);
         uint2 s_cur = s_next, z_cur = z_next;
         bool alive = true;
+        // one lane polls a barrier for its warp (256 polling threads would compete with the converting ones for issue
+        // slots); the shuffle hands the outcome, and the ordering the wait established, to the other lanes
+        auto warp_wait = [&](uint32_t bar, uint32_t parity) {
+            int ok = 1;
+            if (lane == 0) ok = mbar_wait(bar, parity, abortp, a.dev_err) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, ok, 0) != 0;
+        };
         for (int i = 0; i < nkb_run && alive; ++i) {
             const int kq = i & (kW4Super - 1), sb = i / kW4Super, rb = sb % kW4RawBufs, s = i % S;
             if (kq == 0) {
@@ -281,9 +288,9 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
                     s_next = *reinterpret_cast<const uint2 *>(sp + (sb + 1) * kW4Super);
                     z_next = *reinterpret_cast<const uint2 *>(zp + (sb + 1) * kW4Super);
                 }
-                if (!mbar_wait(smem_u32(&b_rfull[rb]), (sb / kW4RawBufs) & 1, abortp, a.dev_err)) { alive = false; break; }
+                if (!warp_wait(smem_u32(&b_rfull[rb]), (sb / kW4RawBufs) & 1)) { alive = false; break; }
             }
-            if (i >= S && !mbar_wait(smem_u32(&b_empty[s]), ((i / S) - 1) & 1, abortp, a.dev_err)) { alive = false; break; }
+            if (i >= S && !warp_wait(smem_u32(&b_empty[s]), ((i / S) - 1) & 1)) { alive = false; break; }
             const uint32_t sw = (kq < 2 ? s_cur.x : s_cur.y), zw = (kq < 2 ? z_cur.x : z_cur.y);
             const float sf = (kq & 1) ? bf16hi(sw) : bf16lo(sw), zf = (kq & 1) ? bf16hi(zw) : bf16lo(zw);
             const __half2 s2 = __float2half2_rn(sf), z2 = __float2half2_rn(zf);  // bf16 values are exact in f16 range here
@@ -297,8 +304,11 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
                 *reinterpret_cast<uint4 *>(arow + ((cc ^ (r & 7)) * 16)) = w4_word_to_f16(cw[j], z2, s2);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores -> tensor-core reads
-            mbar_arrive(smem_u32(&b_afull[s]));
-            if (kq == kW4Super - 1) mbar_arrive(smem_u32(&b_rempty[rb]));
+            __syncwarp();  // every lane's stores are fenced (and its reads of the raw tile done): one arrival per warp
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&b_afull[s]));
+                if (kq == kW4Super - 1) mbar_arrive(smem_u32(&b_rempty[rb]));
+            }
         }
     }
     __syncwarp();
