@@ -163,6 +163,17 @@ def test_mini8_wide_batches_other_gemm_geometries(rows):
     assert r["n_early"] > 0
 
 
+@pytest.mark.parametrize("lens,flags", [([2200, 130, 700, 1, 1500, 300], 0), ([2500, 40], 32), ([1900], 0)])
+def test_mini8_long_ragged_contexts_split_kv(lens, flags):
+    # contexts of hundreds to thousands of positions, mixed in one batch: the KV range of a (row, KV head) is cut into
+    # several splits that meet through the partial buffers and the ticket (six rows: the TMA-fed kernel with the split
+    # count of the host's cost model; flag 32: the same kernel for a two-row step; one row: the small-step kernel with
+    # 30 splits), next to rows with a single, partly filled tile.  Stands in for the exit-aware attention microbenchmark:
+    # scheduled exits differ per row, exit-layer K/V go to the same slots, and the whole cache is compared.
+    r = run_scheduled(model("mini8"), lens, 3, "uniform", page_seed=len(lens), flags=flags, max_batch=8, kv_store=1)
+    assert r["n_early"] > 0
+
+
 # ------------------------------------------------------------------ invariants on the GPU
 def test_identity_river_makes_exits_invisible_on_gpu():
     m = model("tiny", identity=True)
