@@ -260,6 +260,8 @@ def ours(args, wl):
         shape = dataclasses.replace(shape, L=args.layers)
     if args.prompt:
         plo = phi = args.prompt
+    if args.batch:
+        B = args.batch
     L = shape.L
     K, W = args.steps, args.warmup
     n_cal, n_prof, n_e2e = 8, 4, min(K, 64)
@@ -482,6 +484,7 @@ def main():
     ap.add_argument("--no-variant", action="store_true", help="skip the chain-kernel variant measured beside the main arm")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")
     ap.add_argument("--prompt", type=int, default=0, help="profiling aid: override the prompt length")
+    ap.add_argument("--batch", type=int, default=0, help="profiling aid: override the row count (attention sweeps)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -282,8 +282,10 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
         for (int i = 0; i < n; ++i) items += (mh[kMetaHdr + g.max_batch + i] + ch) / ch;  // ceil((pos + 1) / ch)
         items *= g.Hkv;
         const int longest = std::min(ch, max_pos + 1);
-        const double t = std::max(total * g.Hkv / slots + 0.5 * longest, (double)longest) + ovh * std::max(1.0, items / slots) +
-                         (s > 1 ? merge : 0.0);
+        // whole waves of items of the mean length bound it from below as well (equal lengths: 1.3 waves cost 2)
+        const double waves = std::ceil(items / slots), mean_item = total * g.Hkv / items;
+        const double t = std::max(std::max(total * g.Hkv / slots + 0.5 * longest, waves * mean_item), (double)longest) +
+                         ovh * std::max(1.0, items / slots) + (s > 1 ? merge : 0.0);
         if (chunk == 0 || t < best * 0.97) { best = t; S = s; chunk = ch; }
         if (ch == 2 * kAttnTile) break;  // finer splits do not exist
     }
