@@ -1,14 +1,13 @@
 // a3: ragged GQA decode attention over the paged bf16 KV cache (sm_100a).
 //
 // Work item = (row, kv head, KV split).  A producer warp stages K/V pages of the split in shared memory with TMA
-// (2-D tiled copies, 128-byte swizzle, one mbarrier pair per pipeline stage); the consumer warps each own one page
-// (16 positions) of every 64-position tile - and, when the group has an even number of query heads, one half of the
-// heads, so that eight warps instead of four hide each other's latencies - and run an independent online softmax over
-// their share: a lane owns one position and half of the head dim for q.K (the query heads of the warp share every
-// K/V read), the tile maximum and the probabilities move with warp shuffles, and for P.V a lane owns DH/32 head dims.
-// The warp states merge through shared memory into one partial (max, sum, unnormalised output) per (row, head,
-// split); the last split of a (row, kv head) to finish merges the splits.  All arithmetic is fp32, exponentials are
-// base 2 (q is pre-scaled by log2 e).
+// (2-D tiled copies, 128-byte swizzle, one mbarrier pair per pipeline stage); eight consumer warps each own one half
+// page (8 positions) of every 64-position tile and run an independent online softmax over their share: a lane owns one
+// position and a quarter of the head dim for q.K (the GQ query heads of the group share every K/V read, and no K or V
+// element is unpacked twice), the tile maximum and the probabilities move with warp shuffles, and for P.V a lane owns
+// DH/32 head dims.  The eight warp states merge through shared memory (the pipeline stages, free by then) into one
+// partial (max, sum, unnormalised output) per (row, head, split); the last split of a (row, kv head) to finish merges
+// the splits.  All arithmetic is fp32, exponentials are base 2 (q is pre-scaled by log2 e).
 #pragma once
 #include <cuda.h>
 
@@ -19,8 +18,8 @@ namespace river {
 constexpr int kAttnTile = 64;      // positions per pipeline stage (4 pages)
 constexpr int kAttnStages = 3;
 constexpr int kAttnConsumers = 4;  // pages per tile
-__host__ __device__ constexpr int attn_head_split(int gq) { return gq % 2 == 0 ? 2 : 1; }                          // warps per page
-__host__ __device__ constexpr int attn_threads(int gq) { return 32 * (kAttnConsumers * attn_head_split(gq) + 1); }  // consumers + producer
+constexpr int kAttnWarps = 2 * kAttnConsumers;         // consumer warps: two per page, 8 positions each
+constexpr int kAttnThreads = 32 * (kAttnWarps + 1);    // consumers + producer
 constexpr uint32_t kWaitLimit = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -82,16 +81,14 @@ struct AttnArgs {
 };
 
 template <int DH, int GQ>
-__global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
-                                                                      const AttnArgs a) {
-    constexpr int GS = attn_head_split(GQ);      // warps per page
-    constexpr int GW = GQ / GS;                  // query heads per warp
-    constexpr int NW = kAttnConsumers * GS;      // consumer warps
-    constexpr int kAttnThreads = attn_threads(GQ);
+__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                  const AttnArgs a) {
+    constexpr int NW = kAttnWarps;               // consumer warps
+    constexpr int HP = kPage / 2;                // positions per warp and tile
     constexpr int NB = DH / 64;                  // 128-byte boxes per cache row
     constexpr int PAGE_BYTES = kPage * DH * 2;   // one page of K (or V) of one kv head
     constexpr int STAGE_BYTES = 2 * kAttnConsumers * PAGE_BYTES;
-    constexpr int NCH = DH / 16;                 // 16-byte chunks per lane half in q.K
+    constexpr int NCH = DH / 32;                 // 16-byte chunks per lane quarter in q.K
     constexpr int VE = DH / 32;                  // head dims per lane in P.V
 
     const int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
@@ -102,9 +99,9 @@ __global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __gr
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *stages = smem;                                            // kAttnStages * STAGE_BYTES, 1024-aligned
     float *sq = reinterpret_cast<float *>(stages + kAttnStages * STAGE_BYTES);  // [GQ][DH]
-    float *sp = sq + GQ * DH;                                          // [NW warps][16][GW]
-    float *sm = sp + kAttnConsumers * kPage * GQ;                      // merge: [4][GQ][DH + 2]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sm + kAttnConsumers * GQ * (DH + 2));  // full[S], empty[S]
+    float *sp = sq + GQ * DH;                                          // [NW warps][8 positions][GQ]
+    float *sm = reinterpret_cast<float *>(stages);                     // merge: [NW][GQ][DH + 2], in the drained stages
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sp + NW * HP * GQ);  // full[S], empty[S]
     __shared__ int s_abort;
     __shared__ bool s_last;
     const bool is_producer = tid == NW * 32;
@@ -161,76 +158,78 @@ __global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __gr
         sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
     __syncthreads();
 
+    // ---------------- consumers: warp w owns positions [8 (w / 4), + 8) of page w % 4 of every tile
+    const int r8 = lane & 7, qtr = lane >> 3;
+    const int pg = warp & (kAttnConsumers - 1), ph = warp / kAttnConsumers;
+    const int r = ph * HP + r8;  // this lane's position inside the page
+    float m[GQ], l[GQ], acc[GQ][VE];
+#pragma unroll
+    for (int g = 0; g < GQ; ++g) {
+        m[g] = -CUDART_INF_F;
+        l[g] = 0.f;
+#pragma unroll
+        for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
+    }
     if (warp == NW) {
         if (lane == 0)
             for (int t = kAttnStages; t < n_tiles; ++t)
                 if (!issue_tile(t)) break;
     } else {
-        // ---------------- consumers: warp w owns page w % 4 of every tile and the heads [g0, g0 + GW) of the group
-        const int r = lane & 15, hsel = lane >> 4;
-        const int pg = warp & (kAttnConsumers - 1), g0 = (warp / kAttnConsumers) * GW;
-        const float *wq = sq + g0 * DH;
-        float m[GW], l[GW], acc[GW][VE];
-#pragma unroll
-        for (int g = 0; g < GW; ++g) {
-            m[g] = -CUDART_INF_F;
-            l[g] = 0.f;
-#pragma unroll
-            for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
-        }
-        float *my_sp = sp + warp * kPage * GW;
+        float *my_sp = sp + warp * HP * GQ;
         for (int t = 0; t < n_tiles; ++t) {
             const int s = t % kAttnStages;
             if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
-            const int page_pos0 = p0 + t * kAttnTile + pg * kPage;  // first position of this warp's page
-            if (page_pos0 < p1) {
+            const int pos0 = p0 + t * kAttnTile + pg * kPage + ph * HP;  // first position of this warp's half page
+            if (pos0 < p1) {
                 const uint8_t *kpg = stages + s * STAGE_BYTES + pg * PAGE_BYTES;
                 const uint8_t *vpg = kpg + kAttnConsumers * PAGE_BYTES;
-                // q.K for position r, dims [hsel*DH/2, (hsel+1)*DH/2)
-                float sc[GW];
+                // q.K for position r, dims [qtr*DH/4, (qtr+1)*DH/4)
+                float sc[GQ];
 #pragma unroll
-                for (int g = 0; g < GW; ++g) sc[g] = 0.f;
+                for (int g = 0; g < GQ; ++g) sc[g] = 0.f;
 #pragma unroll
                 for (int i = 0; i < NCH; ++i) {
-                    const int cg = hsel * NCH + i, box = cg >> 3, c = cg & 7;
+                    const int cg = qtr * NCH + i, box = cg >> 3, c = cg & 7;
                     const uint4 kw = *reinterpret_cast<const uint4 *>(kpg + box * (kPage * 128) + r * 128 +
                                                                      ((c ^ (r & 7)) << 4));
                     const float k0 = bf16lo(kw.x), k1 = bf16hi(kw.x), k2 = bf16lo(kw.y), k3 = bf16hi(kw.y);
                     const float k4 = bf16lo(kw.z), k5 = bf16hi(kw.z), k6 = bf16lo(kw.w), k7 = bf16hi(kw.w);
 #pragma unroll
-                    for (int g = 0; g < GW; ++g) {
-                        const float4 qa = *reinterpret_cast<const float4 *>(wq + g * DH + cg * 8);
-                        const float4 qb = *reinterpret_cast<const float4 *>(wq + g * DH + cg * 8 + 4);
+                    for (int g = 0; g < GQ; ++g) {
+                        const float4 qa = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8);
+                        const float4 qb = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8 + 4);
                         float v = sc[g];
                         v = fmaf(qa.x, k0, v); v = fmaf(qa.y, k1, v); v = fmaf(qa.z, k2, v); v = fmaf(qa.w, k3, v);
                         v = fmaf(qb.x, k4, v); v = fmaf(qb.y, k5, v); v = fmaf(qb.z, k6, v); v = fmaf(qb.w, k7, v);
                         sc[g] = v;
                     }
                 }
-                const bool live = page_pos0 + r < p1;
-                float corr[GW];
+                const bool live = pos0 + r8 < p1;
+                float corr[GQ];
 #pragma unroll
-                for (int g = 0; g < GW; ++g) {
-                    float v = sc[g] + __shfl_xor_sync(0xffffffffu, sc[g], 16);
+                for (int g = 0; g < GQ; ++g) {
+                    float v = sc[g] + __shfl_xor_sync(0xffffffffu, sc[g], 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
                     v = live ? v : -CUDART_INF_F;  // select, never arithmetic: stale cache rows may hold anything
                     float mx = v;
 #pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    const float mn = fmaxf(m[g], mx);  // finite: position page_pos0 is live
+                    for (int o = 4; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    const float mn = fmaxf(m[g], mx);  // finite: position pos0 is live
                     corr[g] = ex2(m[g] - mn);
                     m[g] = mn;
                     const float p = live ? ex2(v - mn) : 0.f;
-                    if (hsel == 0) my_sp[r * GW + g] = p;
-                    l[g] = fmaf(l[g], corr[g], hsel == 0 ? p : 0.f);  // this lane's share of the sum; added up at the end
+                    if (qtr == 0) my_sp[r8 * GQ + g] = p;
+                    l[g] = fmaf(l[g], corr[g], qtr == 0 ? p : 0.f);  // this lane's share of the sum; added up at the end
 #pragma unroll
                     for (int e = 0; e < VE; ++e) acc[g][e] *= corr[g];
                 }
                 __syncwarp();
                 // P.V: lane owns dims [lane*VE, lane*VE + VE)
-                const int n_live = min(kPage, p1 - page_pos0);
+                const int n_live = min(HP, p1 - pos0);
                 const int vbyte = lane * VE * 2, vbox = vbyte >> 7, vc = (vbyte & 127) >> 4, vo = vbyte & 15;
                 for (int j = 0; j < n_live; ++j) {
-                    const uint8_t *vp = vpg + vbox * (kPage * 128) + j * 128 + ((vc ^ (j & 7)) << 4) + vo;
+                    const int vr = ph * HP + j;
+                    const uint8_t *vp = vpg + vbox * (kPage * 128) + vr * 128 + ((vc ^ (vr & 7)) << 4) + vo;
                     float vf[VE];
                     if (VE == 4) {
                         const uint2 w = *reinterpret_cast<const uint2 *>(vp);
@@ -240,8 +239,8 @@ __global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __gr
                         vf[0] = bf16lo(w); vf[1] = bf16hi(w);
                     }
 #pragma unroll
-                    for (int g = 0; g < GW; ++g) {
-                        const float p = my_sp[j * GW + g];
+                    for (int g = 0; g < GQ; ++g) {
+                        const float p = my_sp[j * GQ + g];
 #pragma unroll
                         for (int e = 0; e < VE; ++e) acc[g][e] = fmaf(p, vf[e], acc[g][e]);
                     }
@@ -250,10 +249,14 @@ __global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __gr
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars[kAttnStages + s]));
         }
-        // publish this warp's state
+    }
+    // every tile that was requested has landed and has been read by every consumer warp (unless the CTA gave up): the
+    // stages may now hold the warp states
+    __syncthreads();
+    if (warp < NW && !s_abort) {
 #pragma unroll
-        for (int g = 0; g < GW; ++g) {
-            float *dst = sm + (pg * GQ + g0 + g) * (DH + 2);
+        for (int g = 0; g < GQ; ++g) {
+            float *dst = sm + (warp * GQ + g) * (DH + 2);
 #pragma unroll
             for (int e = 0; e < VE; ++e) dst[lane * VE + e] = acc[g][e];
             const float lsum = warp_sum(l[g]);
@@ -266,16 +269,16 @@ __global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __gr
         for (int i = 0; i < 2000; ++i) __nanosleep(100);
         return;
     }
-    // merge the four warp states -> one result per head for this split
+    // merge the eight warp states -> one result per head for this split
     const int ns = pos / chunk + 1;  // splits of this row
     for (int t = tid; t < GQ * DH; t += kAttnThreads) {
         const int g = t / DH, e = t % DH;
         float M = -CUDART_INF_F;
 #pragma unroll
-        for (int w = 0; w < kAttnConsumers; ++w) M = fmaxf(M, sm[(w * GQ + g) * (DH + 2) + DH]);
+        for (int w = 0; w < NW; ++w) M = fmaxf(M, sm[(w * GQ + g) * (DH + 2) + DH]);
         float num = 0.f, den = 0.f;
 #pragma unroll
-        for (int w = 0; w < kAttnConsumers; ++w) {
+        for (int w = 0; w < NW; ++w) {
             const float *src = sm + (w * GQ + g) * (DH + 2);
             const float c = (src[DH] == -CUDART_INF_F) ? 0.f : ex2(src[DH] - M);
             num = fmaf(c, src[e], num);
@@ -332,9 +335,8 @@ __global__ void __launch_bounds__(attn_threads(GQ)) attn_split_kernel(const __gr
 }
 
 inline size_t attn_smem_bytes(int DH, int GQ) {
-    const size_t stage = 2 * kAttnConsumers * (size_t)(kPage * DH * 2);
-    return 1024 + kAttnStages * stage + sizeof(float) * ((size_t)GQ * DH + kAttnConsumers * kPage * GQ +
-                                                         (size_t)kAttnConsumers * GQ * (DH + 2)) +
+    const size_t stage = 2 * kAttnConsumers * (size_t)(kPage * DH * 2);  // the warp states reuse the stages
+    return 1024 + kAttnStages * stage + sizeof(float) * ((size_t)GQ * DH + (size_t)kAttnWarps * (kPage / 2) * GQ) +
            2 * kAttnStages * sizeof(uint64_t) + 64;
 }
 

@@ -330,7 +330,7 @@ cudaError_t launch_attn(river_ctx *c, int n, int layer0, bool pdl) {
         cudaFuncSetAttribute(attn_split_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_set = true;
     }
-    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(attn_threads(GQ)), smem, c->stream,
+    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(kAttnThreads), smem, c->stream,
                     pdl, c->kv_tmap, a);
 }
 
