@@ -521,12 +521,12 @@ const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
 // K-splits per tile: fill whole waves of the CTA slots, keep at least four 64-wide k-blocks per split; no split at
 // all when there is a tile for every SM.  The kernel is memory-bound, so what matters is that all CTAs are resident
 // together and every SM slot streams.
-int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots) {
+int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots, int min_kb = 4) {
     int best = 1;
     double best_eff = 0.0;
     if (tiles >= c->num_sms) return 1;  // every SM has a tile of its own: splitting only adds reductions
     for (int s = 1; s <= 8; ++s) {  // a cluster holds at most 8 CTAs
-        if (s > 1 && kb_total / s < 4) break;
+        if (s > 1 && kb_total / s < min_kb) break;
         const int ctas = tiles * s, waves = (ctas + slots - 1) / slots;
         const double eff = (double)ctas / ((double)waves * slots);
         if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
@@ -608,7 +608,10 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
     const bool two = 2 * stage + raw + 4096 <= 110 * 1024;
     a.n_stages = two ? (int)std::min<size_t>(4, (110 * 1024 - raw - 4096) / stage)
                      : (int)std::max<size_t>(2, std::min<size_t>(6, (214 * 1024 - raw) / stage));
-    a.splits = tc_pick_splits(c, tiles, K / (kTcBK * kW4Super), c->num_sms * (two ? 2 : 1));
+    // in raw tiles of four k-blocks: at least four per split, two when K is so short that four would allow only two
+    // splits (measured on the 1B shape, K = 2048: 2 -> 4 splits 35 -> 31 us per layer for QKV, 33 -> 27 us for O)
+    const int raw_tiles = K / (kTcBK * kW4Super);
+    a.splits = tc_pick_splits(c, tiles, raw_tiles, c->num_sms * (two ? 2 : 1), raw_tiles <= 8 ? 2 : 4);
     if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage + raw) return cudaErrorInvalidValue;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
