@@ -16,7 +16,7 @@
 namespace river {
 
 constexpr int kAttnTile = 64;      // positions per pipeline stage (4 pages)
-constexpr int kAttnStages = 3;
+constexpr int kAttnStages = 2;     // two stages of 32 KB (head dim 128): three CTAs per SM, 24 consumer warps
 constexpr int kAttnConsumers = 4;  // pages per tile
 constexpr int kAttnWarps = 2 * kAttnConsumers;         // consumer warps: two per page, 8 positions each
 constexpr int kAttnThreads = 32 * (kAttnWarps + 1);    // consumers + producer

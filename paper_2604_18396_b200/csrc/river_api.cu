@@ -266,7 +266,8 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
         max_pos = std::max(max_pos, pos);
         total += pos + 1;
     }
-    const double slots = 2.0 * c->num_sms, ovh = 120.0 * 128.0 / g.dh, merge = 350.0 * 128.0 / g.dh;
+    // three CTAs of the attention kernel fit per SM (registers; shared memory at head dim 128)
+    const double slots = 3.0 * c->num_sms, ovh = 120.0 * 128.0 / g.dh, merge = 350.0 * 128.0 / g.dh;
     const int s_cap = std::max(1, std::min(64, (g.max_batch + 600) / n));  // the partials hold max_batch + 600 (row, split) slots
     static const int cand[] = {1, 2, 3, 4, 5, 6, 8, 12, 16, 24, 32, 48, 64};
     int S = 1, chunk = 0;
