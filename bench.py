@@ -126,12 +126,10 @@ def draw_model(shape, device):
     return bb, rv
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (taken on a
-# 4-layer model of the same layer shape: kernel, geometry and operands per launch are those of the full model).
-NCU_TRAFFIC = {("8b", "gateup_swiglu"): 235.0e6}
-# decode_chain_kernel: DRAM read + write = 1.0016 x the algorithmic bytes of the captured step; every layer moves the same
-# bytes, so the ratio carries over to the full model.
-NCU_TRAFFIC_RATIO = {("8b", "decode_chain"): 1.0016}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised under
+# profiles/ (taken on a 4-layer model of the same layer shape: kernel, geometry and operands per launch are those of
+# the full model).  None: no capture of the current kernel is on file.
+NCU_TRAFFIC = {}
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle timing
@@ -358,8 +356,8 @@ def ours(args, wl):
     ms_e2e = dist_max((time.perf_counter() - t0) * 1e3)
     step += n_e2e
 
-    # ---- per-kernel timing passes (outside every timed region): events around every launch; for the persistent
-    # chain kernel additionally its phases as CTA 0 saw them on the global timer.  Full depth, then scheduled exits.
+    # ---- per-kernel timing passes (outside every timed region): events around every launch.  Full depth, then
+    # scheduled exits.
     def profile_pass(thresholds):
         nonlocal step
         rv.profile(True)
@@ -378,21 +376,11 @@ def ours(args, wl):
     line = None
     if rank == 0:
         def table(pr):
-            chain = any(r["name"] == "decode_chain" for r in pr)
-            phase_names = ("qkv_rope_kv", "attn_decode", "o_proj_resid", "gateup_swiglu", "down_resid", "exit_score", "lm_head")
-            launches_k = [r for r in pr if not (chain and r["name"] in phase_names)]
-            tot = sum(r["ms_total"] for r in launches_k)
-            row = lambda r, den: {"launches_per_step": r["launches"] // n_prof, "ms_per_step": round(r["ms_total"] / n_prof, 4),
-                                  "share": round(r["ms_total"] / den, 4),
-                                  "GBps": round(r["alg_bytes_total"] / max(r["ms_total"], 1e-9) / 1e6, 1)}
-            out = {r["name"]: row(r, tot) for r in launches_k}
-            if chain:
-                ph = [r for r in pr if r["name"] in phase_names]
-                tot_ph = sum(r["ms_total"] for r in ph)
-                out["decode_chain"]["phases"] = {r["name"]: row(r, tot_ph) for r in ph}
-            return out
-        names = {r["name"]: r for r in prof}
-        dom = names["decode_chain"] if "decode_chain" in names else max(prof, key=lambda r: r["ms_total"])
+            tot = sum(r["ms_total"] for r in pr)
+            return {r["name"]: {"launches_per_step": r["launches"] // n_prof, "ms_per_step": round(r["ms_total"] / n_prof, 4),
+                                "share": round(r["ms_total"] / tot, 4),
+                                "GBps": round(r["alg_bytes_total"] / max(r["ms_total"], 1e-9) / 1e6, 1)} for r in pr}
+        dom = max(prof, key=lambda r: r["ms_total"])
         per_launch_ms = dom["ms_total"] / dom["launches"]
         ach = dom["alg_bytes_total"] / dom["launches"] / (per_launch_ms * 1e-3) / 1e9
         kernels = table(prof)
@@ -418,9 +406,7 @@ def ours(args, wl):
             "early_exit_speedup_vs_full_depth": ms_full / ms,
             "roofline": {"bound": "hbm", "kernel": dom["name"], "achieved": ach, "peak": peak, "unit": "GB/s",
                          "frac": ach / peak,
-                         "traffic": NCU_TRAFFIC.get((shape_name, dom["name"])) or (
-                             NCU_TRAFFIC_RATIO[(shape_name, dom["name"])] * dom["alg_bytes_total"] / dom["launches"]
-                             if (shape_name, dom["name"]) in NCU_TRAFFIC_RATIO else None),
+                         "traffic": NCU_TRAFFIC.get((shape_name, dom["name"])),
                          "peak_kind": peak_kind,
                          "launch_ms": per_launch_ms, "alg_bytes_per_launch": dom["alg_bytes_total"] / dom["launches"],
                          "pass": "full depth, events around every launch"},
@@ -447,27 +433,6 @@ def ours(args, wl):
         line["cpu_baseline"] = None
     stream_ctx.__exit__(None, None, None)
     rv.close()
-    # ---- the other launch plan for 1-4 rows (persistent chain kernel), same model, prompt, tokens and thresholds:
-    # printed beside the main numbers, outside every timed region of the main arm
-    if rank == 0 and world == 1 and B <= 4 and not (flags & 8) and not args.no_variant:
-        cfg2 = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=n_pages, max_batch=max(B, 8),
-                           page_shuffle_seed=seed + 1, flags=flags | 8)
-        rv2 = River(cfg2, bb, rvw)
-        with torch.cuda.stream(rv2.stream):
-            rv2.prefill(slots, prompt, offs)
-            K2 = min(K, 64)
-            t0s = n_cal  # same tokens / thresholds as the main arm's timed exit run
-            timed_steps(rv2, slots_c, slots, toks, inf, logits, nxt, exits, 0, n_cal)
-            timed_steps(rv2, slots_c, slots, toks, taus, logits, nxt, exits, t0s, W)
-            ms_x = timed_steps(rv2, slots_c, slots, toks, taus, logits, nxt, exits, t0s + W, K2)
-            timed_steps(rv2, slots_c, slots, toks, inf, logits, nxt, exits, t0s + W + K2, W)
-            ms_f = timed_steps(rv2, slots_c, slots, toks, inf, logits, nxt, exits, t0s + 2 * W + K2, K2)
-        rv2.close()
-        line["chain_kernel_variant"] = {
-            "flags": flags | 8, "steps": K2, "ms_per_step": ms_x / K2, "tokens_per_s": B * K2 / (ms_x / 1e3),
-            "full_depth_ms_per_step": ms_f / K2,
-            "full_depth_frac_of_measured_peak": bytes_full / (ms_f / K2 * 1e-3) / 1e9 / peak,
-            "note": "steps of 1-4 rows as ONE cooperative launch (river_config.flags | 8)"}
     if rank == 0:
         print(json.dumps(line), flush=True)
 
@@ -479,9 +444,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b_b1", choices=sorted(WORKLOADS))
-    ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay, 8 = persistent chain kernel for 1-4 rows)")
+    ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-variant", action="store_true", help="skip the chain-kernel variant measured beside the main arm")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")
     ap.add_argument("--prompt", type=int, default=0, help="profiling aid: override the prompt length")
     ap.add_argument("--batch", type=int, default=0, help="profiling aid: override the row count (attention sweeps)")

@@ -45,17 +45,12 @@ enum { RIVER_EXIT_PER_TOKEN = 0, RIVER_EXIT_BATCH_MIN = 1 };
 
 /* flags */
 enum {
-    RIVER_F_GRAPH = 1,   /* replay each decode step as a CUDA graph (captured on first use) */
-    RIVER_F_NO_TC = 2,   /* run every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
-    RIVER_F_SIMPLE_ATTN = 4, /* debugging aid: the plain one-CTA-per-(row, kv head) attention kernel without TMA */
-    RIVER_F_CHAIN = 8,       /* steps of 1-4 rows through the persistent chain kernel (one cooperative launch for all
-                                layers and the LM head) instead of one kernel per stage */
-    RIVER_F_NO_W4TC = 16,    /* exit-layer rows of batches on the CUDA-core kernel instead of the dequantising tcgen05 GEMM */
-    RIVER_F_TMA_ATTN = 32,   /* steps of 1-4 rows through the TMA-fed attention kernel too (default: the small-step kernel) */
-    RIVER_F_FUSED_SCORE = 64 /* small steps: exit score / decision / compaction by the last CTA of the down projection
-                                instead of a kernel of its own (measured 1 % slower: the separate kernel overlaps) */
-    /* bits 8-15: tuning aid for the chain kernel, KiB of the next phase's weights each warp requests from the L2
-       ahead of time (0 = default 4) */
+    RIVER_F_GRAPH = 1,    /* replay each decode step as a CUDA graph (captured on first use) */
+    RIVER_F_NO_TC = 2,    /* diagnostic: every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
+    RIVER_F_NO_W4TC = 16, /* diagnostic: exit-layer rows of batches on the CUDA-core kernel instead of the dequantising
+                             tcgen05 GEMM */
+    RIVER_F_TMA_ATTN = 32 /* diagnostic: steps of 1-4 rows through the TMA-fed attention kernel too (default: the
+                             small-step kernel) */
 };
 
 typedef struct river_config {
@@ -113,14 +108,19 @@ size_t river_kv_pool_bytes(const river_config *cfg);
 int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, size_t kv_pool_bytes,
                void *workspace, size_t workspace_bytes, void *cuda_stream, river_ctx **out);
 
-/* Prefill with sequence-level exit (Section 4.2, "Prefill Phase"): every prompt token runs backbone blocks
- * 1..prefill_exit_layer and exit layers above it (prefill_exit_layer = L: the whole backbone), causal attention,
- * and fills the KV cache of every (token, layer).
+/* Prefill with sequence-level exit (Section 4.2, "Prefill Phase"): every token of a prompt runs backbone blocks
+ * 1..e and exit layers above e (e = L: the whole backbone), causal attention, and fills the KV cache of every
+ * (token, layer).
+ *   prefill_exit_layer  e in [entry_layer, L] for every prompt of the call, or -1: chosen per prompt by Eq. 1 with
+ *       the prompt as the batch - the first block l in [max(entry_layer, 1), L-1] after which every position of the
+ *       prompt has s > tau, else L (costs a second pass over the prompts whose depth comes out below L);
+ *   tau     threshold of the -1 rule (unused otherwise);
  *   slots   [host] n_seqs empty sequence slots;   tok [dev] int32 token ids, all prompts concatenated;
  *   offsets [host] n_seqs+1 prefix offsets into tok;
- *   logits_last [dev] fp32 [n_seqs, V] or NULL;  next_tok [dev] int32 [n_seqs] or NULL (greedy, ties -> lowest id). */
+ *   logits_last [dev] fp32 [n_seqs, V] or NULL;  next_tok [dev] int32 [n_seqs] or NULL (greedy, ties -> lowest id);
+ *   depth_out [host] int32 [n_seqs] or NULL: the depth each prompt left the backbone at. */
 int river_prefill(river_ctx *ctx, int n_seqs, const int32_t *slots, const int32_t *tok, const int32_t *offsets,
-                  int prefill_exit_layer, float *logits_last, int32_t *next_tok);
+                  int prefill_exit_layer, float tau, float *logits_last, int32_t *next_tok, int32_t *depth_out);
 
 /* One token-level early-exit decode step (Section 4.2, "Generation Phase"; Eq. 1).
  * Row b appends token tok[b] to sequence slots[b] (distinct slots).  After backbone block l with
@@ -137,7 +137,14 @@ int river_decode_step(river_ctx *ctx, int batch, const int32_t *slots, const int
                       float *scores);
 
 /* The same step with HOST buffers: copies tok / tau / forced_exit to the device, runs the step, copies
- * next_tok / exit_layer (and logits, scores if not NULL) back, and synchronises the stream. */
+ * next_tok / exit_layer (and logits, scores if not NULL) back, and synchronises the stream.
+ *
+ * Device-side errors (a token id or page id out of range, a forced exit layer out of range, a bounded wait that
+ * ran out) are recorded in a sticky error word and the offending access is skipped or redirected; the kernels always
+ * return.  This call, river_stats and river_selftest_wait_timeout read the word back and return RIVER_E_TIMEOUT for
+ * a wait that ran out, RIVER_E_DEVICE otherwise; river_decode_step and river_prefill (which do not synchronise) report
+ * it at the next such call.  Once the host has seen the word the context refuses further steps with the same code
+ * until river_clear_device_error. */
 int river_decode_step_host(river_ctx *ctx, int batch, const int32_t *slots, const int32_t *tok, const float *tau,
                            const int32_t *forced_exit, float *logits, int32_t *next_tok, int32_t *exit_layer,
                            float *scores);
@@ -174,9 +181,12 @@ int river_profile_read(river_ctx *ctx, river_kernel_time *out, int cap, int *n_o
  * allocation would serialise the device.  The scratch (per-CTA partial maxima, per-row arrival counters, 66 KB)
  * is a fixed array in the library's device image; every GPU that loads the library holds it until process exit.
  *   logits [dev] fp32 [n_rows, V];  next_tok [dev] int32 [n_rows]: index of the row maximum, ties -> lowest id
- *   (the rule river_decode_step uses);  cuda_stream: a cudaStream_t (NULL = default stream); the call is
+ *   (the rule river_decode_step uses; NaNs never win, and a row that holds nothing but NaNs yields token 0, as in
+ *   river_decode_step);  cuda_stream: a cudaStream_t (NULL = default stream); the call is
  *   asynchronous on it.
- * n_rows > RIVER_NOALLOC_MAX_ROWS returns RIVER_E_NOMEM (split the batch); bad pointers / sizes RIVER_E_BADARG.
+ * n_rows > RIVER_NOALLOC_MAX_ROWS returns RIVER_E_NOMEM (split the batch); null pointers, n_rows <= 0, V <= 0 or
+ * V > INT_MAX - 128 return RIVER_E_BADARG.  Every call clears the per-row arrival counters with a memset on the
+ * stream before its launch.
  * The first call on a device looks up the scratch array's device address (with that device current); make that
  * first call before any stream capture.  Calls no cudaMalloc / cudaFree or allocating library routine.  All calls
  * on a device share the one array: two calls that overlap on the GPU (different streams) race; issue them on one
@@ -184,9 +194,18 @@ int river_profile_read(river_ctx *ctx, river_kernel_time *out, int cap, int *n_o
 #define RIVER_NOALLOC_MAX_ROWS 64
 int river_argmax_noalloc(const float *logits, int n_rows, int V, int32_t *next_tok, void *cuda_stream);
 
+/* Reset the sticky device error word (synchronises the stream). */
+int river_clear_device_error(river_ctx *ctx);
+
+/* Self-test of the bounded device-side waits: runs the library's mbarrier wait on a barrier nobody completes, with a
+ * poll limit of poll_limit (1 .. 2^20).  The kernel gives up after that many polls, records the time-out and returns;
+ * the call synchronises and returns RIVER_E_TIMEOUT (the expected outcome), leaving the error word set. */
+int river_selftest_wait_timeout(river_ctx *ctx, int poll_limit);
+
 int river_seq_len(const river_ctx *ctx, int slot);       /* tokens cached in the slot, or RIVER_E_BADSLOT */
 int river_release(river_ctx *ctx, int slot);             /* free the slot's pages */
-int river_stats(river_ctx *ctx, river_stats_t *host_out); /* synchronises the stream */
+int river_stats(river_ctx *ctx, river_stats_t *host_out); /* synchronises the stream; fills host_out even when it
+                                                             returns a device-error code */
 void river_destroy(river_ctx *ctx);
 const char *river_last_error(const river_ctx *ctx);      /* ctx may be NULL: error of the last failed river_init */
 

@@ -482,6 +482,35 @@ int orc_prefill(orc_ctx *o, int slot, const int32_t *tokens, int n, int e_p, flo
     return 0;
 }
 
+/*
+ * Prefill whose unified depth is chosen by the exit rule itself (Section 4.2, "Prefill Phase": all tokens of the
+ * prompt exit at one depth; Eq. 1 with the prompt's positions as the batch): the depth is the first block l with
+ * max(entry_layer, 1) <= l <= L-1 after which EVERY prompt position has s^l > tau, else L.  The scores up to that
+ * block involve backbone blocks only, so a first pass runs the whole backbone over the prompt and collects the
+ * scores; the prompt is then redone with orc_prefill at the depth found.  Returns the depth, or a negative code.
+ */
+int orc_prefill_auto(orc_ctx *o, int slot, const int32_t *tokens, int n, float tau, float *logits_last, int32_t *next) {
+    const int L = o->c.L;
+    int32_t nt = 0, el = 0;
+    const int32_t never = L;
+    const float inf = INFINITY;
+    float *sc = (float *)malloc(sizeof(float) * (size_t)L);
+    unsigned char *some_fail = (unsigned char *)calloc((size_t)L + 1, 1);
+    for (int i = 0; i < n; ++i) {
+        const int rc = orc_decode_step(o, 1, &slot, &tokens[i], &inf, &never, NULL, &nt, &el, sc);
+        if (rc) { free(sc); free(some_fail); return rc; }
+        for (int l = 1; l <= L; ++l)
+            if (!(sc[l - 1] > tau)) some_fail[l] = 1;
+    }
+    int depth = L;
+    for (int l = (o->c.entry_layer > 1 ? o->c.entry_layer : 1); l < L; ++l)
+        if (!some_fail[l]) { depth = l; break; }
+    free(sc); free(some_fail);
+    orc_release(o, slot);
+    const int rc = orc_prefill(o, slot, tokens, n, depth, logits_last, next);
+    return rc ? rc : depth;
+}
+
 /* cache access, fp32 [n][Hkv*dh]; K is stored after RoPE */
 int orc_read_kv(const orc_ctx *o, int slot, int layer0, int pos0, int n, float *k_out, float *v_out) {
     const size_t w = (size_t)o->c.Hkv * o->c.dh;

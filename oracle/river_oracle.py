@@ -70,6 +70,7 @@ def lib():
         L.orc_last_lists.argtypes = [C.c_void_p, C.c_int] + [C.c_void_p] * 4
         L.orc_plain_step.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_prefill.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_prefill_auto.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_float, C.c_void_p, C.c_void_p]
         L.orc_read_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_write_kv.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_write_count.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
@@ -195,6 +196,16 @@ class Oracle:
         if rc:
             raise ValueError(f"orc_prefill failed: {rc}")
         return logits, int(nxt.value)
+
+    def prefill_auto(self, slot: int, tokens, tau: float):
+        """Prefill at the depth the exit rule picks for the whole prompt -> (logits, next token, depth)."""
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        logits = np.empty(self.cfg.V, np.float32)
+        nxt = C.c_int32(0)
+        rc = lib().orc_prefill_auto(self.h, slot, _p(tokens), len(tokens), C.c_float(tau), _p(logits), C.addressof(nxt))
+        if rc < 0:
+            raise ValueError(f"orc_prefill_auto failed: {rc}")
+        return logits, int(nxt.value), rc
 
     def read_kv(self, slot: int, layer0: int, pos0: int, n: int):
         w = self.cfg.Hkv * self.cfg.dh

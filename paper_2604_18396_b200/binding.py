@@ -17,8 +17,7 @@ from . import buildlib as _build
 # ---------------------------------------------------------------- C structs (mirror include/river.h)
 RIVER_OK = 0
 RIVER_EXIT_PER_TOKEN, RIVER_EXIT_BATCH_MIN = 0, 1
-RIVER_F_GRAPH, RIVER_F_NO_TC, RIVER_F_SIMPLE_ATTN, RIVER_F_CHAIN, RIVER_F_NO_W4TC, RIVER_F_TMA_ATTN = 1, 2, 4, 8, 16, 32
-RIVER_F_FUSED_SCORE = 64
+RIVER_F_GRAPH, RIVER_F_NO_TC, RIVER_F_NO_W4TC, RIVER_F_TMA_ATTN = 1, 2, 16, 32
 ERR_NAMES = {-1: "BADARG", -2: "SHAPE", -3: "NOMEM", -4: "NOPAGE", -5: "BADSLOT", -6: "DEVICE", -7: "TIMEOUT"}
 
 
@@ -57,7 +56,8 @@ class river_kernel_time(C.Structure):
 
 EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
-           "river_release", "river_stats", "river_destroy", "river_last_error")
+           "river_release", "river_stats", "river_destroy", "river_last_error", "river_clear_device_error",
+           "river_selftest_wait_timeout")
 
 _lib = None
 
@@ -81,7 +81,7 @@ def load():
     L.river_kv_pool_bytes.argtypes = [C.POINTER(river_config)]
     L.river_init.argtypes = [C.POINTER(river_config), C.POINTER(river_weights), vp, C.c_size_t, vp, C.c_size_t, vp,
                              C.POINTER(vp)]
-    L.river_prefill.argtypes = [vp, C.c_int, i32p, vp, i32p, C.c_int, vp, vp]
+    L.river_prefill.argtypes = [vp, C.c_int, i32p, vp, i32p, C.c_int, C.c_float, vp, vp, i32p]
     L.river_decode_step.argtypes = [vp, C.c_int, i32p, vp, vp, vp, vp, vp, vp, vp]
     L.river_decode_step_host.argtypes = [vp, C.c_int, i32p, vp, vp, vp, vp, vp, vp, vp]
     L.river_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
@@ -93,6 +93,8 @@ def load():
     L.river_profile.argtypes = [vp, C.c_int]
     L.river_profile_read.argtypes = [vp, C.POINTER(river_kernel_time), C.c_int, C.POINTER(C.c_int)]
     L.river_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, vp]
+    L.river_clear_device_error.argtypes = [vp]
+    L.river_selftest_wait_timeout.argtypes = [vp, C.c_int]
     L.river_destroy.argtypes = [vp]
     L.river_destroy.restype = None
     L.river_last_error.argtypes = [vp]
@@ -221,11 +223,16 @@ class River:
 
     # -- API (same names as the C entry points)
     def prefill(self, slots: Sequence[int], tok: torch.Tensor, offsets: Sequence[int], prefill_exit_layer=None,
-                logits_last: Optional[torch.Tensor] = None, next_tok: Optional[torch.Tensor] = None):
+                logits_last: Optional[torch.Tensor] = None, next_tok: Optional[torch.Tensor] = None,
+                tau: float = float("inf")) -> List[int]:
+        """river_prefill; prefill_exit_layer None = the whole backbone, -1 = per prompt by Eq. 1 with threshold tau.
+        Returns the depth each prompt left the backbone at."""
         e = self.cfg.L if prefill_exit_layer is None else prefill_exit_layer
+        depth = (C.c_int32 * len(slots))()
         self._order_after_current()
         self._check(load().river_prefill(self.h, len(slots), _i32_host(slots), _dp(tok), _i32_host(offsets), e,
-                                         _dp(logits_last), _dp(next_tok)))
+                                         C.c_float(tau), _dp(logits_last), _dp(next_tok), depth))
+        return list(depth)
 
     def decode_step(self, slots: Sequence[int], tok: torch.Tensor, tau: torch.Tensor,
                     forced_exit: Optional[torch.Tensor], logits: Optional[torch.Tensor], next_tok: torch.Tensor,
@@ -282,8 +289,16 @@ class River:
                      alg_bytes_total=buf[i].alg_bytes_total) for i in range(n.value)]
 
     def stats(self) -> river_stats_t:
+        """river_stats; a device-error return code (-6, -7) is reported through st.device_error, not raised."""
         st = river_stats_t()
         rc = load().river_stats(self.h, C.byref(st))
-        if rc and rc != -6:
+        if rc and rc not in (-6, -7):
             self._check(rc)
         return st
+
+    def clear_device_error(self):
+        self._check(load().river_clear_device_error(self.h))
+
+    def selftest_wait_timeout(self, poll_limit: int) -> int:
+        """river_selftest_wait_timeout: returns the C return code (-7 = the wait ran out, as it should)."""
+        return load().river_selftest_wait_timeout(self.h, poll_limit)

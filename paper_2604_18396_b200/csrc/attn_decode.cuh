@@ -9,9 +9,7 @@
 // partial (max, sum, unnormalised output) per (row, head, split); the last split of a (row, kv head) to finish merges
 // the splits.  All arithmetic is fp32, exponentials are base 2 (q is pre-scaled by log2 e).
 #pragma once
-#include <cuda.h>
-
-#include "river_kernels.cuh"
+#include "mbar_tma.cuh"
 
 namespace river {
 
@@ -20,53 +18,6 @@ constexpr int kAttnStages = 2;     // two stages of 32 KB (head dim 128): three 
 constexpr int kAttnConsumers = 4;  // pages per tile
 constexpr int kAttnWarps = 2 * kAttnConsumers;         // consumer warps: two per page, 8 positions each
 constexpr int kAttnThreads = 32 * (kAttnWarps + 1);    // consumers + producer
-constexpr uint32_t kWaitLimit = 1u << 20;
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after kWaitLimit polls (or when another thread of the CTA already gave up), records the
-// timeout in the device error word and raises the CTA's abort flag.  Returns false on give-up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *dev_err) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicExch(dev_err, DEV_WAIT_TIMEOUT);
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 struct AttnArgs {
     const StepMeta *meta;
     const float *q;        // [rows][Hq*DH]

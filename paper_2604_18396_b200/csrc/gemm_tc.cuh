@@ -14,8 +14,7 @@
 // write, residual add, SwiGLU, logits + argmax partials).
 // Weights do not depend on the previous kernel: their first tiles are requested before the grid dependency resolves.
 #pragma once
-#include "attn_decode.cuh"
-#include "gemv_stream.cuh"
+#include "mbar_tma.cuh"
 
 namespace river {
 
@@ -83,7 +82,7 @@ __device__ __forceinline__ float tc_prep_scale(const ProjIn &in, const float4 *s
     for (int w = 0; w < 8; ++w) ss += red[w];
     return rsqrtf(ss / (float)K + in.eps);
 }
-__global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
+static __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
                                                       __nv_bfloat16 *xhi, __nv_bfloat16 *xlo) {
     __shared__ float red[8];
     pdl_launch();
@@ -256,16 +255,7 @@ struct TcArgs {
     const int32_t *cnt;    // live operand rows (device)
     const int32_t *hint;   // a count of those rows that is never too low: 0 means there are certainly none
     int *dev_err;
-    unsigned long long *probe;  // optional [8]: global timer at the milestones of CTA 0 (debugging aid)
 };
-
-__device__ __forceinline__ void tc_stamp(unsigned long long *probe, int k) {
-    if (probe && blockIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        probe[k] = t;
-    }
-}
 
 // ---------------------------------------------------------------- the common tail of the tensor-core GEMM kernels
 // Called by every thread once the accumulator is complete and the pipeline memory is free: moves the accumulator
@@ -280,7 +270,7 @@ __device__ __forceinline__ void tc_stamp(unsigned long long *probe, int k) {
 template <class Epi>
 __device__ __forceinline__ void tc_finish(const Epi &epi, float *tile, uint32_t tmem_d, uint32_t tmem_cols, int NP,
                                           int splits, int split, int tile_idx, int n_live, const int32_t *rows, bool ok,
-                                          const int *s_abort, int nthr, unsigned long long *probe) {
+                                          const int *s_abort, int nthr) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (warp >= 2 && warp < 6 && ok && n_live > 0) {
         const int q = warp & 3;  // TMEM lane quarter this warp may read
@@ -334,9 +324,7 @@ __device__ __forceinline__ void tc_finish(const Epi &epi, float *tile, uint32_t 
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         __syncthreads();
     }
-    if (tid == 64) tc_stamp(probe, 6);
     if (good) epi.run(tile, kTcLd, tile_idx, n_live, rows, tid, nthr, pr0, pr1);
-    if (tid == 64) tc_stamp(probe, 7);
     if (splits > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
@@ -366,7 +354,6 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     while ((int)tmem_cols < NP) tmem_cols <<= 1;
 
     pdl_launch();
-    if (tid == 0) tc_stamp(a.probe, 0);
     if (tid == 0) s_some = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
     __syncthreads();
     if (!s_some) {  // every row has left the backbone: nothing to fetch, nothing to compute (uniform over the cluster:
@@ -425,9 +412,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     const int pre = min(S, nkb);
     if (tid == 0)
         for (int i = 0; i < pre; ++i) load_a(i);
-    if (tid == 0) tc_stamp(a.probe, 1);
     pdl_wait();
-    if (tid == 0) tc_stamp(a.probe, 2);
     const int n_live = *a.cnt;  // rows of the backbone list; the stream kernel serves the exit-layer rows
     // even with no live row the requested weight tiles must land before the CTA may exit: run the pipeline once
     const int nkb_run = n_live > 0 ? nkb : pre;
@@ -448,8 +433,6 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
             for (int i = 0; i < nkb_run; ++i) {
                 const int s = i % S;
                 if (!mbar_wait(smem_u32(&bars[s]), (i / S) & 1, abortp, a.dev_err)) break;
-                if (i == 0) tc_stamp(a.probe, 3);
-                if (i == nkb_run - 1) tc_stamp(a.probe, 4);
                 tc_fence_after();
                 const uint32_t sa = smem_u32(stages + (size_t)s * stage_bytes);
                 const uint64_t da = tc_smem_desc(sa), dhi = tc_smem_desc(sa + a_bytes), dlo = tc_smem_desc(sa + a_bytes + b_bytes);
@@ -468,11 +451,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     __syncwarp();
     // everyone: wait for the accumulator (bounded), then move it out of TMEM
     bool ok = mbar_wait(smem_u32(&bars[2 * S]), 0, abortp, a.dev_err);
-    if (tid == 64) tc_stamp(a.probe, 5);
     tc_fence_after();
     __syncthreads();  // all TMA writes and MMA reads of the pipeline memory are over: it now holds the tile
-    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kTcThreads,
-              a.probe);
+    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kTcThreads);
 }
 
 inline size_t tc_smem_bytes(int n_pad, int n_stages) {

@@ -36,7 +36,7 @@ __device__ __forceinline__ uint32_t tc_idesc_f16(int n) {  // D fp32, A and B f1
 // ---------------------------------------------------------------- activation rows -> f16 hi / lo operand buffers
 // As tc_prep_kernel (CTA (i, j): inputs [2048 j, 2048 j + 2048) of operand row i, eight per thread), but f16 and with
 // the inputs of every group of eight in the order (0,4,1,5,2,6,3,7).
-__global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
+static __global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
                                                          __half *xhi, __half *xlo) {
     __shared__ float red[8];
     pdl_launch();
@@ -315,8 +315,7 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
     bool ok = n_live > 0 ? mbar_wait(smem_u32(b_acc), 0, abortp, a.dev_err) : true;
     tc_fence_after();
     __syncthreads();  // all copies into and MMA reads of the pipeline memory are over: it now holds the tile
-    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kW4Threads,
-              nullptr);
+    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kW4Threads);
 }
 
 inline size_t tc_w4_smem_bytes(int n_pad, int n_stages) {

@@ -10,7 +10,7 @@
 // the rows still in the backbone (bf16 weights) and the rows in the exit layers (4-bit codes + bf16 scale / zero
 // per group, dequantised on the fly as (q - z) * s); which set is non-empty is read on the device.
 #pragma once
-#include "river_kernels.cuh"
+#include "river_common.cuh"
 
 namespace river {
 
@@ -21,7 +21,8 @@ struct RowLists {
     const int32_t *act_idx, *n_act, *riv_idx, *n_riv;
     const int32_t *hint_act;  // backbone row count as of the latest compaction; never under-counts (a prefetch hint)
     const int32_t *n_rows;    // rows of the step (per-step metadata, stable while the step runs)
-    const uint8_t *exited;    // the sticky exit flags the lists were built from
+    const uint8_t *state;     // sticky exit flags of the rows entering this block (steps of up to four rows build
+                              // their lists from these: one load instead of count -> index)
 };
 
 struct QkvProblem {
@@ -183,6 +184,25 @@ struct GateUpProblem {  // act[row][f] = silu(Wg[f] . y) * (Wu[f] . y)
 };
 
 
+// The exit decision of the block that has just finished, taken by the kernel that consumes its output (steps of up
+// to four rows): Eq. 1 on the block's input and output, strict s > tau in fp32, the eligibility window
+// entry_layer <= l < L, the forced-exit hook and the batch mode.  Every CTA of the launch computes it from the same
+// data with the same reduction order (all CTAs of a launch have the same shape), so all CTAs agree on which weight
+// set every row takes and no kernel boundary is spent on the decision; CTA 0 publishes exit flags, exit layers,
+// scores, the two row lists and the prefetch hint for the kernels and host queries that follow.
+struct DecideArgs {
+    const StepMeta *meta;      // null: this launch takes no decision
+    int l;                     // the block being scored (1-based); its output is this launch's input rows
+    int L, entry_layer, exit_mode;
+    const float *h_prev;       // input of block l, fp32 [rows][K]
+    const uint8_t *state_in;   // exit flags entering block l
+    uint8_t *state_out;        // exit flags entering block l + 1
+    Lists lists;
+    int32_t *hint_act;
+    int32_t *fail;             // optional [slots][L + 1]: set to 1 where a row's score does NOT pass its threshold (the
+    const int32_t *row_slot;   // prefill pass that looks for the unified depth); row_slot maps rows to sequence slots
+};
+
 // Sums of every 32-input chunk of the rows staged in the E = 32 order (all threads of the CTA; ends with a barrier).
 template <int N>
 __device__ __forceinline__ void stream_chunk_sums(const float *xs, float *xsum, int K, int xstride) {
@@ -317,60 +337,104 @@ __device__ __forceinline__ void stream_dots_bf16(const uint16_t *const (&wrow)[R
 }
 
 // 4-bit weights: lane owns the 32-input chunks lane, lane + 32, ... (16 bytes of codes each).
-// sum_k (q_k - z) s x_k over a chunk = s * (sum_k (128 + q_k) x_k - (z + 128) * sum_k x_k), with 128 + q read off
-// the bf16 bit pattern 0x4300 | q; the chunk sums of x are precomputed.
+// sum_k (q_k - z) s x_k over a chunk = s * (sum_k (128 + q_k) x_k - (z + 128) * sum_k x_k): 128 + q is exact in fp32
+// as the bit pattern 0x43000000 | q << 16, which ONE byte permute builds from a word of isolated nibbles, and the
+// products go through the packed two-lane fp32 FMA, so a weight costs one permute and half an FMA issue slot; the
+// chunk sums of x are precomputed.
+template <int R>
+struct W4Batch {
+    static constexpr int PF = R <= 2 ? kStreamPF : kStreamPF / 2;  // chunks per row in flight: 8 code loads per lane
+    uint4 q[R][kStreamPF];      // (sized for the bf16 prefetch that shares these registers)
+    uint32_t sz[R][PF];         // scale (low half) and zero (high half) of the chunk's group, bf16 bits
+};
+
+template <int R>
+__device__ __forceinline__ void stream_issue_w4(const W4 (&wrow)[R], int nch, int gshift, int it0, int lane,
+                                                W4Batch<R> &b) {
+#pragma unroll
+    for (int u = 0; u < W4Batch<R>::PF; ++u) {
+        const int c = (it0 + u) * 32 + lane;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (c < nch) {
+                b.q[r][u] = ldg_stream16(wrow[r].codes + (size_t)c * 16);
+                b.sz[r][u] = (uint32_t)ldg_u16(wrow[r].scale + (c >> gshift)) |
+                             ((uint32_t)ldg_u16(wrow[r].zero + (c >> gshift)) << 16);
+            } else {
+                b.q[r][u] = make_uint4(0u, 0u, 0u, 0u);
+                b.sz[r][u] = 0u;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void ffma2(float2 &acc, const float2 a, const float2 b) {
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%0, %1};\n\t"
+        "fma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
+        : "+f"(acc.x), "+f"(acc.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+}
+// byte j of a word of isolated nibbles -> the fp32 value 128 + nibble
+template <int J>
+__device__ __forceinline__ float w4_byte_f32(uint32_t nib) {
+    return __uint_as_float(__byte_perm(nib, 0x43000000u, 0x7044 | (J << 8)));
+}
+
 template <int N, int R>
 __device__ __forceinline__ void stream_dots_w4(const W4 (&wrow)[R], const float *xs, const float *xsum, int K,
-                                               int xstride, int group, float (&acc)[R][N]) {
+                                               int xstride, int group, bool have_pre, const W4Batch<R> &pre,
+                                               float (&acc)[R][N]) {
     const int lane = threadIdx.x & 31;
-    const int nch = K >> 5;
+    const int nch = K >> 5, nit = (nch + 31) >> 5;
     const int gshift = (group == 64) ? 1 : (group == 32 ? 0 : 2);
 #pragma unroll
     for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
-#pragma unroll 4
-    for (int c = lane; c < nch; c += 32) {
-        uint4 q[R];
-        float s[R], zz[R];
+    for (int it0 = 0; it0 < nit; it0 += W4Batch<R>::PF) {
+        W4Batch<R> b;
+        if (it0 == 0 && have_pre) b = pre;
+        else stream_issue_w4<R>(wrow, nch, gshift, it0, lane, b);
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            q[r] = ldg_stream16(wrow[r].codes + (size_t)c * 16);
-            s[r] = bf16f(ldg_u16(wrow[r].scale + (c >> gshift)));
-            zz[r] = bf16f(ldg_u16(wrow[r].zero + (c >> gshift))) + 128.f;
-        }
+        for (int u = 0; u < W4Batch<R>::PF; ++u) {
+            const int c = (it0 + u) * 32 + lane;
+            if (c < nch) {
 #pragma unroll
-        for (int n = 0; n < N; ++n) {
-            const float *xb = xs + n * xstride + (c >> 5) * 1024 + lane * 4;
-            float p0[R], p1[R];
+                for (int n = 0; n < N; ++n) {
+                    const float *xb = xs + n * xstride + (c >> 5) * 1024 + lane * 4;
+                    float2 p[R];
 #pragma unroll
-            for (int r = 0; r < R; ++r) { p0[r] = 0.f; p1[r] = 0.f; }
+                    for (int r = 0; r < R; ++r) p[r] = make_float2(0.f, 0.f);
 #pragma unroll
-            for (int wd = 0; wd < 4; ++wd) {  // code word wd holds inputs 8*wd .. 8*wd+7 of the chunk
-                const float4 x0 = *reinterpret_cast<const float4 *>(xb + (2 * wd) * 128);
-                const float4 x1 = *reinterpret_cast<const float4 *>(xb + (2 * wd + 1) * 128);
+                    for (int wd = 0; wd < 4; ++wd) {  // code word wd holds inputs 8*wd .. 8*wd+7 of the chunk
+                        const float4 x0 = *reinterpret_cast<const float4 *>(xb + (2 * wd) * 128);
+                        const float4 x1 = *reinterpret_cast<const float4 *>(xb + (2 * wd + 1) * 128);
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const uint32_t v = wd == 0 ? q[r].x : (wd == 1 ? q[r].y : (wd == 2 ? q[r].z : q[r].w));
-                    const uint32_t b0 = (v & 0x000f000fu) | 0x43004300u;          // inputs 0, 4
-                    const uint32_t b1 = ((v >> 4) & 0x000f000fu) | 0x43004300u;   // inputs 1, 5
-                    const uint32_t b2 = ((v >> 8) & 0x000f000fu) | 0x43004300u;   // inputs 2, 6
-                    const uint32_t b3 = ((v >> 12) & 0x000f000fu) | 0x43004300u;  // inputs 3, 7
-                    p0[r] = fmaf(bf16lo(b0), x0.x, p0[r]); p1[r] = fmaf(bf16lo(b1), x0.y, p1[r]);
-                    p0[r] = fmaf(bf16lo(b2), x0.z, p0[r]); p1[r] = fmaf(bf16lo(b3), x0.w, p1[r]);
-                    p0[r] = fmaf(bf16hi(b0), x1.x, p0[r]); p1[r] = fmaf(bf16hi(b1), x1.y, p1[r]);
-                    p0[r] = fmaf(bf16hi(b2), x1.z, p0[r]); p1[r] = fmaf(bf16hi(b3), x1.w, p1[r]);
+                        for (int r = 0; r < R; ++r) {
+                            const uint4 q = b.q[r][u];
+                            const uint32_t v = wd == 0 ? q.x : (wd == 1 ? q.y : (wd == 2 ? q.z : q.w));
+                            const uint32_t e = v & 0x0f0f0f0fu;         // bytes: inputs 0, 2, 4, 6
+                            const uint32_t o = (v >> 4) & 0x0f0f0f0fu;  // bytes: inputs 1, 3, 5, 7
+                            ffma2(p[r], make_float2(w4_byte_f32<0>(e), w4_byte_f32<0>(o)), make_float2(x0.x, x0.y));
+                            ffma2(p[r], make_float2(w4_byte_f32<1>(e), w4_byte_f32<1>(o)), make_float2(x0.z, x0.w));
+                            ffma2(p[r], make_float2(w4_byte_f32<2>(e), w4_byte_f32<2>(o)), make_float2(x1.x, x1.y));
+                            ffma2(p[r], make_float2(w4_byte_f32<3>(e), w4_byte_f32<3>(o)), make_float2(x1.z, x1.w));
+                        }
+                    }
+                    const float sx = xsum[n * nch + c];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const float s = bf16lo(b.sz[r][u]), zz = bf16hi(b.sz[r][u]) + 128.f;
+                        acc[r][n] = fmaf(s, (p[r].x + p[r].y) - zz * sx, acc[r][n]);
+                    }
                 }
             }
-            const float sx = xsum[n * nch + c];
-#pragma unroll
-            for (int r = 0; r < R; ++r) acc[r][n] = fmaf(s[r], (p0[r] + p1[r]) - zz[r] * sx, acc[r][n]);
         }
     }
 }
 
 // ---------------------------------------------------------------- the kernel
-template <class P, int N, int R>
+template <class P, int R>
 __device__ __forceinline__ void stream_rows_bf16(const P &p, int t, const uint16_t *(&rows)[R]) {
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -378,15 +442,189 @@ __device__ __forceinline__ void stream_rows_bf16(const P &p, int t, const uint16
         rows[r] = p.template bf16_base<R>(t, run) + (p.template run_row<R>(t, run) + j) * (size_t)p.K;
     }
 }
+template <class P, int R>
+__device__ __forceinline__ void stream_rows_w4(const P &p, int t, W4 (&rows)[R]) {
+    const int ng = p.K / p.group;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int run = r / (R / P::NRUN), j = r % (R / P::NRUN);
+        const W4 b = p.template w4_base<R>(t, run);
+        const size_t row = p.template run_row<R>(t, run) + j;
+        rows[r] = W4{b.codes + row * (size_t)(p.K >> 1), b.scale + row * ng, b.zero + row * ng};
+    }
+}
+
+// The rest of a warp's first weight rows, and its following tasks up to `budget` bytes, requested from the L2
+// (bulk prefetch, no registers held): issued before the grid dependency resolves, so that while the predecessor
+// drains and this kernel stages its activation rows the HBM queue stays full and the first loads after the wait are
+// L2 hits.
+template <class P, int R, bool W4MODE>
+__device__ __forceinline__ void stream_l2_prefetch(const P &p, int t_first, int t1, int nwarps, int lane, int budget) {
+    const int row_bytes = W4MODE ? (p.K >> 1) : (p.K << 1);
+    int skip = min(row_bytes, (W4MODE ? W4Batch<R>::PF : kStreamPF) * 512);  // the first chunks of the first task travel in registers
+    for (int t = t_first; t < t1 && budget >= 16 * R; t += nwarps) {
+        const int per_row = min(row_bytes - skip, budget / R) & ~15;
+        if (per_row > 0) {
+            if constexpr (W4MODE) {
+                W4 rows[R];
+                stream_rows_w4<P, R>(p, t, rows);
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    if (lane == r) l2_prefetch(rows[r].codes + skip, per_row);
+            } else {
+                const uint16_t *rows[R];
+                stream_rows_bf16<P, R>(p, t, rows);
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    if (lane == r) l2_prefetch(reinterpret_cast<const uint8_t *>(rows[r]) + skip, per_row);
+            }
+        }
+        budget -= per_row * R;
+        skip = 0;
+    }
+}
+
+// Eq. 1 score from the three sums, as the score kernel computes it: a zero norm gives 0, no epsilon.
+__device__ __forceinline__ float transition_score(float ab, float aa, float bb) {
+    return (aa > 0.f && bb > 0.f) ? ab / (sqrtf(aa) * sqrtf(bb)) : 0.f;
+}
+
+// The decision for up to four rows from their scores (every thread computes the same): flags entering block l + 1.
+// CTA 0 / thread 0 publishes.  gone_in / sc are indexed by row; returns the new flags as bits.
+template <int N>
+__device__ __forceinline__ uint32_t stream_decide(const DecideArgs &dec, int n, uint32_t gone_in, const float (&sc)[N],
+                                                  const float (&tau)[N], const int (&forced)[N]) {
+    const int l = dec.l;
+    const bool eligible = (l >= 1) && (l >= dec.entry_layer) && (l < dec.L);
+    bool allpass = true;
+#pragma unroll
+    for (int b = 0; b < N; ++b)
+        if (b < n && !((gone_in >> b) & 1u) && !(eligible && sc[b] > tau[b])) allpass = false;
+    uint32_t gone = gone_in;
+#pragma unroll
+    for (int b = 0; b < N; ++b) {
+        if (b >= n || ((gone_in >> b) & 1u)) continue;
+        bool leave = eligible && (dec.exit_mode == 1 ? allpass : (sc[b] > tau[b]));
+        if (forced[b] >= 0) leave = (forced[b] == l) && (l < dec.L);
+        if (leave) gone |= 1u << b;
+    }
+    return gone;
+}
+
+template <int N>
+__device__ __forceinline__ void stream_publish(const DecideArgs &dec, int n, uint32_t gone_in, uint32_t gone,
+                                               const float (&sc)[N], const float (&tau)[N]) {
+    const int l = dec.l;
+    int32_t *exit_layer = dec.meta->exit_layer;
+    float *scores = dec.meta->scores;
+    int32_t *A = dec.lists.act_idx + (size_t)l * dec.lists.max_batch;
+    int32_t *Rv = dec.lists.riv_idx + (size_t)l * dec.lists.max_batch;
+    int na = 0, nr = 0;
+#pragma unroll
+    for (int b = 0; b < N; ++b) {
+        if (b >= n) continue;
+        const bool was = (gone_in >> b) & 1u, is = (gone >> b) & 1u;
+        dec.state_out[b] = is ? 1 : 0;
+        if (!was) {
+            if (scores) scores[(size_t)b * dec.L + (l - 1)] = sc[b];
+            if (is) exit_layer[b] = l;
+            if (dec.fail && !(sc[b] > tau[b])) dec.fail[(size_t)dec.row_slot[b] * (dec.L + 1) + l] = 1;
+        }
+        if (is) Rv[nr++] = b;
+        else A[na++] = b;
+    }
+    dec.lists.n_act[l] = na;
+    dec.lists.n_riv[l] = nr;
+    *dec.hint_act = na;
+}
+
+// ---------------------------------------------------------------- the two passes over a CTA's tasks
+template <class P, int N, int R>
+__device__ __forceinline__ void stream_pass_bf16(const P &p, const ProjIn &in, const int32_t *act_idx, int na, int xstride,
+                                                 float *xs, float *xsum, float *red, int t0, int t1, bool prestaged,
+                                                 bool fast, bool have_pre, uint4 (&pre)[R][kStreamPF]) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int K = p.K;
+    for (int i0 = 0; i0 < na; i0 += N) {
+        if (!prestaged) {
+            __syncthreads();
+            stream_load_rows<N, 8>(in, act_idx, i0, na, K, xstride, xs, xsum, red);
+        }
+        for (int t = t0 + warp; t < t1; t += nwarps) {
+            const uint16_t *rows[R];
+            stream_rows_bf16<P, R>(p, t, rows);
+            float acc[R][N];
+            float ep[4] = {0.f, 0.f, 0.f, 0.f};
+            if constexpr (N == 1 && R == 2) {
+                if (fast && lane == 0) p.epi_pre(t, 0, ep);  // travels while the dot products are computed
+            }
+            stream_dots_bf16<N, R>(rows, xs, K, xstride, have_pre && i0 == 0 && t == t0 + warp, pre, acc);
+#pragma unroll
+            for (int n2 = 0; n2 < N; ++n2) {
+                float res[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n2]);
+                if (lane == n2 && i0 + n2 < na) {
+                    if constexpr (N == 1 && R == 2) {
+                        if (fast) p.epilogue_pre(t, 0, res, ep);
+                        else p.template epilogue<R>(t, act_idx[i0 + n2], res);
+                    } else {
+                        p.template epilogue<R>(t, act_idx[i0 + n2], res);
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <class P, int N, int R, bool PRE>
+__device__ __forceinline__ void stream_pass_w4(const P &p, const ProjIn &in, const int32_t *riv_idx, int nr, int xstride,
+                                               float *xs, float *xsum, float *red, int t0, int t1, bool prestaged,
+                                               bool fast, const W4Batch<R> &pre) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int K = p.K;
+    for (int i0 = 0; i0 < nr; i0 += N) {
+        if (!prestaged) {
+            __syncthreads();
+            stream_load_rows<N, 32>(in, riv_idx, i0, nr, K, xstride, xs, xsum, red);
+        }
+        for (int t = t0 + warp; t < t1; t += nwarps) {
+            W4 rows[R];
+            stream_rows_w4<P, R>(p, t, rows);
+            float acc[R][N];
+            float ep[4] = {0.f, 0.f, 0.f, 0.f};
+            if constexpr (N == 1 && R == 2) {
+                if (fast && lane == 0) p.epi_pre(t, 0, ep);
+            }
+            stream_dots_w4<N, R>(rows, xs, xsum, K, xstride, p.group, PRE && i0 == 0 && t == t0 + warp, pre, acc);
+#pragma unroll
+            for (int n2 = 0; n2 < N; ++n2) {
+                float res[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n2]);
+                if (lane == n2 && i0 + n2 < nr) {
+                    if constexpr (N == 1 && R == 2) {
+                        if (fast) p.epilogue_pre(t, 0, res, ep);
+                        else p.template epilogue<R>(t, riv_idx[i0 + n2], res);
+                    } else {
+                        p.template epilogue<R>(t, riv_idx[i0 + n2], res);
+                    }
+                }
+            }
+        }
+    }
+}
 
 template <class P, int N, int R>
 __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjIn in, const RowLists rl, int has_river,
-                                                          int xstride, int skip_backbone, const ScoreTail tail) {
+                                                          int xstride, int skip_backbone, int pf_budget,
+                                                          const DecideArgs dec) {
     extern __shared__ __align__(16) float stream_smem[];
     const int K = p.K;
-    float *red = stream_smem;            // 32
-    float *xsum = stream_smem + 32;      // N * K/32
+    float *red = stream_smem;            // 64: block reductions (up to three sums x 16 warps)
+    float *xsum = stream_smem + 64;      // N * K/32
     float *xs = xsum + N * (K >> 5);     // N * xstride
+    __shared__ int32_t s_act[4], s_riv[4];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     pdl_launch();
 
@@ -394,23 +632,48 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     const int t0 = (int)(((long long)tasks * blockIdx.x) / gridDim.x);
     const int t1 = (int)(((long long)tasks * (blockIdx.x + 1)) / gridDim.x);
 
-    // ---- before the grid dependency: the first loads of this warp's first backbone task (weights depend on
-    // nothing).  The hint never under-counts the backbone rows, so zero means they are certainly not needed.
-    uint4 pre[R][kStreamPF];
-    bool have_pre = false;
-    if (!skip_backbone && t0 + warp < t1 && *reinterpret_cast<const volatile int32_t *>(rl.hint_act) > 0) {
-        const uint16_t *rows[R];
-        stream_rows_bf16<P, N, R>(p, t0 + warp, rows);
-        stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre);
-        have_pre = true;
+    // ---- before the grid dependency: the first loads of this warp's first task into registers and the following
+    // bytes into the L2 (weights depend on nothing).  The hint never under-counts the backbone rows: positive, the
+    // bf16 set is (almost certainly) needed; zero, every row has left the backbone and the 4-bit set is.
+    W4Batch<R> pre4;   // its q registers also carry the bf16 weights when that set is prefetched
+    int pre_kind = 0;  // 1: pre4.q holds bf16 weights, 2: pre4 holds codes with their scales / zeros
+    const int gshift = (p.group == 64) ? 1 : (p.group == 32 ? 0 : 2);
+    if (t0 + warp < t1) {
+        const int hint = *reinterpret_cast<const volatile int32_t *>(rl.hint_act);
+        if (hint > 0 && !skip_backbone) {
+            const uint16_t *rows[R];
+            stream_rows_bf16<P, R>(p, t0 + warp, rows);
+            stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre4.q);
+            pre_kind = 1;
+            if (pf_budget > 0) stream_l2_prefetch<P, R, false>(p, t0 + warp, t1, nwarps, lane, pf_budget);
+        } else if (hint == 0 && has_river) {
+            W4 rows[R];
+            stream_rows_w4<P, R>(p, t0 + warp, rows);
+            stream_issue_w4<R>(rows, K >> 5, gshift, 0, lane, pre4);
+            pre_kind = 2;
+            if (pf_budget > 0) stream_l2_prefetch<P, R, true>(p, t0 + warp, t1, nwarps, lane, pf_budget / 4);
+        }
     }
-    // A step of ONE row (the latency-critical case): which weight set the row takes follows from its exit flag, its
-    // index is 0, and its data can be requested at once - one memory round trip after the grid dependency instead of
-    // three (count -> index -> data).  The norm gain, a constant, is fetched before the wait.
-    constexpr int XF = 4;  // 128-bit pieces of the row a thread keeps in registers
+    // Per-step constants of the decision and the norm gain, fetched before the wait.
+    constexpr int XF = R == 2 ? 4 : 2;  // 128-bit pieces of a row a thread keeps in registers (one-row steps)
     const int nv = K >> 2, tid = threadIdx.x, nthr = blockDim.x;
-    const bool single = N == 1 && *rl.n_rows == 1;
-    const bool fast = single && nv <= XF * nthr;
+    const int n = *rl.n_rows;
+    const bool small = n <= N;       // the whole step in one pass: lists come from the exit flags
+    const bool fast = N == 1 && n == 1 && nv <= XF * nthr;
+    float tau[N];
+    int forced[N];
+#pragma unroll
+    for (int b = 0; b < N; ++b) { tau[b] = 0.f; forced[b] = -1; }
+    if (dec.meta && small) {
+        const float *tp = dec.meta->tau;
+        const int32_t *fp = dec.meta->forced;
+#pragma unroll
+        for (int b = 0; b < N; ++b)
+            if (b < n) {
+                tau[b] = tp[b];
+                if (fp) forced[b] = fp[b];
+            }
+    }
     uint2 gr[XF];
     if (fast && in.gain) {
 #pragma unroll
@@ -422,126 +685,156 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     pdl_wait();
     int na, nr;
     bool prestaged = false;
-    __shared__ int32_t s_row0;
     const int32_t *act_idx = rl.act_idx, *riv_idx = rl.riv_idx;
-    if (single) {
-        if (tid == 0) s_row0 = 0;
-        const bool riv = rl.exited[0] != 0;
+    if (fast) {
+        // ---- a step of ONE row (the latency-critical case): exit flag, the row and (when this launch decides) the
+        // previous block's input are requested together - one memory round trip after the grid dependency.
+        const uint8_t flag_in = dec.meta ? __ldcg(dec.state_in) : __ldcg(rl.state);
+        float4 xr[XF];
+        float bb = 0.f, ab = 0.f, aa = 0.f;
+        const float4 *src = reinterpret_cast<const float4 *>(in.src);
+#pragma unroll
+        for (int k = 0; k < XF; ++k) {
+            const int v = tid + k * nthr;
+            xr[k] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (dec.meta) {
+            const float4 *prv = reinterpret_cast<const float4 *>(dec.h_prev);
+            float4 xp[XF];
+#pragma unroll
+            for (int k = 0; k < XF; ++k) {
+                const int v = tid + k * nthr;
+                xp[k] = v < nv ? __ldcg(prv + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int k = 0; k < XF; ++k) {
+                ab += xp[k].x * xr[k].x + xp[k].y * xr[k].y + xp[k].z * xr[k].z + xp[k].w * xr[k].w;
+                aa += xp[k].x * xp[k].x + xp[k].y * xp[k].y + xp[k].z * xp[k].z + xp[k].w * xp[k].w;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < XF; ++k) bb += xr[k].x * xr[k].x + xr[k].y * xr[k].y + xr[k].z * xr[k].z + xr[k].w * xr[k].w;
+        bool riv = flag_in != 0;
+        if (in.gain || dec.meta) {
+            bb = warp_sum(bb);
+            if (dec.meta) { ab = warp_sum(ab); aa = warp_sum(aa); }
+            if (lane == 0) { red[warp] = bb; red[16 + warp] = ab; red[32 + warp] = aa; }
+            __syncthreads();
+            bb = ab = aa = 0.f;
+            for (int w = 0; w < nwarps; ++w) { bb += red[w]; ab += red[16 + w]; aa += red[32 + w]; }
+        }
+        if (dec.meta) {
+            float sc[N];
+#pragma unroll
+            for (int b = 0; b < N; ++b) sc[b] = 0.f;
+            sc[0] = transition_score(ab, aa, bb);
+            const uint32_t gone_in = flag_in ? 1u : 0u;
+            const uint32_t gone = stream_decide<N>(dec, 1, gone_in, sc, tau, forced);
+            if (blockIdx.x == 0 && tid == 0) stream_publish<N>(dec, 1, gone_in, gone, sc, tau);
+            riv = gone != 0;
+        }
+        const float scale = in.gain ? rsqrtf(bb / (float)K + in.eps) : 1.f;
+#pragma unroll
+        for (int k = 0; k < XF; ++k) {
+            const int v = tid + k * nthr;
+            if (v < nv) {
+                float4 y = xr[k];
+                if (in.gain) {
+                    y.x *= scale * bf16lo(gr[k].x); y.y *= scale * bf16hi(gr[k].x);
+                    y.z *= scale * bf16lo(gr[k].y); y.w *= scale * bf16hi(gr[k].y);
+                }
+                if (riv) *reinterpret_cast<float4 *>(xs + xs_index<32>(4 * v)) = y;
+                else *reinterpret_cast<float4 *>(xs + xs_index<8>(4 * v)) = y;
+            }
+        }
+        if (tid == 0) { s_act[0] = 0; s_riv[0] = 0; }
+        __syncthreads();
+        if (riv) stream_chunk_sums<1>(xs, xsum, K, xstride);
         na = (riv || skip_backbone) ? 0 : 1;
         nr = (riv && has_river) ? 1 : 0;
-        act_idx = riv_idx = &s_row0;
-        if (fast && na + nr == 1) {
-            float4 xr[XF];
-            float ss = 0.f;
-            const float4 *src = reinterpret_cast<const float4 *>(in.src);
+        act_idx = s_act;
+        riv_idx = s_riv;
+        prestaged = true;
+    } else if (small) {
+        // ---- up to four rows: flags (and, when this launch decides, Eq. 1 for every row: the warps split over the
+        // rows, the per-row sums meet in shared memory in a fixed order), then the lists in shared memory
+        uint32_t gone = 0u;
+        const uint8_t *st = dec.meta ? dec.state_in : rl.state;
 #pragma unroll
-            for (int k = 0; k < XF; ++k) {
-                const int v = tid + k * nthr;
-                xr[k] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-                ss += xr[k].x * xr[k].x + xr[k].y * xr[k].y + xr[k].z * xr[k].z + xr[k].w * xr[k].w;
-            }
-            float scale = 1.f;
-            if (in.gain) {
-                ss = warp_sum(ss);
-                if (lane == 0) red[warp] = ss;
-                __syncthreads();
-                ss = 0.f;
-                for (int w = 0; w < nwarps; ++w) ss += red[w];
-                scale = rsqrtf(ss / (float)K + in.eps);
-            }
+        for (int b = 0; b < N; ++b)
+            if (b < n && __ldcg(st + b)) gone |= 1u << b;
+        if (dec.meta) {
+            const int wpr = nwarps / n;  // warps per row (n <= 4 <= nwarps)
+            const int row = warp % n, member = warp / n;
+            float ab = 0.f, aa = 0.f, bb = 0.f;
+            if (member < wpr) {
+                const float4 *a4 = reinterpret_cast<const float4 *>(dec.h_prev + (size_t)row * K);
+                const float4 *b4 = reinterpret_cast<const float4 *>(in.src + (size_t)row * K);
+                const int stride = wpr * 32;
+                for (int v0 = member * 32 + lane; v0 < nv; v0 += 4 * stride) {
+                    float4 x[4], y[4];
 #pragma unroll
-            for (int k = 0; k < XF; ++k) {
-                const int v = tid + k * nthr;
-                if (v < nv) {
-                    float4 y = xr[k];
-                    if (in.gain) {
-                        y.x *= scale * bf16lo(gr[k].x); y.y *= scale * bf16hi(gr[k].x);
-                        y.z *= scale * bf16lo(gr[k].y); y.w *= scale * bf16hi(gr[k].y);
+                    for (int u = 0; u < 4; ++u) {
+                        const int v = v0 + u * stride;
+                        x[u] = v < nv ? __ldcg(a4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        y[u] = v < nv ? __ldcg(b4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
-                    if (riv) *reinterpret_cast<float4 *>(xs + xs_index<32>(4 * v)) = y;
-                    else *reinterpret_cast<float4 *>(xs + xs_index<8>(4 * v)) = y;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        ab += x[u].x * y[u].x + x[u].y * y[u].y + x[u].z * y[u].z + x[u].w * y[u].w;
+                        aa += x[u].x * x[u].x + x[u].y * x[u].y + x[u].z * x[u].z + x[u].w * x[u].w;
+                        bb += y[u].x * y[u].x + y[u].y * y[u].y + y[u].z * y[u].z + y[u].w * y[u].w;
+                    }
                 }
             }
+            ab = warp_sum(ab); aa = warp_sum(aa); bb = warp_sum(bb);
+            if (lane == 0) { red[warp] = ab; red[16 + warp] = aa; red[32 + warp] = bb; }
             __syncthreads();
-            if (riv) stream_chunk_sums<1>(xs, xsum, K, xstride);
-            prestaged = true;
-        } else {
-            __syncthreads();  // s_row0
+            float sc[N];
+#pragma unroll
+            for (int b = 0; b < N; ++b) {
+                sc[b] = 0.f;
+                if (b >= n) continue;
+                float sab = 0.f, saa = 0.f, sbb = 0.f;
+                for (int m = 0; m < wpr; ++m) { sab += red[m * n + b]; saa += red[16 + m * n + b]; sbb += red[32 + m * n + b]; }
+                sc[b] = transition_score(sab, saa, sbb);
+            }
+            const uint32_t gone_in = gone;
+            gone = stream_decide<N>(dec, n, gone_in, sc, tau, forced);
+            if (blockIdx.x == 0 && tid == 0) stream_publish<N>(dec, n, gone_in, gone, sc, tau);
         }
+        na = 0; nr = 0;
+        if (tid == 0) {
+            int a = 0, r = 0;
+#pragma unroll
+            for (int b = 0; b < N; ++b)
+                if (b < n) {
+                    if ((gone >> b) & 1u) s_riv[r++] = b;
+                    else s_act[a++] = b;
+                }
+        }
+        na = n - __popc(gone);
+        nr = has_river ? __popc(gone) : 0;
+        if (skip_backbone) na = 0;
+        act_idx = s_act;
+        riv_idx = s_riv;
+        __syncthreads();
     } else {
         // skip_backbone: the backbone rows of this step are served by the tensor-core kernel
         na = skip_backbone ? 0 : *rl.n_act;
         nr = has_river ? *rl.n_riv : 0;
     }
 
-    for (int i0 = 0; i0 < na; i0 += N) {
-        if (!prestaged) {
-            __syncthreads();
-            stream_load_rows<N, 8>(in, act_idx, i0, na, K, xstride, xs, xsum, red);
-        }
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            const uint16_t *rows[R];
-            stream_rows_bf16<P, N, R>(p, t, rows);
-            float acc[R][N];
-            float ep[4] = {0.f, 0.f, 0.f, 0.f};
-            if constexpr (N == 1 && R == 2) {
-                if (single && lane == 0) p.epi_pre(t, 0, ep);  // travels while the dot products are computed
-            }
-            stream_dots_bf16<N, R>(rows, xs, K, xstride, have_pre && i0 == 0 && t == t0 + warp, pre, acc);
-#pragma unroll
-            for (int n = 0; n < N; ++n) {
-                float res[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n]);
-                if (lane == n && i0 + n < na) {
-                    if constexpr (N == 1 && R == 2) {
-                        if (single) p.epilogue_pre(t, 0, res, ep);
-                        else p.template epilogue<R>(t, act_idx[i0 + n], res);
-                    } else {
-                        p.template epilogue<R>(t, single ? 0 : act_idx[i0 + n], res);
-                    }
-                }
-            }
-        }
+    // hint == 0 promised that no row is left in the backbone: then only the 4-bit pass runs, with the prefetched
+    // registers; otherwise the bf16 pass (which may hold prefetched registers) and the 4-bit pass without them, so
+    // that neither pass keeps the other's prefetch registers alive
+    if (pre_kind == 2) {
+        if (na == 0)
+            stream_pass_w4<P, N, R, true>(p, in, riv_idx, nr, xstride, xs, xsum, red, t0, t1, prestaged, fast, pre4);
+    } else {
+        stream_pass_bf16<P, N, R>(p, in, act_idx, na, xstride, xs, xsum, red, t0, t1, prestaged, fast, pre_kind == 1, pre4.q);
+        stream_pass_w4<P, N, R, false>(p, in, riv_idx, nr, xstride, xs, xsum, red, t0, t1, prestaged, fast, pre4);
     }
-    for (int i0 = 0; i0 < nr; i0 += N) {
-        if (!prestaged) {
-            __syncthreads();
-            stream_load_rows<N, 32>(in, riv_idx, i0, nr, K, xstride, xs, xsum, red);
-        }
-        const int ng = K / p.group;
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            W4 rows[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int run = r / (R / P::NRUN), j = r % (R / P::NRUN);
-                const W4 b = p.template w4_base<R>(t, run);
-                const size_t row = p.template run_row<R>(t, run) + j;
-                rows[r] = W4{b.codes + row * (K >> 1), b.scale + row * ng, b.zero + row * ng};
-            }
-            float acc[R][N];
-            float ep[4] = {0.f, 0.f, 0.f, 0.f};
-            if constexpr (N == 1 && R == 2) {
-                if (single && lane == 0) p.epi_pre(t, 0, ep);
-            }
-            stream_dots_w4<N, R>(rows, xs, xsum, K, xstride, p.group, acc);
-#pragma unroll
-            for (int n = 0; n < N; ++n) {
-                float res[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) res[r] = warp_sum(acc[r][n]);
-                if (lane == n && i0 + n < nr) {
-                    if constexpr (N == 1 && R == 2) {
-                        if (single) p.epilogue_pre(t, 0, res, ep);
-                        else p.template epilogue<R>(t, riv_idx[i0 + n], res);
-                    } else {
-                        p.template epilogue<R>(t, single ? 0 : riv_idx[i0 + n], res);
-                    }
-                }
-            }
-        }
-    }
-    if (tail.meta) score_tail(tail);  // the kernel that ends a block also scores it (small steps)
 }
 
 // ---------------------------------------------------------------- a8: final norm + LM head + argmax partials
@@ -559,7 +852,7 @@ struct HeadArgs {
 };
 
 template <int N, int R>
-__global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstride) {
+__global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstride, int pf_budget) {
     extern __shared__ __align__(16) float stream_smem[];
     float *red = stream_smem;
     float *xs = stream_smem + 32;
@@ -579,6 +872,15 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstr
         for (int r = 0; r < R; ++r) rows[r] = a.w + ((size_t)(t0 + warp) * R + r) * K;
         stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre);
         have_pre = true;
+        // the following bytes of this warp's rows into the L2, so that HBM keeps streaming while the last block drains
+        int budget = pf_budget, skip = min(2 * K, kStreamPF * 512);
+        for (int t = t0 + warp; t < t1 && budget >= 16 * R; t += nwarps) {
+            const int per_row = min(2 * K - skip, budget / R) & ~15;
+            if (per_row > 0 && lane < R)
+                l2_prefetch(reinterpret_cast<const uint8_t *>(a.w + ((size_t)t * R + lane) * K) + skip, per_row);
+            budget -= per_row * R;
+            skip = 0;
+        }
     }
     pdl_wait();
     const int cnt = a.meta->n_head_rows;
@@ -625,7 +927,7 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstr
     }
 }
 
-__global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts) {
+static __global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts) {
     pdl_launch();
     pdl_wait();
     const int i = blockIdx.x;
@@ -651,12 +953,12 @@ __global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val,
     if (threadIdx.x == 0) {
         for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
             if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
-        next_tok[i] = bi;
+        next_tok[i] = bi == 0x7fffffff ? 0 : bi;  // a row without any comparable logit (all NaN) yields token 0
     }
 }
 
 inline size_t stream_smem_bytes(int N, int K) {
-    return sizeof(float) * (32 + (size_t)N * (K >> 5) + (size_t)N * xs_stride(K, 32));
+    return sizeof(float) * (64 + (size_t)N * (K >> 5) + (size_t)N * xs_stride(K, 32));
 }
 
 }  // namespace river

@@ -1,0 +1,81 @@
+// Launches of the tensor-core projection kernel for backbone rows (5 <= rows <= 256) and its operand kernel.
+#include <algorithm>
+
+#include "launch_tc.h"
+#include "tensor_maps.h"
+
+namespace river {
+
+const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
+    for (auto &b : c->tc_bmaps)
+        if (b.K == K && b.np == np) return &b;
+    river_ctx::BMap b{K, np, {}, {}};
+    if (!make_map_bf16(&b.hi, c->tc_xhi, K, np, np) || !make_map_bf16(&b.lo, c->tc_xlo, K, np, np)) return nullptr;
+    c->tc_bmaps.push_back(b);
+    return &c->tc_bmaps.back();
+}
+
+// K-splits per tile: fill whole waves of the CTA slots, keep at least four 64-wide k-blocks per split; no split at
+// all when there is a tile for every SM.  The kernel is memory-bound, so what matters is that all CTAs are resident
+// together and every SM slot streams.
+int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots, int min_kb) {
+    int best = 1;
+    double best_eff = 0.0;
+    if (tiles >= c->num_sms) return 1;  // every SM has a tile of its own: splitting only adds reductions
+    for (int s = 1; s <= 8; ++s) {  // a cluster holds at most 8 CTAs
+        if (s > 1 && kb_total / s < min_kb) break;
+        const int ctas = tiles * s, waves = (ctas + slots - 1) / slots;
+        const double eff = (double)ctas / ((double)waves * slots);
+        if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+    }
+    return best;
+}
+
+template <class Epi>
+cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
+                      int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
+                      const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint) {
+    const int np = (n + 15) / 16 * 16;
+    const river_ctx::BMap *bm = tc_bmap(c, K, np);
+    if (!bm) return cudaErrorInvalidValue;
+    cudaError_t e = launch_k(tc_prep_kernel, dim3(np, (K + kPrepChunk - 1) / kPrepChunk), dim3(256), 0, c->stream, true, in, rows, cnt, K,
+                             c->tc_xhi, c->tc_xlo);
+    if (e != cudaSuccess) return e;
+    ++c->st.launches_last_step;
+    TcArgs a{};
+    a.K = K; a.n_pad = np;
+    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
+    // CTAs per SM: two with three stages each, or three with two when that puts more CTAs of one wave to work (while
+    // one CTA drains its accumulator and takes part in the cluster reduction the others keep the weight stream going);
+    // one with deep stages when the operand tiles are too large for that.
+    const size_t sm_smem = 228 * 1024, fixed = 1024 + 1024 + 256;  // per CTA: system reserve, alignment slack, barriers
+    auto stages_at = [&](int occ) {
+        const size_t room = std::min<size_t>(sm_smem / occ, 227 * 1024);
+        return room < fixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : 3, (room - fixed) / stage);
+    };
+    int occ = stages_at(2) ? 2 : 1;
+    a.splits = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * occ);
+    if (occ == 2 && stages_at(3) && allow_split) {
+        const int s3 = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * 3);
+        if (tiles * s3 > tiles * a.splits && tiles * s3 <= c->num_sms * 3) { occ = 3; a.splits = s3; }
+    }
+    a.n_stages = stages_at(occ);
+    // the finished tile lives in the pipeline memory
+    if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage) return cudaErrorInvalidValue;
+    if (!allow_split) a.splits = 1;
+    a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
+    a.rows = rows; a.cnt = cnt; a.dev_err = c->dev_err;
+    a.hint = hint ? hint : cnt;
+    const size_t smem = tc_smem_bytes(np, a.n_stages);
+    e = ensure_smem(c, tc_gemm_kernel<Epi>, smem);
+    if (e != cudaSuccess) return e;
+    return launch_kc(tc_gemm_kernel<Epi>, dim3(tiles * a.splits), dim3(kTcThreads), smem, c->stream, true, a.splits, a0,
+                     a1, a2, bm->hi, bm->lo, a, epi);
+}
+#define RIVER_TC_INST(E) \
+    template cudaError_t launch_tc<E>(river_ctx *, const ProjIn &, const CUtensorMap &, const CUtensorMap &, const CUtensorMap &, \
+                                      int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *);
+RIVER_TC_INST(TcQkvEpi) RIVER_TC_INST(TcResidEpi) RIVER_TC_INST(TcGateUpEpi) RIVER_TC_INST(TcHeadEpi)
+#undef RIVER_TC_INST
+
+}  // namespace river

@@ -1,0 +1,49 @@
+// Launches of the dequantising tensor-core kernel for exit-layer rows (5 <= rows <= 256) and its operand kernel.
+#include <algorithm>
+
+#include "launch_tc.h"
+#include "gemm_tc_w4.cuh"
+
+namespace river {
+
+template <class Epi>
+cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
+                         int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
+                         const int32_t *cnt, const int32_t *hint, const Epi &epi) {
+    const int np = (n + 15) / 16 * 16;
+    const river_ctx::BMap *bm = tc_bmap(c, K, np);
+    if (!bm) return cudaErrorInvalidValue;
+    cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np, (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk)), dim3(256), 0, c->stream, true, in, rows,
+                             cnt, K,
+                             reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(c->tc_xlo));
+    if (e != cudaSuccess) return e;
+    ++c->st.launches_last_step;
+    TcW4Args a{};
+    a.K = K; a.n_pad = np;
+    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
+    const size_t raw = (size_t)kW4RawBufs * kW4RawBytes;
+    // two CTAs per SM (16 dequantisation warps) when two operand stages fit in half of the shared memory
+    const bool two = 2 * stage + raw + 4096 <= 110 * 1024;
+    a.n_stages = two ? (int)std::min<size_t>(4, (110 * 1024 - raw - 4096) / stage)
+                     : (int)std::max<size_t>(2, std::min<size_t>(6, (214 * 1024 - raw) / stage));
+    // in raw tiles of four k-blocks: at least four per split, two when K is so short that four would allow only two
+    // splits (measured on the 1B shape, K = 2048: 2 -> 4 splits 35 -> 31 us per layer for QKV, 33 -> 27 us for O)
+    const int raw_tiles = K / (kTcBK * kW4Super);
+    a.splits = tc_pick_splits(c, tiles, raw_tiles, c->num_sms * (two ? 2 : 1), raw_tiles <= 8 ? 2 : 4);
+    if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage + raw) return cudaErrorInvalidValue;
+    a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
+    for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
+    a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
+    const size_t smem = tc_w4_smem_bytes(np, a.n_stages);
+    e = ensure_smem(c, tc_gemm_w4_kernel<Epi>, smem);
+    if (e != cudaSuccess) return e;
+    return launch_kc(tc_gemm_w4_kernel<Epi>, dim3(tiles * a.splits), dim3(kW4Threads), smem, c->stream, true, a.splits,
+                     *m[0], *m[1], *m[2], bm->hi, bm->lo, a, epi);
+}
+#define RIVER_TCW4_INST(E) \
+    template cudaError_t launch_tc_w4<E>(river_ctx *, const ProjIn &, const CUtensorMap *const (&)[3], const river_w4 *const (&)[3], \
+                                         int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &);
+RIVER_TCW4_INST(TcQkvEpi) RIVER_TCW4_INST(TcResidEpi) RIVER_TCW4_INST(TcGateUpEpi)
+#undef RIVER_TCW4_INST
+
+}  // namespace river

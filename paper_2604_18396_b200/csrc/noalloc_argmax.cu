@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(256) argmax_noalloc_kernel(const float *logits
     if (threadIdx.x == 0) {
         for (int w = 1; w < 8; ++w)
             if (better(sv[w], si[w], bv, bi)) { bv = sv[w]; bi = si[w]; }
-        next_tok[row] = bi;
+        next_tok[row] = bi == 0x7fffffff ? 0 : bi;  // a row without any comparable value (all NaN) yields token 0
         s->arrived[row] = 0;
     }
 }
@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(256) argmax_noalloc_kernel(const float *logits
 }  // namespace
 
 extern "C" int river_argmax_noalloc(const float *logits, int n_rows, int V, int32_t *next_tok, void *cuda_stream) {
-    if (!logits || !next_tok || n_rows <= 0 || V <= 0) return RIVER_E_BADARG;
+    if (!logits || !next_tok || n_rows <= 0 || V <= 0 || V > 0x7fffffff - kParts) return RIVER_E_BADARG;
     if (n_rows > kMaxRows) return RIVER_E_NOMEM;  // beyond the fixed scratch: split the batch
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RIVER_E_DEVICE;
@@ -108,7 +108,8 @@ extern "C" int river_argmax_noalloc(const float *logits, int n_rows, int V, int3
     }
     Scratch *s = g_scratch_addr[dev];
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    // the array keeps whatever the last call left: the counters have to start at zero
+    // the array keeps whatever the last call left and the counters have to start at zero: this memset is what the
+    // call relies on (the kernel also returns them to zero, so an aborted earlier launch cannot poison a later one)
     if (cudaMemsetAsync(s->arrived, 0, sizeof(unsigned) * n_rows, st) != cudaSuccess) return RIVER_E_DEVICE;
     argmax_noalloc_kernel<<<dim3(kParts, n_rows), 256, 0, st>>>(logits, V, next_tok, s);
     return cudaGetLastError() == cudaSuccess ? RIVER_OK : RIVER_E_DEVICE;

@@ -9,15 +9,13 @@
 #include <string>
 #include <vector>
 
-#include "../../include/river.h"
+#include "river_ctx.h"
+#include "launch.h"
+#include "launch_tc.h"
+#include "tensor_maps.h"
 #include "river_kernels.cuh"
 #include "attn_decode.cuh"
-#include "gemv_stream.cuh"
-#include <cstdio>
-#include <cstdlib>
-#include "gemm_tc.cuh"
-#include "decode_chain.cuh"
-#include "gemm_tc_w4.cuh"
+#include "attn_small.cuh"
 
 using namespace river;
 
@@ -25,11 +23,8 @@ namespace {
 
 thread_local std::string g_init_error;
 
-constexpr int kStaging = 4;        // pinned metadata buffers in flight
-enum KernelClass { K_BEGIN, K_COMPACT, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, K_CHAIN, kNumClasses };
-const char *const kClassNames[kNumClasses] = {"step_begin", "compact", "qkv_rope_kv", "attn_decode", "o_proj_resid",
-                                              "gateup_swiglu", "down_resid", "exit_score", "lm_head", "argmax_final",
-                                              "decode_chain"};
+const char *const kClassNames[kNumClasses] = {"step_begin", "qkv_rope_kv", "attn_decode", "o_proj_resid", "gateup_swiglu",
+                                              "down_resid", "exit_score", "lm_head", "argmax_final", "prefill_attn"};
 
 struct Carver {
     char *base;
@@ -44,79 +39,6 @@ struct Carver {
 };
 
 }  // namespace
-
-struct river_ctx {
-    river_config cfg;
-    std::vector<river_layer_weights> layers;
-    const uint16_t *embed, *lm_head, *final_norm;
-    cudaStream_t stream;
-    int num_sms = 0;
-    __nv_bfloat16 *pool = nullptr;
-
-    // workspace
-    float *h[3], *qbuf, *obuf, *act, *part_val, *tau_i, *logits_i, *scores_i;
-    float2 *rope_cs, *part_ml;
-    float *part_o;
-    CUtensorMap kv_tmap;
-    int attn_splits_now = 1;
-    bool attn_small_now = false;  // this step's attention runs on the small-step kernel (short contexts, 1-4 rows)
-    unsigned *attn_tickets, *tickets;  // [max_batch*Hkv], [4]
-    // tensor-core path: operand buffers, split-K partials, tickets, tensor maps of every weight matrix
-    __nv_bfloat16 *tc_xhi = nullptr, *tc_xlo = nullptr;
-    int tc_max_pad = 0, tc_kmax = 0;
-    bool tc_ok = false;
-    struct LayerMaps { CUtensorMap q, k, v, o, g, u, d; };
-    std::vector<LayerMaps> tc_maps;
-    std::vector<LayerMaps> w4_maps;  // code matrices of the exit layers (u8 [rows][K/2], 128-byte boxes)
-    bool w4tc_ok = false;
-    CUtensorMap tc_map_head;
-    struct BMap { int K, np; CUtensorMap hi, lo; };
-    std::vector<BMap> tc_bmaps;
-    int32_t *hint_act;
-    // persistent layer-chain kernel for steps of at most four rows
-    LayerDev *layers_dev = nullptr;
-    unsigned long long *chain_stamps = nullptr;
-    bool chain_ok = false;
-    bool rows_distinct = true;  // every row of the current step is a different sequence (decode), not a prefill chunk
-    int chain_grid = 0, chain_pf_bytes = 4 * 1024;
-    struct GraphEntry { int n; bool small_attn; int attn_splits; cudaGraphExec_t exec; int launches; };
-    std::vector<GraphEntry> graphs;
-    double *inv_freq;
-    int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
-    int32_t *meta_dev;  // [kMetaHdr + 7*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows, row_page
-    uint8_t *exited, *pass;
-    int *dev_err;
-    size_t ws_bytes = 0;
-
-    // host state
-    std::vector<int32_t> page_tbl, seq_len, free_pages;
-    int32_t *meta_host[kStaging] = {nullptr, nullptr, nullptr, nullptr};
-    cudaEvent_t meta_ev[kStaging];
-    int meta_next = 0;
-    void *pin_io = nullptr;  // pinned staging for the *_host entry point
-    size_t pin_io_bytes = 0;
-    std::vector<int32_t> last_pos;  // positions of the rows of the last decode step
-    int head_grid = 0;
-
-    river_stats_t st{};
-    std::string err;
-
-    // optional per-kernel timing (river_profile): events around every launch of a step
-    bool profiling = false;
-    std::vector<cudaEvent_t> prof_ev;
-    struct ProfRec { int cls; double bytes_act, bytes_riv; int list_idx; };
-    std::vector<ProfRec> prof_rec;
-    double prof_ms[kNumClasses] = {0}, prof_bytes[kNumClasses] = {0};
-    int64_t prof_launches[kNumClasses] = {0};
-
-    int meta_ints() const { return kMetaHdr + 7 * cfg.max_batch; }
-    StepMeta *meta() const { return reinterpret_cast<StepMeta *>(meta_dev); }
-    int32_t *row_slot() const { return meta_dev + kMetaHdr; }
-    int32_t *row_pos() const { return meta_dev + kMetaHdr + cfg.max_batch; }
-    int32_t *upd() const { return meta_dev + kMetaHdr + 2 * cfg.max_batch; }
-    int32_t *head_rows() const { return meta_dev + kMetaHdr + 5 * cfg.max_batch; }
-    int32_t *row_page() const { return meta_dev + kMetaHdr + 6 * cfg.max_batch; }  // page of each row's new position
-};
 
 namespace {
 
@@ -171,83 +93,28 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     int32_t *na = cv.take<int32_t>(L + 1), *nr = cv.take<int32_t>(L + 1);
     int32_t *pt = cv.take<int32_t>((size_t)c->max_seqs * c->max_pages_per_seq);
     int32_t *tk = cv.take<int32_t>(B), *fo = cv.take<int32_t>(B), *ex = cv.take<int32_t>(B), *nx = cv.take<int32_t>(B);
-    int32_t *md = cv.take<int32_t>(kMetaHdr + 7 * B);
+    int32_t *md = cv.take<int32_t>(kMetaHdr + 8 * B);
+    int32_t *pff = cv.take<int32_t>((size_t)c->max_seqs * (L + 1));
     float *po = cv.take<float>((B + 600) * (size_t)c->Hq * c->dh);
     float2 *pml = cv.take<float2>((B + 600) * (size_t)c->Hq);
-    uint8_t *exd = cv.take<uint8_t>(B), *ps = cv.take<uint8_t>(B);
+    const size_t sstride = (B + 15) / 16 * 16;
+    uint8_t *exd = cv.take<uint8_t>((L + 1) * sstride), *ps = cv.take<uint8_t>(B);
     int *de = cv.take<int>(1);
     unsigned *atk = cv.take<unsigned>(B * (size_t)c->Hkv), *tk4 = cv.take<unsigned>(4);
     int32_t *hint = md ? md + 5 : nullptr;  // StepMeta::hint_act
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
-    LayerDev *ld = cv.take<LayerDev>(L);
-    unsigned long long *stp = cv.take<unsigned long long>(2 + 6 * L + 48);
 
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
         x->part_val = pv; x->part_idx = pi; x->tau_i = tau; x->logits_i = lg; x->scores_i = sc; x->rope_cs = cs;
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
-        x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->exited = exd;
+        x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->state = exd; x->state_stride = (int)sstride; x->prefill_fail = pff;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
-        x->layers_dev = ld; x->chain_stamps = stp;
         x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
-}
-
-// Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the
-// stream is still running and orders itself with griddepcontrol.wait.  Every kernel launched this way calls
-// griddepcontrol.wait before it touches anything a predecessor writes.
-template <class... KArgs, class... Args>
-cudaError_t launch_kc(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
-                      int cluster_x, Args &&...args) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute at[2];
-    int na = 0;
-    if (pdl) {
-        at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[na].val.programmaticStreamSerializationAllowed = 1;
-        ++na;
-    }
-    if (cluster_x > 1) {  // consecutive CTAs along x form a thread-block cluster
-        at[na].id = cudaLaunchAttributeClusterDimension;
-        at[na].val.clusterDim.x = cluster_x;
-        at[na].val.clusterDim.y = 1;
-        at[na].val.clusterDim.z = 1;
-        ++na;
-    }
-    cfg.attrs = at;
-    cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
-}
-template <class... KArgs, class... Args>
-cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
-                     Args &&...args) {
-    return launch_kc(kern, grid, block, smem, st, pdl, 1, std::forward<Args>(args)...);
-}
-
-KvAddr kv_addr(const river_ctx *c, int layer0) {
-    KvAddr k;
-    k.pool = c->pool;
-    k.page_tbl = c->page_tbl_dev;
-    k.row_slot = c->row_slot();
-    k.row_pos = c->row_pos();
-    k.row_page = c->row_page();
-    k.n_pages = c->cfg.n_pages;
-    k.max_pages_per_seq = c->cfg.max_pages_per_seq;
-    k.Hkv = c->cfg.Hkv;
-    k.dh = c->cfg.dh;
-    k.layer0 = layer0;
-    return k;
-}
-
-W4 w4(const river_w4 &r) {
-    return W4{(const uint8_t *)r.codes, (const uint16_t *)r.scale, (const uint16_t *)r.zero};
 }
 
 // KV split geometry of this step.  A (row, kv head, split) item costs its positions plus a fixed start-up overhead
@@ -293,15 +160,15 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     mh[3] = chunk;
     mh[4] = S;
     mh[5] = n;  // hint_act: every row starts in the backbone
-    // the persistent chain kernel: one CTA per (row, kv head, split), chunks in whole pages
-    int Sc = std::max(1, std::min(64, c->num_sms / (n * g.Hkv)));
+    // the small-step kernel: one CTA per (row, kv head, split), chunks in whole pages
+    const int Sc = small_attn_splits(c->num_sms, n, g.Hkv);
     int cchunk = (max_pos + 1 + Sc - 1) / Sc;
     cchunk = std::max(kPage, (cchunk + kPage - 1) / kPage * kPage);
     mh[6] = cchunk;  // StepMeta::pad[0]
     mh[7] = Sc;      // StepMeta::pad[1]
     // the small-step kernel walks a split in batches of 4 positions per warp without a load pipeline: worth it up to
     // two batches per warp, beyond that the TMA-fed kernel's staging pays
-    c->attn_small_now = n <= 4 && cchunk <= 2 * 4 * kChainWarps && !(g.flags & (RIVER_F_SIMPLE_ATTN | RIVER_F_TMA_ATTN));
+    c->attn_small_now = n <= 4 && cchunk <= 2 * 4 * kSmallAttnWarps && !(g.flags & RIVER_F_TMA_ATTN);
     c->attn_splits_now = S;
 }
 
@@ -312,166 +179,7 @@ void set_io_meta(int32_t *mh, const int32_t *tok, const float *tau, const int32_
     m->exit_layer = exit_layer; m->scores = scores;
 }
 
-template <int DH, int GQ>
-cudaError_t launch_attn(river_ctx *c, int n, int layer0, bool pdl) {
-    const river_config &g = c->cfg;
-    if (g.flags & RIVER_F_SIMPLE_ATTN) {
-        attn_decode_kernel<DH, GQ><<<dim3(g.Hkv, n), 128, 0, c->stream>>>(
-            c->meta(), c->qbuf, kv_addr(c, layer0), 1.0f / std::sqrt((float)DH), g.Hq, c->obuf);
-        return cudaGetLastError();
-    }
-    AttnArgs a{};
-    a.meta = c->meta(); a.q = c->qbuf; a.page_tbl = c->page_tbl_dev; a.row_slot = c->row_slot(); a.row_pos = c->row_pos();
-    a.n_pages = g.n_pages; a.max_pages_per_seq = g.max_pages_per_seq; a.Hkv = g.Hkv; a.Hq = g.Hq; a.layer0 = layer0;
-    a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.tickets = c->attn_tickets; a.out = c->obuf; a.dev_err = c->dev_err;
-    const size_t smem = attn_smem_bytes(DH, GQ);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(attn_split_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_set = true;
-    }
-    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(kAttnThreads), smem, c->stream,
-                    pdl, c->kv_tmap, a);
-}
-
-// Steps of 1-4 rows: the split-KV kernel that fetches the cached positions before the grid dependency resolves.
-template <int DH, int GQ>
-cudaError_t launch_attn_small(river_ctx *c, int n, int layer0, int early) {
-    const river_config &g = c->cfg;
-    ChainArgs a{};
-    a.meta = c->meta();
-    a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh;
-    a.qscale = 1.4426950408889634f / std::sqrt((float)g.dh);
-    a.qbuf = c->qbuf; a.obuf = c->obuf; a.kv = kv_addr(c, layer0);
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.attn_tickets = c->attn_tickets; a.dev_err = c->dev_err;
-    const int S = std::max(1, std::min(64, c->num_sms / (n * g.Hkv)));  // as set_attn_meta puts into the metadata
-    const size_t smem = sizeof(float) * (size_t)kChainWarps * GQ * (DH + 2);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(attn_small_kernel<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_set = true;
-    }
-    return launch_k(attn_small_kernel<DH, GQ>, dim3(n * g.Hkv * S), dim3(kChainThreads), smem, c->stream, true, a, layer0, early);
-}
-
-cudaError_t launch_attention(river_ctx *c, int n, int layer0, bool pdl) {
-    const int gq = c->cfg.Hq / c->cfg.Hkv;
-    if (c->attn_small_now) {
-#define ATTS(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn_small<DH_, GQ_>(c, n, layer0, c->rows_distinct ? 1 : 0);
-        ATTS(64, 1) ATTS(64, 2) ATTS(64, 4) ATTS(64, 8) ATTS(128, 1) ATTS(128, 2) ATTS(128, 4) ATTS(128, 8)
-#undef ATTS
-    }
-#define ATT(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn<DH_, GQ_>(c, n, layer0, pdl);
-    ATT(64, 1) ATT(64, 2) ATT(64, 4) ATT(64, 8) ATT(128, 1) ATT(128, 2) ATT(128, 4) ATT(128, 8)
-#undef ATT
-    return cudaErrorInvalidValue;
-}
-
-// ---- streaming projection launch
-// Launch geometry: warps per CTA and CTAs per SM such that every warp gets the same number of tasks (a task is R
-// weight rows) and at least 16 warps per SM have loads in flight; searched once per (kernel, task count).
-struct StreamGeom { int threads, grid; };
-
-template <class Kern>
-StreamGeom pick_geometry(river_ctx *c, Kern kern, int tasks, size_t smem) {
-    StreamGeom best{256, c->num_sms};
-    double best_cost = 1e30;
-    int best_w = 0;
-    for (int w = 4; w <= 16; ++w) {
-        int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, w * 32, smem) != cudaSuccess || occ < 1) continue;
-        occ = std::min(occ, 64 / w);
-        for (int o = 1; o <= occ; ++o) {
-            const int ctas = c->num_sms * o;
-            const int per_cta = (tasks + ctas - 1) / ctas;
-            const int rounds = (per_cta + w - 1) / w;
-            const int W = w * o;
-            const double cost = rounds * (W < 16 ? 16.0 / W : 1.0) * (1.0 + 0.002 * o);  // few large CTAs share x loads
-            if (cost < best_cost - 1e-9 || (std::fabs(cost - best_cost) < 1e-9 && W > best_w)) {
-                best_cost = cost; best_w = W; best = StreamGeom{w * 32, ctas};
-            }
-        }
-    }
-    return best;
-}
-
-template <class P, int N, int R>
-cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks,
-                            int has_river, bool pdl, int skip_backbone, const ScoreTail &tail) {
-    const size_t smem = stream_smem_bytes(N, K);
-    // one kernel instantiation serves several projections (O and down): cache the geometry per (tasks, K)
-    struct Entry { int tasks, K; StreamGeom g; };
-    static std::vector<Entry> cache;
-    static size_t attr_smem = 0;
-    const StreamGeom *geom = nullptr;
-    for (auto &e : cache)
-        if (e.tasks == tasks && e.K == K) geom = &e.g;
-    if (!geom) {
-        if (smem > attr_smem) attr_smem = smem;
-        cudaFuncSetAttribute(stream_proj_kernel<P, N, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attr_smem);
-        cache.push_back({tasks, K, pick_geometry(c, stream_proj_kernel<P, N, R>, tasks, smem)});
-        geom = &cache.back().g;
-    }
-    return launch_k(stream_proj_kernel<P, N, R>, dim3(geom->grid), dim3(geom->threads), smem, c->stream, pdl, p, in, rl,
-                    has_river, xs_stride(K, 32), skip_backbone, tail);
-}
-
-int stream_rows_per_task(int K) { return K >= 4096 ? 2 : 4; }
-
-template <class P>
-cudaError_t launch_stream(river_ctx *c, const P &p, const ProjIn &in, const RowLists &rl, int K, int tasks_r2, int n,
-                          int has_river, bool pdl, int skip_backbone = 0, const ScoreTail &tail = ScoreTail{}) {
-    int n_sel = 1;
-    while (n_sel < n && n_sel < 4 && stream_smem_bytes(n_sel * 2, K) <= 200 * 1024) n_sel *= 2;
-    const int r = stream_rows_per_task(K);
-    const int tasks = tasks_r2 * 2 / r;
-#define STREAM_CASE(N_, R_) if (n_sel == N_ && r == R_) return launch_stream_t<P, N_, R_>(c, p, in, rl, K, tasks, has_river, pdl, skip_backbone, tail);
-    STREAM_CASE(1, 2) STREAM_CASE(2, 2) STREAM_CASE(4, 2)
-    STREAM_CASE(1, 4) STREAM_CASE(2, 4) STREAM_CASE(4, 4)
-#undef STREAM_CASE
-    return cudaErrorInvalidValue;
-}
-
-typedef CUresult (*TmapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-TmapEncodeFn tmap_encoder() {
-    static TmapEncodeFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess) fn = (TmapEncodeFn)p;
-    }
-    return fn;
-}
-// bf16 row-major matrix [rows][inner] -> tiled map with a (box_rows x 64) box and the 128-byte swizzle
-bool make_map_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
-    TmapEncodeFn fn = tmap_encoder();
-    if (!fn) return false;
-    const cuuint64_t gdim[2] = {inner, rows};
-    const cuuint64_t gstride[1] = {inner * 2};
-    const cuuint32_t box[2] = {64, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// u8 code matrix [rows][inner_bytes] -> tiled map with a (box_rows x 128 byte) box and the 128-byte swizzle
-bool make_map_codes(CUtensorMap *m, const void *base, uint64_t inner_bytes, uint64_t rows, uint32_t box_rows) {
-    TmapEncodeFn fn = tmap_encoder();
-    if (!fn) return false;
-    const cuuint64_t gdim[2] = {inner_bytes, rows};
-    const cuuint64_t gstride[1] = {inner_bytes};
-    const cuuint32_t box[2] = {128, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// ---- tensor-core projection launch
+// ---- tensor maps of the weights for the tensor-core projections
 // The shapes the tensor-core path takes: every output dimension in whole 128-feature tiles.
 bool tc_shape_ok(const river_config &g) {
     return g.d % 128 == 0 && (g.Hq * g.dh) % 128 == 0 && (g.Hkv * g.dh) % 128 == 0 && g.F % 64 == 0 && g.V % 128 == 0 &&
@@ -510,121 +218,6 @@ bool make_w4_maps(river_ctx *c) {
             return false;
     }
     return true;
-}
-const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
-    for (auto &b : c->tc_bmaps)
-        if (b.K == K && b.np == np) return &b;
-    river_ctx::BMap b{K, np, {}, {}};
-    if (!make_map_bf16(&b.hi, c->tc_xhi, K, np, np) || !make_map_bf16(&b.lo, c->tc_xlo, K, np, np)) return nullptr;
-    c->tc_bmaps.push_back(b);
-    return &c->tc_bmaps.back();
-}
-// K-splits per tile: fill whole waves of the CTA slots, keep at least four 64-wide k-blocks per split; no split at
-// all when there is a tile for every SM.  The kernel is memory-bound, so what matters is that all CTAs are resident
-// together and every SM slot streams.
-int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots, int min_kb = 4) {
-    int best = 1;
-    double best_eff = 0.0;
-    if (tiles >= c->num_sms) return 1;  // every SM has a tile of its own: splitting only adds reductions
-    for (int s = 1; s <= 8; ++s) {  // a cluster holds at most 8 CTAs
-        if (s > 1 && kb_total / s < min_kb) break;
-        const int ctas = tiles * s, waves = (ctas + slots - 1) / slots;
-        const double eff = (double)ctas / ((double)waves * slots);
-        if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
-    }
-    return best;
-}
-
-template <class Epi>
-cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
-                      int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                      const int32_t *cnt, const Epi &epi, bool allow_split = true, const int32_t *hint = nullptr) {
-    const int np = (n + 15) / 16 * 16;
-    const river_ctx::BMap *bm = tc_bmap(c, K, np);
-    if (!bm) return cudaErrorInvalidValue;
-    cudaError_t e = launch_k(tc_prep_kernel, dim3(np, (K + kPrepChunk - 1) / kPrepChunk), dim3(256), 0, c->stream, true, in, rows, cnt, K,
-                             c->tc_xhi, c->tc_xlo);
-    if (e != cudaSuccess) return e;
-    ++c->st.launches_last_step;
-    TcArgs a{};
-    a.K = K; a.n_pad = np;
-    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
-    // CTAs per SM: two with three stages each, or three with two when that puts more CTAs of one wave to work (while
-    // one CTA drains its accumulator and takes part in the cluster reduction the others keep the weight stream going);
-    // one with deep stages when the operand tiles are too large for that.
-    const size_t sm_smem = 228 * 1024, fixed = 1024 + 1024 + 256;  // per CTA: system reserve, alignment slack, barriers
-    auto stages_at = [&](int occ) {
-        const size_t room = std::min<size_t>(sm_smem / occ, 227 * 1024);
-        return room < fixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : 3, (room - fixed) / stage);
-    };
-    int occ = stages_at(2) ? 2 : 1;
-    a.splits = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * occ);
-    if (occ == 2 && stages_at(3) && allow_split) {
-        const int s3 = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * 3);
-        if (tiles * s3 > tiles * a.splits && tiles * s3 <= c->num_sms * 3) { occ = 3; a.splits = s3; }
-    }
-    a.n_stages = stages_at(occ);
-    // the finished tile lives in the pipeline memory
-    if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage) return cudaErrorInvalidValue;
-    if (!allow_split) a.splits = 1;
-    a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
-    a.rows = rows; a.cnt = cnt; a.dev_err = c->dev_err;
-    a.hint = hint ? hint : cnt;
-    static const bool probe_on = std::getenv("RIVER_TC_PROBE") != nullptr;
-    if (probe_on && c->profiling) {
-        const int kind = gateup ? 2 : q_tiles ? 0 : K > c->cfg.d ? 3 : 1;
-        a.probe = c->chain_stamps + 2 + 6 * (size_t)c->cfg.L + 8 * kind;
-        static int printed = 0;
-        if (printed++ < 8) std::fprintf(stderr, "tc kind %d: tiles %d splits %d stages %d np %d nkb %d\n", kind, tiles, a.splits, a.n_stages, np, K / kTcBK / a.splits);
-    }
-    const size_t smem = tc_smem_bytes(np, a.n_stages);
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaFuncSetAttribute(tc_gemm_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_smem = smem;
-    }
-    return launch_kc(tc_gemm_kernel<Epi>, dim3(tiles * a.splits), dim3(kTcThreads), smem, c->stream, true, a.splits, a0,
-                     a1, a2, bm->hi, bm->lo, a, epi);
-}
-
-// Exit-layer rows through the dequantising tensor-core kernel: m[0..2] are the code maps, w[0..2] the matching
-// scale / zero arrays (one matrix, gate + up, or q + k + v).
-template <class Epi>
-cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
-                         int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                         const int32_t *cnt, const int32_t *hint, const Epi &epi) {
-    const int np = (n + 15) / 16 * 16;
-    const river_ctx::BMap *bm = tc_bmap(c, K, np);
-    if (!bm) return cudaErrorInvalidValue;
-    cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np, (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk)), dim3(256), 0, c->stream, true, in, rows,
-                             cnt, K,
-                             reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(c->tc_xlo));
-    if (e != cudaSuccess) return e;
-    ++c->st.launches_last_step;
-    TcW4Args a{};
-    a.K = K; a.n_pad = np;
-    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
-    const size_t raw = (size_t)kW4RawBufs * kW4RawBytes;
-    // two CTAs per SM (16 dequantisation warps) when two operand stages fit in half of the shared memory
-    const bool two = 2 * stage + raw + 4096 <= 110 * 1024;
-    a.n_stages = two ? (int)std::min<size_t>(4, (110 * 1024 - raw - 4096) / stage)
-                     : (int)std::max<size_t>(2, std::min<size_t>(6, (214 * 1024 - raw) / stage));
-    // in raw tiles of four k-blocks: at least four per split, two when K is so short that four would allow only two
-    // splits (measured on the 1B shape, K = 2048: 2 -> 4 splits 35 -> 31 us per layer for QKV, 33 -> 27 us for O)
-    const int raw_tiles = K / (kTcBK * kW4Super);
-    a.splits = tc_pick_splits(c, tiles, raw_tiles, c->num_sms * (two ? 2 : 1), raw_tiles <= 8 ? 2 : 4);
-    if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage + raw) return cudaErrorInvalidValue;
-    a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
-    for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
-    a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
-    const size_t smem = tc_w4_smem_bytes(np, a.n_stages);
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaFuncSetAttribute(tc_gemm_w4_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_smem = smem;
-    }
-    return launch_kc(tc_gemm_w4_kernel<Epi>, dim3(tiles * a.splits), dim3(kW4Threads), smem, c->stream, true, a.splits,
-                     *m[0], *m[1], *m[2], bm->hi, bm->lo, a, epi);
 }
 
 // 2-D tiled tensor map over the KV pool seen as [all cache rows][dh] bf16, box = 16 rows x 64 elements (128 bytes),
@@ -701,34 +294,13 @@ struct LaunchScope {
     }
 };
 
-int profile_collect(river_ctx *c, int n = 0, int n_head = 0, const int32_t *row_pos_host = nullptr) {
+int profile_collect(river_ctx *c) {
     const river_config &g = c->cfg;
     const int L = g.L;
     std::vector<int32_t> na(L + 1), nr(L + 1);
-    std::vector<unsigned long long> stamps(2 + 6 * (size_t)L + 48);
     CUDA_TRY(c, cudaMemcpyAsync(na.data(), c->n_act, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(nr.data(), c->n_riv, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
-    CUDA_TRY(c, cudaMemcpyAsync(stamps.data(), c->chain_stamps, sizeof(unsigned long long) * stamps.size(),
-                                cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-    if (std::getenv("RIVER_TC_PROBE")) {  // debugging aid: milestones of CTA 0 of the last tensor-core GEMMs
-        const unsigned long long *sub = stamps.data() + 2 + 6 * (size_t)L;
-        const char *names[4] = {"qkv", "o", "gateup", "down"};
-        for (int k = 0; k < 4; ++k) {
-            const unsigned long long *t = sub + 8 * k;
-            std::fprintf(stderr, "tc probe %-7s setup+prefetch %6.2f wait %6.2f first-full %6.2f mainloop %6.2f acc %6.2f drain+reduce %6.2f epilogue %6.2f total %6.2f us\n",
-                         names[k], (t[1] - t[0]) * 1e-3, (t[2] - t[1]) * 1e-3, (t[3] - t[2]) * 1e-3, (t[4] - t[3]) * 1e-3,
-                         (t[5] - t[4]) * 1e-3, (t[6] - t[5]) * 1e-3, (t[7] - t[6]) * 1e-3, (t[7] - t[0]) * 1e-3);
-        }
-    }
-    if (std::getenv("RIVER_CHAIN_PROBE")) {  // debugging aid: where CTA 0 of the chain kernel spent the last step
-        const unsigned long long *sub = stamps.data() + 2 + 6 * (size_t)L;
-        const char *names[6] = {"qkv", "o", "gateup", "down", "attn/decide", "head"};
-        for (int k = 0; k < 6; ++k)
-            std::fprintf(stderr, "chain probe %-12s bf16: stage %7.1f stream %7.1f join %7.1f finish %7.1f wait %7.1f | w4: stage %7.1f stream %7.1f finish %7.1f (us per step)\n",
-                         names[k], sub[8 * k] * 1e-3, sub[8 * k + 1] * 1e-3, sub[8 * k + 7] * 1e-3, sub[8 * k + 2] * 1e-3, sub[8 * k + 3] * 1e-3,
-                         sub[8 * k + 4] * 1e-3, sub[8 * k + 5] * 1e-3, sub[8 * k + 6] * 1e-3);
-    }
     for (size_t i = 0; i < c->prof_rec.size(); ++i) {
         const auto &r = c->prof_rec[i];
         float ms = 0.f;
@@ -736,34 +308,7 @@ int profile_collect(river_ctx *c, int n = 0, int n_head = 0, const int32_t *row_
         c->prof_ms[r.cls] += ms;
         c->prof_launches[r.cls] += 1;
         double bytes = 0.0;
-        if (r.list_idx == -2) {
-            // the chain kernel: weights of the executed (layer, weight set) pairs, cache traffic, LM head; its phases
-            // as CTA 0 saw them (global timer at the phase boundaries) are booked under the per-phase classes
-            const int qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
-            const double w4f = 0.25 + 2.0 / g.group;
-            const double wb[4] = {2.0 * (qdim + 2.0 * kvdim) * g.d, 2.0 * qdim * g.d, 4.0 * g.F * g.d, 2.0 * g.F * g.d};
-            const int cls[6] = {K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE};
-            double kv_read = 0.0;
-            for (int b = 0; b < n; ++b) kv_read += (double)(row_pos_host[b] + 1) * 2.0 * kvdim * 2.0;
-            const double kv_write = (double)n * 2.0 * kvdim * 2.0;
-            for (int l = 0; l < L; ++l) {
-                const double f = (na[l] > 0 ? 1.0 : 0.0) + (nr[l] > 0 ? w4f : 0.0);
-                const double pb[6] = {wb[0] * f + kv_write, kv_read, wb[1] * f, wb[2] * f, wb[3] * f, (double)n * g.d * 8.0};
-                for (int ph = 0; ph < 6; ++ph) {
-                    c->prof_ms[cls[ph]] += (double)(stamps[1 + 6 * l + ph] - stamps[6 * l + ph]) * 1e-6;
-                    c->prof_launches[cls[ph]] += 1;
-                    c->prof_bytes[cls[ph]] += pb[ph];
-                    if (ph != 5) bytes += pb[ph];
-                }
-            }
-            if (n_head > 0) {
-                const double hb = 2.0 * g.V * g.d + 4.0 * n_head * g.V;
-                c->prof_ms[K_HEAD] += (double)(stamps[1 + 6 * (size_t)L] - stamps[6 * (size_t)L]) * 1e-6;
-                c->prof_launches[K_HEAD] += 1;
-                c->prof_bytes[K_HEAD] += hb;
-                bytes += hb;
-            }
-        } else if (r.list_idx < 0) bytes = r.bytes_act;
+        if (r.list_idx < 0) bytes = r.bytes_act;
         else bytes = (na[r.list_idx] > 0 ? r.bytes_act : 0.0) + (nr[r.list_idx] > 0 ? r.bytes_riv : 0.0);
         c->prof_bytes[r.cls] += bytes;
     }
@@ -772,9 +317,16 @@ int profile_collect(river_ctx *c, int n = 0, int n_head = 0, const int32_t *row_
 }
 
 // The launch sequence of one step over the rows described in the device metadata (rows, positions, caller buffers).
-int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
+//
+// Steps of up to four rows: per block QKV, attention, O, gate/up, down - the exit decision of block l is taken by the
+// QKV kernel of block l + 1 (every CTA computes Eq. 1 for itself while it stages the rows, see gemv_stream.cuh), so
+// no kernel boundary is spent on it; one score kernel after the LM head records the last block's score and the final
+// row lists.  Steps of five and more rows: backbone rows on the tensor-core GEMM, exit-layer rows on its dequantising
+// variant, and the score / compaction kernel after every block.
+int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool record_fail = false) {
     const river_config &g = c->cfg;
     const int L = g.L, d = g.d, B = g.max_batch;
+    int32_t *fail_buf = record_fail ? c->prefill_fail : nullptr;
     c->st.launches_last_step = 0;
     Lists lists{c->act_idx, c->riv_idx, c->n_act, c->n_riv, B};
     const int qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
@@ -784,20 +336,29 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
     const double kv_write = (double)n * 2.0 * kvdim * 2.0;
     cudaError_t err = cudaSuccess;
     auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
+    const bool fold = n <= 4;  // the decisions ride in the QKV kernels
+    const DecideArgs no_dec{};
 
     {
         LaunchScope ls(c, K_BEGIN, (double)n * d * 2.0, 0, -1);
         note(launch_k(step_begin_kernel, dim3(std::max(n, 1)), dim3(128), 0, c->stream, false, c->meta(), c->upd(),
                       c->page_tbl_dev, g.max_pages_per_seq, B, c->embed, d, g.V, c->h[0], c->row_pos(), c->inv_freq,
-                      g.dh / 2, c->rope_cs, L, g.entry_layer, c->exited, c->dev_err, lists, c->hint_act, c->tickets));
+                      g.dh / 2, c->rope_cs, L, g.entry_layer, c->state_at(0), c->dev_err, lists, c->hint_act, c->tickets));
     }
+    auto launch_score = [&](int l, const float *h_in, const float *h_out) {
+        LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
+        note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, true, c->meta(), l, L, g.entry_layer,
+                      g.exit_mode, h_in, h_out, d, c->pass, (const uint8_t *)c->state_at(l - 1), c->state_at(l), lists,
+                      c->hint_act, c->tickets + 1, fail_buf, (const int32_t *)c->row_slot()));
+    };
     int hi = 0;                  // h[hi] = block input
+    const float *prev_in = nullptr;  // input of the previous block (its output is h[hi])
     for (int l = 1; l <= L; ++l) {
         const river_layer_weights &w = c->layers[l - 1];
         const int has_river = w.rq.codes != nullptr;
         const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
         const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
-        const RowLists rl{ai, na, ri, nr, c->hint_act, c->meta_dev /* StepMeta::n_rows */, c->exited};
+        const RowLists rl{ai, na, ri, nr, c->hint_act, c->meta_dev /* StepMeta::n_rows */, c->state_at(l - 1)};
         float *h_in = c->h[hi], *h_mid = c->h[(hi + 1) % 3], *h_out = c->h[(hi + 2) % 3];
         // With more rows than one CUDA-core pass takes, the backbone rows go to the tensor-core GEMM and the stream
         // kernel only serves the exit-layer rows of the same launch slot.
@@ -805,18 +366,23 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
         const river_ctx::LayerMaps *tm = tc ? &c->tc_maps[l - 1] : nullptr;
         const river_ctx::LayerMaps *wm = (tc && c->w4tc_ok && has_river) ? &c->w4_maps[l - 1] : nullptr;
         const int32_t *nrh = c->n_riv + std::max(0, l - 2);  // never above the count entering this block
-        const bool fuse_score = !tc && (g.flags & RIVER_F_FUSED_SCORE);  // opt-in; needs the down projection on the stream kernel
         const int skip_bb = tc ? 1 : 0;
-        // ---- a2: attention norm + QKV + RoPE + KV write
+        // ---- a2: attention norm + QKV + RoPE + KV write (+ a6 / a7 of the previous block when the step is small)
         {
             const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
             LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
             QkvProblem p{};
             p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
-            p.rq = w4(w.rq); p.rk = w4(w.rk); p.rv = w4(w.rv);
+            p.rq = w4_of(w.rq); p.rk = w4_of(w.rk); p.rv = w4_of(w.rv);
             p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
             p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
             const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
+            DecideArgs dec{};
+            if (fold && l >= 2) {
+                dec.meta = c->meta(); dec.l = l - 1; dec.L = L; dec.entry_layer = g.entry_layer; dec.exit_mode = g.exit_mode;
+                dec.h_prev = prev_in; dec.state_in = c->state_at(l - 2); dec.state_out = c->state_at(l - 1);
+                dec.lists = lists; dec.hint_act = c->hint_act; dec.fail = fail_buf; dec.row_slot = c->row_slot();
+            }
             if (tc) {
                 TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
                 note(launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM,
@@ -828,19 +394,19 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
                 const river_w4 *const cw[3] = {&w.rq, &w.rk, &w.rv};
                 note(launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ri, nr, nrh, e));
             } else if (!tc || has_river)
-                note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, skip_bb));
+                note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, skip_bb, dec));
         }
         // ---- a3: paged GQA decode attention
         {
             LaunchScope ls(c, K_ATTN, kv_read, 0, -1);
-            note(launch_attention(c, n, l - 1, !(g.flags & RIVER_F_SIMPLE_ATTN)));
+            note(launch_attention(c, n, l - 1));
         }
         // ---- a4: O projection + residual
         {
             const double wb = 2.0 * qdim * d;
             LaunchScope ls(c, K_OPROJ, wb, wb * w4f, l - 1);
             ResidProblem p{};
-            p.w = (const uint16_t *)w.wo; p.rw = w4(w.ro); p.K = qdim; p.out_dim = d; p.group = g.group;
+            p.w = (const uint16_t *)w.wo; p.rw = w4_of(w.ro); p.K = qdim; p.out_dim = d; p.group = g.group;
             p.resid = h_in; p.out = h_mid;
             const ProjIn in{c->obuf, nullptr, 0.f};
             if (tc) {
@@ -853,14 +419,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
                 const river_w4 *const cw[3] = {&w.ro, &w.ro, &w.ro};
                 note(launch_tc_w4(c, in, cm, cw, qdim, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
             } else if (!tc || has_river)
-                note(launch_stream(c, p, in, rl, qdim, d / 2, n, has_river, tc || !(g.flags & RIVER_F_SIMPLE_ATTN), skip_bb));
+                note(launch_stream(c, p, in, rl, qdim, d / 2, n, has_river, true, skip_bb, no_dec));
         }
         // ---- a5: FFN norm + gate/up + SwiGLU
         {
             const double wb = 2.0 * 2.0 * g.F * d;
             LaunchScope ls(c, K_GATEUP, wb, wb * w4f, l - 1);
             GateUpProblem p{};
-            p.wg = (const uint16_t *)w.wg; p.wu = (const uint16_t *)w.wu; p.rg = w4(w.rg); p.ru = w4(w.ru);
+            p.wg = (const uint16_t *)w.wg; p.wu = (const uint16_t *)w.wu; p.rg = w4_of(w.rg); p.ru = w4_of(w.ru);
             p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
             const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
             if (tc) {
@@ -872,14 +438,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
                 const CUtensorMap *const cm[3] = {&wm->g, &wm->u, &wm->u};
                 const river_w4 *const cw[3] = {&w.rg, &w.ru, &w.ru};
                 note(launch_tc_w4(c, in, cm, cw, d, g.F / 64, n, 1, 0, 0, ri, nr, nrh, e));
-            } else if (!tc || has_river) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb));
+            } else if (!tc || has_river) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb, no_dec));
         }
         // ---- a5: down projection + residual
         {
             const double wb = 2.0 * g.F * d;
             LaunchScope ls(c, K_DOWN, wb, wb * w4f, l - 1);
             ResidProblem p{};
-            p.w = (const uint16_t *)w.wd; p.rw = w4(w.rd); p.K = g.F; p.out_dim = d; p.group = g.group;
+            p.w = (const uint16_t *)w.wd; p.rw = w4_of(w.rd); p.K = g.F; p.out_dim = d; p.group = g.group;
             p.resid = h_mid; p.out = h_out;
             const ProjIn in{c->act, nullptr, 0.f};
             if (tc) {
@@ -891,24 +457,12 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
                 const CUtensorMap *const cm[3] = {&wm->d, &wm->d, &wm->d};
                 const river_w4 *const cw[3] = {&w.rd, &w.rd, &w.rd};
                 note(launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
-            } else if (!tc || has_river) {
-                ScoreTail st{};
-                if (fuse_score) {
-                    st.meta = c->meta(); st.l = l; st.L = L; st.entry_layer = g.entry_layer; st.exit_mode = g.exit_mode;
-                    st.d = d; st.h_in = h_in; st.h_out = h_out; st.pass = c->pass; st.exited = c->exited; st.lists = lists;
-                    st.hint_act = c->hint_act; st.ticket = c->tickets + 1;
-                }
-                note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb, st));
-            }
+            } else if (!tc || has_river)
+                note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb, no_dec));
         }
-        // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1 (with RIVER_F_FUSED_SCORE: done
-        // by the last CTA of the down projection above)
-        if (!fuse_score) {
-            LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
-            note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, true, c->meta(), l, L,
-                          g.entry_layer, g.exit_mode, (const float *)h_in, (const float *)h_out, d, c->pass, c->exited,
-                          lists, c->hint_act, c->tickets + 1));
-        }
+        // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
+        if (!fold) launch_score(l, h_in, h_out);
+        prev_in = h_in;
         hi = (hi + 2) % 3;
     }
     if (n_head > 0) {
@@ -923,28 +477,18 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
             n_parts = g.V / kTcBM;
             TcHeadEpi e{c->meta(), g.V, c->part_val, c->part_idx, n_parts};
             note(launch_tc(c, a.in, c->tc_map_head, c->tc_map_head, c->tc_map_head, d, n_parts, n_head, 0, 0, 0,
-                           c->head_rows(), c->meta_dev + 2 /* StepMeta::n_head_rows */, e, false));
+                           c->head_rows(), c->meta_dev + 2 /* StepMeta::n_head_rows */, e, false, nullptr));
         } else {
-            int n_sel = 1;
-            while (n_sel < n_head && n_sel < 4) n_sel *= 2;
-            const int xstride = xs_stride(d, 8);
-            const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xstride);
             LaunchScope ls(c, K_HEAD, 2.0 * g.V * d + 4.0 * n_head * g.V, 0, -1);
-            switch (n_sel) {
-                case 1: cudaFuncSetAttribute(lm_head_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        note(launch_k(lm_head_kernel<1, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride)); break;
-                case 2: cudaFuncSetAttribute(lm_head_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        note(launch_k(lm_head_kernel<2, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride)); break;
-                default: cudaFuncSetAttribute(lm_head_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                        note(launch_k(lm_head_kernel<4, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride)); break;
-            }
+            note(launch_head_stream(c, a, n_head));
         }
         {
             LaunchScope ls(c, K_ARGMAX, 0, 0, -1);
-            note(launch_k(argmax_final_kernel, dim3(n_head), dim3(128), 0, c->stream, true, c->meta(),
-                          (const float *)c->part_val, (const int32_t *)c->part_idx, n_parts));
+            note(launch_argmax_final(c, n_head, n_parts));
         }
     }
+    // small steps: the last block's score (a diagnostic: no exit is taken after block L) and the final row lists
+    if (fold) launch_score(L, prev_in, c->h[hi]);
     if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(err));
     c->st.launches_total += c->st.launches_last_step;
@@ -952,162 +496,9 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host) {
     return 0;
 }
 
-// ---- persistent layer-chain kernel (steps of at most four rows)
-int chain_part_cap(const river_config &g, int grid) {  // most units (task x K-slice) a CTA owns in any pass
-    auto cap_for = [&](int tasks, int K, bool w4) {
-        const int nch = w4 ? K / 32 : K / 8;
-        const int nit = (nch + 31) / 32, its = w4 ? kW4Its : kBfIts;
-        const int nsl = std::max(1, (nit + its - 1) / its);
-        return ((tasks + grid - 1) / grid) * nsl;
-    };
-    const int qdim = g.Hq * g.dh;
-    int cap = 2;
-    for (int w4 = 0; w4 < 2; ++w4) {
-        cap = std::max(cap, cap_for((g.Hq + 2 * g.Hkv) * (g.dh / 2), g.d, w4));
-        cap = std::max(cap, cap_for(g.d / 2, qdim, w4));
-        cap = std::max(cap, cap_for(g.F, g.d, w4));
-        cap = std::max(cap, cap_for(g.d / 2, g.F, w4));
-    }
-    return std::max(cap, cap_for(g.V / 2, g.d, false));
-}
-
-struct ChainPlan { ChainLayout lay; };
-ChainPlan chain_plan(const river_ctx *c, int N) {  // bytes == 0: N rows per pass do not fit in shared memory
-    const river_config &g = c->cfg;
-    const int Kmax = std::max(std::max(g.d, g.F), g.Hq * g.dh);
-    const ChainLayout l = chain_layout(N, Kmax, chain_part_cap(g, c->chain_grid), g.dh, g.Hq / g.Hkv);
-    if (l.bytes <= 200 * 1024) return ChainPlan{l};
-    return ChainPlan{ChainLayout{0, 0, 0}};
-}
-
-typedef void (*ChainKern)(const ChainArgs);
-ChainKern chain_kernel_for(int N, int dh, int gq) {
-#define CHAIN_CASE(N_, DH_, GQ_) if (N == N_ && dh == DH_ && gq == GQ_) return decode_chain_kernel<N_, DH_, GQ_>;
-    CHAIN_CASE(1, 64, 2) CHAIN_CASE(2, 64, 2) CHAIN_CASE(4, 64, 2)
-    CHAIN_CASE(1, 64, 4) CHAIN_CASE(2, 64, 4) CHAIN_CASE(4, 64, 4)
-    CHAIN_CASE(1, 128, 4) CHAIN_CASE(2, 128, 4) CHAIN_CASE(4, 128, 4)
-#undef CHAIN_CASE
-    return nullptr;
-}
-
-// Rows per pass for a step of n rows, or 0 if the chain kernel does not take this step.
-int chain_rows_per_pass(const river_ctx *c, int n) {
-    const river_config &g = c->cfg;
-    if (!c->chain_ok || n < 1 || n > 4) return 0;
-    const int N = n == 1 ? 1 : (n == 2 ? 2 : 4);
-    if (chain_plan(c, N).lay.bytes == 0) return 0;
-    return N;
-}
-
-bool chain_setup(river_ctx *c) {
-    const river_config &g = c->cfg;
-    if (!(g.flags & RIVER_F_CHAIN)) return false;
-    if (g.V % 2 || g.d % 4 || g.F % 2) return false;
-    if (!chain_kernel_for(1, g.dh, g.Hq / g.Hkv)) return false;
-    int dev = 0, coop = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return false;
-    c->chain_grid = c->num_sms;
-    bool any = false;
-    for (int N = 1; N <= 4; N *= 2) {
-        const ChainPlan pl = chain_plan(c, N);
-        if (pl.lay.bytes == 0) continue;
-        ChainKern k = chain_kernel_for(N, g.dh, g.Hq / g.Hkv);
-        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.lay.bytes) != cudaSuccess) return false;
-        int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kChainThreads, pl.lay.bytes) != cudaSuccess || occ < 1) return false;
-        any = true;
-    }
-    if (!any) return false;
-    std::vector<LayerDev> ld(g.L);
-    for (int l = 0; l < g.L; ++l) {
-        const river_layer_weights &w = c->layers[l];
-        LayerDev &x = ld[l];
-        x.attn_norm = (const uint16_t *)w.attn_norm; x.ffn_norm = (const uint16_t *)w.ffn_norm;
-        x.wq = (const uint16_t *)w.wq; x.wk = (const uint16_t *)w.wk; x.wv = (const uint16_t *)w.wv;
-        x.wo = (const uint16_t *)w.wo; x.wg = (const uint16_t *)w.wg; x.wu = (const uint16_t *)w.wu;
-        x.wd = (const uint16_t *)w.wd;
-        x.rq = w4(w.rq); x.rk = w4(w.rk); x.rv = w4(w.rv); x.ro = w4(w.ro); x.rg = w4(w.rg); x.ru = w4(w.ru); x.rd = w4(w.rd);
-        x.has_river = w.rq.codes != nullptr;
-        x.pad = 0;
-    }
-    if (cudaMemcpy(c->layers_dev, ld.data(), sizeof(LayerDev) * g.L, cudaMemcpyHostToDevice) != cudaSuccess) return false;
-    const int kb = (g.flags >> 8) & 0xff;  // tuning aid: KiB of the next phase each warp requests from the L2
-    if (kb) c->chain_pf_bytes = kb * 1024;
-    return true;
-}
-
-int run_chain(river_ctx *c, int n, int n_head, int N, const int32_t *row_pos_host) {
-    const river_config &g = c->cfg;
-    const int L = g.L, d = g.d, B = g.max_batch;
-    c->st.launches_last_step = 0;
-    Lists lists{c->act_idx, c->riv_idx, c->n_act, c->n_riv, B};
-    cudaError_t err = cudaSuccess;
-    auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
-    {
-        LaunchScope ls(c, K_BEGIN, (double)n * d * 2.0, 0, -1);
-        note(launch_k(step_begin_kernel, dim3(std::max(n, 1)), dim3(128), 0, c->stream, false, c->meta(), c->upd(),
-                      c->page_tbl_dev, g.max_pages_per_seq, B, c->embed, d, g.V, c->h[0], c->row_pos(), c->inv_freq,
-                      g.dh / 2, c->rope_cs, L, g.entry_layer, c->exited, c->dev_err, lists, c->hint_act, c->tickets));
-    }
-    note(cudaMemsetAsync(c->tickets + 2, 0, sizeof(unsigned), c->stream));
-    if (c->profiling) note(cudaMemsetAsync(c->chain_stamps + 2 + 6 * (size_t)L, 0, sizeof(unsigned long long) * 48, c->stream));
-    ChainArgs a{};
-    a.meta = c->meta(); a.layers = c->layers_dev;
-    a.L = L; a.d = d; a.Hq = g.Hq; a.Hkv = g.Hkv; a.dh = g.dh; a.F = g.F; a.V = g.V; a.group = g.group;
-    a.entry_layer = g.entry_layer; a.exit_mode = g.exit_mode; a.eps = g.rms_eps;
-    a.qscale = 1.4426950408889634f / std::sqrt((float)g.dh);
-    a.h[0] = c->h[0]; a.h[1] = c->h[1]; a.h[2] = c->h[2]; a.qbuf = c->qbuf; a.obuf = c->obuf; a.act = c->act;
-    a.rope_cs = c->rope_cs; a.kv = kv_addr(c, 0);
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.attn_tickets = c->attn_tickets;
-    a.exited = c->exited; a.lists = lists;
-    a.lm_head = c->lm_head; a.final_norm = c->final_norm; a.head_rows = c->head_rows();
-    a.part_val = c->part_val; a.part_idx = c->part_idx;
-    a.bar = c->tickets + 2; a.dev_err = c->dev_err;
-    a.stamps = c->profiling ? c->chain_stamps : nullptr;
-    a.sub = c->profiling ? c->chain_stamps + 2 + 6 * (size_t)L : nullptr;
-    a.part_cap = chain_part_cap(g, c->chain_grid);
-    a.pf_bytes = c->chain_pf_bytes;
-    const ChainPlan pl = chain_plan(c, N);
-    a.xs_floats = pl.lay.xs_floats;
-    a.part_floats = pl.lay.part_floats;
-    const size_t smem = pl.lay.bytes;
-    {
-        LaunchScope ls(c, K_CHAIN, 0, 0, -2);
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(c->chain_grid);
-        cfg.blockDim = dim3(kChainThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = c->stream;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeCooperative;
-        at[0].val.cooperative = 1;
-        cfg.attrs = at;
-        cfg.numAttrs = 1;
-        note(cudaLaunchKernelEx(&cfg, chain_kernel_for(N, g.dh, g.Hq / g.Hkv), a));
-    }
-    if (n_head > 0) {
-        LaunchScope ls(c, K_ARGMAX, 0, 0, -1);
-        note(launch_k(argmax_final_kernel, dim3(n_head), dim3(128), 0, c->stream, false, c->meta(),
-                      (const float *)c->part_val, (const int32_t *)c->part_idx, c->chain_grid));
-    }
-    if (err == cudaSuccess) err = cudaGetLastError();
-    if (err != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(err));
-    c->st.launches_total += c->st.launches_last_step;
-    if (c->profiling) return profile_collect(c, n, n_head, row_pos_host);
-    return 0;
-}
-
 // One decode step through a CUDA graph of the launch sequence (captured the second time a row count is seen; the
 // per-step inputs live in device memory, so the graph never needs new parameters).
 int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
-    if (const int N = chain_rows_per_pass(c, n)) {
-        const int rc = run_chain(c, n, n, N, row_pos_host);
-        if (rc != RIVER_E_DEVICE || cudaPeekAtLastError() != cudaSuccess) return rc;
-        // the cooperative launch was refused (co-residency cannot be guaranteed in this context): use the
-        // one-kernel-per-stage plan from now on; its first kernel redoes the step prologue
-        c->chain_ok = false;
-    }
     const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
     if (!use_graph) return run_rows(c, n, n, row_pos_host);
     const int key_splits = c->attn_small_now ? 0 : c->attn_splits_now;  // the attention grid of the captured launches
@@ -1133,6 +524,89 @@ int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
         }
     c->graphs.push_back({n, c->attn_small_now, key_splits, nullptr, 0});
     return run_rows(c, n, n, row_pos_host);  // first use: plain launches (also sets the kernels' attributes)
+}
+
+// Device error word -> return code.  The word is sticky on the device; once the host has seen it, the context
+// refuses further steps with the same code until river_clear_device_error.
+int note_device_error(river_ctx *c, int de) {
+    c->st.device_error = de;
+    if (de == 0) return RIVER_OK;
+    static const char *const names[] = {"", "forced exit layer out of range", "token id out of range",
+                                        "page id out of range", "a bounded device-side wait ran out", "internal"};
+    const std::string what = de > 0 && de < 6 ? names[de] : "unknown";
+    return fail(c, de == DEV_WAIT_TIMEOUT ? RIVER_E_TIMEOUT : RIVER_E_DEVICE,
+                "a kernel flagged an error (" + std::to_string(de) + ": " + what + "); river_clear_device_error resets it");
+}
+int refuse_if_flagged(river_ctx *c) {
+    if (c->st.device_error == 0) return RIVER_OK;
+    return note_device_error(c, c->st.device_error);
+}
+
+// Give back the pages a failed call took: the host table entries return to -1 and the pages to the free list, in
+// reverse order, so that the retry finds the state it would have found at first.
+void rollback_pages(river_ctx *c, const int32_t *mh, int n_upd) {
+    const river_config &g = c->cfg;
+    const int32_t *u = mh + kMetaHdr + 2 * g.max_batch;
+    for (int i = n_upd - 1; i >= 0; --i) {
+        const int slot = u[i], pi = u[g.max_batch + i], page = u[2 * g.max_batch + i];
+        c->page_tbl[(size_t)slot * g.max_pages_per_seq + pi] = -1;
+        c->free_pages.push_back(page);
+    }
+}
+
+
+// One pass of the prompts through the decode kernels in chunks of rows (slot, position): rows of a chunk are
+// consecutive prompt positions, possibly of several sequences; K/V of the whole chunk are written before its attention
+// runs, and a row attends to positions <= its own, so causality holds inside a chunk.  depth[s]: the unified exit depth
+// of sequence s (L = the whole backbone).  record_fail: note per (sequence, block) whether some position failed Eq. 1.
+int prefill_pass(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t *tok, const int32_t *offsets,
+                 const int32_t *depth, float tau, bool record_fail, float *logits_last, int32_t *next_tok) {
+    const river_config &g = c->cfg;
+    {
+        std::vector<float> ta(g.max_batch, tau);
+        CUDA_TRY(c, cudaMemcpyAsync(c->tau_i, ta.data(), sizeof(float) * ta.size(), cudaMemcpyHostToDevice, c->stream));
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    }
+    int s = 0, p = 0;  // next (sequence, position) to schedule
+    while (s < n_seqs) {
+        int32_t *mh = next_meta(c);
+        int n = 0, n_upd = 0, n_head = 0;
+        const int tok0 = offsets[s] + p;
+        int head_seq[kMaxBatch];
+        while (s < n_seqs && n < g.max_batch) {
+            const int len = offsets[s + 1] - offsets[s];
+            if (offsets[s] + p != tok0 + n) break;  // token ids of a chunk must be contiguous in tok
+            if (int rc = ensure_page(c, slots[s], p, mh, n_upd)) { rollback_pages(c, mh, n_upd); return rc; }
+            mh[kMetaHdr + n] = slots[s];
+            mh[kMetaHdr + g.max_batch + n] = p;
+            mh[kMetaHdr + 6 * g.max_batch + n] = c->page_tbl[(size_t)slots[s] * g.max_pages_per_seq + p / kPage];
+            mh[kMetaHdr + 7 * g.max_batch + n] = depth[s];
+            if (p == len - 1) {
+                mh[kMetaHdr + 5 * g.max_batch + n_head] = n;
+                head_seq[n_head++] = s;
+            }
+            ++n;
+            if (++p == len) { c->seq_len[slots[s]] = len; ++s; p = 0; }
+        }
+        mh[0] = n; mh[1] = n_upd; mh[2] = n_head;
+        set_attn_meta(c, mh, n);
+        const bool want_logits = logits_last && n_head > 0;
+        set_io_meta(mh, tok + tok0, c->tau_i, c->row_forced(), want_logits ? c->logits_i : nullptr, c->next_i, c->exit_i,
+                    nullptr);
+        if (int rc = push_meta(c, mh)) return rc;
+        c->rows_distinct = false;  // consecutive positions of one sequence share a chunk
+        const int rc_rows = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch, record_fail);
+        c->rows_distinct = true;
+        if (rc_rows) return rc_rows;
+        for (int i = 0; i < n_head; ++i) {
+            if (logits_last)
+                CUDA_TRY(c, cudaMemcpyAsync(logits_last + (size_t)head_seq[i] * g.V, c->logits_i + (size_t)i * g.V,
+                                            sizeof(float) * g.V, cudaMemcpyDeviceToDevice, c->stream));
+            if (next_tok)
+                CUDA_TRY(c, cudaMemcpyAsync(next_tok + head_seq[i], c->next_i + i, sizeof(int32_t), cudaMemcpyDeviceToDevice, c->stream));
+        }
+    }
+    return RIVER_OK;
 }
 
 int check_slot(const river_ctx *c, int slot) { return slot >= 0 && slot < c->cfg.max_seqs; }
@@ -1191,21 +665,21 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
         river_destroy(c);
         return RIVER_E_DEVICE;
     };
-    int dev = 0;
+    int dev = 0, cc_major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return bail("cudaGetDevice failed (no CUDA device?)");
-    cudaDeviceProp prop;
-    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return bail("cudaGetDeviceProperties failed");
-    if (prop.major != 10) return bail("this library is built for sm_100a (B200) only");
-    c->num_sms = prop.multiProcessorCount;
+    if (cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return bail("cudaDeviceGetAttribute failed");
+    if (cc_major != 10) return bail("this library is built for sm_100a (B200) only");
+    c->device = dev;
     if (make_kv_tensor_map(c)) { river_destroy(c); return RIVER_E_DEVICE; }
     c->tc_ok = !(cfg->flags & RIVER_F_NO_TC) && tc_shape_ok(*cfg) && make_tc_maps(c);
     c->w4tc_ok = c->tc_ok && !(cfg->flags & RIVER_F_NO_W4TC) && make_w4_maps(c);
-    c->chain_ok = chain_setup(c);
     for (int i = 0; i < kStaging; ++i) {
         if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");
         if (cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail("cudaEventCreate failed");
     }
-    c->pin_io_bytes = (size_t)cfg->max_batch * (4 * sizeof(int32_t) + sizeof(float));
+    c->pin_io_bytes = (size_t)cfg->max_batch * (4 * sizeof(int32_t) + sizeof(float)) + sizeof(int32_t);
     if (cudaMallocHost(&c->pin_io, c->pin_io_bytes) != cudaSuccess) return bail("cudaMallocHost failed");
     c->page_tbl.assign((size_t)cfg->max_seqs * cfg->max_pages_per_seq, -1);
     c->seq_len.assign(cfg->max_seqs, 0);
@@ -1224,6 +698,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     cudaError_t e = cudaMemcpyAsync(c->inv_freq, fr.data(), sizeof(double) * fr.size(), cudaMemcpyHostToDevice, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->page_tbl_dev, 0xff, sizeof(int32_t) * c->page_tbl.size(), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->state, 0, (size_t)(cfg->L + 1) * c->state_stride, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
 
@@ -1240,20 +715,26 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
                       float *scores) {
     if (!c) return RIVER_E_BADARG;
     const river_config &g = c->cfg;
+    if (int rc = refuse_if_flagged(c)) return rc;
     if (batch <= 0 || batch > g.max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
     if (!slots || !tok || !tau || !next_tok || !exit_layer) return fail(c, RIVER_E_BADARG, "null argument");
+    // everything that can fail is checked before any page is taken: slots, lengths, and the pages the whole batch needs
+    int new_pages = 0;
     for (int b = 0; b < batch; ++b) {
         if (!check_slot(c, slots[b])) return fail(c, RIVER_E_BADSLOT, "slot out of range");
         for (int b2 = 0; b2 < b; ++b2)
             if (slots[b2] == slots[b]) return fail(c, RIVER_E_BADSLOT, "a slot appears twice in one step");
-        if (c->seq_len[slots[b]] >= g.max_pages_per_seq * kPage) return fail(c, RIVER_E_NOPAGE, "sequence full");
+        const int pos = c->seq_len[slots[b]];
+        if (pos >= g.max_pages_per_seq * kPage) return fail(c, RIVER_E_NOPAGE, "sequence full");
+        if (c->page_tbl[(size_t)slots[b] * g.max_pages_per_seq + pos / kPage] < 0) ++new_pages;
     }
+    if (new_pages > (int)c->free_pages.size()) return fail(c, RIVER_E_NOPAGE, "KV pool exhausted");
     int32_t *mh = next_meta(c);
     int n_upd = 0;
     c->last_pos.resize(batch);
     for (int b = 0; b < batch; ++b) {
         const int pos = c->seq_len[slots[b]];
-        if (int rc = ensure_page(c, slots[b], pos, mh, n_upd)) return rc;
+        if (int rc = ensure_page(c, slots[b], pos, mh, n_upd)) { rollback_pages(c, mh, n_upd); return rc; }
         mh[kMetaHdr + b] = slots[b];
         mh[kMetaHdr + g.max_batch + b] = pos;
         mh[kMetaHdr + 5 * g.max_batch + b] = b;
@@ -1263,7 +744,7 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
     mh[0] = batch; mh[1] = n_upd; mh[2] = batch;
     set_attn_meta(c, mh, batch);
     set_io_meta(mh, tok, tau, forced_exit, logits, next_tok, exit_layer, scores);
-    if (int rc = push_meta(c, mh)) return rc;
+    if (int rc = push_meta(c, mh)) { rollback_pages(c, mh, n_upd); return rc; }
     if (int rc = run_step(c, batch, c->last_pos.data())) return rc;
     for (int b = 0; b < batch; ++b) c->seq_len[slots[b]] += 1;
     c->st.steps += 1;
@@ -1285,6 +766,7 @@ int river_decode_step_host(river_ctx *c, int batch, const int32_t *slots, const 
     const size_t B = g.max_batch;
     int32_t *p_tok = (int32_t *)c->pin_io, *p_forced = p_tok + B, *p_next = p_forced + B, *p_exit = p_next + B;
     float *p_tau = (float *)(p_exit + B);
+    int32_t *p_err = (int32_t *)(p_tau + B);  // pin_io holds 5 arrays of max_batch entries and this word
     std::memcpy(p_tok, tok, sizeof(int32_t) * batch);
     std::memcpy(p_tau, tau, sizeof(float) * batch);
     if (forced_exit) std::memcpy(p_forced, forced_exit, sizeof(int32_t) * batch);
@@ -1297,6 +779,7 @@ int river_decode_step_host(river_ctx *c, int batch, const int32_t *slots, const 
         return rc;
     CUDA_TRY(c, cudaMemcpyAsync(p_next, c->next_i, sizeof(int32_t) * batch, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(p_exit, c->exit_i, sizeof(int32_t) * batch, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(p_err, c->dev_err, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
     if (logits)
         CUDA_TRY(c, cudaMemcpyAsync(logits, c->logits_i, sizeof(float) * (size_t)batch * g.V, cudaMemcpyDeviceToHost, c->stream));
     if (scores)
@@ -1304,16 +787,19 @@ int river_decode_step_host(river_ctx *c, int batch, const int32_t *slots, const 
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     std::memcpy(next_tok, p_next, sizeof(int32_t) * batch);
     std::memcpy(exit_layer, p_exit, sizeof(int32_t) * batch);
-    return RIVER_OK;
+    return note_device_error(c, *p_err);
 }
 
 int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t *tok, const int32_t *offsets,
-                  int prefill_exit_layer, float *logits_last, int32_t *next_tok) {
+                  int prefill_exit_layer, float tau, float *logits_last, int32_t *next_tok, int32_t *depth_out) {
     if (!c) return RIVER_E_BADARG;
     const river_config &g = c->cfg;
+    if (int rc = refuse_if_flagged(c)) return rc;
     if (n_seqs <= 0 || !slots || !tok || !offsets) return fail(c, RIVER_E_BADARG, "null / empty argument");
-    if (prefill_exit_layer < std::max(g.entry_layer, 0) || prefill_exit_layer > g.L)
-        return fail(c, RIVER_E_BADARG, "prefill_exit_layer must lie in [entry_layer, L]");
+    const bool auto_depth = prefill_exit_layer == -1;
+    if (!auto_depth && (prefill_exit_layer < std::max(g.entry_layer, 0) || prefill_exit_layer > g.L))
+        return fail(c, RIVER_E_BADARG, "prefill_exit_layer must be -1 or lie in [entry_layer, L]");
+    long long new_pages = 0;
     for (int s = 0; s < n_seqs; ++s) {
         if (!check_slot(c, slots[s])) return fail(c, RIVER_E_BADSLOT, "slot out of range");
         if (c->seq_len[slots[s]] != 0) return fail(c, RIVER_E_BADSLOT, "prefill needs an empty slot");
@@ -1322,56 +808,52 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
         const int n = offsets[s + 1] - offsets[s];
         if (n <= 0) return fail(c, RIVER_E_BADARG, "empty prompt");
         if (n > g.max_pages_per_seq * kPage) return fail(c, RIVER_E_NOPAGE, "prompt longer than the page table");
+        for (int pi = 0; pi < (n + kPage - 1) / kPage; ++pi)
+            if (c->page_tbl[(size_t)slots[s] * g.max_pages_per_seq + pi] < 0) ++new_pages;
     }
-    // constant per-row inputs of every chunk: exit forced at the unified depth, threshold unused
-    {
-        std::vector<int32_t> fe(g.max_batch, prefill_exit_layer);
-        std::vector<float> ta(g.max_batch, INFINITY);
-        CUDA_TRY(c, cudaMemcpyAsync(c->forced_i, fe.data(), sizeof(int32_t) * fe.size(), cudaMemcpyHostToDevice, c->stream));
-        CUDA_TRY(c, cudaMemcpyAsync(c->tau_i, ta.data(), sizeof(float) * ta.size(), cudaMemcpyHostToDevice, c->stream));
+    if (new_pages > (long long)c->free_pages.size()) return fail(c, RIVER_E_NOPAGE, "KV pool exhausted");
+    // Unified depth (Section 4.2, "Prefill Phase": all tokens of a prompt leave at one depth).  -1: per sequence, the
+    // first block l in [max(entry_layer, 1), L - 1] after which EVERY position of the prompt passes Eq. 1 (s > tau),
+    // else L.  Scores up to that block only involve backbone blocks, so a first pass runs the whole backbone over the
+    // prompts and notes per (sequence, block) whether some position failed; if some depth is below L a second pass
+    // redoes the prompts with the exit layers above each sequence's depth (the cache entries are simply rewritten).
+    std::vector<int32_t> depth(n_seqs, auto_depth ? g.L : prefill_exit_layer);
+    if (auto_depth) {
+        CUDA_TRY(c, cudaMemsetAsync(c->prefill_fail, 0, sizeof(int32_t) * (size_t)g.max_seqs * (g.L + 1), c->stream));
+        if (int rc = prefill_pass(c, n_seqs, slots, tok, offsets, depth.data(), tau, true, logits_last, next_tok)) return rc;
+        std::vector<int32_t> failed((size_t)g.max_seqs * (g.L + 1));
+        CUDA_TRY(c, cudaMemcpyAsync(failed.data(), c->prefill_fail, sizeof(int32_t) * failed.size(), cudaMemcpyDeviceToHost, c->stream));
         CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        bool again = false;
+        for (int s = 0; s < n_seqs; ++s)
+            for (int l = std::max(g.entry_layer, 1); l < g.L; ++l)
+                if (!failed[(size_t)slots[s] * (g.L + 1) + l]) { depth[s] = l; again = true; break; }
+        if (depth_out) std::memcpy(depth_out, depth.data(), sizeof(int32_t) * n_seqs);
+        if (!again) return RIVER_OK;  // the first pass is the result
+        for (int s = 0; s < n_seqs; ++s) c->seq_len[slots[s]] = 0;  // the pages stay; every position is rewritten
+    } else if (depth_out) {
+        std::memcpy(depth_out, depth.data(), sizeof(int32_t) * n_seqs);
     }
-    // Rows of a chunk are consecutive prompt positions, possibly of several sequences; K/V of the whole chunk are
-    // written before its attention runs, and a row attends to positions <= its own, so causality holds inside a chunk.
-    int s = 0, p = 0;  // next (sequence, position) to schedule
-    while (s < n_seqs) {
-        int32_t *mh = next_meta(c);
-        int n = 0, n_upd = 0, n_head = 0;
-        const int tok0 = offsets[s] + p;
-        int head_seq[kMaxBatch];
-        while (s < n_seqs && n < g.max_batch) {
-            const int len = offsets[s + 1] - offsets[s];
-            if (offsets[s] + p != tok0 + n) break;  // token ids of a chunk must be contiguous in tok
-            if (int rc = ensure_page(c, slots[s], p, mh, n_upd)) return rc;
-            mh[kMetaHdr + n] = slots[s];
-            mh[kMetaHdr + g.max_batch + n] = p;
-            mh[kMetaHdr + 6 * g.max_batch + n] = c->page_tbl[(size_t)slots[s] * g.max_pages_per_seq + p / kPage];
-            if (p == len - 1) {
-                mh[kMetaHdr + 5 * g.max_batch + n_head] = n;
-                head_seq[n_head++] = s;
-            }
-            ++n;
-            if (++p == len) { c->seq_len[slots[s]] = len; ++s; p = 0; }
-        }
-        mh[0] = n; mh[1] = n_upd; mh[2] = n_head;
-        set_attn_meta(c, mh, n);
-        const bool want_logits = logits_last && n_head > 0;
-        set_io_meta(mh, tok + tok0, c->tau_i, c->forced_i, want_logits ? c->logits_i : nullptr, c->next_i, c->exit_i,
-                    nullptr);
-        if (int rc = push_meta(c, mh)) return rc;
-        c->rows_distinct = false;  // consecutive positions of one sequence share a chunk
-        const int rc_rows = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch);
-        c->rows_distinct = true;
-        if (rc_rows) return rc_rows;
-        for (int i = 0; i < n_head; ++i) {
-            if (logits_last)
-                CUDA_TRY(c, cudaMemcpyAsync(logits_last + (size_t)head_seq[i] * g.V, c->logits_i + (size_t)i * g.V,
-                                            sizeof(float) * g.V, cudaMemcpyDeviceToDevice, c->stream));
-            if (next_tok)
-                CUDA_TRY(c, cudaMemcpyAsync(next_tok + head_seq[i], c->next_i + i, sizeof(int32_t), cudaMemcpyDeviceToDevice, c->stream));
-        }
-    }
+    return prefill_pass(c, n_seqs, slots, tok, offsets, depth.data(), tau, false, logits_last, next_tok);
+}
+
+int river_clear_device_error(river_ctx *c) {
+    if (!c) return RIVER_E_BADARG;
+    CUDA_TRY(c, cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    c->st.device_error = 0;
     return RIVER_OK;
+}
+
+int river_selftest_wait_timeout(river_ctx *c, int poll_limit) {
+    if (!c) return RIVER_E_BADARG;
+    if (poll_limit < 1 || poll_limit > (1 << 20)) return fail(c, RIVER_E_BADARG, "poll_limit out of range");
+    wait_timeout_probe_kernel<<<1, 32, 0, c->stream>>>(c->dev_err, (uint32_t)poll_limit);
+    CUDA_TRY(c, cudaGetLastError());
+    int de = 0;
+    CUDA_TRY(c, cudaMemcpyAsync(&de, c->dev_err, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    return note_device_error(c, de);
 }
 
 static int kv_copy(river_ctx *c, int slot, int layer, int pos0, int n, void *k, void *v, int to_cache) {
@@ -1458,7 +940,6 @@ int river_stats(river_ctx *c, river_stats_t *out) {
     CUDA_TRY(c, cudaMemcpyAsync(nr.data(), c->n_riv, sizeof(int32_t) * (L + 1), cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(&de, c->dev_err, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-    c->st.device_error = de;
     c->st.pages_in_use = g.n_pages - (int)c->free_pages.size();
     // algorithmic bytes of the last decode step from its actual exit pattern
     double bytes = 0.0, layers_run = 0.0;
@@ -1475,8 +956,9 @@ int river_stats(river_ctx *c, river_stats_t *out) {
         c->st.layers_executed_last = layers_run / ((double)B * L);
     }
     c->st.alg_bytes_last_step = bytes;
+    const int rc = note_device_error(c, de);
     *out = c->st;
-    return de ? RIVER_E_DEVICE : RIVER_OK;
+    return rc;
 }
 
 int river_profile(river_ctx *c, int enable) {

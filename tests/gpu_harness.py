@@ -18,10 +18,10 @@ LOGIT_COS = 0.999
 KV_RTOL = 1e-2       # |a-b| <= KV_RTOL*|b| + KV_RTOL*rms(b)
 
 
-def draw_model(name: str, n_layers=None, identity: bool = False):
+def draw_model(name: str, n_layers=None, identity: bool = False, device=None):
     """Draw the model once (on the GPU when there is one: faster) and return CPU and CUDA copies of the same bits."""
     shape = synth.SHAPES[name]
-    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    dev = device or ("cuda" if torch.cuda.is_available() else "cpu")
     bb = synth.make_backbone(shape, dev, n_layers)
     if identity:
         rv = []
@@ -54,22 +54,20 @@ class StepOut:
     scores: np.ndarray
 
 
-EXTRA_FLAGS = 0  # OR-ed into every context's river_config.flags (the parity tests run under both launch plans)
-
-
 class Pair:
     """An oracle and a CUDA context over the same model, fed the same tokens."""
 
     def __init__(self, model, max_seqs: int, max_len: int, max_batch: int, exit_mode: int = 0,
-                 entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0, kv_store: int = 0):
+                 entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0, kv_store: int = 0,
+                 n_pages: Optional[int] = None):
         self.shape, (bb_c, rv_c), (bb_g, rv_g) = model
         self.L = len(bb_c["layers"])
         self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, kv_store)
         pages_per_seq = (max_len + 15) // 16
         cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
-                          n_pages=max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
+                          n_pages=n_pages or max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
                           entry_layer=entry_layer, exit_mode=exit_mode, page_shuffle_seed=page_shuffle_seed,
-                          flags=flags | EXTRA_FLAGS)
+                          flags=flags)
         self.gpu = River(cfg, bb_g, rv_g)
         self.entry = self.shape.entry_layer if entry_layer is None else entry_layer
         self.V = self.shape.V
@@ -81,6 +79,19 @@ class Pair:
         tok = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
         offs = np.concatenate([[0], np.cumsum([len(p) for p in prompts])]).tolist()
         self.gpu.prefill(slots, tok, offs, exit_layer)
+
+    def fill_history(self, lens: List[int], seed: int = 31):
+        """The same N(0,1) bf16 K/V history of lens[b] positions in slot b of both caches (an oracle prefill of long
+        prompts would take minutes)."""
+        w = self.shape.Hkv * self.shape.dh
+        for b, n in enumerate(lens):
+            for l in range(self.L):
+                k = synth.normal(seed, 1000 * b + 2 * l, (n, w), 1.0, "cuda")
+                v = synth.normal(seed, 1000 * b + 2 * l + 1, (n, w), 1.0, "cuda")
+                self.gpu.write_kv(b, l + 1, 0, k, v)
+                self.oracle.write_kv(b, l, 0, k.float().cpu().numpy(), v.float().cpu().numpy())
+            self.oracle.set_len(b, n)
+            assert self.gpu.seq_len(b) == n
 
     def gpu_step(self, slots, tok, tau, forced=None, want_logits=True) -> StepOut:
         B = len(slots)

@@ -31,16 +31,6 @@ def model(name, n_layers=None, identity=False):
     return _models[key]
 
 
-@pytest.fixture(autouse=True, params=[0, 8], ids=["stage-kernels", "chain-kernel"])
-def launch_plan(request):
-    """Every test runs twice: steps of 1-4 rows as one kernel per stage (default), and through the persistent chain
-    kernel (flag 8).  Steps of five or more rows take the same tensor-core kernels either way."""
-    import tests.gpu_harness as gh
-    gh.EXTRA_FLAGS = request.param
-    yield
-    gh.EXTRA_FLAGS = 0
-
-
 def toks(shape, n, stream):
     return synth.tokens(shape.seed, stream, n, shape.V).numpy()
 
@@ -133,13 +123,20 @@ def test_tiny_geometric_exits_and_wide_batch():
     assert r["n_early"] > r["total"] // 2
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2, 4, 5, 8, 9, 12, 32, 33, 64, 97])
+@pytest.mark.parametrize("flags", [0, 1, 32, 33])
 def test_launch_modes_agree_with_oracle(flags):
-    # 1: CUDA-graph replay; 2: no tensor-core projections; 4: plain attention kernel; 8: the persistent chain kernel
-    # (three rows per step: the chain kernel takes them when 8 is set, by the parameter or by the fixture);
-    # 32: the TMA-fed attention kernel for small steps too (default there: the kernel that fetches the cache early);
-    # 64: exit score / decision / compaction by the last CTA of the down projection instead of a kernel of its own
+    # 1: CUDA-graph replay; 32: the TMA-fed attention kernel for small steps too (default there: the kernel that
+    # fetches the cache early).  Three rows per step: the exit decisions ride in the QKV kernels.
     r = run_scheduled(model("mini8"), [37, 16, 3], 6, "uniform", page_seed=11, flags=flags, max_batch=4)
+    assert r["n_early"] > 0
+
+
+@pytest.mark.parametrize("rows", [1, 2, 4])
+def test_small_steps_every_row_count(rows):
+    # one, two and four rows per step (each its own kernel instantiation; the decision of block l is taken by the QKV
+    # kernel of block l + 1), graph replay on, mixed exit layers
+    lens = [29, 5, 18, 40][:rows]
+    r = run_scheduled(model("mini8"), lens, 8, "uniform", page_seed=3 + rows, flags=1, max_batch=4)
     assert r["n_early"] > 0
 
 
@@ -358,32 +355,19 @@ def test_8b_class_six_rows_tensor_core_paths():
     print("8b six rows:", r)
 
 
-@pytest.mark.parametrize("lens,flags", [([1024], 1), ([1024, 300, 2050, 17, 640, 1500], 1)])
-def test_8b_class_full_size_step_on_synthetic_history(lens, flags):
-    # The benchmark's own configuration - all 32 layers of the 8B shape, context ~1024, CUDA-graph replay - checked
-    # output by output: an oracle prefill of such prompts would take minutes, so both caches are filled with the same
-    # N(0,1) bf16 history through the write hook, then three scheduled steps run on both sides (one row: the
-    # small-step kernels the default bench line times; six rows of mixed lengths: the tensor-core GEMMs, the
-    # dequantising GEMM and the TMA-fed attention with several splits per row).  Logits, exit layers, scores, row lists
-    # and the K/V of every layer and position are compared as in every other test.
-    m = model("8b")
+def run_on_history(m, lens, n_steps, flags=1, exit_mode=0, max_batch=None, page_seed=9, sched_seed=23, kv_check=None):
+    """Scheduled steps on a synthetic cache history (both caches hold the same N(0,1) bf16 entries): logits, exit
+    layers, scores, row lists and the K/V of every layer and position are compared as in every other test."""
     shape = m[0]
-    B, n_steps = len(lens), 3
-    p = Pair(m, B, max(lens) + n_steps + 1, max(B, 8), page_shuffle_seed=9, kv_store=1, flags=flags)
-    w = shape.Hkv * shape.dh
-    for b, n in enumerate(lens):
-        for l in range(p.L):
-            k = synth.normal(31, 1000 * b + 2 * l, (n, w), 1.0, "cuda")
-            v = synth.normal(31, 1000 * b + 2 * l + 1, (n, w), 1.0, "cuda")
-            p.gpu.write_kv(b, l + 1, 0, k, v)
-            p.oracle.write_kv(b, l, 0, k.float().cpu().numpy(), v.float().cpu().numpy())
-        p.oracle.set_len(b, n)
-        assert p.gpu.seq_len(b) == n
+    B = len(lens)
+    p = Pair(m, B, max(lens) + n_steps + 1, max_batch or max(B, 8), page_shuffle_seed=page_seed, kv_store=1, flags=flags,
+             exit_mode=exit_mode)
+    p.fill_history(lens)
     slots = list(range(B))
     n_early = 0
     for t in range(n_steps):
         tk = toks(shape, B, 300 + t)
-        targets = synth.forced_exit_schedule(23, t, B, p.L, shape.entry_layer, "uniform").numpy()
+        targets = synth.forced_exit_schedule(sched_seed, t, B, p.L, shape.entry_layer, "uniform").numpy()
         tau, o = p.oracle_scheduled_step(slots, tk, targets)
         g = p.gpu_step(slots, tk, tau)
         assert np.array_equal(g.exit_layer, o.exit_layer), f"step {t}: exit layers {g.exit_layer} vs {o.exit_layer}"
@@ -393,25 +377,242 @@ def test_8b_class_full_size_step_on_synthetic_history(lens, flags):
         assert np.array_equal(ran, ~np.isnan(g.scores))
         assert np.abs(g.scores[ran] - o.scores[ran]).max() < NEAR
         n_early += int((o.exit_layer < p.L).sum())
-    for s_ in slots:
+    for s_ in (slots if kv_check is None else kv_check):
         p.compare_kv(s_, p.oracle.seq_len(s_))
         assert p.gpu.seq_len(s_) == p.oracle.seq_len(s_)
     assert p.gpu.stats().device_error == 0
-    assert n_early > 0
     p.close()
+    return n_early
 
 
-def test_fp32_cache_oracle_deviation_is_storage_noise():
-    # against the oracle with an fp32 cache: direction preserved (cosine bound), max-abs reported
-    m = model("8b")
+@pytest.mark.parametrize("lens", [[1024], [1024, 300, 2050, 17, 640, 1500]])
+def test_8b_class_full_size_step_on_synthetic_history(lens):
+    # The benchmark's own configuration - all 32 layers of the 8B shape, context ~1024, CUDA-graph replay - checked
+    # output by output (one row: the small-step kernels the default bench line times; six rows of mixed lengths: the
+    # tensor-core GEMMs, the dequantising GEMM and the TMA-fed attention with several splits per row).
+    assert run_on_history(model("8b"), lens, 3) > 0
+
+
+def test_8b_layer_shape_64_rows_ragged_both_weight_sets():
+    # The wide-batch configuration's geometry: the 8B layer shape (its K-splits and 64-row operand tiles in the
+    # tensor-core GEMM and in the dequantising GEMM), 64 rows with prompt lengths drawn uniformly from 256-4096 (seed 3,
+    # as the benchmark draws them), scheduled exits so that both weight sets are live in most layers.  Eight blocks of
+    # that shape instead of 32: depth does not change any kernel's geometry, and the oracle's fp32 cache of 64 x 4096
+    # positions x 32 layers would not fit in host memory.  The K/V of eight rows are compared in full.
+    lens = synth.prompt_lengths(3, 64, 256, 4096)
+    n_early = run_on_history(model("8b", 8), lens, 2, max_batch=64, kv_check=list(range(0, 64, 8)))
+    assert 8 < n_early < 120
+
+
+def test_1b_class_8_rows_context_512():
+    # the 1B configuration as stated: 16 layers, 8 rows, context 512
+    assert run_on_history(model("1b"), [512] * 8, 3, max_batch=8) > 0
+
+
+def test_batch_min_mode_on_the_tensor_core_path():
+    # Eq. 1 literally (the batch leaves together) with six rows: backbone rows on the tcgen05 GEMM, then all rows on
+    # the dequantising GEMM
+    m = model("mini8")
     shape = m[0]
-    p = Pair(m, 1, 24, 1, kv_store=0)
-    p.prefill([0], [toks(shape, 10, 100)])
-    o = p.oracle_step([0], toks(shape, 1, 200), INF)
-    g = p.gpu_step([0], toks(shape, 1, 200), INF)
-    a, w = g.logits[0].astype(np.float64), o.logits[0].astype(np.float64)
-    cos = a @ w / (np.linalg.norm(a) * np.linalg.norm(w))
-    err = np.abs(a - w).max()
-    print(f"8b vs fp32-cache oracle: cosine {cos:.6f}, max-abs {err:.4f}, logit std {w.std():.3f}")
-    assert cos >= 0.999 and err < 0.1 * w.std()
+    B = 6
+    p = Pair(m, B, 64, 8, exit_mode=1, page_shuffle_seed=2)
+    slots = list(range(B))
+    p.prefill(slots, [toks(shape, 5 + 4 * b, b) for b in range(B)])
+    seen = set()
+    lo = max(shape.entry_layer, 1)
+    for t, tau in enumerate([0.4, 0.8, 0.9, 0.95, 0.98, 0.995, 0.9995]):
+        tk = toks(shape, B, 40 + t)
+        o = p.oracle_step(slots, tk, tau)
+        g = p.gpu_step(slots, tk, tau)
+        assert len(set(o.exit_layer.tolist())) == 1
+        if np.abs(o.scores[:, lo - 1:p.L - 1] - tau).min() <= NEAR:
+            break  # a score within 1e-3 of the threshold may flip the batch's decision: histories would differ
+        assert np.array_equal(g.exit_layer, o.exit_layer)
+        p.compare_lists(B)
+        p.compare_logits(g.logits, o.logits, f"batch-min step {t}")
+        seen.add(int(o.exit_layer[0]))
+    assert len(seen) >= 2
     p.close()
+
+
+def free_tau_pass(m, prompt_lens, n_steps, frac, max_batch, kv_store=0, flags=1):
+    """One threshold for the whole run, the GPU decides: exit layers must equal the oracle's except for tokens with an
+    oracle score within 1e-3 of the threshold (counted and printed).  A row whose decision flipped has a different
+    history from then on and leaves the comparison; the other rows go on."""
+    shape = m[0]
+    B = len(prompt_lens)
+    prompts = [toks(shape, n, 100 + b) for b, n in enumerate(prompt_lens)]
+    steps = np.stack([toks(shape, B, 200 + t) for t in range(n_steps)])
+    tau = natural_tau(m, prompts, steps, frac)
+    p = Pair(m, B, max(prompt_lens) + n_steps + 1, max_batch, kv_store=kv_store, flags=flags, page_shuffle_seed=17)
+    slots = list(range(B))
+    p.prefill(slots, prompts)
+    alive = np.ones(B, bool)
+    n_cmp = n_near = n_early = 0
+    for t in range(n_steps):
+        o = p.oracle_step(slots, steps[t], tau)
+        g = p.gpu_step(slots, steps[t], tau)
+        for b in range(B):
+            if not alive[b]:
+                continue
+            n_cmp += 1
+            n_early += int(o.exit_layer[b] < p.L)
+            if g.exit_layer[b] != o.exit_layer[b]:
+                assert p.near_threshold(o.scores[b], tau, max(g.exit_layer[b], o.exit_layer[b])), \
+                    f"step {t} row {b}: exit {g.exit_layer[b]} vs {o.exit_layer[b]} with no score within 1e-3 of tau"
+                n_near += 1
+                alive[b] = False
+        if alive.any():
+            p.compare_logits(g.logits[alive], o.logits[alive], f"free step {t}")
+    print(f"free-tau pass {shape.name}: tau={tau:.5f}, {n_cmp} decisions compared, {n_early} early exits, "
+          f"{n_near} near-threshold flips")
+    p.close()
+    return n_cmp, n_early, n_near
+
+
+def test_free_tau_pass_mini8_and_1b():
+    n_cmp, n_early, n_near = free_tau_pass(model("mini8"), [21, 9, 33, 14, 5, 27], 12, 0.5, 8)
+    assert n_early > 0 and n_near <= n_cmp // 4
+    n_cmp, n_early, n_near = free_tau_pass(model("mini8"), [19], 16, 0.5, 1)
+    assert n_near <= n_cmp // 4
+    n_cmp, n_early, n_near = free_tau_pass(model("1b"), [40, 23], 6, 0.5, 8, kv_store=1)
+    assert n_near <= n_cmp // 2
+
+
+@pytest.mark.parametrize("name,prompt_len", [("1b", 40), ("8b", 12)])
+def test_bf16_cache_storage_noise_oracle_vs_oracle_and_gpu(name, prompt_len):
+    # Why the large shapes are compared with the oracle whose cache entries are rounded to bf16 (Section 4.1 keeps
+    # the KV cache in a 16-bit format): the SAME inputs through the oracle with an fp32 cache and through the oracle
+    # with bf16 storage - no kernel involved - already differ by more than the 2e-2 logit bound on these random-weight
+    # models.  The GPU, which stores bf16, must sit within the stated bound of the bf16-storage oracle, and its
+    # distance from the fp32-cache oracle may exceed the oracle-to-oracle distance by at most that bound.
+    m = model(name)
+    shape = m[0]
+    prompt, steps = toks(shape, prompt_len, 100), toks(shape, 3, 200)
+    a = Pair(m, 1, prompt_len + 8, 1, kv_store=0)
+    b = Pair(m, 1, prompt_len + 8, 1, kv_store=1)
+    a.prefill([0], [prompt])
+    b.oracle.prefill(0, prompt)
+    worst_oo = worst_g32 = worst_g16 = 0.0
+    for t in range(3):
+        oa = a.oracle_step([0], [steps[t]], INF)
+        ob = b.oracle_step([0], [steps[t]], INF)
+        g = a.gpu_step([0], [steps[t]], INF)
+        x32, x16, xg = (v.logits[0].astype(np.float64) for v in (oa, ob, g))
+        cos = lambda u, v: u @ v / (np.linalg.norm(u) * np.linalg.norm(v))
+        assert cos(x32, x16) >= 0.999 and cos(xg, x32) >= 0.999 and cos(xg, x16) >= 0.999
+        worst_oo = max(worst_oo, np.abs(x32 - x16).max())
+        worst_g32 = max(worst_g32, np.abs(xg - x32).max())
+        worst_g16 = max(worst_g16, np.abs(xg - x16).max())
+    print(f"{name}: logits max-abs  fp32-cache oracle vs bf16-cache oracle {worst_oo:.4f}   GPU vs fp32-cache oracle "
+          f"{worst_g32:.4f}   GPU vs bf16-cache oracle {worst_g16:.4f}   (logit std {x32.std():.3f})")
+    assert worst_g16 <= 2e-2
+    assert worst_oo <= 0.1 * x32.std()
+    assert worst_g32 <= worst_oo + 2e-2
+    a.close()
+    b.close()
+
+
+def test_pool_exhaustion_fails_cleanly_and_the_retry_is_exact():
+    # a step that needs more pages than are free takes none (no half-updated page table), and the same rows step
+    # correctly once pages have been released
+    from paper_2604_18396_b200 import RiverError
+    m = model("tiny")
+    shape = m[0]
+    p = Pair(m, 3, 48, 4, n_pages=4, page_shuffle_seed=8)
+    prompts = [toks(shape, 16, b) for b in range(3)]  # one full page each: every row's next token needs a new page
+    p.prefill([0, 1, 2], prompts)
+    assert p.gpu.stats().pages_in_use == 3
+    tk = toks(shape, 3, 70)
+    with pytest.raises(RiverError) as e:
+        p.gpu_step([0, 1, 2], tk, INF)  # three new pages needed, one free
+    assert e.value.code == -4
+    assert p.gpu.stats().pages_in_use == 3 and [p.gpu.seq_len(s) for s in range(3)] == [16, 16, 16]
+    p.gpu.release(2)
+    p.oracle.release(2)
+    for t in range(3):
+        tk = toks(shape, 2, 71 + t)
+        targets = synth.forced_exit_schedule(5, t, 2, shape.L, shape.entry_layer).numpy()
+        tau, o = p.oracle_scheduled_step([0, 1], tk, targets)
+        g = p.gpu_step([0, 1], tk, tau)
+        assert np.array_equal(g.exit_layer, o.exit_layer)
+        p.compare_logits(g.logits, o.logits, f"retry step {t}")
+    p.compare_kv(0, 19)
+    p.compare_kv(1, 19)
+    st = p.gpu.stats()
+    assert st.device_error == 0 and st.pages_in_use == 4
+    with pytest.raises(RiverError) as e:  # prefill: two pages needed, none free
+        p.gpu.prefill([2], torch.zeros(20, dtype=torch.int32, device="cuda"), [0, 20])
+    assert e.value.code == -4 and p.gpu.seq_len(2) == 0 and p.gpu.stats().pages_in_use == 4
+    p.close()
+
+
+def test_bounded_wait_runs_out_and_is_reported():
+    # the library's bounded mbarrier wait on a barrier nobody completes: the kernel returns, the error word says
+    # "wait ran out", the call returns RIVER_E_TIMEOUT, further steps are refused until the word is cleared
+    from paper_2604_18396_b200 import RiverError
+    m = model("tiny")
+    shape = m[0]
+    p = Pair(m, 1, 32, 1)
+    p.prefill([0], [toks(shape, 5, 0)])
+    ref = p.gpu_step([0], [3], INF)
+    assert p.gpu.selftest_wait_timeout(4000) == -7
+    assert p.gpu.stats().device_error == 4
+    with pytest.raises(RiverError) as e:
+        p.gpu_step([0], [4], INF)
+    assert e.value.code == -7 and p.gpu.seq_len(0) == 6
+    p.gpu.clear_device_error()
+    assert p.gpu.stats().device_error == 0
+    o1 = p.oracle_step([0], [3], INF)
+    o2 = p.oracle_step([0], [4], INF)
+    g2 = p.gpu_step([0], [4], INF)  # the context is usable again
+    p.compare_logits(ref.logits, o1.logits, "before the time-out")
+    p.compare_logits(g2.logits, o2.logits, "after the time-out")
+    p.close()
+
+
+@pytest.mark.parametrize("name,lens", [("tiny", [14, 3, 22]), ("mini8", [40, 9, 75, 18, 31, 6, 12])])
+def test_prefill_depth_chosen_by_the_exit_rule(name, lens):
+    # prefill_exit_layer = -1: per prompt, the first block after which every position passes Eq. 1.  Thresholds are
+    # placed between the per-block minima of the oracle's full-depth scores (never within 2.5e-3 of one), so the depth
+    # is unambiguous; depth, last-position logits and the K/V of every layer are compared with the oracle.
+    m = model(name)
+    shape = m[0]
+    B = len(lens)
+    prompts = [toks(shape, n, 300 + b) for b, n in enumerate(lens)]
+    lo = max(shape.entry_layer, 1)
+    L = shape.L
+    probe = Pair(m, 1, max(lens) + 2, 4)
+    mins = []
+    for pr in prompts:  # per-block minima over the prompt's positions, full depth
+        sc = []
+        for tk in pr:
+            sc.append(probe.oracle.decode_step([0], [tk], INF)["scores"][0])
+        probe.oracle.release(0)
+        mins.append(np.stack(sc)[:, lo - 1:L - 1].min(axis=0))
+    probe.close()
+    mins = np.stack(mins)  # [B, eligible blocks]
+    cands = sorted(set([-1.0, 2.0] + [float(0.5 * (a + b)) for a, b in zip(np.sort(mins.ravel())[:-1], np.sort(mins.ravel())[1:])]))
+    cands = [t for t in cands if np.abs(mins - t).min() > 2.5e-3]
+    picked = [cands[0], cands[len(cands) // 3], cands[2 * len(cands) // 3], cands[-1]]
+    seen = set()
+    for tau in picked:
+        p = Pair(m, B, max(lens) + 2, 8, page_shuffle_seed=4)
+        want, o_logits = [], []
+        for b, pr in enumerate(prompts):
+            lg, _, depth = p.oracle.prefill_auto(b, pr, tau)
+            want.append(depth)
+            o_logits.append(lg)
+        tok = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
+        offs = np.concatenate([[0], np.cumsum(lens)]).tolist()
+        lg_g = torch.empty((B, shape.V), dtype=torch.float32, device="cuda")
+        got = p.gpu.prefill(list(range(B)), tok, offs, -1, lg_g, None, tau)
+        torch.cuda.synchronize()
+        assert got == want, (tau, got, want)
+        p.compare_logits(lg_g.cpu().numpy(), np.stack(o_logits), f"auto prefill tau={tau}")
+        for b in range(B):
+            p.compare_kv(b, lens[b])
+        assert p.gpu.stats().device_error == 0
+        seen.update(want)
+        p.close()
+    assert len(seen) >= 2

@@ -421,3 +421,54 @@ def test_argmax_ties_and_bad_arguments(tiny):
         o.decode_step([0], [5], INF)  # sequence full
     r = o.decode_step([1], [7], INF)
     assert r["next_tok"][0] == int(np.argmax(r["logits"][0]))
+
+
+# ------------------------------------------------------------------ prefill at the depth the exit rule picks
+def test_prefill_auto_depth_matches_bruteforce_rule(tiny):
+    # Section 4.2, "Prefill Phase": one depth for the whole prompt.  The depth the oracle picks is checked against the
+    # rule applied to an independent no-cache recompute of the full-depth scores (every position of the prompt must
+    # pass s > tau at that block and at least one position must fail at every earlier eligible block), and the cache
+    # and logits it leaves behind against a recompute with every token leaving at that depth.
+    shape, bb, rv = tiny
+    prompt = _tokens(shape, 14, 7)
+    _, _, _, sc_full = bruteforce.recompute(shape, bb, rv, prompt, [shape.L] * len(prompt))
+    lo = max(shape.entry_layer, 1)
+    col_min = sc_full[:, lo - 1:shape.L - 1].min(axis=0)  # min over positions, per eligible block
+    seen = set()
+    taus = [-1.0] + [float(m) - 1e-4 for m in col_min] + [float(m) + 1e-4 for m in col_min] + [2.0]
+    for tau in taus:
+        if np.abs(col_min - tau).min() < 5e-5:
+            continue
+        want = shape.L
+        for l in range(lo, shape.L):
+            if col_min[l - lo] > tau:
+                want = l
+                break
+        o = orc.Oracle(shape, bb, rv, 1, 32)
+        logits, nxt, depth = o.prefill_auto(0, prompt, tau)
+        assert depth == want, (tau, depth, want, col_min)
+        seen.add(depth)
+        lg, K, V, _ = bruteforce.recompute(shape, bb, rv, prompt, [depth] * len(prompt))
+        assert np.abs(logits - lg[-1]).max() < 2e-4
+        for l in range(shape.L):
+            k, v = o.read_kv(0, l, 0, len(prompt))
+            assert np.abs(k - K[l]).max() < 1e-4 and np.abs(v - V[l]).max() < 1e-4
+            for pos in range(len(prompt)):
+                assert o.write_count(0, l, pos) == 1  # the second pass leaves every slot written exactly once
+        assert o.seq_len(0) == len(prompt)
+        o.close()
+    assert lo in seen and shape.L in seen and len(seen) >= 3
+
+
+def test_prefill_auto_limits(tiny):
+    shape, bb, rv = tiny
+    prompt = _tokens(shape, 9, 3)
+    a = orc.Oracle(shape, bb, rv, 1, 16)
+    b = orc.Oracle(shape, bb, rv, 1, 16)
+    la, na, depth = a.prefill_auto(0, prompt, INF)       # nothing passes: the whole backbone
+    lb, nb = b.prefill(0, prompt, shape.L)
+    assert depth == shape.L and np.array_equal(la, lb) and na == nb
+    a.release(0), b.release(0)
+    la, na, depth = a.prefill_auto(0, prompt, -2.0)      # everything passes: the entry layer
+    lb, nb = b.prefill(0, prompt, max(shape.entry_layer, 1))
+    assert depth == max(shape.entry_layer, 1) and np.array_equal(la, lb) and na == nb
