@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the early-exit decode step (one JSON line on stdout).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8b_b1|1b_b8|8b_b64|tiny] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8b_b1|1b_b8|8b_b64|tiny|attn_micro] [--impl reference]
 
 A step is one decode step of the whole hot path (embed, every block on the backbone or exit-layer weights with
 paged GQA attention, exit score, compaction, LM head) over one batch of synthetic, seeded input.  The default
@@ -437,13 +437,135 @@ def ours(args, wl):
         print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------- attention microbenchmark
+def attn_micro(args):
+    """Exit-aware decode-attention microbenchmark (8B-class GQA geometry: 32/8 heads, head dim 128, bf16 cache).
+
+    For every (context, batch, skip density) point the rows of the batch get exit layers drawn (seed 4) so that the
+    mean share of bypassed blocks equals the skip density; masks are sticky in depth.  Per block l three pieces are
+    timed with CUDA events through the library's single-stage entry points and summed over the blocks:
+      M1  attention over the compacted rows still in the backbone (river_attention on A_l),
+      M2  exit-layer K/V generation + RoPE + paged cache write for the rows that left it (river_project_kv on R_l),
+      M3  attention of those rows (river_attention on R_l): an exit layer is a whole block, so they attend too.
+    The method's total is M1 + M2 + M3; M1 + M2 alone would be a K/V-only exit path.  Prints one JSON line."""
+    import ctypes
+    import dataclasses
+    from paper_2604_18396_b200 import River, buildlib, make_config
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    buildlib.build()
+    dev = torch.device("cuda", 0)
+    peak, peak_kind = peaks()
+    shape0 = synth.SHAPES["8b"]
+    contexts = [int(x) for x in args.micro_contexts.split(",")]
+    batches = [int(x) for x in args.micro_batches.split(",")]
+    densities = [float(x) for x in args.micro_densities.split(",")]
+    pool_cap = args.micro_pool_gib * 2 ** 30
+    kv_tok_layer = 2 * shape0.Hkv * shape0.dh * 2  # bytes of K+V per token and block
+    qkv_rows = (shape0.Hq + 2 * shape0.Hkv) * shape0.dh
+    w4_qkv_bytes = qkv_rows * shape0.d * (0.5 + 4.0 / shape0.group)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    results = []
+    models = {}
+    for ctx in contexts:
+        for B in batches:
+            per_layer = B * (ctx + 16) * kv_tok_layer
+            L = int(max(1, min(shape0.L, pool_cap // per_layer)))
+            shape = dataclasses.replace(shape0, L=L)
+            if L not in models:
+                models.clear()
+                torch.cuda.empty_cache()
+                models[L] = draw_model(shape, dev)
+            bb, rvw = models[L]
+            pages_per_seq = (ctx + 15) // 16
+            cfg = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=B * pages_per_seq,
+                              max_batch=max(B, 8), page_shuffle_seed=5, flags=0)
+            rv = River(cfg, bb, rvw)
+            with torch.cuda.stream(rv.stream):
+                w = shape.Hkv * shape.dh
+                z = torch.zeros((ctx, w), dtype=torch.bfloat16, device=dev)
+                for b in range(B):
+                    rv.write_kv(b, 1, 0, z, z)  # allocates the row's pages and sets its length
+                del z
+                flat = rv.kv_pool.view(-1)
+                for i0 in range(0, flat.numel(), 1 << 30):  # N(0,1) bf16 everywhere: every block's K and V
+                    flat[i0:i0 + (1 << 30)].normal_()
+                q = torch.randn((B, shape.Hq * shape.dh), device=dev)
+                h = torch.randn((B, shape.d), device=dev)
+                out = torch.empty_like(q)
+                torch.cuda.synchronize()
+                for dens in densities:
+                    # exit layer per row: mean (L - e) / L = dens, e in [1, L]; rows with e = L never leave
+                    u = synth.uniform_int(4, int(1000 * dens) + 7 * B + ctx, B, 0, 10 ** 6).numpy() / 1e6
+                    frac_left = u ** ((1.0 - dens) / dens) if dens > 0 else np.zeros(B)  # mean dens: E[u^k] = 1 / (k + 1)
+                    depth_left = np.clip(np.round(frac_left * shape0.L), 0, shape0.L - 1)
+                    e_rel = 1.0 - depth_left / shape0.L
+                    t = {"M1": 0.0, "M2": 0.0, "M3": 0.0}
+                    by = {"M1": 0.0, "M2": 0.0, "M3": 0.0}
+                    n_riv_total = 0
+                    for rep in range(2):  # first pass warms up (launch geometry, attributes), second is timed
+                        for l in range(1, L + 1):
+                            rel = l / L
+                            riv = [b for b in range(B) if e_rel[b] < rel - 1e-9]
+                            act = [b for b in range(B) if not e_rel[b] < rel - 1e-9]
+                            pieces = (("M1", act), ("M2", riv), ("M3", riv))
+                            for name, rows in pieces:
+                                if not rows:
+                                    continue
+                                if per_layer < (256 << 20):
+                                    flush.zero_()  # the block's cache would otherwise sit in the L2 from the last pass
+                                sc = (ctypes.c_int32 * len(rows))(*rows)
+                                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                                e0.record()
+                                if name == "M2":
+                                    rv.project_kv(l, True, rows, h[:len(rows)], None, slots_c=sc)
+                                else:
+                                    rv.attention(l, rows, q[:len(rows)], out[:len(rows)], slots_c=sc)
+                                e1.record()
+                                if rep == 1:
+                                    torch.cuda.synchronize()
+                                    t[name] += e0.elapsed_time(e1) * 1e-3
+                                    by[name] += (w4_qkv_bytes + len(rows) * kv_tok_layer) if name == "M2" else \
+                                        len(rows) * ctx * kv_tok_layer
+                                    if name == "M2":
+                                        n_riv_total += len(rows)
+                    tot_t, tot_b = sum(t.values()), sum(by.values())
+                    results.append({
+                        "context": ctx, "batch": B, "skip_density": dens, "blocks": L,
+                        "achieved_skip": n_riv_total / (B * L),
+                        "us_per_block": {k: round(1e6 * v / L, 2) for k, v in t.items()},
+                        "us_per_block_sum": round(1e6 * tot_t / L, 2),
+                        "GBps": {k: (round(by[k] / t[k] / 1e9, 1) if t[k] > 0 else None) for k in t},
+                        "frac_of_peak_sum": round(tot_b / tot_t / 1e9 / peak, 4) if tot_t > 0 else None,
+                        "frac_of_peak_attention": round((by["M1"] + by["M3"]) / max(t["M1"] + t["M3"], 1e-12) / 1e9 / peak, 4),
+                    })
+                st = rv.stats()
+                assert st.device_error == 0, st.device_error
+            rv.close()
+            del rv
+            torch.cuda.empty_cache()
+    line = {"metric": "exit_aware_decode_attention", "unit": "us per block (M1 + M2 + M3)", "n_gpus": 1, "dtype": "bf16",
+            "data": "synthetic", "peak_GBps": peak, "peak_kind": peak_kind,
+            "config": {"workload": "attn_micro", "shape": "8b (32/8 heads, head dim 128, 16-token pages)",
+                       "contexts": contexts, "batches": batches, "skip_densities": densities, "seed": 4,
+                       "pool_cap_GiB": args.micro_pool_gib,
+                       "l2": "cache of a block flushed from the L2 before each timed call when it is below 256 MB",
+                       "timing": "CUDA events around each single-stage call (metadata upload + kernels)"},
+            "points": results}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="8b_b1", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="8b_b1", choices=sorted(WORKLOADS) + ["attn_micro"])
+    ap.add_argument("--micro-contexts", default="1024,8192,32768")
+    ap.add_argument("--micro-batches", default="1,16,128")
+    ap.add_argument("--micro-densities", default="0,0.2,0.4,0.6,0.8")
+    ap.add_argument("--micro-pool-gib", type=int, default=64, help="attn_micro: cap of the KV pool (fewer blocks are run when a point needs more)")
     ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")
@@ -452,7 +574,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.workload == "attn_micro":
+        attn_micro(args)
+    elif args.impl == "reference":
         reference_arm(args, args.workload)
     else:
         ours(args, args.workload)

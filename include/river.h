@@ -154,6 +154,20 @@ int river_decode_step_host(river_ctx *ctx, int batch, const int32_t *slots, cons
 int river_read_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, void *k_out, void *v_out);
 int river_write_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, const void *k_in, const void *v_in);
 
+/* Two stages of the path on their own, for kernel-level tests and the exit-aware attention microbenchmark.  Both take
+ * a compacted list of rows: row i belongs to sequence slots[i] ([host], distinct, non-empty) and sits at that
+ * sequence's LAST cached position p_i; both enqueue on the context's stream like a decode step.
+ *
+ * river_attention - step a3, paged GQA decode attention: out[i] = softmax(q[i] K^T / sqrt(dh)) V over the cached
+ *   positions 0..p_i of block `layer` (1-based);  q, out [dev] fp32 [n_rows, Hq*dh].
+ * river_project_kv - step a2: x = RMSNorm(h[i]) with the block's attention-norm gain, q, k, v = W x on the block's
+ *   bf16 weights (use_exit_layer = 0) or on its 4-bit exit-layer copy (1: the K/V generation of a bypassed block,
+ *   Section 4.1), rotary embedding at position p_i, and k, v stored (bf16) over the cache entry of position p_i - the
+ *   slot both weight sets share;  h [dev] fp32 [n_rows, d];  q_out [dev] fp32 [n_rows, Hq*dh] or NULL. */
+int river_attention(river_ctx *ctx, int layer, int n_rows, const int32_t *slots, const float *q, float *out);
+int river_project_kv(river_ctx *ctx, int layer, int use_exit_layer, int n_rows, const int32_t *slots, const float *h,
+                     float *q_out);
+
 /* Row lists of the last decode step, [host] out: act_idx / riv_idx int32 [(L+1), batch] (entry l-1: rows in the
  * backbone / in the exit layers entering block l, ascending, -1 padded; entry L: at the LM head) and their counts
  * int32 [L+1].  Synchronises the stream. */

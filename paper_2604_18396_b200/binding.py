@@ -57,7 +57,7 @@ class river_kernel_time(C.Structure):
 EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error", "river_clear_device_error",
-           "river_selftest_wait_timeout")
+           "river_selftest_wait_timeout", "river_attention", "river_project_kv")
 
 _lib = None
 
@@ -93,6 +93,8 @@ def load():
     L.river_profile.argtypes = [vp, C.c_int]
     L.river_profile_read.argtypes = [vp, C.POINTER(river_kernel_time), C.c_int, C.POINTER(C.c_int)]
     L.river_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, vp]
+    L.river_attention.argtypes = [vp, C.c_int, C.c_int, i32p, vp, vp]
+    L.river_project_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, vp]
     L.river_clear_device_error.argtypes = [vp]
     L.river_selftest_wait_timeout.argtypes = [vp, C.c_int]
     L.river_destroy.argtypes = [vp]
@@ -260,6 +262,17 @@ class River:
     def write_kv(self, slot: int, layer: int, pos0: int, k: torch.Tensor, v: torch.Tensor):
         self._order_after_current()
         self._check(load().river_write_kv(self.h, slot, layer, pos0, k.shape[0], _dp(k), _dp(v)))
+
+    def attention(self, layer: int, slots: Sequence[int], q: torch.Tensor, out: torch.Tensor, slots_c=None):
+        sc = slots_c if slots_c is not None else _i32_host(slots)
+        self._order_after_current()
+        self._check(load().river_attention(self.h, layer, len(slots), sc, _dp(q), _dp(out)))
+
+    def project_kv(self, layer: int, use_exit_layer: bool, slots: Sequence[int], h: torch.Tensor,
+                   q_out: Optional[torch.Tensor] = None, slots_c=None):
+        sc = slots_c if slots_c is not None else _i32_host(slots)
+        self._order_after_current()
+        self._check(load().river_project_kv(self.h, layer, int(use_exit_layer), len(slots), sc, _dp(h), _dp(q_out)))
 
     def last_lists(self, batch: int):
         import numpy as np

@@ -203,31 +203,77 @@ struct DecideArgs {
     const int32_t *row_slot;   // prefill pass that looks for the unified depth); row_slot maps rows to sequence slots
 };
 
-// Sums of every 32-input chunk of the rows staged in the E = 32 order (all threads of the CTA; ends with a barrier).
+// Activation rows of the exit layers as 16-bit block floating point (the A16 of the paper's W4A16, Section 4.1): every
+// 32-input chunk of a row shares one fp32 scale (max |x| / 16383), an input is a signed 15-bit integer v = 128 hi + lo
+// split into two byte digits, so that a 4-bit code times an input is an exact integer product and four of them are ONE
+// dp4a.  Per chunk c the digits sit in four 16-byte pieces [hi of code words 0-1 | hi of words 2-3 | lo of words 0-1 |
+// lo of words 2-3], a piece holding (even inputs of word a, odd inputs of word a, even of word b, odd of word b) - the
+// byte order of the isolated even / odd nibbles of a code word; piece p of the 32 chunks of a group is contiguous, so
+// a lane that owns a chunk reads its pieces with conflict-free 128-bit loads.  xsc[c] is the scale, xsum[c] = scale *
+// sum of v over the chunk (what the zero-point multiplies).  Rows are read in plain fp32 order from xs.
+__host__ __device__ inline int xq_stride16(int K) { return (((K >> 5) + 31) >> 5) * 128; }  // uint4 per row
+
 template <int N>
-__device__ __forceinline__ void stream_chunk_sums(const float *xs, float *xsum, int K, int xstride) {
+__device__ __forceinline__ void stream_quantise_rows(const float *xs, int K, int xstride, uint4 *xq, float *xsc,
+                                                     float *xsum) {
     const int tid = threadIdx.x, nthr = blockDim.x;
-    const int nch = K >> 5;
-    for (int t = tid; t < N * nch; t += nthr) {
-        const int n = t / nch, c = t % nch;
-        const float *xb = xs + n * xstride + (c >> 5) * 1024 + (c & 31) * 4;
-        float sx = 0.f;
+    const int nw = K >> 3, nch = K >> 5;  // 8-input words (four per chunk: four adjacent lanes share a chunk)
+    const int total = N * nw;
+    uint32_t *xq32 = reinterpret_cast<uint32_t *>(xq);
+    for (int u0 = 0; u0 < total; u0 += nthr) {
+        const int unit = u0 + tid;
+        const bool valid = unit < total;
+        const int n = valid ? unit / nw : 0, w = valid ? unit % nw : 0;
+        const int c = w >> 2, wd = w & 3;
+        float x[8];
+        if (valid) {
+            const float4 a = *reinterpret_cast<const float4 *>(xs + n * xstride + 8 * w);
+            const float4 b = *reinterpret_cast<const float4 *>(xs + n * xstride + 8 * w + 4);
+            x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+        } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float4 v = *reinterpret_cast<const float4 *>(xb + j * 128);
-            sx += (v.x + v.y) + (v.z + v.w);
+            for (int i = 0; i < 8; ++i) x[i] = 0.f;
         }
-        xsum[n * nch + c] = sx;
+        float m = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(x[i]));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        const float inv = m > 0.f ? 16383.f / m : 0.f;
+        int v[8], sv = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { v[i] = __float2int_rn(x[i] * inv); sv += v[i]; }
+        sv += __shfl_xor_sync(0xffffffffu, sv, 1);
+        sv += __shfl_xor_sync(0xffffffffu, sv, 2);
+        if (valid) {
+            auto pack = [](int b0, int b1, int b2, int b3) {
+                return (uint32_t)(b0 & 255) | ((uint32_t)(b1 & 255) << 8) | ((uint32_t)(b2 & 255) << 16) | ((uint32_t)(b3 & 255) << 24);
+            };
+            const uint32_t hi_e = pack(v[0] >> 7, v[2] >> 7, v[4] >> 7, v[6] >> 7), hi_o = pack(v[1] >> 7, v[3] >> 7, v[5] >> 7, v[7] >> 7);
+            const uint32_t lo_e = pack(v[0] & 127, v[2] & 127, v[4] & 127, v[6] & 127), lo_o = pack(v[1] & 127, v[3] & 127, v[5] & 127, v[7] & 127);
+            uint32_t *row = xq32 + (size_t)n * xq_stride16(K) * 4;
+            const int g = c >> 5, cl = c & 31;
+            uint32_t *ph = row + ((g * 4 + (wd >> 1)) * 32 + cl) * 4 + (wd & 1) * 2;
+            uint32_t *pl = row + ((g * 4 + 2 + (wd >> 1)) * 32 + cl) * 4 + (wd & 1) * 2;
+            *reinterpret_cast<uint2 *>(ph) = make_uint2(hi_e, hi_o);
+            *reinterpret_cast<uint2 *>(pl) = make_uint2(lo_e, lo_o);
+            if (wd == 0) {
+                const float sc = m * (1.f / 16383.f);
+                xsc[n * nch + c] = sc;
+                xsum[n * nch + c] = sc * (float)sv;
+            }
+        }
     }
     __syncthreads();
 }
 
 // ---------------------------------------------------------------- activation rows -> shared memory
 // All threads of the CTA load up to N rows idx[i0..], optionally RMS-normalise them, and store them fp32 in the
-// lane-interleaved order for E inputs per chunk (8: bf16 weights, 32: 4-bit codes, plus the sums of every chunk).
+// lane-interleaved order for E inputs per chunk (8: bf16 weights) or in plain order (E = 0: the exit-layer rows, which
+// the caller then turns into block-floating-point digits).
 template <int N, int E>
 __device__ __forceinline__ void stream_load_rows(const ProjIn &in, const int32_t *idx, int i0, int cnt, int K,
-                                                 int xstride, float *xs, float *xsum, float *red) {
+                                                 int xstride, float *xs, float *red) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     for (int n = 0; n < N; ++n) {
         float *dst = xs + n * xstride;
@@ -273,7 +319,6 @@ __device__ __forceinline__ void stream_load_rows(const ProjIn &in, const int32_t
         }
     }
     __syncthreads();
-    if (E == 32) stream_chunk_sums<N>(xs, xsum, K, xstride);
 }
 
 // ---------------------------------------------------------------- one task = R weight rows against N activation rows
@@ -336,11 +381,10 @@ __device__ __forceinline__ void stream_dots_bf16(const uint16_t *const (&wrow)[R
     }
 }
 
-// 4-bit weights: lane owns the 32-input chunks lane, lane + 32, ... (16 bytes of codes each).
-// sum_k (q_k - z) s x_k over a chunk = s * (sum_k (128 + q_k) x_k - (z + 128) * sum_k x_k): 128 + q is exact in fp32
-// as the bit pattern 0x43000000 | q << 16, which ONE byte permute builds from a word of isolated nibbles, and the
-// products go through the packed two-lane fp32 FMA, so a weight costs one permute and half an FMA issue slot; the
-// chunk sums of x are precomputed.
+// 4-bit weights: lane owns the 32-input chunks lane, lane + 32, ... (16 bytes of codes each) and multiplies them with
+// the block-floating-point digits of the activations: the even and the odd nibbles of a code word, isolated with one
+// mask each, are four byte operands of dp4a, so eight weights cost three logic operations and four integer dot
+// products (two digits), and the chunk's scale and zero-point enter once per 32 weights.
 template <int R>
 struct W4Batch {
     static constexpr int PF = R <= 2 ? kStreamPF : kStreamPF / 2;  // chunks per row in flight: 8 code loads per lane
@@ -368,65 +412,65 @@ __device__ __forceinline__ void stream_issue_w4(const W4 (&wrow)[R], int nch, in
     }
 }
 
-__device__ __forceinline__ void ffma2(float2 &acc, const float2 a, const float2 b) {
-    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%0, %1};\n\t"
-        "fma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
-        : "+f"(acc.x), "+f"(acc.y)
-        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-}
-// byte j of a word of isolated nibbles -> the fp32 value 128 + nibble
-template <int J>
-__device__ __forceinline__ float w4_byte_f32(uint32_t nib) {
-    return __uint_as_float(__byte_perm(nib, 0x43000000u, 0x7044 | (J << 8)));
+// One batch of chunks (already in registers) against the staged rows: the inner step of the pipelined passes below.
+template <int N, int R>
+__device__ __forceinline__ void stream_fma_bf16(const uint4 (&w)[R][kStreamPF], const float *xs, int xstride, int it0,
+                                                int nch, int lane, float (&acc)[R][N]) {
+#pragma unroll
+    for (int u = 0; u < kStreamPF; ++u) {
+        const int c = (it0 + u) * 32 + lane;
+        if (c < nch) {
+            const float *xb = xs + (c >> 5) * 256 + lane * 4;
+#pragma unroll
+            for (int n = 0; n < N; ++n) {
+                const float4 x0 = *reinterpret_cast<const float4 *>(xb + n * xstride);
+                const float4 x1 = *reinterpret_cast<const float4 *>(xb + n * xstride + 128);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const uint4 v = w[r][u];
+                    float a0 = bf16lo(v.x) * x0.x, a1 = bf16hi(v.x) * x0.y;
+                    a0 = fmaf(bf16lo(v.y), x0.z, a0); a1 = fmaf(bf16hi(v.y), x0.w, a1);
+                    a0 = fmaf(bf16lo(v.z), x1.x, a0); a1 = fmaf(bf16hi(v.z), x1.y, a1);
+                    a0 = fmaf(bf16lo(v.w), x1.z, a0); a1 = fmaf(bf16hi(v.w), x1.w, a1);
+                    acc[r][n] += a0 + a1;
+                }
+            }
+        }
+    }
 }
 
 template <int N, int R>
-__device__ __forceinline__ void stream_dots_w4(const W4 (&wrow)[R], const float *xs, const float *xsum, int K,
-                                               int xstride, int group, bool have_pre, const W4Batch<R> &pre,
-                                               float (&acc)[R][N]) {
-    const int lane = threadIdx.x & 31;
-    const int nch = K >> 5, nit = (nch + 31) >> 5;
-    const int gshift = (group == 64) ? 1 : (group == 32 ? 0 : 2);
+__device__ __forceinline__ void stream_fma_w4(const W4Batch<R> &b, const uint4 *xq, const float *xsc, const float *xsum,
+                                              int xqs, int it0, int nch, int lane, float (&acc)[R][N]) {
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+    for (int u = 0; u < W4Batch<R>::PF; ++u) {
+        const int c = (it0 + u) * 32 + lane;
+        if (c < nch) {
 #pragma unroll
-        for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
-    for (int it0 = 0; it0 < nit; it0 += W4Batch<R>::PF) {
-        W4Batch<R> b;
-        if (it0 == 0 && have_pre) b = pre;
-        else stream_issue_w4<R>(wrow, nch, gshift, it0, lane, b);
+            for (int n = 0; n < N; ++n) {
+                const uint4 *xb = xq + n * xqs + (c >> 5) * 128 + lane;
+                const uint4 h01 = xb[0], h23 = xb[32], l01 = xb[64], l23 = xb[96];
+                const float sc = xsc[n * nch + c], sx = xsum[n * nch + c];
 #pragma unroll
-        for (int u = 0; u < W4Batch<R>::PF; ++u) {
-            const int c = (it0 + u) * 32 + lane;
-            if (c < nch) {
-#pragma unroll
-                for (int n = 0; n < N; ++n) {
-                    const float *xb = xs + n * xstride + (c >> 5) * 1024 + lane * 4;
-                    float2 p[R];
-#pragma unroll
-                    for (int r = 0; r < R; ++r) p[r] = make_float2(0.f, 0.f);
-#pragma unroll
-                    for (int wd = 0; wd < 4; ++wd) {  // code word wd holds inputs 8*wd .. 8*wd+7 of the chunk
-                        const float4 x0 = *reinterpret_cast<const float4 *>(xb + (2 * wd) * 128);
-                        const float4 x1 = *reinterpret_cast<const float4 *>(xb + (2 * wd + 1) * 128);
-#pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            const uint4 q = b.q[r][u];
-                            const uint32_t v = wd == 0 ? q.x : (wd == 1 ? q.y : (wd == 2 ? q.z : q.w));
-                            const uint32_t e = v & 0x0f0f0f0fu;         // bytes: inputs 0, 2, 4, 6
-                            const uint32_t o = (v >> 4) & 0x0f0f0f0fu;  // bytes: inputs 1, 3, 5, 7
-                            ffma2(p[r], make_float2(w4_byte_f32<0>(e), w4_byte_f32<0>(o)), make_float2(x0.x, x0.y));
-                            ffma2(p[r], make_float2(w4_byte_f32<1>(e), w4_byte_f32<1>(o)), make_float2(x0.z, x0.w));
-                            ffma2(p[r], make_float2(w4_byte_f32<2>(e), w4_byte_f32<2>(o)), make_float2(x1.x, x1.y));
-                            ffma2(p[r], make_float2(w4_byte_f32<3>(e), w4_byte_f32<3>(o)), make_float2(x1.z, x1.w));
-                        }
-                    }
-                    const float sx = xsum[n * nch + c];
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const float s = bf16lo(b.sz[r][u]), zz = bf16hi(b.sz[r][u]) + 128.f;
-                        acc[r][n] = fmaf(s, (p[r].x + p[r].y) - zz * sx, acc[r][n]);
-                    }
+                for (int r = 0; r < R; ++r) {
+                    const uint4 q = b.q[r][u];
+                    int dh = 0, dl = 0;
+                    uint32_t e, o;
+                    e = q.x & 0x0f0f0f0fu; o = (q.x >> 4) & 0x0f0f0f0fu;  // bytes: even / odd inputs of the code word
+                    dh = __dp4a((int)e, (int)h01.x, dh); dh = __dp4a((int)o, (int)h01.y, dh);
+                    dl = __dp4a((int)e, (int)l01.x, dl); dl = __dp4a((int)o, (int)l01.y, dl);
+                    e = q.y & 0x0f0f0f0fu; o = (q.y >> 4) & 0x0f0f0f0fu;
+                    dh = __dp4a((int)e, (int)h01.z, dh); dh = __dp4a((int)o, (int)h01.w, dh);
+                    dl = __dp4a((int)e, (int)l01.z, dl); dl = __dp4a((int)o, (int)l01.w, dl);
+                    e = q.z & 0x0f0f0f0fu; o = (q.z >> 4) & 0x0f0f0f0fu;
+                    dh = __dp4a((int)e, (int)h23.x, dh); dh = __dp4a((int)o, (int)h23.y, dh);
+                    dl = __dp4a((int)e, (int)l23.x, dl); dl = __dp4a((int)o, (int)l23.y, dl);
+                    e = q.w & 0x0f0f0f0fu; o = (q.w >> 4) & 0x0f0f0f0fu;
+                    dh = __dp4a((int)e, (int)h23.z, dh); dh = __dp4a((int)o, (int)h23.w, dh);
+                    dl = __dp4a((int)e, (int)l23.z, dl); dl = __dp4a((int)o, (int)l23.w, dl);
+                    // sum_k (q_k - z) s x_k = s (scale * sum_k q_k v_k - z * scale * sum_k v_k), the integer sum exact
+                    const float s = bf16lo(b.sz[r][u]), z = bf16hi(b.sz[r][u]);
+                    acc[r][n] = fmaf(s, fmaf(sc, (float)(dh * 128 + dl), -z * sx), acc[r][n]);
                 }
             }
         }
@@ -451,36 +495,6 @@ __device__ __forceinline__ void stream_rows_w4(const P &p, int t, W4 (&rows)[R])
         const W4 b = p.template w4_base<R>(t, run);
         const size_t row = p.template run_row<R>(t, run) + j;
         rows[r] = W4{b.codes + row * (size_t)(p.K >> 1), b.scale + row * ng, b.zero + row * ng};
-    }
-}
-
-// The rest of a warp's first weight rows, and its following tasks up to `budget` bytes, requested from the L2
-// (bulk prefetch, no registers held): issued before the grid dependency resolves, so that while the predecessor
-// drains and this kernel stages its activation rows the HBM queue stays full and the first loads after the wait are
-// L2 hits.
-template <class P, int R, bool W4MODE>
-__device__ __forceinline__ void stream_l2_prefetch(const P &p, int t_first, int t1, int nwarps, int lane, int budget) {
-    const int row_bytes = W4MODE ? (p.K >> 1) : (p.K << 1);
-    int skip = min(row_bytes, (W4MODE ? W4Batch<R>::PF : kStreamPF) * 512);  // the first chunks of the first task travel in registers
-    for (int t = t_first; t < t1 && budget >= 16 * R; t += nwarps) {
-        const int per_row = min(row_bytes - skip, budget / R) & ~15;
-        if (per_row > 0) {
-            if constexpr (W4MODE) {
-                W4 rows[R];
-                stream_rows_w4<P, R>(p, t, rows);
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-                    if (lane == r) l2_prefetch(rows[r].codes + skip, per_row);
-            } else {
-                const uint16_t *rows[R];
-                stream_rows_bf16<P, R>(p, t, rows);
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-                    if (lane == r) l2_prefetch(reinterpret_cast<const uint8_t *>(rows[r]) + skip, per_row);
-            }
-        }
-        budget -= per_row * R;
-        skip = 0;
     }
 }
 
@@ -539,26 +553,61 @@ __device__ __forceinline__ void stream_publish(const DecideArgs &dec, int n, uin
 }
 
 // ---------------------------------------------------------------- the two passes over a CTA's tasks
+// A warp walks its tasks batch by batch (kStreamPF chunks of each of the R rows) with the NEXT batch's loads - the
+// same task's next chunks or the next task's first ones - issued before the current batch is multiplied, so its
+// loads are in flight during the arithmetic, the warp reduction and the epilogue of a task as well as across task
+// boundaries.  The very first batch may have been loaded before the grid dependency resolved.
 template <class P, int N, int R>
 __device__ __forceinline__ void stream_pass_bf16(const P &p, const ProjIn &in, const int32_t *act_idx, int na, int xstride,
-                                                 float *xs, float *xsum, float *red, int t0, int t1, bool prestaged,
+                                                 float *xs, float *red, int t0, int t1, bool prestaged,
                                                  bool fast, bool have_pre, uint4 (&pre)[R][kStreamPF]) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    const int K = p.K;
+    const int K = p.K, nch = K >> 3, nit = (nch + 31) >> 5;
+    constexpr bool PIPE = N * R <= 2;  // more rows: the second register set would spill
     for (int i0 = 0; i0 < na; i0 += N) {
         if (!prestaged) {
             __syncthreads();
-            stream_load_rows<N, 8>(in, act_idx, i0, na, K, xstride, xs, xsum, red);
+            stream_load_rows<N, 8>(in, act_idx, i0, na, K, xstride, xs, red);
         }
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            const uint16_t *rows[R];
-            stream_rows_bf16<P, R>(p, t, rows);
+        int t = t0 + warp;
+        if (t >= t1) continue;
+        const uint16_t *rows[R];
+        stream_rows_bf16<P, R>(p, t, rows);
+        bool loaded = have_pre && i0 == 0;  // `pre` already holds the batch that comes next
+        if constexpr (PIPE) {
+            if (!loaded) stream_issue_bf16<R>(rows, nch, 0, lane, pre);
+        }
+        for (; t < t1; t += nwarps) {
             float acc[R][N];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
             float ep[4] = {0.f, 0.f, 0.f, 0.f};
             if constexpr (N == 1 && R == 2) {
                 if (fast && lane == 0) p.epi_pre(t, 0, ep);  // travels while the dot products are computed
             }
-            stream_dots_bf16<N, R>(rows, xs, K, xstride, have_pre && i0 == 0 && t == t0 + warp, pre, acc);
+            for (int it0 = 0; it0 < nit; it0 += kStreamPF) {
+                if constexpr (PIPE) {
+                    uint4 w[R][kStreamPF];
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int u = 0; u < kStreamPF; ++u) w[r][u] = pre[r][u];
+                    if (it0 + kStreamPF < nit) {
+                        stream_issue_bf16<R>(rows, nch, it0 + kStreamPF, lane, pre);
+                    } else if (t + nwarps < t1) {
+                        const uint16_t *nrows[R];
+                        stream_rows_bf16<P, R>(p, t + nwarps, nrows);
+                        stream_issue_bf16<R>(nrows, nch, 0, lane, pre);
+                    }
+                    stream_fma_bf16<N, R>(w, xs, xstride, it0, nch, lane, acc);
+                } else {
+                    if (!loaded) stream_issue_bf16<R>(rows, nch, it0, lane, pre);
+                    loaded = false;
+                    stream_fma_bf16<N, R>(pre, xs, xstride, it0, nch, lane, acc);
+                }
+            }
 #pragma unroll
             for (int n2 = 0; n2 < N; ++n2) {
                 float res[R];
@@ -573,30 +622,66 @@ __device__ __forceinline__ void stream_pass_bf16(const P &p, const ProjIn &in, c
                     }
                 }
             }
+            if (t + nwarps < t1) stream_rows_bf16<P, R>(p, t + nwarps, rows);
         }
     }
 }
 
 template <class P, int N, int R, bool PRE>
 __device__ __forceinline__ void stream_pass_w4(const P &p, const ProjIn &in, const int32_t *riv_idx, int nr, int xstride,
-                                               float *xs, float *xsum, float *red, int t0, int t1, bool prestaged,
-                                               bool fast, const W4Batch<R> &pre) {
+                                               float *xs, uint4 *xq, float *xsc, float *xsum, float *red, int t0, int t1,
+                                               bool prestaged,
+                                               bool fast, W4Batch<R> &pre) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    const int K = p.K;
+    const int K = p.K, nch = K >> 5, nit = (nch + 31) >> 5;
+    const int gshift = (p.group == 64) ? 1 : (p.group == 32 ? 0 : 2);
+    constexpr int PF = W4Batch<R>::PF;
+    const int xqs = xq_stride16(K);
+#ifndef RIVER_W4_PIPE
+#define RIVER_W4_PIPE 0
+#endif
+    constexpr bool PIPE = RIVER_W4_PIPE && N * R <= 2;
     for (int i0 = 0; i0 < nr; i0 += N) {
         if (!prestaged) {
             __syncthreads();
-            stream_load_rows<N, 32>(in, riv_idx, i0, nr, K, xstride, xs, xsum, red);
+            stream_load_rows<N, 0>(in, riv_idx, i0, nr, K, xstride, xs, red);
+            stream_quantise_rows<N>(xs, K, xstride, xq, xsc, xsum);
         }
-        for (int t = t0 + warp; t < t1; t += nwarps) {
-            W4 rows[R];
-            stream_rows_w4<P, R>(p, t, rows);
+        int t = t0 + warp;
+        if (t >= t1) continue;
+        W4 rows[R];
+        stream_rows_w4<P, R>(p, t, rows);
+        bool loaded = PRE && i0 == 0;
+        if constexpr (PIPE) {
+            if (!loaded) stream_issue_w4<R>(rows, nch, gshift, 0, lane, pre);
+        }
+        for (; t < t1; t += nwarps) {
             float acc[R][N];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int n = 0; n < N; ++n) acc[r][n] = 0.f;
             float ep[4] = {0.f, 0.f, 0.f, 0.f};
             if constexpr (N == 1 && R == 2) {
                 if (fast && lane == 0) p.epi_pre(t, 0, ep);
             }
-            stream_dots_w4<N, R>(rows, xs, xsum, K, xstride, p.group, PRE && i0 == 0 && t == t0 + warp, pre, acc);
+            for (int it0 = 0; it0 < nit; it0 += PF) {
+                if constexpr (PIPE) {
+                    const W4Batch<R> b = pre;
+                    if (it0 + PF < nit) {
+                        stream_issue_w4<R>(rows, nch, gshift, it0 + PF, lane, pre);
+                    } else if (t + nwarps < t1) {
+                        W4 nrows[R];
+                        stream_rows_w4<P, R>(p, t + nwarps, nrows);
+                        stream_issue_w4<R>(nrows, nch, gshift, 0, lane, pre);
+                    }
+                    stream_fma_w4<N, R>(b, xq, xsc, xsum, xqs, it0, nch, lane, acc);
+                } else {
+                    if (!loaded) stream_issue_w4<R>(rows, nch, gshift, it0, lane, pre);
+                    loaded = false;
+                    stream_fma_w4<N, R>(pre, xq, xsc, xsum, xqs, it0, nch, lane, acc);
+                }
+            }
 #pragma unroll
             for (int n2 = 0; n2 < N; ++n2) {
                 float res[R];
@@ -611,19 +696,22 @@ __device__ __forceinline__ void stream_pass_w4(const P &p, const ProjIn &in, con
                     }
                 }
             }
+            if (t + nwarps < t1) stream_rows_w4<P, R>(p, t + nwarps, rows);
         }
     }
 }
 
 template <class P, int N, int R>
 __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjIn in, const RowLists rl, int has_river,
-                                                          int xstride, int skip_backbone, int pf_budget,
-                                                          const DecideArgs dec) {
+                                                          int xstride, int skip_backbone, const DecideArgs dec) {
     extern __shared__ __align__(16) float stream_smem[];
     const int K = p.K;
     float *red = stream_smem;            // 64: block reductions (up to three sums x 16 warps)
+    const int nchp = ((K >> 5) + 3) & ~3;  // keeps what follows 16-byte aligned
     float *xsum = stream_smem + 64;      // N * K/32
-    float *xs = xsum + N * (K >> 5);     // N * xstride
+    float *xsc = xsum + N * nchp;        // N * K/32
+    float *xs = xsc + N * nchp;          // N * xstride
+    uint4 *xq = reinterpret_cast<uint4 *>(xs + N * xstride);  // N * xq_stride16(K): digits of the exit-layer rows
     __shared__ int32_t s_act[4], s_riv[4];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     pdl_launch();
@@ -632,8 +720,7 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     const int t0 = (int)(((long long)tasks * blockIdx.x) / gridDim.x);
     const int t1 = (int)(((long long)tasks * (blockIdx.x + 1)) / gridDim.x);
 
-    // ---- before the grid dependency: the first loads of this warp's first task into registers and the following
-    // bytes into the L2 (weights depend on nothing).  The hint never under-counts the backbone rows: positive, the
+    // ---- before the grid dependency: the first loads of this warp's first task (weights depend on nothing).  The hint never under-counts the backbone rows: positive, the
     // bf16 set is (almost certainly) needed; zero, every row has left the backbone and the 4-bit set is.
     W4Batch<R> pre4;   // its q registers also carry the bf16 weights when that set is prefetched
     int pre_kind = 0;  // 1: pre4.q holds bf16 weights, 2: pre4 holds codes with their scales / zeros
@@ -645,13 +732,11 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
             stream_rows_bf16<P, R>(p, t0 + warp, rows);
             stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre4.q);
             pre_kind = 1;
-            if (pf_budget > 0) stream_l2_prefetch<P, R, false>(p, t0 + warp, t1, nwarps, lane, pf_budget);
         } else if (hint == 0 && has_river) {
             W4 rows[R];
             stream_rows_w4<P, R>(p, t0 + warp, rows);
             stream_issue_w4<R>(rows, K >> 5, gshift, 0, lane, pre4);
             pre_kind = 2;
-            if (pf_budget > 0) stream_l2_prefetch<P, R, true>(p, t0 + warp, t1, nwarps, lane, pf_budget / 4);
         }
     }
     // Per-step constants of the decision and the norm gain, fetched before the wait.
@@ -743,13 +828,13 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
                     y.x *= scale * bf16lo(gr[k].x); y.y *= scale * bf16hi(gr[k].x);
                     y.z *= scale * bf16lo(gr[k].y); y.w *= scale * bf16hi(gr[k].y);
                 }
-                if (riv) *reinterpret_cast<float4 *>(xs + xs_index<32>(4 * v)) = y;
+                if (riv) *reinterpret_cast<float4 *>(xs + 4 * v) = y;
                 else *reinterpret_cast<float4 *>(xs + xs_index<8>(4 * v)) = y;
             }
         }
         if (tid == 0) { s_act[0] = 0; s_riv[0] = 0; }
         __syncthreads();
-        if (riv) stream_chunk_sums<1>(xs, xsum, K, xstride);
+        if (riv) stream_quantise_rows<1>(xs, K, xstride, xq, xsc, xsum);
         na = (riv || skip_backbone) ? 0 : 1;
         nr = (riv && has_river) ? 1 : 0;
         act_idx = s_act;
@@ -830,10 +915,10 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     // that neither pass keeps the other's prefetch registers alive
     if (pre_kind == 2) {
         if (na == 0)
-            stream_pass_w4<P, N, R, true>(p, in, riv_idx, nr, xstride, xs, xsum, red, t0, t1, prestaged, fast, pre4);
+            stream_pass_w4<P, N, R, true>(p, in, riv_idx, nr, xstride, xs, xq, xsc, xsum, red, t0, t1, prestaged, fast, pre4);
     } else {
-        stream_pass_bf16<P, N, R>(p, in, act_idx, na, xstride, xs, xsum, red, t0, t1, prestaged, fast, pre_kind == 1, pre4.q);
-        stream_pass_w4<P, N, R, false>(p, in, riv_idx, nr, xstride, xs, xsum, red, t0, t1, prestaged, fast, pre4);
+        stream_pass_bf16<P, N, R>(p, in, act_idx, na, xstride, xs, red, t0, t1, prestaged, fast, pre_kind == 1, pre4.q);
+        stream_pass_w4<P, N, R, false>(p, in, riv_idx, nr, xstride, xs, xq, xsc, xsum, red, t0, t1, prestaged, fast, pre4);
     }
 }
 
@@ -852,7 +937,7 @@ struct HeadArgs {
 };
 
 template <int N, int R>
-__global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstride, int pf_budget) {
+__global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstride) {
     extern __shared__ __align__(16) float stream_smem[];
     float *red = stream_smem;
     float *xs = stream_smem + 32;
@@ -872,22 +957,13 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstr
         for (int r = 0; r < R; ++r) rows[r] = a.w + ((size_t)(t0 + warp) * R + r) * K;
         stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre);
         have_pre = true;
-        // the following bytes of this warp's rows into the L2, so that HBM keeps streaming while the last block drains
-        int budget = pf_budget, skip = min(2 * K, kStreamPF * 512);
-        for (int t = t0 + warp; t < t1 && budget >= 16 * R; t += nwarps) {
-            const int per_row = min(2 * K - skip, budget / R) & ~15;
-            if (per_row > 0 && lane < R)
-                l2_prefetch(reinterpret_cast<const uint8_t *>(a.w + ((size_t)t * R + lane) * K) + skip, per_row);
-            budget -= per_row * R;
-            skip = 0;
-        }
     }
     pdl_wait();
     const int cnt = a.meta->n_head_rows;
     float *logits = a.meta->logits;
     for (int i0 = 0; i0 < cnt; i0 += N) {
         __syncthreads();
-        stream_load_rows<N, 8>(a.in, a.rows, i0, cnt, K, xstride, xs, nullptr, red);
+        stream_load_rows<N, 8>(a.in, a.rows, i0, cnt, K, xstride, xs, red);
         float best[N];
         int besti[N];
 #pragma unroll
@@ -958,7 +1034,8 @@ static __global__ void argmax_final_kernel(const StepMeta *meta, const float *pa
 }
 
 inline size_t stream_smem_bytes(int N, int K) {
-    return sizeof(float) * (64 + (size_t)N * (K >> 5) + (size_t)N * xs_stride(K, 32));
+    return sizeof(float) * (64 + 2 * (size_t)N * (((K >> 5) + 3) & ~3) + (size_t)N * xs_stride(K, 32)) +
+           16 * (size_t)N * xq_stride16(K);
 }
 
 }  // namespace river

@@ -7,10 +7,6 @@
 
 namespace river {
 
-#ifndef RIVER_PF_BUDGET
-#define RIVER_PF_BUDGET (16 * 1024)  // bytes of weights each warp asks the L2 for before the grid dependency resolves
-#endif
-
 namespace {
 
 // Launch geometry: warps per CTA and CTAs per SM such that every warp gets the same number of tasks (a task is R
@@ -57,7 +53,7 @@ cudaError_t launch_stream_t(river_ctx *c, const P &p, const ProjIn &in, const Ro
         geom = &c->geoms.back();
     }
     return launch_k(kern, dim3(geom->grid), dim3(geom->threads), smem, c->stream, pdl, p, in, rl, has_river,
-                    xs_stride(K, 32), skip_backbone, (int)RIVER_PF_BUDGET, dec);
+                    xs_stride(K, 32), skip_backbone, dec);
 }
 
 }  // namespace
@@ -84,12 +80,11 @@ cudaError_t launch_head_stream(river_ctx *c, const HeadArgs &a, int n_head) {
     while (n_sel < n_head && n_sel < 4) n_sel *= 2;
     const int xstride = xs_stride(a.d, 8);
     const size_t smem = sizeof(float) * (32 + (size_t)n_sel * xstride);
-    const int pf = 4 * (int)RIVER_PF_BUDGET;
 #define HEAD_CASE(N_)                                                                                              \
     if (n_sel == N_) {                                                                                             \
         const cudaError_t e = ensure_smem(c, lm_head_kernel<N_, 4>, smem);                                         \
         if (e != cudaSuccess) return e;                                                                            \
-        return launch_k(lm_head_kernel<N_, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride, pf); \
+        return launch_k(lm_head_kernel<N_, 4>, dim3(c->head_grid), dim3(256), smem, c->stream, true, a, xstride); \
     }
     HEAD_CASE(1) HEAD_CASE(2) HEAD_CASE(4)
 #undef HEAD_CASE

@@ -316,6 +316,47 @@ int profile_collect(river_ctx *c) {
     return 0;
 }
 
+// a2 of block l for the n rows of the step: attention norm + QKV + RoPE + KV write, on the weight set(s) the row
+// lists name (small steps: from the exit flags).
+cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const DecideArgs &dec, double kv_write) {
+    const river_config &g = c->cfg;
+    const int d = g.d, B = g.max_batch, qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
+    const double w4f = 0.25 + 2.0 / g.group;
+    const river_layer_weights &w = c->layers[l - 1];
+    const int has_river = w.rq.codes != nullptr;
+    const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
+    const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
+    const RowLists rl{ai, na, ri, nr, c->hint_act, c->meta_dev /* StepMeta::n_rows */, c->state_at(l - 1)};
+    const bool tc = c->tc_ok && n >= 5 && n <= c->tc_max_pad;
+    const river_ctx::LayerMaps *tm = tc ? &c->tc_maps[l - 1] : nullptr;
+    const river_ctx::LayerMaps *wm = (tc && c->w4tc_ok && has_river) ? &c->w4_maps[l - 1] : nullptr;
+    const int32_t *nrh = c->n_riv + std::max(0, l - 2);  // never above the count entering this block
+    cudaError_t err = cudaSuccess;
+    auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
+    const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
+    LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
+    QkvProblem p{};
+    p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
+    p.rq = w4_of(w.rq); p.rk = w4_of(w.rk); p.rv = w4_of(w.rv);
+    p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
+    p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
+    const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
+    if (tc) {
+        TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
+        note(launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ai, na,
+                       e, true, c->hint_act));
+    }
+    if (wm) {
+        TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
+        const CUtensorMap *const cm[3] = {&wm->q, &wm->k, &wm->v};
+        const river_w4 *const cw[3] = {&w.rq, &w.rk, &w.rv};
+        note(launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ri, nr, nrh, e));
+    } else if (!tc || has_river) {
+        note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, tc ? 1 : 0, dec));
+    }
+    return err;
+}
+
 // The launch sequence of one step over the rows described in the device metadata (rows, positions, caller buffers).
 //
 // Steps of up to four rows: per block QKV, attention, O, gate/up, down - the exit decision of block l is taken by the
@@ -369,32 +410,13 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
         const int skip_bb = tc ? 1 : 0;
         // ---- a2: attention norm + QKV + RoPE + KV write (+ a6 / a7 of the previous block when the step is small)
         {
-            const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
-            LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
-            QkvProblem p{};
-            p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
-            p.rq = w4_of(w.rq); p.rk = w4_of(w.rk); p.rv = w4_of(w.rv);
-            p.K = d; p.Hq = g.Hq; p.Hkv = g.Hkv; p.dh = g.dh; p.group = g.group;
-            p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
-            const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
             DecideArgs dec{};
             if (fold && l >= 2) {
                 dec.meta = c->meta(); dec.l = l - 1; dec.L = L; dec.entry_layer = g.entry_layer; dec.exit_mode = g.exit_mode;
                 dec.h_prev = prev_in; dec.state_in = c->state_at(l - 2); dec.state_out = c->state_at(l - 1);
                 dec.lists = lists; dec.hint_act = c->hint_act; dec.fail = fail_buf; dec.row_slot = c->row_slot();
             }
-            if (tc) {
-                TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
-                note(launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM,
-                               kvdim / kTcBM, ai, na, e, true, c->hint_act));
-            }
-            if (wm) {
-                TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
-                const CUtensorMap *const cm[3] = {&wm->q, &wm->k, &wm->v};
-                const river_w4 *const cw[3] = {&w.rq, &w.rk, &w.rv};
-                note(launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ri, nr, nrh, e));
-            } else if (!tc || has_river)
-                note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, skip_bb, dec));
+            note(launch_qkv(c, l, n, h_in, dec, kv_write));
         }
         // ---- a3: paged GQA decode attention
         {
@@ -835,6 +857,79 @@ int river_prefill(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t 
         std::memcpy(depth_out, depth.data(), sizeof(int32_t) * n_seqs);
     }
     return prefill_pass(c, n_seqs, slots, tok, offsets, depth.data(), tau, false, logits_last, next_tok);
+}
+
+// Common front of the single-stage entry points: rows (slot, last cached position) into the step metadata.
+static int stage_rows(river_ctx *c, int layer, int n_rows, const int32_t *slots, int on_exit_layer) {
+    const river_config &g = c->cfg;
+    if (int rc = refuse_if_flagged(c)) return rc;
+    if (layer < 1 || layer > g.L) return fail(c, RIVER_E_BADARG, "layer out of range");
+    if (n_rows <= 0 || n_rows > g.max_batch || !slots) return fail(c, RIVER_E_BADARG, "rows out of range");
+    if (on_exit_layer && !c->layers[layer - 1].rq.codes) return fail(c, RIVER_E_BADARG, "this block has no exit-layer copy");
+    for (int b = 0; b < n_rows; ++b) {
+        if (!check_slot(c, slots[b])) return fail(c, RIVER_E_BADSLOT, "slot out of range");
+        if (c->seq_len[slots[b]] <= 0) return fail(c, RIVER_E_BADSLOT, "empty sequence");
+        for (int b2 = 0; b2 < b; ++b2)
+            if (slots[b2] == slots[b]) return fail(c, RIVER_E_BADSLOT, "a slot appears twice");
+    }
+    int32_t *mh = next_meta(c);
+    c->last_pos.resize(n_rows);
+    for (int b = 0; b < n_rows; ++b) {
+        const int pos = c->seq_len[slots[b]] - 1;
+        mh[kMetaHdr + b] = slots[b];
+        mh[kMetaHdr + g.max_batch + b] = pos;
+        mh[kMetaHdr + 6 * g.max_batch + b] = c->page_tbl[(size_t)slots[b] * g.max_pages_per_seq + pos / kPage];
+        c->last_pos[b] = pos;
+    }
+    mh[0] = n_rows; mh[1] = 0; mh[2] = 0;
+    set_attn_meta(c, mh, n_rows);
+    set_io_meta(mh, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+    if (int rc = push_meta(c, mh)) return rc;
+    Lists lists{c->act_idx, c->riv_idx, c->n_act, c->n_riv, g.max_batch};
+    stage_begin_kernel<<<n_rows, 64, 0, c->stream>>>(c->meta(), c->row_pos(), c->inv_freq, g.dh / 2, c->rope_cs,
+                                                      c->state_at(layer - 1), lists, layer - 1, on_exit_layer, c->hint_act);
+    CUDA_TRY(c, cudaGetLastError());
+    c->st.launches_total += 1;
+    return RIVER_OK;
+}
+
+int river_attention(river_ctx *c, int layer, int n_rows, const int32_t *slots, const float *q, float *out) {
+    if (!c) return RIVER_E_BADARG;
+    if (!q || !out) return fail(c, RIVER_E_BADARG, "null argument");
+    if (int rc = stage_rows(c, layer, n_rows, slots, 0)) return rc;
+    float *q_keep = c->qbuf, *o_keep = c->obuf;
+    c->qbuf = const_cast<float *>(q);
+    c->obuf = out;
+    c->st.launches_last_step = 0;
+    cudaError_t e;
+    {
+        double kv_read = 0.0;
+        for (int b = 0; b < n_rows; ++b) kv_read += (double)(c->last_pos[b] + 1) * 4.0 * c->cfg.Hkv * c->cfg.dh;
+        LaunchScope ls(c, K_ATTN, kv_read, 0, -1);
+        e = launch_attention(c, n_rows, layer - 1);
+    }
+    c->qbuf = q_keep;
+    c->obuf = o_keep;
+    if (e != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(e));
+    c->st.launches_total += c->st.launches_last_step;
+    if (c->profiling) return profile_collect(c);
+    return RIVER_OK;
+}
+
+int river_project_kv(river_ctx *c, int layer, int use_exit_layer, int n_rows, const int32_t *slots, const float *h,
+                     float *q_out) {
+    if (!c) return RIVER_E_BADARG;
+    if (!h) return fail(c, RIVER_E_BADARG, "null argument");
+    if (int rc = stage_rows(c, layer, n_rows, slots, use_exit_layer ? 1 : 0)) return rc;
+    float *q_keep = c->qbuf;
+    if (q_out) c->qbuf = q_out;
+    c->st.launches_last_step = 0;
+    const cudaError_t e = launch_qkv(c, layer, n_rows, h, DecideArgs{}, (double)n_rows * 4.0 * c->cfg.Hkv * c->cfg.dh);
+    c->qbuf = q_keep;
+    if (e != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(e));
+    c->st.launches_total += c->st.launches_last_step;
+    if (c->profiling) return profile_collect(c);
+    return RIVER_OK;
 }
 
 int river_clear_device_error(river_ctx *c) {

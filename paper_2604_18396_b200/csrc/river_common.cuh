@@ -36,19 +36,6 @@ __device__ __forceinline__ uint16_t ldg_u16(const void *p) {
     asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
     return v;
 }
-// Ask the L2 to fetch [p, p + bytes) (never a byte outside the range; 16-byte granules).
-__device__ __forceinline__ void l2_prefetch(const void *p, size_t bytes) {
-    const uintptr_t a = reinterpret_cast<uintptr_t>(p);
-    uintptr_t a0 = (a + 15) & ~(uintptr_t)15;
-    if (a0 - a >= bytes) return;
-    size_t n = (bytes - (a0 - a)) & ~(size_t)15;
-    while (n) {
-        const uint32_t c = n > 32768 ? 32768u : (uint32_t)n;
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a0), "r"(c) : "memory");
-        a0 += c;
-        n -= c;
-    }
-}
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -64,7 +51,8 @@ __device__ __forceinline__ float warp_max(float v) {
 // inputs of "chunk" c reads them with conflict-free 128-bit loads: index of input k (c = k / E, j = k % E).
 template <int E>
 __device__ __forceinline__ int xs_index(int k) {
-    const int c = k / E, j = k % E;
+    if constexpr (E == 0) return k;  // plain order
+    const int c = k / (E ? E : 1), j = k % (E ? E : 1);
     return (c >> 5) * (32 * E) + (j >> 2) * 128 + (c & 31) * 4 + (j & 3);
 }
 // KV splits per (row, KV head) of the small-step attention kernel: about one CTA per SM.

@@ -210,6 +210,32 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
     if (threadIdx.x == 0 && gridDim.x > 1) *ticket = 0;
 }
 
+// ---------------------------------------------------------------- prologue of the single-stage entry points
+// river_attention / river_project_kv run one stage of the path for a caller-given list of rows: this kernel tabulates
+// the rotary angles of the rows' positions and puts all rows on one weight set of block `l0 + 1` (exit flags, row
+// lists, counts, prefetch hint), as the step prologue and the compaction would have.
+static __global__ void stage_begin_kernel(const StepMeta *meta, const int32_t *row_pos, const double *inv_freq, int half_dh,
+                                          float2 *rope_cs, uint8_t *state, Lists lists, int l0, int on_exit_layer,
+                                          int32_t *hint_act) {
+    const int b = blockIdx.x, n = meta->n_rows;
+    if (b >= n) return;
+    const int pos = row_pos[b];
+    for (int i = threadIdx.x; i < half_dh; i += blockDim.x) {
+        double s, c;
+        sincos((double)pos * inv_freq[i], &s, &c);
+        rope_cs[(size_t)b * half_dh + i] = make_float2((float)c, (float)s);
+    }
+    if (threadIdx.x == 0) {
+        state[b] = on_exit_layer ? 1 : 0;
+        (on_exit_layer ? lists.riv_idx : lists.act_idx)[(size_t)l0 * lists.max_batch + b] = b;
+        if (b == 0) {
+            lists.n_act[l0] = on_exit_layer ? 0 : n;
+            lists.n_riv[l0] = on_exit_layer ? n : 0;
+            *hint_act = on_exit_layer ? 0 : n;
+        }
+    }
+}
+
 // ---------------------------------------------------------------- self-test of the bounded waits
 // Runs the library's bounded mbarrier wait on a barrier that nobody completes: after `limit` polls the wait gives up,
 // records DEV_WAIT_TIMEOUT in the error word and the kernel returns normally (no trap, no endless loop).

@@ -186,8 +186,9 @@ def test_identity_river_makes_exits_invisible_on_gpu():
             lg.append(g.logits[0])
         outs.append(np.stack(lg))
         p.close()
-    # same weights either way: only fp32 summation order differs between the two projection kernels
-    assert np.abs(outs[0] - outs[1]).max() < 2e-4
+    # same weights either way: what differs is the summation order and the 16-bit block-floating-point form the
+    # exit-layer kernels give their activations (the A16 of W4A16)
+    assert np.abs(outs[0] - outs[1]).max() < 1e-3
 
 
 def test_full_quant_limit_and_entry_layer_zero():
