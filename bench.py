@@ -271,7 +271,7 @@ def ours(args, wl):
     n_pages = sum((l + total_steps + 15) // 16 for l in lens)
     flags = args.flags
     cfg = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=n_pages, max_batch=max(B, 8),
-                      page_shuffle_seed=seed + 1, flags=flags)
+                      page_shuffle_seed=seed + 1, flags=flags, prefill_chunk=256)
     rv = River(cfg, bb, rvw)
     torch.cuda.synchronize()
     # everything below runs on the context's stream (its own stream when graph replay is on)

@@ -66,6 +66,9 @@ typedef struct river_config {
     int32_t exit_mode;         /* RIVER_EXIT_PER_TOKEN: Eq. 1 per row; RIVER_EXIT_BATCH_MIN: Eq. 1 literally */
     uint32_t page_shuffle_seed;/* != 0: hand pages out in a seeded shuffled order */
     uint32_t flags;
+    int32_t prefill_chunk;     /* prompt positions river_prefill runs per pass through the blocks (0 = max_batch, at most
+                                  256): every pass streams the weights once, so larger chunks make prefill cheaper; the
+                                  workspace grows with max(max_batch, prefill_chunk) */
 } river_config;
 
 typedef struct river_w4 {

@@ -552,6 +552,78 @@ __device__ __forceinline__ void stream_publish(const DecideArgs &dec, int n, uin
     *dec.hint_act = na;
 }
 
+// A step of ONE row (the latency-critical case): exit flag, the row and (when this launch decides) the previous
+// block's input are requested together - one memory round trip after the grid dependency - then Eq. 1, the decision
+// (published by CTA 0), the RMS norm, and the row in shared memory in the layout of the weight set it takes: fp32 in
+// the lane-interleaved order for the bf16 weights, block-floating-point digits for the 4-bit ones.  Returns whether
+// the row is on the exit layers.  gr: the norm gain of this thread's pieces, fetched before the wait.
+template <int XF>
+__device__ __forceinline__ bool stream_stage_one(const ProjIn &in, const DecideArgs &dec, const uint8_t *state, int K,
+                                                 int xstride, float *red, float *xs, uint4 *xq, float *xsc, float *xsum,
+                                                 const uint2 (&gr)[XF], float tau0, int forced0) {
+    const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarps = nthr >> 5;
+    const int nv = K >> 2;
+    const uint8_t flag_in = __ldcg(state);
+    float4 xr[XF];
+    float bb = 0.f, ab = 0.f, aa = 0.f;
+    const float4 *src = reinterpret_cast<const float4 *>(in.src);
+#pragma unroll
+    for (int k = 0; k < XF; ++k) {
+        const int v = tid + k * nthr;
+        xr[k] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (dec.meta) {
+        const float4 *prv = reinterpret_cast<const float4 *>(dec.h_prev);
+        float4 xp[XF];
+#pragma unroll
+        for (int k = 0; k < XF; ++k) {
+            const int v = tid + k * nthr;
+            xp[k] = v < nv ? __ldcg(prv + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < XF; ++k) {
+            ab += xp[k].x * xr[k].x + xp[k].y * xr[k].y + xp[k].z * xr[k].z + xp[k].w * xr[k].w;
+            aa += xp[k].x * xp[k].x + xp[k].y * xp[k].y + xp[k].z * xp[k].z + xp[k].w * xp[k].w;
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < XF; ++k) bb += xr[k].x * xr[k].x + xr[k].y * xr[k].y + xr[k].z * xr[k].z + xr[k].w * xr[k].w;
+    bool riv = flag_in != 0;
+    if (in.gain || dec.meta) {
+        bb = warp_sum(bb);
+        if (dec.meta) { ab = warp_sum(ab); aa = warp_sum(aa); }
+        if (lane == 0) { red[warp] = bb; red[16 + warp] = ab; red[32 + warp] = aa; }
+        __syncthreads();
+        bb = ab = aa = 0.f;
+        for (int w = 0; w < nwarps; ++w) { bb += red[w]; ab += red[16 + w]; aa += red[32 + w]; }
+    }
+    if (dec.meta) {
+        const float sc[1] = {transition_score(ab, aa, bb)}, tau[1] = {tau0};
+        const int forced[1] = {forced0};
+        const uint32_t gone_in = flag_in ? 1u : 0u;
+        const uint32_t gone = stream_decide<1>(dec, 1, gone_in, sc, tau, forced);
+        if (blockIdx.x == 0 && tid == 0) stream_publish<1>(dec, 1, gone_in, gone, sc, tau);
+        riv = gone != 0;
+    }
+    const float scale = in.gain ? rsqrtf(bb / (float)K + in.eps) : 1.f;
+#pragma unroll
+    for (int k = 0; k < XF; ++k) {
+        const int v = tid + k * nthr;
+        if (v < nv) {
+            float4 y = xr[k];
+            if (in.gain) {
+                y.x *= scale * bf16lo(gr[k].x); y.y *= scale * bf16hi(gr[k].x);
+                y.z *= scale * bf16lo(gr[k].y); y.w *= scale * bf16hi(gr[k].y);
+            }
+            if (riv) *reinterpret_cast<float4 *>(xs + 4 * v) = y;
+            else *reinterpret_cast<float4 *>(xs + xs_index<8>(4 * v)) = y;
+        }
+    }
+    __syncthreads();
+    if (riv) stream_quantise_rows<1>(xs, K, xstride, xq, xsc, xsum);
+    return riv;
+}
+
 // ---------------------------------------------------------------- the two passes over a CTA's tasks
 // A warp walks its tasks batch by batch (kStreamPF chunks of each of the R rows) with the NEXT batch's loads - the
 // same task's next chunks or the next task's first ones - issued before the current batch is multiplied, so its
@@ -637,10 +709,7 @@ __device__ __forceinline__ void stream_pass_w4(const P &p, const ProjIn &in, con
     const int gshift = (p.group == 64) ? 1 : (p.group == 32 ? 0 : 2);
     constexpr int PF = W4Batch<R>::PF;
     const int xqs = xq_stride16(K);
-#ifndef RIVER_W4_PIPE
-#define RIVER_W4_PIPE 0
-#endif
-    constexpr bool PIPE = RIVER_W4_PIPE && N * R <= 2;
+    constexpr bool PIPE = false;  // measured: issuing the next batch early makes the 4-bit pass slower, not faster
     for (int i0 = 0; i0 < nr; i0 += N) {
         if (!prestaged) {
             __syncthreads();
@@ -772,69 +841,10 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     bool prestaged = false;
     const int32_t *act_idx = rl.act_idx, *riv_idx = rl.riv_idx;
     if (fast) {
-        // ---- a step of ONE row (the latency-critical case): exit flag, the row and (when this launch decides) the
-        // previous block's input are requested together - one memory round trip after the grid dependency.
-        const uint8_t flag_in = dec.meta ? __ldcg(dec.state_in) : __ldcg(rl.state);
-        float4 xr[XF];
-        float bb = 0.f, ab = 0.f, aa = 0.f;
-        const float4 *src = reinterpret_cast<const float4 *>(in.src);
-#pragma unroll
-        for (int k = 0; k < XF; ++k) {
-            const int v = tid + k * nthr;
-            xr[k] = v < nv ? __ldcg(src + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (dec.meta) {
-            const float4 *prv = reinterpret_cast<const float4 *>(dec.h_prev);
-            float4 xp[XF];
-#pragma unroll
-            for (int k = 0; k < XF; ++k) {
-                const int v = tid + k * nthr;
-                xp[k] = v < nv ? __ldcg(prv + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int k = 0; k < XF; ++k) {
-                ab += xp[k].x * xr[k].x + xp[k].y * xr[k].y + xp[k].z * xr[k].z + xp[k].w * xr[k].w;
-                aa += xp[k].x * xp[k].x + xp[k].y * xp[k].y + xp[k].z * xp[k].z + xp[k].w * xp[k].w;
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < XF; ++k) bb += xr[k].x * xr[k].x + xr[k].y * xr[k].y + xr[k].z * xr[k].z + xr[k].w * xr[k].w;
-        bool riv = flag_in != 0;
-        if (in.gain || dec.meta) {
-            bb = warp_sum(bb);
-            if (dec.meta) { ab = warp_sum(ab); aa = warp_sum(aa); }
-            if (lane == 0) { red[warp] = bb; red[16 + warp] = ab; red[32 + warp] = aa; }
-            __syncthreads();
-            bb = ab = aa = 0.f;
-            for (int w = 0; w < nwarps; ++w) { bb += red[w]; ab += red[16 + w]; aa += red[32 + w]; }
-        }
-        if (dec.meta) {
-            float sc[N];
-#pragma unroll
-            for (int b = 0; b < N; ++b) sc[b] = 0.f;
-            sc[0] = transition_score(ab, aa, bb);
-            const uint32_t gone_in = flag_in ? 1u : 0u;
-            const uint32_t gone = stream_decide<N>(dec, 1, gone_in, sc, tau, forced);
-            if (blockIdx.x == 0 && tid == 0) stream_publish<N>(dec, 1, gone_in, gone, sc, tau);
-            riv = gone != 0;
-        }
-        const float scale = in.gain ? rsqrtf(bb / (float)K + in.eps) : 1.f;
-#pragma unroll
-        for (int k = 0; k < XF; ++k) {
-            const int v = tid + k * nthr;
-            if (v < nv) {
-                float4 y = xr[k];
-                if (in.gain) {
-                    y.x *= scale * bf16lo(gr[k].x); y.y *= scale * bf16hi(gr[k].x);
-                    y.z *= scale * bf16lo(gr[k].y); y.w *= scale * bf16hi(gr[k].y);
-                }
-                if (riv) *reinterpret_cast<float4 *>(xs + 4 * v) = y;
-                else *reinterpret_cast<float4 *>(xs + xs_index<8>(4 * v)) = y;
-            }
-        }
+        const bool riv = stream_stage_one<XF>(in, dec, dec.meta ? dec.state_in : rl.state, K, xstride, red, xs, xq, xsc, xsum,
+                                              gr, tau[0], forced[0]);
         if (tid == 0) { s_act[0] = 0; s_riv[0] = 0; }
         __syncthreads();
-        if (riv) stream_quantise_rows<1>(xs, K, xstride, xq, xsc, xsum);
         na = (riv || skip_backbone) ? 0 : 1;
         nr = (riv && has_river) ? 1 : 0;
         act_idx = s_act;

@@ -68,6 +68,7 @@ const char *check_config(const river_config *c) {
     if (c->page_size != kPage) return "page_size must be 16";
     if (c->entry_layer < 0 || c->entry_layer >= c->L) return "entry_layer out of range";
     if (c->max_batch <= 0 || c->max_batch > kMaxBatch) return "max_batch out of range";
+    if (c->prefill_chunk < 0 || c->prefill_chunk > 256) return "prefill_chunk out of range (0 .. 256)";
     if (c->max_seqs <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return "bad cache geometry";
     if (!(c->exit_mode == RIVER_EXIT_PER_TOKEN || c->exit_mode == RIVER_EXIT_BATCH_MIN)) return "bad exit_mode";
     return nullptr;
@@ -76,7 +77,16 @@ const char *check_config(const river_config *c) {
 int head_grid_for(const river_config *c) { return 148 * 2 > c->V / 4 ? std::max(1, c->V / 4) : 148 * 2; }
 int head_parts_for(const river_config *c) { return std::max(head_grid_for(c), c->V / 128 + 1); }  // argmax partials per row
 
-size_t carve(const river_config *c, river_ctx *x, char *base) {
+// Row-indexed buffers are sized for the larger of a decode step and a prefill chunk; the logits staging only for the
+// rows that can need logits at once (a decode step's rows, or as many prompt ends in a chunk).
+river_config effective(const river_config *cfg, int *user_max_batch) {
+    river_config e = *cfg;
+    if (user_max_batch) *user_max_batch = cfg->max_batch;
+    e.max_batch = std::max(cfg->max_batch, cfg->prefill_chunk);
+    return e;
+}
+
+size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     Carver cv{base};
     const size_t B = c->max_batch, d = c->d, L = c->L;
     float *h0 = cv.take<float>(B * d), *h1 = cv.take<float>(B * d), *h2 = cv.take<float>(B * d);
@@ -85,7 +95,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base) {
     float *pv = cv.take<float>(B * (size_t)head_parts_for(c));
     int32_t *pi = cv.take<int32_t>(B * (size_t)head_parts_for(c));
     float *tau = cv.take<float>(B);
-    float *lg = cv.take<float>(B * (size_t)c->V);
+    float *lg = cv.take<float>((size_t)head_rows * (size_t)c->V);
     float *sc = cv.take<float>(B * L);
     float2 *cs = cv.take<float2>(B * (c->dh / 2));
     double *fr = cv.take<double>(c->dh / 2);
@@ -595,7 +605,7 @@ int prefill_pass(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t *
         int n = 0, n_upd = 0, n_head = 0;
         const int tok0 = offsets[s] + p;
         int head_seq[kMaxBatch];
-        while (s < n_seqs && n < g.max_batch) {
+        while (s < n_seqs && n < g.max_batch && n_head < c->user_max_batch) {
             const int len = offsets[s + 1] - offsets[s];
             if (offsets[s] + p != tok0 + n) break;  // token ids of a chunk must be contiguous in tok
             if (int rc = ensure_page(c, slots[s], p, mh, n_upd)) { rollback_pages(c, mh, n_upd); return rc; }
@@ -639,7 +649,9 @@ extern "C" {
 
 size_t river_workspace_bytes(const river_config *cfg) {
     if (check_config(cfg)) return 0;
-    return carve(cfg, nullptr, nullptr);
+    int mb = 0;
+    const river_config e = effective(cfg, &mb);
+    return carve(&e, nullptr, nullptr, mb);
 }
 
 size_t river_kv_pool_bytes(const river_config *cfg) {
@@ -669,7 +681,8 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
             return fail(nullptr, RIVER_E_BADARG, "layer " + std::to_string(l + 1) + " is above entry_layer but has no exit-layer copy");
     }
     river_ctx *c = new river_ctx();
-    c->cfg = *cfg;
+    c->cfg = effective(cfg, &c->user_max_batch);
+    cfg = &c->cfg;  // from here on max_batch means rows per launch sequence (a decode step or a prefill chunk)
     c->layers.assign(w->layers, w->layers + cfg->L);
     c->embed = (const uint16_t *)w->embed;
     c->lm_head = (const uint16_t *)w->lm_head;
@@ -680,7 +693,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
         return fail(nullptr, RIVER_E_BADARG, "RIVER_F_GRAPH needs a stream other than the default stream");
     }
     c->pool = (__nv_bfloat16 *)kv_pool;
-    c->ws_bytes = carve(cfg, c, (char *)workspace);
+    c->ws_bytes = carve(cfg, c, (char *)workspace, c->user_max_batch);
     c->head_grid = head_grid_for(cfg);
     auto bail = [&](const std::string &m) {
         g_init_error = m;
@@ -738,7 +751,7 @@ int river_decode_step(river_ctx *c, int batch, const int32_t *slots, const int32
     if (!c) return RIVER_E_BADARG;
     const river_config &g = c->cfg;
     if (int rc = refuse_if_flagged(c)) return rc;
-    if (batch <= 0 || batch > g.max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
+    if (batch <= 0 || batch > c->user_max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
     if (!slots || !tok || !tau || !next_tok || !exit_layer) return fail(c, RIVER_E_BADARG, "null argument");
     // everything that can fail is checked before any page is taken: slots, lengths, and the pages the whole batch needs
     int new_pages = 0;
@@ -779,7 +792,7 @@ int river_decode_step_host(river_ctx *c, int batch, const int32_t *slots, const 
                            float *scores) {
     if (!c) return RIVER_E_BADARG;
     const river_config &g = c->cfg;
-    if (batch <= 0 || batch > g.max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
+    if (batch <= 0 || batch > c->user_max_batch) return fail(c, RIVER_E_BADARG, "batch out of range");
     if (!slots || !tok || !tau || !next_tok || !exit_layer) return fail(c, RIVER_E_BADARG, "null argument");
     if (forced_exit)
         for (int b = 0; b < batch; ++b)
@@ -864,7 +877,7 @@ static int stage_rows(river_ctx *c, int layer, int n_rows, const int32_t *slots,
     const river_config &g = c->cfg;
     if (int rc = refuse_if_flagged(c)) return rc;
     if (layer < 1 || layer > g.L) return fail(c, RIVER_E_BADARG, "layer out of range");
-    if (n_rows <= 0 || n_rows > g.max_batch || !slots) return fail(c, RIVER_E_BADARG, "rows out of range");
+    if (n_rows <= 0 || n_rows > c->user_max_batch || !slots) return fail(c, RIVER_E_BADARG, "rows out of range");
     if (on_exit_layer && !c->layers[layer - 1].rq.codes) return fail(c, RIVER_E_BADARG, "this block has no exit-layer copy");
     for (int b = 0; b < n_rows; ++b) {
         if (!check_slot(c, slots[b])) return fail(c, RIVER_E_BADSLOT, "slot out of range");

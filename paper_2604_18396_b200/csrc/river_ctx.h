@@ -17,7 +17,8 @@ constexpr int kStaging = 4;  // pinned metadata buffers in flight
 enum KernelClass { K_BEGIN, K_QKV, K_ATTN, K_OPROJ, K_GATEUP, K_DOWN, K_SCORE, K_HEAD, K_ARGMAX, K_PREFILL_ATTN, kNumClasses };
 
 struct river_ctx {
-    river_config cfg;
+    river_config cfg;        // as given, except max_batch = max(max_batch, prefill_chunk): rows per launch sequence
+    int user_max_batch = 0;  // rows per decode step the caller asked for
     std::vector<river_layer_weights> layers;
     const uint16_t *embed, *lm_head, *final_norm;
     cudaStream_t stream;

@@ -59,7 +59,7 @@ class Pair:
 
     def __init__(self, model, max_seqs: int, max_len: int, max_batch: int, exit_mode: int = 0,
                  entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0, kv_store: int = 0,
-                 n_pages: Optional[int] = None):
+                 n_pages: Optional[int] = None, prefill_chunk: int = 0):
         self.shape, (bb_c, rv_c), (bb_g, rv_g) = model
         self.L = len(bb_c["layers"])
         self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, kv_store)
@@ -67,7 +67,7 @@ class Pair:
         cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
                           n_pages=n_pages or max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
                           entry_layer=entry_layer, exit_mode=exit_mode, page_shuffle_seed=page_shuffle_seed,
-                          flags=flags)
+                          flags=flags, prefill_chunk=prefill_chunk)
         self.gpu = River(cfg, bb_g, rv_g)
         self.entry = self.shape.entry_layer if entry_layer is None else entry_layer
         self.V = self.shape.V

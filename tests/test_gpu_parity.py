@@ -572,6 +572,41 @@ def test_bounded_wait_runs_out_and_is_reported():
     p.close()
 
 
+@pytest.mark.parametrize("depth", [None, 2])
+def test_prefill_in_chunks_of_256_positions(depth):
+    # prefill_chunk = 256 with max_batch = 4: prompt positions go through the blocks 256 at a time (tensor-core GEMMs
+    # with 256-row operand tiles, TMA-fed attention over rows of one sequence at consecutive positions), chunks that
+    # hold the end of one prompt and the start of the next, a prompt of one token, and more prompt ends in a chunk
+    # than the logits staging has rows for (max_batch).  Last-position logits, every cached K/V and two decode steps
+    # afterwards are compared with the oracle.
+    m = model("mini8")
+    shape = m[0]
+    lens = [300, 70, 1, 513, 2, 3, 1, 1, 5, 140]
+    B = len(lens)
+    p = Pair(m, B, max(lens) + 4, 4, page_shuffle_seed=6, prefill_chunk=256, kv_store=1)
+    prompts = [toks(shape, n, 400 + b) for b, n in enumerate(lens)]
+    o_logits = np.stack([p.oracle.prefill(b, pr, depth)[0] for b, pr in enumerate(prompts)])
+    tok = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
+    offs = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    lg = torch.empty((B, shape.V), dtype=torch.float32, device="cuda")
+    nx = torch.empty(B, dtype=torch.int32, device="cuda")
+    p.gpu.prefill(list(range(B)), tok, offs, depth, lg, nx)
+    torch.cuda.synchronize()
+    p.compare_logits(lg.cpu().numpy(), o_logits, "chunked prefill")
+    for b in range(B):
+        p.compare_kv(b, lens[b])
+    for t in range(2):
+        sl = [0, 3, 9, 2]
+        tk = toks(shape, 4, 500 + t)
+        targets = synth.forced_exit_schedule(7, t, 4, p.L, shape.entry_layer).numpy()
+        tau, o = p.oracle_scheduled_step(sl, tk, targets)
+        g = p.gpu_step(sl, tk, tau)
+        assert np.array_equal(g.exit_layer, o.exit_layer)
+        p.compare_logits(g.logits, o.logits, f"step {t} after chunked prefill")
+    assert p.gpu.stats().device_error == 0
+    p.close()
+
+
 @pytest.mark.parametrize("name,lens", [("tiny", [14, 3, 22]), ("mini8", [40, 9, 75, 18, 31, 6, 12])])
 def test_prefill_depth_chosen_by_the_exit_rule(name, lens):
     # prefill_exit_layer = -1: per prompt, the first block after which every position passes Eq. 1.  Thresholds are
