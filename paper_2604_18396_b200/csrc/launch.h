@@ -17,5 +17,7 @@ cudaError_t launch_argmax_final(river_ctx *c, int n_head, int n_parts);
 
 // launch_attn.cu: paged GQA decode attention (TMA-fed split-KV kernel; small-step kernel for 1-4 rows)
 cudaError_t launch_attention(river_ctx *c, int n, int layer0);
+bool prefill_attn_supported(const river_ctx *c);
+cudaError_t launch_attention_prefill(river_ctx *c, int n, int layer0);  // tensor-core causal attention of a prefill chunk
 
 }  // namespace river

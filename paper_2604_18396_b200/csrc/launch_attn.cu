@@ -6,6 +6,7 @@
 #include "launch.h"
 #include "attn_decode.cuh"
 #include "attn_small.cuh"
+#include "attn_prefill.cuh"
 
 namespace river {
 
@@ -45,6 +46,36 @@ cudaError_t launch_attn_small(river_ctx *c, int n, int layer0, int early) {
 }
 
 }  // namespace
+
+bool prefill_attn_supported(const river_ctx *c) {
+    const int gq = c->cfg.Hq / c->cfg.Hkv;
+    return (c->cfg.dh == 64 || c->cfg.dh == 128) && (gq == 1 || gq == 2 || gq == 4 || gq == 8);
+}
+
+namespace {
+template <int DH, int GQ>
+cudaError_t launch_attn_prefill_t(river_ctx *c, int n, int layer0) {
+    const river_config &g = c->cfg;
+    PrefillAttnArgs a{};
+    a.meta = c->meta(); a.tile_row0 = c->tile_row0(); a.tile_rows = c->tile_rows();
+    a.q = c->qbuf; a.out = c->obuf; a.kv = kv_addr(c, layer0); a.Hq = g.Hq;
+    a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
+    a.dev_err = c->dev_err;
+    const size_t smem = attn_prefill_smem_bytes(DH);
+    const cudaError_t e = ensure_smem(c, attn_prefill_kernel<DH, GQ>, smem);
+    if (e != cudaSuccess) return e;
+    // at most one tile per row; the kernel reads the tile count of the chunk from the step metadata
+    return launch_k(attn_prefill_kernel<DH, GQ>, dim3(n, g.Hkv), dim3(32 * GQ), smem, c->stream, true, a);
+}
+}  // namespace
+
+cudaError_t launch_attention_prefill(river_ctx *c, int n, int layer0) {
+    const int gq = c->cfg.Hq / c->cfg.Hkv;
+#define ATTP(DH_, GQ_) if (c->cfg.dh == DH_ && gq == GQ_) return launch_attn_prefill_t<DH_, GQ_>(c, n, layer0);
+    ATTP(64, 1) ATTP(64, 2) ATTP(64, 4) ATTP(64, 8) ATTP(128, 1) ATTP(128, 2) ATTP(128, 4) ATTP(128, 8)
+#undef ATTP
+    return cudaErrorInvalidValue;
+}
 
 cudaError_t launch_attention(river_ctx *c, int n, int layer0) {
     const int gq = c->cfg.Hq / c->cfg.Hkv;

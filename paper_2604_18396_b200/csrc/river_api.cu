@@ -16,6 +16,7 @@
 #include "river_kernels.cuh"
 #include "attn_decode.cuh"
 #include "attn_small.cuh"
+#include "attn_prefill.cuh"
 
 using namespace river;
 
@@ -103,7 +104,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     int32_t *na = cv.take<int32_t>(L + 1), *nr = cv.take<int32_t>(L + 1);
     int32_t *pt = cv.take<int32_t>((size_t)c->max_seqs * c->max_pages_per_seq);
     int32_t *tk = cv.take<int32_t>(B), *fo = cv.take<int32_t>(B), *ex = cv.take<int32_t>(B), *nx = cv.take<int32_t>(B);
-    int32_t *md = cv.take<int32_t>(kMetaHdr + 8 * B);
+    int32_t *md = cv.take<int32_t>(kMetaHdr + 10 * B);
     int32_t *pff = cv.take<int32_t>((size_t)c->max_seqs * (L + 1));
     float *po = cv.take<float>((B + 600) * (size_t)c->Hq * c->dh);
     float2 *pml = cv.take<float2>((B + 600) * (size_t)c->Hq);
@@ -429,7 +430,10 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
             note(launch_qkv(c, l, n, h_in, dec, kv_write));
         }
         // ---- a3: paged GQA decode attention
-        {
+        if (c->prefill_attn_now) {
+            LaunchScope ls(c, K_PREFILL_ATTN, kv_read, 0, -1);
+            note(launch_attention_prefill(c, n, l - 1));
+        } else {
             LaunchScope ls(c, K_ATTN, kv_read, 0, -1);
             note(launch_attention(c, n, l - 1));
         }
@@ -622,6 +626,20 @@ int prefill_pass(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t *
         }
         mh[0] = n; mh[1] = n_upd; mh[2] = n_head;
         set_attn_meta(c, mh, n);
+        // query tiles for the tensor-core prefill attention: up to 16 consecutive positions of one sequence each
+        int n_tiles = 0;
+        for (int i = 0; i < n;) {
+            int j = i + 1;
+            while (j < n && j - i < kPfBM && mh[kMetaHdr + j] == mh[kMetaHdr + i] &&
+                   mh[kMetaHdr + g.max_batch + j] == mh[kMetaHdr + g.max_batch + i] + (j - i))
+                ++j;
+            mh[kMetaHdr + 8 * g.max_batch + n_tiles] = i;
+            mh[kMetaHdr + 9 * g.max_batch + n_tiles] = j - i;
+            ++n_tiles;
+            i = j;
+        }
+        reinterpret_cast<StepMeta *>(mh)->pad2[0] = n_tiles;
+        c->prefill_attn_now = n >= 5 && prefill_attn_supported(c);
         const bool want_logits = logits_last && n_head > 0;
         set_io_meta(mh, tok + tok0, c->tau_i, c->row_forced(), want_logits ? c->logits_i : nullptr, c->next_i, c->exit_i,
                     nullptr);
@@ -629,6 +647,7 @@ int prefill_pass(river_ctx *c, int n_seqs, const int32_t *slots, const int32_t *
         c->rows_distinct = false;  // consecutive positions of one sequence share a chunk
         const int rc_rows = run_rows(c, n, n_head, mh + kMetaHdr + g.max_batch, record_fail);
         c->rows_distinct = true;
+        c->prefill_attn_now = false;
         if (rc_rows) return rc_rows;
         for (int i = 0; i < n_head; ++i) {
             if (logits_last)

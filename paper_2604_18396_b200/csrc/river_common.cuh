@@ -70,7 +70,8 @@ struct StepMeta {  // device-resident, rewritten by the host before every step
     int32_t attn_chunk;   // positions per KV split of the attention kernel (multiple of 64)
     int32_t attn_splits;  // split slots per (row, head) in the partial buffers
     int32_t hint_act;     // rows still in the backbone as of the latest compaction (reset to n_rows by the host)
-    int32_t pad[2];
+    int32_t pad[2];       // small-step attention: positions per split, splits per (row, KV head)
+    int32_t pad2[2];      // [0]: query tiles of a prefill chunk (attn_prefill_kernel)
     // the caller's device buffers of this step (read through here so that a captured launch sequence never changes)
     const int32_t *tok;
     const float *tau;
