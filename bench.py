@@ -128,8 +128,8 @@ def draw_model(shape, device):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised under
 # profiles/ (taken on a 4-layer model of the same layer shape: kernel, geometry and operands per launch are those of
-# the full model).  None: no capture of the current kernel is on file.
-NCU_TRAFFIC = {}
+# the full model).  Missing key: no capture of that kernel is on file (traffic is then reported as null).
+NCU_TRAFFIC = {("8b", "gateup_swiglu"): 235068160.0}  # profiles/stream_proj_kernel_8b4L_b1.md
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle timing
