@@ -219,6 +219,17 @@ int river_clear_device_error(river_ctx *ctx);
  * the call synchronises and returns RIVER_E_TIMEOUT (the expected outcome), leaving the error word set. */
 int river_selftest_wait_timeout(river_ctx *ctx, int poll_limit);
 
+/* The exit layers' weights from the backbone's (Section 4.1: an exit layer is a copy of its backbone block whose
+ * Attention and FFN matrices go through a training-free 4-bit weight-only quantisation with a refined zero-point).
+ *   w [dev] bf16 row-major [out, in], 16-byte aligned;  group in {32, 64, 128} dividing `in`;
+ *   refine_iters: rounds of the half-quadratic zero-point refinement (0 = plain min/max round-to-nearest grid; 20 is
+ *       the published default);
+ *   codes [dev] u8 [out, in/2] (low nibble = even input), scale / zero [dev] bf16 [out, in/group]: the layout
+ *       river_init takes.  No context needed; asynchronous on cuda_stream.  Returns RIVER_E_SHAPE for an unsupported
+ *       group, RIVER_E_BADARG for null / misaligned pointers or non-positive sizes. */
+int river_quantize_w4(const void *w, int out, int in, int group, int refine_iters, void *codes, void *scale, void *zero,
+                      void *cuda_stream);
+
 int river_seq_len(const river_ctx *ctx, int slot);       /* tokens cached in the slot, or RIVER_E_BADSLOT */
 int river_release(river_ctx *ctx, int slot);             /* free the slot's pages */
 int river_stats(river_ctx *ctx, river_stats_t *host_out); /* synchronises the stream; fills host_out even when it

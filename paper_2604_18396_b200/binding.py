@@ -57,7 +57,7 @@ class river_kernel_time(C.Structure):
 EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error", "river_clear_device_error",
-           "river_selftest_wait_timeout", "river_attention", "river_project_kv")
+           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4")
 
 _lib = None
 
@@ -95,6 +95,7 @@ def load():
     L.river_argmax_noalloc.argtypes = [vp, C.c_int, C.c_int, vp, vp]
     L.river_attention.argtypes = [vp, C.c_int, C.c_int, i32p, vp, vp]
     L.river_project_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, vp]
+    L.river_quantize_w4.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp]
     L.river_clear_device_error.argtypes = [vp]
     L.river_selftest_wait_timeout.argtypes = [vp, C.c_int]
     L.river_destroy.argtypes = [vp]
@@ -153,6 +154,22 @@ def argmax_noalloc(logits: torch.Tensor, next_tok: torch.Tensor, stream=None) ->
                                          C.c_void_p(st.cuda_stream))
     if rc:
         raise RiverError(rc, "river_argmax_noalloc rejected the call")
+
+
+def quantize_w4(w: torch.Tensor, group: int = 64, refine_iters: int = 20, stream=None):
+    """river_quantize_w4: CUDA bf16 [out, in] -> (codes u8 [out, in/2], scale bf16 [out, in/group], zero bf16 [...])."""
+    assert w.is_cuda and w.dtype == torch.bfloat16 and w.dim() == 2 and w.is_contiguous()
+    out, inn = w.shape
+    codes = torch.empty((out, inn // 2), dtype=torch.uint8, device=w.device)
+    scale = torch.empty((out, inn // group), dtype=torch.bfloat16, device=w.device)
+    zero = torch.empty_like(scale)
+    st = stream if stream is not None else torch.cuda.current_stream(w.device)
+    with torch.cuda.device(w.device):
+        rc = load().river_quantize_w4(_dp(w), out, inn, group, refine_iters, _dp(codes), _dp(scale), _dp(zero),
+                                      C.c_void_p(st.cuda_stream))
+    if rc:
+        raise RiverError(rc, "river_quantize_w4 rejected the call")
+    return codes, scale, zero
 
 
 class River:

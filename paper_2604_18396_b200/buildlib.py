@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 OBJ = os.path.join(_HERE, "build")
 LIB = os.path.join(_HERE, "libriver_b200.so")
-SOURCES = ["river_api.cu", "launch_stream.cu", "launch_attn.cu", "launch_tc.cu", "launch_tc_w4.cu", "noalloc_argmax.cu"]
+SOURCES = ["river_api.cu", "launch_stream.cu", "launch_attn.cu", "launch_tc.cu", "launch_tc_w4.cu", "noalloc_argmax.cu", "quantize_w4.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 
