@@ -157,6 +157,15 @@ int river_decode_step_host(river_ctx *ctx, int batch, const int32_t *slots, cons
 int river_read_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, void *k_out, void *v_out);
 int river_write_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, const void *k_in, const void *v_in);
 
+/* Free-running greedy generation (Section 4.2, "Generation Phase"): n_steps decode steps in which every row's next
+ * token is fed back on the device - step t reads the tokens step t-1 wrote - with no host synchronisation in between
+ * (the host only enqueues; with RIVER_F_GRAPH every step is one graph launch).  Thresholds are the same for all steps.
+ *   tok0 [dev] int32 [batch] first input tokens;  tau [dev] fp32 [batch];
+ *   out_tok [dev] int32 [n_steps, batch] generated tokens;  out_exit [dev] int32 [n_steps, batch] or NULL.
+ * Fails like river_decode_step (e.g. RIVER_E_NOPAGE when a sequence fills up); steps enqueued before stay valid. */
+int river_generate(river_ctx *ctx, int batch, const int32_t *slots, const int32_t *tok0, const float *tau, int n_steps,
+                   int32_t *out_tok, int32_t *out_exit);
+
 /* Two stages of the path on their own, for kernel-level tests and the exit-aware attention microbenchmark.  Both take
  * a compacted list of rows: row i belongs to sequence slots[i] ([host], distinct, non-empty) and sits at that
  * sequence's LAST cached position p_i; both enqueue on the context's stream like a decode step.

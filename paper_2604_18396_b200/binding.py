@@ -57,7 +57,7 @@ class river_kernel_time(C.Structure):
 EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error", "river_clear_device_error",
-           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4")
+           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4", "river_generate")
 
 _lib = None
 
@@ -96,6 +96,7 @@ def load():
     L.river_attention.argtypes = [vp, C.c_int, C.c_int, i32p, vp, vp]
     L.river_project_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, vp]
     L.river_quantize_w4.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp]
+    L.river_generate.argtypes = [vp, C.c_int, i32p, vp, vp, C.c_int, vp, vp]
     L.river_clear_device_error.argtypes = [vp]
     L.river_selftest_wait_timeout.argtypes = [vp, C.c_int]
     L.river_destroy.argtypes = [vp]
@@ -268,6 +269,16 @@ class River:
         sc = slots_c if slots_c is not None else _i32_host(slots)
         self._check(load().river_decode_step_host(self.h, len(slots), sc, _hp(tok), _hp(tau), _hp(forced_exit),
                                                   _hp(logits), _hp(next_tok), _hp(exit_layer), _hp(scores)))
+
+    def generate(self, slots: Sequence[int], tok0: torch.Tensor, tau: torch.Tensor, n_steps: int):
+        """river_generate -> (tokens int32 [n_steps, batch], exit layers int32 [n_steps, batch]), both on the device."""
+        B = len(slots)
+        out_tok = torch.empty((n_steps, B), dtype=torch.int32, device=self.device)
+        out_exit = torch.empty((n_steps, B), dtype=torch.int32, device=self.device)
+        self._order_after_current()
+        self._check(load().river_generate(self.h, B, _i32_host(slots), _dp(tok0), _dp(tau), n_steps, _dp(out_tok),
+                                          _dp(out_exit)))
+        return out_tok, out_exit
 
     def read_kv(self, slot: int, layer: int, pos0: int, n: int):
         w = self.cfg.Hkv * self.cfg.dh

@@ -964,6 +964,19 @@ int river_project_kv(river_ctx *c, int layer, int use_exit_layer, int n_rows, co
     return RIVER_OK;
 }
 
+int river_generate(river_ctx *c, int batch, const int32_t *slots, const int32_t *tok0, const float *tau, int n_steps,
+                   int32_t *out_tok, int32_t *out_exit) {
+    if (!c) return RIVER_E_BADARG;
+    if (!tok0 || !tau || !out_tok || n_steps <= 0) return fail(c, RIVER_E_BADARG, "null argument / no steps");
+    for (int t = 0; t < n_steps; ++t) {
+        const int32_t *tok = t == 0 ? tok0 : out_tok + (size_t)(t - 1) * batch;  // fed back on the device
+        int32_t *ex = out_exit ? out_exit + (size_t)t * batch : c->exit_i;
+        if (int rc = river_decode_step(c, batch, slots, tok, tau, nullptr, nullptr, out_tok + (size_t)t * batch, ex, nullptr))
+            return rc;
+    }
+    return RIVER_OK;
+}
+
 int river_clear_device_error(river_ctx *c) {
     if (!c) return RIVER_E_BADARG;
     CUDA_TRY(c, cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream));

@@ -514,6 +514,49 @@ def test_bf16_cache_storage_noise_oracle_vs_oracle_and_gpu(name, prompt_len):
     b.close()
 
 
+@pytest.mark.parametrize("flags", [0, 1])
+def test_free_running_generation_feeds_tokens_back_on_the_device(flags):
+    # river_generate against the oracle generating greedily from its own tokens: the token streams must agree up to
+    # the first step at which the oracle's choice is ambiguous (top-2 logit gap below twice the logit tolerance) or an
+    # exit score lies within 1e-3 of the threshold; at least a few steps have to be comparable
+    m = model("mini8")
+    shape = m[0]
+    prompts = [toks(shape, 12, 0), toks(shape, 30, 1), toks(shape, 5, 2)]
+    steps_tok = np.stack([toks(shape, 3, 50 + t) for t in range(6)])
+    tau = natural_tau(m, prompts, steps_tok, 0.5)
+    n_steps = 24
+    p = Pair(m, 3, 30 + n_steps + 2, 4, flags=flags, page_shuffle_seed=2)
+    p.prefill([0, 1, 2], prompts)
+    tok0 = toks(shape, 3, 77)
+    g_tok, g_exit = p.gpu.generate([0, 1, 2], torch.from_numpy(tok0.astype(np.int32)).cuda(),
+                                   torch.full((3,), tau, dtype=torch.float32, device="cuda"), n_steps)
+    torch.cuda.synchronize()
+    g_tok, g_exit = g_tok.cpu().numpy(), g_exit.cpu().numpy()
+    alive = np.ones(3, bool)
+    cur = tok0.copy()
+    compared = 0
+    for t in range(n_steps):
+        o = p.oracle_step([0, 1, 2], cur, tau)
+        top2 = np.sort(o.logits, axis=1)[:, -2:]
+        for b in range(3):
+            if not alive[b]:
+                continue
+            if p.near_threshold(o.scores[b], tau, p.L) or top2[b, 1] - top2[b, 0] < 4e-2:
+                alive[b] = False  # from here on the two sides may legitimately differ
+                continue
+            assert g_exit[t, b] == o.exit_layer[b] and g_tok[t, b] == o.next_tok[b], (t, b)
+            compared += 1
+        cur = np.where(alive, o.next_tok, g_tok[t]).astype(np.int32)
+        if not alive.any():
+            break
+    print(f"free-running generation: {compared} (step, row) pairs compared before ambiguity")
+    assert compared >= 6
+    for b in range(3):
+        assert p.gpu.seq_len(b) == len(prompts[b]) + n_steps
+    assert p.gpu.stats().device_error == 0
+    p.close()
+
+
 def test_pool_exhaustion_fails_cleanly_and_the_retry_is_exact():
     # a step that needs more pages than are free takes none (no half-updated page table), and the same rows step
     # correctly once pages have been released
