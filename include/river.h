@@ -95,6 +95,7 @@ typedef struct river_stats_t {
     double alg_bytes_last_step;  /* algorithmic HBM bytes of the last step (executed-layer weights + KV read/written
                                     + LM head + embedding rows + logits), from its actual exit pattern */
     double layers_executed_last; /* mean exit_layer / L over the rows of the last step */
+    int64_t offload_fetches;     /* backbone blocks copied from host memory since river_init (river_offload) */
 } river_stats_t;
 
 typedef struct river_ctx river_ctx;
@@ -165,6 +166,18 @@ int river_write_kv(river_ctx *ctx, int slot, int layer, int pos0, int n, const v
  * Fails like river_decode_step (e.g. RIVER_E_NOPAGE when a sequence fills up); steps enqueued before stay valid. */
 int river_generate(river_ctx *ctx, int batch, const int32_t *slots, const int32_t *tok0, const float *tau, int n_steps,
                    int32_t *out_tok, int32_t *out_exit);
+
+/* Backbone offloading (Section 4.2, "Backbone Offloading"): the bf16 matrices of backbone blocks
+ * first_offloaded_layer..L live in PINNED HOST memory and are copied into device memory only for a step whose rows are
+ * still in the backbone when they reach such a block (the exit layers, which carry most tokens, stay resident).
+ *   host_layers [host] array of L entries; in entries >= first_offloaded_layer wq, wk, wv, wo, wg, wu, wd are pinned
+ *       host pointers to the bf16 matrices (norm gains and exit-layer weights stay as given to river_init);
+ *   device side: at river_init the offloaded blocks must have been given device matrices that alternate between TWO
+ *       staging slots (blocks l and l + 2 the same seven pointers): a block is staged while the previous one runs.
+ * With offloading on, a step synchronises with the host once per offloaded block (the host must see whether any row is
+ * still in the backbone before it copies 2 P bytes), graph replay is off and the exit score runs as a kernel of its
+ * own.  first_offloaded_layer = 0 turns it off.  river_stats.offload_fetches counts the block copies. */
+int river_offload(river_ctx *ctx, int first_offloaded_layer, const river_layer_weights *host_layers);
 
 /* Two stages of the path on their own, for kernel-level tests and the exit-aware attention microbenchmark.  Both take
  * a compacted list of rows: row i belongs to sequence slots[i] ([host], distinct, non-empty) and sits at that

@@ -46,7 +46,8 @@ class river_weights(C.Structure):
 class river_stats_t(C.Structure):
     _fields_ = [("steps", C.c_int64), ("launches_total", C.c_int64), ("launches_last_step", C.c_int32),
                 ("batch_last", C.c_int32), ("device_error", C.c_int32), ("pages_in_use", C.c_int32),
-                ("alg_bytes_last_step", C.c_double), ("layers_executed_last", C.c_double)]
+                ("alg_bytes_last_step", C.c_double), ("layers_executed_last", C.c_double),
+                ("offload_fetches", C.c_int64)]
 
 
 class river_kernel_time(C.Structure):
@@ -57,7 +58,7 @@ class river_kernel_time(C.Structure):
 EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error", "river_clear_device_error",
-           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4", "river_generate")
+           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4", "river_generate", "river_offload")
 
 _lib = None
 
@@ -96,6 +97,7 @@ def load():
     L.river_attention.argtypes = [vp, C.c_int, C.c_int, i32p, vp, vp]
     L.river_project_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, vp]
     L.river_quantize_w4.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp]
+    L.river_offload.argtypes = [vp, C.c_int, C.POINTER(river_layer_weights)]
     L.river_generate.argtypes = [vp, C.c_int, i32p, vp, vp, C.c_int, vp, vp]
     L.river_clear_device_error.argtypes = [vp]
     L.river_selftest_wait_timeout.argtypes = [vp, C.c_int]
@@ -269,6 +271,20 @@ class River:
         sc = slots_c if slots_c is not None else _i32_host(slots)
         self._check(load().river_decode_step_host(self.h, len(slots), sc, _hp(tok), _hp(tau), _hp(forced_exit),
                                                   _hp(logits), _hp(next_tok), _hp(exit_layer), _hp(scores)))
+
+    def offload(self, first_offloaded_layer: int, host_layers: Optional[List[dict]] = None):
+        """river_offload; host_layers: per layer a dict of pinned CPU bf16 tensors (wq .. wd) or None."""
+        nl = self.cfg.L
+        arr = (river_layer_weights * nl)()
+        if host_layers is not None:
+            for l in range(nl):
+                if host_layers[l] is not None:
+                    for n in ("wq", "wk", "wv", "wo", "wg", "wu", "wd"):
+                        t = host_layers[l][n]
+                        assert t.is_pinned() and t.is_contiguous() and t.dtype == torch.bfloat16
+                        setattr(arr[l], n, t.data_ptr())
+        self._keep_host = host_layers
+        self._check(load().river_offload(self.h, first_offloaded_layer, arr))
 
     def generate(self, slots: Sequence[int], tok0: torch.Tensor, tau: torch.Tensor, n_steps: int):
         """river_generate -> (tokens int32 [n_steps, batch], exit layers int32 [n_steps, batch]), both on the device."""

@@ -327,6 +327,43 @@ int profile_collect(river_ctx *c) {
     return 0;
 }
 
+// ---- backbone offloading (Section 4.2, "Backbone Offloading")
+// Stage block l's seven bf16 matrices from pinned host memory into the device slot its layer entry points at, unless
+// the slot already holds them; the copy runs on its own stream, after the kernels that last used the slot.
+int offload_fetch(river_ctx *c, int l) {
+    const river_config &g = c->cfg;
+    const int slot = (l - c->off_first) & 1;
+    if (c->off_slot_layer[slot] == l) return RIVER_OK;
+    const river_layer_weights &dst = c->layers[l - 1], &src = c->off_host[l - 1];
+    const size_t qdim = (size_t)g.Hq * g.dh, kvdim = (size_t)g.Hkv * g.dh, d = g.d, F = g.F;
+    const void *dp[7] = {dst.wq, dst.wk, dst.wv, dst.wo, dst.wg, dst.wu, dst.wd};
+    const void *sp[7] = {src.wq, src.wk, src.wv, src.wo, src.wg, src.wu, src.wd};
+    const size_t nb[7] = {qdim * d * 2, kvdim * d * 2, kvdim * d * 2, d * qdim * 2, F * d * 2, F * d * 2, d * F * 2};
+    CUDA_TRY(c, cudaStreamWaitEvent(c->off_copy, c->off_freed[slot], 0));
+    for (int i = 0; i < 7; ++i)
+        CUDA_TRY(c, cudaMemcpyAsync(const_cast<void *>(dp[i]), sp[i], nb[i], cudaMemcpyHostToDevice, c->off_copy));
+    CUDA_TRY(c, cudaEventRecord(c->off_ready[slot], c->off_copy));
+    c->off_slot_layer[slot] = l;
+    c->st.offload_fetches += 1;
+    return RIVER_OK;
+}
+
+// Before block l >= off_first: are rows still in the backbone?  (A host decision: the one place where a step with
+// offloading synchronises.)  If so the block's weights are staged and the next block's copy is started behind them.
+int offload_before_layer(river_ctx *c, int l, bool *staged) {
+    *staged = false;
+    int32_t na = 0;
+    CUDA_TRY(c, cudaMemcpyAsync(&na, c->n_act + (l - 1), sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (na <= 0) return RIVER_OK;
+    if (int rc = offload_fetch(c, l)) return rc;
+    CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->off_ready[(l - c->off_first) & 1], 0));
+    if (l + 1 <= c->cfg.L)
+        if (int rc = offload_fetch(c, l + 1)) return rc;
+    *staged = true;
+    return RIVER_OK;
+}
+
 // a2 of block l for the n rows of the step: attention norm + QKV + RoPE + KV write, on the weight set(s) the row
 // lists name (small steps: from the exit flags).
 cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const DecideArgs &dec, double kv_write) {
@@ -388,7 +425,8 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
     const double kv_write = (double)n * 2.0 * kvdim * 2.0;
     cudaError_t err = cudaSuccess;
     auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
-    const bool fold = n <= 4;  // the decisions ride in the QKV kernels
+    const bool fold = n <= 4 && !c->off_first;  // the decisions ride in the QKV kernels (with offloading the host has to
+                                                // see every decision before it stages a block: score kernel per block)
     const DecideArgs no_dec{};
 
     {
@@ -419,6 +457,9 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
         const river_ctx::LayerMaps *wm = (tc && c->w4tc_ok && has_river) ? &c->w4_maps[l - 1] : nullptr;
         const int32_t *nrh = c->n_riv + std::max(0, l - 2);  // never above the count entering this block
         const int skip_bb = tc ? 1 : 0;
+        bool staged = false;
+        if (c->off_first && l >= c->off_first)
+            if (int rc = offload_before_layer(c, l, &staged)) return rc;
         // ---- a2: attention norm + QKV + RoPE + KV write (+ a6 / a7 of the previous block when the step is small)
         {
             DecideArgs dec{};
@@ -498,6 +539,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
         }
         // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
         if (!fold) launch_score(l, h_in, h_out);
+        if (staged) note(cudaEventRecord(c->off_freed[(l - c->off_first) & 1], c->stream));  // the slot may be refilled
         prev_in = h_in;
         hi = (hi + 2) % 3;
     }
@@ -535,7 +577,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
 // One decode step through a CUDA graph of the launch sequence (captured the second time a row count is seen; the
 // per-step inputs live in device memory, so the graph never needs new parameters).
 int run_step(river_ctx *c, int n, const int32_t *row_pos_host) {
-    const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling;
+    const bool use_graph = (c->cfg.flags & RIVER_F_GRAPH) && !c->profiling && !c->off_first;
     if (!use_graph) return run_rows(c, n, n, row_pos_host);
     const int key_splits = c->attn_small_now ? 0 : c->attn_splits_now;  // the attention grid of the captured launches
     for (auto &ge : c->graphs)
@@ -953,12 +995,18 @@ int river_project_kv(river_ctx *c, int layer, int use_exit_layer, int n_rows, co
     if (!c) return RIVER_E_BADARG;
     if (!h) return fail(c, RIVER_E_BADARG, "null argument");
     if (int rc = stage_rows(c, layer, n_rows, slots, use_exit_layer ? 1 : 0)) return rc;
+    if (!use_exit_layer && c->off_first && layer >= c->off_first) {  // an offloaded backbone block: stage it first
+        if (int rc = offload_fetch(c, layer)) return rc;
+        CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->off_ready[(layer - c->off_first) & 1], 0));
+    }
     float *q_keep = c->qbuf;
     if (q_out) c->qbuf = q_out;
     c->st.launches_last_step = 0;
     const cudaError_t e = launch_qkv(c, layer, n_rows, h, DecideArgs{}, (double)n_rows * 4.0 * c->cfg.Hkv * c->cfg.dh);
     c->qbuf = q_keep;
     if (e != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(e));
+    if (!use_exit_layer && c->off_first && layer >= c->off_first)
+        CUDA_TRY(c, cudaEventRecord(c->off_freed[(layer - c->off_first) & 1], c->stream));
     c->st.launches_total += c->st.launches_last_step;
     if (c->profiling) return profile_collect(c);
     return RIVER_OK;
@@ -974,6 +1022,36 @@ int river_generate(river_ctx *c, int batch, const int32_t *slots, const int32_t 
         if (int rc = river_decode_step(c, batch, slots, tok, tau, nullptr, nullptr, out_tok + (size_t)t * batch, ex, nullptr))
             return rc;
     }
+    return RIVER_OK;
+}
+
+int river_offload(river_ctx *c, int first_offloaded_layer, const river_layer_weights *host_layers) {
+    if (!c) return RIVER_E_BADARG;
+    const river_config &g = c->cfg;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (first_offloaded_layer == 0) { c->off_first = 0; return RIVER_OK; }
+    if (first_offloaded_layer < 2 || first_offloaded_layer > g.L || !host_layers)
+        return fail(c, RIVER_E_BADARG, "first_offloaded_layer must be 0 or lie in [2, L], with the host copies given");
+    for (int l = first_offloaded_layer; l <= g.L; ++l) {
+        const river_layer_weights &h = host_layers[l - 1], &dv = c->layers[l - 1];
+        if (!h.wq || !h.wk || !h.wv || !h.wo || !h.wg || !h.wu || !h.wd)
+            return fail(c, RIVER_E_BADARG, "null host copy in an offloaded layer");
+        if (l + 2 <= g.L) {  // blocks two apart must share a device slot
+            const river_layer_weights &d2 = c->layers[l + 1];
+            if (dv.wq != d2.wq || dv.wk != d2.wk || dv.wv != d2.wv || dv.wo != d2.wo || dv.wg != d2.wg || dv.wu != d2.wu || dv.wd != d2.wd)
+                return fail(c, RIVER_E_BADARG, "offloaded blocks l and l + 2 must be given the same device matrices (two staging slots)");
+        }
+    }
+    if (!c->off_copy) {
+        CUDA_TRY(c, cudaStreamCreateWithFlags(&c->off_copy, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CUDA_TRY(c, cudaEventCreateWithFlags(&c->off_ready[i], cudaEventDisableTiming));
+            CUDA_TRY(c, cudaEventCreateWithFlags(&c->off_freed[i], cudaEventDisableTiming));
+        }
+    }
+    c->off_host.assign(host_layers, host_layers + g.L);
+    c->off_first = first_offloaded_layer;
+    c->off_slot_layer[0] = c->off_slot_layer[1] = -1;
     return RIVER_OK;
 }
 
@@ -1141,6 +1219,11 @@ void river_destroy(river_ctx *c) {
         if (c->meta_host[i]) { cudaFreeHost(c->meta_host[i]); cudaEventDestroy(c->meta_ev[i]); }
     }
     if (c->pin_io) cudaFreeHost(c->pin_io);
+    if (c->off_copy) {
+        cudaStreamSynchronize(c->off_copy);
+        for (int i = 0; i < 2; ++i) { cudaEventDestroy(c->off_ready[i]); cudaEventDestroy(c->off_freed[i]); }
+        cudaStreamDestroy(c->off_copy);
+    }
     delete c;
 }
 

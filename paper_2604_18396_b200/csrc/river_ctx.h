@@ -73,6 +73,14 @@ struct river_ctx {
     river_stats_t st{};
     std::string err;
 
+    // backbone offloading: blocks >= off_first keep their bf16 matrices in pinned host memory and are staged, on
+    // demand, into the two device slots their layer entries alias
+    int off_first = 0;  // 0 = off
+    std::vector<river_layer_weights> off_host;
+    cudaStream_t off_copy = nullptr;
+    cudaEvent_t off_ready[2] = {nullptr, nullptr}, off_freed[2] = {nullptr, nullptr};
+    int off_slot_layer[2] = {-1, -1};
+
     // per-context launch bookkeeping: the largest dynamic shared memory size set per kernel, and the launch geometry
     // of the streaming kernels per (kernel, task count, K)
     struct SmemAttr { const void *fn; size_t bytes; };

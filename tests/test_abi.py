@@ -43,7 +43,7 @@ def test_struct_layouts_match_header():
     assert fields == [f[0] for f in binding.river_config._fields_]
     assert ctypes.sizeof(binding.river_config) == 4 * len(fields)
     assert ctypes.sizeof(binding.river_layer_weights) == 8 * (9 + 21)
-    assert ctypes.sizeof(binding.river_stats_t) == 8 + 8 + 4 * 4 + 8 + 8
+    assert ctypes.sizeof(binding.river_stats_t) == 8 + 8 + 4 * 4 + 8 + 8 + 8
 
 
 def test_size_queries_and_config_checks_need_no_gpu(lib):
