@@ -8,16 +8,30 @@
 // DH/32 head dims.  The eight warp states merge through shared memory (the pipeline stages, free by then) into one
 // partial (max, sum, unnormalised output) per (row, head, split); the last split of a (row, kv head) to finish merges
 // the splits.  All arithmetic is fp32, exponentials are base 2 (q is pre-scaled by log2 e).
+//
+// Groups of up to four query heads run the two contractions on the warp-level tensor cores instead (MMA = true; the
+// CUDA-core consumers above retire ~1500 warp instructions per 8 KB page and are bound by instruction issue at half the
+// HBM rate).  Four consumer warps, one page of every tile each:
+//   * S = Q K^T as mma.sync m16n8k16 with the pre-scaled queries as the A operand, held in registers for the whole
+//     kernel: row g carries the bf16 head of q_g, row 4 + g its bf16 remainder (q = hi + lo keeps 16 mantissa bits);
+//     the K page is the B operand, read from the swizzled stage with ldmatrix exactly as TMA laid it down;
+//   * the two partial scores of a head meet with one shuffle; the online softmax runs in the accumulator layout (a lane
+//     holds one head row and four positions of the page);
+//   * O^T = V^T P^T: the V page is the A operand (ldmatrix.trans of the same swizzled rows), the probabilities are the
+//     B operand - again split p = hi + lo into columns g and 4 + g - and the accumulator layout of S is already the
+//     fragment layout of that operand, so nothing is exchanged between lanes; O^T keeps DH x 8 fp32 values per warp.
+//   Cache rows past the row's position are never multiplied: their scores are replaced, their V fragments zeroed.
 #pragma once
 #include "mbar_tma.cuh"
+#include "mma_sync.cuh"
 
 namespace river {
 
 constexpr int kAttnTile = 64;      // positions per pipeline stage (4 pages)
 constexpr int kAttnStages = 2;     // two stages of 32 KB (head dim 128): three CTAs per SM, 24 consumer warps
 constexpr int kAttnConsumers = 4;  // pages per tile
-constexpr int kAttnWarps = 2 * kAttnConsumers;         // consumer warps: two per page, 8 positions each
-constexpr int kAttnThreads = 32 * (kAttnWarps + 1);    // consumers + producer
+constexpr int kAttnWarps = 2 * kAttnConsumers;         // CUDA-core consumer warps: two per page, 8 positions each
+__host__ __device__ constexpr int attn_threads(bool mma) { return 32 * ((mma ? kAttnConsumers : kAttnWarps) + 1); }  // consumers + producer
 struct AttnArgs {
     const StepMeta *meta;
     const float *q;        // [rows][Hq*DH]
@@ -31,10 +45,12 @@ struct AttnArgs {
     int *dev_err;
 };
 
-template <int DH, int GQ>
-__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
-                                                                  const AttnArgs a) {
-    constexpr int NW = kAttnWarps;               // consumer warps
+template <int DH, int GQ, bool MMA>
+__global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                       const AttnArgs a) {
+    static_assert(!MMA || GQ <= 4, "the tensor-core consumers carry hi and lo parts of four heads in eight columns");
+    constexpr int NW = MMA ? kAttnConsumers : kAttnWarps;  // consumer warps
+    constexpr int kAttnThreads = attn_threads(MMA);
     constexpr int HP = kPage / 2;                // positions per warp and tile
     constexpr int NB = DH / 64;                  // 128-byte boxes per cache row
     constexpr int PAGE_BYTES = kPage * DH * 2;   // one page of K (or V) of one kv head
@@ -105,122 +121,261 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     };
     if (is_producer)
         for (int t = 0; t < min(n_tiles, kAttnStages); ++t) issue_tile(t);
-    for (int i = tid; i < GQ * DH; i += kAttnThreads)
-        sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
+    if constexpr (!MMA) {
+        for (int i = tid; i < GQ * DH; i += kAttnThreads)
+            sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
+    }
     __syncthreads();
 
-    // ---------------- consumers: warp w owns positions [8 (w / 4), + 8) of page w % 4 of every tile
-    const int r8 = lane & 7, qtr = lane >> 3;
-    const int pg = warp & (kAttnConsumers - 1), ph = warp / kAttnConsumers;
-    const int r = ph * HP + r8;  // this lane's position inside the page
-    float m[GQ], l[GQ], acc[GQ][VE];
+    if constexpr (MMA) {
+        // ---------------- tensor-core consumers: warp w owns page w of every tile
+        constexpr int KS = DH / 16;  // k-steps of S = Q K^T, and 16-dim row tiles of O^T
+        const int t4 = lane & 3, r8 = lane >> 2;
+        const int g = r8 & 3;
+        const bool lo_row = r8 >= 4;
+        uint32_t qa[KS][2];  // A fragments of Q: rows 0-3 hi parts, rows 4-7 remainders, rows 8-15 zero
 #pragma unroll
-    for (int g = 0; g < GQ; ++g) {
-        m[g] = -CUDART_INF_F;
-        l[g] = 0.f;
+        for (int ks = 0; ks < KS; ++ks) {
+            float2 x0 = make_float2(0.f, 0.f), x1 = x0;
+            if (g < GQ && warp < NW) {
+                const float *qp = a.q + (size_t)row * a.Hq * DH + (size_t)(kvh * GQ + g) * DH + ks * 16 + 2 * t4;
+                x0 = *reinterpret_cast<const float2 *>(qp);
+                x1 = *reinterpret_cast<const float2 *>(qp + 8);
+            }
+            x0.x *= a.qscale; x0.y *= a.qscale; x1.x *= a.qscale; x1.y *= a.qscale;
+            const uint32_t h0 = pack_bf16x2(x0.x, x0.y), h1 = pack_bf16x2(x1.x, x1.y);
+            qa[ks][0] = lo_row ? pack_bf16x2(x0.x - bf16lo(h0), x0.y - bf16hi(h0)) : h0;
+            qa[ks][1] = lo_row ? pack_bf16x2(x1.x - bf16lo(h1), x1.y - bf16hi(h1)) : h1;
+        }
+        float m = -CUDART_INF_F, l = 0.f;  // head g's state (held twice: by the lanes of row g and of row 4 + g)
+        float acc[KS][4];                  // O^T: dims 16 mt + r8 (+ 8), columns 2 t4, 2 t4 + 1
 #pragma unroll
-        for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
-    }
-    if (warp == NW) {
-        if (lane == 0)
-            for (int t = kAttnStages; t < n_tiles; ++t)
-                if (!issue_tile(t)) break;
-    } else {
-        float *my_sp = sp + warp * HP * GQ;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int s = t % kAttnStages;
-            if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
-            const int pos0 = p0 + t * kAttnTile + pg * kPage + ph * HP;  // first position of this warp's half page
-            if (pos0 < p1) {
-                const uint8_t *kpg = stages + s * STAGE_BYTES + pg * PAGE_BYTES;
-                const uint8_t *vpg = kpg + kAttnConsumers * PAGE_BYTES;
-                // q.K for position r, dims [qtr*DH/4, (qtr+1)*DH/4)
-                float sc[GQ];
+        for (int mt = 0; mt < KS; ++mt)
 #pragma unroll
-                for (int g = 0; g < GQ; ++g) sc[g] = 0.f;
+            for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
+        if (warp == NW) {
+            if (lane == 0)
+                for (int t = kAttnStages; t < n_tiles; ++t)
+                    if (!issue_tile(t)) break;
+        } else {
+            // ldmatrix row of this lane: matrix lane / 8 -> positions 8 (lane / 16) .., 16-byte chunk parity (lane / 8) & 1
+            const int lpos = (lane & 7) + 8 * (lane >> 4), lodd = (lane >> 3) & 1;
+            for (int t = 0; t < n_tiles; ++t) {
+                const int s = t % kAttnStages;
+                if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
+                const int pos0 = p0 + t * kAttnTile + warp * kPage;  // first position of this warp's page
+                if (pos0 < p1) {
+                    const int n_live = min(kPage, p1 - pos0);
+                    const uint32_t kpg = smem_u32(stages + s * STAGE_BYTES + warp * PAGE_BYTES);
+                    const uint32_t vpg = kpg + kAttnConsumers * PAGE_BYTES;
+                    float sc[2][4];  // S: row r8, positions 8 j + 2 t4 (+ 1) in [j][0..1]; rows 8-15 (unused) in [j][2..3]
 #pragma unroll
-                for (int i = 0; i < NCH; ++i) {
-                    const int cg = qtr * NCH + i, box = cg >> 3, c = cg & 7;
-                    const uint4 kw = *reinterpret_cast<const uint4 *>(kpg + box * (kPage * 128) + r * 128 +
-                                                                     ((c ^ (r & 7)) << 4));
-                    const float k0 = bf16lo(kw.x), k1 = bf16hi(kw.x), k2 = bf16lo(kw.y), k3 = bf16hi(kw.y);
-                    const float k4 = bf16lo(kw.z), k5 = bf16hi(kw.z), k6 = bf16lo(kw.w), k7 = bf16hi(kw.w);
+                    for (int j = 0; j < 2; ++j)
 #pragma unroll
-                    for (int g = 0; g < GQ; ++g) {
-                        const float4 qa = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8);
-                        const float4 qb = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8 + 4);
-                        float v = sc[g];
-                        v = fmaf(qa.x, k0, v); v = fmaf(qa.y, k1, v); v = fmaf(qa.z, k2, v); v = fmaf(qa.w, k3, v);
-                        v = fmaf(qb.x, k4, v); v = fmaf(qb.y, k5, v); v = fmaf(qb.z, k6, v); v = fmaf(qb.w, k7, v);
-                        sc[g] = v;
+                        for (int e = 0; e < 4; ++e) sc[j][e] = 0.f;
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        const int cg = 2 * ks + lodd, box = cg >> 3, c = cg & 7;
+                        uint32_t kf[4];
+                        ldsm_x4(kf, kpg + box * (kPage * 128) + lpos * 128 + ((c ^ (lpos & 7)) << 4));
+                        const uint32_t af[4] = {qa[ks][0], 0u, qa[ks][1], 0u};
+                        mma_bf16_m16n8k16(sc[0], af, kf[0], kf[1]);
+                        mma_bf16_m16n8k16(sc[1], af, kf[2], kf[3]);
                     }
-                }
-                const bool live = pos0 + r8 < p1;
-                float corr[GQ];
+                    float p[2][2], mx = -CUDART_INF_F;
 #pragma unroll
-                for (int g = 0; g < GQ; ++g) {
-                    float v = sc[g] + __shfl_xor_sync(0xffffffffu, sc[g], 8);
-                    v += __shfl_xor_sync(0xffffffffu, v, 16);
-                    v = live ? v : -CUDART_INF_F;  // select, never arithmetic: stale cache rows may hold anything
-                    float mx = v;
+                    for (int j = 0; j < 2; ++j)
 #pragma unroll
-                    for (int o = 4; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    const float mn = fmaxf(m[g], mx);  // finite: position pos0 is live
-                    corr[g] = ex2(m[g] - mn);
-                    m[g] = mn;
-                    const float p = live ? ex2(v - mn) : 0.f;
-                    if (qtr == 0) my_sp[r8 * GQ + g] = p;
-                    l[g] = fmaf(l[g], corr[g], qtr == 0 ? p : 0.f);  // this lane's share of the sum; added up at the end
+                        for (int e = 0; e < 2; ++e) {
+                            float v = sc[j][e] + __shfl_xor_sync(0xffffffffu, sc[j][e], 16);  // hi row + remainder row
+                            v = (8 * j + 2 * t4 + e < n_live) ? v : -CUDART_INF_F;  // select: stale rows may hold anything
+                            p[j][e] = v;
+                            mx = fmaxf(mx, v);
+                        }
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float mn = fmaxf(m, mx);  // finite: position pos0 is live
+                    const float corr = ex2(m - mn);
+                    m = mn;
+                    float psum = 0.f;
+                    uint32_t pb[2];
 #pragma unroll
-                    for (int e = 0; e < VE; ++e) acc[g][e] *= corr[g];
+                    for (int j = 0; j < 2; ++j) {
+                        const float e0 = ex2(p[j][0] - mn), e1 = ex2(p[j][1] - mn);  // masked positions: exactly 0
+                        psum += e0 + e1;
+                        const uint32_t h = pack_bf16x2(e0, e1);
+                        pb[j] = lo_row ? pack_bf16x2(e0 - bf16lo(h), e1 - bf16hi(h)) : h;
+                    }
+                    l = fmaf(l, corr, psum);
+                    // the accumulator columns 2 t4, 2 t4 + 1 belong to heads (2 t4) & 3 and (2 t4 + 1) & 3
+                    const float c0 = __shfl_sync(0xffffffffu, corr, ((2 * t4) & 3) * 4);
+                    const float c1 = __shfl_sync(0xffffffffu, corr, ((2 * t4 + 1) & 3) * 4);
+                    const bool cut = n_live < kPage;
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt) {
+                        const int cg = 2 * mt + lodd, box = cg >> 3, c = cg & 7;
+                        uint32_t vf[4];
+                        ldsm_x4_trans(vf, vpg + box * (kPage * 128) + lpos * 128 + ((c ^ (lpos & 7)) << 4));
+                        if (cut) {  // vf[0..1]: positions 2 t4, 2 t4 + 1; vf[2..3]: positions 8 + 2 t4, 9 + 2 t4
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int pp = 2 * t4 + 8 * (q >> 1);
+                                if (pp >= n_live) vf[q] = 0u;
+                                else if (pp + 1 >= n_live) vf[q] &= 0x0000ffffu;
+                            }
+                        }
+                        acc[mt][0] *= c0; acc[mt][1] *= c1; acc[mt][2] *= c0; acc[mt][3] *= c1;
+                        mma_bf16_m16n8k16(acc[mt], vf, pb[0], pb[1]);
+                    }
                 }
                 __syncwarp();
-                // P.V: lane owns dims [lane*VE, lane*VE + VE)
-                const int n_live = min(HP, p1 - pos0);
-                const int vbyte = lane * VE * 2, vbox = vbyte >> 7, vc = (vbyte & 127) >> 4, vo = vbyte & 15;
-                for (int j = 0; j < n_live; ++j) {
-                    const int vr = ph * HP + j;
-                    const uint8_t *vp = vpg + vbox * (kPage * 128) + vr * 128 + ((vc ^ (vr & 7)) << 4) + vo;
-                    float vf[VE];
-                    if (VE == 4) {
-                        const uint2 w = *reinterpret_cast<const uint2 *>(vp);
-                        vf[0] = bf16lo(w.x); vf[1] = bf16hi(w.x); vf[2 % VE] = bf16lo(w.y); vf[3 % VE] = bf16hi(w.y);
-                    } else {
-                        const uint32_t w = *reinterpret_cast<const uint32_t *>(vp);
-                        vf[0] = bf16lo(w); vf[1] = bf16hi(w);
-                    }
+                if (lane == 0) mbar_arrive(smem_u32(&bars[kAttnStages + s]));
+            }
+        }
+        __syncthreads();
+        if (warp < NW && !s_abort) {
+            // column 4 + g holds the remainder part of head g: add it to column g, then lanes t4 < 2 own heads 2 t4, 2 t4 + 1
 #pragma unroll
-                    for (int g = 0; g < GQ; ++g) {
-                        const float p = my_sp[j * GQ + g];
+            for (int mt = 0; mt < KS; ++mt)
 #pragma unroll
-                        for (int e = 0; e < VE; ++e) acc[g][e] = fmaf(p, vf[e], acc[g][e]);
+                for (int e = 0; e < 4; ++e) acc[mt][e] += __shfl_xor_sync(0xffffffffu, acc[mt][e], 2);
+            if (t4 < 2) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int hg = 2 * t4 + e;
+                    if (hg < GQ) {
+                        float *dst = sm + (warp * GQ + hg) * (DH + 2);
+#pragma unroll
+                        for (int mt = 0; mt < KS; ++mt) {
+                            dst[mt * 16 + r8] = acc[mt][e];
+                            dst[mt * 16 + r8 + 8] = acc[mt][2 + e];
+                        }
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars[kAttnStages + s]));
+            float lsum = l + __shfl_xor_sync(0xffffffffu, l, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            if (t4 == 0 && r8 < GQ) {
+                float *dst = sm + (warp * GQ + r8) * (DH + 2);
+                dst[DH] = m;
+                dst[DH + 1] = lsum;
+            }
         }
-    }
-    // every tile that was requested has landed and has been read by every consumer warp (unless the CTA gave up): the
-    // stages may now hold the warp states
-    __syncthreads();
-    if (warp < NW && !s_abort) {
-#pragma unroll
+        __syncthreads();
+    } else {
+        // ---------------- consumers: warp w owns positions [8 (w / 4), + 8) of page w % 4 of every tile
+        const int r8 = lane & 7, qtr = lane >> 3;
+        const int pg = warp & (kAttnConsumers - 1), ph = warp / kAttnConsumers;
+        const int r = ph * HP + r8;  // this lane's position inside the page
+        float m[GQ], l[GQ], acc[GQ][VE];
+    #pragma unroll
         for (int g = 0; g < GQ; ++g) {
-            float *dst = sm + (warp * GQ + g) * (DH + 2);
-#pragma unroll
-            for (int e = 0; e < VE; ++e) dst[lane * VE + e] = acc[g][e];
-            const float lsum = warp_sum(l[g]);
-            if (lane == 0) { dst[DH] = m[g]; dst[DH + 1] = lsum; }
+            m[g] = -CUDART_INF_F;
+            l[g] = 0.f;
+    #pragma unroll
+            for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
         }
+        if (warp == NW) {
+            if (lane == 0)
+                for (int t = kAttnStages; t < n_tiles; ++t)
+                    if (!issue_tile(t)) break;
+        } else {
+            float *my_sp = sp + warp * HP * GQ;
+            for (int t = 0; t < n_tiles; ++t) {
+                const int s = t % kAttnStages;
+                if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
+                const int pos0 = p0 + t * kAttnTile + pg * kPage + ph * HP;  // first position of this warp's half page
+                if (pos0 < p1) {
+                    const uint8_t *kpg = stages + s * STAGE_BYTES + pg * PAGE_BYTES;
+                    const uint8_t *vpg = kpg + kAttnConsumers * PAGE_BYTES;
+                    // q.K for position r, dims [qtr*DH/4, (qtr+1)*DH/4)
+                    float sc[GQ];
+    #pragma unroll
+                    for (int g = 0; g < GQ; ++g) sc[g] = 0.f;
+    #pragma unroll
+                    for (int i = 0; i < NCH; ++i) {
+                        const int cg = qtr * NCH + i, box = cg >> 3, c = cg & 7;
+                        const uint4 kw = *reinterpret_cast<const uint4 *>(kpg + box * (kPage * 128) + r * 128 +
+                                                                         ((c ^ (r & 7)) << 4));
+                        const float k0 = bf16lo(kw.x), k1 = bf16hi(kw.x), k2 = bf16lo(kw.y), k3 = bf16hi(kw.y);
+                        const float k4 = bf16lo(kw.z), k5 = bf16hi(kw.z), k6 = bf16lo(kw.w), k7 = bf16hi(kw.w);
+    #pragma unroll
+                        for (int g = 0; g < GQ; ++g) {
+                            const float4 qa = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8);
+                            const float4 qb = *reinterpret_cast<const float4 *>(sq + g * DH + cg * 8 + 4);
+                            float v = sc[g];
+                            v = fmaf(qa.x, k0, v); v = fmaf(qa.y, k1, v); v = fmaf(qa.z, k2, v); v = fmaf(qa.w, k3, v);
+                            v = fmaf(qb.x, k4, v); v = fmaf(qb.y, k5, v); v = fmaf(qb.z, k6, v); v = fmaf(qb.w, k7, v);
+                            sc[g] = v;
+                        }
+                    }
+                    const bool live = pos0 + r8 < p1;
+                    float corr[GQ];
+    #pragma unroll
+                    for (int g = 0; g < GQ; ++g) {
+                        float v = sc[g] + __shfl_xor_sync(0xffffffffu, sc[g], 8);
+                        v += __shfl_xor_sync(0xffffffffu, v, 16);
+                        v = live ? v : -CUDART_INF_F;  // select, never arithmetic: stale cache rows may hold anything
+                        float mx = v;
+    #pragma unroll
+                        for (int o = 4; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                        const float mn = fmaxf(m[g], mx);  // finite: position pos0 is live
+                        corr[g] = ex2(m[g] - mn);
+                        m[g] = mn;
+                        const float p = live ? ex2(v - mn) : 0.f;
+                        if (qtr == 0) my_sp[r8 * GQ + g] = p;
+                        l[g] = fmaf(l[g], corr[g], qtr == 0 ? p : 0.f);  // this lane's share of the sum; added up at the end
+    #pragma unroll
+                        for (int e = 0; e < VE; ++e) acc[g][e] *= corr[g];
+                    }
+                    __syncwarp();
+                    // P.V: lane owns dims [lane*VE, lane*VE + VE)
+                    const int n_live = min(HP, p1 - pos0);
+                    const int vbyte = lane * VE * 2, vbox = vbyte >> 7, vc = (vbyte & 127) >> 4, vo = vbyte & 15;
+                    for (int j = 0; j < n_live; ++j) {
+                        const int vr = ph * HP + j;
+                        const uint8_t *vp = vpg + vbox * (kPage * 128) + vr * 128 + ((vc ^ (vr & 7)) << 4) + vo;
+                        float vf[VE];
+                        if (VE == 4) {
+                            const uint2 w = *reinterpret_cast<const uint2 *>(vp);
+                            vf[0] = bf16lo(w.x); vf[1] = bf16hi(w.x); vf[2 % VE] = bf16lo(w.y); vf[3 % VE] = bf16hi(w.y);
+                        } else {
+                            const uint32_t w = *reinterpret_cast<const uint32_t *>(vp);
+                            vf[0] = bf16lo(w); vf[1] = bf16hi(w);
+                        }
+    #pragma unroll
+                        for (int g = 0; g < GQ; ++g) {
+                            const float p = my_sp[j * GQ + g];
+    #pragma unroll
+                            for (int e = 0; e < VE; ++e) acc[g][e] = fmaf(p, vf[e], acc[g][e]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars[kAttnStages + s]));
+            }
+        }
+        // every tile that was requested has landed and has been read by every consumer warp (unless the CTA gave up): the
+        // stages may now hold the warp states
+        __syncthreads();
+        if (warp < NW && !s_abort) {
+    #pragma unroll
+            for (int g = 0; g < GQ; ++g) {
+                float *dst = sm + (warp * GQ + g) * (DH + 2);
+    #pragma unroll
+                for (int e = 0; e < VE; ++e) dst[lane * VE + e] = acc[g][e];
+                const float lsum = warp_sum(l[g]);
+                if (lane == 0) { dst[DH] = m[g]; dst[DH + 1] = lsum; }
+            }
+        }
+        __syncthreads();
     }
-    __syncthreads();
     if (s_abort) {
         // give copies that are still in flight time to land before the CTA's shared memory is handed on
         for (int i = 0; i < 2000; ++i) __nanosleep(100);
         return;
     }
-    // merge the eight warp states -> one result per head for this split
+    // merge the warp states -> one result per head for this split
     const int ns = pos / chunk + 1;  // splits of this row
     for (int t = tid; t < GQ * DH; t += kAttnThreads) {
         const int g = t / DH, e = t % DH;
@@ -285,7 +440,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_c
     if (tid == 0) a.tickets[row * a.Hkv + kvh] = 0;
 }
 
-inline size_t attn_smem_bytes(int DH, int GQ) {
+inline size_t attn_smem_bytes(int DH, int GQ) {  // (both consumer kinds: the tensor-core one leaves sq / sp unused)
     const size_t stage = 2 * kAttnConsumers * (size_t)(kPage * DH * 2);  // the warp states reuse the stages
     return 1024 + kAttnStages * stage + sizeof(float) * ((size_t)GQ * DH + (size_t)kAttnWarps * (kPage / 2) * GQ) +
            2 * kAttnStages * sizeof(uint64_t) + 64;

@@ -9,7 +9,7 @@
 // run as mma.sync with fp32 accumulators, the softmax is online in fp32 (base-2 exponentials, causal mask by position).
 // The GQ query heads of the group share every K/V tile.  K and V are the cache's bf16 values, exactly.
 #pragma once
-#include "river_common.cuh"
+#include "mma_sync.cuh"
 
 namespace river {
 
@@ -29,24 +29,8 @@ struct PrefillAttnArgs {
     int *dev_err;
 };
 
-__device__ __forceinline__ void pf_ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
-}
-__device__ __forceinline__ void pf_ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
-}
-__device__ __forceinline__ void pf_mma(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ void pf_cp16(uint32_t dst, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ uint32_t pf_pack_bf16(float lo, float hi) {
-    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
 }
 __device__ __forceinline__ float pf_ex2(float x) {
     float y;
@@ -87,7 +71,7 @@ __global__ void __launch_bounds__(32 * GQ) attn_prefill_kernel(const PrefillAttn
             v.x *= a.qscale; v.y *= a.qscale;
             const __nv_bfloat16 hx = __float2bfloat16_rn(v.x), hy = __float2bfloat16_rn(v.y);
             qhi[kk][h] = (uint32_t)__bfloat16_as_ushort(hx) | ((uint32_t)__bfloat16_as_ushort(hy) << 16);
-            qlo[kk][h] = pf_pack_bf16(v.x - __bfloat162float(hx), v.y - __bfloat162float(hy));
+            qlo[kk][h] = pack_bf16x2(v.x - __bfloat162float(hx), v.y - __bfloat162float(hy));
         }
     }
     float o[DT][4], m[2], l[2];
@@ -143,18 +127,18 @@ __global__ void __launch_bounds__(32 * GQ) attn_prefill_kernel(const PrefillAttn
 #pragma unroll
             for (int np = 0; np < NT / 2; ++np) {  // two n-tiles (16 keys) per ldmatrix.x4
                 const int key = np * 16 + (lane >> 4) * 8 + (lane & 7), dim = kk * 16 + ((lane >> 3) & 1) * 8;
-                pf_ldmatrix_x4(kf[np], pf_smem_u32(kb + (size_t)key * LD + dim));
+                ldsm_x4(kf[np], pf_smem_u32(kb + (size_t)key * LD + dim));
             }
             // eight independent accumulators per round: no mma waits for the one issued just before it
 #pragma unroll
             for (int np = 0; np < NT / 2; ++np) {
-                pf_mma(s[2 * np], qhi[kk], kf[np][0], kf[np][1]);
-                pf_mma(s[2 * np + 1], qhi[kk], kf[np][2], kf[np][3]);
+                mma_bf16_m16n8k16(s[2 * np], qhi[kk], kf[np][0], kf[np][1]);
+                mma_bf16_m16n8k16(s[2 * np + 1], qhi[kk], kf[np][2], kf[np][3]);
             }
 #pragma unroll
             for (int np = 0; np < NT / 2; ++np) {
-                pf_mma(s[2 * np], qlo[kk], kf[np][0], kf[np][1]);
-                pf_mma(s[2 * np + 1], qlo[kk], kf[np][2], kf[np][3]);
+                mma_bf16_m16n8k16(s[2 * np], qlo[kk], kf[np][0], kf[np][1]);
+                mma_bf16_m16n8k16(s[2 * np + 1], qlo[kk], kf[np][2], kf[np][3]);
             }
         }
         // ---- causal mask, online softmax (rows qr and qr + 8 of the block; a quad of lanes shares a row)
@@ -187,10 +171,10 @@ __global__ void __launch_bounds__(32 * GQ) attn_prefill_kernel(const PrefillAttn
             float r[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) r[e] = p[e] - __bfloat162float(__float2bfloat16_rn(p[e]));
-            pa[nt >> 1][(nt & 1) * 2 + 0] = pf_pack_bf16(p[0], p[1]);
-            pa[nt >> 1][(nt & 1) * 2 + 1] = pf_pack_bf16(p[2], p[3]);
-            pb[nt >> 1][(nt & 1) * 2 + 0] = pf_pack_bf16(r[0], r[1]);
-            pb[nt >> 1][(nt & 1) * 2 + 1] = pf_pack_bf16(r[2], r[3]);
+            pa[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16x2(p[0], p[1]);
+            pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16x2(p[2], p[3]);
+            pb[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16x2(r[0], r[1]);
+            pb[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16x2(r[2], r[3]);
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -213,17 +197,17 @@ __global__ void __launch_bounds__(32 * GQ) attn_prefill_kernel(const PrefillAttn
 #pragma unroll
                 for (int dp = 0; dp < 4; ++dp) {  // two n-tiles (16 dims) per ldmatrix.x4.trans
                     const int key = j * 16 + ((lane >> 3) & 1) * 8 + (lane & 7), dim = (d0 + dp) * 16 + (lane >> 4) * 8;
-                    pf_ldmatrix_x4_trans(vf[dp], pf_smem_u32(vb + (size_t)key * LD + dim));
+                    ldsm_x4_trans(vf[dp], pf_smem_u32(vb + (size_t)key * LD + dim));
                 }
 #pragma unroll
                 for (int dp = 0; dp < 4; ++dp) {
-                    pf_mma(o[2 * (d0 + dp)], pa[j], vf[dp][0], vf[dp][1]);
-                    pf_mma(o[2 * (d0 + dp) + 1], pa[j], vf[dp][2], vf[dp][3]);
+                    mma_bf16_m16n8k16(o[2 * (d0 + dp)], pa[j], vf[dp][0], vf[dp][1]);
+                    mma_bf16_m16n8k16(o[2 * (d0 + dp) + 1], pa[j], vf[dp][2], vf[dp][3]);
                 }
 #pragma unroll
                 for (int dp = 0; dp < 4; ++dp) {
-                    pf_mma(o[2 * (d0 + dp)], pb[j], vf[dp][0], vf[dp][1]);
-                    pf_mma(o[2 * (d0 + dp) + 1], pb[j], vf[dp][2], vf[dp][3]);
+                    mma_bf16_m16n8k16(o[2 * (d0 + dp)], pb[j], vf[dp][0], vf[dp][1]);
+                    mma_bf16_m16n8k16(o[2 * (d0 + dp) + 1], pb[j], vf[dp][2], vf[dp][3]);
                 }
             }
         }

@@ -21,10 +21,11 @@ cudaError_t launch_attn_split(river_ctx *c, int n, int layer0) {
     a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.tickets = c->attn_tickets; a.out = c->obuf; a.dev_err = c->dev_err;
     const size_t smem = attn_smem_bytes(DH, GQ);
-    const cudaError_t e = ensure_smem(c, attn_split_kernel<DH, GQ>, smem);
+    constexpr bool MMA = GQ <= 4;  // groups of up to four query heads: contractions on the warp-level tensor cores
+    const cudaError_t e = ensure_smem(c, attn_split_kernel<DH, GQ, MMA>, smem);
     if (e != cudaSuccess) return e;
-    return launch_k(attn_split_kernel<DH, GQ>, dim3(c->attn_splits_now, g.Hkv, n), dim3(kAttnThreads), smem, c->stream,
-                    true, c->kv_tmap, a);
+    return launch_k(attn_split_kernel<DH, GQ, MMA>, dim3(c->attn_splits_now, g.Hkv, n), dim3(attn_threads(MMA)), smem,
+                    c->stream, true, c->kv_tmap, a);
 }
 
 // Steps of 1-4 rows: the split-KV kernel that fetches the cached positions before the grid dependency resolves.
