@@ -131,13 +131,35 @@ struct TcResidEpi {  // out[row][row0 + r] = resid[row][row0 + r] + tile(r, n)
     float *out;
     int out_dim;
     __device__ int quad_row(int i, int q0, int) const { return 8 * q0 + 4 * i; }  // pairs (2 pr, 2 pr + 1): one range
+    // Four consecutive features per access; the residual values of a batch are all requested before the first sum is
+    // stored (`out` and `resid` never overlap, but the compiler cannot know: left alone it waits for every load).
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
-                        int pr0, int pr1) const {
-        const int row0 = tile_idx * kTcBM, nr = 2 * (pr1 - pr0);
-        for (int t = tid; t < n_live * nr; t += nthr) {
-            const int n = t / nr, r = 2 * pr0 + t % nr;
-            const size_t o = (size_t)rows[n] * out_dim + row0 + r;
-            out[o] = resid[o] + tile[n * ld + r];
+                        int pr0, int pr1, int = 0) const {
+        constexpr int UB = 4;
+        const int row0 = tile_idx * kTcBM, nr4 = (pr1 - pr0) / 2, total = n_live * nr4;  // slices are whole quads of pairs
+        for (int t0 = tid; t0 < total; t0 += UB * nthr) {
+            float4 res[UB];
+            size_t o[UB];
+            int src[UB];
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const int t = t0 + u * nthr;
+                res[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                o[u] = 0; src[u] = -1;
+                if (t < total) {
+                    const int n = t / nr4, r = 2 * pr0 + 4 * (t % nr4);
+                    o[u] = (size_t)rows[n] * out_dim + row0 + r;
+                    src[u] = n * ld + r;
+                    res[u] = __ldcg(reinterpret_cast<const float4 *>(resid + o[u]));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UB; ++u)
+                if (src[u] >= 0) {
+                    const float4 x = *reinterpret_cast<const float4 *>(tile + src[u]);
+                    *reinterpret_cast<float4 *>(out + o[u]) =
+                        make_float4(res[u].x + x.x, res[u].y + x.y, res[u].z + x.z, res[u].w + x.w);
+                }
         }
     }
 };
@@ -146,7 +168,7 @@ struct TcGateUpEpi {  // tile rows 0..63: gate features f0.., rows 64..127: up f
     int F;
     __device__ int quad_row(int i, int q0, int nq) const { return i < nq ? 4 * (q0 + i) : 64 + 4 * (q0 + i - nq); }
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
-                        int pr0, int pr1) const {
+                        int pr0, int pr1, int = 0) const {
         const int f0 = tile_idx * 64, np = pr1 - pr0;
         for (int t = tid; t < n_live * np; t += nthr) {
             const int n = t / np, r = pr0 + t % np;
@@ -166,37 +188,53 @@ struct TcQkvEpi {  // tiles walk the concatenated [q heads | k heads | v heads] 
         return (pr / half) * dh + pr % half + (i < nq ? 0 : half);
     }
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
-                        int pr0, int pr1) const {
+                        int pr0, int pr1, int = 0) const {
         const int half = dh >> 1, heads_per_tile = kTcBM / dh;
         const int feat0 = tile_idx * kTcBM;
         const int qdim = Hq * dh, kvdim = Hkv * dh;
         const int which = feat0 < qdim ? 0 : (feat0 < qdim + kvdim ? 1 : 2);
         const int base = which == 0 ? feat0 : (which == 1 ? feat0 - qdim : feat0 - qdim - kvdim);  // inside its matrix
-        const int np = pr1 - pr0;
-        for (int t = tid; t < n_live * np; t += nthr) {
-            const int n = t / np, pr = pr0 + t % np;
-            const int hh = pr / half, i = pr % half;  // head inside the tile, pair index
-            if (hh >= heads_per_tile) continue;
-            const int r_lo = hh * dh + i, r_hi = r_lo + half;
-            const int row = rows[n];
-            float lo = tile[n * ld + r_lo], hi = tile[n * ld + r_hi];
-            if (which != 2) {
-                const float2 cs = rope_cs[(size_t)row * half + i];
-                const float a = lo * cs.x - hi * cs.y, b = hi * cs.x + lo * cs.y;
-                lo = a; hi = b;
+        const int np = pr1 - pr0, total = n_live * np;
+        // batches of four (row, pair) items: everything an item reads from global memory (its rotation, its cache slot)
+        // is requested for the whole batch before the first result is stored
+        constexpr int UB = 4;
+        for (int t0 = tid; t0 < total; t0 += UB * nthr) {
+            int row[UB], src[UB], ii[UB], hl[UB], pos[UB], page[UB];
+            float2 cs[UB];
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const int t = t0 + u * nthr;
+                src[u] = -1; row[u] = 0; ii[u] = 0; hl[u] = 0; pos[u] = 0; page[u] = 0;
+                cs[u] = make_float2(1.f, 0.f);
+                if (t >= total) continue;
+                const int n = t / np, pr = pr0 + t % np;
+                const int hh = pr / half, i = pr % half;  // head inside the tile, pair index
+                if (hh >= heads_per_tile) continue;
+                row[u] = rows[n];
+                src[u] = n * ld + hh * dh + i;
+                ii[u] = i;
+                hl[u] = (base + hh * dh) / dh;
+                if (which != 2) cs[u] = rope_cs[(size_t)row[u] * half + i];
+                if (which != 0) { pos[u] = kv.row_pos[row[u]]; page[u] = kv.row_page[row[u]]; }
             }
-            const int hl = (base + hh * dh) / dh;
-            if (which == 0) {
-                float *q = q_out + (size_t)row * qdim + (size_t)hl * dh;
-                q[i] = lo;
-                q[i + half] = hi;
-            } else {
-                const int pos = kv.row_pos[row];
-                const int page = kv.row_page[row];
-                if (page < 0 || page >= kv.n_pages) { atomicExch(dev_err, DEV_BAD_PAGE); continue; }
-                const size_t o = kv.base(page, which - 1, hl, pos % kPage);
-                kv.pool[o + i] = __float2bfloat16_rn(lo);
-                kv.pool[o + i + half] = __float2bfloat16_rn(hi);
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                if (src[u] < 0) continue;
+                float lo = tile[src[u]], hi = tile[src[u] + half];
+                if (which != 2) {
+                    const float a = lo * cs[u].x - hi * cs[u].y, b = hi * cs[u].x + lo * cs[u].y;
+                    lo = a; hi = b;
+                }
+                if (which == 0) {
+                    float *q = q_out + (size_t)row[u] * qdim + (size_t)hl[u] * dh;
+                    q[ii[u]] = lo;
+                    q[ii[u] + half] = hi;
+                } else {
+                    if (page[u] < 0 || page[u] >= kv.n_pages) { atomicExch(dev_err, DEV_BAD_PAGE); continue; }
+                    const size_t o = kv.base(page[u], which - 1, hl[u], pos[u] % kPage);
+                    kv.pool[o + ii[u]] = __float2bfloat16_rn(lo);
+                    kv.pool[o + ii[u] + half] = __float2bfloat16_rn(hi);
+                }
             }
         }
     }
@@ -209,14 +247,15 @@ struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row
     int n_parts;
     __device__ int quad_row(int i, int q0, int) const { return 8 * q0 + 4 * i; }
     // (the LM head is never K-split: the argmax partial below needs all 128 rows of the tile)
+    // n0: operand row behind column 0 of `tile` (a tile may be handed over in column chunks)
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *, int tid, int nthr, int,
-                        int) const {
+                        int, int n0 = 0) const {
         float *logits = meta->logits;
         const int v0 = tile_idx * kTcBM;
         if (logits)
             for (int t = tid; t < n_live * kTcBM; t += nthr) {
                 const int n = t / kTcBM, r = t % kTcBM;
-                logits[(size_t)n * V + v0 + r] = tile[n * ld + r];
+                logits[(size_t)(n0 + n) * V + v0 + r] = tile[n * ld + r];
             }
         // one warp per column: a lane scans four consecutive features, then (max, lowest id) over the warp
         const int lane = tid & 31;
@@ -235,8 +274,8 @@ struct TcHeadEpi {  // logits (optional) and the tile's (max, lowest id) per row
                 if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
             }
             if (lane == 0) {
-                part_val[(size_t)n * n_parts + tile_idx] = bv;
-                part_idx[(size_t)n * n_parts + tile_idx] = bi;
+                part_val[(size_t)(n0 + n) * n_parts + tile_idx] = bv;
+                part_idx[(size_t)(n0 + n) * n_parts + tile_idx] = bi;
             }
         }
     }
@@ -248,6 +287,7 @@ struct TcArgs {
     int n_pad;        // N operand rows (multiple of 16, <= 256)
     int splits;       // K splits per tile = CTAs per cluster (<= 8)
     int n_stages;     // pipeline depth
+    int wide;         // 1: hi and lo operand rows as one operand of 2 n_pad rows (the host checks the TMEM budget)
     int a_rows_per_map;  // a tile's 128 rows come from map tile_idx / (rows_per_map / 128) ... see tile_map()
     int gateup;       // 1: a tile is 64 rows of map 0 + 64 rows of map 1
     int qkv_q_tiles, qkv_k_tiles;  // QKV: tiles per matrix (0 otherwise)
@@ -267,10 +307,11 @@ struct TcArgs {
 // sums replace its own partial values in place (peers only ever read the rows of THEIR slices).  A CTA may not
 // exit while a peer still reads its tile: it arrives at the second cluster barrier right after its own reads and waits
 // for it after its epilogue.  Even a CTA that gave up takes part in both barriers: a cluster barrier has no time-out.
+// `wide`: the accumulator has 2 NP columns, W hi^T in [0, NP) and W lo^T in [NP, 2 NP), to be added up here.
 template <class Epi>
 __device__ __forceinline__ void tc_finish(const Epi &epi, float *tile, uint32_t tmem_d, uint32_t tmem_cols, int NP,
                                           int splits, int split, int tile_idx, int n_live, const int32_t *rows, bool ok,
-                                          const int *s_abort, int nthr) {
+                                          const int *s_abort, int nthr, bool wide = false) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (warp >= 2 && warp < 6 && ok && n_live > 0) {
         const int q = warp & 3;  // TMEM lane quarter this warp may read
@@ -278,6 +319,12 @@ __device__ __forceinline__ void tc_finish(const Epi &epi, float *tile, uint32_t 
         for (int c0 = 0; c0 < NP; c0 += 16) {
             float v[16];
             tc_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+            if (wide) {
+                float w[16];
+                tc_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)(NP + c0), w);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] += w[j];
+            }
 #pragma unroll
             for (int j = 0; j < 16; ++j) col[(c0 + j) * kTcLd] = v[j];
         }
@@ -350,8 +397,13 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     const int kb_total = a.K / kTcBK;
     const int kb0 = (int)(((long long)kb_total * split) / a.splits), kb1 = (int)(((long long)kb_total * (split + 1)) / a.splits);
     const int nkb = kb1 - kb0;
+    // Up to 128 operand rows the hi and the lo boxes (adjacent in a stage) are ONE operand of 2 NP rows: a single MMA per
+    // 16 inputs, D = [W hi^T | W lo^T] in 2 NP columns, added up when the tile leaves TMEM.  (An instruction costs ~85
+    // cycles or more whatever its N, and it reads the weight box from shared memory once instead of twice.)
+    const bool wide = a.wide != 0;
+    const int acc_n = wide ? 2 * NP : NP;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < NP) tmem_cols <<= 1;
+    while ((int)tmem_cols < acc_n) tmem_cols <<= 1;
 
     pdl_launch();
     if (tid == 0) s_some = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
@@ -385,25 +437,24 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         if (tile_idx >= a.qkv_q_tiles + a.qkv_k_tiles) { ma = &map_a2; ay = (tile_idx - a.qkv_q_tiles - a.qkv_k_tiles) * kTcBM; }
         else if (tile_idx >= a.qkv_q_tiles) { ma = &map_a1; ay = (tile_idx - a.qkv_q_tiles) * kTcBM; }
     }
-    auto load_a = [&](int i) {  // weight tile of k-block kb0 + i into stage i % S (expects the stage's whole byte count)
-        const int s = i % S;
-        const uint32_t full = smem_u32(&bars[s]), dst = smem_u32(stages + (size_t)s * stage_bytes);
+    // The two issuing lanes advance their state incrementally (stage, parity, addresses: no division or multiplication
+    // per k-block): a single thread retires an instruction every few cycles, and a k-block it handles late is 16 KB of
+    // weights not streamed.
+    const uint32_t stage0 = smem_u32(stages), full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[S]);
+    int ax = kb0 * kTcBK;  // inner coordinate of the next weight tile to request
+    auto load_a = [&](uint32_t s) {  // ... into stage s (expects the stage's whole byte count)
+        const uint32_t full = full0 + 8 * s, dst = stage0 + s * stage_bytes;
         mbar_expect_tx(full, stage_bytes);
-        const int x = (kb0 + i) * kTcBK;
-        if (ma2) {
-            // two 64-row boxes: gate rows then up rows (each box 64 x 64 bf16 = 8 KB, 1024-aligned)
-            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                         ::"r"(dst), "l"(ma), "r"(x), "r"(ay), "r"(full) : "memory");
-            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                         ::"r"(dst + a_bytes / 2), "l"(ma2), "r"(x), "r"(ay2), "r"(full) : "memory");
+        if (ma2) {  // two 64-row boxes: gate rows then up rows (each box 64 x 64 bf16 = 8 KB, 1024-aligned)
+            tma_load_2d(dst, ma, ax, ay, full);
+            tma_load_2d(dst + a_bytes / 2, ma2, ax, ay2, full);
         } else {
-            tma_load_2d(dst, ma, x, ay, full);
+            tma_load_2d(dst, ma, ax, ay, full);
         }
+        ax += kTcBK;
     };
-    auto load_b = [&](int i) {
-        const int s = i % S;
-        const uint32_t full = smem_u32(&bars[s]), dst = smem_u32(stages + (size_t)s * stage_bytes) + a_bytes;
-        const int x = (kb0 + i) * kTcBK;
+    auto load_b = [&](uint32_t s, int x) {
+        const uint32_t full = full0 + 8 * s, dst = stage0 + s * stage_bytes + a_bytes;
         tma_load_2d(dst, &map_bhi, x, 0, full);
         tma_load_2d(dst + b_bytes, &map_blo, x, 0, full);
     };
@@ -411,7 +462,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     // weights first: they depend on nothing
     const int pre = min(S, nkb);
     if (tid == 0)
-        for (int i = 0; i < pre; ++i) load_a(i);
+        for (int i = 0; i < pre; ++i) load_a((uint32_t)i);
     pdl_wait();
     const int n_live = *a.cnt;  // rows of the backbone list; the stream kernel serves the exit-layer rows
     // even with no live row the requested weight tiles must land before the CTA may exit: run the pipeline once
@@ -419,29 +470,35 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int i = 0; i < nkb_run; ++i) {
-                if (i >= S) {
-                    if (!mbar_wait(smem_u32(&bars[S + i % S]), ((i / S) - 1) & 1, abortp, a.dev_err)) break;
-                    load_a(i);
-                }
-                load_b(i);
+            for (int i = 0; i < pre; ++i) load_b((uint32_t)i, (kb0 + i) * kTcBK);
+            uint32_t s = 0, par = 0;  // (k-block `pre` is the first to reuse a stage: stage 0, first completion of its barrier)
+            for (int i = pre; i < nkb_run; ++i) {
+                if (!mbar_wait(empty0 + 8 * s, par, abortp, a.dev_err)) break;
+                const int x = ax;
+                load_a(s);
+                load_b(s, x);
+                if (++s == (uint32_t)S) { s = 0; par ^= 1u; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = tc_idesc(NP);
+            const uint32_t idesc = tc_idesc(acc_n);
+            const uint64_t dfix = tc_smem_desc(0);  // everything but the address field
+            const uint32_t stage16 = stage_bytes >> 4, a16 = a_bytes >> 4, b16 = b_bytes >> 4;
+            uint32_t s = 0, par = 0, addr16 = stage0 >> 4;
             for (int i = 0; i < nkb_run; ++i) {
-                const int s = i % S;
-                if (!mbar_wait(smem_u32(&bars[s]), (i / S) & 1, abortp, a.dev_err)) break;
+                if (!mbar_wait(full0 + 8 * s, par, abortp, a.dev_err)) break;
                 tc_fence_after();
-                const uint32_t sa = smem_u32(stages + (size_t)s * stage_bytes);
-                const uint64_t da = tc_smem_desc(sa), dhi = tc_smem_desc(sa + a_bytes), dlo = tc_smem_desc(sa + a_bytes + b_bytes);
+                const uint64_t da = dfix | addr16, dhi = da + a16, dlo = dhi + b16;  // (addresses below 256 KB: no carry)
+                tc_mma(tmem_d, da, dhi, idesc, i > 0 ? 1u : 0u);
+                if (!wide) tc_mma(tmem_d, da, dlo, idesc, 1u);
 #pragma unroll
-                for (int k = 0; k < kTcBK / 16; ++k) {  // UMMA K = 16 bf16 = 32 bytes: +2 in the 16-byte address field
-                    tc_mma(tmem_d, da + 2 * k, dhi + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                    tc_mma(tmem_d, da + 2 * k, dlo + 2 * k, idesc, 1u);
+                for (int k = 1; k < kTcBK / 16; ++k) {  // UMMA K = 16 bf16 = 32 bytes: +2 in the 16-byte address field
+                    tc_mma(tmem_d, da + 2 * k, dhi + 2 * k, idesc, 1u);
+                    if (!wide) tc_mma(tmem_d, da + 2 * k, dlo + 2 * k, idesc, 1u);
                 }
-                tc_commit(smem_u32(&bars[S + s]));  // frees the stage once these MMAs have read it
+                tc_commit(empty0 + 8 * s);  // frees the stage once these MMAs have read it
+                if (++s == (uint32_t)S) { s = 0; par ^= 1u; addr16 = stage0 >> 4; } else addr16 += stage16;
             }
             tc_commit(smem_u32(&bars[2 * S]));      // accumulator complete
         }
@@ -449,11 +506,12 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     // The other lanes of the two single-lane warps park at a warp barrier: a spinning (and possibly suspending)
     // mbarrier wait in the same warp would steal the issuing lane's cycles.
     __syncwarp();
-    // everyone: wait for the accumulator (bounded), then move it out of TMEM
-    bool ok = mbar_wait(smem_u32(&bars[2 * S]), 0, abortp, a.dev_err);
+    // everyone: wait for the accumulator (bounded; sleeping between polls, so that the waiting warps leave the issue slots
+    // to the two issuing lanes), then move it out of TMEM
+    bool ok = mbar_wait_sleepy(smem_u32(&bars[2 * S]), 0, abortp, a.dev_err);
     tc_fence_after();
     __syncthreads();  // all TMA writes and MMA reads of the pipeline memory are over: it now holds the tile
-    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kTcThreads);
+    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kTcThreads, wide);
 }
 
 inline size_t tc_smem_bytes(int n_pad, int n_stages) {

@@ -60,6 +60,11 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
         if (tiles * s3 > tiles * a.splits && tiles * s3 <= c->num_sms * 3) { occ = 3; a.splits = s3; }
     }
     a.n_stages = stages_at(occ);
+    // hi | lo as one operand doubles the accumulator columns; all CTAs that can be resident on an SM must get their
+    // tensor memory at once (a CTA stuck in the allocation while its cluster waits for it could not be waited out)
+    int cols = 32;
+    while (cols < 2 * np) cols <<= 1;
+    a.wide = (2 * np <= 256 && occ * cols <= 512) ? 1 : 0;
     // the finished tile lives in the pipeline memory
     if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage) return cudaErrorInvalidValue;
     if (!allow_split) a.splits = 1;

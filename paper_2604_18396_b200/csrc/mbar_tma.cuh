@@ -43,6 +43,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     atomicExch(dev_err, DEV_WAIT_TIMEOUT);
     return false;
 }
+// The same for waits that are expected to last long: sleeps between polls so that the waiting warps leave the issue
+// slots to the warps that work (the limit counts polls of ~0.3 us).
+__device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *dev_err,
+                                                 uint32_t limit = kWaitLimit) {
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        __nanosleep(256);
+    }
+    *abort_flag = 1;
+    atomicExch(dev_err, DEV_WAIT_TIMEOUT);
+    return false;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"

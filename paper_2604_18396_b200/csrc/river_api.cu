@@ -1058,6 +1058,8 @@ int river_offload(river_ctx *c, int first_offloaded_layer, const river_layer_wei
 int river_clear_device_error(river_ctx *c) {
     if (!c) return RIVER_E_BADARG;
     CUDA_TRY(c, cudaMemsetAsync(c->dev_err, 0, sizeof(int), c->stream));
+    // a launch that gave up may have left tickets of unfinished attention merges behind
+    CUDA_TRY(c, cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)c->cfg.max_batch * c->cfg.Hkv, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     c->st.device_error = 0;
     return RIVER_OK;

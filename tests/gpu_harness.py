@@ -59,10 +59,16 @@ class Pair:
 
     def __init__(self, model, max_seqs: int, max_len: int, max_batch: int, exit_mode: int = 0,
                  entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0, kv_store: int = 0,
-                 n_pages: Optional[int] = None, prefill_chunk: int = 0):
+                 n_pages: Optional[int] = None, prefill_chunk: int = 0, storage_yardstick: bool = False):
         self.shape, (bb_c, rv_c), (bb_g, rv_g) = model
         self.L = len(bb_c["layers"])
         self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, kv_store)
+        # A second oracle with an fp32 cache that is forced down the first one's exit path: how far 16-bit cache storage
+        # ALONE moves every later K/V entry (no kernel involved).  On the random-weight 8B-class model a single bf16
+        # rounding of a cache entry is amplified layer by layer, so the two sides of a comparison (both store bf16, both
+        # round differently here and there) can only be held to that distance where it exceeds the plain tolerance.
+        self.twin = (orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, 0)
+                     if storage_yardstick and kv_store else None)
         pages_per_seq = (max_len + 15) // 16
         cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
                           n_pages=n_pages or max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
@@ -76,6 +82,8 @@ class Pair:
     def prefill(self, slots: List[int], prompts: List[np.ndarray], exit_layer: Optional[int] = None):
         for s, p in zip(slots, prompts):
             self.oracle.prefill(s, p, exit_layer)
+            if self.twin:
+                self.twin.prefill(s, p, exit_layer)
         tok = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
         offs = np.concatenate([[0], np.cumsum([len(p) for p in prompts])]).tolist()
         self.gpu.prefill(slots, tok, offs, exit_layer)
@@ -90,7 +98,11 @@ class Pair:
                 v = synth.normal(seed, 1000 * b + 2 * l + 1, (n, w), 1.0, "cuda")
                 self.gpu.write_kv(b, l + 1, 0, k, v)
                 self.oracle.write_kv(b, l, 0, k.float().cpu().numpy(), v.float().cpu().numpy())
+                if self.twin:
+                    self.twin.write_kv(b, l, 0, k.float().cpu().numpy(), v.float().cpu().numpy())
             self.oracle.set_len(b, n)
+            if self.twin:
+                self.twin.set_len(b, n)
             assert self.gpu.seq_len(b) == n
 
     def gpu_step(self, slots, tok, tau, forced=None, want_logits=True) -> StepOut:
@@ -109,6 +121,8 @@ class Pair:
 
     def oracle_step(self, slots, tok, tau, forced=None) -> StepOut:
         r = self.oracle.decode_step(slots, tok, tau, forced)
+        if self.twin:
+            self.twin.decode_step(slots, tok, INF, r["exit_layer"])
         return StepOut(r["logits"], r["next_tok"], r["exit_layer"], r["scores"])
 
     def oracle_scheduled_step(self, slots, tok, targets, margin: float = 2.5 * NEAR):
@@ -147,16 +161,19 @@ class Pair:
         worst = 0.0
         for l in range(1, self.L + 1):
             ko, vo = self.oracle.read_kv(slot, l - 1, 0, n)
+            kt, vt = self.twin.read_kv(slot, l - 1, 0, n) if self.twin else (None, None)
             kg, vg = self.gpu.read_kv(slot, l, 0, n)
             torch.cuda.synchronize()
-            for name, o, g in (("K", ko, kg), ("V", vo, vg)):
+            for name, o, g, tw in (("K", ko, kg, kt), ("V", vo, vg, vt)):
                 g = g.float().cpu().numpy()
                 assert np.isfinite(g).all(), f"{what}: {name} layer {l} slot {slot}: unwritten (NaN) cache entry"
                 rms = np.sqrt((o.astype(np.float64) ** 2).mean())
                 bound = KV_RTOL * np.abs(o) + KV_RTOL * rms
                 ratio = (np.abs(g - o) / bound).max()
-                worst = max(worst, ratio)
-                assert ratio <= 1.0, f"{what}: {name} layer {l} slot {slot}: error {ratio:.3f} x tolerance"
+                allowed = 1.0 if tw is None else max(1.0, float((np.abs(tw - o) / bound).max()))
+                worst = max(worst, ratio / allowed)
+                assert ratio <= allowed, (f"{what}: {name} layer {l} slot {slot}: error {ratio:.3f} x tolerance "
+                                          f"(16-bit storage alone: {allowed:.3f} x)")
         return worst
 
     def compare_lists(self, B: int):
@@ -174,6 +191,8 @@ class Pair:
     def close(self):
         self.gpu.close()
         self.oracle.close()
+        if self.twin:
+            self.twin.close()
 
 
 def natural_tau(model, prompts, steps_tok, frac_exit: float, entry_layer=None) -> float:

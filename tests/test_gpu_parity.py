@@ -36,12 +36,12 @@ def toks(shape, n, stream):
 
 
 def run_scheduled(m, prompt_lens, n_steps, kind="uniform", prefill_exit=None, page_seed=0, max_batch=None,
-                  seed=21, kv_store=0, flags=0):
+                  seed=21, kv_store=0, flags=0, storage_yardstick=False):
     shape = m[0]
     B = len(prompt_lens)
     L = len(m[1][0]["layers"])
     p = Pair(m, B, max(prompt_lens) + n_steps + 1, max_batch or max(B, 8), page_shuffle_seed=page_seed,
-             kv_store=kv_store, flags=flags)
+             kv_store=kv_store, flags=flags, storage_yardstick=storage_yardstick)
     prompts = [toks(shape, n, 100 + b) for b, n in enumerate(prompt_lens)]
     slots = list(range(B))
     p.prefill(slots, prompts, prefill_exit)
@@ -351,7 +351,10 @@ def test_8b_class_batch_rows_on_both_paths():
 def test_8b_class_six_rows_tensor_core_paths():
     # from five rows on: backbone rows on the tcgen05 GEMM, exit-layer rows on the dequantising tcgen05 GEMM, at the
     # full 8B layer shape (cluster K-splits of every projection, 128-head-dim cache writes from the GEMM epilogue)
-    r = run_scheduled(model("8b"), [6, 11, 3, 9, 4, 7], 2, "uniform", max_batch=8, kv_store=1, page_seed=5)
+    # (32 layers of the random-weight 8B shape amplify a single bf16 rounding of a cache entry: deep-layer K/V are held
+    # to the plain tolerance or to the distance that 16-bit storage alone produces, whichever is larger)
+    r = run_scheduled(model("8b"), [6, 11, 3, 9, 4, 7], 2, "uniform", max_batch=8, kv_store=1, page_seed=5,
+                      storage_yardstick=True)
     assert r["n_early"] > 0
     print("8b six rows:", r)
 
@@ -362,7 +365,7 @@ def run_on_history(m, lens, n_steps, flags=1, exit_mode=0, max_batch=None, page_
     shape = m[0]
     B = len(lens)
     p = Pair(m, B, max(lens) + n_steps + 1, max_batch or max(B, 8), page_shuffle_seed=page_seed, kv_store=1, flags=flags,
-             exit_mode=exit_mode)
+             exit_mode=exit_mode, storage_yardstick=shape.name == "8b")
     p.fill_history(lens)
     slots = list(range(B))
     n_early = 0
