@@ -89,6 +89,7 @@ struct TcW4Args {
     int n_pad;         // N operand rows (multiple of 16, <= 256)
     int splits;        // K splits per tile = CTAs per cluster (<= 8), in whole raw tiles
     int n_stages;      // operand stages
+    int wide;          // 1: hi and lo activation rows as one operand of 2 n_pad rows (the host checks the TMEM budget)
     int gateup;        // 1: a tile is 64 rows of matrix 0 + 64 rows of matrix 1
     int qkv_q_tiles, qkv_k_tiles;  // QKV: tiles per matrix (0 otherwise)
     const uint16_t *scale[3], *zero[3];  // bf16 [rows][K/64] of the up to three matrices behind the code maps
@@ -145,8 +146,10 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
     const int sb_total = a.K / (kTcBK * kW4Super);
     const int sb0 = (int)(((long long)sb_total * split) / a.splits), sb1 = (int)(((long long)sb_total * (split + 1)) / a.splits);
     const int nsb = sb1 - sb0, kb0 = sb0 * kW4Super, nkb = nsb * kW4Super;
+    const bool wide = a.wide != 0;  // as in tc_gemm_kernel: one MMA per 16 inputs, D = [W hi^T | W lo^T]
+    const int acc_n = wide ? 2 * NP : NP;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < NP) tmem_cols <<= 1;
+    while ((int)tmem_cols < acc_n) tmem_cols <<= 1;
 
     pdl_launch();
     if (tid == 0) {
@@ -245,20 +248,25 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = tc_idesc_f16(NP);
+            const uint32_t idesc = tc_idesc_f16(acc_n);
+            const uint64_t dfix = tc_smem_desc(0);  // everything but the address field
+            const uint32_t stage16 = stage_bytes >> 4, a16 = a_bytes >> 4, b16 = b_bytes >> 4;
+            const uint32_t afull0 = smem_u32(b_afull), bfull0 = smem_u32(b_bfull), empty0 = smem_u32(b_empty);
+            uint32_t s = 0, par = 0, addr16 = smem_u32(stages) >> 4;  // incremental: no division per k-block
             for (int i = 0; i < nkb_run; ++i) {
-                const int s = i % S;
-                if (!mbar_wait(smem_u32(&b_afull[s]), (i / S) & 1, abortp, a.dev_err)) break;
-                if (!mbar_wait(smem_u32(&b_bfull[s]), (i / S) & 1, abortp, a.dev_err)) break;
+                if (!mbar_wait(afull0 + 8 * s, par, abortp, a.dev_err)) break;
+                if (!mbar_wait(bfull0 + 8 * s, par, abortp, a.dev_err)) break;
                 tc_fence_after();
-                const uint32_t sa = smem_u32(stages + (size_t)s * stage_bytes);
-                const uint64_t da = tc_smem_desc(sa), dhi = tc_smem_desc(sa + a_bytes), dlo = tc_smem_desc(sa + a_bytes + b_bytes);
+                const uint64_t da = dfix | addr16, dhi = da + a16, dlo = dhi + b16;  // (addresses below 256 KB: no carry)
+                tc_mma(tmem_d, da, dhi, idesc, i > 0 ? 1u : 0u);
+                if (!wide) tc_mma(tmem_d, da, dlo, idesc, 1u);
 #pragma unroll
-                for (int k = 0; k < kTcBK / 16; ++k) {
-                    tc_mma(tmem_d, da + 2 * k, dhi + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                    tc_mma(tmem_d, da + 2 * k, dlo + 2 * k, idesc, 1u);
+                for (int k = 1; k < kTcBK / 16; ++k) {
+                    tc_mma(tmem_d, da + 2 * k, dhi + 2 * k, idesc, 1u);
+                    if (!wide) tc_mma(tmem_d, da + 2 * k, dlo + 2 * k, idesc, 1u);
                 }
-                tc_commit(smem_u32(&b_empty[s]));
+                tc_commit(empty0 + 8 * s);
+                if (++s == (uint32_t)S) { s = 0; par ^= 1u; addr16 = smem_u32(stages) >> 4; } else addr16 += stage16;
             }
             tc_commit(smem_u32(b_acc));
         }
@@ -280,8 +288,10 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
             if (lane == 0) ok = mbar_wait(bar, parity, abortp, a.dev_err) ? 1 : 0;
             return __shfl_sync(0xffffffffu, ok, 0) != 0;
         };
+        int s = 0;
+        uint32_t epar = 1;  // parity of the stage's `empty` barrier to wait for from the second round on: ((i / S) - 1) & 1
         for (int i = 0; i < nkb_run && alive; ++i) {
-            const int kq = i & (kW4Super - 1), sb = i / kW4Super, rb = sb % kW4RawBufs, s = i % S;
+            const int kq = i & (kW4Super - 1), sb = i / kW4Super, rb = sb % kW4RawBufs;
             if (kq == 0) {
                 s_cur = s_next; z_cur = z_next;
                 if (sb + 1 < nsb) {  // the next raw tile's scales / zeros travel while this one is processed
@@ -290,7 +300,7 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
                 }
                 if (!warp_wait(smem_u32(&b_rfull[rb]), (sb / kW4RawBufs) & 1)) { alive = false; break; }
             }
-            if (i >= S && !warp_wait(smem_u32(&b_empty[s]), ((i / S) - 1) & 1)) { alive = false; break; }
+            if (i >= S && !warp_wait(smem_u32(&b_empty[s]), epar)) { alive = false; break; }
             const uint32_t sw = (kq < 2 ? s_cur.x : s_cur.y), zw = (kq < 2 ? z_cur.x : z_cur.y);
             const float sf = (kq & 1) ? bf16hi(sw) : bf16lo(sw), zf = (kq & 1) ? bf16hi(zw) : bf16lo(zw);
             const __half2 s2 = __float2half2_rn(sf), z2 = __float2half2_rn(zf);  // bf16 values are exact in f16 range here
@@ -309,13 +319,14 @@ __global__ void __launch_bounds__(kW4Threads) tc_gemm_w4_kernel(const __grid_con
                 mbar_arrive(smem_u32(&b_afull[s]));
                 if (kq == kW4Super - 1) mbar_arrive(smem_u32(&b_rempty[rb]));
             }
+            if (++s == S) { s = 0; epar ^= 1u; }
         }
     }
     __syncwarp();
     bool ok = n_live > 0 ? mbar_wait(smem_u32(b_acc), 0, abortp, a.dev_err) : true;
     tc_fence_after();
     __syncthreads();  // all copies into and MMA reads of the pipeline memory are over: it now holds the tile
-    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kW4Threads);
+    tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kW4Threads, wide);
 }
 
 inline size_t tc_w4_smem_bytes(int n_pad, int n_stages) {

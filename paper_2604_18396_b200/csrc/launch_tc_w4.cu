@@ -31,6 +31,9 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
     const int raw_tiles = K / (kTcBK * kW4Super);
     a.splits = tc_pick_splits(c, tiles, raw_tiles, c->num_sms * (two ? 2 : 1), raw_tiles <= 8 ? 2 : 4);
     if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage + raw) return cudaErrorInvalidValue;
+    int cols = 32;  // (see launch_tc: every CTA resident on an SM must get its accumulator columns at once)
+    while (cols < 2 * np) cols <<= 1;
+    a.wide = (2 * np <= 256 && (two ? 2 : 1) * cols <= 512) ? 1 : 0;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
     a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
