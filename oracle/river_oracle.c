@@ -47,6 +47,12 @@ typedef struct {
     int32_t exit_mode;   /* 0 = per token, 1 = whole batch switches together (Eq. 1 literal) */
     int32_t kv_store;    /* 0 = cache holds fp32 values; 1 = cache entries are rounded to bf16 when stored: the
                             method keeps the KV cache in a 16-bit format (Section 4.1) */
+    int32_t kv_strategy; /* what happens in the blocks a token skips (Section 3, the strategies the method is compared
+                            with): 0 = the KV-Shared Exit River (Section 4.1: the quantised copy of the block runs and
+                            writes K/V into the shared slot); 1 = State Propagation: the hidden state at the exit is the
+                            input of every later block's K/V projection (backbone weights), nothing else runs there;
+                            2 = Mono-Decreasing Exit: nothing runs in a skipped block, and a token leaves no later than
+                            the previous token of its sequence did, so no cache entry it needs is ever missing */
 } orc_config;
 
 /* backbone pointers per layer: attn_norm, wq, wk, wv, wo, ffn_norm, wg, wu, wd (all bf16) */
@@ -62,6 +68,7 @@ typedef struct {
     float *K, *V;    /* [L][max_seqs][max_len][Hkv*dh] */
     uint8_t *written;/* [L][max_seqs][max_len] number of writes (saturating) */
     int32_t *len;    /* [max_seqs] */
+    int32_t *cap;    /* [max_seqs] Mono-Decreasing Exit: the depth the sequence's last token reached (L to begin with) */
     /* lists of the last decode step: rows in the backbone / in the river entering layer l (1-based) */
     int32_t *act_idx, *riv_idx, *n_act, *n_riv; /* [(L+1)][maxB], [(L+1)] */
     int32_t lists_cap;
@@ -250,6 +257,30 @@ static void block(orc_ctx *o, int l0, int river, int slot, int pos, const float 
     free(x); free(q); free(att); free(hmid); free(tmp); free(gate); free(up);
 }
 
+/*
+ * State Propagation (Section 3): block l0 + 1 is skipped, but its K/V for this position are computed from the hidden
+ * state the token left the backbone with - that block's attention norm and its backbone K / V projections - and
+ * stored in the block's cache slot.  No attention, no feed-forward: the hidden state itself is unchanged.
+ */
+static void propagate_kv(orc_ctx *o, int l0, int slot, int pos, const float *h) {
+    const orc_config *c = &o->c;
+    const int d = c->d, Hkv = c->Hkv, dh = c->dh;
+    mat_t m[7];
+    get_mats(o, l0, 0, m);
+    float *x = (float *)malloc(sizeof(float) * (size_t)d);
+    rmsnorm(h, (const uint16_t *)o->bb[l0 * BB_N + BB_ATTN_NORM], d, c->rms_eps, x);
+    float *kdst = o->K + kv_off(o, l0, slot, pos);
+    float *vdst = o->V + kv_off(o, l0, slot, pos);
+    matvec(&m[1], Hkv * dh, d, x, kdst);
+    matvec(&m[2], Hkv * dh, d, x, vdst);
+    for (int j = 0; j < Hkv; ++j) rope(kdst + (size_t)j * dh, dh, pos, c->rope_theta);
+    if (c->kv_store == 1)
+        for (int i = 0; i < Hkv * dh; ++i) { kdst[i] = round_to_bf16(kdst[i]); vdst[i] = round_to_bf16(vdst[i]); }
+    uint8_t *w = &o->written[((size_t)l0 * c->max_seqs + slot) * c->max_len + pos];
+    if (*w < 255) ++*w;
+    free(x);
+}
+
 /* Eq. 1: s = <a,b> / (|a| |b|); zero norm -> 0 */
 static float transition_similarity(const float *a, const float *b, int d) {
     double ab = 0.0, aa = 0.0, bb = 0.0;
@@ -305,13 +336,16 @@ orc_ctx *orc_create(const orc_config *cfg, const void *embed, const void *lm_hea
     o->V = (float *)calloc(n * cfg->Hkv * cfg->dh, sizeof(float));
     o->written = (uint8_t *)calloc(n, 1);
     o->len = (int32_t *)calloc((size_t)cfg->max_seqs, sizeof(int32_t));
-    if (!o->K || !o->V || !o->written) return NULL;
+    o->cap = (int32_t *)malloc(sizeof(int32_t) * (size_t)cfg->max_seqs);
+    if (!o->K || !o->V || !o->written || !o->cap) return NULL;
+    for (int s = 0; s < cfg->max_seqs; ++s) o->cap[s] = cfg->L;
+    if (cfg->kv_strategy < 0 || cfg->kv_strategy > 2) return NULL;
     return o;
 }
 
 void orc_destroy(orc_ctx *o) {
     if (!o) return;
-    free(o->K); free(o->V); free(o->written); free(o->len);
+    free(o->K); free(o->V); free(o->written); free(o->len); free(o->cap);
     free((void *)o->bb); free((void *)o->rv);
     free(o->act_idx); free(o->riv_idx); free(o->n_act); free(o->n_riv);
     free(o);
@@ -321,6 +355,7 @@ int orc_seq_len(const orc_ctx *o, int slot) { return o->len[slot]; }
 void orc_set_len(orc_ctx *o, int slot, int n) { o->len[slot] = n; }
 void orc_release(orc_ctx *o, int slot) {
     o->len[slot] = 0;
+    o->cap[slot] = o->c.L;
     for (int l = 0; l < o->c.L; ++l)
         memset(&o->written[((size_t)l * o->c.max_seqs + slot) * o->c.max_len], 0, (size_t)o->c.max_len);
 }
@@ -385,6 +420,11 @@ int orc_decode_step(orc_ctx *o, int B, const int32_t *slots, const int32_t *tok,
         }
         o->n_act[l - 1] = na; o->n_riv[l - 1] = nr;
         for (int b = 0; b < B; ++b) {
+            if (exited[b] && c->kv_strategy != 0) {  /* a skipped block under one of the other strategies */
+                if (c->kv_strategy == 1) propagate_kv(o, l - 1, slots[b], o->len[slots[b]], h + (size_t)b * d);
+                memcpy(h2 + (size_t)b * d, h + (size_t)b * d, sizeof(float) * (size_t)d);
+                continue;
+            }
             if (exited[b] && !river_exists(o, l - 1)) { free(h); free(h2); free(exited); free(s_now); return -6; }
             block(o, l - 1, exited[b], slots[b], o->len[slots[b]], h + (size_t)b * d, h2 + (size_t)b * d);
         }
@@ -408,6 +448,8 @@ int orc_decode_step(orc_ctx *o, int B, const int32_t *slots, const int32_t *tok,
                 if (c->exit_mode == 0) leave = eligible && (s_now[b] > tau[b]);
                 else leave = eligible && any_active && all_pass;
             }
+            /* Mono-Decreasing Exit: never deeper than the sequence's previous token */
+            if (c->kv_strategy == 2 && l < L && l >= o->cap[slots[b]]) leave = 1;
             if (leave) { exited[b] = 1; exit_layer[b] = l; }
         }
         float *t = h; h = h2; h2 = t;
@@ -423,6 +465,7 @@ int orc_decode_step(orc_ctx *o, int B, const int32_t *slots, const int32_t *tok,
     for (int b = 0; b < B; ++b) {
         lm_head(o, h + (size_t)b * d, logits ? logits + (size_t)b * c->V : NULL, &next_tok[b]);
         o->len[slots[b]] += 1;
+        if (c->kv_strategy == 2) o->cap[slots[b]] = exit_layer[b];
     }
     free(h); free(h2); free(exited); free(s_now);
     return 0;

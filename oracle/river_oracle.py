@@ -49,7 +49,7 @@ def build(verbose: bool = False) -> str:
 class OrcConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("L", "d", "Hq", "Hkv", "dh", "F", "V")] + [
         ("rms_eps", C.c_float), ("rope_theta", C.c_float)] + [
-        (n, C.c_int32) for n in ("entry_layer", "group", "max_seqs", "max_len", "exit_mode", "kv_store")]
+        (n, C.c_int32) for n in ("entry_layer", "group", "max_seqs", "max_len", "exit_mode", "kv_store", "kv_strategy")]
 
 
 _lib = None
@@ -101,20 +101,22 @@ def _p(a) -> int:
 
 
 def make_config(shape, max_seqs: int, max_len: int, exit_mode: int = 0, entry_layer: Optional[int] = None,
-                n_layers: Optional[int] = None, kv_store: int = 0) -> OrcConfig:
+                n_layers: Optional[int] = None, kv_store: int = 0, kv_strategy: int = 0) -> OrcConfig:
     return OrcConfig(L=n_layers or shape.L, d=shape.d, Hq=shape.Hq, Hkv=shape.Hkv, dh=shape.dh, F=shape.F,
                      V=shape.V, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta,
                      entry_layer=shape.entry_layer if entry_layer is None else entry_layer, group=shape.group,
-                     max_seqs=max_seqs, max_len=max_len, exit_mode=exit_mode, kv_store=kv_store)
+                     max_seqs=max_seqs, max_len=max_len, exit_mode=exit_mode, kv_store=kv_store,
+                     kv_strategy=kv_strategy)
 
 
 class Oracle:
     """The oracle over one model (CPU tensors: bf16 backbone, (codes, scale, zero) river)."""
 
     def __init__(self, shape, backbone: dict, river: List[Optional[dict]], max_seqs: int, max_len: int,
-                 exit_mode: int = 0, entry_layer: Optional[int] = None, kv_store: int = 0):
+                 exit_mode: int = 0, entry_layer: Optional[int] = None, kv_store: int = 0, kv_strategy: int = 0):
         self.L = len(backbone["layers"])
-        self.cfg = make_config(shape, max_seqs, max_len, exit_mode, entry_layer, n_layers=self.L, kv_store=kv_store)
+        self.cfg = make_config(shape, max_seqs, max_len, exit_mode, entry_layer, n_layers=self.L, kv_store=kv_store,
+                               kv_strategy=kv_strategy)
         self.shape = shape
         self._keep = (backbone, river)
         bb = (C.c_void_p * (self.L * 9))()

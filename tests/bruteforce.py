@@ -36,9 +36,13 @@ def _bf16(x):
     return torch.from_numpy(x).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
 
 
-def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False):
+def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False, strategy=0):
     """-> logits [T,V], K [L,T,Hkv*dh] (after RoPE), V [L,T,Hkv*dh], scores [T,L].
-    kv_bf16: keys and values are rounded to bf16 (through torch's cast) before they are used or returned."""
+    kv_bf16: keys and values are rounded to bf16 (through torch's cast) before they are used or returned.
+    strategy (what a skipped block does, Section 3): 0 = the quantised copy of the block runs (Section 4.1); 1 = State
+    Propagation: K/V of the block from the hidden state at the exit through the BACKBONE's K / V projections, the
+    hidden state itself unchanged; 2 = Mono-Decreasing Exit: nothing (the block's K/V rows of that token come back as
+    NaN; no later token may need them, which holds when the exit layers never increase)."""
     tokens = np.asarray(tokens)
     e = np.asarray(exit_layers)
     T = len(tokens)
@@ -54,7 +58,7 @@ def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False):
 
         def proj(name, X):
             Y = X @ f64(lay[name]).T
-            if in_river.any():
+            if in_river.any() and strategy == 0:
                 Wr = dequant_np(*rv[l - 1][name], shape.group)
                 Y = np.where(in_river[:, None], X @ Wr.T, Y)
             return Y
@@ -65,9 +69,13 @@ def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False):
         v = proj("wv", x)
         if kv_bf16:
             k, v = _bf16(k), _bf16(v)
+        if strategy == 2:
+            assert all(e[j] <= e[i] for i in range(T) for j in range(i + 1, T)), "exit layers must not increase"
+            k = np.where(in_river[:, None], np.nan, k)
+            v = np.where(in_river[:, None], np.nan, v)
         Ks.append(k)
         Vs.append(v)
-        k3, v3 = k.reshape(T, Hkv, dh), v.reshape(T, Hkv, dh)
+        k3, v3 = np.nan_to_num(k).reshape(T, Hkv, dh), np.nan_to_num(v).reshape(T, Hkv, dh)
         att = np.empty((T, Hq, dh))
         for i in range(Hq):
             j = i // (Hq // Hkv)
@@ -83,6 +91,6 @@ def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False):
         Hn = Hm + proj("wd", g / (1.0 + np.exp(-g)) * u)
         s = (H * Hn).sum(1) / (np.linalg.norm(H, axis=1) * np.linalg.norm(Hn, axis=1))
         scores[:, l - 1] = np.where(in_river, np.nan, s)
-        H = Hn
+        H = Hn if strategy == 0 else np.where(in_river[:, None], H, Hn)
     logits = _rms(H, f64(bb["final_norm"]), shape.rms_eps) @ f64(bb["lm_head"]).T
     return logits, np.stack(Ks), np.stack(Vs), scores

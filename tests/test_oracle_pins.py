@@ -472,3 +472,65 @@ def test_prefill_auto_limits(tiny):
     la, na, depth = a.prefill_auto(0, prompt, -2.0)      # everything passes: the entry layer
     lb, nb = b.prefill(0, prompt, max(shape.entry_layer, 1))
     assert depth == max(shape.entry_layer, 1) and np.array_equal(la, lb) and na == nb
+
+
+# ------------------------------------------------------------------ the other KV strategies (Section 3)
+def test_state_propagation_matches_whole_sequence_recompute(tiny):
+    # kv_strategy = 1: a skipped block's K/V come from the hidden state at the exit through the backbone's K / V
+    # projections; checked against the cache-free numpy recompute (logits, every K / V entry, scores)
+    shape, bb, rv = tiny
+    toks = _tokens(shape, 11, 7)
+    rng = np.random.default_rng(3)
+    e = rng.integers(max(shape.entry_layer, 1), shape.L + 1, len(toks))
+    o = orc.Oracle(shape, bb, rv, 1, 16, kv_strategy=1)
+    lg = []
+    for t, tk in enumerate(toks):
+        r = o.decode_step([0], [tk], INF, [int(e[t])])
+        assert r["exit_layer"][0] == e[t]
+        lg.append(r["logits"][0])
+    logits, K, V, sc = bruteforce.recompute(shape, bb, rv, toks, e, strategy=1)
+    assert np.abs(np.stack(lg) - logits).max() < 2e-4
+    for l in range(shape.L):
+        k, v = o.read_kv(0, l, 0, len(toks))
+        assert np.abs(k - K[l]).max() < 2e-4 and np.abs(v - V[l]).max() < 2e-4
+        assert all(o.write_count(0, l, p) == 1 for p in range(len(toks)))  # every (token, layer) slot written once
+    # and it is NOT the river: with some early exits the logits differ from strategy 0 on the same path
+    o0 = orc.Oracle(shape, bb, rv, 1, 16)
+    d = max(np.abs(o0.decode_step([0], [tk], INF, [int(e[t])])["logits"][0] - lg[t]).max() for t, tk in enumerate(toks))
+    assert (e < shape.L).any() and d > 1e-3
+    o.close(); o0.close()
+
+
+def test_mono_decreasing_exit_caps_depth_and_writes_no_skipped_slot(tiny):
+    # kv_strategy = 2: a token leaves no later than the previous token of its sequence did (whatever its score or
+    # the forced schedule says), skipped blocks write nothing, and the result equals the cache-free recompute
+    shape, bb, rv = tiny
+    L = shape.L
+    toks = _tokens(shape, 9, 8)
+    wish = [L, L, 3, L, 2, 3, 2, 1, L]  # requested exit layers; the cap makes them non-increasing
+    want, cap = [], L
+    for w in wish:
+        cap = min(cap, w)
+        want.append(cap)
+    o = orc.Oracle(shape, bb, rv, 2, 16, entry_layer=1, kv_strategy=2)
+    lg, got = [], []
+    for t, tk in enumerate(toks):
+        r = o.decode_step([1], [tk], INF, [wish[t]])
+        got.append(int(r["exit_layer"][0]))
+        lg.append(r["logits"][0])
+    assert got == want
+    logits, K, V, _ = bruteforce.recompute(shape, bb, rv, toks, want, strategy=2)
+    assert np.abs(np.stack(lg) - logits).max() < 2e-4
+    for l in range(L):
+        k, v = o.read_kv(1, l, 0, len(toks))
+        for p in range(len(toks)):
+            ran = want[p] >= l + 1
+            assert o.write_count(1, l, p) == (1 if ran else 0)
+            if ran:
+                assert np.abs(k[p] - K[l][p]).max() < 2e-4 and np.abs(v[p] - V[l][p]).max() < 2e-4
+    # a second sequence starts with a fresh cap; releasing a slot resets it
+    r = o.decode_step([0], [toks[0]], INF)
+    assert r["exit_layer"][0] == L
+    o.release(1)
+    assert o.decode_step([1], [toks[0]], INF)["exit_layer"][0] == L
+    o.close()
