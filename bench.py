@@ -95,20 +95,29 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(mhz)}
 
 
-def alg_bytes_step(shape, L, exit_layers, positions, want_logits=True):
+def alg_bytes_step(shape, L, exit_layers, positions, want_logits=True, kv_strategy=0):
     """Algorithmic HBM bytes of one decode step from its exit pattern: weights of every (layer, weight set) that
-    ran, KV read by every row in every layer (exit-layer rows attend too), KV written, LM head, embedding rows."""
+    ran, KV read by every row in every layer it attends in (exit-layer rows attend too), KV written, LM head,
+    embedding rows.  kv_strategy 1 (State Propagation): a skipped block costs its bf16 K and V matrices and a KV
+    write, no attention; 2 (Mono-Decreasing Exit): nothing."""
     P = shape.layer_params()
     B = len(exit_layers)
+    kv_tok = 2.0 * shape.Hkv * shape.dh * 2.0
     total = 0.0
     for l in range(1, L + 1):
         n_act = sum(1 for e in exit_layers if e >= l)
         if n_act > 0:
             total += 2.0 * P
         if n_act < B:
-            total += P / 2.0 + 4.0 * P / shape.group
-    kv_tok = 2.0 * shape.Hkv * shape.dh * 2.0
-    total += L * sum((p + 1) * kv_tok + kv_tok for p in positions)
+            if kv_strategy == 0:
+                total += P / 2.0 + 4.0 * P / shape.group
+            elif kv_strategy == 1:
+                total += 2.0 * 2.0 * shape.Hkv * shape.dh * shape.d
+        for e, p in zip(exit_layers, positions):
+            if kv_strategy == 0 or e >= l:
+                total += (p + 1) * kv_tok + kv_tok
+            elif kv_strategy == 1:
+                total += kv_tok
     total += 2.0 * shape.V * shape.d + B * shape.d * 2.0 + (4.0 * B * shape.V if want_logits else 0.0)
     return total
 
@@ -283,7 +292,7 @@ def ours(args, wl):
     n_pages = sum((l + total_steps + 15) // 16 for l in lens)
     flags = args.flags
     cfg = make_config(shape, max_seqs=B, max_pages_per_seq=pages_per_seq, n_pages=n_pages, max_batch=max(B, 8),
-                      page_shuffle_seed=seed + 1, flags=flags, prefill_chunk=256)
+                      page_shuffle_seed=seed + 1, flags=flags, prefill_chunk=256, kv_strategy=args.kv_strategy)
     rv = River(cfg, bb, rvw)
     if off_host is not None:
         rv.offload(args.offload_from, off_host)
@@ -343,7 +352,8 @@ def ours(args, wl):
     ex = exits[step:step + K].cpu().numpy()
     step += K
     ms = dist_max(ms)
-    bytes_exit = sum(alg_bytes_step(shape, L, ex[t], [p + t for p in pos0]) for t in range(K)) / K
+    bytes_exit = sum(alg_bytes_step(shape, L, ex[t], [p + t for p in pos0], kv_strategy=args.kv_strategy)
+                     for t in range(K)) / K
 
     timed_steps(rv, slots_c, slots, toks, inf, logits, nxt, exits, step, W)
     step += W
@@ -411,6 +421,7 @@ def ours(args, wl):
                        "early_exit_target_fraction": EARLY_FRACTION, "thresholds": "per-step, from calibrated mean scores",
                        "l2": "inputs (weights + KV) larger than L2, no flush", "flags": flags, "layers": L,
                        "parallelism": "replicas only" if world > 1 else "1 GPU", "prefill_s": round(t_pf, 3),
+                       "kv_strategy": ["exit river", "state propagation", "mono-decreasing exit"][args.kv_strategy],
                        **({"offload": {"first_offloaded_layer": args.offload_from, "device_bytes_saved": off_saved,
                                        "block_copies_per_step": (off_fetches - off_fetches0) / K}}
                           if args.offload_from else {})},
@@ -587,6 +598,9 @@ def main():
     ap.add_argument("--micro-pool-gib", type=int, default=64, help="attn_micro: cap of the KV pool (fewer blocks are run when a point needs more)")
     ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv-strategy", type=int, default=0, choices=[0, 1, 2],
+                    help="what a skipped block does: 0 = the 4-bit exit river (the method), 1 = State Propagation, "
+                         "2 = Mono-Decreasing Exit (river_config.kv_strategy)")
     ap.add_argument("--offload-from", type=int, default=0,
                     help="keep backbone blocks >= this layer in pinned host memory (river_offload); 0 = all resident")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")

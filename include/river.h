@@ -69,7 +69,24 @@ typedef struct river_config {
     int32_t prefill_chunk;     /* prompt positions river_prefill runs per pass through the blocks (0 = max_batch, at most
                                   256): every pass streams the weights once, so larger chunks make prefill cheaper; the
                                   workspace grows with max(max_batch, prefill_chunk) */
+    int32_t kv_strategy;       /* what happens in the blocks a token skips (Section 3; RIVER_KV_*): the method's KV-Shared
+                                  Exit River, or one of the strategies it is compared with, on the same kernels */
 } river_config;
+
+/* river_config.kv_strategy.  In all of them the rows that have left still get their logits from the original LM head.
+ *   RIVER_KV_RIVER             (Section 4.1) the 4-bit copy of every skipped block runs and writes the token's K/V into
+ *                              the backbone's cache slot.
+ *   RIVER_KV_STATE_PROPAGATION (Section 3) the hidden state at the exit is the input of every later block's K / V
+ *                              projection (that block's norm and bf16 weights); no attention, no feed-forward there,
+ *                              the hidden state reaches the LM head unchanged.  Needs no exit-layer weights.
+ *   RIVER_KV_MONO_DECREASING   (Section 3) nothing runs in a skipped block, and a token leaves no later than the previous
+ *                              token of its sequence did (whatever its score, and before a later forced exit), so no
+ *                              cache entry it attends to is ever missing; the cap of a sequence starts at L, follows
+ *                              every token (prefill: the prefill depth) and is reset by river_release.
+ * (KV Mask, the fourth strategy of Section 3, is not built.) */
+#define RIVER_KV_RIVER 0
+#define RIVER_KV_STATE_PROPAGATION 1
+#define RIVER_KV_MONO_DECREASING 2
 
 typedef struct river_w4 {
     const void *codes, *scale, *zero; /* [dev] */

@@ -26,7 +26,7 @@ class river_config(C.Structure):
         ("rms_eps", C.c_float), ("rope_theta", C.c_float)] + [
         (n, C.c_int32) for n in ("entry_layer", "group", "page_size", "max_seqs", "max_pages_per_seq", "n_pages",
                                  "max_batch", "exit_mode")] + [("page_shuffle_seed", C.c_uint32),
-                                                               ("flags", C.c_uint32), ("prefill_chunk", C.c_int32)]
+                                                               ("flags", C.c_uint32), ("prefill_chunk", C.c_int32), ("kv_strategy", C.c_int32)]
 
 
 class river_w4(C.Structure):
@@ -117,14 +117,15 @@ class RiverError(RuntimeError):
 
 def make_config(shape, *, max_seqs: int, max_pages_per_seq: int, n_pages: int, max_batch: int,
                 n_layers: Optional[int] = None, entry_layer: Optional[int] = None, exit_mode: int = 0,
-                page_shuffle_seed: int = 0, flags: int = 0, prefill_chunk: int = 0) -> river_config:
+                page_shuffle_seed: int = 0, flags: int = 0, prefill_chunk: int = 0,
+                kv_strategy: int = 0) -> river_config:
     """river_config from a model shape (anything with L,d,Hq,Hkv,dh,F,V,rms_eps,rope_theta,entry_layer,group)."""
     return river_config(L=n_layers or shape.L, d=shape.d, Hq=shape.Hq, Hkv=shape.Hkv, dh=shape.dh, F=shape.F,
                         V=shape.V, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta,
                         entry_layer=shape.entry_layer if entry_layer is None else entry_layer, group=shape.group,
                         page_size=16, max_seqs=max_seqs, max_pages_per_seq=max_pages_per_seq, n_pages=n_pages,
                         max_batch=max_batch, exit_mode=exit_mode, page_shuffle_seed=page_shuffle_seed, flags=flags,
-                        prefill_chunk=prefill_chunk)
+                        prefill_chunk=prefill_chunk, kv_strategy=kv_strategy)
 
 
 def _dp(t: Optional[torch.Tensor]) -> int:

@@ -43,6 +43,7 @@ struct AttnArgs {
     unsigned *tickets;     // [rows][Hkv], zero between launches: the last split of a (row, kv head) merges them all
     float *out;            // [rows][Hq*DH]
     int *dev_err;
+    const uint8_t *skip;   // rows whose flag is set do not attend (they have left and run nothing here), or null
 };
 
 template <int DH, int GQ, bool MMA>
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
     // independent loads first, decisions after (every index below is valid for any row of the grid)
     const int n_rows = a.meta->n_rows, chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
     const int pos = a.row_pos[row], slot = a.row_slot[row];
-    if (row >= n_rows) return;
+    if (row >= n_rows || (a.skip && a.skip[row])) return;
     const int p0 = split * chunk;
     if (p0 > pos) return;
     const int p1 = min(p0 + chunk, pos + 1);     // positions [p0, p1)

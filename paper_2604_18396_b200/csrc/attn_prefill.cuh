@@ -27,6 +27,7 @@ struct PrefillAttnArgs {
     int Hq;
     float qscale;                // log2(e) / sqrt(DH)
     int *dev_err;
+    const uint8_t *skip;         // a tile whose first row's flag is set does not attend (its rows have left), or null
 };
 
 __device__ __forceinline__ void pf_cp16(uint32_t dst, const void *src) {
@@ -54,6 +55,7 @@ __global__ void __launch_bounds__(32 * GQ) attn_prefill_kernel(const PrefillAttn
     const int tile = blockIdx.x, kvh = blockIdx.y;
     if (tile >= a.meta->pad2[0]) return;
     const int row0 = a.tile_row0[tile], n_rows = a.tile_rows[tile];
+    if (a.skip && a.skip[row0]) return;  // (the rows of a chunk leave together: prefill exits at one depth)
     const int slot = a.kv.row_slot[row0], pos0 = a.kv.row_pos[row0];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
     const int head = kvh * GQ + warp;

@@ -27,6 +27,7 @@ struct SmallAttnArgs {
     float2 *part_ml;          // [row][Hq][splits]
     unsigned *attn_tickets;   // [row][Hkv], zero between launches
     int *dev_err;
+    const uint8_t *skip;      // rows whose flag is set do not attend (they have left and run nothing here), or null
 };
 
 __device__ __forceinline__ float small_ex2(float x) {
@@ -89,6 +90,7 @@ __device__ __forceinline__ void small_attn_body(const SmallAttnArgs &a, const Kv
     const int Hq = a.Hq;
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int sp = item % S, kvh = (item / S) % a.Hkv, row = item / (S * a.Hkv);
+        if (a.skip && a.skip[row]) continue;
         const int pos = kv.row_pos[row], slot = kv.row_slot[row];
         const int p0 = sp * chunk, p1 = min(pos + 1, p0 + chunk);
         float qr[GQ][VE], acc[GQ][VE], m[GQ], l[GQ];

@@ -801,7 +801,7 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
             stream_rows_bf16<P, R>(p, t0 + warp, rows);
             stream_issue_bf16<R>(rows, K >> 3, 0, lane, pre4.q);
             pre_kind = 1;
-        } else if (hint == 0 && has_river) {
+        } else if (hint == 0 && has_river == 1) {
             W4 rows[R];
             stream_rows_w4<P, R>(p, t0 + warp, rows);
             stream_issue_w4<R>(rows, K >> 5, gshift, 0, lane, pre4);
@@ -813,7 +813,7 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
     const int nv = K >> 2, tid = threadIdx.x, nthr = blockDim.x;
     const int n = *rl.n_rows;
     const bool small = n <= N;       // the whole step in one pass: lists come from the exit flags
-    const bool fast = N == 1 && n == 1 && nv <= XF * nthr;
+    const bool fast = N == 1 && n == 1 && nv <= XF * nthr && has_river != 2;
     float tau[N];
     int forced[N];
 #pragma unroll
@@ -920,6 +920,13 @@ __global__ void __launch_bounds__(512) stream_proj_kernel(const P p, const ProjI
         nr = has_river ? *rl.n_riv : 0;
     }
 
+    // has_river == 2 (State Propagation, Section 3): this launch serves the rows that have LEFT the backbone, on the bf16
+    // weights - the two lists trade places and nothing runs on 4-bit codes
+    if (has_river == 2) {
+        const int32_t *t = act_idx; act_idx = riv_idx; riv_idx = t;
+        na = nr;
+        nr = 0;
+    }
     // hint == 0 promised that no row is left in the backbone: then only the 4-bit pass runs, with the prefetched
     // registers; otherwise the bf16 pass (which may hold prefetched registers) and the 4-bit pass without them, so
     // that neither pass keeps the other's prefetch registers alive

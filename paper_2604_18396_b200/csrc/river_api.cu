@@ -72,6 +72,7 @@ const char *check_config(const river_config *c) {
     if (c->prefill_chunk < 0 || c->prefill_chunk > 256) return "prefill_chunk out of range (0 .. 256)";
     if (c->max_seqs <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return "bad cache geometry";
     if (!(c->exit_mode == RIVER_EXIT_PER_TOKEN || c->exit_mode == RIVER_EXIT_BATCH_MIN)) return "bad exit_mode";
+    if (c->kv_strategy < RIVER_KV_RIVER || c->kv_strategy > RIVER_KV_MONO_DECREASING) return "bad kv_strategy";
     return nullptr;
 }
 
@@ -113,6 +114,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     int *de = cv.take<int>(1);
     unsigned *atk = cv.take<unsigned>(B * (size_t)c->Hkv), *tk4 = cv.take<unsigned>(4);
     int32_t *hint = md ? md + 5 : nullptr;  // StepMeta::hint_act
+    int32_t *scap = cv.take<int32_t>((size_t)c->max_seqs);
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
@@ -123,6 +125,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->state = exd; x->state_stride = (int)sstride; x->prefill_fail = pff;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
+        x->slot_cap = scap;
         x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
@@ -371,7 +374,8 @@ cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const Deci
     const int d = g.d, B = g.max_batch, qdim = g.Hq * g.dh, kvdim = g.Hkv * g.dh;
     const double w4f = 0.25 + 2.0 / g.group;
     const river_layer_weights &w = c->layers[l - 1];
-    const int has_river = w.rq.codes != nullptr;
+    const int strat = g.kv_strategy;
+    const int has_river = strat == RIVER_KV_RIVER && w.rq.codes != nullptr;
     const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
     const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
     const RowLists rl{ai, na, ri, nr, c->hint_act, c->meta_dev /* StepMeta::n_rows */, c->state_at(l - 1)};
@@ -382,7 +386,10 @@ cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const Deci
     cudaError_t err = cudaSuccess;
     auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
     const double wb = 2.0 * (qdim + 2.0 * kvdim) * d;
-    LaunchScope ls(c, K_QKV, wb + kv_write, wb * w4f + kv_write, l - 1);
+    // bytes the rows that have left cost here: the 4-bit copy; the bf16 K and V matrices (State Propagation); nothing
+    const double riv_bytes = strat == RIVER_KV_RIVER ? wb * w4f + kv_write
+                           : strat == RIVER_KV_STATE_PROPAGATION ? 2.0 * 2.0 * kvdim * d + kv_write : 0.0;
+    LaunchScope ls(c, K_QKV, wb + kv_write, riv_bytes, l - 1);
     QkvProblem p{};
     p.wq = (const uint16_t *)w.wq; p.wk = (const uint16_t *)w.wk; p.wv = (const uint16_t *)w.wv;
     p.rq = w4_of(w.rq); p.rk = w4_of(w.rk); p.rv = w4_of(w.rv);
@@ -401,6 +408,24 @@ cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const Deci
         note(launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ri, nr, nrh, e));
     } else if (!tc || has_river) {
         note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, tc ? 1 : 0, dec));
+    }
+    if (strat == RIVER_KV_STATE_PROPAGATION) {
+        // Section 3: K / V of this block for the rows that have left, from their hidden state at the exit (this block's
+        // norm, the backbone's K and V matrices); the same kernels on a K / V-only problem (no query heads) and on the
+        // list of the rows that left
+        if (tc) {
+            TcQkvEpi e{0, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
+            // (the kernel's early-out hint must never under-count; the count of rows that left only grows, so the
+            // hint is the step's row count: the kernel always waits for the real count)
+            note(launch_tc(c, in, tm->k, tm->v, tm->v, d, 2 * kvdim / kTcBM, n, 0, kvdim / kTcBM, kvdim / kTcBM, ri, nr, e,
+                           true, c->meta_dev /* StepMeta::n_rows */));
+            ++c->st.launches_last_step;
+        } else {
+            QkvProblem pk = p;
+            pk.Hq = 0;
+            note(launch_stream(c, pk, in, rl, d, 2 * g.Hkv * (g.dh / 2), n, 2, true, 0, DecideArgs{}));
+            ++c->st.launches_last_step;
+        }
     }
     return err;
 }
@@ -425,8 +450,10 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
     const double kv_write = (double)n * 2.0 * kvdim * 2.0;
     cudaError_t err = cudaSuccess;
     auto note = [&](cudaError_t e) { if (err == cudaSuccess) err = e; };
-    const bool fold = n <= 4 && !c->off_first;  // the decisions ride in the QKV kernels (with offloading the host has to
-                                                // see every decision before it stages a block: score kernel per block)
+    const int strat = g.kv_strategy;
+    // the decisions ride in the QKV kernels - unless the host has to see every decision before it stages a block
+    // (offloading) or the rows that left take another route than the 4-bit copies (then: score kernel per block)
+    const bool fold = n <= 4 && !c->off_first && strat == RIVER_KV_RIVER;
     const DecideArgs no_dec{};
 
     {
@@ -439,13 +466,14 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
         LaunchScope ls(c, K_SCORE, (double)n * d * 8.0, 0, -1);
         note(launch_k(score_compact_kernel, dim3(n), dim3(256), 0, c->stream, true, c->meta(), l, L, g.entry_layer,
                       g.exit_mode, h_in, h_out, d, c->pass, (const uint8_t *)c->state_at(l - 1), c->state_at(l), lists,
-                      c->hint_act, c->tickets + 1, fail_buf, (const int32_t *)c->row_slot()));
+                      c->hint_act, c->tickets + 1, fail_buf, (const int32_t *)c->row_slot(),
+                      strat == RIVER_KV_MONO_DECREASING ? c->slot_cap : (int32_t *)nullptr));
     };
     int hi = 0;                  // h[hi] = block input
     const float *prev_in = nullptr;  // input of the previous block (its output is h[hi])
     for (int l = 1; l <= L; ++l) {
         const river_layer_weights &w = c->layers[l - 1];
-        const int has_river = w.rq.codes != nullptr;
+        const int has_river = strat == RIVER_KV_RIVER && w.rq.codes != nullptr;
         const int32_t *ai = c->act_idx + (size_t)(l - 1) * B, *ri = c->riv_idx + (size_t)(l - 1) * B;
         const int32_t *na = c->n_act + (l - 1), *nr = c->n_riv + (l - 1);
         const RowLists rl{ai, na, ri, nr, c->hint_act, c->meta_dev /* StepMeta::n_rows */, c->state_at(l - 1)};
@@ -469,6 +497,13 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
                 dec.lists = lists; dec.hint_act = c->hint_act; dec.fail = fail_buf; dec.row_slot = c->row_slot();
             }
             note(launch_qkv(c, l, n, h_in, dec, kv_write));
+        }
+        // the other KV strategies (Section 3): a row that has left neither attends nor changes its hidden state
+        c->attn_skip = strat == RIVER_KV_RIVER ? nullptr : c->state_at(l - 1);
+        if (strat != RIVER_KV_RIVER) {
+            LaunchScope ls(c, K_SCORE, 0, 0, -1);
+            note(launch_k(carry_rows_kernel, dim3(n, (d / 4 + 255) / 256), dim3(256), 0, c->stream, true, c->meta(),
+                          (const uint8_t *)c->state_at(l - 1), (const float *)h_in, h_out, d));
         }
         // ---- a3: paged GQA decode attention
         if (c->prefill_attn_now) {
@@ -797,6 +832,10 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (e == cudaSuccess) e = cudaMemsetAsync(c->state, 0, (size_t)(cfg->L + 1) * c->state_stride, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
+    {
+        const std::vector<int32_t> caps((size_t)cfg->max_seqs, cfg->L);  // Mono-Decreasing Exit: every sequence starts at L
+        if (e == cudaSuccess) e = cudaMemcpy(c->slot_cap, caps.data(), sizeof(int32_t) * caps.size(), cudaMemcpyHostToDevice);
+    }
 
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_act, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->n_riv, 0, sizeof(int32_t) * (cfg->L + 1), c->stream);
@@ -974,6 +1013,7 @@ int river_attention(river_ctx *c, int layer, int n_rows, const int32_t *slots, c
     float *q_keep = c->qbuf, *o_keep = c->obuf;
     c->qbuf = const_cast<float *>(q);
     c->obuf = out;
+    c->attn_skip = nullptr;  // every listed row attends
     c->st.launches_last_step = 0;
     cudaError_t e;
     {
@@ -1147,6 +1187,9 @@ int river_release(river_ctx *c, int slot) {
     c->seq_len[slot] = 0;
     CUDA_TRY(c, cudaMemsetAsync(c->page_tbl_dev + (size_t)slot * g.max_pages_per_seq, 0xff,
                                 sizeof(int32_t) * g.max_pages_per_seq, c->stream));
+    const int32_t cap0 = g.L;  // a new sequence in this slot may go to full depth again
+    CUDA_TRY(c, cudaMemcpyAsync(c->slot_cap + slot, &cap0, sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     return RIVER_OK;
 }
 

@@ -45,6 +45,8 @@ struct river_ctx {
     struct BMap { int K, np; CUtensorMap hi, lo; };
     std::vector<BMap> tc_bmaps;
     int32_t *hint_act;
+    const uint8_t *attn_skip = nullptr;  // exit flags of the block whose attention is being launched (strategies that run nothing for rows that left), else null
+    int32_t *slot_cap = nullptr;  // [max_seqs] Mono-Decreasing Exit: the depth the sequence's last token reached
     bool prefill_attn_now = false;  // this chunk's attention runs on the tensor-core prefill kernel
     bool rows_distinct = true;  // every row of the current step is a different sequence (decode), not a prefill chunk
     struct GraphEntry { int n; bool small_attn; int attn_splits; cudaGraphExec_t exec; int launches; };

@@ -79,7 +79,10 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
                                                             int exit_mode, const float *h_in, const float *h_out,
                                                             int d, uint8_t *pass, const uint8_t *state_in,
                                                             uint8_t *state_out, Lists lists, int32_t *hint_act,
-                                                            unsigned *ticket, int32_t *fail, const int32_t *row_slot) {
+                                                            unsigned *ticket, int32_t *fail, const int32_t *row_slot,
+                                                            int32_t *slot_cap) {
+    // slot_cap (Mono-Decreasing Exit only, else null): per sequence the depth its previous token reached; a row leaves
+    // at that depth at the latest, and its own exit layer becomes the sequence's new cap
     __shared__ float red[3][8];
     __shared__ int s_cnt[66];
     __shared__ bool s_last;
@@ -132,8 +135,10 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
             if (!gone) {
                 bool leave = eligible && pass1;  // with one row the batch minimum is the row itself
                 if (forced_mine >= 0) leave = (forced_mine == l) && (l < L);
+                if (slot_cap && l < L && l >= slot_cap[row_slot[0]]) leave = true;
                 if (leave) {
                     exit_layer[0] = l;
+                    if (slot_cap) slot_cap[row_slot[0]] = l;
                     gone = true;
                 }
             }
@@ -202,12 +207,30 @@ __global__ void __launch_bounds__(256) score_compact_kernel(const StepMeta *meta
         bool leave = eligible && (exit_mode == 1 ? (s_allpass != 0) : (pass[b] != 0));
         const int f = forced ? (b == (int)threadIdx.x ? forced_mine : forced[b]) : -1;
         if (f >= 0) leave = (f == l) && (l < L);
-        if (leave) exit_layer[b] = l;
+        if (slot_cap && l < L && l >= slot_cap[row_slot[b]]) leave = true;
+        if (leave) {
+            exit_layer[b] = l;
+            if (slot_cap) slot_cap[row_slot[b]] = l;  // (rows of one prefill chunk share a slot: they all write l)
+        }
         state_out[b] = leave ? 1 : 0;
     }
     __syncthreads();
     build_lists(n, state_out, l, lists, hint_act, s_cnt);
     if (threadIdx.x == 0 && gridDim.x > 1) *ticket = 0;
+}
+
+// ---------------------------------------------------------------- skipped blocks of the other KV strategies
+// State Propagation and Mono-Decreasing Exit (Section 3): a row that has left runs nothing that changes its hidden
+// state, so the block's output row is its input row.  CTA (b, j): floats [1024 j, 1024 j + 1024) of row b.
+static __global__ void __launch_bounds__(256) carry_rows_kernel(const StepMeta *meta, const uint8_t *state, const float *h_in,
+                                                                float *h_out, int d) {
+    pdl_launch();
+    pdl_wait();
+    const int b = blockIdx.x;
+    if (b >= meta->n_rows || state[b] == 0) return;
+    const int i = blockIdx.y * 256 + threadIdx.x;
+    if (i < d / 4)
+        reinterpret_cast<float4 *>(h_out + (size_t)b * d)[i] = __ldcg(reinterpret_cast<const float4 *>(h_in + (size_t)b * d) + i);
 }
 
 // ---------------------------------------------------------------- prologue of the single-stage entry points

@@ -59,10 +59,14 @@ class Pair:
 
     def __init__(self, model, max_seqs: int, max_len: int, max_batch: int, exit_mode: int = 0,
                  entry_layer: Optional[int] = None, page_shuffle_seed: int = 0, flags: int = 0, kv_store: int = 0,
-                 n_pages: Optional[int] = None, prefill_chunk: int = 0, storage_yardstick: bool = False):
+                 n_pages: Optional[int] = None, prefill_chunk: int = 0, storage_yardstick: bool = False,
+                 kv_strategy: int = 0):
         self.shape, (bb_c, rv_c), (bb_g, rv_g) = model
         self.L = len(bb_c["layers"])
-        self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, kv_store)
+        self.kv_strategy = kv_strategy
+        self.depth = {}  # slot -> number of backbone blocks every cached position ran (what Mono-Decreasing Exit wrote)
+        self.oracle = orc.Oracle(self.shape, bb_c, rv_c, max_seqs, max_len, exit_mode, entry_layer, kv_store,
+                                 kv_strategy=kv_strategy)
         # A second oracle with an fp32 cache that is forced down the first one's exit path: how far 16-bit cache storage
         # ALONE moves every later K/V entry (no kernel involved).  On the random-weight 8B-class model a single bf16
         # rounding of a cache entry is amplified layer by layer, so the two sides of a comparison (both store bf16, both
@@ -73,7 +77,7 @@ class Pair:
         cfg = make_config(self.shape, max_seqs=max_seqs, max_pages_per_seq=pages_per_seq,
                           n_pages=n_pages or max_seqs * pages_per_seq, max_batch=max_batch, n_layers=self.L,
                           entry_layer=entry_layer, exit_mode=exit_mode, page_shuffle_seed=page_shuffle_seed,
-                          flags=flags, prefill_chunk=prefill_chunk)
+                          flags=flags, prefill_chunk=prefill_chunk, kv_strategy=kv_strategy)
         self.gpu = River(cfg, bb_g, rv_g)
         self.entry = self.shape.entry_layer if entry_layer is None else entry_layer
         self.V = self.shape.V
@@ -82,6 +86,7 @@ class Pair:
     def prefill(self, slots: List[int], prompts: List[np.ndarray], exit_layer: Optional[int] = None):
         for s, p in zip(slots, prompts):
             self.oracle.prefill(s, p, exit_layer)
+            self.depth.setdefault(s, []).extend([self.L if exit_layer is None else exit_layer] * len(p))
             if self.twin:
                 self.twin.prefill(s, p, exit_layer)
         tok = torch.from_numpy(np.concatenate(prompts).astype(np.int32)).cuda()
@@ -121,6 +126,8 @@ class Pair:
 
     def oracle_step(self, slots, tok, tau, forced=None) -> StepOut:
         r = self.oracle.decode_step(slots, tok, tau, forced)
+        for s, e in zip(slots, r["exit_layer"]):
+            self.depth.setdefault(s, []).append(int(e))
         if self.twin:
             self.twin.decode_step(slots, tok, INF, r["exit_layer"])
         return StepOut(r["logits"], r["next_tok"], r["exit_layer"], r["scores"])
@@ -164,8 +171,17 @@ class Pair:
             kt, vt = self.twin.read_kv(slot, l - 1, 0, n) if self.twin else (None, None)
             kg, vg = self.gpu.read_kv(slot, l, 0, n)
             torch.cuda.synchronize()
+            # Mono-Decreasing Exit writes nothing in a skipped block: those slots must still hold the pool's NaN filling
+            # (taken from the exit layers the oracle reported: its own write counts also see the trial steps)
+            wr = np.array(self.depth[slot][:n]) >= l if self.kv_strategy == 2 else np.ones(n, bool)
             for name, o, g, tw in (("K", ko, kg, kt), ("V", vo, vg, vt)):
                 g = g.float().cpu().numpy()
+                assert np.isnan(g[~wr]).all(), f"{what}: {name} layer {l} slot {slot}: a skipped block wrote the cache"
+                o, g = o[wr], g[wr]
+                if tw is not None:
+                    tw = tw[wr]
+                if not wr.any():
+                    continue
                 assert np.isfinite(g).all(), f"{what}: {name} layer {l} slot {slot}: unwritten (NaN) cache entry"
                 rms = np.sqrt((o.astype(np.float64) ** 2).mean())
                 bound = KV_RTOL * np.abs(o) + KV_RTOL * rms

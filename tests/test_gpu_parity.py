@@ -36,12 +36,12 @@ def toks(shape, n, stream):
 
 
 def run_scheduled(m, prompt_lens, n_steps, kind="uniform", prefill_exit=None, page_seed=0, max_batch=None,
-                  seed=21, kv_store=0, flags=0, storage_yardstick=False):
+                  seed=21, kv_store=0, flags=0, storage_yardstick=False, kv_strategy=0):
     shape = m[0]
     B = len(prompt_lens)
     L = len(m[1][0]["layers"])
     p = Pair(m, B, max(prompt_lens) + n_steps + 1, max_batch or max(B, 8), page_shuffle_seed=page_seed,
-             kv_store=kv_store, flags=flags, storage_yardstick=storage_yardstick)
+             kv_store=kv_store, flags=flags, storage_yardstick=storage_yardstick, kv_strategy=kv_strategy)
     prompts = [toks(shape, n, 100 + b) for b, n in enumerate(prompt_lens)]
     slots = list(range(B))
     p.prefill(slots, prompts, prefill_exit)
