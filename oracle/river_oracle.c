@@ -52,7 +52,9 @@ typedef struct {
                             writes K/V into the shared slot); 1 = State Propagation: the hidden state at the exit is the
                             input of every later block's K/V projection (backbone weights), nothing else runs there;
                             2 = Mono-Decreasing Exit: nothing runs in a skipped block, and a token leaves no later than
-                            the previous token of its sequence did, so no cache entry it needs is ever missing */
+                            the previous token of its sequence did, so no cache entry it needs is ever missing;
+                            3 = KV Mask: nothing runs in a skipped block, and a later token's attention in block l sees
+                            only the positions whose token ran block l (and itself) */
 } orc_config;
 
 /* backbone pointers per layer: attn_norm, wq, wk, wv, wo, ffn_norm, wg, wu, wd (all bf16) */
@@ -69,6 +71,7 @@ typedef struct {
     uint8_t *written;/* [L][max_seqs][max_len] number of writes (saturating) */
     int32_t *len;    /* [max_seqs] */
     int32_t *cap;    /* [max_seqs] Mono-Decreasing Exit: the depth the sequence's last token reached (L to begin with) */
+    uint8_t *depth;  /* [max_seqs][max_len] KV Mask: number of backbone blocks the token at each position ran */
     /* lists of the last decode step: rows in the backbone / in the river entering layer l (1-based) */
     int32_t *act_idx, *riv_idx, *n_act, *n_riv; /* [(L+1)][maxB], [(L+1)] */
     int32_t lists_cap;
@@ -175,17 +178,21 @@ static void get_mats(const orc_ctx *o, int l0, int river, mat_t m[7]) {
  * Causal GQA attention for one row: query heads q [Hq][dh] (already rotated) against the
  * cached positions 0..pos of sequence slot at layer l0; head i reads kv head i/(Hq/Hkv);
  * att [Hq][dh] = softmax_p(q_i . K_p / sqrt(dh)) . V_p.
+ * KV Mask (kv_strategy 3, Section 3): an earlier position whose token did not run block l0 + 1 has no K/V there and is
+ * invisible (the softmax runs over the other positions; the row's own position is always among them).
  */
 static void attend(const orc_ctx *o, int l0, int slot, int pos, const float *q, float *att) {
     const orc_config *c = &o->c;
     const int Hq = c->Hq, dh = c->dh, grp = c->Hq / c->Hkv;
     const double scale = 1.0 / sqrt((double)dh);
+    const uint8_t *depth = c->kv_strategy == 3 ? o->depth + (size_t)slot * c->max_len : NULL;
 #pragma omp parallel for schedule(static)
     for (int i = 0; i < Hq; ++i) {
         const int kvh = i / grp;
         double *sc = (double *)malloc(sizeof(double) * (size_t)(pos + 1));
         double mx = -INFINITY;
         for (int p = 0; p <= pos; ++p) {
+            if (depth && p < pos && depth[p] < l0 + 1) { sc[p] = -INFINITY; continue; }
             const float *kp = o->K + kv_off(o, l0, slot, p) + (size_t)kvh * dh;
             double a = 0.0;
             for (int e = 0; e < dh; ++e) a += (double)q[(size_t)i * dh + e] * (double)kp[e];
@@ -194,13 +201,13 @@ static void attend(const orc_ctx *o, int l0, int slot, int pos, const float *q, 
         }
         double den = 0.0;
         for (int p = 0; p <= pos; ++p) {
-            sc[p] = exp(sc[p] - mx);
+            sc[p] = exp(sc[p] - mx);  /* exactly 0 for an invisible position */
             den += sc[p];
         }
         for (int e = 0; e < dh; ++e) {
             double a = 0.0;
             for (int p = 0; p <= pos; ++p)
-                a += sc[p] * (double)(o->V + kv_off(o, l0, slot, p))[(size_t)kvh * dh + e];
+                if (sc[p] != 0.0) a += sc[p] * (double)(o->V + kv_off(o, l0, slot, p))[(size_t)kvh * dh + e];
             att[(size_t)i * dh + e] = (float)(a / den);
         }
         free(sc);
@@ -339,13 +346,15 @@ orc_ctx *orc_create(const orc_config *cfg, const void *embed, const void *lm_hea
     o->cap = (int32_t *)malloc(sizeof(int32_t) * (size_t)cfg->max_seqs);
     if (!o->K || !o->V || !o->written || !o->cap) return NULL;
     for (int s = 0; s < cfg->max_seqs; ++s) o->cap[s] = cfg->L;
-    if (cfg->kv_strategy < 0 || cfg->kv_strategy > 2) return NULL;
+    if (cfg->kv_strategy < 0 || cfg->kv_strategy > 3 || cfg->L > 255) return NULL;
+    o->depth = (uint8_t *)calloc((size_t)cfg->max_seqs * cfg->max_len, 1);
+    if (!o->depth) return NULL;
     return o;
 }
 
 void orc_destroy(orc_ctx *o) {
     if (!o) return;
-    free(o->K); free(o->V); free(o->written); free(o->len); free(o->cap);
+    free(o->K); free(o->V); free(o->written); free(o->len); free(o->cap); free(o->depth);
     free((void *)o->bb); free((void *)o->rv);
     free(o->act_idx); free(o->riv_idx); free(o->n_act); free(o->n_riv);
     free(o);
@@ -420,7 +429,7 @@ int orc_decode_step(orc_ctx *o, int B, const int32_t *slots, const int32_t *tok,
         }
         o->n_act[l - 1] = na; o->n_riv[l - 1] = nr;
         for (int b = 0; b < B; ++b) {
-            if (exited[b] && c->kv_strategy != 0) {  /* a skipped block under one of the other strategies */
+            if (exited[b] && c->kv_strategy != 0) {  /* a skipped block under one of the other strategies (2, 3: nothing) */
                 if (c->kv_strategy == 1) propagate_kv(o, l - 1, slots[b], o->len[slots[b]], h + (size_t)b * d);
                 memcpy(h2 + (size_t)b * d, h + (size_t)b * d, sizeof(float) * (size_t)d);
                 continue;
@@ -466,6 +475,7 @@ int orc_decode_step(orc_ctx *o, int B, const int32_t *slots, const int32_t *tok,
         lm_head(o, h + (size_t)b * d, logits ? logits + (size_t)b * c->V : NULL, &next_tok[b]);
         o->len[slots[b]] += 1;
         if (c->kv_strategy == 2) o->cap[slots[b]] = exit_layer[b];
+        o->depth[(size_t)slots[b] * c->max_len + (o->len[slots[b]] - 1)] = (uint8_t)exit_layer[b];
     }
     free(h); free(h2); free(exited); free(s_now);
     return 0;

@@ -42,7 +42,8 @@ def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False, strategy=0):
     strategy (what a skipped block does, Section 3): 0 = the quantised copy of the block runs (Section 4.1); 1 = State
     Propagation: K/V of the block from the hidden state at the exit through the BACKBONE's K / V projections, the
     hidden state itself unchanged; 2 = Mono-Decreasing Exit: nothing (the block's K/V rows of that token come back as
-    NaN; no later token may need them, which holds when the exit layers never increase)."""
+    NaN; no later token may need them, which holds when the exit layers never increase); 3 = KV Mask: nothing either,
+    and a token's attention in a block sees only the earlier positions whose token ran that block, and itself."""
     tokens = np.asarray(tokens)
     e = np.asarray(exit_layers)
     T = len(tokens)
@@ -71,8 +72,10 @@ def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False, strategy=0):
             k, v = _bf16(k), _bf16(v)
         if strategy == 2:
             assert all(e[j] <= e[i] for i in range(T) for j in range(i + 1, T)), "exit layers must not increase"
+        if strategy in (2, 3):
             k = np.where(in_river[:, None], np.nan, k)
             v = np.where(in_river[:, None], np.nan, v)
+        visible = causal if strategy != 3 else causal & (~in_river[None, :] | np.eye(T, dtype=bool))
         Ks.append(k)
         Vs.append(v)
         k3, v3 = np.nan_to_num(k).reshape(T, Hkv, dh), np.nan_to_num(v).reshape(T, Hkv, dh)
@@ -80,7 +83,7 @@ def recompute(shape, bb, rv, tokens, exit_layers, kv_bf16=False, strategy=0):
         for i in range(Hq):
             j = i // (Hq // Hkv)
             sc = q[:, i, :] @ k3[:, j, :].T / np.sqrt(dh)
-            sc = np.where(causal, sc, -np.inf)
+            sc = np.where(visible, sc, -np.inf)
             p = np.exp(sc - sc.max(axis=1, keepdims=True))
             p /= p.sum(axis=1, keepdims=True)
             att[:, i, :] = p @ v3[:, j, :]
