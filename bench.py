@@ -99,7 +99,8 @@ def alg_bytes_step(shape, L, exit_layers, positions, want_logits=True, kv_strate
     """Algorithmic HBM bytes of one decode step from its exit pattern: weights of every (layer, weight set) that
     ran, KV read by every row in every layer it attends in (exit-layer rows attend too), KV written, LM head,
     embedding rows.  kv_strategy 1 (State Propagation): a skipped block costs its bf16 K and V matrices and a KV
-    write, no attention; 2 (Mono-Decreasing Exit): nothing."""
+    write, no attention; 2 (Mono-Decreasing Exit) and 3 (KV Mask): nothing (KV Mask rows read fewer cache entries than
+    counted here: positions without an entry in a block are skipped)."""
     P = shape.layer_params()
     B = len(exit_layers)
     kv_tok = 2.0 * shape.Hkv * shape.dh * 2.0
@@ -421,7 +422,7 @@ def ours(args, wl):
                        "early_exit_target_fraction": EARLY_FRACTION, "thresholds": "per-step, from calibrated mean scores",
                        "l2": "inputs (weights + KV) larger than L2, no flush", "flags": flags, "layers": L,
                        "parallelism": "replicas only" if world > 1 else "1 GPU", "prefill_s": round(t_pf, 3),
-                       "kv_strategy": ["exit river", "state propagation", "mono-decreasing exit"][args.kv_strategy],
+                       "kv_strategy": ["exit river", "state propagation", "mono-decreasing exit", "kv mask"][args.kv_strategy],
                        **({"offload": {"first_offloaded_layer": args.offload_from, "device_bytes_saved": off_saved,
                                        "block_copies_per_step": (off_fetches - off_fetches0) / K}}
                           if args.offload_from else {})},
@@ -598,9 +599,9 @@ def main():
     ap.add_argument("--micro-pool-gib", type=int, default=64, help="attn_micro: cap of the KV pool (fewer blocks are run when a point needs more)")
     ap.add_argument("--flags", type=int, default=1, help="river_config.flags (1 = CUDA-graph replay)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kv-strategy", type=int, default=0, choices=[0, 1, 2],
+    ap.add_argument("--kv-strategy", type=int, default=0, choices=[0, 1, 2, 3],
                     help="what a skipped block does: 0 = the 4-bit exit river (the method), 1 = State Propagation, "
-                         "2 = Mono-Decreasing Exit (river_config.kv_strategy)")
+                         "2 = Mono-Decreasing Exit, 3 = KV Mask (river_config.kv_strategy)")
     ap.add_argument("--offload-from", type=int, default=0,
                     help="keep backbone blocks >= this layer in pinned host memory (river_offload); 0 = all resident")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the shape")

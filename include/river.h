@@ -83,10 +83,13 @@ typedef struct river_config {
  *                              token of its sequence did (whatever its score, and before a later forced exit), so no
  *                              cache entry it attends to is ever missing; the cap of a sequence starts at L, follows
  *                              every token (prefill: the prefill depth) and is reset by river_release.
- * (KV Mask, the fourth strategy of Section 3, is not built.) */
+ *   RIVER_KV_MASK              (Section 3) nothing runs in a skipped block either, and exits are free: attention in block
+ *                              l sees only the cached positions whose token ran block l (and the row's own position).
+ *                              Needs groups of at most four query heads per KV head. */
 #define RIVER_KV_RIVER 0
 #define RIVER_KV_STATE_PROPAGATION 1
 #define RIVER_KV_MONO_DECREASING 2
+#define RIVER_KV_MASK 3
 
 typedef struct river_w4 {
     const void *codes, *scale, *zero; /* [dev] */

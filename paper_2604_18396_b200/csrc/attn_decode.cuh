@@ -44,6 +44,8 @@ struct AttnArgs {
     float *out;            // [rows][Hq*DH]
     int *dev_err;
     const uint8_t *skip;   // rows whose flag is set do not attend (they have left and run nothing here), or null
+    const uint8_t *pos_depth;  // KV Mask: [slot][depth_stride] backbone blocks the token at each position ran, or null
+    int depth_stride, layer1;  // ... a position is visible in block layer1 if that number is >= layer1 (or it is the row's own)
 };
 
 template <int DH, int GQ, bool MMA>
@@ -165,8 +167,21 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
                 const int s = t % kAttnStages;
                 if (!mbar_wait(smem_u32(&bars[s]), (t / kAttnStages) & 1, abortp, a.dev_err)) break;
                 const int pos0 = p0 + t * kAttnTile + warp * kPage;  // first position of this warp's page
+                // positions of this page that take part: inside the split, and (KV Mask) with an entry in this block
+                uint32_t seen = 0u;
                 if (pos0 < p1) {
-                    const int n_live = min(kPage, p1 - pos0);
+                    seen = (1u << min(kPage, p1 - pos0)) - 1u;
+                    if (a.pos_depth) {
+                        const uint4 dv = *reinterpret_cast<const uint4 *>(a.pos_depth + (size_t)slot * a.depth_stride + pos0);
+                        const uint32_t dw[4] = {dv.x, dv.y, dv.z, dv.w};
+                        uint32_t ok = 0u;
+#pragma unroll
+                        for (int i = 0; i < kPage; ++i)
+                            if ((int)((dw[i >> 2] >> (8 * (i & 3))) & 0xffu) >= a.layer1 || pos0 + i == pos) ok |= 1u << i;
+                        seen &= ok;
+                    }
+                }
+                if (seen) {
                     const uint32_t kpg = smem_u32(stages + s * STAGE_BYTES + warp * PAGE_BYTES);
                     const uint32_t vpg = kpg + kAttnConsumers * PAGE_BYTES;
                     float sc[2][4];  // S: row r8, positions 8 j + 2 t4 (+ 1) in [j][0..1]; rows 8-15 (unused) in [j][2..3]
@@ -189,13 +204,13 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             float v = sc[j][e] + __shfl_xor_sync(0xffffffffu, sc[j][e], 16);  // hi row + remainder row
-                            v = (8 * j + 2 * t4 + e < n_live) ? v : -CUDART_INF_F;  // select: stale rows may hold anything
+                            v = ((seen >> (8 * j + 2 * t4 + e)) & 1u) ? v : -CUDART_INF_F;  // select: other rows may hold anything
                             p[j][e] = v;
                             mx = fmaxf(mx, v);
                         }
                     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    const float mn = fmaxf(m, mx);  // finite: position pos0 is live
+                    const float mn = fmaxf(m, mx);  // finite: at least one position of the page takes part
                     const float corr = ex2(m - mn);
                     m = mn;
                     float psum = 0.f;
@@ -211,7 +226,7 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
                     // the accumulator columns 2 t4, 2 t4 + 1 belong to heads (2 t4) & 3 and (2 t4 + 1) & 3
                     const float c0 = __shfl_sync(0xffffffffu, corr, ((2 * t4) & 3) * 4);
                     const float c1 = __shfl_sync(0xffffffffu, corr, ((2 * t4 + 1) & 3) * 4);
-                    const bool cut = n_live < kPage;
+                    const bool cut = seen != 0xffffu;
 #pragma unroll
                     for (int mt = 0; mt < KS; ++mt) {
                         const int cg = 2 * mt + lodd, box = cg >> 3, c = cg & 7;
@@ -221,8 +236,8 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 const int pp = 2 * t4 + 8 * (q >> 1);
-                                if (pp >= n_live) vf[q] = 0u;
-                                else if (pp + 1 >= n_live) vf[q] &= 0x0000ffffu;
+                                if (!((seen >> pp) & 1u)) vf[q] &= 0xffff0000u;
+                                if (!((seen >> (pp + 1)) & 1u)) vf[q] &= 0x0000ffffu;
                             }
                         }
                         acc[mt][0] *= c0; acc[mt][1] *= c1; acc[mt][2] *= c0; acc[mt][3] *= c1;

@@ -28,6 +28,8 @@ struct SmallAttnArgs {
     unsigned *attn_tickets;   // [row][Hkv], zero between launches
     int *dev_err;
     const uint8_t *skip;      // rows whose flag is set do not attend (they have left and run nothing here), or null
+    const uint8_t *pos_depth; // KV Mask: [slot][depth_stride] backbone blocks the token at each position ran, or null
+    int depth_stride, layer1; // ... a position is visible in block layer1 if that number is >= layer1 (or it is the row's own)
 };
 
 __device__ __forceinline__ float small_ex2(float x) {
@@ -118,6 +120,8 @@ __device__ __forceinline__ void small_attn_body(const SmallAttnArgs &a, const Kv
             }
             float kf[U][VE], vf[U][VE];
             const bool first = item == (int)blockIdx.x && pb == p0 + warp * U;
+            uint32_t dw = 0xffffffffu;  // depth bytes of positions pb .. pb + 3 (pb is a multiple of 4)
+            if (a.pos_depth) dw = *reinterpret_cast<const uint32_t *>(a.pos_depth + (size_t)slot * a.depth_stride + pb);
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int p = pb + u;
@@ -138,7 +142,9 @@ __device__ __forceinline__ void small_attn_body(const SmallAttnArgs &a, const Kv
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (pb + u < p1) {  // warp-uniform
+                // warp-uniform; KV Mask: a position whose token skipped this block has no entry here (its slot may hold
+                // anything) and is not seen - the row's own position always is
+                if (pb + u < p1 && (pb + u == pos || (int)((dw >> (8 * u)) & 0xffu) >= a.layer1)) {
 #pragma unroll
                     for (int g = 0; g < GQ; ++g) {
                         float s = 0.f;

@@ -21,6 +21,7 @@ cudaError_t launch_attn_split(river_ctx *c, int n, int layer0) {
     a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.tickets = c->attn_tickets; a.out = c->obuf; a.dev_err = c->dev_err;
     a.skip = c->attn_skip;
+    a.pos_depth = c->attn_layer1 ? c->pos_depth : nullptr; a.depth_stride = g.max_pages_per_seq * kPage; a.layer1 = c->attn_layer1;
     const size_t smem = attn_smem_bytes(DH, GQ);
     constexpr bool MMA = GQ <= 4;  // groups of up to four query heads: contractions on the warp-level tensor cores
     const cudaError_t e = ensure_smem(c, attn_split_kernel<DH, GQ, MMA>, smem);
@@ -40,6 +41,7 @@ cudaError_t launch_attn_small(river_ctx *c, int n, int layer0, int early) {
     a.qbuf = c->qbuf; a.obuf = c->obuf; a.kv = kv_addr(c, layer0);
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.attn_tickets = c->attn_tickets; a.dev_err = c->dev_err;
     a.skip = c->attn_skip;
+    a.pos_depth = c->attn_layer1 ? c->pos_depth : nullptr; a.depth_stride = g.max_pages_per_seq * kPage; a.layer1 = c->attn_layer1;
     if (a.skip) early = 0;  // the flags belong to this block: nothing may be fetched before the dependency resolves
     const int S = small_attn_splits(c->num_sms, n, g.Hkv);  // as the step metadata says
     const size_t smem = sizeof(float) * (size_t)kSmallAttnWarps * GQ * (DH + 2);

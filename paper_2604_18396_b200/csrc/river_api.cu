@@ -72,7 +72,9 @@ const char *check_config(const river_config *c) {
     if (c->prefill_chunk < 0 || c->prefill_chunk > 256) return "prefill_chunk out of range (0 .. 256)";
     if (c->max_seqs <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return "bad cache geometry";
     if (!(c->exit_mode == RIVER_EXIT_PER_TOKEN || c->exit_mode == RIVER_EXIT_BATCH_MIN)) return "bad exit_mode";
-    if (c->kv_strategy < RIVER_KV_RIVER || c->kv_strategy > RIVER_KV_MONO_DECREASING) return "bad kv_strategy";
+    if (c->kv_strategy < RIVER_KV_RIVER || c->kv_strategy > RIVER_KV_MASK) return "bad kv_strategy";
+    if (c->kv_strategy == RIVER_KV_MASK && (c->Hq / c->Hkv > 4 || c->L > 255))
+        return "KV Mask needs groups of at most four query heads per KV head";
     return nullptr;
 }
 
@@ -115,6 +117,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     unsigned *atk = cv.take<unsigned>(B * (size_t)c->Hkv), *tk4 = cv.take<unsigned>(4);
     int32_t *hint = md ? md + 5 : nullptr;  // StepMeta::hint_act
     int32_t *scap = cv.take<int32_t>((size_t)c->max_seqs);
+    uint8_t *pdep = cv.take<uint8_t>((size_t)c->max_seqs * c->max_pages_per_seq * kPage);
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
@@ -125,7 +128,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->state = exd; x->state_stride = (int)sstride; x->prefill_fail = pff;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
-        x->slot_cap = scap;
+        x->slot_cap = scap; x->pos_depth = pdep;
         x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
@@ -500,6 +503,10 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
         }
         // the other KV strategies (Section 3): a row that has left neither attends nor changes its hidden state
         c->attn_skip = strat == RIVER_KV_RIVER ? nullptr : c->state_at(l - 1);
+        // (a prefill chunk needs no visibility test: a prompt starts in an empty slot and all its positions stop at one
+        // depth, so whatever a row that still runs may look back at has an entry - and the chunk's own positions have
+        // not been noted yet)
+        c->attn_layer1 = (strat == RIVER_KV_MASK && c->rows_distinct) ? l : 0;
         if (strat != RIVER_KV_RIVER) {
             LaunchScope ls(c, K_SCORE, 0, 0, -1);
             note(launch_k(carry_rows_kernel, dim3(n, (d / 4 + 255) / 256), dim3(256), 0, c->stream, true, c->meta(),
@@ -602,6 +609,11 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
     }
     // small steps: the last block's score (a diagnostic: no exit is taken after block L) and the final row lists
     if (fold) launch_score(L, prev_in, c->h[hi]);
+    if (strat == RIVER_KV_MASK) {  // what the later tokens' attention may see of this step's positions
+        LaunchScope ls(c, K_SCORE, 0, 0, -1);
+        note(launch_k(depth_note_kernel, dim3((n + 127) / 128), dim3(128), 0, c->stream, true, c->meta(),
+                      (const int32_t *)c->row_slot(), (const int32_t *)c->row_pos(), c->pos_depth, g.max_pages_per_seq * kPage));
+    }
     if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) return fail(c, RIVER_E_DEVICE, std::string("kernel launch failed: ") + cudaGetErrorString(err));
     c->st.launches_total += c->st.launches_last_step;
@@ -1014,6 +1026,7 @@ int river_attention(river_ctx *c, int layer, int n_rows, const int32_t *slots, c
     c->qbuf = const_cast<float *>(q);
     c->obuf = out;
     c->attn_skip = nullptr;  // every listed row attends
+    c->attn_layer1 = 0;      // ... to every cached position
     c->st.launches_last_step = 0;
     cudaError_t e;
     {

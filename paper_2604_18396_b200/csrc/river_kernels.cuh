@@ -233,6 +233,16 @@ static __global__ void __launch_bounds__(256) carry_rows_kernel(const StepMeta *
         reinterpret_cast<float4 *>(h_out + (size_t)b * d)[i] = __ldcg(reinterpret_cast<const float4 *>(h_in + (size_t)b * d) + i);
 }
 
+// KV Mask (Section 3): at the end of a step, note for every row's position how many backbone blocks its token ran -
+// the later tokens' attention in block l sees a position only if that number is at least l.
+static __global__ void depth_note_kernel(const StepMeta *meta, const int32_t *row_slot, const int32_t *row_pos,
+                                         uint8_t *pos_depth, int stride) {
+    pdl_launch();
+    pdl_wait();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < meta->n_rows) pos_depth[(size_t)row_slot[b] * stride + row_pos[b]] = (uint8_t)meta->exit_layer[b];
+}
+
 // ---------------------------------------------------------------- prologue of the single-stage entry points
 // river_attention / river_project_kv run one stage of the path for a caller-given list of rows: this kernel tabulates
 // the rotary angles of the rows' positions and puts all rows on one weight set of block `l0 + 1` (exit flags, row

@@ -171,9 +171,9 @@ class Pair:
             kt, vt = self.twin.read_kv(slot, l - 1, 0, n) if self.twin else (None, None)
             kg, vg = self.gpu.read_kv(slot, l, 0, n)
             torch.cuda.synchronize()
-            # Mono-Decreasing Exit writes nothing in a skipped block: those slots must still hold the pool's NaN filling
+            # Mono-Decreasing Exit and KV Mask write nothing in a skipped block: those slots must still hold the pool's NaN filling
             # (taken from the exit layers the oracle reported: its own write counts also see the trial steps)
-            wr = np.array(self.depth[slot][:n]) >= l if self.kv_strategy == 2 else np.ones(n, bool)
+            wr = np.array(self.depth[slot][:n]) >= l if self.kv_strategy in (2, 3) else np.ones(n, bool)
             for name, o, g, tw in (("K", ko, kg, kt), ("V", vo, vg, vt)):
                 g = g.float().cpu().numpy()
                 assert np.isnan(g[~wr]).all(), f"{what}: {name} layer {l} slot {slot}: a skipped block wrote the cache"

@@ -8,7 +8,7 @@ from tests.test_gpu_parity import model, run_scheduled, toks
 
 pytestmark = pytest.mark.gpu
 
-SP, MONO = 1, 2
+SP, MONO, MASK = 1, 2, 3
 
 
 @pytest.mark.parametrize("rows,flags", [(1, 1), (3, 0), (3, 1), (6, 1)])
@@ -58,5 +58,35 @@ def test_mono_decreasing_cap_follows_prefill_depth_and_release():
     g = p.gpu_step([0], tk, INF)
     assert g.exit_layer[0] == o.exit_layer[0] == L
     p.compare_logits(g.logits, o.logits, "after release")
+    assert p.gpu.stats().device_error == 0
+    p.close()
+
+
+@pytest.mark.parametrize("rows,flags,steps", [(1, 1, 14), (3, 1, 10), (6, 1, 8)])
+def test_kv_mask_steps(rows, flags, steps):
+    # exits are free; skipped blocks write nothing; a later token's attention in block l must see exactly the positions
+    # whose token ran block l (the small-step kernel for 1-3 rows, the TMA-fed tensor-core kernel for 6): any position
+    # seen by mistake would bring the pool's NaN filling into the logits
+    lens = [23, 9, 40, 5, 31, 16][:rows]
+    r = run_scheduled(model("mini8"), lens, steps, "uniform", prefill_exit=4, page_seed=13 + rows, flags=flags,
+                      max_batch=max(rows, 4), kv_strategy=MASK, kv_store=1)
+    assert r["n_early"] > 0
+    print("kv mask:", r)
+
+
+def test_kv_mask_long_context_split_attention():
+    # one row with a context long enough for the TMA-fed kernel with several splits, early exits in the history
+    m = model("mini8")
+    shape = m[0]
+    p = Pair(m, 1, 400, 4, kv_strategy=MASK, kv_store=1, flags=33)  # 32: the TMA-fed kernel for small steps too
+    p.prefill([0], [toks(shape, 300, 3)], 3)  # blocks 4..L see nothing of the prompt
+    rng = np.random.default_rng(1)
+    for t in range(6):
+        tk = toks(shape, 1, 60 + t)
+        tau, o = p.oracle_scheduled_step([0], tk, rng.integers(1, p.L + 1, 1))
+        g = p.gpu_step([0], tk, tau)
+        assert np.array_equal(g.exit_layer, o.exit_layer)
+        p.compare_logits(g.logits, o.logits, f"step {t}")
+    p.compare_kv(0, p.oracle.seq_len(0))
     assert p.gpu.stats().device_error == 0
     p.close()
