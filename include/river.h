@@ -199,6 +199,15 @@ int river_generate(river_ctx *ctx, int batch, const int32_t *slots, const int32_
  * own.  first_offloaded_layer = 0 turns it off.  river_stats.offload_fetches counts the block copies. */
 int river_offload(river_ctx *ctx, int first_offloaded_layer, const river_layer_weights *host_layers);
 
+/* Which blocks are sparsely used (Section 4.2: the blocks to offload follow from where the tokens leave).
+ * river_exit_histogram: counts [host] L + 1 entries, counts[e] = decoded tokens so far (decode steps and river_generate,
+ *   not prompts) that ran e backbone blocks; reset != 0 clears the counters afterwards.  Synchronises the stream.
+ * river_suggest_offload: the first block l >= 2 that at most max_deep_fraction of the decoded tokens have reached (exit
+ *   layer >= l) - the value to hand to river_offload - or 0 when no block qualifies or nothing has been decoded yet;
+ *   negative on error. */
+int river_exit_histogram(river_ctx *ctx, int64_t *counts, int reset);
+int river_suggest_offload(river_ctx *ctx, double max_deep_fraction);
+
 /* Two stages of the path on their own, for kernel-level tests and the exit-aware attention microbenchmark.  Both take
  * a compacted list of rows: row i belongs to sequence slots[i] ([host], distinct, non-empty) and sits at that
  * sequence's LAST cached position p_i; both enqueue on the context's stream like a decode step.

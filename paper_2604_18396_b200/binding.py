@@ -58,7 +58,8 @@ class river_kernel_time(C.Structure):
 EXPORTS = ("river_argmax_noalloc", "river_profile", "river_profile_read", "river_workspace_bytes", "river_kv_pool_bytes", "river_init", "river_prefill", "river_decode_step",
            "river_decode_step_host", "river_read_kv", "river_write_kv", "river_last_lists", "river_seq_len",
            "river_release", "river_stats", "river_destroy", "river_last_error", "river_clear_device_error",
-           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4", "river_generate", "river_offload")
+           "river_selftest_wait_timeout", "river_attention", "river_project_kv", "river_quantize_w4", "river_generate", "river_offload", "river_exit_histogram",
+           "river_suggest_offload")
 
 _lib = None
 
@@ -98,6 +99,8 @@ def load():
     L.river_project_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, vp]
     L.river_quantize_w4.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp]
     L.river_offload.argtypes = [vp, C.c_int, C.POINTER(river_layer_weights)]
+    L.river_exit_histogram.argtypes = [vp, C.POINTER(C.c_int64), C.c_int]
+    L.river_suggest_offload.argtypes = [vp, C.c_double]
     L.river_generate.argtypes = [vp, C.c_int, i32p, vp, vp, C.c_int, vp, vp]
     L.river_clear_device_error.argtypes = [vp]
     L.river_selftest_wait_timeout.argtypes = [vp, C.c_int]
@@ -286,6 +289,18 @@ class River:
                         setattr(arr[l], n, t.data_ptr())
         self._keep_host = host_layers
         self._check(load().river_offload(self.h, first_offloaded_layer, arr))
+
+    def exit_histogram(self, reset: bool = False):
+        """river_exit_histogram -> list of L + 1 counts."""
+        buf = (C.c_int64 * (self.cfg.L + 1))()
+        self._check(load().river_exit_histogram(self.h, buf, 1 if reset else 0))
+        return list(buf)
+
+    def suggest_offload(self, max_deep_fraction: float) -> int:
+        rc = load().river_suggest_offload(self.h, float(max_deep_fraction))
+        if rc < 0:
+            self._check(rc)
+        return rc
 
     def generate(self, slots: Sequence[int], tok0: torch.Tensor, tau: torch.Tensor, n_steps: int):
         """river_generate -> (tokens int32 [n_steps, batch], exit layers int32 [n_steps, batch]), both on the device."""

@@ -1020,11 +1020,15 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const HeadArgs a, int xstr
     }
 }
 
-static __global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts) {
+// exit_hist (decode steps only, else null): [L + 1] counters of the exit layers taken so far - the head rows of a decode
+// step are its rows, and their exit layers are final by now.
+static __global__ void argmax_final_kernel(const StepMeta *meta, const float *part_val, const int32_t *part_idx, int nparts,
+                                           unsigned long long *exit_hist) {
     pdl_launch();
     pdl_wait();
     const int i = blockIdx.x;
     if (i >= meta->n_head_rows) return;
+    if (exit_hist && threadIdx.x == 0) atomicAdd(exit_hist + meta->exit_layer[i], 1ull);
     int32_t *next_tok = meta->next_tok;  // indexed by position in the head-row list
     float bv = -CUDART_INF_F;
     int bi = 0x7fffffff;

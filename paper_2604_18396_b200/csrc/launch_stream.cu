@@ -93,7 +93,8 @@ cudaError_t launch_head_stream(river_ctx *c, const HeadArgs &a, int n_head) {
 
 cudaError_t launch_argmax_final(river_ctx *c, int n_head, int n_parts) {
     return launch_k(argmax_final_kernel, dim3(n_head), dim3(128), 0, c->stream, true, c->meta(),
-                    (const float *)c->part_val, (const int32_t *)c->part_idx, n_parts);
+                    (const float *)c->part_val, (const int32_t *)c->part_idx, n_parts,
+                    c->rows_distinct ? c->exit_hist : (unsigned long long *)nullptr);  // (not for prefill chunks)
 }
 
 }  // namespace river

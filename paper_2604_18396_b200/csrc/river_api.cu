@@ -118,6 +118,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     int32_t *hint = md ? md + 5 : nullptr;  // StepMeta::hint_act
     int32_t *scap = cv.take<int32_t>((size_t)c->max_seqs);
     uint8_t *pdep = cv.take<uint8_t>((size_t)c->max_seqs * c->max_pages_per_seq * kPage);
+    unsigned long long *ehist = cv.take<unsigned long long>((size_t)c->L + 1);
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
@@ -128,7 +129,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
         x->inv_freq = fr; x->act_idx = ai; x->riv_idx = ri; x->n_act = na; x->n_riv = nr; x->page_tbl_dev = pt;
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->state = exd; x->state_stride = (int)sstride; x->prefill_fail = pff;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
-        x->slot_cap = scap; x->pos_depth = pdep;
+        x->slot_cap = scap; x->pos_depth = pdep; x->exit_hist = ehist;
         x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
@@ -844,6 +845,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     if (e == cudaSuccess) e = cudaMemsetAsync(c->state, 0, (size_t)(cfg->L + 1) * c->state_stride, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->attn_tickets, 0, sizeof(unsigned) * (size_t)cfg->max_batch * cfg->Hkv, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * 4, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->exit_hist, 0, sizeof(unsigned long long) * (cfg->L + 1), c->stream);
     {
         const std::vector<int32_t> caps((size_t)cfg->max_seqs, cfg->L);  // Mono-Decreasing Exit: every sequence starts at L
         if (e == cudaSuccess) e = cudaMemcpy(c->slot_cap, caps.data(), sizeof(int32_t) * caps.size(), cudaMemcpyHostToDevice);
@@ -1106,6 +1108,33 @@ int river_offload(river_ctx *c, int first_offloaded_layer, const river_layer_wei
     c->off_first = first_offloaded_layer;
     c->off_slot_layer[0] = c->off_slot_layer[1] = -1;
     return RIVER_OK;
+}
+
+int river_exit_histogram(river_ctx *c, int64_t *counts, int reset) {
+    if (!c || !counts) return RIVER_E_BADARG;
+    const int n = c->cfg.L + 1;
+    CUDA_TRY(c, cudaMemcpyAsync(counts, c->exit_hist, sizeof(int64_t) * n, cudaMemcpyDeviceToHost, c->stream));
+    if (reset) CUDA_TRY(c, cudaMemsetAsync(c->exit_hist, 0, sizeof(unsigned long long) * n, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    return RIVER_OK;
+}
+
+int river_suggest_offload(river_ctx *c, double max_deep_fraction) {
+    if (!c || !(max_deep_fraction >= 0.0)) return RIVER_E_BADARG;
+    const int L = c->cfg.L;
+    std::vector<int64_t> h((size_t)L + 1);
+    if (int rc = river_exit_histogram(c, h.data(), 0)) return rc;
+    int64_t total = 0;
+    for (int64_t v : h) total += v;
+    if (total == 0) return 0;  // nothing decoded yet: no advice
+    // tokens that reach block l are those whose exit layer is >= l; the first block (>= 2) that at most the given
+    // fraction of the tokens reaches
+    int64_t reach = total - h[0];  // exit layer >= 1
+    for (int l = 1; l <= L; ++l) {
+        if (l >= 2 && (double)reach <= max_deep_fraction * (double)total) return l;
+        reach -= h[l];
+    }
+    return 0;  // every block is reached too often
 }
 
 int river_clear_device_error(river_ctx *c) {

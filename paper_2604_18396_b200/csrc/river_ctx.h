@@ -48,6 +48,7 @@ struct river_ctx {
     const uint8_t *attn_skip = nullptr;  // exit flags of the block whose attention is being launched (strategies that run nothing for rows that left), else null
     uint8_t *pos_depth = nullptr;  // [max_seqs][max_pages_per_seq * 16] KV Mask: backbone blocks the token at each position ran
     int attn_layer1 = 0;           // block (1-based) whose attention is being launched (KV Mask: the visibility test)
+    unsigned long long *exit_hist = nullptr;  // [L + 1] exit layers of all decoded tokens so far (river_exit_histogram)
     int32_t *slot_cap = nullptr;  // [max_seqs] Mono-Decreasing Exit: the depth the sequence's last token reached
     bool prefill_attn_now = false;  // this chunk's attention runs on the tensor-core prefill kernel
     bool rows_distinct = true;  // every row of the current step is a different sequence (decode), not a prefill chunk

@@ -86,3 +86,35 @@ def test_offload_rejects_unaliased_layers():
         p.gpu.offload(1, host)
     p.gpu.offload(0, None)
     p.close()
+
+
+def test_exit_histogram_and_offload_suggestion():
+    # the counters follow the exit layers of the decoded tokens (not the prompt's), and the suggested first offloaded
+    # block is the first one that at most the given fraction of them reached
+    model = draw_model("mini8")
+    p = Pair(model, max_seqs=3, max_len=64, max_batch=4)
+    L = p.L
+    prompts = [synth.tokens(5, b, 9 + 4 * b, p.shape.V) for b in range(3)]
+    p.prefill([0, 1, 2], prompts)
+    assert p.gpu.suggest_offload(0.5) == 0 and sum(p.gpu.exit_histogram()) == 0
+    tok = np.array([pr[-1] for pr in prompts], np.int32)
+    want = np.zeros(L + 1, np.int64)
+    schedule = [[2, 2, 6], [1, 3, 2], [2, 6, 2], [2, 1, 4]]
+    for forced in schedule:
+        o = p.oracle_step([0, 1, 2], tok, INF, forced)
+        g = p.gpu_step([0, 1, 2], tok, INF, forced)
+        assert np.array_equal(g.exit_layer, o.exit_layer)
+        for e in o.exit_layer:
+            want[e] += 1
+        tok = o.next_tok.astype(np.int32)
+    assert p.gpu.exit_histogram() == want.tolist()
+    total = int(want.sum())
+    for frac in (0.0, 0.1, 0.2, 0.5, 1.0):
+        expect = 0
+        for l in range(2, L + 1):
+            if int(want[l:].sum()) <= frac * total:
+                expect = l
+                break
+        assert p.gpu.suggest_offload(frac) == expect, frac
+    assert p.gpu.exit_histogram(reset=True) == want.tolist() and sum(p.gpu.exit_histogram()) == 0
+    p.close()
