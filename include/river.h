@@ -196,7 +196,8 @@ int river_generate(river_ctx *ctx, int batch, const int32_t *slots, const int32_
  *       staging slots (blocks l and l + 2 the same seven pointers): a block is staged while the previous one runs.
  * With offloading on, a step synchronises with the host once per offloaded block (the host must see whether any row is
  * still in the backbone before it copies 2 P bytes), graph replay is off and the exit score runs as a kernel of its
- * own.  first_offloaded_layer = 0 turns it off.  river_stats.offload_fetches counts the block copies. */
+ * own.  first_offloaded_layer = 0 turns it off.  river_stats.offload_fetches counts the block copies.  Not with
+ * RIVER_KV_STATE_PROPAGATION (which needs the backbone K / V matrices of every skipped block). */
 int river_offload(river_ctx *ctx, int first_offloaded_layer, const river_layer_weights *host_layers);
 
 /* Which blocks are sparsely used (Section 4.2: the blocks to offload follow from where the tokens leave).

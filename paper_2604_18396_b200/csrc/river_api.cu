@@ -1085,6 +1085,8 @@ int river_offload(river_ctx *c, int first_offloaded_layer, const river_layer_wei
     const river_config &g = c->cfg;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     if (first_offloaded_layer == 0) { c->off_first = 0; return RIVER_OK; }
+    if (g.kv_strategy == RIVER_KV_STATE_PROPAGATION)
+        return fail(c, RIVER_E_BADARG, "State Propagation projects K / V with every skipped block's backbone matrices: they cannot be offloaded");
     if (first_offloaded_layer < 2 || first_offloaded_layer > g.L || !host_layers)
         return fail(c, RIVER_E_BADARG, "first_offloaded_layer must be 0 or lie in [2, L], with the host copies given");
     for (int l = first_offloaded_layer; l <= g.L; ++l) {

@@ -118,3 +118,12 @@ def test_exit_histogram_and_offload_suggestion():
         assert p.gpu.suggest_offload(frac) == expect, frac
     assert p.gpu.exit_histogram(reset=True) == want.tolist() and sum(p.gpu.exit_histogram()) == 0
     p.close()
+
+
+def test_offload_is_refused_under_state_propagation():
+    # State Propagation projects K / V with every skipped block's backbone matrices: none of them may live on the host
+    model, host = offloaded_model("mini8", 3)
+    p = Pair(model, max_seqs=1, max_len=32, max_batch=4, kv_strategy=1)
+    with pytest.raises(RuntimeError):
+        p.gpu.offload(3, host)
+    p.close()
