@@ -287,6 +287,7 @@ struct TcArgs {
     int n_pad;        // N operand rows (multiple of 16, <= 256)
     int splits;       // K splits per tile = CTAs per cluster (<= 8)
     int n_stages;     // pipeline depth
+    int one_box;      // 1: map_bhi covers the hi rows AND the lo rows behind them: one copy of 2 n_pad rows per k-block
     int wide;         // 1: hi and lo operand rows as one operand of 2 n_pad rows (the host checks the TMEM budget)
     int a_rows_per_map;  // a tile's 128 rows come from map tile_idx / (rows_per_map / 128) ... see tile_map()
     int gateup;       // 1: a tile is 64 rows of map 0 + 64 rows of map 1
@@ -456,7 +457,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     auto load_b = [&](uint32_t s, int x) {
         const uint32_t full = full0 + 8 * s, dst = stage0 + s * stage_bytes + a_bytes;
         tma_load_2d(dst, &map_bhi, x, 0, full);
-        tma_load_2d(dst + b_bytes, &map_blo, x, 0, full);
+        if (!a.one_box) tma_load_2d(dst + b_bytes, &map_blo, x, 0, full);
     };
 
     // weights first: they depend on nothing

@@ -9,8 +9,10 @@ namespace river {
 const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
     for (auto &b : c->tc_bmaps)
         if (b.K == K && b.np == np) return &b;
-    river_ctx::BMap b{K, np, {}, {}};
-    if (!make_map_bf16(&b.hi, c->tc_xhi, K, np, np) || !make_map_bf16(&b.lo, c->tc_xlo, K, np, np)) return nullptr;
+    river_ctx::BMap b{K, np, 2 * np <= 256, nullptr, {}, {}};
+    b.lo_ptr = b.one ? c->tc_xhi + (size_t)np * K : c->tc_xlo;
+    const int hi_rows = b.one ? 2 * np : np;  // a box holds at most 256 rows
+    if (!make_map_bf16(&b.hi, c->tc_xhi, K, hi_rows, hi_rows) || !make_map_bf16(&b.lo, b.lo_ptr, K, np, np)) return nullptr;
     c->tc_bmaps.push_back(b);
     return &c->tc_bmaps.back();
 }
@@ -39,11 +41,11 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
     const river_ctx::BMap *bm = tc_bmap(c, K, np);
     if (!bm) return cudaErrorInvalidValue;
     cudaError_t e = launch_k(tc_prep_kernel, dim3(np, (K + kPrepChunk - 1) / kPrepChunk), dim3(256), 0, c->stream, true, in, rows, cnt, K,
-                             c->tc_xhi, c->tc_xlo);
+                             c->tc_xhi, bm->lo_ptr);
     if (e != cudaSuccess) return e;
     ++c->st.launches_last_step;
     TcArgs a{};
-    a.K = K; a.n_pad = np;
+    a.K = K; a.n_pad = np; a.one_box = bm->one ? 1 : 0;
     const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
     // CTAs per SM: two with three stages each, or three with two when that puts more CTAs of one wave to work (while
     // one CTA drains its accumulator and takes part in the cluster reduction the others keep the weight stream going);

@@ -15,29 +15,35 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
     if (!bm) return cudaErrorInvalidValue;
     cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np, (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk)), dim3(256), 0, c->stream, true, in, rows,
                              cnt, K,
-                             reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(c->tc_xlo));
+                             reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(bm->lo_ptr));
     if (e != cudaSuccess) return e;
     ++c->st.launches_last_step;
     TcW4Args a{};
-    a.K = K; a.n_pad = np;
-    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
+    a.K = K; a.n_pad = np; a.one_box = bm->one ? 1 : 0;
+    const size_t stage = 2 * (size_t)np * kTcBK * 2;  // the activations' hi and lo tiles; the A tiles are in tensor memory
     const size_t raw = (size_t)kW4RawBufs * kW4RawBytes;
-    // two CTAs per SM (16 dequantisation warps) when two operand stages fit in half of the shared memory
+    // two CTAs per SM (16 dequantisation warps) when two stages fit in half of the shared memory; an even number of
+    // stages (the two dequantisation warps of a lane quarter alternate)
     const bool two = 2 * stage + raw + 4096 <= 110 * 1024;
     a.n_stages = two ? (int)std::min<size_t>(4, (110 * 1024 - raw - 4096) / stage)
-                     : (int)std::max<size_t>(2, std::min<size_t>(6, (214 * 1024 - raw) / stage));
+                     : (int)std::max<size_t>(2, std::min<size_t>(4, (214 * 1024 - raw) / stage));
+    a.n_stages &= ~1;
     // in raw tiles of four k-blocks: at least four per split, two when K is so short that four would allow only two
     // splits (measured on the 1B shape, K = 2048: 2 -> 4 splits 35 -> 31 us per layer for QKV, 33 -> 27 us for O)
     const int raw_tiles = K / (kTcBK * kW4Super);
     a.splits = tc_pick_splits(c, tiles, raw_tiles, c->num_sms * (two ? 2 : 1), raw_tiles <= 8 ? 2 : 4);
     if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage + raw) return cudaErrorInvalidValue;
-    int cols = 32;  // (see launch_tc: every CTA resident on an SM must get its accumulator columns at once)
-    while (cols < 2 * np) cols <<= 1;
-    a.wide = (2 * np <= 256 && (two ? 2 : 1) * cols <= 512) ? 1 : 0;
+    // tensor memory: accumulator + A tiles, a power of two of columns; every CTA that can be resident on an SM must get
+    // its columns at once (a CTA stuck in the allocation while its cluster waits for it could not be waited out), so
+    // the shared-memory request is padded until no more than `occ` CTAs fit
+    const int occ = two ? 2 : 1;
+    auto cols_for = [&](int acc) { int cols = 32; while (cols < acc + a.n_stages * (int)kW4ACols) cols <<= 1; return cols; };
+    a.wide = (2 * np <= 256 && occ * cols_for(2 * np) <= 512) ? 1 : 0;
+    if (occ * cols_for(a.wide ? 2 * np : np) > 512) return cudaErrorInvalidValue;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
     a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
-    const size_t smem = tc_w4_smem_bytes(np, a.n_stages);
+    const size_t smem = std::max(tc_w4_smem_bytes(np, a.n_stages), (size_t)(228 * 1024) / (occ + 1) + 1024);
     e = ensure_smem(c, tc_gemm_w4_kernel<Epi>, smem);
     if (e != cudaSuccess) return e;
     return launch_kc(tc_gemm_w4_kernel<Epi>, dim3(tiles * a.splits), dim3(kW4Threads), smem, c->stream, true, a.splits,

@@ -121,7 +121,8 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     unsigned long long *ehist = cv.take<unsigned long long>((size_t)c->L + 1);
     const size_t tc_pad = std::min<size_t>(256, (B + 15) / 16 * 16);
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
-    __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(tc_pad * tc_kmax), *txl = cv.take<__nv_bfloat16>(tc_pad * tc_kmax);
+    // one allocation: lo rows may start right behind the hi rows in use (launch_tc.cu: tc_bmap)
+    __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax), *txl = txh ? txh + tc_pad * tc_kmax : nullptr;
 
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;

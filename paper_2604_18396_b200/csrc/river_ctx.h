@@ -42,7 +42,9 @@ struct river_ctx {
     std::vector<LayerMaps> w4_maps;  // code matrices of the exit layers (u8 [rows][K/2], 128-byte boxes)
     bool w4tc_ok = false;
     CUtensorMap tc_map_head;
-    struct BMap { int K, np; CUtensorMap hi, lo; };
+    // operand maps of the tensor-core projections for (K, padded rows): up to 128 rows the lo rows follow the hi rows
+    // in one buffer (`lo_ptr` = tc_xhi + np K) and `hi` covers both (one copy per k-block); beyond, two buffers
+    struct BMap { int K, np; bool one; __nv_bfloat16 *lo_ptr; CUtensorMap hi, lo; };
     std::vector<BMap> tc_bmaps;
     int32_t *hint_act;
     const uint8_t *attn_skip = nullptr;  // exit flags of the block whose attention is being launched (strategies that run nothing for rows that left), else null
