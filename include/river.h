@@ -49,8 +49,10 @@ enum {
     RIVER_F_NO_TC = 2,    /* diagnostic: every projection on the CUDA-core kernels, never the tcgen05 GEMMs */
     RIVER_F_NO_W4TC = 16, /* diagnostic: exit-layer rows of batches on the CUDA-core kernel instead of the dequantising
                              tcgen05 GEMM */
-    RIVER_F_TMA_ATTN = 32 /* diagnostic: steps of 1-4 rows through the TMA-fed attention kernel too (default: the
-                             small-step kernel) */
+    RIVER_F_TMA_ATTN = 32, /* diagnostic: steps of 1-4 rows through the TMA-fed attention kernel too (default: the
+                              small-step kernel) */
+    RIVER_F_SERIAL_TC = 64 /* diagnostic: the two tcgen05 GEMMs of a projection (backbone rows, exit-layer rows) one
+                              after the other (default: in flight together) */
 };
 
 typedef struct river_config {

@@ -17,7 +17,7 @@ from . import buildlib as _build
 # ---------------------------------------------------------------- C structs (mirror include/river.h)
 RIVER_OK = 0
 RIVER_EXIT_PER_TOKEN, RIVER_EXIT_BATCH_MIN = 0, 1
-RIVER_F_GRAPH, RIVER_F_NO_TC, RIVER_F_NO_W4TC, RIVER_F_TMA_ATTN = 1, 2, 16, 32
+RIVER_F_GRAPH, RIVER_F_NO_TC, RIVER_F_NO_W4TC, RIVER_F_TMA_ATTN, RIVER_F_SERIAL_TC = 1, 2, 16, 32, 64
 ERR_NAMES = {-1: "BADARG", -2: "SHAPE", -3: "NOMEM", -4: "NOPAGE", -5: "BADSLOT", -6: "DEVICE", -7: "TIMEOUT"}
 
 

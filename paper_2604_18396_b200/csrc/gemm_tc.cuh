@@ -287,6 +287,7 @@ struct TcArgs {
     int n_pad;        // N operand rows (multiple of 16, <= 256)
     int splits;       // K splits per tile = CTAs per cluster (<= 8)
     int n_stages;     // pipeline depth
+    int late_release; // 1: dependent grids may start only once this grid's own dependency is met (see the kernel)
     int one_box;      // 1: map_bhi covers the hi rows AND the lo rows behind them: one copy of 2 n_pad rows per k-block
     int wide;         // 1: hi and lo operand rows as one operand of 2 n_pad rows (the host checks the TMEM budget)
     int a_rows_per_map;  // a tile's 128 rows come from map tile_idx / (rows_per_map / 128) ... see tile_map()
@@ -406,7 +407,10 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < acc_n) tmem_cols <<= 1;
 
-    pdl_launch();
+    // `late_release`: the next grid in the stream is the dequantising kernel of the same projection, which runs beside
+    // this one instead of behind it: it never waits for this grid at its start, so it may only start once everything
+    // BOTH read (the operand kernels' output) is complete - that is when every CTA here is past its own wait.
+    if (!a.late_release) pdl_launch();
     if (tid == 0) s_some = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
     __syncthreads();
     if (!s_some) {  // every row has left the backbone: nothing to fetch, nothing to compute (uniform over the cluster:
@@ -465,6 +469,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     if (tid == 0)
         for (int i = 0; i < pre; ++i) load_a((uint32_t)i);
     pdl_wait();
+    if (a.late_release) pdl_launch();
     const int n_live = *a.cnt;  // rows of the backbone list; the stream kernel serves the exit-layer rows
     // even with no live row the requested weight tiles must land before the CTA may exit: run the pipeline once
     const int nkb_run = n_live > 0 ? nkb : pre;

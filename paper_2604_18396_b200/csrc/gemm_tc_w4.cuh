@@ -115,6 +115,8 @@ struct TcW4Args {
     int n_pad;         // N operand rows (multiple of 16, <= 256)
     int splits;        // K splits per tile = CTAs per cluster (<= 8), in whole raw tiles
     int n_stages;      // stages: activation tiles in shared memory AND A tiles in tensor memory (even)
+    int overlap;       // 1: runs beside the preceding grid (tc_gemm_kernel of the same projection, launched with
+                       // late_release): no wait at the start, the wait for that grid comes before the CTA exits
     int one_box;       // 1: map_bhi covers the hi rows AND the lo rows behind them: one copy of 2 n_pad rows per k-block
     int wide;          // 1: hi and lo activation rows as one operand of 2 n_pad rows (the host checks the TMEM budget)
     int gateup;        // 1: a tile is 64 rows of matrix 0 + 64 rows of matrix 1
@@ -224,9 +226,16 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
     const int pre = early ? min(kW4RawBufs, nsb) : 0;
     if (tid == 0)
         for (int sb = 0; sb < pre; ++sb) load_raw(sb);
-    pdl_wait();
+    // Beside the backbone kernel of the same projection (`overlap`): that grid let this one start only after the
+    // operand kernels of both had completed, the two write disjoint rows, and the row count dates from the previous
+    // block - nothing here depends on it.  Whoever comes next in the stream waits for THIS grid, so this grid must not
+    // complete before that one: every CTA waits for it just before it exits.
+    if (!a.overlap) pdl_wait();
     const int n_live = *a.cnt;
-    if (n_live <= 0 && pre == 0) return;  // uniform over the CTA and the cluster (nobody reaches a cluster barrier)
+    if (n_live <= 0 && pre == 0) {  // uniform over the CTA and the cluster (nobody reaches a cluster barrier)
+        if (a.overlap) pdl_wait();
+        return;
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(tmem_cols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
@@ -366,6 +375,7 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
     tc_fence_after();
     __syncthreads();  // all copies into and MMA reads of the pipeline memory are over: it now holds the tile
     tc_finish(epi, tile, tmem_d, tmem_cols, NP, a.splits, split, tile_idx, n_live, a.rows, ok, &s_abort, kW4Threads, wide);
+    if (a.overlap) pdl_wait();
 }
 
 inline size_t tc_w4_smem_bytes(int n_pad, int n_stages) {

@@ -6,13 +6,14 @@
 
 namespace river {
 
-const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np) {
+const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np, bool w4) {
     for (auto &b : c->tc_bmaps)
-        if (b.K == K && b.np == np) return &b;
-    river_ctx::BMap b{K, np, 2 * np <= 256, nullptr, {}, {}};
-    b.lo_ptr = b.one ? c->tc_xhi + (size_t)np * K : c->tc_xlo;
+        if (b.K == K && b.np == np && b.w4 == w4) return &b;
+    river_ctx::BMap b{K, np, w4, 2 * np <= 256, nullptr, {}, {}};
+    __nv_bfloat16 *base = w4 ? c->tc_x4 : c->tc_xhi;
+    b.lo_ptr = b.one ? base + (size_t)np * K : base + (size_t)c->tc_max_pad * c->tc_kmax;
     const int hi_rows = b.one ? 2 * np : np;  // a box holds at most 256 rows
-    if (!make_map_bf16(&b.hi, c->tc_xhi, K, hi_rows, hi_rows) || !make_map_bf16(&b.lo, b.lo_ptr, K, np, np)) return nullptr;
+    if (!make_map_bf16(&b.hi, base, K, hi_rows, hi_rows) || !make_map_bf16(&b.lo, b.lo_ptr, K, np, np)) return nullptr;
     c->tc_bmaps.push_back(b);
     return &c->tc_bmaps.back();
 }
@@ -33,40 +34,72 @@ int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots, int m
     return best;
 }
 
+namespace {
+
+constexpr size_t kSmSmem = 228 * 1024;
+constexpr size_t kCtaFixed = 1024 + 1024 + 256;  // per CTA: system reserve, alignment slack, barriers
+
+size_t tc_stage_bytes(int np) { return (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2; }
+// pipeline stages with `occ` CTAs per SM (0: they do not fit)
+int tc_stages_at(int np, int occ) {
+    const size_t stage = tc_stage_bytes(np), room = std::min<size_t>(kSmSmem / occ, 227 * 1024);
+    return room < kCtaFixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : 3, (room - kCtaFixed) / stage);
+}
+// hi | lo as one operand doubles the accumulator columns; all CTAs that can be resident on an SM must get their
+// tensor memory at once (a CTA stuck in the allocation while its cluster waits for it could not be waited out)
+int tc_cols(int np, int occ, int *wide) {
+    int cols = 32;
+    while (cols < 2 * np) cols <<= 1;
+    *wide = (2 * np <= 256 && occ * cols <= 512) ? 1 : 0;
+    if (!*wide) { cols = 32; while (cols < np) cols <<= 1; }
+    return cols;
+}
+
+}  // namespace
+
+int tc_footprints(int np, TcFootprint (&out)[2]) {
+    int n = 0;
+    for (int occ = tc_stages_at(np, 2) ? 2 : 1; occ <= 3; ++occ) {
+        const int st = tc_stages_at(np, occ);
+        if (!st) break;
+        int wide;
+        out[n].cols = tc_cols(np, occ, &wide);
+        out[n].smem = tc_smem_bytes(np, st);
+        if (++n == 2 || occ == 1) break;
+    }
+    return n;
+}
+
 template <class Epi>
 cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
                       int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                      const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint) {
+                      const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint, int phase,
+                      bool late_release) {
     const int np = (n + 15) / 16 * 16;
     const river_ctx::BMap *bm = tc_bmap(c, K, np);
     if (!bm) return cudaErrorInvalidValue;
-    cudaError_t e = launch_k(tc_prep_kernel, dim3(np, (K + kPrepChunk - 1) / kPrepChunk), dim3(256), 0, c->stream, true, in, rows, cnt, K,
-                             c->tc_xhi, bm->lo_ptr);
-    if (e != cudaSuccess) return e;
-    ++c->st.launches_last_step;
+    cudaError_t e = cudaSuccess;
+    if (phase & kTcPrep) {
+        e = launch_k(tc_prep_kernel, dim3(np, (K + kPrepChunk - 1) / kPrepChunk), dim3(256), 0, c->stream, true, in, rows, cnt, K,
+                     c->tc_xhi, bm->lo_ptr);
+        if (e != cudaSuccess) return e;
+        ++c->st.launches_last_step;
+    }
+    if (!(phase & kTcGemm)) return e;
     TcArgs a{};
-    a.K = K; a.n_pad = np; a.one_box = bm->one ? 1 : 0;
-    const size_t stage = (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)np * kTcBK * 2;
+    a.K = K; a.n_pad = np; a.one_box = bm->one ? 1 : 0; a.late_release = late_release ? 1 : 0;
+    const size_t stage = tc_stage_bytes(np);
     // CTAs per SM: two with three stages each, or three with two when that puts more CTAs of one wave to work (while
     // one CTA drains its accumulator and takes part in the cluster reduction the others keep the weight stream going);
     // one with deep stages when the operand tiles are too large for that.
-    const size_t sm_smem = 228 * 1024, fixed = 1024 + 1024 + 256;  // per CTA: system reserve, alignment slack, barriers
-    auto stages_at = [&](int occ) {
-        const size_t room = std::min<size_t>(sm_smem / occ, 227 * 1024);
-        return room < fixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : 3, (room - fixed) / stage);
-    };
-    int occ = stages_at(2) ? 2 : 1;
+    int occ = tc_stages_at(np, 2) ? 2 : 1;
     a.splits = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * occ);
-    if (occ == 2 && stages_at(3) && allow_split) {
+    if (occ == 2 && tc_stages_at(np, 3) && allow_split) {
         const int s3 = tc_pick_splits(c, tiles, K / kTcBK, c->num_sms * 3);
         if (tiles * s3 > tiles * a.splits && tiles * s3 <= c->num_sms * 3) { occ = 3; a.splits = s3; }
     }
-    a.n_stages = stages_at(occ);
-    // hi | lo as one operand doubles the accumulator columns; all CTAs that can be resident on an SM must get their
-    // tensor memory at once (a CTA stuck in the allocation while its cluster waits for it could not be waited out)
-    int cols = 32;
-    while (cols < 2 * np) cols <<= 1;
-    a.wide = (2 * np <= 256 && occ * cols <= 512) ? 1 : 0;
+    a.n_stages = tc_stages_at(np, occ);
+    tc_cols(np, occ, &a.wide);
     // the finished tile lives in the pipeline memory
     if (sizeof(float) * (size_t)np * kTcLd > (size_t)a.n_stages * stage) return cudaErrorInvalidValue;
     if (!allow_split) a.splits = 1;
@@ -81,7 +114,8 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
 }
 #define RIVER_TC_INST(E) \
     template cudaError_t launch_tc<E>(river_ctx *, const ProjIn &, const CUtensorMap &, const CUtensorMap &, const CUtensorMap &, \
-                                      int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *);
+                                      int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *, \
+                                      int, bool);
 RIVER_TC_INST(TcQkvEpi) RIVER_TC_INST(TcResidEpi) RIVER_TC_INST(TcGateUpEpi) RIVER_TC_INST(TcHeadEpi)
 #undef RIVER_TC_INST
 

@@ -5,17 +5,27 @@
 
 namespace river {
 
-const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np);
+const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np, bool w4 = false);
+
+// Both kernels of a projection (backbone rows, exit-layer rows) are in flight together: `phase` says which part of a
+// launch function runs - the operand kernel, the GEMM, or both in a row.
+enum : int { kTcPrep = 1, kTcGemm = 2, kTcBoth = 3 };
+// Shared memory and tensor-memory columns per CTA of the configurations tc_gemm_kernel may run in for `np` operand
+// rows (two or three CTAs per SM): what a kernel that shares the SMs with it must budget against.
+struct TcFootprint { size_t smem; int cols; };
+int tc_footprints(int np, TcFootprint (&out)[2]);
 int tc_pick_splits(const river_ctx *c, int tiles, int kb_total, int slots, int min_kb = 4);
 
 // launch_tc.cu: backbone rows, 5 <= rows <= 256
 template <class Epi>
 cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
                       int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                      const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint);
+                      const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint, int phase = kTcBoth,
+                      bool late_release = false);
 #define RIVER_TC_DECL(E) \
     extern template cudaError_t launch_tc<E>(river_ctx *, const ProjIn &, const CUtensorMap &, const CUtensorMap &, const CUtensorMap &, \
-                                             int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *);
+                                             int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *, \
+                                             int, bool);
 RIVER_TC_DECL(TcQkvEpi) RIVER_TC_DECL(TcResidEpi) RIVER_TC_DECL(TcGateUpEpi) RIVER_TC_DECL(TcHeadEpi)
 #undef RIVER_TC_DECL
 
@@ -24,10 +34,11 @@ RIVER_TC_DECL(TcQkvEpi) RIVER_TC_DECL(TcResidEpi) RIVER_TC_DECL(TcGateUpEpi) RIV
 template <class Epi>
 cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
                          int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                         const int32_t *cnt, const int32_t *hint, const Epi &epi);
+                         const int32_t *cnt, const int32_t *hint, const Epi &epi, int phase = kTcBoth, bool overlap = false);
 #define RIVER_TCW4_DECL(E) \
     extern template cudaError_t launch_tc_w4<E>(river_ctx *, const ProjIn &, const CUtensorMap *const (&)[3], const river_w4 *const (&)[3], \
-                                                int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &);
+                                                int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &, \
+                                                int, bool);
 RIVER_TCW4_DECL(TcQkvEpi) RIVER_TCW4_DECL(TcResidEpi) RIVER_TCW4_DECL(TcGateUpEpi)
 #undef RIVER_TCW4_DECL
 

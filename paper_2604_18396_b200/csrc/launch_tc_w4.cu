@@ -9,15 +9,18 @@ namespace river {
 template <class Epi>
 cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
                          int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                         const int32_t *cnt, const int32_t *hint, const Epi &epi) {
+                         const int32_t *cnt, const int32_t *hint, const Epi &epi, int phase, bool overlap) {
     const int np = (n + 15) / 16 * 16;
-    const river_ctx::BMap *bm = tc_bmap(c, K, np);
+    const river_ctx::BMap *bm = tc_bmap(c, K, np, true);
     if (!bm) return cudaErrorInvalidValue;
-    cudaError_t e = launch_k(tc_prep_w4_kernel, dim3(np, (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk)), dim3(256), 0, c->stream, true, in, rows,
-                             cnt, K,
-                             reinterpret_cast<__half *>(c->tc_xhi), reinterpret_cast<__half *>(bm->lo_ptr));
-    if (e != cudaSuccess) return e;
-    ++c->st.launches_last_step;
+    cudaError_t e = cudaSuccess;
+    if (phase & kTcPrep) {
+        e = launch_k(tc_prep_w4_kernel, dim3(np, (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk)), dim3(256), 0, c->stream, true, in,
+                     rows, cnt, K, reinterpret_cast<__half *>(c->tc_x4), reinterpret_cast<__half *>(bm->lo_ptr));
+        if (e != cudaSuccess) return e;
+        ++c->st.launches_last_step;
+    }
+    if (!(phase & kTcGemm)) return e;
     TcW4Args a{};
     a.K = K; a.n_pad = np; a.one_box = bm->one ? 1 : 0;
     const size_t stage = 2 * (size_t)np * kTcBK * 2;  // the activations' hi and lo tiles; the A tiles are in tensor memory
@@ -39,11 +42,28 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
     const int occ = two ? 2 : 1;
     auto cols_for = [&](int acc) { int cols = 32; while (cols < acc + a.n_stages * (int)kW4ACols) cols <<= 1; return cols; };
     a.wide = (2 * np <= 256 && occ * cols_for(2 * np) <= 512) ? 1 : 0;
-    if (occ * cols_for(a.wide ? 2 * np : np) > 512) return cudaErrorInvalidValue;
+    const int cols = cols_for(a.wide ? 2 * np : np);
+    if (occ * cols > 512) return cudaErrorInvalidValue;
+    const size_t sm_smem = 228 * 1024;
+    size_t smem = std::max(tc_w4_smem_bytes(np, a.n_stages), sm_smem / (occ + 1) + 1024);
+    // CTAs of tc_gemm_kernel share the SMs with this kernel (beside it when `overlap`, and the next projection's may
+    // take their tensor memory while CTAs of this grid are still to come): whatever mix of the two fits into an SM's
+    // shared memory must fit into its 512 columns as well - pad the request until it does
+    TcFootprint fp[2];
+    const int nfp = tc_footprints(np, fp);
+    auto mix_ok = [&](size_t mine) {
+        for (int f = 0; f < nfp; ++f)
+            for (int i = 0; i <= 8; ++i)
+                for (int j = 0; j <= occ; ++j)
+                    if (i * fp[f].smem + j * mine <= sm_smem && i * fp[f].cols + j * cols > 512) return false;
+        return true;
+    };
+    while (!mix_ok(smem) && smem + 4096 <= sm_smem / occ - 1024) smem += 4096;
+    if (!mix_ok(smem)) return cudaErrorInvalidValue;
+    a.overlap = overlap ? 1 : 0;
     a.gateup = gateup; a.qkv_q_tiles = q_tiles; a.qkv_k_tiles = k_tiles;
     for (int i = 0; i < 3; ++i) { a.scale[i] = (const uint16_t *)w[i]->scale; a.zero[i] = (const uint16_t *)w[i]->zero; }
     a.rows = rows; a.cnt = cnt; a.hint = hint; a.dev_err = c->dev_err;
-    const size_t smem = std::max(tc_w4_smem_bytes(np, a.n_stages), (size_t)(228 * 1024) / (occ + 1) + 1024);
     e = ensure_smem(c, tc_gemm_w4_kernel<Epi>, smem);
     if (e != cudaSuccess) return e;
     return launch_kc(tc_gemm_w4_kernel<Epi>, dim3(tiles * a.splits), dim3(kW4Threads), smem, c->stream, true, a.splits,
@@ -51,7 +71,8 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
 }
 #define RIVER_TCW4_INST(E) \
     template cudaError_t launch_tc_w4<E>(river_ctx *, const ProjIn &, const CUtensorMap *const (&)[3], const river_w4 *const (&)[3], \
-                                         int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &);
+                                         int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &, \
+                                         int, bool);
 RIVER_TCW4_INST(TcQkvEpi) RIVER_TCW4_INST(TcResidEpi) RIVER_TCW4_INST(TcGateUpEpi)
 #undef RIVER_TCW4_INST
 

@@ -123,6 +123,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     const size_t tc_kmax = std::max<size_t>(std::max<size_t>(c->d, c->F), (size_t)c->Hq * c->dh);
     // one allocation: lo rows may start right behind the hi rows in use (launch_tc.cu: tc_bmap)
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax), *txl = txh ? txh + tc_pad * tc_kmax : nullptr;
+    __nv_bfloat16 *tx4 = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax);
 
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
@@ -131,7 +132,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->state = exd; x->state_stride = (int)sstride; x->prefill_fail = pff;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
         x->slot_cap = scap; x->pos_depth = pdep; x->exit_hist = ehist;
-        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
+        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_x4 = tx4; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
 }
@@ -372,6 +373,24 @@ int offload_before_layer(river_ctx *c, int l, bool *staged) {
     return RIVER_OK;
 }
 
+// The tensor-core kernels of one projection: `backbone(phase, late_release)` launches tc_gemm_kernel's part,
+// `river(phase, beside)` the dequantising kernel's.  With both, the two operand kernels go first and the two GEMMs
+// share the device: the first lets the second start once the operands are complete, the second waits for the first
+// before it ends (the kernels' comments say why that is enough); RIVER_F_SERIAL_TC keeps them one after the other.
+template <class Bb, class Rv>
+cudaError_t tc_pair(river_ctx *c, bool with_river, Bb &&backbone, Rv &&river) {
+    if (!with_river) return backbone(kTcBoth, false);
+    cudaError_t e;
+    if (c->cfg.flags & RIVER_F_SERIAL_TC) {
+        if ((e = backbone(kTcBoth, false)) != cudaSuccess) return e;
+        return river(kTcBoth, false);
+    }
+    if ((e = backbone(kTcPrep, false)) != cudaSuccess) return e;
+    if ((e = river(kTcPrep, false)) != cudaSuccess) return e;
+    if ((e = backbone(kTcGemm, true)) != cudaSuccess) return e;
+    return river(kTcGemm, true);
+}
+
 // a2 of block l for the n rows of the step: attention norm + QKV + RoPE + KV write, on the weight set(s) the row
 // lists name (small steps: from the exit flags).
 cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const DecideArgs &dec, double kv_write) {
@@ -402,16 +421,20 @@ cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const Deci
     p.rope_cs = c->rope_cs; p.q_out = c->qbuf; p.kv = kv_addr(c, l - 1); p.dev_err = c->dev_err;
     const ProjIn in{h_in, (const uint16_t *)w.attn_norm, g.rms_eps};
     if (tc) {
-        TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
-        note(launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ai, na,
-                       e, true, c->hint_act));
-    }
-    if (wm) {
-        TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
-        const CUtensorMap *const cm[3] = {&wm->q, &wm->k, &wm->v};
+        const TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
+        const CUtensorMap *const cm[3] = {wm ? &wm->q : nullptr, wm ? &wm->k : nullptr, wm ? &wm->v : nullptr};
         const river_w4 *const cw[3] = {&w.rq, &w.rk, &w.rv};
-        note(launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM, ri, nr, nrh, e));
-    } else if (!tc || has_river) {
+        note(tc_pair(c, wm != nullptr,
+                     [&](int phase, bool late) {
+                         return launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM,
+                                          kvdim / kTcBM, ai, na, e, true, c->hint_act, phase, late);
+                     },
+                     [&](int phase, bool beside) {
+                         return launch_tc_w4(c, in, cm, cw, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM, kvdim / kTcBM,
+                                             ri, nr, nrh, e, phase, beside);
+                     }));
+    }
+    if (!wm && (!tc || has_river)) {
         note(launch_stream(c, p, in, rl, d, (g.Hq + 2 * g.Hkv) * (g.dh / 2), n, has_river, true, tc ? 1 : 0, dec));
     }
     if (strat == RIVER_KV_STATE_PROPAGATION) {
@@ -531,15 +554,19 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
             p.resid = h_in; p.out = h_mid;
             const ProjIn in{c->obuf, nullptr, 0.f};
             if (tc) {
-                TcResidEpi e{h_in, h_mid, d};
-                note(launch_tc(c, in, tm->o, tm->o, tm->o, qdim, d / kTcBM, n, 0, 0, 0, ai, na, e, true, c->hint_act));
-            }
-            if (wm) {
-                TcResidEpi e{h_in, h_mid, d};
-                const CUtensorMap *const cm[3] = {&wm->o, &wm->o, &wm->o};
+                const TcResidEpi e{h_in, h_mid, d};
+                const CUtensorMap *const cm[3] = {wm ? &wm->o : nullptr, wm ? &wm->o : nullptr, wm ? &wm->o : nullptr};
                 const river_w4 *const cw[3] = {&w.ro, &w.ro, &w.ro};
-                note(launch_tc_w4(c, in, cm, cw, qdim, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
-            } else if (!tc || has_river)
+                note(tc_pair(c, wm != nullptr,
+                             [&](int phase, bool late) {
+                                 return launch_tc(c, in, tm->o, tm->o, tm->o, qdim, d / kTcBM, n, 0, 0, 0, ai, na, e, true,
+                                                  c->hint_act, phase, late);
+                             },
+                             [&](int phase, bool beside) {
+                                 return launch_tc_w4(c, in, cm, cw, qdim, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e, phase, beside);
+                             }));
+            }
+            if (!wm && (!tc || has_river))
                 note(launch_stream(c, p, in, rl, qdim, d / 2, n, has_river, true, skip_bb, no_dec));
         }
         // ---- a5: FFN norm + gate/up + SwiGLU
@@ -551,15 +578,19 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
             p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
             const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
             if (tc) {
-                TcGateUpEpi e{c->act, g.F};
-                note(launch_tc(c, in, tm->g, tm->u, tm->u, d, g.F / 64, n, 1, 0, 0, ai, na, e, true, c->hint_act));
-            }
-            if (wm) {
-                TcGateUpEpi e{c->act, g.F};
-                const CUtensorMap *const cm[3] = {&wm->g, &wm->u, &wm->u};
+                const TcGateUpEpi e{c->act, g.F};
+                const CUtensorMap *const cm[3] = {wm ? &wm->g : nullptr, wm ? &wm->u : nullptr, wm ? &wm->u : nullptr};
                 const river_w4 *const cw[3] = {&w.rg, &w.ru, &w.ru};
-                note(launch_tc_w4(c, in, cm, cw, d, g.F / 64, n, 1, 0, 0, ri, nr, nrh, e));
-            } else if (!tc || has_river) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb, no_dec));
+                note(tc_pair(c, wm != nullptr,
+                             [&](int phase, bool late) {
+                                 return launch_tc(c, in, tm->g, tm->u, tm->u, d, g.F / 64, n, 1, 0, 0, ai, na, e, true,
+                                                  c->hint_act, phase, late);
+                             },
+                             [&](int phase, bool beside) {
+                                 return launch_tc_w4(c, in, cm, cw, d, g.F / 64, n, 1, 0, 0, ri, nr, nrh, e, phase, beside);
+                             }));
+            }
+            if (!wm && (!tc || has_river)) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb, no_dec));
         }
         // ---- a5: down projection + residual
         {
@@ -570,15 +601,19 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
             p.resid = h_mid; p.out = h_out;
             const ProjIn in{c->act, nullptr, 0.f};
             if (tc) {
-                TcResidEpi e{h_mid, h_out, d};
-                note(launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e, true, c->hint_act));
-            }
-            if (wm) {
-                TcResidEpi e{h_mid, h_out, d};
-                const CUtensorMap *const cm[3] = {&wm->d, &wm->d, &wm->d};
+                const TcResidEpi e{h_mid, h_out, d};
+                const CUtensorMap *const cm[3] = {wm ? &wm->d : nullptr, wm ? &wm->d : nullptr, wm ? &wm->d : nullptr};
                 const river_w4 *const cw[3] = {&w.rd, &w.rd, &w.rd};
-                note(launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e));
-            } else if (!tc || has_river)
+                note(tc_pair(c, wm != nullptr,
+                             [&](int phase, bool late) {
+                                 return launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e, true,
+                                                  c->hint_act, phase, late);
+                             },
+                             [&](int phase, bool beside) {
+                                 return launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e, phase, beside);
+                             }));
+            }
+            if (!wm && (!tc || has_river))
                 note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb, no_dec));
         }
         // ---- a6 + a7: exit score, decision, compaction -> row lists entering block l+1
