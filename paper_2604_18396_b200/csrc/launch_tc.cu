@@ -43,7 +43,7 @@ size_t tc_stage_bytes(int np) { return (size_t)kTcBM * kTcBK * 2 + 2 * (size_t)n
 // pipeline stages with `occ` CTAs per SM (0: they do not fit)
 int tc_stages_at(int np, int occ) {
     const size_t stage = tc_stage_bytes(np), room = std::min<size_t>(kSmSmem / occ, 227 * 1024);
-    return room < kCtaFixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : 3, (room - kCtaFixed) / stage);
+    return room < kCtaFixed + 2 * stage ? 0 : (int)std::min<size_t>(occ == 1 ? 8 : occ == 2 ? 4 : 3, (room - kCtaFixed) / stage);
 }
 // hi | lo as one operand doubles the accumulator columns; all CTAs that can be resident on an SM must get their
 // tensor memory at once (a CTA stuck in the allocation while its cluster waits for it could not be waited out)
