@@ -82,14 +82,12 @@ __device__ __forceinline__ float tc_prep_scale(const ProjIn &in, const float4 *s
     for (int w = 0; w < 8; ++w) ss += red[w];
     return rsqrtf(ss / (float)K + in.eps);
 }
-static __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
-                                                      __nv_bfloat16 *xhi, __nv_bfloat16 *xlo) {
-    __shared__ float red[8];
-    pdl_launch();
-    pdl_wait();
-    const int i = blockIdx.x, n = *cnt;
+// (the body of CTA (i, by); `red`: eight floats of shared memory)
+__device__ __forceinline__ void tc_prep_body(const ProjIn &in, const int32_t *idx, const int32_t *cnt, int K,
+                                             __nv_bfloat16 *xhi, __nv_bfloat16 *xlo, int i, int by, float *red) {
+    const int n = *cnt;
     if (n <= 0) return;  // no row in the backbone any more: the GEMM returns before it reads an operand
-    const int v = blockIdx.y * (kPrepChunk / 4) + threadIdx.x;  // 4-input group of the row
+    const int v = by * (kPrepChunk / 4) + threadIdx.x;  // 4-input group of the row
     const bool mine = v < (K >> 2);
     uint2 *hi = reinterpret_cast<uint2 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint2 *>(xlo + (size_t)i * K);
     if (i >= n) {
@@ -117,6 +115,13 @@ static __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, co
     split2(y.z, y.w, h.y, l.y);
     hi[v] = h;
     lo[v] = l;
+}
+static __global__ void __launch_bounds__(256) tc_prep_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
+                                                      __nv_bfloat16 *xhi, __nv_bfloat16 *xlo) {
+    __shared__ float red[8];
+    pdl_launch();
+    pdl_wait();
+    tc_prep_body(in, idx, cnt, K, xhi, xlo, blockIdx.x, blockIdx.y, red);
 }
 
 // ---------------------------------------------------------------- epilogues on a finished 128 x N tile in smem

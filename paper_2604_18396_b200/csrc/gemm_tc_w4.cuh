@@ -62,14 +62,11 @@ __device__ __forceinline__ uint32_t tc_idesc_f16(int n) {  // D fp32, A and B f1
 // ---------------------------------------------------------------- activation rows -> f16 hi / lo operand buffers
 // As tc_prep_kernel (CTA (i, j): inputs [2048 j, 2048 j + 2048) of operand row i, eight per thread), but f16 and with
 // the inputs of every group of eight in the order (0,4,1,5,2,6,3,7).
-static __global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
-                                                         __half *xhi, __half *xlo) {
-    __shared__ float red[8];
-    pdl_launch();
-    pdl_wait();
-    const int i = blockIdx.x, n = *cnt;
+__device__ __forceinline__ void tc_prep_w4_body(const ProjIn &in, const int32_t *idx, const int32_t *cnt, int K,
+                                                __half *xhi, __half *xlo, int i, int by, float *red) {
+    const int n = *cnt;
     if (n <= 0) return;  // no row on the exit layers: the GEMM returns before it reads an operand
-    const int v = blockIdx.y * (2 * kPrepChunk / 8) + threadIdx.x;  // 8-input group of the row
+    const int v = by * (2 * kPrepChunk / 8) + threadIdx.x;  // 8-input group of the row
     const bool mine = v < (K >> 3);
     uint4 *hi = reinterpret_cast<uint4 *>(xhi + (size_t)i * K), *lo = reinterpret_cast<uint4 *>(xlo + (size_t)i * K);
     if (i >= n) {
@@ -107,6 +104,28 @@ static __global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in,
                        (uint32_t)h[2] | ((uint32_t)h[6] << 16), (uint32_t)h[3] | ((uint32_t)h[7] << 16));
     lo[v] = make_uint4((uint32_t)l[0] | ((uint32_t)l[4] << 16), (uint32_t)l[1] | ((uint32_t)l[5] << 16),
                        (uint32_t)l[2] | ((uint32_t)l[6] << 16), (uint32_t)l[3] | ((uint32_t)l[7] << 16));
+}
+static __global__ void __launch_bounds__(256) tc_prep_w4_kernel(const ProjIn in, const int32_t *idx, const int32_t *cnt, int K,
+                                                         __half *xhi, __half *xlo) {
+    __shared__ float red[8];
+    pdl_launch();
+    pdl_wait();
+    tc_prep_w4_body(in, idx, cnt, K, xhi, xlo, blockIdx.x, blockIdx.y, red);
+}
+// Both operand sets of a projection in one launch: CTAs (i, j < ya) are tc_prep_kernel's for the backbone list, CTAs
+// (i, ya + j) tc_prep_w4_kernel's for the list of the rows on the exit layers.
+struct PrepPair {
+    const int32_t *idx_a, *cnt_a, *idx_r, *cnt_r;
+    __nv_bfloat16 *ahi, *alo;
+    __half *rhi, *rlo;
+    int ya;
+};
+static __global__ void __launch_bounds__(256) tc_prep_pair_kernel(const ProjIn in, const PrepPair p, int K) {
+    __shared__ float red[8];
+    pdl_launch();
+    pdl_wait();
+    if ((int)blockIdx.y < p.ya) tc_prep_body(in, p.idx_a, p.cnt_a, K, p.ahi, p.alo, blockIdx.x, blockIdx.y, red);
+    else tc_prep_w4_body(in, p.idx_r, p.cnt_r, K, p.rhi, p.rlo, blockIdx.x, (int)blockIdx.y - p.ya, red);
 }
 
 // ---------------------------------------------------------------- the kernel

@@ -29,6 +29,10 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
 RIVER_TC_DECL(TcQkvEpi) RIVER_TC_DECL(TcResidEpi) RIVER_TC_DECL(TcGateUpEpi) RIVER_TC_DECL(TcHeadEpi)
 #undef RIVER_TC_DECL
 
+// launch_tc_w4.cu: the operand kernels of both lists as one launch (then launch_tc / launch_tc_w4 with kTcGemm)
+cudaError_t launch_tc_prep_pair(river_ctx *c, const ProjIn &in, int K, int n, const int32_t *rows_a, const int32_t *cnt_a,
+                                const int32_t *rows_r, const int32_t *cnt_r);
+
 // launch_tc_w4.cu: exit-layer rows through the dequantising kernel: m[0..2] are the code maps, w[0..2] the matching
 // scale / zero arrays (one matrix, gate + up, or q + k + v)
 template <class Epi>

@@ -6,6 +6,21 @@
 
 namespace river {
 
+cudaError_t launch_tc_prep_pair(river_ctx *c, const ProjIn &in, int K, int n, const int32_t *rows_a, const int32_t *cnt_a,
+                                const int32_t *rows_r, const int32_t *cnt_r) {
+    const int np = (n + 15) / 16 * 16;
+    const river_ctx::BMap *ba = tc_bmap(c, K, np, false);
+    if (!ba) return cudaErrorInvalidValue;
+    __nv_bfloat16 *alo = ba->lo_ptr;  // (the next call may move the map table)
+    const river_ctx::BMap *br = tc_bmap(c, K, np, true);
+    if (!br) return cudaErrorInvalidValue;
+    PrepPair p{rows_a, cnt_a, rows_r, cnt_r, c->tc_xhi, alo, reinterpret_cast<__half *>(c->tc_x4),
+               reinterpret_cast<__half *>(br->lo_ptr), (K + kPrepChunk - 1) / kPrepChunk};
+    const int yr = (K + 2 * kPrepChunk - 1) / (2 * kPrepChunk);
+    ++c->st.launches_last_step;
+    return launch_k(tc_prep_pair_kernel, dim3(np, p.ya + yr), dim3(256), 0, c->stream, true, in, p, K);
+}
+
 template <class Epi>
 cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
                          int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,

@@ -374,19 +374,19 @@ int offload_before_layer(river_ctx *c, int l, bool *staged) {
 }
 
 // The tensor-core kernels of one projection: `backbone(phase, late_release)` launches tc_gemm_kernel's part,
-// `river(phase, beside)` the dequantising kernel's.  With both, the two operand kernels go first and the two GEMMs
+// `river(phase, beside)` the dequantising kernel's.  With both, one operand kernel serves both lists and the two GEMMs
 // share the device: the first lets the second start once the operands are complete, the second waits for the first
 // before it ends (the kernels' comments say why that is enough); RIVER_F_SERIAL_TC keeps them one after the other.
 template <class Bb, class Rv>
-cudaError_t tc_pair(river_ctx *c, bool with_river, Bb &&backbone, Rv &&river) {
+cudaError_t tc_pair(river_ctx *c, bool with_river, const ProjIn &in, int K, int n, const RowLists &rl, Bb &&backbone,
+                    Rv &&river) {
     if (!with_river) return backbone(kTcBoth, false);
     cudaError_t e;
     if (c->cfg.flags & RIVER_F_SERIAL_TC) {
         if ((e = backbone(kTcBoth, false)) != cudaSuccess) return e;
         return river(kTcBoth, false);
     }
-    if ((e = backbone(kTcPrep, false)) != cudaSuccess) return e;
-    if ((e = river(kTcPrep, false)) != cudaSuccess) return e;
+    if ((e = launch_tc_prep_pair(c, in, K, n, rl.act_idx, rl.n_act, rl.riv_idx, rl.n_riv)) != cudaSuccess) return e;
     if ((e = backbone(kTcGemm, true)) != cudaSuccess) return e;
     return river(kTcGemm, true);
 }
@@ -424,7 +424,7 @@ cudaError_t launch_qkv(river_ctx *c, int l, int n, const float *h_in, const Deci
         const TcQkvEpi e{g.Hq, g.Hkv, g.dh, c->rope_cs, c->qbuf, kv_addr(c, l - 1), c->dev_err};
         const CUtensorMap *const cm[3] = {wm ? &wm->q : nullptr, wm ? &wm->k : nullptr, wm ? &wm->v : nullptr};
         const river_w4 *const cw[3] = {&w.rq, &w.rk, &w.rv};
-        note(tc_pair(c, wm != nullptr,
+        note(tc_pair(c, wm != nullptr, in, d, n, rl,
                      [&](int phase, bool late) {
                          return launch_tc(c, in, tm->q, tm->k, tm->v, d, (qdim + 2 * kvdim) / kTcBM, n, 0, qdim / kTcBM,
                                           kvdim / kTcBM, ai, na, e, true, c->hint_act, phase, late);
@@ -557,7 +557,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
                 const TcResidEpi e{h_in, h_mid, d};
                 const CUtensorMap *const cm[3] = {wm ? &wm->o : nullptr, wm ? &wm->o : nullptr, wm ? &wm->o : nullptr};
                 const river_w4 *const cw[3] = {&w.ro, &w.ro, &w.ro};
-                note(tc_pair(c, wm != nullptr,
+                note(tc_pair(c, wm != nullptr, in, qdim, n, rl,
                              [&](int phase, bool late) {
                                  return launch_tc(c, in, tm->o, tm->o, tm->o, qdim, d / kTcBM, n, 0, 0, 0, ai, na, e, true,
                                                   c->hint_act, phase, late);
@@ -581,7 +581,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
                 const TcGateUpEpi e{c->act, g.F};
                 const CUtensorMap *const cm[3] = {wm ? &wm->g : nullptr, wm ? &wm->u : nullptr, wm ? &wm->u : nullptr};
                 const river_w4 *const cw[3] = {&w.rg, &w.ru, &w.ru};
-                note(tc_pair(c, wm != nullptr,
+                note(tc_pair(c, wm != nullptr, in, d, n, rl,
                              [&](int phase, bool late) {
                                  return launch_tc(c, in, tm->g, tm->u, tm->u, d, g.F / 64, n, 1, 0, 0, ai, na, e, true,
                                                   c->hint_act, phase, late);
@@ -604,7 +604,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
                 const TcResidEpi e{h_mid, h_out, d};
                 const CUtensorMap *const cm[3] = {wm ? &wm->d : nullptr, wm ? &wm->d : nullptr, wm ? &wm->d : nullptr};
                 const river_w4 *const cw[3] = {&w.rd, &w.rd, &w.rd};
-                note(tc_pair(c, wm != nullptr,
+                note(tc_pair(c, wm != nullptr, in, g.F, n, rl,
                              [&](int phase, bool late) {
                                  return launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e, true,
                                                   c->hint_act, phase, late);
