@@ -36,6 +36,7 @@ struct AttnArgs {
     const StepMeta *meta;
     const float *q;        // [rows][Hq*DH]
     const int32_t *page_tbl, *row_slot, *row_pos;
+    const int32_t *order;  // grid z -> row (longest context first), a permutation of the step's rows
     int n_pages, max_pages_per_seq, Hkv, Hq, layer0;
     float qscale;          // log2(e) / sqrt(DH)
     float *part_o;         // [(row*Hq + head)*splits + split][DH]  unnormalised
@@ -61,7 +62,7 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
     constexpr int NCH = DH / 32;                 // 16-byte chunks per lane quarter in q.K
     constexpr int VE = DH / 32;                  // head dims per lane in P.V
 
-    const int split = blockIdx.x, kvh = blockIdx.y, row = blockIdx.z;
+    const int split = blockIdx.x, kvh = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     pdl_launch();
 
@@ -87,43 +88,47 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
     pdl_wait();
     // independent loads first, decisions after (every index below is valid for any row of the grid)
     const int n_rows = a.meta->n_rows, chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
+    const int row = a.order[blockIdx.z];  // (entries past the step's rows hold 0 or an earlier step's row id)
     const int pos = a.row_pos[row], slot = a.row_slot[row];
-    if (row >= n_rows || (a.skip && a.skip[row])) return;
+    if ((int)blockIdx.z >= n_rows || (a.skip && a.skip[row])) return;
     const int p0 = split * chunk;
     if (p0 > pos) return;
     const int p1 = min(p0 + chunk, pos + 1);     // positions [p0, p1)
     const int n_tiles = (p1 - p0 + kAttnTile - 1) / kAttnTile;
     volatile int *abortp = &s_abort;
 
-    // one lane issues the TMA copies, at most kAttnStages tiles ahead; the first tiles go out before anything else
+    // The producer WARP issues the TMA copies of a tile, at most kAttnStages tiles ahead - one copy per lane (a tile is
+    // 2 NB copies per page: a single lane, retiring an instruction every few tens of cycles, would take about as long
+    // to issue them as the tile takes to arrive); the first tiles go out before anything else.  Called by all lanes.
+    static_assert(kAttnConsumers * 2 * NB <= 32, "one copy per producer lane");
     auto issue_tile = [&](int t) {
-        const int32_t *pt = a.page_tbl + (size_t)slot * a.max_pages_per_seq;
         const int s = t % kAttnStages;
-        if (t >= kAttnStages &&
-            !mbar_wait(smem_u32(&bars[kAttnStages + s]), ((t / kAttnStages) - 1) & 1, abortp, a.dev_err))
-            return false;
+        if (t >= kAttnStages) {
+            int ok = 1;
+            if (lane == 0)
+                ok = mbar_wait(smem_u32(&bars[kAttnStages + s]), ((t / kAttnStages) - 1) & 1, abortp, a.dev_err) ? 1 : 0;
+            if (!__shfl_sync(0xffffffffu, ok, 0)) return false;
+        }
         const int first_page = (p0 + t * kAttnTile) / kPage;
         const int n_valid = min(kAttnConsumers, (p1 - 1) / kPage - first_page + 1);
         const uint32_t full = smem_u32(&bars[s]);
-        mbar_expect_tx(full, (uint32_t)(n_valid * 2 * PAGE_BYTES));
-        for (int j = 0; j < n_valid; ++j) {
-            int page = pt[first_page + j];
+        if (lane == 0) mbar_expect_tx(full, (uint32_t)(n_valid * 2 * PAGE_BYTES));
+        __syncwarp();
+        if (lane < n_valid * 2 * NB) {
+            const int j = lane / (2 * NB), kv = (lane / NB) & 1, b = lane % NB;  // page of the tile, K or V, 128-byte box
+            int page = a.page_tbl[(size_t)slot * a.max_pages_per_seq + first_page + j];
             if (page < 0 || page >= a.n_pages) { atomicExch(a.dev_err, DEV_BAD_PAGE); page = 0; }
             // cache rows of (layer, page, K|V, kv head): 16 consecutive rows of the [rows][DH] view
-            const int yk = ((((a.layer0 * a.n_pages + page) * 2 + 0) * a.Hkv) + kvh) * kPage;
-            const int yv = ((((a.layer0 * a.n_pages + page) * 2 + 1) * a.Hkv) + kvh) * kPage;
-            const uint32_t dk = smem_u32(stages + s * STAGE_BYTES + j * PAGE_BYTES);
-            const uint32_t dv = dk + kAttnConsumers * PAGE_BYTES;
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                tma_load_2d(dk + b * (kPage * 128), &tmap, b * 64, yk, full);
-                tma_load_2d(dv + b * (kPage * 128), &tmap, b * 64, yv, full);
-            }
+            const int y = ((((a.layer0 * a.n_pages + page) * 2 + kv) * a.Hkv) + kvh) * kPage;
+            const uint32_t dst = smem_u32(stages + s * STAGE_BYTES + (kv * kAttnConsumers + j) * PAGE_BYTES) + b * (kPage * 128);
+            tma_load_2d(dst, &tmap, b * 64, y, full);
         }
         return true;
     };
-    if (is_producer)
+    if (warp == NW) {
+        __syncwarp();  // the barriers lane 0 initialised
         for (int t = 0; t < min(n_tiles, kAttnStages); ++t) issue_tile(t);
+    }
     if constexpr (!MMA) {
         for (int i = tid; i < GQ * DH; i += kAttnThreads)
             sq[i] = a.q[(size_t)row * a.Hq * DH + (size_t)kvh * GQ * DH + i] * a.qscale;
@@ -157,9 +162,8 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
         if (warp == NW) {
-            if (lane == 0)
-                for (int t = kAttnStages; t < n_tiles; ++t)
-                    if (!issue_tile(t)) break;
+            for (int t = kAttnStages; t < n_tiles; ++t)
+                if (!issue_tile(t)) break;
         } else {
             // ldmatrix row of this lane: matrix lane / 8 -> positions 8 (lane / 16) .., 16-byte chunk parity (lane / 8) & 1
             const int lpos = (lane & 7) + 8 * (lane >> 4), lodd = (lane >> 3) & 1;
@@ -292,9 +296,8 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
             for (int e = 0; e < VE; ++e) acc[g][e] = 0.f;
         }
         if (warp == NW) {
-            if (lane == 0)
-                for (int t = kAttnStages; t < n_tiles; ++t)
-                    if (!issue_tile(t)) break;
+            for (int t = kAttnStages; t < n_tiles; ++t)
+                if (!issue_tile(t)) break;
         } else {
             float *my_sp = sp + warp * HP * GQ;
             for (int t = 0; t < n_tiles; ++t) {

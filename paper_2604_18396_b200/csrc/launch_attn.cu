@@ -17,6 +17,7 @@ cudaError_t launch_attn_split(river_ctx *c, int n, int layer0) {
     const river_config &g = c->cfg;
     AttnArgs a{};
     a.meta = c->meta(); a.q = c->qbuf; a.page_tbl = c->page_tbl_dev; a.row_slot = c->row_slot(); a.row_pos = c->row_pos();
+    a.order = c->attn_order();
     a.n_pages = g.n_pages; a.max_pages_per_seq = g.max_pages_per_seq; a.Hkv = g.Hkv; a.Hq = g.Hq; a.layer0 = layer0;
     a.qscale = 1.4426950408889634f / std::sqrt((float)DH);
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.tickets = c->attn_tickets; a.out = c->obuf; a.dev_err = c->dev_err;

@@ -107,7 +107,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     int32_t *na = cv.take<int32_t>(L + 1), *nr = cv.take<int32_t>(L + 1);
     int32_t *pt = cv.take<int32_t>((size_t)c->max_seqs * c->max_pages_per_seq);
     int32_t *tk = cv.take<int32_t>(B), *fo = cv.take<int32_t>(B), *ex = cv.take<int32_t>(B), *nx = cv.take<int32_t>(B);
-    int32_t *md = cv.take<int32_t>(kMetaHdr + 10 * B);
+    int32_t *md = cv.take<int32_t>(kMetaHdr + 11 * B);
     int32_t *pff = cv.take<int32_t>((size_t)c->max_seqs * (L + 1));
     float *po = cv.take<float>((B + 600) * (size_t)c->Hq * c->dh);
     float2 *pml = cv.take<float2>((B + 600) * (size_t)c->Hq);
@@ -180,6 +180,13 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     mh[3] = chunk;
     mh[4] = S;
     mh[5] = n;  // hint_act: every row starts in the backbone
+    // the attention grid takes its rows longest context first: CTA slots are handed out in launch order, and a long
+    // item that starts last is what the step ends on
+    int32_t *order = mh + kMetaHdr + 10 * g.max_batch;
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order, order + n, [&](int32_t x, int32_t y) {
+        return mh[kMetaHdr + g.max_batch + x] > mh[kMetaHdr + g.max_batch + y];
+    });
     // the small-step kernel: one CTA per (row, kv head, split), chunks in whole pages
     const int Sc = small_attn_splits(c->num_sms, n, g.Hkv);
     int cchunk = (max_pos + 1 + Sc - 1) / Sc;
@@ -857,6 +864,7 @@ int river_init(const river_config *cfg, const river_weights *w, void *kv_pool, s
     c->w4tc_ok = c->tc_ok && !(cfg->flags & RIVER_F_NO_W4TC) && make_w4_maps(c);
     for (int i = 0; i < kStaging; ++i) {
         if (cudaMallocHost((void **)&c->meta_host[i], sizeof(int32_t) * c->meta_ints()) != cudaSuccess) return bail("cudaMallocHost failed");
+        std::memset(c->meta_host[i], 0, sizeof(int32_t) * c->meta_ints());  // entries past a step's rows stay valid row ids
         if (cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail("cudaEventCreate failed");
     }
     c->pin_io_bytes = (size_t)cfg->max_batch * (4 * sizeof(int32_t) + sizeof(float)) + sizeof(int32_t);

@@ -59,8 +59,8 @@ struct river_ctx {
     std::vector<GraphEntry> graphs;
     double *inv_freq;
     int32_t *act_idx, *riv_idx, *n_act, *n_riv, *page_tbl_dev, *part_idx, *tok_i, *forced_i, *exit_i, *next_i;
-    int32_t *meta_dev;  // [kMetaHdr + 10*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows, row_page, row_forced,
-                        // tile_row0, tile_rows (query tiles of a prefill chunk)
+    int32_t *meta_dev;  // [kMetaHdr + 11*max_batch]: StepMeta, row_slot, row_pos, upd[3], head_rows, row_page, row_forced,
+                        // tile_row0, tile_rows (query tiles of a prefill chunk), attn_order
     int32_t *prefill_fail;  // [max_seqs][L+1]: 1 where some prompt position of the sequence failed Eq. 1 after block l
     uint8_t *state;     // [(L+1)][state_stride]: sticky exit flags of the rows entering block l + 1 (entry L: at the LM head)
     int state_stride = 0;
@@ -104,7 +104,7 @@ struct river_ctx {
     double prof_ms[kNumClasses] = {0}, prof_bytes[kNumClasses] = {0};
     int64_t prof_launches[kNumClasses] = {0};
 
-    int meta_ints() const { return river::kMetaHdr + 10 * cfg.max_batch; }
+    int meta_ints() const { return river::kMetaHdr + 11 * cfg.max_batch; }
     river::StepMeta *meta() const { return reinterpret_cast<river::StepMeta *>(meta_dev); }
     int32_t *row_slot() const { return meta_dev + river::kMetaHdr; }
     int32_t *row_pos() const { return meta_dev + river::kMetaHdr + cfg.max_batch; }
@@ -114,6 +114,7 @@ struct river_ctx {
     int32_t *row_forced() const { return meta_dev + river::kMetaHdr + 7 * cfg.max_batch; }  // prefill: forced exit per row
     int32_t *tile_row0() const { return meta_dev + river::kMetaHdr + 8 * cfg.max_batch; }
     int32_t *tile_rows() const { return meta_dev + river::kMetaHdr + 9 * cfg.max_batch; }
+    int32_t *attn_order() const { return meta_dev + river::kMetaHdr + 10 * cfg.max_batch; }  // rows, longest context first
     uint8_t *state_at(int l) const { return state + (size_t)l * state_stride; }
 };
 
