@@ -140,10 +140,11 @@ def test_small_steps_every_row_count(rows):
     assert r["n_early"] > 0
 
 
-@pytest.mark.parametrize("flags", [0, 16, 2])
+@pytest.mark.parametrize("flags", [0, 16, 2, 64, 1, 65])
 def test_mini8_head_dim_128_gqa4(flags):
-    # five rows: backbone rows on the tcgen05 GEMM; exit-layer rows on the dequantising tcgen05 GEMM (0), on the
-    # CUDA-core kernel (16), everything on CUDA cores (2)
+    # five rows: backbone rows on the tcgen05 GEMM; exit-layer rows on the dequantising tcgen05 GEMM - beside it (0)
+    # or behind it (64) -, on the CUDA-core kernel (16), everything on CUDA cores (2); 1, 65: the same two orders
+    # replayed from a CUDA graph
     r = run_scheduled(model("mini8"), [70, 16, 31, 48, 5], 18, "uniform", prefill_exit=3, page_seed=7, flags=flags)
     assert r["n_early"] > 0
     print(r)
