@@ -150,10 +150,12 @@ def test_mini8_head_dim_128_gqa4(flags):
     print(r)
 
 
-@pytest.mark.parametrize("rows", [70, 150])
+@pytest.mark.parametrize("rows", [70, 120, 150])
 def test_mini8_wide_batches_other_gemm_geometries(rows):
-    # 70 rows: operand tiles of 80 rows, three CTAs per SM; 150 rows: 160-row operand tiles, one CTA per SM with deep
-    # stages; both weight sets live in most layers, lengths mixed so that the attention splits differ per row.  The
+    # 70 rows: operand tiles of 80 rows, three CTAs per SM; 120 rows: 128-row tiles, hi and lo still one TMA box but two
+    # MMAs per k-step in the dequantising kernel (its tensor-memory ring leaves no room for a 256-column accumulator
+    # twice per SM); 150 rows: 160-row operand tiles, one CTA per SM with deep stages, separate hi / lo boxes; both
+    # weight sets live in most layers, lengths mixed so that the attention splits differ per row.  The
     # oracle stores its cache in bf16 here as the large-shape tests do: over millions of cache entries the tail of the
     # fp32-cache deviation (Section 4.1's shared slots hold bf16) reaches the K/V tolerance without any kernel error.
     r = run_scheduled(model("mini8"), [3 + (11 * b) % 29 for b in range(rows)], 3, "uniform", page_seed=rows, max_batch=rows,
