@@ -137,13 +137,16 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     return (cv.off + 255) & ~(size_t)255;
 }
 
-// KV split geometry of this step.  A (row, kv head, split) item costs its positions plus a fixed start-up overhead
-// worth about two 64-position tiles, and splitting at all adds the merge through global memory (about five tiles'
-// time, once); items are handed to the CTA slots in launch order, so a step lasts about (all positions / slots) +
-// half of the longest item + the overheads a slot pays (constants fitted to measurements at 64 rows with equal and
-// with mixed lengths).  The split count that minimises this estimate is taken from a short list: one split when the rows are equally long and outnumber the slots
-// (splitting only adds overhead), several when the lengths are mixed, and at least enough to give every slot an item.  Splits are whole tiles,
-// at least two.  The split count is part of a captured launch's key; the chunk length lives in the step metadata.
+// KV split geometry of this step.  A (row, kv head, split) item costs its positions plus a fixed start and end worth
+// about four 64-position tiles, and splitting at all adds the merge through global memory (about five tiles' time,
+// once); items are handed to the CTA slots in launch order, rows longest first.  One wave of items lasts as long as its
+// longest item; more waves last about (all positions / slots) + a quarter of the longest item (what a slot still
+// holds when the others run dry), and with rows of equal length no less than whole waves of the mean item; every slot
+// pays the fixed part once per item (constants fitted to measurements at 16, 64 and 128 rows with equal and with mixed
+// lengths).  The split count that minimises this estimate is taken from a short list - one split when the rows are
+// equally long and outnumber the slots, a few when the lengths are mixed, and with few rows enough to fill three
+// quarters of the slots.  Splits are whole tiles, at least two.  The split count is part of a captured launch's key;
+// the chunk length lives in the step metadata.
 void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
     const river_config &g = c->cfg;
     int max_pos = 0;
@@ -154,13 +157,15 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
         total += pos + 1;
     }
     // three CTAs of the attention kernel fit per SM (registers; shared memory at head dim 128)
-    const double slots = 3.0 * c->num_sms, ovh = 120.0 * 128.0 / g.dh, merge = 350.0 * 128.0 / g.dh;
+    const double slots = 3.0 * c->num_sms, ovh = 250.0 * 128.0 / g.dh, merge = 350.0 * 128.0 / g.dh;
+    const bool uniform = (max_pos + 1) <= 1.3 * total / n;  // whole waves of equal items bound the time only then
     const int s_cap = std::max(1, std::min(64, (g.max_batch + 600) / n));  // the partials hold max_batch + 600 (row, split) slots
     static const int cand[] = {1, 2, 3, 4, 5, 6, 8, 12, 16, 24, 32, 48, 64};
     int S = 1, chunk = 0;
     double best = 0.0;
-    // fewer items than slots: at least fill the slots
-    const int s_lo = std::min(s_cap, (int)((slots + n * g.Hkv - 1) / (n * g.Hkv)));
+    // fewer items than slots: at least fill three quarters of them (three CTAs share an SM: one wave that leaves some
+    // slots empty beats a second, nearly empty wave)
+    const int s_lo = std::max(1, std::min(s_cap, (int)std::ceil(0.75 * slots / (n * g.Hkv))));
     for (int k = -1; k < (int)(sizeof(cand) / sizeof(cand[0])); ++k) {
         const int s = k < 0 ? s_lo : cand[k];
         if (k >= 0 && (s <= s_lo || s > s_cap)) continue;
@@ -172,8 +177,12 @@ void set_attn_meta(river_ctx *c, int32_t *mh, int n) {
         const int longest = std::min(ch, max_pos + 1);
         // whole waves of items of the mean length bound it from below as well (equal lengths: 1.3 waves cost 2)
         const double waves = std::ceil(items / slots), mean_item = total * g.Hkv / items;
-        const double t = std::max(std::max(total * g.Hkv / slots + 0.5 * longest, waves * mean_item), (double)longest) +
-                         ovh * std::max(1.0, items / slots) + (s > 1 ? merge : 0.0);
+        // one wave: the longest item; more: the slots' mean load plus a tail (the rows enter longest first, so what a
+        // slot still holds at the end is a fraction of an item)
+        const double body = items <= slots ? (double)longest
+                                           : std::max(std::max(total * g.Hkv / slots + 0.25 * longest, uniform ? waves * mean_item : 0.0),
+                                                      (double)longest);
+        const double t = body + ovh * std::max(1.0, items / slots) + (s > 1 ? merge : 0.0);
         if (chunk == 0 || t < best * 0.97) { best = t; S = s; chunk = ch; }
         if (ch == 2 * kAttnTile) break;  // finer splits do not exist
     }
