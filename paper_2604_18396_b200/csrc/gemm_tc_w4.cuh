@@ -183,10 +183,10 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
     uint8_t *stages = smem;
     uint8_t *raw = stages + (size_t)S * stage_bytes;                 // kW4RawBufs raw code tiles, 1024-aligned
     float *tile = reinterpret_cast<float *>(stages);                 // the finished tile reuses stages + raw
-    // barriers: a_full[S], b_full[S], empty[S], raw_full[R], raw_empty[R], acc
+    // barriers: full[S] (A tile written and activation tile landed), empty[S], raw_full[R], raw_empty[R], acc
     uint64_t *bars = reinterpret_cast<uint64_t *>(raw + (size_t)kW4RawBufs * kW4RawBytes);
-    uint64_t *b_afull = bars, *b_bfull = bars + S, *b_empty = bars + 2 * S, *b_rfull = bars + 3 * S,
-             *b_rempty = bars + 3 * S + kW4RawBufs, *b_acc = bars + 3 * S + 2 * kW4RawBufs;
+    uint64_t *b_afull = bars, *b_empty = bars + S, *b_rfull = bars + 2 * S, *b_rempty = bars + 2 * S + kW4RawBufs,
+             *b_acc = bars + 2 * S + 2 * kW4RawBufs;
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort, s_early;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -204,8 +204,9 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
         s_abort = 0;
         s_early = *reinterpret_cast<const volatile int32_t *>(a.hint) > 0;  // one read for the whole CTA
         for (int s = 0; s < S; ++s) {
-            mbar_init(smem_u32(&b_afull[s]), 4);  // one arrival per lane quarter
-            mbar_init(smem_u32(&b_bfull[s]), 1);
+            // a stage is full when its A tile is written (one arrival per lane quarter) AND its activation tile has
+            // landed (the producer's arrival with the byte count): ONE barrier, one poll per k-block for the MMA lane
+            mbar_init(smem_u32(&b_afull[s]), 4 + 1);
             mbar_init(smem_u32(&b_empty[s]), 1);
         }
         for (int r = 0; r < kW4RawBufs; ++r) {
@@ -276,7 +277,7 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
             }
             // stage, parity and addresses advance incrementally (a single lane retires an instruction every few
             // cycles: divisions by the runtime stage count cost more here than the copies they address)
-            const uint32_t bfull0 = smem_u32(b_bfull), empty0 = smem_u32(b_empty), rempty0 = smem_u32(b_rempty);
+            const uint32_t bfull0 = smem_u32(b_afull), empty0 = smem_u32(b_empty), rempty0 = smem_u32(b_rempty);
             const uint32_t stage0 = smem_u32(stages);
             uint32_t s = 0, epar = 1, dst = stage0;  // epar: parity of `empty` to wait for from the second round on
             int x = kb0 * kTcBK;
@@ -308,11 +309,10 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
             const uint32_t idesc = tc_idesc_f16(acc_n);
             const uint64_t dfix = tc_smem_desc(0);  // everything but the address field
             const uint32_t stage16 = stage_bytes >> 4, b16 = b_bytes >> 4;
-            const uint32_t afull0 = smem_u32(b_afull), bfull0 = smem_u32(b_bfull), empty0 = smem_u32(b_empty);
+            const uint32_t afull0 = smem_u32(b_afull), empty0 = smem_u32(b_empty);
             const uint32_t ta0 = tmem_d + (uint32_t)acc_n;
             uint32_t s = 0, par = 0, addr16 = smem_u32(stages) >> 4, ta = ta0;  // incremental: no division per k-block
             for (int i = 0; i < nkb_run; ++i) {
-                if (!mbar_wait(bfull0 + 8 * s, par, abortp, a.dev_err)) break;
                 if (!mbar_wait(afull0 + 8 * s, par, abortp, a.dev_err)) break;
                 tc_fence_after();
                 const uint64_t dhi = dfix | addr16, dlo = dhi + b16;  // (addresses below 256 KB: no carry)
@@ -400,7 +400,7 @@ __global__ void __launch_bounds__(kW4Threads, 2) tc_gemm_w4_kernel(const __grid_
 inline size_t tc_w4_smem_bytes(int n_pad, int n_stages) {
     const size_t stage = 2 * (size_t)n_pad * kTcBK * 2;
     return 1024 + (size_t)n_stages * stage + (size_t)kW4RawBufs * kW4RawBytes +
-           sizeof(uint64_t) * (3 * n_stages + 2 * kW4RawBufs + 1) + 64;
+           sizeof(uint64_t) * (2 * n_stages + 2 * kW4RawBufs + 1) + 64;
 }
 
 }  // namespace river
