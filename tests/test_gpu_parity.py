@@ -163,6 +163,17 @@ def test_mini8_wide_batches_other_gemm_geometries(rows):
     assert r["n_early"] > 0
 
 
+@pytest.mark.parametrize("rows", [5, 9, 17, 33, 48, 65, 97, 129, 200, 256])
+def test_mini8_row_count_sweep_on_the_tensor_core_kernels(rows):
+    # every operand-tile height of the two tcgen05 kernels from 16 to 256 rows (one or two accumulators, hi and lo rows
+    # in one TMA box or two, two to four stages, one to three CTAs per SM, with and without K-split clusters), the two
+    # GEMMs of a projection side by side, geometric exit layers so that both weight sets are live from the second
+    # block on; bf16 cache in the oracle as in the other wide-batch tests
+    r = run_scheduled(model("mini8"), [2 + (13 * b + rows) % 41 for b in range(rows)], 2, "geometric", page_seed=100 + rows,
+                      max_batch=rows, kv_store=1)
+    assert r["n_early"] > 0
+
+
 @pytest.mark.parametrize("lens,flags", [([2200, 130, 700, 1, 1500, 300], 0), ([2500, 40], 32), ([1900], 0)])
 def test_mini8_long_ragged_contexts_split_kv(lens, flags):
     # contexts of hundreds to thousands of positions, mixed in one batch: the KV range of a (row, KV head) is cut into
