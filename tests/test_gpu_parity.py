@@ -163,7 +163,7 @@ def test_mini8_wide_batches_other_gemm_geometries(rows):
     assert r["n_early"] > 0
 
 
-@pytest.mark.parametrize("rows", [5, 9, 17, 33, 48, 65, 97, 129, 200, 256])
+@pytest.mark.parametrize("rows", [5, 9, 17, 33, 48, 65, 90, 97, 129, 170, 185, 200, 220, 235, 256])
 def test_mini8_row_count_sweep_on_the_tensor_core_kernels(rows):
     # every operand-tile height of the two tcgen05 kernels from 16 to 256 rows (one or two accumulators, hi and lo rows
     # in one TMA box or two, two to four stages, one to three CTAs per SM, with and without K-split clusters), the two
