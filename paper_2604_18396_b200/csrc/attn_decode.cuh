@@ -47,6 +47,8 @@ struct AttnArgs {
     const uint8_t *skip;   // rows whose flag is set do not attend (they have left and run nothing here), or null
     const uint8_t *pos_depth;  // KV Mask: [slot][depth_stride] backbone blocks the token at each position ran, or null
     int depth_stride, layer1;  // ... a position is visible in block layer1 if that number is >= layer1 (or it is the row's own)
+    int early;             // 1: every row is a different sequence (a decode step): the kernel still in flight writes nothing
+                           // but each row's newest position, so tiles that end before it are requested BEFORE the wait
 };
 
 template <int DH, int GQ, bool MMA>
@@ -85,7 +87,8 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    pdl_wait();
+    if (!a.early) pdl_wait();
+    // (the step metadata and the page table are the host's: complete before the step's first kernel)
     // independent loads first, decisions after (every index below is valid for any row of the grid)
     const int n_rows = a.meta->n_rows, chunk = a.meta->attn_chunk, n_splits = a.meta->attn_splits;
     const int row = a.order[blockIdx.z];  // (entries past the step's rows hold 0 or an earlier step's row id)
@@ -127,7 +130,14 @@ __global__ void __launch_bounds__(attn_threads(MMA)) attn_split_kernel(const __g
     };
     if (warp == NW) {
         __syncwarp();  // the barriers lane 0 initialised
-        for (int t = 0; t < min(n_tiles, kAttnStages); ++t) issue_tile(t);
+        for (int t = 0; t < min(n_tiles, kAttnStages); ++t)
+            if (!a.early || p0 + (t + 1) * kAttnTile <= pos) issue_tile(t);  // (early: only tiles the row's new position is not in)
+    }
+    if (a.early) {
+        pdl_wait();
+        if (warp == NW)
+            for (int t = 0; t < min(n_tiles, kAttnStages); ++t)
+                if (p0 + (t + 1) * kAttnTile > pos) issue_tile(t);
     }
     if constexpr (!MMA) {
         for (int i = tid; i < GQ * DH; i += kAttnThreads)

@@ -23,6 +23,7 @@ cudaError_t launch_attn_split(river_ctx *c, int n, int layer0) {
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.tickets = c->attn_tickets; a.out = c->obuf; a.dev_err = c->dev_err;
     a.skip = c->attn_skip;
     a.pos_depth = c->attn_layer1 ? c->pos_depth : nullptr; a.depth_stride = g.max_pages_per_seq * kPage; a.layer1 = c->attn_layer1;
+    a.early = (c->rows_distinct && !a.skip) ? 1 : 0;  // (the exit flags of a skipping strategy belong to this block: wait first)
     const size_t smem = attn_smem_bytes(DH, GQ);
     constexpr bool MMA = GQ <= 4;  // groups of up to four query heads: contractions on the warp-level tensor cores
     const cudaError_t e = ensure_smem(c, attn_split_kernel<DH, GQ, MMA>, smem);
