@@ -14,6 +14,7 @@
 // write, residual add, SwiGLU, logits + argmax partials).
 // Weights do not depend on the previous kernel: their first tiles are requested before the grid dependency resolves.
 #pragma once
+#include <cuda_fp16.h>
 #include "mbar_tma.cuh"
 
 namespace river {
@@ -171,6 +172,11 @@ struct TcResidEpi {  // out[row][row0 + r] = resid[row][row0 + r] + tile(r, n)
 struct TcGateUpEpi {  // tile rows 0..63: gate features f0.., rows 64..127: up features f0..
     float *act;
     int F;
+    // optional: the down projection's operand rows, so that it needs no operand kernel: row n of the list, split
+    // v = hi + lo exactly as tc_prep_kernel (omode 1: bf16) or tc_prep_w4_kernel (omode 2: f16, the inputs of every
+    // group of eight in the order (0,4,1,5,2,6,3,7)) would split act[rows[n]]
+    uint16_t *ohi = nullptr, *olo = nullptr;
+    int omode = 0;
     __device__ int quad_row(int i, int q0, int nq) const { return i < nq ? 4 * (q0 + i) : 64 + 4 * (q0 + i - nq); }
     __device__ void run(const float *tile, int ld, int tile_idx, int n_live, const int32_t *rows, int tid, int nthr,
                         int pr0, int pr1, int = 0) const {
@@ -178,7 +184,20 @@ struct TcGateUpEpi {  // tile rows 0..63: gate features f0.., rows 64..127: up f
         for (int t = tid; t < n_live * np; t += nthr) {
             const int n = t / np, r = pr0 + t % np;
             const float g = tile[n * ld + r], u = tile[n * ld + 64 + r];
-            act[(size_t)rows[n] * F + f0 + r] = g / (1.f + __expf(-g)) * u;
+            const float v = g / (1.f + __expf(-g)) * u;
+            act[(size_t)rows[n] * F + f0 + r] = v;
+            if (omode == 1) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                const size_t o = (size_t)n * F + f0 + r;
+                ohi[o] = __bfloat16_as_ushort(h);
+                olo[o] = __bfloat16_as_ushort(__float2bfloat16_rn(v - __bfloat162float(h)));
+            } else if (omode == 2) {
+                const __half h = __float2half_rn(v);
+                const int f = f0 + r, j = f & 7;
+                const size_t o = (size_t)n * F + (f & ~7) + (j < 4 ? 2 * j : 2 * (j - 4) + 1);
+                ohi[o] = __half_as_ushort(h);
+                olo[o] = __half_as_ushort(__float2half_rn(v - __half2float(h)));
+            }
         }
     }
 };

@@ -6,11 +6,12 @@
 
 namespace river {
 
-const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np, bool w4) {
+const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np, bool w4, bool alt) {
     for (auto &b : c->tc_bmaps)
-        if (b.K == K && b.np == np && b.w4 == w4) return &b;
-    river_ctx::BMap b{K, np, w4, 2 * np <= 256, nullptr, {}, {}};
-    __nv_bfloat16 *base = w4 ? c->tc_x4 : c->tc_xhi;
+        if (b.K == K && b.np == np && b.w4 == w4 && b.alt == alt) return &b;
+    river_ctx::BMap b{K, np, w4, alt, 2 * np <= 256, nullptr, nullptr, {}, {}};
+    __nv_bfloat16 *base = alt ? (w4 ? c->tc_x4alt : c->tc_xalt) : (w4 ? c->tc_x4 : c->tc_xhi);
+    b.base = base;
     b.lo_ptr = b.one ? base + (size_t)np * K : base + (size_t)c->tc_max_pad * c->tc_kmax;
     const int hi_rows = b.one ? 2 * np : np;  // a box holds at most 256 rows
     if (!make_map_bf16(&b.hi, base, K, hi_rows, hi_rows) || !make_map_bf16(&b.lo, b.lo_ptr, K, np, np)) return nullptr;
@@ -74,9 +75,10 @@ template <class Epi>
 cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
                       int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
                       const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint, int phase,
-                      bool late_release) {
+                      bool late_release, bool alt_operand) {
     const int np = (n + 15) / 16 * 16;
-    const river_ctx::BMap *bm = tc_bmap(c, K, np);
+    const river_ctx::BMap *bm = tc_bmap(c, K, np, false, alt_operand);
+    if (alt_operand) phase &= ~kTcPrep;  // the operand rows are there already (the previous projection's epilogues)
     if (!bm) return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
     if (phase & kTcPrep) {
@@ -115,7 +117,7 @@ cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, con
 #define RIVER_TC_INST(E) \
     template cudaError_t launch_tc<E>(river_ctx *, const ProjIn &, const CUtensorMap &, const CUtensorMap &, const CUtensorMap &, \
                                       int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *, \
-                                      int, bool);
+                                      int, bool, bool);
 RIVER_TC_INST(TcQkvEpi) RIVER_TC_INST(TcResidEpi) RIVER_TC_INST(TcGateUpEpi) RIVER_TC_INST(TcHeadEpi)
 #undef RIVER_TC_INST
 

@@ -5,7 +5,7 @@
 
 namespace river {
 
-const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np, bool w4 = false);
+const river_ctx::BMap *tc_bmap(river_ctx *c, int K, int np, bool w4 = false, bool alt = false);
 
 // Both kernels of a projection (backbone rows, exit-layer rows) are in flight together: `phase` says which part of a
 // launch function runs - the operand kernel, the GEMM, or both in a row.
@@ -21,11 +21,11 @@ template <class Epi>
 cudaError_t launch_tc(river_ctx *c, const ProjIn &in, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
                       int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
                       const int32_t *cnt, const Epi &epi, bool allow_split, const int32_t *hint, int phase = kTcBoth,
-                      bool late_release = false);
+                      bool late_release = false, bool alt_operand = false);
 #define RIVER_TC_DECL(E) \
     extern template cudaError_t launch_tc<E>(river_ctx *, const ProjIn &, const CUtensorMap &, const CUtensorMap &, const CUtensorMap &, \
                                              int, int, int, int, int, int, const int32_t *, const int32_t *, const E &, bool, const int32_t *, \
-                                             int, bool);
+                                             int, bool, bool);
 RIVER_TC_DECL(TcQkvEpi) RIVER_TC_DECL(TcResidEpi) RIVER_TC_DECL(TcGateUpEpi) RIVER_TC_DECL(TcHeadEpi)
 #undef RIVER_TC_DECL
 
@@ -38,11 +38,12 @@ cudaError_t launch_tc_prep_pair(river_ctx *c, const ProjIn &in, int K, int n, co
 template <class Epi>
 cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
                          int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                         const int32_t *cnt, const int32_t *hint, const Epi &epi, int phase = kTcBoth, bool overlap = false);
+                         const int32_t *cnt, const int32_t *hint, const Epi &epi, int phase = kTcBoth, bool overlap = false,
+                         bool alt_operand = false);
 #define RIVER_TCW4_DECL(E) \
     extern template cudaError_t launch_tc_w4<E>(river_ctx *, const ProjIn &, const CUtensorMap *const (&)[3], const river_w4 *const (&)[3], \
                                                 int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &, \
-                                                int, bool);
+                                                int, bool, bool);
 RIVER_TCW4_DECL(TcQkvEpi) RIVER_TCW4_DECL(TcResidEpi) RIVER_TCW4_DECL(TcGateUpEpi)
 #undef RIVER_TCW4_DECL
 

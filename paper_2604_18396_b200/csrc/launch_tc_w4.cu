@@ -24,9 +24,10 @@ cudaError_t launch_tc_prep_pair(river_ctx *c, const ProjIn &in, int K, int n, co
 template <class Epi>
 cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *const (&m)[3], const river_w4 *const (&w)[3],
                          int K, int tiles, int n, int gateup, int q_tiles, int k_tiles, const int32_t *rows,
-                         const int32_t *cnt, const int32_t *hint, const Epi &epi, int phase, bool overlap) {
+                         const int32_t *cnt, const int32_t *hint, const Epi &epi, int phase, bool overlap, bool alt_operand) {
     const int np = (n + 15) / 16 * 16;
-    const river_ctx::BMap *bm = tc_bmap(c, K, np, true);
+    const river_ctx::BMap *bm = tc_bmap(c, K, np, true, alt_operand);
+    if (alt_operand) phase &= ~kTcPrep;  // the operand rows are there already (the previous projection's epilogues)
     if (!bm) return cudaErrorInvalidValue;
     cudaError_t e = cudaSuccess;
     if (phase & kTcPrep) {
@@ -87,7 +88,7 @@ cudaError_t launch_tc_w4(river_ctx *c, const ProjIn &in, const CUtensorMap *cons
 #define RIVER_TCW4_INST(E) \
     template cudaError_t launch_tc_w4<E>(river_ctx *, const ProjIn &, const CUtensorMap *const (&)[3], const river_w4 *const (&)[3], \
                                          int, int, int, int, int, int, const int32_t *, const int32_t *, const int32_t *, const E &, \
-                                         int, bool);
+                                         int, bool, bool);
 RIVER_TCW4_INST(TcQkvEpi) RIVER_TCW4_INST(TcResidEpi) RIVER_TCW4_INST(TcGateUpEpi)
 #undef RIVER_TCW4_INST
 

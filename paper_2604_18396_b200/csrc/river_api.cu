@@ -124,6 +124,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
     // one allocation: lo rows may start right behind the hi rows in use (launch_tc.cu: tc_bmap)
     __nv_bfloat16 *txh = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax), *txl = txh ? txh + tc_pad * tc_kmax : nullptr;
     __nv_bfloat16 *tx4 = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax);
+    __nv_bfloat16 *txa = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax), *tx4a = cv.take<__nv_bfloat16>(2 * tc_pad * tc_kmax);
 
     if (x) {
         x->h[0] = h0; x->h[1] = h1; x->h[2] = h2; x->qbuf = qb; x->obuf = ob; x->act = act;
@@ -132,7 +133,7 @@ size_t carve(const river_config *c, river_ctx *x, char *base, int head_rows) {
         x->tok_i = tk; x->forced_i = fo; x->exit_i = ex; x->next_i = nx; x->meta_dev = md; x->state = exd; x->state_stride = (int)sstride; x->prefill_fail = pff;
         x->pass = ps; x->dev_err = de; x->part_o = po; x->part_ml = pml; x->attn_tickets = atk; x->tickets = tk4; x->hint_act = hint;
         x->slot_cap = scap; x->pos_depth = pdep; x->exit_hist = ehist;
-        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_x4 = tx4; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
+        x->tc_xhi = txh; x->tc_xlo = txl; x->tc_x4 = tx4; x->tc_xalt = txa; x->tc_x4alt = tx4a; x->tc_max_pad = (int)tc_pad; x->tc_kmax = (int)tc_kmax;
     }
     return (cv.off + 255) & ~(size_t)255;
 }
@@ -394,16 +395,20 @@ int offload_before_layer(river_ctx *c, int l, bool *staged) {
 // `river(phase, beside)` the dequantising kernel's.  With both, one operand kernel serves both lists and the two GEMMs
 // share the device: the first lets the second start once the operands are complete, the second waits for the first
 // before it ends (the kernels' comments say why that is enough); RIVER_F_SERIAL_TC keeps them one after the other.
+// `operand_ready`: the operand rows of both lists were written by the previous projection's epilogues: no operand kernel.
 template <class Bb, class Rv>
 cudaError_t tc_pair(river_ctx *c, bool with_river, const ProjIn &in, int K, int n, const RowLists &rl, Bb &&backbone,
-                    Rv &&river) {
-    if (!with_river) return backbone(kTcBoth, false);
+                    Rv &&river, bool operand_ready = false) {
+    const int whole = operand_ready ? kTcGemm : kTcBoth;
+    if (!with_river) return backbone(whole, false);
     cudaError_t e;
     if (c->cfg.flags & RIVER_F_SERIAL_TC) {
-        if ((e = backbone(kTcBoth, false)) != cudaSuccess) return e;
-        return river(kTcBoth, false);
+        if ((e = backbone(whole, false)) != cudaSuccess) return e;
+        return river(whole, false);
     }
-    if ((e = launch_tc_prep_pair(c, in, K, n, rl.act_idx, rl.n_act, rl.riv_idx, rl.n_riv)) != cudaSuccess) return e;
+    if (!operand_ready &&
+        (e = launch_tc_prep_pair(c, in, K, n, rl.act_idx, rl.n_act, rl.riv_idx, rl.n_riv)) != cudaSuccess)
+        return e;
     if ((e = backbone(kTcGemm, true)) != cudaSuccess) return e;
     return river(kTcGemm, true);
 }
@@ -595,7 +600,18 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
             p.K = d; p.F = g.F; p.group = g.group; p.act = c->act;
             const ProjIn in{h_mid, (const uint16_t *)w.ffn_norm, g.rms_eps};
             if (tc) {
-                const TcGateUpEpi e{c->act, g.F};
+                // the epilogues also write the down projection's operand rows (second operand buffers: this
+                // projection's own operand is still being read while they do)
+                const int npad = (n + 15) / 16 * 16;
+                TcGateUpEpi e{c->act, g.F}, e4{c->act, g.F};
+                if (const river_ctx::BMap *bd = tc_bmap(c, g.F, npad, false, true)) {
+                    e.ohi = reinterpret_cast<uint16_t *>(bd->base); e.olo = reinterpret_cast<uint16_t *>(bd->lo_ptr); e.omode = 1;
+                } else note(cudaErrorInvalidValue);
+                if (wm) {
+                    if (const river_ctx::BMap *bd = tc_bmap(c, g.F, npad, true, true)) {
+                        e4.ohi = reinterpret_cast<uint16_t *>(bd->base); e4.olo = reinterpret_cast<uint16_t *>(bd->lo_ptr); e4.omode = 2;
+                    } else note(cudaErrorInvalidValue);
+                }
                 const CUtensorMap *const cm[3] = {wm ? &wm->g : nullptr, wm ? &wm->u : nullptr, wm ? &wm->u : nullptr};
                 const river_w4 *const cw[3] = {&w.rg, &w.ru, &w.ru};
                 note(tc_pair(c, wm != nullptr, in, d, n, rl,
@@ -604,7 +620,7 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
                                                   c->hint_act, phase, late);
                              },
                              [&](int phase, bool beside) {
-                                 return launch_tc_w4(c, in, cm, cw, d, g.F / 64, n, 1, 0, 0, ri, nr, nrh, e, phase, beside);
+                                 return launch_tc_w4(c, in, cm, cw, d, g.F / 64, n, 1, 0, 0, ri, nr, nrh, e4, phase, beside);
                              }));
             }
             if (!wm && (!tc || has_river)) note(launch_stream(c, p, in, rl, d, g.F, n, has_river, true, skip_bb, no_dec));
@@ -624,11 +640,12 @@ int run_rows(river_ctx *c, int n, int n_head, const int32_t *row_pos_host, bool 
                 note(tc_pair(c, wm != nullptr, in, g.F, n, rl,
                              [&](int phase, bool late) {
                                  return launch_tc(c, in, tm->d, tm->d, tm->d, g.F, d / kTcBM, n, 0, 0, 0, ai, na, e, true,
-                                                  c->hint_act, phase, late);
+                                                  c->hint_act, phase, late, true);
                              },
                              [&](int phase, bool beside) {
-                                 return launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e, phase, beside);
-                             }));
+                                 return launch_tc_w4(c, in, cm, cw, g.F, d / kTcBM, n, 0, 0, 0, ri, nr, nrh, e, phase, beside, true);
+                             },
+                             true));  // operand rows: written by the gate/up epilogues
             }
             if (!wm && (!tc || has_river))
                 note(launch_stream(c, p, in, rl, g.F, d / 2, n, has_river, true, skip_bb, no_dec));

@@ -36,6 +36,8 @@ struct river_ctx {
     // tensor-core path: operand buffers, tensor maps of every weight matrix
     __nv_bfloat16 *tc_xhi = nullptr, *tc_xlo = nullptr;
     __nv_bfloat16 *tc_x4 = nullptr;  // the same pair for the exit-layer rows (f16 bits): both kernels of a projection run at once
+    __nv_bfloat16 *tc_xalt = nullptr, *tc_x4alt = nullptr;  // second set: operand rows written by the PREVIOUS projection's
+                                                            // epilogues (gate/up -> down) while that projection still reads its own
     int tc_max_pad = 0, tc_kmax = 0;
     bool tc_ok = false;
     struct LayerMaps { CUtensorMap q, k, v, o, g, u, d; };
@@ -45,7 +47,7 @@ struct river_ctx {
     CUtensorMap tc_map_head;
     // operand maps of the tensor-core projections for (K, padded rows): up to 128 rows the lo rows follow the hi rows
     // in one buffer (`lo_ptr` = tc_xhi + np K) and `hi` covers both (one copy per k-block); beyond, two buffers
-    struct BMap { int K, np; bool w4, one; __nv_bfloat16 *lo_ptr; CUtensorMap hi, lo; };
+    struct BMap { int K, np; bool w4, alt, one; __nv_bfloat16 *base, *lo_ptr; CUtensorMap hi, lo; };
     std::vector<BMap> tc_bmaps;
     int32_t *hint_act;
     const uint8_t *attn_skip = nullptr;  // exit flags of the block whose attention is being launched (strategies that run nothing for rows that left), else null
